@@ -1,0 +1,386 @@
+"""Pins for the CPU oracle: it is checked against things other than itself -- the paper's printed
+worked examples (tests/golden), closed forms, invariants, brute force on tiny inputs and
+torch-CPU fp64 library routines -- before anything on the GPU is trusted against it."""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import blocked, core, operators, relational
+
+RNG = np.random.default_rng(3905)
+
+
+def _golden(golden_dir, name):
+    with open(os.path.join(golden_dir, name)) as f:
+        return json.load(f)
+
+
+# ---------------------------------------------------------------------------------------------
+# rounding
+# ---------------------------------------------------------------------------------------------
+def test_round_bf16_matches_torch_and_ties_to_even():
+    x = np.concatenate([RNG.standard_normal(20000) * 10.0 ** RNG.integers(-30, 30, 20000),
+                        [0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38, 1e-40, -1e-45, 65504.0]])
+    x32 = x.astype(np.float32).astype(np.float64)  # torch rounds from fp32; feed fp32-representable values
+    want = torch.from_numpy(x32.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    got = core.round_to(x32, "bf16")
+    assert np.array_equal(got, want)
+    # exact ties: 1 + 2^-8 lies midway between 1 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    assert core.round_to([1.0 + 2.0 ** -8], "bf16")[0] == 1.0
+    assert core.round_to([1.0 + 3 * 2.0 ** -8], "bf16")[0] == 1.0 + 2.0 ** -6
+    # one rounding from fp64, not two: just above the tie must round up
+    assert core.round_to([1.0 + 2.0 ** -8 + 2.0 ** -40], "bf16")[0] == 1.0 + 2.0 ** -7
+    assert np.array_equal(core.round_to(x, "f32"), x.astype(np.float32).astype(np.float64))
+
+
+# ---------------------------------------------------------------------------------------------
+# the three engines against brute force (tiny inputs, every extent <= 6)
+# ---------------------------------------------------------------------------------------------
+CASES = [
+    ("ij,jk->ik", "mul", "sum", ()),
+    ("ij,kj->ik", "mul", "sum", ()),
+    ("bqhd,bkhd->bhqk", "mul", "sum", ()),
+    ("ij->i", "square", "sum", ()),
+    ("hij->hi", "ident", "max", ()),
+    ("hij,hi->hi", "exp_sub", "sum", ()),
+    ("hij,hi,hi->hij", "exp_sub_div", "none", ()),
+    ("ij,ij->ij", "silu_mul", "none", ()),
+    ("ij,ij->ij", "add", "none", ()),
+    ("ij,i,j->ij", "rms_scale", "none", (1e-5, 5.0)),
+    ("ij,jk,kl->il", "mul", "sum", ()),
+    ("i,j->ij", "mul", "none", ()),
+]
+
+
+@pytest.mark.parametrize("einsum,fn,agg,params", CASES)
+def test_engines_agree_with_brute_force(einsum, fn, agg, params):
+    ins, out, letters = core.parse_einsum(einsum)
+    ext = {c: int(RNG.integers(2, 6)) for c in letters}
+    if fn == "rms_scale":
+        ext["j"] = 5
+    inputs = [RNG.standard_normal([ext[c] for c in t]) for t in ins]
+    if fn in ("rms_scale",):
+        inputs[1] = np.abs(inputs[1]) + 0.1
+    if fn == "exp_sub_div":
+        inputs[2] = np.abs(inputs[2]) + 0.5
+    want = relational.brute_einsum(einsum, inputs, fn, agg, params)
+    t1 = core.join_agg(einsum, inputs, fn, agg, params)
+    t0 = relational.t0_join_agg(einsum, inputs, fn, agg, params)
+    np.testing.assert_allclose(t1, want, rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(t0, want, rtol=1e-13, atol=1e-13)
+    # ascending fold order is the same in T0 and T1 => identical bits (numpy's exp may differ from libm's)
+    if fn in ("mul", "ident", "square", "add"):
+        assert np.array_equal(t0, t1)
+
+
+def test_selection_predicate_against_brute_force():
+    S = RNG.standard_normal((2, 5, 5))
+    for eng in (core.join_agg, relational.t0_join_agg):
+        got = eng("hqk->hq", [S], fn="ident", agg="max", pred=("k", "q"))
+        want = relational.brute_einsum("hqk->hq", [S], "ident", "max", (), pred=("k", "q"))
+        assert np.array_equal(got, want)
+        assert np.array_equal(got, np.array([[S[h, q, : q + 1].max() for q in range(5)] for h in range(2)]))
+
+
+def test_t0_equals_t1_on_config1_shape():
+    """Config 1 through the literal tuple engine: 256^3 = 16.8 M joined tuples."""
+    A = RNG.standard_normal((256, 256)).astype(np.float32).astype(np.float64)
+    B = RNG.standard_normal((256, 256)).astype(np.float32).astype(np.float64)
+    t1 = core.matmul(A, B)
+    t0 = relational.t0_join_agg("ij,jk->ik", [A[:64], B])
+    assert np.array_equal(t0, t1[:64])
+    assert np.array_equal(core.join_agg("ij,jk->ik", [A, B]), t1)
+
+
+# ---------------------------------------------------------------------------------------------
+# paper pins: spec enumeration, multiplicities, cost counts, overlay
+# ---------------------------------------------------------------------------------------------
+def _distinct_out_types(spec):
+    seen = {}
+    for cell in spec.cells:
+        c = spec.block_coords(cell, -1)
+        lo, hi = spec.bounds(c, -1)
+        seen[spec.flat_key(c, -1)] = {"lower": lo, "upper": hi}
+    return [seen[k] for k in sorted(seen)]
+
+
+def test_matmul_decomposed_example(golden_dir):
+    g = _golden(golden_dir, "matmul_decomposed.json")
+    two = blocked.Spec(g["einsum"], g["two_spec"]["parts"])
+    assert two.p == g["two_spec"]["num_function_specs"]
+    assert _distinct_out_types(two) == g["two_spec"]["distinct_output_types"]
+    assert two.multiplicity().tolist() == g["two_spec"]["multiplicity"]
+    cols = [two.bounds(two.block_coords(c, 0), 0) for c in two.cells]
+    assert [[lo[1], hi[1]] for lo, hi in cols] == g["two_spec"]["A_columns"]
+    four = blocked.Spec(g["einsum"], g["four_spec"]["parts"])
+    assert [four.nb[c] for c in "ijk"] == [g["four_spec"]["intervals"][c] for c in "ijk"]
+    assert four.p == g["four_spec"]["num_function_specs"] == 2 * 2 * 1
+    assert _distinct_out_types(four) == g["four_spec"]["distinct_output_types"]
+    assert four.multiplicity().tolist() == g["four_spec"]["multiplicity"]
+    # F_{m,n}: rows in the m-th half of i, columns in the n-th half of j, times rows in the n-th half of j
+    ink, outk = four.tuples()
+    assert ink.tolist() == [[0, 0], [1, 1], [2, 0], [3, 1]] and outk.tolist() == [0, 0, 1, 1]
+
+
+def test_cost_closed_form(golden_dir):
+    g = _golden(golden_dir, "cost_3d_matmul.json")
+    for c in g["cases"]:
+        N = c["N"]
+        spec = blocked.Spec("ij,jk->ik", {"i": blocked.equal_splits(N, c["a"]), "j": blocked.equal_splits(N, c["b"]),
+                                          "k": blocked.equal_splits(N, c["c"])})
+        assert spec.p == c["a"] * c["b"] * c["c"]
+        assert spec.cost_terms() == (c["join"], c["agg"]) == ((c["a"] + c["c"]) * N * N, (c["b"] - 1) * N * N)
+
+
+def test_overlay_example(golden_dir):
+    g = _golden(golden_dir, "overlay_example.json")
+    over, atoms = blocked.overlay_atoms(g["producer_splits"], g["consumer_splits"])
+    assert over[0] == g["overlay_row_split_points"] and over[1] == [0, 256]
+    assert len(atoms) == g["num_atoms"]
+    assert [a[2] for a in atoms] == g["atom_to_producer_block"]
+    assert [a[3] for a in atoms] == g["atom_to_consumer_block"]
+    assert all(g["atom_to_producer_block"].count(b) == g["atoms_per_producer_block"] for b in (0, 1))
+
+
+def test_overlay_invariants_random():
+    for _ in range(20):
+        rank = int(RNG.integers(1, 4))
+        ext = [int(RNG.integers(3, 12)) for _ in range(rank)]
+
+        def rand_splits(e):
+            cuts = sorted(set(RNG.integers(1, e, int(RNG.integers(0, 4))).tolist()))
+            return [0] + cuts + [e]
+
+        src = [rand_splits(e) for e in ext]
+        dst = [rand_splits(e) for e in ext]
+        _, atoms = blocked.overlay_atoms(src, dst)
+        cover = np.zeros(ext, dtype=np.int32)
+        _, slo, sup, _, _ = blocked.relation_keys(ext, src, 2)
+        _, dlo, dup, _, _ = blocked.relation_keys(ext, dst, 2)
+        for lo, hi, sb, db in atoms:
+            cover[tuple(slice(l, h) for l, h in zip(lo, hi))] += 1
+            for blo, bup in ((slo[sb], sup[sb]), (dlo[db], dup[db])):  # atom inside exactly one block of each family
+                assert all(bl <= l and h <= bu for l, h, bl, bu in zip(lo, hi, blo, bup))
+        assert (cover == 1).all()  # atoms tile the tensor
+
+
+def test_tiling_validation():
+    blocked.check_splits(8, [0, 3, 8])
+    for bad in ([0, 3], [1, 8], [0, 5, 5, 8], [0, 6, 4, 8], [0]):
+        with pytest.raises(ValueError):
+            blocked.check_splits(8, bad)
+    # brute-force cover + disjointness of the block types of a key table (Definition 3.2)
+    ext, splits = [7, 5, 4], [[0, 2, 7], [0, 5], [0, 1, 3, 4]]
+    _, lo, up, off, total = blocked.relation_keys(ext, splits, 2)
+    cover = np.zeros(ext, dtype=int)
+    for l, u in zip(lo, up):
+        cover[tuple(slice(a, b) for a, b in zip(l, u))] += 1
+    assert (cover == 1).all() and (off % 128 == 0).all() and total % 128 == 0
+    assert blocked.equal_splits(10, 4) == [0, 2, 5, 7, 10]
+
+
+# ---------------------------------------------------------------------------------------------
+# decomposition invariance (Definition 3.7: every spec recovers the same output)
+# ---------------------------------------------------------------------------------------------
+def test_decomposition_invariance_config1():
+    A = RNG.standard_normal((256, 256)).astype(np.float32).astype(np.float64)
+    B = RNG.standard_normal((256, 256)).astype(np.float32).astype(np.float64)
+    ref = core.matmul(A, B)
+    for grid in ((4, 4, 4), (2, 8, 4), (1, 1, 1), (4, 8, 4)):
+        parts = {c: blocked.equal_splits(256, n) for c, n in zip("ijk", grid)}
+        got = blocked.t2_join_agg("ij,jk->ik", parts, [A, B])
+        assert np.abs(got - ref).max() <= 1e-12 * np.abs(ref).max()
+    np.testing.assert_allclose(ref, torch.from_numpy(A).matmul(torch.from_numpy(B)).numpy(), rtol=0, atol=1e-11)
+
+
+@pytest.mark.parametrize("einsum,fn,agg", [("ij->i", "square", "sum"), ("hij->hi", "ident", "max"),
+                                           ("ij,ij->ij", "silu_mul", "none"), ("ij,kj->ik", "mul", "sum")])
+def test_decomposition_invariance_uneven(einsum, fn, agg):
+    ins, out, letters = core.parse_einsum(einsum)
+    ext = {c: int(RNG.integers(5, 11)) for c in letters}
+    inputs = [RNG.standard_normal([ext[c] for c in t]) for t in ins]
+    ref = core.join_agg(einsum, inputs, fn, agg)
+    for _ in range(3):
+        parts = {c: blocked.equal_splits(ext[c], int(RNG.integers(1, 4))) for c in letters}
+        got = blocked.t2_join_agg(einsum, parts, inputs, fn, agg)
+        np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-12)
+        if agg == "max":
+            assert np.array_equal(got, ref)
+
+
+# ---------------------------------------------------------------------------------------------
+# relation layout and repartition
+# ---------------------------------------------------------------------------------------------
+def test_pack_unpack_repartition():
+    ext = [12, 10, 6]
+    dense = RNG.integers(0, 60000, ext).astype(np.uint16)
+    one = [[0, e] for e in ext]
+    t1 = [[0, 5, 12], [0, 10], [0, 2, 6]]
+    t2 = [[0, 4, 8, 12], [0, 3, 10], [0, 6]]
+    p1 = blocked.pack(dense, t1)
+    assert np.array_equal(blocked.unpack(p1, ext, t1), dense)
+    # repartition to the one-block tiling = the dense row-major tensor
+    assert np.array_equal(blocked.repartition(p1, ext, t1, one)[: dense.size], dense.reshape(-1))
+    p2 = blocked.repartition(p1, ext, t1, t2)
+    assert np.array_equal(p2, blocked.pack(dense, t2))                       # direct
+    assert np.array_equal(blocked.repartition(p2, ext, t2, t1), p1)          # round trip
+    via = blocked.repartition(blocked.repartition(p1, ext, t1, one), ext, one, t2)
+    assert np.array_equal(via, p2)                                           # via an intermediate tiling
+
+
+# ---------------------------------------------------------------------------------------------
+# operators against closed forms and library routines
+# ---------------------------------------------------------------------------------------------
+def test_matmul_special_cases():
+    A = RNG.standard_normal((9, 9))
+    assert np.array_equal(core.matmul(A, np.eye(9)), A)
+    perm = np.eye(9)[RNG.permutation(9)]
+    assert np.array_equal(core.matmul(perm, A), perm @ A)
+    # transposed operands would give A^T: the join must pair A's SECOND index with B's FIRST
+    B = RNG.standard_normal((9, 4))
+    assert np.abs(core.matmul(A, B) - A @ B).max() < 1e-13 and np.abs(core.matmul(A, B) - A.T @ B).max() > 1e-3
+
+
+def test_silu_mul():
+    t = RNG.standard_normal((7, 9)) * 4
+    one = np.ones_like(t)
+    s = core.join_agg("ij,ij->ij", [t, one], "silu_mul", "none")
+    s_neg = core.join_agg("ij,ij->ij", [-t, one], "silu_mul", "none")
+    np.testing.assert_allclose(s - s_neg, t, rtol=1e-13, atol=1e-13)          # silu(t) - silu(-t) = t
+    assert core.join_agg("ij,ij->ij", [np.zeros((1, 1)), np.ones((1, 1))], "silu_mul", "none")[0, 0] == 0.0
+    b = RNG.standard_normal((7, 9))
+    want = (torch.nn.functional.silu(torch.from_numpy(t)) * torch.from_numpy(b)).numpy()
+    np.testing.assert_allclose(core.join_agg("ij,ij->ij", [t, b], "silu_mul", "none"), want, rtol=1e-13, atol=1e-14)
+
+
+def test_rmsnorm():
+    X = RNG.standard_normal((6, 32)) * 2
+    g = 1 + 0.1 * RNG.standard_normal(32)
+    eps = 1e-5
+    out = operators.rmsnorm(X, g, eps, out_dtype=None)
+    want = torch.nn.functional.rms_norm(torch.from_numpy(X), (32,), torch.from_numpy(g), eps).numpy()
+    np.testing.assert_allclose(out["y"], want, rtol=1e-6, atol=1e-7)  # ss is stored in fp32
+    y1 = operators.rmsnorm(X, np.ones(32), eps, out_dtype=None)["y"]
+    ms = (X * X).mean(axis=1)
+    np.testing.assert_allclose((y1 * y1).mean(axis=1), ms / (ms + eps), rtol=1e-6)  # closed form with gamma = 1
+    y_scaled = operators.rmsnorm(1000 * X, g, eps, out_dtype=None)["y"]
+    np.testing.assert_allclose(y_scaled, out["y"], rtol=1e-4)                        # scale invariance (eps small)
+
+
+def test_softmax():
+    S = RNG.standard_normal((3, 5, 16)) * 2
+    out = operators.softmax_rows(S, out_dtype=None)
+    np.testing.assert_allclose(out["p"].sum(axis=-1), 1.0, rtol=1e-6)
+    np.testing.assert_allclose(out["p"], torch.softmax(torch.from_numpy(S), -1).numpy(), rtol=1e-6, atol=1e-9)
+    shifted = operators.softmax_rows(S + 3.0, out_dtype=None)["p"]
+    np.testing.assert_allclose(shifted, out["p"], rtol=1e-6)
+    assert np.array_equal(out["m"], S.max(axis=-1).astype(np.float32).astype(np.float64))
+
+
+def test_attention_closed_forms_and_library():
+    B, S, H, D = 2, 12, 3, 8
+    Q, K, V = (RNG.standard_normal((B, S, H, D)) for _ in range(3))
+    O = operators.attention(Q, K, V, out_dtype=None)
+    t = lambda a: torch.from_numpy(a).permute(0, 2, 1, 3)
+    want = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V), is_causal=True).permute(0, 2, 1, 3).numpy()
+    np.testing.assert_allclose(O, want, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(O[:, 0], V[:, 0], rtol=1e-14)                               # row 0 sees only key 0
+    prefix_mean = np.cumsum(V, axis=1) / np.arange(1, S + 1)[None, :, None, None]
+    np.testing.assert_allclose(operators.attention(0 * Q, K, V, out_dtype=None), prefix_mean, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(operators.attention(Q, K, np.ones_like(V), out_dtype=None), 1.0, rtol=1e-13)
+    want_nc = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V)).permute(0, 2, 1, 3).numpy()
+    np.testing.assert_allclose(operators.attention(Q, K, V, causal=False, out_dtype=None), want_nc, rtol=1e-12, atol=1e-13)
+    # S = 1: O = V
+    np.testing.assert_allclose(operators.attention(Q[:, :1], K[:, :1], V[:, :1], out_dtype=None), V[:, :1], rtol=1e-14)
+    # a subset of query rows, given their positions
+    rows = np.array([0, 5, 11])
+    np.testing.assert_array_equal(operators.attention(Q[:, rows], K, V, out_dtype=None, qpos=rows), O[:, rows])
+    # the operator as an explicit chain of scalar-keyed join-aggs
+    np.testing.assert_allclose(operators.attention_as_join_aggs(Q, K, V), O, rtol=1e-12, atol=1e-13)
+    # Definition 3.7 with the KV index split inside the sequence and the triple aggregation
+    for qs, ks in (([0, 4, 8, 12], [0, 4, 8, 12]), ([0, 12], [0, 3, 12]), ([0, 5, 12], [0, 2, 7, 12])):
+        np.testing.assert_allclose(operators.attention_blocked(Q, K, V, qs, ks), O, rtol=1e-12, atol=1e-13)
+
+
+def test_online_softmax_aggregation_is_a_valid_aggregation():
+    def rand_triple():
+        return RNG.standard_normal((4, 3)), RNG.standard_normal(4) * 3, np.abs(RNG.standard_normal(4)) + 0.1
+
+    a, b, c = rand_triple(), rand_triple(), rand_triple()
+    comb = operators.softmax_triple_combine
+    for x, y in zip(comb(a, b), comb(b, a)):
+        np.testing.assert_allclose(x, y, rtol=1e-14)                       # commutative
+    for x, y in zip(comb(comb(a, b), c), comb(a, comb(b, c))):
+        np.testing.assert_allclose(x, y, rtol=1e-12)                       # associative
+    ident = (np.zeros((4, 3)), np.full(4, -np.inf), np.zeros(4))
+    for x, y in zip(comb(a, ident), a):
+        np.testing.assert_array_equal(x, y)                                # identity (0, -inf, 0)
+    for x, y in zip(comb(ident, ident), ident):
+        np.testing.assert_array_equal(x, y)
+
+
+def test_rope_properties():
+    B, S, H, D = 1, 9, 2, 8
+    x, y = RNG.standard_normal((B, S, H, D)), RNG.standard_normal((B, S, H, D))
+    rx = operators.rope(x, 1e4, out_dtype=None)
+    np.testing.assert_allclose(rx[:, 0], x[:, 0], rtol=1e-15)                               # t = 0 is the identity
+    pair_norm = lambda a: a.reshape(B, S, H, D // 2, 2) ** 2
+    np.testing.assert_allclose(pair_norm(rx).sum(-1), pair_norm(x).sum(-1), rtol=1e-12)     # rotation
+    # <RoPE(q, t1), RoPE(k, t2)> depends on t1 - t2 only
+    q, k = x[0, 0, 0], y[0, 0, 0]
+
+    def at(vec, t):
+        return operators.rope(vec.reshape(1, 1, 1, D), 1e4, out_dtype=None, pos=[t])[0, 0, 0]
+
+    assert abs(at(q, 7) @ at(k, 3) - at(q, 5) @ at(k, 1)) < 1e-12
+    assert abs(at(q, 7) @ at(k, 3) - at(q, 4) @ at(k, 1)) > 1e-6
+    # pair p = 0 rotates by exactly t radians; pair p by t * theta^(-2p/d); (1, 0) -> (cos, sin)
+    e = np.zeros((1, 1, 1, 4)); e[..., 0] = 1.0; e[..., 2] = 1.0
+    r = operators.rope(e, 100.0, out_dtype=None, pos=[3])[0, 0, 0]
+    np.testing.assert_allclose(r, [math.cos(3), math.sin(3), math.cos(3 / 10.0), math.sin(3 / 10.0)], rtol=1e-14)
+
+
+def _torch_block(x, w, n_heads, theta, eps):
+    """An independent composition from torch-CPU fp64 library routines (no rounding anywhere)."""
+    T = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    x = T(x)
+    S, hidden = x.shape
+    d = hidden // n_heads
+    n1 = torch.nn.functional.rms_norm(x, (hidden,), T(w["g1"]), eps)
+    q, k, v = (n1 @ T(w[n]) for n in ("wq", "wk", "wv"))
+
+    def rot(t):
+        t = t.reshape(S, n_heads, d // 2, 2)
+        ang = torch.arange(S, dtype=torch.float64)[:, None] * theta ** (-torch.arange(0, d, 2, dtype=torch.float64) / d)
+        z = torch.view_as_complex(t.contiguous()) * torch.polar(torch.ones_like(ang), ang)[:, None, :]
+        return torch.view_as_real(z).reshape(S, n_heads, d)
+
+    q, k, v = rot(q), rot(k), v.reshape(S, n_heads, d)
+    att = torch.nn.functional.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1),
+                                                           is_causal=True).transpose(0, 1).reshape(S, hidden)
+    h = x + att @ T(w["wo"])
+    n2 = torch.nn.functional.rms_norm(h, (hidden,), T(w["g2"]), eps)
+    y = (torch.nn.functional.silu(n2 @ T(w["w1"])) * (n2 @ T(w["w3"]))) @ T(w["w2"])
+    return (h + y).numpy()
+
+
+def test_llama_block_composition():
+    S, hidden, ffn, H = 10, 16, 24, 2
+    x = RNG.standard_normal((S, hidden))
+    w = {n: RNG.standard_normal(s) * 0.3 for n, s in (("wq", (hidden, hidden)), ("wk", (hidden, hidden)),
+         ("wv", (hidden, hidden)), ("wo", (hidden, hidden)), ("w1", (hidden, ffn)), ("w3", (hidden, ffn)),
+         ("w2", (ffn, hidden)))}
+    w["g1"], w["g2"] = 1 + 0.1 * RNG.standard_normal(hidden), 1 + 0.1 * RNG.standard_normal(hidden)
+    full = operators.llama_block(x, w, H, 1e4, 1e-5, dtype=None)
+    np.testing.assert_allclose(full["out"], _torch_block(x, w, H, 1e4, 1e-5), rtol=1e-5, atol=1e-6)
+    rows = np.array([0, 3, 9])
+    sub = operators.llama_block(x, w, H, 1e4, 1e-5, rows=rows, dtype=None)
+    np.testing.assert_array_equal(sub["out"], full["out"][rows])
+    # with storage rounding the result stays within bf16 distance of the unrounded one
+    b16 = operators.llama_block(x, w, H, 1e4, 1e-5, dtype="bf16")["out"]
+    assert np.linalg.norm(b16 - full["out"]) / np.linalg.norm(full["out"]) < 2e-2
