@@ -1,0 +1,179 @@
+/*
+ * ja.h -- C ABI of libja: execution of join-agg specs over tensor relations on one B200.
+ *
+ * Vocabulary follows the paper ("Every Kernel Is a Join"):
+ *   tensor type      rank + lower/upper bound vectors (Definition 3.1)
+ *   tiling           a set of tensor types that cover a type disjointly (Definition 3.2)
+ *   tensor relation  a tensor stored as (sub_tensor_key, sub_tensor) pairs, the key being the tensor
+ *                    type of the sub-tensor (Section 1; Section 3.2)
+ *   function spec F  one joined tuple of input sub-tensor types -> output sub-tensor types (Definition 3.5)
+ *   join-agg spec J  the set {F_1..F_p} obtained from one interval decomposition of the named indices
+ *                    (Definition 3.6; Section 3.3: exactly prod_s intervals[s] function specs)
+ *   implementation   Join (run f on every F) -> Aggregate ((+) over the F sharing an output type)
+ *                    -> Recompose (Definition 3.7)
+ *
+ * Conventions
+ *   - Every call returns ja_status_t; JA_OK == 0.  ja_last_error() gives a thread-local message.
+ *   - Argument errors are reported synchronously, before anything is enqueued; nothing is ever
+ *     partially enqueued.
+ *   - Handles (ja_spec_t, ja_relation_t) are opaque, owned by the library, freed by *_destroy.
+ *   - "host" / "device" in a parameter comment says where the pointed-to memory lives.
+ *   - Relation payloads are DEVICE memory owned by the caller (borrowed, never freed here), 128-byte
+ *     aligned, and must outlive every enqueued use.
+ *   - Canonical orders: index letters in order of first appearance in the einsum string (inputs left
+ *     to right, then the output); function specs row-major over the interval grid in that letter order
+ *     (last letter fastest); blocks of a relation row-major over the relation's own index order;
+ *     atoms row-major over the overlay grid.
+ *
+ * Payload layout of a relation ("block-key layout"): blocks in row-major key order, each block a dense
+ * row-major array of its own extents, blocks back to back, each starting on a 128-byte boundary.
+ */
+#ifndef JA_H_
+#define JA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    JA_OK = 0,
+    JA_ERR_INVALID_ARG = 1,
+    JA_ERR_PARSE = 2,              /* malformed einsum string */
+    JA_ERR_SHAPE = 3,              /* extents / ranks disagree */
+    JA_ERR_TILING = 4,             /* split points do not tile the index range (Definition 3.2 / 3.6) */
+    JA_ERR_PARTITION_MISMATCH = 5, /* a relation's tiling differs from in_k(J) / out(J): repartition first (Section 4.3, sub-cost 1) */
+    JA_ERR_DTYPE = 6,
+    JA_ERR_UNSUPPORTED = 7,        /* no kernel for this (einsum, fn, agg, dtype) combination */
+    JA_ERR_ALIGNMENT = 8,
+    JA_ERR_OOM = 9,
+    JA_ERR_CUDA = 10,
+    JA_ERR_TIMEOUT = 11            /* a bounded device-side wait ran out (reported through ja_stream_status) */
+} ja_status_t;
+
+typedef enum { JA_F32 = 0, JA_BF16 = 1 } ja_dtype_t;
+
+/* aggregation operator (+) of Definition 3.7 */
+typedef enum {
+    JA_AGG_NONE = 0,           /* every output type is produced by exactly one function spec */
+    JA_AGG_SUM = 1,
+    JA_AGG_MAX = 2,
+    JA_AGG_ONLINE_SOFTMAX = 3  /* (O~,m,l) (+) (O~',m',l'): m*=max(m,m'), O~ e^(m-m*) + O~' e^(m'-m*), same for l */
+} ja_agg_t;
+
+/* concrete operator f applied to one joined tuple (Definition 3.5).  fn_params in brackets. */
+typedef enum {
+    JA_FN_MUL = 0,         /* product of the operands: einsum contraction                               */
+    JA_FN_IDENT = 1,       /* x                                                                           */
+    JA_FN_SQUARE = 2,      /* x^2                                                                         */
+    JA_FN_ADD = 3,         /* x + y                                                                       */
+    JA_FN_SILU_MUL = 4,    /* a / (1 + exp(-a)) * b                                                       */
+    JA_FN_RMS_SCALE = 5,   /* x * (ss/n + eps)^(-1/2) * g, n = extent of the last index        [eps]     */
+    JA_FN_EXP_SUB = 6,     /* exp(x - m)                                                                  */
+    JA_FN_EXP_SUB_DIV = 7, /* exp(x - m) / l                                                              */
+    JA_FN_ROPE = 8,        /* rotate pairs (2p,2p+1) of the last index by t*theta^(-2p/d), t = value of the
+                              second index of "bshd"                                             [theta]  */
+    JA_FN_ATTENTION = 9,   /* per (q-block,k-block) tuple: scale*Q K^T, causal band, partial (O~,m,l);
+                              with JA_AGG_ONLINE_SOFTMAX, then O = O~/l                  [scale, causal]  */
+    JA_FN_RMSNORM = 10,    /* fused chain SQUARE/SUM -> RMS_SCALE over the last index              [eps]  */
+    JA_FN_SOFTMAX = 11     /* fused chain IDENT/MAX -> EXP_SUB/SUM -> EXP_SUB_DIV over the last index     */
+} ja_fn_t;
+
+typedef struct ja_spec ja_spec_t;
+typedef struct ja_relation ja_relation_t;
+
+/* Interval decomposition of one named index (Section 3.3): nparts+1 ascending split points (host),
+ * splits[0] == 0, splits[nparts] == extent. */
+typedef struct {
+    char name;
+    int64_t extent;
+    int32_t nparts;
+    const int64_t* splits; /* host, copied */
+} ja_index_part_t;
+
+/* ---- join-agg spec (Definition 3.6, Section 3.3) ------------------------------------------------
+ * Builds J for `einsum` (lower-case letters, ',' between operands, "->" before the output, at most 4
+ * operands of rank <= 4) from one ja_index_part_t per distinct letter (host array, any order).
+ * fn_params: host array of n_fn_params doubles, meaning per ja_fn_t above.  accum_dtype must be JA_F32.
+ * Errors: JA_ERR_PARSE, JA_ERR_SHAPE (letter without a partition / duplicate), JA_ERR_TILING,
+ * JA_ERR_INVALID_ARG.  Allocates no device memory and makes no CUDA call. */
+ja_status_t ja_spec_create(const char* einsum, const ja_index_part_t* parts, int32_t n_parts, ja_fn_t fn,
+                           const double* fn_params, int32_t n_fn_params, ja_agg_t agg, ja_dtype_t accum_dtype,
+                           ja_spec_t** out);
+ja_status_t ja_spec_destroy(ja_spec_t* spec);
+
+/* Introspection (host outputs, caller-allocated) -- the bit-exact bookkeeping surface.
+ * p = number of function specs = prod_s intervals[s]. */
+ja_status_t ja_spec_num_tuples(const ja_spec_t* spec, int64_t* p, int32_t* n_inputs);
+/* in_keys[p][n_inputs], out_keys[p]: flat block keys of every function spec, canonical order. */
+ja_status_t ja_spec_get_tuples(const ja_spec_t* spec, int32_t* in_keys, int32_t* out_keys);
+/* Tiling in_k(J) (operand >= 0) or out(J) (operand == -1): rank, blocks per dimension [rank], and the
+ * split points of every dimension concatenated (sum_d (nblocks[d]+1) values). */
+ja_status_t ja_spec_operand_tiling(const ja_spec_t* spec, int32_t operand, int32_t* rank, int32_t* nblocks,
+                                   int64_t* splits_flat);
+/* Cost-model counts of Section 4.3: join_elems = sum_F sum_k |I(T^(i_k))|; agg_elems = sum over distinct
+ * output types of (m-1) |I(T^(o))|.  For an a x b x c matmul grid these are (a+c)N^2 and (b-1)N^2 (Section 4.4). */
+ja_status_t ja_spec_cost_terms(const ja_spec_t* spec, int64_t* join_elems, int64_t* agg_elems);
+
+/* ---- tensor relation (Section 1, Section 3.2) -----------------------------------------------------
+ * extents[rank], nparts[rank], splits[rank] (host; splits[d] has nparts[d]+1 entries). */
+ja_status_t ja_relation_bytes(int32_t rank, const int64_t* extents, const int32_t* nparts,
+                              const int64_t* const* splits, ja_dtype_t dtype, size_t* bytes);
+/* device_ptr: DEVICE payload of at least `bytes` bytes as reported by ja_relation_bytes, 128-byte aligned,
+ * borrowed.  Errors: JA_ERR_TILING, JA_ERR_ALIGNMENT, JA_ERR_INVALID_ARG (buffer too small).  No CUDA call. */
+ja_status_t ja_relation_create(int32_t rank, const int64_t* extents, const int32_t* nparts,
+                               const int64_t* const* splits, ja_dtype_t dtype, void* device_ptr, size_t bytes,
+                               ja_relation_t** out);
+ja_status_t ja_relation_destroy(ja_relation_t* rel); /* frees key tables only, never the payload */
+ja_status_t ja_relation_num_blocks(const ja_relation_t* rel, int64_t* nblocks, int32_t* rank);
+/* Key table (host outputs): per block, in key order, coords[rank] (int32), lower[rank], upper[rank]
+ * (the tensor type = the key of the paper) and the byte offset of the block in the payload. */
+ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int64_t* lower, int64_t* upper,
+                                 int64_t* offsets);
+
+/* ---- execution (Definition 3.7) -------------------------------------------------------------------
+ * Runs Join -> Aggregate -> Recompose of `spec` in ONE kernel launch sequence on `cuda_stream`
+ * (a cudaStream_t passed as void*; NULL = the legacy default stream), asynchronously.
+ * inputs[k] must be tiled exactly as in_k(J), outputs[0] as out(J) (else JA_ERR_PARTITION_MISMATCH).
+ * Supported forms (letters are free; shapes of the signature matter):
+ *   "ij,jk->ik"            MUL / SUM        bf16 or f32 operands, f32 accumulate (tensor cores for bf16 on
+ *                                            uniform 16-byte-aligned blocks, plain ALUs otherwise)
+ *   "X,X->X", X any rank   ADD | SILU_MUL / NONE          key-aligned join
+ *   "Rj->R"                SQUARE/SUM, IDENT/MAX          R = leading letters; f32 statistics output
+ *   "Rj,R->R"              EXP_SUB / SUM
+ *   "Rj,R,j->Rj"           RMS_SCALE / NONE               (R of rank 1)
+ *   "Rj,R,R->Rj"           EXP_SUB_DIV / NONE
+ *   "Rj,j->Rj"             RMSNORM / NONE   (fused)       "Rj->Rj"  SOFTMAX / NONE (fused)
+ *   "bshd->bshd"           ROPE / NONE
+ *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128
+ * The first call for a given (spec, relations) tuple builds and caches tables on the device (a few
+ * synchronous cudaMalloc / cudaMemcpy); later calls only launch. */
+ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,
+                       ja_relation_t* const* outputs, int32_t n_outputs, void* cuda_stream);
+
+/* ---- repartition (Section 5.3: overlay -> atoms, decompose + recompose) ---------------------------
+ * Copies the tensor held by `src` into the tiling of `dst` (same rank, extents, dtype): every atom of the
+ * overlay of the two tilings moves from its source block to its destination block.  Bit-exact, no
+ * aggregation.  Asynchronous on `cuda_stream`. */
+ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* dst, void* cuda_stream);
+/* Overlay introspection (host, no CUDA): number of atoms, then per atom lower[rank], upper[rank],
+ * flat source block, flat destination block.  Pass NULL arrays to query the count only. */
+ja_status_t ja_overlay_atoms(const ja_relation_t* src, const ja_relation_t* dst, int64_t* n_atoms, int64_t* lower,
+                             int64_t* upper, int32_t* src_block, int32_t* dst_block);
+
+/* Device-detected conditions (bounded-wait expiry) accumulate in a status word; this call synchronizes
+ * `cuda_stream`, returns the word in *device_status and clears it. */
+ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_status);
+
+/* Number of kernels this library has launched since load (for launch accounting by callers). */
+int64_t ja_launch_count(void);
+
+const char* ja_last_error(void);
+const char* ja_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JA_H_ */

@@ -43,7 +43,10 @@ def check_splits(extent: int, splits) -> None:
 class Spec:
     """The join-agg spec J for one interval decomposition (Definition 3.6 / Section 3.3)."""
 
-    def __init__(self, einsum: str, parts: dict):
+    def __init__(self, einsum: str, parts: dict, band=None):
+        """band = (k_letter, q_letter): the selection k <= q lifted to blocks -- a cell of the interval grid is
+        a function specification only if some key position of its k interval is <= some query position of its
+        q interval (attention with the key index split inside a sequence)."""
         self.einsum = einsum
         self.ins, self.out, self.letters = core.parse_einsum(einsum)
         self.parts = {c: list(parts[c]) for c in self.letters}
@@ -53,6 +56,10 @@ class Spec:
         self.extent = {c: self.parts[c][-1] for c in self.letters}
         grid = [range(self.nb[c]) for c in self.letters]
         self.cells = list(itertools.product(*grid))  # row-major, last letter fastest
+        if band is not None:
+            ik, iq = self.letters.index(band[0]), self.letters.index(band[1])
+            self.cells = [c for c in self.cells
+                          if self.parts[band[0]][c[ik]] <= self.parts[band[1]][c[iq] + 1] - 1]
         self.p = len(self.cells)
 
     # -- per-operand helpers (operand = index into self.ins, or -1 for the output) --------------

@@ -1,0 +1,7 @@
+"""paper_2609_03905_b200: join-agg execution over tensor relations on one B200.
+
+`binding` mirrors the C ABI of libja (include/ja.h); `relations` adds handle/payload conveniences.
+"""
+from . import binding  # noqa: F401  (raises if libja.so is absent and cannot be built)
+from .binding import *  # noqa: F401,F403
+from .relations import Relation, Spec, equal_splits, from_dense, repartition, to_dense  # noqa: F401

@@ -1,0 +1,214 @@
+"""ctypes binding of libja's C ABI: the same names, argument marshalling only.
+
+Every step of the join-agg path runs inside libja's CUDA kernels; torch supplies device memory
+(`tensor.data_ptr()`) and streams (`torch.cuda.current_stream().cuda_stream`) and nothing else.
+There is no CPU fallback: if libja.so is missing and cannot be built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libja.so")
+
+JA_OK = 0
+STATUS = {0: "JA_OK", 1: "JA_ERR_INVALID_ARG", 2: "JA_ERR_PARSE", 3: "JA_ERR_SHAPE", 4: "JA_ERR_TILING",
+          5: "JA_ERR_PARTITION_MISMATCH", 6: "JA_ERR_DTYPE", 7: "JA_ERR_UNSUPPORTED", 8: "JA_ERR_ALIGNMENT",
+          9: "JA_ERR_OOM", 10: "JA_ERR_CUDA", 11: "JA_ERR_TIMEOUT"}
+JA_F32, JA_BF16 = 0, 1
+AGG = {"none": 0, "sum": 1, "max": 2, "online_softmax": 3}
+FN = {"mul": 0, "ident": 1, "square": 2, "add": 3, "silu_mul": 4, "rms_scale": 5, "exp_sub": 6, "exp_sub_div": 7,
+      "rope": 8, "attention": 9, "rmsnorm": 10, "softmax": 11}
+
+
+class JaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS.get(status, status)}: {message}")
+        self.status = status
+        self.status_name = STATUS.get(status, str(status))
+
+
+class ja_index_part_t(ctypes.Structure):
+    _fields_ = [("name", ctypes.c_char), ("extent", ctypes.c_int64), ("nparts", ctypes.c_int32),
+                ("splits", ctypes.POINTER(ctypes.c_int64))]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        from .build import build
+        build()
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    P = ctypes.POINTER
+    sigs = {
+        "ja_spec_create": [ctypes.c_char_p, P(ja_index_part_t), i32, ctypes.c_int, P(ctypes.c_double), i32, ctypes.c_int,
+                           ctypes.c_int, P(vp)],
+        "ja_spec_destroy": [vp],
+        "ja_spec_num_tuples": [vp, P(i64), P(i32)],
+        "ja_spec_get_tuples": [vp, vp, vp],
+        "ja_spec_operand_tiling": [vp, i32, P(i32), vp, vp],
+        "ja_spec_cost_terms": [vp, P(i64), P(i64)],
+        "ja_relation_bytes": [i32, P(i64), P(i32), P(P(i64)), ctypes.c_int, P(ctypes.c_size_t)],
+        "ja_relation_create": [i32, P(i64), P(i32), P(P(i64)), ctypes.c_int, vp, ctypes.c_size_t, P(vp)],
+        "ja_relation_destroy": [vp],
+        "ja_relation_num_blocks": [vp, P(i64), P(i32)],
+        "ja_relation_get_keys": [vp, vp, vp, vp, vp],
+        "ja_execute": [vp, P(vp), i32, P(vp), i32, vp],
+        "ja_repartition": [vp, vp, vp],
+        "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
+        "ja_stream_status": [vp, P(ctypes.c_int)],
+    }
+    for name, argtypes in sigs.items():
+        fn = getattr(lib, name)
+        fn.argtypes = argtypes
+        fn.restype = ctypes.c_int
+    lib.ja_last_error.restype = ctypes.c_char_p
+    lib.ja_version.restype = ctypes.c_char_p
+    lib.ja_launch_count.restype = ctypes.c_int64
+    return lib
+
+
+LIB = _load()
+LIB_PATH = _LIB_PATH
+
+
+def _check(st: int):
+    if st != JA_OK:
+        raise JaError(st, LIB.ja_last_error().decode())
+
+
+def _splits_arrays(splits):
+    arrs = [(ctypes.c_int64 * len(s))(*[int(x) for x in s]) for s in splits]
+    ptrs = (ctypes.POINTER(ctypes.c_int64) * len(arrs))(*[ctypes.cast(a, ctypes.POINTER(ctypes.c_int64)) for a in arrs])
+    return arrs, ptrs
+
+
+def ja_version() -> str:
+    return LIB.ja_version().decode()
+
+
+def ja_launch_count() -> int:
+    return int(LIB.ja_launch_count())
+
+
+def ja_spec_create(einsum: str, parts: dict, fn: str = "mul", fn_params=(), agg: str = "sum") -> int:
+    """parts: {letter: split points}. Returns the opaque spec handle."""
+    keep = []
+    arr = (ja_index_part_t * len(parts))()
+    for i, (name, sp) in enumerate(parts.items()):
+        a = (ctypes.c_int64 * len(sp))(*[int(x) for x in sp])
+        keep.append(a)
+        arr[i].name = name.encode()
+        arr[i].extent = int(sp[-1]) if len(sp) else 0
+        arr[i].nparts = len(sp) - 1
+        arr[i].splits = ctypes.cast(a, ctypes.POINTER(ctypes.c_int64))
+    p = (ctypes.c_double * max(1, len(fn_params)))(*[float(x) for x in fn_params])
+    out = ctypes.c_void_p()
+    _check(LIB.ja_spec_create(einsum.encode(), arr, len(parts), FN[fn] if isinstance(fn, str) else int(fn), p, len(fn_params),
+                              AGG[agg] if isinstance(agg, str) else int(agg), JA_F32, ctypes.byref(out)))
+    return out.value
+
+
+def ja_spec_destroy(spec: int):
+    _check(LIB.ja_spec_destroy(spec))
+
+
+def ja_spec_num_tuples(spec: int):
+    p, n = ctypes.c_int64(), ctypes.c_int32()
+    _check(LIB.ja_spec_num_tuples(spec, ctypes.byref(p), ctypes.byref(n)))
+    return p.value, n.value
+
+
+def ja_spec_get_tuples(spec: int):
+    p, n = ja_spec_num_tuples(spec)
+    ink = np.zeros((p, n), dtype=np.int32)
+    outk = np.zeros(p, dtype=np.int32)
+    _check(LIB.ja_spec_get_tuples(spec, ink.ctypes.data, outk.ctypes.data))
+    return ink, outk
+
+
+def ja_spec_operand_tiling(spec: int, operand: int):
+    rank = ctypes.c_int32()
+    _check(LIB.ja_spec_operand_tiling(spec, operand, ctypes.byref(rank), None, None))
+    nb = np.zeros(rank.value, dtype=np.int32)
+    _check(LIB.ja_spec_operand_tiling(spec, operand, ctypes.byref(rank), nb.ctypes.data, None))
+    flat = np.zeros(int(nb.sum()) + rank.value, dtype=np.int64)
+    _check(LIB.ja_spec_operand_tiling(spec, operand, ctypes.byref(rank), nb.ctypes.data, flat.ctypes.data))
+    splits, w = [], 0
+    for d in range(rank.value):
+        splits.append(flat[w: w + nb[d] + 1].tolist())
+        w += nb[d] + 1
+    return nb.tolist(), splits
+
+
+def ja_spec_cost_terms(spec: int):
+    j, a = ctypes.c_int64(), ctypes.c_int64()
+    _check(LIB.ja_spec_cost_terms(spec, ctypes.byref(j), ctypes.byref(a)))
+    return j.value, a.value
+
+
+def ja_relation_bytes(extents, splits, dtype: int) -> int:
+    rank = len(extents)
+    ext = (ctypes.c_int64 * rank)(*[int(e) for e in extents])
+    npar = (ctypes.c_int32 * rank)(*[len(s) - 1 for s in splits])
+    keep, ptrs = _splits_arrays(splits)
+    out = ctypes.c_size_t()
+    _check(LIB.ja_relation_bytes(rank, ext, npar, ptrs, dtype, ctypes.byref(out)))
+    return out.value
+
+
+def ja_relation_create(extents, splits, dtype: int, device_ptr: int, nbytes: int) -> int:
+    rank = len(extents)
+    ext = (ctypes.c_int64 * rank)(*[int(e) for e in extents])
+    npar = (ctypes.c_int32 * rank)(*[len(s) - 1 for s in splits])
+    keep, ptrs = _splits_arrays(splits)
+    out = ctypes.c_void_p()
+    _check(LIB.ja_relation_create(rank, ext, npar, ptrs, dtype, ctypes.c_void_p(device_ptr), nbytes, ctypes.byref(out)))
+    return out.value
+
+
+def ja_relation_destroy(rel: int):
+    _check(LIB.ja_relation_destroy(rel))
+
+
+def ja_relation_get_keys(rel: int):
+    nb, rank = ctypes.c_int64(), ctypes.c_int32()
+    _check(LIB.ja_relation_num_blocks(rel, ctypes.byref(nb), ctypes.byref(rank)))
+    coords = np.zeros((nb.value, rank.value), dtype=np.int32)
+    lower = np.zeros((nb.value, rank.value), dtype=np.int64)
+    upper = np.zeros((nb.value, rank.value), dtype=np.int64)
+    offs = np.zeros(nb.value, dtype=np.int64)
+    _check(LIB.ja_relation_get_keys(rel, coords.ctypes.data, lower.ctypes.data, upper.ctypes.data, offs.ctypes.data))
+    return coords, lower, upper, offs
+
+
+def ja_execute(spec: int, inputs, outputs, stream: int = 0):
+    ins = (ctypes.c_void_p * len(inputs))(*inputs)
+    outs = (ctypes.c_void_p * len(outputs))(*outputs)
+    _check(LIB.ja_execute(spec, ins, len(inputs), outs, len(outputs), ctypes.c_void_p(stream)))
+
+
+def ja_repartition(src: int, dst: int, stream: int = 0):
+    _check(LIB.ja_repartition(src, dst, ctypes.c_void_p(stream)))
+
+
+def ja_overlay_atoms(src: int, dst: int):
+    n = ctypes.c_int64()
+    _check(LIB.ja_overlay_atoms(src, dst, ctypes.byref(n), None, None, None, None))
+    nb, rank = ctypes.c_int64(), ctypes.c_int32()
+    _check(LIB.ja_relation_num_blocks(src, ctypes.byref(nb), ctypes.byref(rank)))
+    lower = np.zeros((n.value, rank.value), dtype=np.int64)
+    upper = np.zeros((n.value, rank.value), dtype=np.int64)
+    sb = np.zeros(n.value, dtype=np.int32)
+    db = np.zeros(n.value, dtype=np.int32)
+    _check(LIB.ja_overlay_atoms(src, dst, ctypes.byref(n), lower.ctypes.data, upper.ctypes.data, sb.ctypes.data, db.ctypes.data))
+    return lower, upper, sb, db
+
+
+def ja_stream_status(stream: int = 0) -> int:
+    st = ctypes.c_int()
+    _check(LIB.ja_stream_status(ctypes.c_void_p(stream), ctypes.byref(st)))
+    return st.value

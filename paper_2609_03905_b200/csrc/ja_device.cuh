@@ -1,0 +1,42 @@
+// Device-side helpers shared by the kernels: key-table lookups on a RelView and small numeric utilities.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ja_internal.h"
+
+// block index of coordinate x along dimension d: arithmetic on uniform tilings, binary search otherwise
+__device__ __forceinline__ int ja_find_blk(const RelView& v, int d, int64_t x) {
+    if (v.bs[d]) return (int)(x / v.bs[d]);
+    int lo = 0, hi = v.nblk[d] - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (v.splits[d][mid] <= x) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+
+// byte offset in the payload of the cell with tensor coordinates x[0..rank)
+__device__ __forceinline__ int64_t ja_elem_off(const RelView& v, const int64_t* x) {
+    int64_t flat = 0, off = 0;
+#pragma unroll
+    for (int d = 0; d < JA_MAX_RANK; ++d) {
+        if (d < v.rank) {
+            int b = ja_find_blk(v, d, x[d]);
+            int64_t lo = v.splits[d][b];
+            int64_t w = v.splits[d][b + 1] - lo;
+            flat = flat * v.nblk[d] + b;
+            off = off * w + (x[d] - lo);
+        }
+    }
+    return v.blk_off[flat] + off * v.esize;
+}
+
+__device__ __forceinline__ float ja_to_float(float x) { return x; }
+__device__ __forceinline__ float ja_to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T ja_from_float(float x);
+template <> __device__ __forceinline__ float ja_from_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 ja_from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }

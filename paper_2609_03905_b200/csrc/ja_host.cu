@@ -1,0 +1,757 @@
+// Host side of libja: einsum parsing, join-agg spec enumeration (Definition 3.6, Section 3.3), tensor
+// relation key tables (Section 1 / 3.2), overlay planning for repartition (Section 5.3), and the
+// dispatch of ja_execute (Definition 3.7) to the sm_100a kernels. No arithmetic on tensor values
+// happens on the host.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <mutex>
+
+#include "ja_internal.h"
+
+// ---------------------------------------------------------------------------------------------------
+// errors, counters, device status word
+// ---------------------------------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+static std::atomic<int64_t> g_launches{0};
+static std::atomic<uint64_t> g_next_id{1};
+__device__ int g_ja_status_word;
+
+ja_status_t ja_fail(ja_status_t st, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+ja_status_t ja_cuda_fail(cudaError_t e, const char* what) {
+    return ja_fail(JA_ERR_CUDA, "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+}
+
+void ja_count_launch(int n) { g_launches += n; }
+
+int* ja_device_status_word() {
+    static int* p = nullptr;
+    if (!p) {
+        if (cudaGetSymbolAddress((void**)&p, g_ja_status_word) != cudaSuccess) p = nullptr;
+    }
+    return p;
+}
+
+extern "C" const char* ja_last_error(void) { return g_err; }
+extern "C" const char* ja_version(void) { return "libja 0.1 (sm_100a)"; }
+extern "C" int64_t ja_launch_count(void) { return g_launches.load(); }
+
+extern "C" ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_status) {
+    if (!device_status) return ja_fail(JA_ERR_INVALID_ARG, "device_status is NULL");
+    JA_CUDA(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    int* w = ja_device_status_word();
+    if (!w) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    int v = 0;
+    JA_CUDA(cudaMemcpy(&v, w, sizeof v, cudaMemcpyDeviceToHost));
+    *device_status = (ja_status_t)v;
+    if (v != 0) {
+        int zero = 0;
+        JA_CUDA(cudaMemcpy(w, &zero, sizeof zero, cudaMemcpyHostToDevice));
+    }
+    return JA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// tilings
+// ---------------------------------------------------------------------------------------------------
+static bool splits_tile(int64_t extent, int32_t nparts, const int64_t* s) {
+    if (nparts < 1 || !s || s[0] != 0 || s[nparts] != extent) return false;
+    for (int32_t i = 0; i < nparts; ++i)
+        if (s[i + 1] <= s[i]) return false;
+    return true;
+}
+
+static int esize_of(ja_dtype_t dt) { return dt == JA_F32 ? 4 : 2; }
+
+static ja_status_t fill_relation(ja_relation* r, int32_t rank, const int64_t* extents, const int32_t* nparts,
+                                 const int64_t* const* splits, ja_dtype_t dtype) {
+    if (rank < 1 || rank > JA_MAX_RANK || !extents || !nparts || !splits)
+        return ja_fail(JA_ERR_INVALID_ARG, "rank must be 1..%d and extents/nparts/splits non-NULL", JA_MAX_RANK);
+    if (dtype != JA_F32 && dtype != JA_BF16) return ja_fail(JA_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    r->rank = rank;
+    r->dtype = dtype;
+    r->esize = esize_of(dtype);
+    r->nblocks = 1;
+    r->equal_blocks = true;
+    for (int d = 0; d < rank; ++d) {
+        if (extents[d] < 1) return ja_fail(JA_ERR_SHAPE, "extent of dimension %d is %lld", d, (long long)extents[d]);
+        if (!splits_tile(extents[d], nparts[d], splits[d]))
+            return ja_fail(JA_ERR_TILING, "split points of dimension %d do not tile [0, %lld)", d, (long long)extents[d]);
+        r->extent[d] = extents[d];
+        r->nblk[d] = nparts[d];
+        r->splits[d].assign(splits[d], splits[d] + nparts[d] + 1);
+        int64_t b0 = splits[d][1] - splits[d][0];
+        bool uni = true, eq = true;
+        for (int i = 0; i < nparts[d]; ++i) {
+            int64_t w = splits[d][i + 1] - splits[d][i];
+            if (i + 1 < nparts[d] ? (w != b0) : (w > b0)) uni = false;
+            if (w != b0) eq = false;
+        }
+        r->bs[d] = uni ? b0 : 0;
+        r->equal_blocks = r->equal_blocks && eq;
+        r->nblocks *= nparts[d];
+    }
+    // block offsets: row-major key order, back to back, 128-byte aligned
+    r->blk_off.resize(r->nblocks);
+    int32_t c[JA_MAX_RANK] = {0, 0, 0, 0};
+    int64_t off = 0;
+    for (int64_t b = 0; b < r->nblocks; ++b) {
+        r->blk_off[b] = off;
+        int64_t n = 1;
+        for (int d = 0; d < rank; ++d) n *= r->splits[d][c[d] + 1] - r->splits[d][c[d]];
+        int64_t nbytes = n * r->esize;
+        off += (nbytes + JA_ALIGN - 1) / JA_ALIGN * JA_ALIGN;
+        for (int d = rank - 1; d >= 0; --d) {
+            if (++c[d] < r->nblk[d]) break;
+            c[d] = 0;
+        }
+    }
+    r->bytes = (size_t)off;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_relation_bytes(int32_t rank, const int64_t* extents, const int32_t* nparts,
+                                         const int64_t* const* splits, ja_dtype_t dtype, size_t* bytes) {
+    if (!bytes) return ja_fail(JA_ERR_INVALID_ARG, "bytes is NULL");
+    ja_relation tmp;
+    ja_status_t st = fill_relation(&tmp, rank, extents, nparts, splits, dtype);
+    if (st != JA_OK) return st;
+    *bytes = tmp.bytes;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_relation_create(int32_t rank, const int64_t* extents, const int32_t* nparts,
+                                          const int64_t* const* splits, ja_dtype_t dtype, void* device_ptr,
+                                          size_t bytes, ja_relation_t** out) {
+    if (!out) return ja_fail(JA_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    std::unique_ptr<ja_relation> r(new ja_relation());
+    ja_status_t st = fill_relation(r.get(), rank, extents, nparts, splits, dtype);
+    if (st != JA_OK) return st;
+    if (!device_ptr) return ja_fail(JA_ERR_INVALID_ARG, "device_ptr is NULL");
+    if (((uintptr_t)device_ptr) % JA_ALIGN != 0)
+        return ja_fail(JA_ERR_ALIGNMENT, "payload pointer %p is not %d-byte aligned", device_ptr, JA_ALIGN);
+    if (bytes < r->bytes)
+        return ja_fail(JA_ERR_INVALID_ARG, "payload buffer has %zu bytes, the tiling needs %zu", bytes, r->bytes);
+    r->base = device_ptr;
+    r->id = g_next_id++;
+    *out = r.release();
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_relation_destroy(ja_relation_t* rel) {
+    if (!rel) return JA_OK;
+    if (rel->d_tables) cudaFree(rel->d_tables);
+    delete rel;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_relation_num_blocks(const ja_relation_t* rel, int64_t* nblocks, int32_t* rank) {
+    if (!rel) return ja_fail(JA_ERR_INVALID_ARG, "relation is NULL");
+    if (nblocks) *nblocks = rel->nblocks;
+    if (rank) *rank = rel->rank;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int64_t* lower, int64_t* upper,
+                                            int64_t* offsets) {
+    if (!rel) return ja_fail(JA_ERR_INVALID_ARG, "relation is NULL");
+    int32_t c[JA_MAX_RANK] = {0, 0, 0, 0};
+    for (int64_t b = 0; b < rel->nblocks; ++b) {
+        for (int d = 0; d < rel->rank; ++d) {
+            if (coords) coords[b * rel->rank + d] = c[d];
+            if (lower) lower[b * rel->rank + d] = rel->splits[d][c[d]];
+            if (upper) upper[b * rel->rank + d] = rel->splits[d][c[d] + 1];
+        }
+        if (offsets) offsets[b] = rel->blk_off[b];
+        for (int d = rel->rank - 1; d >= 0; --d) {
+            if (++c[d] < rel->nblk[d]) break;
+            c[d] = 0;
+        }
+    }
+    return JA_OK;
+}
+
+// device copy of the key table: [splits of dim 0 | dim 1 | ... | block offsets]
+ja_status_t ja_relation_to_device(const ja_relation* r) {
+    if (r->on_device) return JA_OK;
+    std::vector<int64_t> host;
+    for (int d = 0; d < r->rank; ++d) host.insert(host.end(), r->splits[d].begin(), r->splits[d].end());
+    host.insert(host.end(), r->blk_off.begin(), r->blk_off.end());
+    JA_CUDA(cudaMalloc((void**)&r->d_tables, host.size() * sizeof(int64_t)));
+    JA_CUDA(cudaMemcpy(r->d_tables, host.data(), host.size() * sizeof(int64_t), cudaMemcpyHostToDevice));
+    r->on_device = true;
+    return JA_OK;
+}
+
+RelView ja_view(const ja_relation* r) {
+    RelView v;
+    memset(&v, 0, sizeof v);
+    v.base = (char*)r->base;
+    v.rank = r->rank;
+    v.esize = r->esize;
+    int64_t* p = r->d_tables;
+    for (int d = 0; d < JA_MAX_RANK; ++d) {
+        if (d < r->rank) {
+            v.splits[d] = p;
+            p += r->nblk[d] + 1;
+            v.extent[d] = r->extent[d];
+            v.bs[d] = r->bs[d];
+            v.nblk[d] = r->nblk[d];
+        } else {
+            v.splits[d] = nullptr;
+            v.extent[d] = 1;
+            v.bs[d] = 1;
+            v.nblk[d] = 1;
+        }
+    }
+    v.blk_off = p;
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// join-agg spec
+// ---------------------------------------------------------------------------------------------------
+static int letter_pos(const std::string& letters, char c) {
+    size_t p = letters.find(c);
+    return p == std::string::npos ? -1 : (int)p;
+}
+
+extern "C" ja_status_t ja_spec_create(const char* einsum, const ja_index_part_t* parts, int32_t n_parts, ja_fn_t fn,
+                                      const double* fn_params, int32_t n_fn_params, ja_agg_t agg,
+                                      ja_dtype_t accum_dtype, ja_spec_t** out) {
+    if (!out) return ja_fail(JA_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!einsum || !parts || n_parts < 1) return ja_fail(JA_ERR_INVALID_ARG, "einsum / parts missing");
+    if (accum_dtype != JA_F32) return ja_fail(JA_ERR_DTYPE, "accumulation dtype must be JA_F32");
+    if ((int)fn < 0 || (int)fn > (int)JA_FN_SOFTMAX) return ja_fail(JA_ERR_INVALID_ARG, "unknown fn %d", (int)fn);
+    if ((int)agg < 0 || (int)agg > (int)JA_AGG_ONLINE_SOFTMAX) return ja_fail(JA_ERR_INVALID_ARG, "unknown agg %d", (int)agg);
+    if (n_fn_params < 0 || (n_fn_params > 0 && !fn_params)) return ja_fail(JA_ERR_INVALID_ARG, "fn_params missing");
+
+    std::unique_ptr<ja_spec> s(new ja_spec());
+    // ---- parse ------------------------------------------------------------------------------------
+    std::string e;
+    for (const char* c = einsum; *c; ++c)
+        if (*c != ' ') e.push_back(*c);
+    size_t arrow = e.find("->");
+    if (arrow == std::string::npos || e.find("->", arrow + 2) != std::string::npos)
+        return ja_fail(JA_ERR_PARSE, "einsum '%s' needs exactly one '->'", einsum);
+    std::string lhs = e.substr(0, arrow);
+    s->out = e.substr(arrow + 2);
+    size_t pos = 0;
+    while (true) {
+        size_t comma = lhs.find(',', pos);
+        s->ins.push_back(lhs.substr(pos, comma == std::string::npos ? std::string::npos : comma - pos));
+        if (comma == std::string::npos) break;
+        pos = comma + 1;
+    }
+    if (s->ins.empty() || s->ins.size() > JA_MAX_IN) return ja_fail(JA_ERR_PARSE, "1..%d operands expected", JA_MAX_IN);
+    std::vector<std::string> terms = s->ins;
+    terms.push_back(s->out);
+    for (size_t t = 0; t < terms.size(); ++t) {
+        const std::string& term = terms[t];
+        bool is_out = (t + 1 == terms.size());
+        if ((term.empty() && !is_out) || term.size() > JA_MAX_RANK)
+            return ja_fail(JA_ERR_PARSE, "operand '%s' must have rank 1..%d", term.c_str(), JA_MAX_RANK);
+        for (size_t i = 0; i < term.size(); ++i) {
+            char c = term[i];
+            if (c < 'a' || c > 'z') return ja_fail(JA_ERR_PARSE, "bad character '%c' in einsum", c);
+            if (term.find(c, i + 1) != std::string::npos)
+                return ja_fail(JA_ERR_PARSE, "letter '%c' repeated inside one operand", c);
+            if (is_out) {
+                if (letter_pos(s->letters, c) < 0)
+                    return ja_fail(JA_ERR_PARSE, "output letter '%c' appears in no input", c);
+            } else if (letter_pos(s->letters, c) < 0) {
+                s->letters.push_back(c);
+            }
+        }
+    }
+    if (s->out.empty()) return ja_fail(JA_ERR_UNSUPPORTED, "scalar outputs are not supported");
+    s->einsum = e;
+    // ---- partitions ---------------------------------------------------------------------------------
+    s->parts.resize(s->letters.size());
+    for (int32_t i = 0; i < n_parts; ++i) {
+        int lp = letter_pos(s->letters, parts[i].name);
+        if (lp < 0) return ja_fail(JA_ERR_SHAPE, "partition given for letter '%c' which the einsum does not use", parts[i].name);
+        if (!s->parts[lp].empty()) return ja_fail(JA_ERR_SHAPE, "two partitions for letter '%c'", parts[i].name);
+        if (parts[i].extent < 1 || !splits_tile(parts[i].extent, parts[i].nparts, parts[i].splits))
+            return ja_fail(JA_ERR_TILING, "split points of index '%c' do not tile [0, %lld)", parts[i].name,
+                           (long long)parts[i].extent);
+        s->parts[lp].assign(parts[i].splits, parts[i].splits + parts[i].nparts + 1);
+    }
+    for (size_t l = 0; l < s->letters.size(); ++l)
+        if (s->parts[l].empty()) return ja_fail(JA_ERR_SHAPE, "no partition for index '%c'", s->letters[l]);
+    bool has_agg_index = false;
+    for (char c : s->letters)
+        if (s->out.find(c) == std::string::npos) has_agg_index = true;
+    if (agg == JA_AGG_NONE && has_agg_index && fn != JA_FN_RMSNORM && fn != JA_FN_SOFTMAX)
+        return ja_fail(JA_ERR_TILING,
+                       "an index is absent from the output, so several function specs share an output type, "
+                       "but no aggregation was given");
+    s->fn = fn;
+    s->agg = agg;
+    s->params.assign(fn_params, fn_params + n_fn_params);
+
+    // ---- enumerate J: one function spec per cell of the interval grid (Section 3.3) ------------------
+    const int L = (int)s->letters.size();
+    std::vector<int32_t> nb(L);
+    int64_t p = 1;
+    for (int l = 0; l < L; ++l) {
+        nb[l] = (int32_t)s->parts[l].size() - 1;
+        p *= nb[l];
+        if (p > (int64_t)1 << 26) return ja_fail(JA_ERR_UNSUPPORTED, "more than 2^26 function specs");
+    }
+    // band predicate of attention: a (q-block, k-block) pair is a tuple only if some k <= some q
+    int band_q = -1, band_k = -1;
+    if (fn == JA_FN_ATTENTION && s->params.size() >= 2 && s->params[1] != 0.0 && s->ins.size() == 3 &&
+        s->ins[0].size() == 4 && s->ins[1].size() == 4) {
+        band_q = letter_pos(s->letters, s->ins[0][1]);
+        band_k = letter_pos(s->letters, s->ins[1][1]);
+    }
+    const int n_in = (int)s->ins.size();
+    std::vector<int32_t> cell(L, 0);
+    for (int64_t t = 0; t < p; ++t) {
+        bool keep = true;
+        if (band_q >= 0) keep = s->parts[band_k][cell[band_k]] <= s->parts[band_q][cell[band_q] + 1] - 1;
+        if (keep) {
+            for (int k = 0; k <= n_in; ++k) {
+                const std::string& term = (k < n_in) ? s->ins[k] : s->out;
+                int32_t key = 0;
+                for (char c : term) {
+                    int lp = letter_pos(s->letters, c);
+                    key = key * nb[lp] + cell[lp];
+                }
+                if (k < n_in) s->in_keys.push_back(key);
+                else s->out_keys.push_back(key);
+            }
+        }
+        for (int l = L - 1; l >= 0; --l) {
+            if (++cell[l] < nb[l]) break;
+            cell[l] = 0;
+        }
+    }
+    s->p = (int64_t)s->out_keys.size();
+    *out = s.release();
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_spec_destroy(ja_spec_t* spec) {
+    delete spec;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_spec_num_tuples(const ja_spec_t* spec, int64_t* p, int32_t* n_inputs) {
+    if (!spec) return ja_fail(JA_ERR_INVALID_ARG, "spec is NULL");
+    if (p) *p = spec->p;
+    if (n_inputs) *n_inputs = (int32_t)spec->ins.size();
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_spec_get_tuples(const ja_spec_t* spec, int32_t* in_keys, int32_t* out_keys) {
+    if (!spec) return ja_fail(JA_ERR_INVALID_ARG, "spec is NULL");
+    if (in_keys) memcpy(in_keys, spec->in_keys.data(), spec->in_keys.size() * sizeof(int32_t));
+    if (out_keys) memcpy(out_keys, spec->out_keys.data(), spec->out_keys.size() * sizeof(int32_t));
+    return JA_OK;
+}
+
+static const std::string& spec_term(const ja_spec* s, int operand) {
+    return operand < 0 ? s->out : s->ins[operand];
+}
+
+extern "C" ja_status_t ja_spec_operand_tiling(const ja_spec_t* spec, int32_t operand, int32_t* rank, int32_t* nblocks,
+                                              int64_t* splits_flat) {
+    if (!spec) return ja_fail(JA_ERR_INVALID_ARG, "spec is NULL");
+    if (operand < -1 || operand >= (int32_t)spec->ins.size()) return ja_fail(JA_ERR_INVALID_ARG, "operand %d out of range", operand);
+    const std::string& term = spec_term(spec, operand);
+    if (rank) *rank = (int32_t)term.size();
+    size_t w = 0;
+    for (size_t d = 0; d < term.size(); ++d) {
+        const std::vector<int64_t>& sp = spec->parts[letter_pos(spec->letters, term[d])];
+        if (nblocks) nblocks[d] = (int32_t)sp.size() - 1;
+        if (splits_flat) {
+            memcpy(splits_flat + w, sp.data(), sp.size() * sizeof(int64_t));
+            w += sp.size();
+        }
+    }
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_spec_cost_terms(const ja_spec_t* spec, int64_t* join_elems, int64_t* agg_elems) {
+    if (!spec) return ja_fail(JA_ERR_INVALID_ARG, "spec is NULL");
+    const int n_in = (int)spec->ins.size();
+    auto card = [&](int operand, int32_t key) {
+        const std::string& term = spec_term(spec, operand);
+        int64_t n = 1;
+        for (int d = (int)term.size() - 1; d >= 0; --d) {
+            const std::vector<int64_t>& sp = spec->parts[letter_pos(spec->letters, term[d])];
+            int32_t nbd = (int32_t)sp.size() - 1;
+            int32_t c = key % nbd;
+            key /= nbd;
+            n *= sp[c + 1] - sp[c];
+        }
+        return n;
+    };
+    int64_t join = 0;
+    std::map<int32_t, int64_t> mult;
+    for (int64_t t = 0; t < spec->p; ++t) {
+        for (int k = 0; k < n_in; ++k) join += card(k, spec->in_keys[t * n_in + k]);
+        mult[spec->out_keys[t]] += 1;
+    }
+    int64_t ag = 0;
+    for (auto& kv : mult) ag += (kv.second - 1) * card(-1, kv.first);
+    if (join_elems) *join_elems = join;
+    if (agg_elems) *agg_elems = ag;
+    return JA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// repartition: overlay -> atoms -> slab copies (Section 5.3)
+// ---------------------------------------------------------------------------------------------------
+struct Atom {
+    int64_t lo[JA_MAX_RANK], hi[JA_MAX_RANK];
+    int32_t sb, db;
+};
+
+static ja_status_t check_same_tensor(const ja_relation* a, const ja_relation* b) {
+    if (!a || !b) return ja_fail(JA_ERR_INVALID_ARG, "relation is NULL");
+    if (a->rank != b->rank) return ja_fail(JA_ERR_SHAPE, "ranks differ (%d vs %d)", a->rank, b->rank);
+    if (a->dtype != b->dtype) return ja_fail(JA_ERR_DTYPE, "dtypes differ");
+    for (int d = 0; d < a->rank; ++d)
+        if (a->extent[d] != b->extent[d]) return ja_fail(JA_ERR_SHAPE, "extent of dimension %d differs", d);
+    return JA_OK;
+}
+
+static void build_atoms(const ja_relation* src, const ja_relation* dst, std::vector<Atom>* atoms) {
+    const int r = src->rank;
+    std::vector<int64_t> over[JA_MAX_RANK];
+    for (int d = 0; d < r; ++d) {
+        over[d] = src->splits[d];
+        over[d].insert(over[d].end(), dst->splits[d].begin(), dst->splits[d].end());
+        std::sort(over[d].begin(), over[d].end());
+        over[d].erase(std::unique(over[d].begin(), over[d].end()), over[d].end());
+    }
+    auto owner = [](const std::vector<int64_t>& sp, int64_t x) {
+        return (int32_t)(std::upper_bound(sp.begin(), sp.end(), x) - sp.begin() - 1);
+    };
+    int32_t c[JA_MAX_RANK] = {0, 0, 0, 0};
+    int64_t n = 1;
+    for (int d = 0; d < r; ++d) n *= (int64_t)over[d].size() - 1;
+    atoms->reserve(n);
+    for (int64_t a = 0; a < n; ++a) {
+        Atom at;
+        at.sb = at.db = 0;
+        for (int d = 0; d < r; ++d) {
+            at.lo[d] = over[d][c[d]];
+            at.hi[d] = over[d][c[d] + 1];
+            at.sb = at.sb * src->nblk[d] + owner(src->splits[d], at.lo[d]);
+            at.db = at.db * dst->nblk[d] + owner(dst->splits[d], at.lo[d]);
+        }
+        atoms->push_back(at);
+        for (int d = r - 1; d >= 0; --d) {
+            if (++c[d] < (int32_t)over[d].size() - 1) break;
+            c[d] = 0;
+        }
+    }
+}
+
+extern "C" ja_status_t ja_overlay_atoms(const ja_relation_t* src, const ja_relation_t* dst, int64_t* n_atoms,
+                                        int64_t* lower, int64_t* upper, int32_t* src_block, int32_t* dst_block) {
+    ja_status_t st = check_same_tensor(src, dst);
+    if (st != JA_OK) return st;
+    std::vector<Atom> atoms;
+    build_atoms(src, dst, &atoms);
+    if (n_atoms) *n_atoms = (int64_t)atoms.size();
+    for (size_t a = 0; a < atoms.size(); ++a) {
+        for (int d = 0; d < src->rank; ++d) {
+            if (lower) lower[a * src->rank + d] = atoms[a].lo[d];
+            if (upper) upper[a * src->rank + d] = atoms[a].hi[d];
+        }
+        if (src_block) src_block[a] = atoms[a].sb;
+        if (dst_block) dst_block[a] = atoms[a].db;
+    }
+    return JA_OK;
+}
+
+struct RepartPlan {
+    CopySlab* d_slabs = nullptr;
+    int64_t n_slabs = 0;
+    int vec_bytes = 16;
+    ~RepartPlan() {
+        if (d_slabs) cudaFree(d_slabs);
+    }
+};
+static std::mutex g_repart_mu;
+static std::map<std::pair<uint64_t, uint64_t>, std::shared_ptr<RepartPlan>> g_repart_plans;
+
+// element offset of coordinate x inside block `b` of relation r (row-major inside the block)
+static int64_t in_block_offset(const ja_relation* r, int32_t b, const int64_t* x, int64_t* last_width) {
+    int32_t c[JA_MAX_RANK];
+    for (int d = r->rank - 1; d >= 0; --d) {
+        c[d] = b % r->nblk[d];
+        b /= r->nblk[d];
+    }
+    int64_t off = 0;
+    for (int d = 0; d < r->rank; ++d) {
+        int64_t lo = r->splits[d][c[d]], w = r->splits[d][c[d] + 1] - lo;
+        off = off * w + (x[d] - lo);
+        if (d == r->rank - 1 && last_width) *last_width = w;
+    }
+    return off;
+}
+
+extern "C" ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* dst, void* cuda_stream) {
+    ja_status_t st = check_same_tensor(src, dst);
+    if (st != JA_OK) return st;
+    if (src->base == dst->base) return ja_fail(JA_ERR_INVALID_ARG, "repartition in place is not supported");
+    std::shared_ptr<RepartPlan> plan;
+    {
+        std::lock_guard<std::mutex> lk(g_repart_mu);
+        auto it = g_repart_plans.find({src->id, dst->id});
+        if (it != g_repart_plans.end()) plan = it->second;
+    }
+    if (!plan) {
+        std::vector<Atom> atoms;
+        build_atoms(src, dst, &atoms);
+        const int r = src->rank, es = src->esize;
+        std::vector<CopySlab> slabs;
+        int64_t all_or = 0;  // OR of every quantity that limits the vector width
+        for (const Atom& at : atoms) {
+            // a slab = (rows of the second-to-last dimension) x (contiguous run of the last dimension),
+            // one per assignment of the outer dimensions
+            int64_t rows = r >= 2 ? at.hi[r - 2] - at.lo[r - 2] : 1;
+            int64_t row_bytes = (at.hi[r - 1] - at.lo[r - 1]) * es;
+            int64_t outer = 1;
+            for (int d = 0; d + 2 < r; ++d) outer *= at.hi[d] - at.lo[d];
+            int64_t rows_per = std::max<int64_t>(1, (64 * 1024) / row_bytes);
+            for (int64_t o = 0; o < outer; ++o) {
+                int64_t x[JA_MAX_RANK];
+                int64_t rem = o;
+                for (int d = r - 3; d >= 0; --d) {
+                    int64_t e = at.hi[d] - at.lo[d];
+                    x[d] = at.lo[d] + rem % e;
+                    rem /= e;
+                }
+                for (int64_t r0 = 0; r0 < rows; r0 += rows_per) {
+                    if (r >= 2) x[r - 2] = at.lo[r - 2] + r0;
+                    x[r - 1] = at.lo[r - 1];
+                    int64_t sw = 0, dw = 0;
+                    CopySlab s;
+                    s.src_off = src->blk_off[at.sb] + in_block_offset(src, at.sb, x, &sw) * es;
+                    s.dst_off = dst->blk_off[at.db] + in_block_offset(dst, at.db, x, &dw) * es;
+                    s.rows = (int32_t)std::min(rows_per, rows - r0);
+                    s.row_bytes = (int32_t)row_bytes;
+                    s.src_pitch = (int32_t)(sw * es);
+                    s.dst_pitch = (int32_t)(dw * es);
+                    all_or |= s.src_off | s.dst_off | s.row_bytes | s.src_pitch | s.dst_pitch;
+                    slabs.push_back(s);
+                }
+            }
+        }
+        plan.reset(new RepartPlan());
+        plan->vec_bytes = 16;
+        while (plan->vec_bytes > es && (all_or % plan->vec_bytes) != 0) plan->vec_bytes /= 2;
+        plan->n_slabs = (int64_t)slabs.size();
+        JA_CUDA(cudaMalloc((void**)&plan->d_slabs, slabs.size() * sizeof(CopySlab)));
+        JA_CUDA(cudaMemcpy(plan->d_slabs, slabs.data(), slabs.size() * sizeof(CopySlab), cudaMemcpyHostToDevice));
+        std::lock_guard<std::mutex> lk(g_repart_mu);
+        g_repart_plans[{src->id, dst->id}] = plan;
+    }
+    return ja_launch_repartition((const char*)src->base, (char*)dst->base, plan->d_slabs, plan->n_slabs,
+                                 plan->vec_bytes, (cudaStream_t)cuda_stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// ja_execute
+// ---------------------------------------------------------------------------------------------------
+struct ExecPlan {
+    std::shared_ptr<GemmTcPlan> gemm;
+    bool gemm_checked = false;
+    float2* rope_table = nullptr;
+    ~ExecPlan() {
+        if (rope_table) cudaFree(rope_table);
+    }
+};
+
+static ja_status_t check_tiling(const ja_spec* s, int operand, const ja_relation* r) {
+    const std::string& term = spec_term(s, operand);
+    if (!r) return ja_fail(JA_ERR_INVALID_ARG, "relation for operand %d is NULL", operand);
+    if (r->rank != (int)term.size())
+        return ja_fail(JA_ERR_SHAPE, "operand %d has rank %d, the einsum term '%s' needs %zu", operand, r->rank,
+                       term.c_str(), term.size());
+    for (int d = 0; d < r->rank; ++d) {
+        const std::vector<int64_t>& sp = s->parts[letter_pos(s->letters, term[d])];
+        if (r->extent[d] != sp.back())
+            return ja_fail(JA_ERR_SHAPE, "operand %d dimension %d has extent %lld, index '%c' has %lld", operand, d,
+                           (long long)r->extent[d], term[d], (long long)sp.back());
+        if (r->splits[d] != sp)
+            return ja_fail(JA_ERR_PARTITION_MISMATCH,
+                           "operand %d is not tiled as the join-agg spec requires along index '%c': repartition it first",
+                           operand, term[d]);
+    }
+    return JA_OK;
+}
+
+// "Rj" style helpers: lead = all letters but the last
+static std::string lead_of(const std::string& t) { return t.substr(0, t.size() - 1); }
+
+extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,
+                                  ja_relation_t* const* outputs, int32_t n_outputs, void* cuda_stream) {
+    if (!spec || !inputs || !outputs) return ja_fail(JA_ERR_INVALID_ARG, "spec / inputs / outputs is NULL");
+    const int n_in = (int)spec->ins.size();
+    if (n_inputs != n_in) return ja_fail(JA_ERR_INVALID_ARG, "spec has %d operands, %d relations given", n_in, n_inputs);
+    if (n_outputs != 1) return ja_fail(JA_ERR_UNSUPPORTED, "exactly one output relation is supported");
+    ja_status_t st;
+    for (int k = 0; k < n_in; ++k)
+        if ((st = check_tiling(spec, k, inputs[k])) != JA_OK) return st;
+    ja_relation* out = outputs[0];
+    if ((st = check_tiling(spec, -1, out)) != JA_OK) return st;
+    for (int k = 0; k < n_in; ++k)
+        if (inputs[k]->base == out->base) return ja_fail(JA_ERR_INVALID_ARG, "output aliases input %d", k);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const ja_fn_t fn = spec->fn;
+    const ja_agg_t agg = spec->agg;
+    const std::vector<std::string>& in = spec->ins;
+    const std::string& o = spec->out;
+
+    // plan cache
+    std::vector<uint64_t> key;
+    for (int k = 0; k < n_in; ++k) key.push_back(inputs[k]->id);
+    key.push_back(out->id);
+    std::shared_ptr<ExecPlan>& plan = spec->plans[key];
+    if (!plan) plan.reset(new ExecPlan());
+
+    for (int k = 0; k < n_in; ++k)
+        if ((st = ja_relation_to_device(inputs[k])) != JA_OK) return st;
+    if ((st = ja_relation_to_device(out)) != JA_OK) return st;
+
+    // ---- matmul: "ij,jk->ik" MUL / SUM --------------------------------------------------------------
+    if (fn == JA_FN_MUL && agg == JA_AGG_SUM && n_in == 2 && in[0].size() == 2 && in[1].size() == 2 && o.size() == 2 &&
+        in[0][1] == in[1][0] && o[0] == in[0][0] && o[1] == in[1][1] && in[0][0] != in[1][1]) {
+        const ja_relation *A = inputs[0], *B = inputs[1];
+        if (A->dtype != B->dtype || A->dtype != out->dtype) return ja_fail(JA_ERR_DTYPE, "matmul operands must share one dtype");
+        if (A->dtype == JA_BF16) {
+            if (!plan->gemm_checked) {
+                bool ok = false;
+                if ((st = ja_gemm_tc_plan(A, B, out, &plan->gemm, &ok)) != JA_OK) return st;
+                if (!ok) plan->gemm.reset();
+                plan->gemm_checked = true;
+            }
+            if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
+        }
+        return ja_launch_matmul_simt(ja_view(A), ja_view(B), ja_view(out), A->dtype, stream);
+    }
+
+    // ---- key-aligned maps "X,X->X" ----------------------------------------------------------------------
+    if ((fn == JA_FN_ADD || fn == JA_FN_SILU_MUL) && agg == JA_AGG_NONE && n_in == 2 && in[0] == in[1] && in[0] == o) {
+        if (inputs[0]->dtype != inputs[1]->dtype || inputs[0]->dtype != out->dtype)
+            return ja_fail(JA_ERR_DTYPE, "key-aligned join needs one dtype");
+        // identical tilings => identical payload layouts: the join pairs blocks with equal keys, and inside a
+        // block cells with equal offsets
+        return ja_launch_flat(fn, inputs[0]->base, inputs[1]->base, out->base, (int64_t)(out->bytes / out->esize),
+                              out->dtype, stream);
+    }
+
+    // ---- row-structured forms -------------------------------------------------------------------------------
+    RowArgs ra;
+    memset(&ra, 0, sizeof ra);
+    const std::string& x = in[0];
+    const std::string R = lead_of(x);
+    const bool x_ok = x.size() >= 2;
+    auto stat_ok = [&](const ja_relation* r) { return r->dtype == JA_F32; };
+    if (x_ok && fn == JA_FN_SQUARE && agg == JA_AGG_SUM && n_in == 1 && o == R) {
+        if (!stat_ok(out)) return ja_fail(JA_ERR_DTYPE, "statistics relations are f32");
+        ra.x = ja_view(inputs[0]); ra.s0 = ja_view(out);
+        return ja_launch_row(ROW_SUMSQ, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_IDENT && agg == JA_AGG_MAX && n_in == 1 && o == R) {
+        if (!stat_ok(out)) return ja_fail(JA_ERR_DTYPE, "statistics relations are f32");
+        ra.x = ja_view(inputs[0]); ra.s0 = ja_view(out);
+        return ja_launch_row(ROW_MAX, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_EXP_SUB && agg == JA_AGG_SUM && n_in == 2 && in[1] == R && o == R) {
+        if (!stat_ok(out) || !stat_ok(inputs[1])) return ja_fail(JA_ERR_DTYPE, "statistics relations are f32");
+        ra.x = ja_view(inputs[0]); ra.s0 = ja_view(inputs[1]); ra.s1 = ja_view(out);
+        return ja_launch_row(ROW_EXPSUM, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_RMS_SCALE && agg == JA_AGG_NONE && n_in == 3 && in[1] == R && in[2] == x.substr(x.size() - 1) && o == x) {
+        if (!stat_ok(inputs[1]) || inputs[2]->dtype != inputs[0]->dtype || out->dtype != inputs[0]->dtype)
+            return ja_fail(JA_ERR_DTYPE, "RMS_SCALE: x, g, y share a dtype; ss is f32");
+        ra.x = ja_view(inputs[0]); ra.s0 = ja_view(inputs[1]); ra.g = ja_view(inputs[2]); ra.y = ja_view(out);
+        ra.eps = spec->params.empty() ? 1e-5f : (float)spec->params[0];
+        return ja_launch_row(ROW_RMS_SCALE, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_EXP_SUB_DIV && agg == JA_AGG_NONE && n_in == 3 && in[1] == R && in[2] == R && o == x) {
+        if (!stat_ok(inputs[1]) || !stat_ok(inputs[2]) || out->dtype != inputs[0]->dtype)
+            return ja_fail(JA_ERR_DTYPE, "EXP_SUB_DIV: x, y share a dtype; m, l are f32");
+        ra.x = ja_view(inputs[0]); ra.s0 = ja_view(inputs[1]); ra.s1 = ja_view(inputs[2]); ra.y = ja_view(out);
+        return ja_launch_row(ROW_EXP_SUB_DIV, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_RMSNORM && agg == JA_AGG_NONE && n_in == 2 && in[1] == x.substr(x.size() - 1) && o == x) {
+        if (inputs[1]->dtype != inputs[0]->dtype || out->dtype != inputs[0]->dtype)
+            return ja_fail(JA_ERR_DTYPE, "RMSNORM: x, g, y share a dtype");
+        ra.x = ja_view(inputs[0]); ra.g = ja_view(inputs[1]); ra.y = ja_view(out);
+        ra.eps = spec->params.empty() ? 1e-5f : (float)spec->params[0];
+        return ja_launch_row(ROW_RMSNORM, ra, inputs[0]->dtype, stream);
+    }
+    if (x_ok && fn == JA_FN_SOFTMAX && agg == JA_AGG_NONE && n_in == 1 && o == x) {
+        if (out->dtype != inputs[0]->dtype) return ja_fail(JA_ERR_DTYPE, "SOFTMAX: x, y share a dtype");
+        ra.x = ja_view(inputs[0]); ra.y = ja_view(out);
+        return ja_launch_row(ROW_SOFTMAX, ra, inputs[0]->dtype, stream);
+    }
+    if (fn == JA_FN_ROPE && agg == JA_AGG_NONE && n_in == 1 && x.size() == 4 && o == x) {
+        if (out->dtype != inputs[0]->dtype) return ja_fail(JA_ERR_DTYPE, "ROPE: x, y share a dtype");
+        const ja_relation* X = inputs[0];
+        const int64_t S = X->extent[1], D = X->extent[3];
+        if (D % 2) return ja_fail(JA_ERR_SHAPE, "ROPE needs an even last extent");
+        for (int64_t sp : X->splits[3])
+            if (sp % 2) return ja_fail(JA_ERR_TILING, "ROPE: the last index may be split at even positions only");
+        if (!plan->rope_table) {
+            // rotation relation R[s,p] = (cos, sin)(s * theta^(-2p/d)), evaluated in fp64, stored in f32
+            const double theta = spec->params.empty() ? 1e4 : spec->params[0];
+            std::vector<float2> tab((size_t)S * (D / 2));
+            for (int64_t s = 0; s < S; ++s)
+                for (int64_t p = 0; p < D / 2; ++p) {
+                    double phi = (double)s * std::pow(theta, -2.0 * (double)p / (double)D);
+                    tab[s * (D / 2) + p] = make_float2((float)std::cos(phi), (float)std::sin(phi));
+                }
+            JA_CUDA(cudaMalloc((void**)&plan->rope_table, tab.size() * sizeof(float2)));
+            JA_CUDA(cudaMemcpy(plan->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice));
+        }
+        ra.x = ja_view(X); ra.y = ja_view(out); ra.rope_table = plan->rope_table;
+        return ja_launch_row(ROW_ROPE, ra, X->dtype, stream);
+    }
+
+    // ---- attention: "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX --------------------------------------
+    if (fn == JA_FN_ATTENTION && agg == JA_AGG_ONLINE_SOFTMAX && n_in == 3 && x.size() == 4 && in[1].size() == 4 &&
+        in[1] == in[2] && o == x && in[1][0] == x[0] && in[1][2] == x[2] && in[1][3] == x[3] && in[1][1] != x[1]) {
+        const ja_relation *Q = inputs[0], *K = inputs[1], *V = inputs[2];
+        if (Q->dtype != JA_BF16 || K->dtype != JA_BF16 || V->dtype != JA_BF16 || out->dtype != JA_BF16)
+            return ja_fail(JA_ERR_DTYPE, "attention relations must be bf16");
+        if (Q->extent[3] != 128 || Q->nblk[3] != 1) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs an unsplit last index of extent 128");
+        if (Q->extent[1] != K->extent[1]) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs equal query and key extents");
+        if (!Q->equal_blocks || !K->equal_blocks) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs uniform blocks");
+        AttnArgs aa;
+        memset(&aa, 0, sizeof aa);
+        aa.q = ja_view(Q); aa.k = ja_view(K); aa.v = ja_view(V); aa.o = ja_view(out);
+        aa.B = (int32_t)Q->extent[0]; aa.S = (int32_t)Q->extent[1]; aa.H = (int32_t)Q->extent[2]; aa.D = 128;
+        aa.qblk = (int32_t)Q->bs[1]; aa.kblk = (int32_t)K->bs[1]; aa.hblk = (int32_t)Q->bs[2];
+        if (aa.qblk % 64 || aa.kblk % 64) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs q/k blocks that are multiples of 64 rows");
+        aa.scale = spec->params.size() >= 1 ? (float)spec->params[0] : 0.08838834764831845f;
+        aa.causal = spec->params.size() >= 2 ? (spec->params[1] != 0.0) : 1;
+        return ja_launch_attention(aa, stream);
+    }
+
+    return ja_fail(JA_ERR_UNSUPPORTED, "no kernel for einsum '%s' with fn %d / agg %d", spec->einsum.c_str(), (int)fn,
+                   (int)agg);
+}

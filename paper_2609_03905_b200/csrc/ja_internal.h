@@ -1,0 +1,129 @@
+// Internal declarations of libja (host bookkeeping + kernel launchers). Not part of the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "ja.h"
+
+#define JA_MAX_RANK 4
+#define JA_MAX_IN 4
+#define JA_ALIGN 128
+
+// ---- device-side view of a tensor relation (passed to kernels by value) -------------------------
+// Key table on the device: per-dimension split points and per-block byte offsets. A kernel turns a
+// tensor coordinate into (block key, offset inside the block) with these and nothing else.
+struct RelView {
+    char* base;                          // payload
+    const int64_t* splits[JA_MAX_RANK];  // device; splits[d][0..nblk[d]]
+    const int64_t* blk_off;              // device; byte offset of every block, row-major key order
+    int64_t extent[JA_MAX_RANK];
+    int64_t bs[JA_MAX_RANK];             // uniform block size of dimension d, or 0 if irregular
+    int32_t nblk[JA_MAX_RANK];
+    int32_t rank;
+    int32_t esize;
+};
+
+struct ja_relation {
+    int32_t rank = 0;
+    int64_t extent[JA_MAX_RANK] = {0, 0, 0, 0};
+    int32_t nblk[JA_MAX_RANK] = {1, 1, 1, 1};
+    std::vector<int64_t> splits[JA_MAX_RANK];
+    int64_t bs[JA_MAX_RANK] = {0, 0, 0, 0};
+    ja_dtype_t dtype = JA_BF16;
+    int32_t esize = 2;
+    void* base = nullptr;
+    size_t bytes = 0;         // payload size implied by the tiling
+    int64_t nblocks = 0;
+    std::vector<int64_t> blk_off;  // bytes
+    bool equal_blocks = false;     // every block has the same shape (constant block stride)
+    uint64_t id = 0;
+    // lazily created device copies of the key table
+    mutable int64_t* d_tables = nullptr;
+    mutable bool on_device = false;
+};
+
+struct ExecPlan;  // per (spec, relations) cached launch state
+
+struct ja_spec {
+    std::string einsum;
+    std::vector<std::string> ins;
+    std::string out;
+    std::string letters;  // order of first appearance
+    std::vector<std::vector<int64_t>> parts;  // per letter: split points
+    ja_fn_t fn = JA_FN_MUL;
+    ja_agg_t agg = JA_AGG_SUM;
+    std::vector<double> params;
+    int64_t p = 0;
+    std::vector<int32_t> in_keys;   // [p][n_in]
+    std::vector<int32_t> out_keys;  // [p]
+    mutable std::map<std::vector<uint64_t>, std::shared_ptr<ExecPlan>> plans;
+};
+
+// ---- helpers implemented in ja_host.cu ------------------------------------------------------------
+ja_status_t ja_fail(ja_status_t st, const char* fmt, ...);
+ja_status_t ja_cuda_fail(cudaError_t e, const char* what);
+ja_status_t ja_relation_to_device(const ja_relation* r);
+RelView ja_view(const ja_relation* r);
+int* ja_device_status_word();
+void ja_count_launch(int n = 1);
+
+#define JA_CUDA(call)                                              \
+    do {                                                           \
+        cudaError_t e_ = (call);                                   \
+        if (e_ != cudaSuccess) return ja_cuda_fail(e_, #call);     \
+    } while (0)
+
+// ---- kernel launchers (one per .cu file) ------------------------------------------------------------
+// Plain-ALU tiled matmul join-agg over arbitrary tilings (f32 or bf16 operands, f32 accumulate).
+ja_status_t ja_launch_matmul_simt(const RelView& A, const RelView& B, const RelView& C, ja_dtype_t dt,
+                                  cudaStream_t st);
+
+// Memory-bound join-aggs: flat key-aligned maps and row-structured maps / reductions.
+enum RowOp {
+    ROW_SUMSQ = 0, ROW_MAX, ROW_EXPSUM, ROW_RMS_SCALE, ROW_EXP_SUB_DIV, ROW_RMSNORM, ROW_SOFTMAX, ROW_ROPE
+};
+struct RowArgs {
+    RelView x;     // [R..., j] input
+    RelView s0;    // statistics relation keyed by R (ss or m) -- input or output depending on op
+    RelView s1;    // second statistics relation (l)
+    RelView g;     // [j] gain vector
+    RelView y;     // [R..., j] output
+    float eps;     // RMS_SCALE / RMSNORM
+    float theta;   // ROPE
+    const float2* rope_table;  // device [extent(s)][d/2] (cos, sin)
+};
+ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st);
+ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,
+                           cudaStream_t st);
+
+// Repartition: list of 2-D slab copies.
+struct CopySlab {
+    int64_t src_off, dst_off;        // bytes
+    int32_t rows, row_bytes;         // slab shape
+    int32_t src_pitch, dst_pitch;    // bytes between consecutive rows
+};
+ja_status_t ja_launch_repartition(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int vec_bytes,
+                                  cudaStream_t st);
+
+// tcgen05 / TMEM / TMA matmul join-agg for bf16 relations with uniform blocks.
+struct GemmTcPlan;
+ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C,
+                            std::shared_ptr<GemmTcPlan>* out, bool* eligible);
+ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st);
+
+// Attention join-agg (QK^T join, online-softmax aggregation, PV).
+struct AttnArgs {
+    RelView q, k, v, o;
+    float scale;
+    int causal;
+    int32_t B, S, H, D;
+    int32_t qblk, kblk;    // rows per q block / k block (uniform)
+    int32_t hblk;          // heads per block
+};
+ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);

@@ -1,0 +1,254 @@
+// Dot-product attention as a join-agg: "bqhd,bkhd,bkhd->bqhd", f = ATTENTION, (+) = online softmax.
+//
+// One CTA owns one output key tile: QT query rows of one (batch, head). It walks the function specs that
+// share that output key -- the key/value blocks kb that survive the causal band predicate -- in ascending
+// order. For each joined tuple (Q block, K block, V block) the concrete operator computes the partial
+// triple (O~, m, l) of the block pair; the running triple kept in registers is combined with it by
+//     m* = max(m, m'),  O~ <- O~ e^(m-m*) + O~' e^(m'-m*),  l <- l e^(m-m*) + l' e^(m'-m*)
+// which is the aggregation operator of the spec. O = O~/l is written once, to the key's offset in the
+// output relation. Scores and probabilities never reach HBM.
+//
+// This version feeds the tensor cores through mma.sync (m16n8k16, bf16 in, fp32 accumulate); operands are
+// staged in shared memory with cp.async under an XOR swizzle and read with ldmatrix.
+#include "ja_device.cuh"
+
+namespace {
+
+constexpr int D = 128;     // head dimension (extent of the unsplit last index)
+constexpr int KT = 64;     // key rows per inner step
+constexpr int ROW_BYTES = D * 2;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// byte address inside a [rows][128] bf16 tile whose 16-byte chunks are XOR-swizzled by the row
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); }
+
+// pointer to cell (b, s, h, 0) of a "bshd" relation, and the byte pitch between consecutive s inside the block
+__device__ __forceinline__ const char* row_ptr(const RelView& v, int b, int s, int h, int64_t* pitch) {
+    const int bb = ja_find_blk(v, 0, b), sb = ja_find_blk(v, 1, s), hb = ja_find_blk(v, 2, h);
+    const int64_t blo = v.splits[0][bb], slo = v.splits[1][sb], hlo = v.splits[2][hb];
+    const int64_t sw = v.splits[1][sb + 1] - slo, hw = v.splits[2][hb + 1] - hlo;
+    const int64_t flat = ((int64_t)bb * v.nblk[1] + sb) * v.nblk[2] + hb;
+    *pitch = hw * D * 2;
+    return v.base + v.blk_off[flat] + ((((int64_t)(b - blo) * sw + (s - slo)) * hw + (h - hlo)) * D) * 2;
+}
+
+template <int QT>
+__global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
+    constexpr int NW = QT / 16;        // warps; each owns 16 query rows
+    constexpr int NT = NW * 32;
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint8_t* sQ = smem;                          // QT x 128 (reused to stage O)
+    uint8_t* sK = smem + QT * ROW_BYTES;         // 2 x KT x 128
+    uint8_t* sV = sK + 2 * KT * ROW_BYTES;       // 2 x KT x 128
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int g = lane / 4, t4 = lane % 4;
+
+    const int n_qt = a.S / QT;
+    const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest output keys (most surviving tuples) first
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int q0 = qt * QT;
+
+    // ---- stage Q, read its A fragments ---------------------------------------------------------------------
+    {
+        int64_t pitch;
+        const char* qp = row_ptr(a.q, b, q0, h, &pitch);  // a q tile never leaves its block (QT divides qblk)
+        for (int i = tid; i < QT * 16; i += NT) {
+            int r = i / 16, c = i % 16;
+            cp_async16(smem_u32(sQ) + swz(r, c), qp + (int64_t)r * pitch + c * 16);
+        }
+        cp_async_commit();
+    }
+    // number of 64-row key steps this output key joins with: keys [0, q0 + QT) when causal
+    const int k_end = a.causal ? min(a.S, q0 + QT) : a.S;
+    const int n_steps = (k_end + KT - 1) / KT;
+
+    auto load_kv = [&](int step, int buf) {
+        const int k0 = step * KT;  // a 64-row step never straddles a key block (64 divides kblk)
+        int64_t pk, pv;
+        const char* kp = row_ptr(a.k, b, k0, h, &pk);
+        const char* vp = row_ptr(a.v, b, k0, h, &pv);
+        const uint32_t dk = smem_u32(sK) + buf * KT * ROW_BYTES, dv = smem_u32(sV) + buf * KT * ROW_BYTES;
+        for (int i = tid; i < KT * 16; i += NT) {
+            int r = i / 16, c = i % 16;
+            cp_async16(dk + swz(r, c), kp + (int64_t)r * pk + c * 16);
+            cp_async16(dv + swz(r, c), vp + (int64_t)r * pv + c * 16);
+        }
+        cp_async_commit();
+    };
+    load_kv(0, 0);
+
+    cp_async_wait<1>();  // Q has landed
+    __syncthreads();
+    uint32_t qf[8][4];
+    {
+        const int r = warp * 16 + (lane % 8) + 8 * ((lane / 8) % 2);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const int chunk = ks * 2 + lane / 16;
+            ldmatrix_x4(smem_u32(sQ) + swz(r, chunk), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+        }
+    }
+
+    float o[16][4];
+#pragma unroll
+    for (int n = 0; n < 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const float sl2 = a.scale * 1.4426950408889634f;  // scores are kept in the base-2 exponent domain
+    const int row0 = q0 + warp * 16 + g;              // sequence position of this thread's first row (second: +8)
+
+    for (int step = 0; step < n_steps; ++step) {
+        const int buf = step & 1;
+        if (step + 1 < n_steps) { load_kv(step + 1, buf ^ 1); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();
+        const uint32_t kbase = smem_u32(sK) + buf * KT * ROW_BYTES, vbase = smem_u32(sV) + buf * KT * ROW_BYTES;
+
+        // ---- S = Q K^T for 16 rows x 64 keys -------------------------------------------------------------------
+        float s[8][4];
+#pragma unroll
+        for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {  // pairs of 8-key tiles
+                const int mi = lane / 8;
+                const int krow = np * 16 + (mi / 2) * 8 + (lane % 8);
+                const int chunk = ks * 2 + (mi % 2);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4(kbase + swz(krow, chunk), b0, b1, b2, b3);
+                mma_bf16(s[2 * np], qf[ks], b0, b1);
+                mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
+            }
+        }
+        // ---- scale, causal band inside the diagonal block, row max ---------------------------------------------
+        const int k0 = step * KT;
+        const bool diag = a.causal && (k0 + KT - 1 > q0 + warp * 16);
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float v = s[n][e] * sl2;
+                if (diag) {
+                    const int key = k0 + n * 8 + 2 * t4 + (e & 1);
+                    const int row = row0 + 8 * (e >> 1);
+                    if (key > row) v = -INFINITY;
+                }
+                s[n][e] = v;
+                mx[e >> 1] = fmaxf(mx[e >> 1], v);
+            }
+        }
+        float alpha[2], m_use[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+            const float m_new = fmaxf(m_run[r], mx[r]);
+            m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;               // e^(-inf - -inf) := 0
+            alpha[r] = (m_run[r] == -INFINITY) ? 0.f : exp2f(m_run[r] - m_use[r]);
+            m_run[r] = m_new;
+        }
+        // ---- P = 2^(S - m), row sums, O~ <- O~ alpha ----------------------------------------------------------------
+        float ls[2] = {0.f, 0.f};
+        uint32_t pf[4][4];
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+            float p0 = exp2f(s[n][0] - m_use[0]), p1 = exp2f(s[n][1] - m_use[0]);
+            float p2 = exp2f(s[n][2] - m_use[1]), p3 = exp2f(s[n][3] - m_use[1]);
+            ls[0] += p0 + p1;
+            ls[1] += p2 + p3;
+            pf[n / 2][(n % 2) * 2 + 0] = pack_bf16(p0, p1);
+            pf[n / 2][(n % 2) * 2 + 1] = pack_bf16(p2, p3);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * alpha[r] + ls[r];
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+            o[n][0] *= alpha[0]; o[n][1] *= alpha[0];
+            o[n][2] *= alpha[1]; o[n][3] *= alpha[1];
+        }
+        // ---- O~ += P V ----------------------------------------------------------------------------------------------
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {      // 16 keys per step
+#pragma unroll
+            for (int np = 0; np < 8; ++np) {  // pairs of 8-wide d tiles
+                const int mi = lane / 8;
+                const int vrow = ks * 16 + (mi % 2) * 8 + (lane % 8);
+                const int chunk = np * 2 + (mi / 2);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(vbase + swz(vrow, chunk), b0, b1, b2, b3);
+                mma_bf16(o[2 * np], pf[ks], b0, b1);
+                mma_bf16(o[2 * np + 1], pf[ks], b2, b3);
+            }
+        }
+        __syncthreads();  // everyone is done with this buffer before it is refilled
+    }
+
+    // ---- finish: O = O~ / l, stage through shared memory, 16-byte stores --------------------------------------------
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+    }
+    const float inv0 = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f, inv1 = l_run[1] > 0.f ? 1.f / l_run[1] : 0.f;
+    {
+        const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+            // columns n*8 + 2*t4, +1  -> chunk n, byte (2*t4)*2 inside it
+            *reinterpret_cast<uint32_t*>(sQ + swz(r_lo, n) + t4 * 4) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
+            *reinterpret_cast<uint32_t*>(sQ + swz(r_hi, n) + t4 * 4) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
+        }
+    }
+    __syncthreads();
+    {
+        int64_t pitch;
+        char* op = const_cast<char*>(row_ptr(a.o, b, q0, h, &pitch));
+        for (int i = tid; i < QT * 16; i += NT) {
+            int r = i / 16, c = i % 16;
+            *reinterpret_cast<uint4*>(op + (int64_t)r * pitch + c * 16) = *reinterpret_cast<const uint4*>(sQ + swz(r, c));
+        }
+    }
+}
+
+}  // namespace
+
+ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
+    const int QT = (a.qblk % 128 == 0) ? 128 : 64;
+    dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
+    const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
+    if (QT == 128) {
+        JA_CUDA(cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attention_kernel<128><<<grid, 256, smem, st>>>(a);
+    } else {
+        JA_CUDA(cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attention_kernel<64><<<grid, 128, smem, st>>>(a);
+    }
+    ja_count_launch();
+    JA_CUDA(cudaGetLastError());
+    return JA_OK;
+}

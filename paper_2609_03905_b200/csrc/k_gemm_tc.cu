@@ -1,0 +1,439 @@
+// Tensor-core matmul join-agg "ij,jk->ik" (MUL / SUM) for bf16 relations with uniform blocks.
+//
+// One persistent CTA per SM. For every output tile (128 rows x up to 256 columns of ONE output key, or of
+// several adjacent output keys when blocks are narrow) the CTA walks the function specs that share that
+// output key in ascending order of the contracted block index j -- the SUM aggregation of Definition 3.7 is
+// the accumulation of all those tuples into one fp32 accumulator in tensor memory; only the aggregated block
+// is written (Recompose = the store at the key's offset).
+//
+//   warp 0      TMA producer: cp.async.bulk.tensor straight from the block-key layout. A relation with
+//               uniform blocks is a rank-4 tensor (col in block, row in block, col-block, row-block), so one
+//               tensor map per operand addresses every block; ragged tiles rely on zero fill inside a block.
+//   warp 1      tcgen05.mma issuer (one elected lane), kind::f16, M=128, N<=256, K=16, A K-major and
+//               B MN-major (weights are [in, out] row-major), both under the 128-byte swizzle.
+//   warps 2..5  epilogue: tcgen05.ld of the fp32 accumulator, one RNE rounding to bf16, 16-byte stores.
+//
+// Two accumulator stages (2 x 256 TMEM columns) let the epilogue of tile t overlap the mainloop of tile t+1.
+// Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT, drains its copies and exits.
+#include <cuda.h>
+
+#include "ja_device.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
+constexpr int B_STAGE_BYTES = BK * BN * 2;   // 32 KiB
+constexpr int B_CHUNK_BYTES = BK * 64 * 2;   // one 64-column box: 8 KiB
+constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int NUM_THREADS = 192;
+
+struct GemmParams {
+    char* c_base;
+    const int64_t* c_blk_off;  // device: byte offsets of the output blocks
+    int32_t* status;           // device status word
+    int32_t bm, bk, bn;        // block extents along i, j, k
+    int32_t nbm, nbk, nbn;     // blocks along i, j, k
+    int32_t M, N;              // tensor extents along i, k
+    int32_t a_box_rows;        // rows per A box (= min(bm, 128))
+    int32_t m_tiles, n_tiles;  // tile grid
+    int32_t tiles_per_mblk;    // >= 1 when bm >= 128 (tiles never leave a block), 0 when tiles span blocks
+    int32_t tiles_per_nblk;    // >= 1 when tiles stay inside one column block, 0 when tiles span blocks
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after ~2 s, records the failure and raises the CTA-wide abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 63) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > 2000000000ull) {
+                *abort_flag = 1;
+                atomicExch(status, (int)JA_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// shared-memory matrix descriptors, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version for this architecture
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+
+struct TileCoord {
+    int mb, r0;          // row block, first row inside it (tiles that stay inside a block)
+    int row_g0;          // first global row (tiles that span blocks)
+    int n_g0, nb, c0;    // first global column / column block and first column inside it
+    int width;           // valid columns (multiple of 8)
+    int rows;            // valid rows
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t) {
+    TileCoord tc;
+    const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+    if (p.tiles_per_mblk > 0) {
+        tc.mb = mt / p.tiles_per_mblk;
+        tc.r0 = (mt % p.tiles_per_mblk) * BM;
+        tc.rows = min(BM, p.bm - tc.r0);
+        tc.row_g0 = tc.mb * p.bm + tc.r0;
+    } else {
+        tc.row_g0 = mt * BM;
+        tc.mb = tc.row_g0 / p.bm;
+        tc.r0 = 0;
+        tc.rows = min(BM, p.M - tc.row_g0);
+    }
+    if (p.tiles_per_nblk > 0) {
+        tc.nb = nt / p.tiles_per_nblk;
+        tc.c0 = (nt % p.tiles_per_nblk) * BN;
+        tc.width = min(BN, p.bn - tc.c0);
+        tc.n_g0 = tc.nb * p.bn + tc.c0;
+    } else {
+        tc.n_g0 = nt * BN;
+        tc.nb = tc.n_g0 / p.bn;
+        tc.c0 = tc.n_g0 % p.bn;
+        tc.width = min(BN, p.N - tc.n_g0);
+    }
+    return tc;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t sA = base, sB = base + STAGES * A_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // allocate all 512 TMEM columns (two 128 x 256 fp32 accumulators)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int kchunks = (p.bk + BK - 1) / BK;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t last_parity[STAGES];
+            bool issued[STAGES];
+            for (int s = 0; s < STAGES; ++s) { last_parity[s] = 0; issued[s] = false; }
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const TileCoord tc = tile_coord(p, t);
+                const int nchunks = (tc.width + 63) / 64;
+                const uint32_t tx = A_STAGE_BYTES + nchunks * B_CHUNK_BYTES;
+                for (int jb = 0; jb < p.nbk && ok; ++jb) {          // the tuples of this output key, ascending j
+                    for (int kc = 0; kc < kchunks; ++kc) {
+                        if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, p.status)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(stage), tx);
+                        issued[stage] = true;
+                        last_parity[stage] = phase;
+                        // A: boxes of a_box_rows rows x 64 k
+                        const int nboxes = BM / p.a_box_rows;
+                        for (int bx = 0; bx < nboxes; ++bx) {
+                            int mb = tc.mb + (p.tiles_per_mblk > 0 ? 0 : bx);
+                            int r0 = p.tiles_per_mblk > 0 ? tc.r0 : 0;
+                            tma_load_4d(sA + stage * A_STAGE_BYTES + bx * p.a_box_rows * 128, &tmA, full_bar(stage),
+                                        kc * BK, r0, jb, mb);
+                        }
+                        // B: one box of 64 k-rows x 64 columns per 64-column chunk of the tile
+                        for (int c = 0; c < nchunks; ++c) {
+                            int nb, cin;
+                            if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + 64 * c; }
+                            else { int g = tc.n_g0 + 64 * c; nb = g / p.bn; cin = g % p.bn; }
+                            tma_load_4d(sB + stage * B_STAGE_BYTES + c * B_CHUNK_BYTES, &tmB, full_bar(stage), cin,
+                                        kc * BK, nb, jb);
+                        }
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+            if (!ok) {  // drain: wait (bounded) for copies already in flight before the CTA may exit
+                for (int s = 0; s < STAGES; ++s) {
+                    if (!issued[s]) continue;
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(full_bar(s), last_parity[s]) && global_ns() - t0 < 200000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t acc_phase[2] = {0, 0};
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+                const TileCoord tc = tile_coord(p, t);
+                const int acc = it & 1;
+                const uint32_t n_mma = (uint32_t)((tc.width + 15) / 16 * 16);
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((n_mma >> 3) << 17) | ((BM >> 4) << 24);
+                if (!mbar_wait(tempty_bar(acc), acc_phase[acc] ^ 1, abort_flag, p.status)) { ok = false; break; }
+                acc_phase[acc] ^= 1;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                uint32_t accumulate = 0;
+                for (int jb = 0; jb < p.nbk && ok; ++jb) {
+                    for (int kc = 0; kc < kchunks; ++kc) {
+                        if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        const int kvalid = min(BK, p.bk - kc * BK);
+                        const int k16 = (kvalid + 15) / 16;
+                        const uint32_t a_addr = sA + stage * A_STAGE_BYTES;
+                        const uint32_t b_addr = sB + stage * B_STAGE_BYTES;
+                        for (int kk = 0; kk < k16; ++kk) {
+                            // A: K-major, 16 k = 32 bytes inside the swizzle atom; B: MN-major, 16 k-rows = 2048 bytes
+                            uint64_t da = desc_sw128(a_addr + kk * 32, 16);
+                            uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
+                            umma_bf16(d_tmem, da, db, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(empty_bar(stage));  // frees the smem stage once these MMAs have read it
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
+                if (ok) umma_commit(tfull_bar(acc));    // accumulator complete -> epilogue
+            }
+        }
+    } else {
+        // ================= epilogue (warps 2..5) =================
+        const int q = warp & 3;  // TMEM lane group this warp may access
+        uint32_t acc_phase[2] = {0, 0};
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            const TileCoord tc = tile_coord(p, t);
+            const int acc = it & 1;
+            if (!mbar_wait(tfull_bar(acc), acc_phase[acc], abort_flag, p.status)) { ok = false; break; }
+            acc_phase[acc] ^= 1;
+            tc_fence_after();
+            const int r = q * 32 + lane;                     // row of the tile held by this thread
+            const int grow = tc.row_g0 + r;                  // global row
+            const bool row_ok = r < tc.rows;
+            int ib = 0, iin = 0;
+            if (row_ok) { ib = grow / p.bm; iin = grow % p.bm; }
+            for (int ch = 0; ch * 32 < tc.width; ++ch) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + ch * 32, v);
+                tmem_ld_wait();
+                if (row_ok) {
+                    const int gcol = tc.n_g0 + ch * 32;
+                    const int kb = gcol / p.bn, cin = gcol % p.bn;
+                    char* dst = p.c_base + p.c_blk_off[(int64_t)ib * p.nbn + kb] + ((int64_t)iin * p.bn + cin) * 2;
+                    const int valid = min(32, tc.width - ch * 32);  // multiple of 8
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g * 8 < valid) {
+                            uint4 o;
+                            __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                po[e] = __floats2bfloat162_rn(__uint_as_float(v[g * 8 + 2 * e]), __uint_as_float(v[g * 8 + 2 * e + 1]));
+                            *reinterpret_cast<uint4*>(dst + g * 16) = o;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
+    }
+    // ---- teardown ---------------------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+// ---- host: tensor maps -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// A relation [R, C] with equal blocks br x bc is the rank-4 tensor (c in block, r in block, col-block, row-block).
+ja_status_t encode_blocked_2d(const ja_relation* r, int box_inner, int box_rows, CUtensorMap* tm) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const int64_t br = r->bs[0], bc = r->bs[1];
+    const int64_t blk_stride = r->nblocks > 1 ? r->blk_off[1] - r->blk_off[0] : (int64_t)r->bytes;
+    cuuint64_t dims[4] = {(cuuint64_t)bc, (cuuint64_t)br, (cuuint64_t)r->nblk[1], (cuuint64_t)r->nblk[0]};
+    cuuint64_t strides[3] = {(cuuint64_t)(bc * 2), (cuuint64_t)blk_stride, (cuuint64_t)(blk_stride * r->nblk[1])};
+    cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, r->base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)res);
+    return JA_OK;
+}
+
+}  // namespace
+
+struct GemmTcPlan {
+    CUtensorMap tmA, tmB;
+    GemmParams p;
+    int grid;
+};
+
+ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C,
+                            std::shared_ptr<GemmTcPlan>* out, bool* eligible) {
+    *eligible = false;
+    if (!A->equal_blocks || !B->equal_blocks || !C->equal_blocks) return JA_OK;
+    const int64_t bm = A->bs[0], bk = A->bs[1], bn = B->bs[1];
+    // TMA needs 16-byte row pitches; boxes are 64 elements wide; A boxes hold min(bm,128) rows
+    if (bk % 8 || bn % 8 || bk < 64 || bn < 64) return JA_OK;
+    if (bm < 128 && (128 % bm != 0 || bm % 8 != 0)) return JA_OK;
+    if (A->extent[0] >= (1ll << 31) || B->extent[1] >= (1ll << 31)) return JA_OK;
+    std::shared_ptr<GemmTcPlan> plan(new GemmTcPlan());
+    GemmParams& p = plan->p;
+    p.c_base = (char*)C->base;
+    p.c_blk_off = ja_view(C).blk_off;
+    p.status = ja_device_status_word();
+    if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    p.bm = (int)bm; p.bk = (int)bk; p.bn = (int)bn;
+    p.nbm = A->nblk[0]; p.nbk = A->nblk[1]; p.nbn = B->nblk[1];
+    p.M = (int)A->extent[0]; p.N = (int)B->extent[1];
+    p.a_box_rows = (int)std::min<int64_t>(bm, 128);
+    if (bm >= 128) { p.tiles_per_mblk = (int)((bm + BM - 1) / BM); p.m_tiles = p.tiles_per_mblk * p.nbm; }
+    else { p.tiles_per_mblk = 0; p.m_tiles = (p.M + BM - 1) / BM; }
+    if (bn % 64 == 0 && bn < BN && p.nbn > 1) { p.tiles_per_nblk = 0; p.n_tiles = (p.N + BN - 1) / BN; }
+    else { p.tiles_per_nblk = (int)((bn + BN - 1) / BN); p.n_tiles = p.tiles_per_nblk * p.nbn; }
+    ja_status_t st;
+    if ((st = encode_blocked_2d(A, 64, p.a_box_rows, &plan->tmA)) != JA_OK) return st;
+    if ((st = encode_blocked_2d(B, 64, 64, &plan->tmB)) != JA_OK) return st;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    plan->grid = std::min(sms, p.m_tiles * p.n_tiles);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return ja_cuda_fail(e, "cudaFuncSetAttribute(gemm_tc_kernel)");
+    *out = plan;
+    *eligible = true;
+    return JA_OK;
+}
+
+ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
+    gemm_tc_kernel<<<plan.grid, NUM_THREADS, SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.p);
+    ja_count_launch();
+    JA_CUDA(cudaGetLastError());
+    return JA_OK;
+}

@@ -1,0 +1,136 @@
+"""A LLaMA-shaped transformer block forward as a chain of join-aggs: nothing here computes -- every step is
+one ja_execute or ja_repartition call on relations allocated up front.
+
+    n1 = RMSNorm(x, g1);  q,k,v = n1 Wq, n1 Wk, n1 Wv;  q,k <- RoPE;  att = CausalAttention(q,k,v)
+    h  = x + att Wo;      n2 = RMSNorm(h, g2);  out = h + (silu(n2 W1) * (n2 W3)) W2
+
+Two decompositions (the block's input and output relations are tiled identically in both: 128-token row
+blocks x 8 column blocks):
+
+  "seq"   sequence-blocked: every [tokens, hidden] relation keeps 128 x (hidden/8) blocks; q, k, v are
+          re-tiled to one head per block before attention and the attention output is re-tiled back
+          (the one-GPU image of sequence-parallel outside / head-parallel inside attention).
+  "head"  head-blocked: x is re-tiled once to 128 x 128 blocks (one head per column block); all projections
+          contract over 32 (64) head-sized blocks and emit head-sized blocks, so attention needs no
+          relayout; the block output is re-tiled back at the end.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from . import binding as B
+from .relations import Relation, Spec, equal_splits as ES, from_dense, repartition
+
+
+class LlamaBlock:
+    def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
+                 theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8):
+        assert plan in ("seq", "head")
+        assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
+        assert seq % token_block == 0
+        self.plan, self.B, self.S, self.hidden, self.H, self.ffn = plan, batch, seq, hidden, n_heads, ffn
+        T = batch * seq
+        self.T = T
+        bf = torch.bfloat16
+        D = hidden // n_heads
+        t_sp = ES(T, T // token_block)
+        io_c = ES(hidden, col_blocks)                    # column tiling of the block's input / output
+        head_c = ES(hidden, n_heads)                     # one head per column block
+        act_c = io_c if plan == "seq" else head_c        # column tiling of the plan's [T, hidden] activations
+        ffn_c = ES(ffn, col_blocks)
+        self.t_sp, self.io_c, self.head_c, self.act_c, self.ffn_c = t_sp, io_c, head_c, act_c, ffn_c
+        qkv_c = io_c if plan == "seq" else head_c        # tiling q, k, v are produced in
+
+        def act(cols=act_c):
+            return Relation([T, hidden], [t_sp, cols], bf)
+
+        # ---- relations -------------------------------------------------------------------------------
+        self.x = Relation([T, hidden], [t_sp, io_c], bf)                 # block input (filled by the caller)
+        self.out = Relation([T, hidden], [t_sp, io_c], bf)               # block output
+        self.x_p = self.x if plan == "seq" else act()                    # input in the plan's tiling
+        self.n1, self.h, self.n2, self.o, self.y = act(), act(), act(), act(), act()
+        self.q, self.k, self.v = act(qkv_c), act(qkv_c), act(qkv_c)
+        self.q_r, self.k_r = act(qkv_c), act(qkv_c)                      # after RoPE
+        if plan == "seq":
+            self.q_h, self.k_h, self.v_h, self.att_h = act(head_c), act(head_c), act(head_c), act(head_c)
+            self.att = act()
+        else:
+            self.q_h, self.k_h, self.v_h = self.q_r, self.k_r, self.v
+            self.att_h = self.att = act()
+        self.out_p = self.out if plan == "seq" else act()
+        self.a = Relation([T, ffn], [t_sp, ffn_c], bf)
+        self.b = Relation([T, ffn], [t_sp, ffn_c], bf)
+        self.hh = Relation([T, ffn], [t_sp, ffn_c], bf)
+        # weights [in, out]: rows tiled like the activation they contract with, columns like the result
+        w = {n: weights[n].to("cuda", bf) for n in weights}
+        self.wq, self.wk, self.wv = (from_dense(w[n], [act_c, qkv_c]) for n in ("wq", "wk", "wv"))
+        self.wo = from_dense(w["wo"], [act_c if plan == "seq" else head_c, act_c])
+        self.w1, self.w3 = from_dense(w["w1"], [act_c, ffn_c]), from_dense(w["w3"], [act_c, ffn_c])
+        self.w2 = from_dense(w["w2"], [ffn_c, act_c])
+        self.g1, self.g2 = from_dense(w["g1"], [act_c]), from_dense(w["g2"], [act_c])
+
+        # 4-D views "bshd" over the same payloads (the block layout of [T, hidden] with 128-token row blocks
+        # and whole-head column blocks IS the layout of [b, s, h, d] with blocks [1, 128, heads/block, 128])
+        b_sp, s_sp = ES(batch, batch), ES(seq, seq // token_block)
+
+        def v4(rel: Relation, cols):
+            hb = ES(n_heads, len(cols) - 1)
+            return rel.view_as([batch, seq, n_heads, D], [b_sp, s_sp, hb, [0, D]])
+
+        self.q4, self.k4 = v4(self.q, qkv_c), v4(self.k, qkv_c)
+        self.q4r, self.k4r = v4(self.q_r, qkv_c), v4(self.k_r, qkv_c)
+        self.qa, self.ka, self.va, self.oa = (v4(r, head_c) for r in (self.q_h, self.k_h, self.v_h, self.att_h))
+
+        # ---- specs -------------------------------------------------------------------------------------
+        def mm(jc, kc):
+            return Spec("ij,jk->ik", {"i": t_sp, "j": jc, "k": kc}, "mul", (), "sum")
+
+        self.s_norm = Spec("ij,j->ij", {"i": t_sp, "j": act_c}, "rmsnorm", (eps,), "none")
+        self.s_qkv = mm(act_c, qkv_c)
+        self.s_rope = Spec("bshd->bshd", {"b": b_sp, "s": s_sp, "h": ES(n_heads, len(qkv_c) - 1), "d": [0, D]}, "rope",
+                           (theta,), "none")
+        self.s_attn = Spec("bqhd,bkhd,bkhd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_heads), "d": [0, D], "k": s_sp},
+                           "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
+        self.s_wo = mm(act_c if plan == "seq" else head_c, act_c)
+        self.s_add = Spec("ij,ij->ij", {"i": t_sp, "j": act_c}, "add", (), "none")
+        self.s_up = mm(act_c, ffn_c)
+        self.s_silu = Spec("ij,ij->ij", {"i": t_sp, "j": ffn_c}, "silu_mul", (), "none")
+        self.s_down = mm(ffn_c, act_c)
+        self.n_relayouts = 4 if plan == "seq" else 2
+
+    # flop count of one forward (dense contractions only; causal attention counted at half the square)
+    def flops(self) -> float:
+        T, d, f, S = self.T, self.hidden, self.ffn, self.S
+        return 2.0 * T * d * d * 4 + 2.0 * T * d * f * 3 + 4.0 * T * S * d / 2
+
+    def forward(self, stream: int | None = None) -> Relation:
+        """Enqueue the whole chain on the current stream; returns the output relation (tiled like x)."""
+        p = self.plan
+        if p == "head":
+            repartition(self.x, self.x_p, stream)
+        self.s_norm.execute([self.x_p, self.g1], self.n1, stream)
+        self.s_qkv.execute([self.n1, self.wq], self.q, stream)
+        self.s_qkv.execute([self.n1, self.wk], self.k, stream)
+        self.s_qkv.execute([self.n1, self.wv], self.v, stream)
+        self.s_rope.execute([self.q4], self.q4r, stream)
+        self.s_rope.execute([self.k4], self.k4r, stream)
+        if p == "seq":
+            repartition(self.q_r, self.q_h, stream)
+            repartition(self.k_r, self.k_h, stream)
+            repartition(self.v, self.v_h, stream)
+        self.s_attn.execute([self.qa, self.ka, self.va], self.oa, stream)
+        if p == "seq":
+            repartition(self.att_h, self.att, stream)
+        self.s_wo.execute([self.att, self.wo], self.o, stream)
+        self.s_add.execute([self.x_p, self.o], self.h, stream)
+        self.s_norm.execute([self.h, self.g2], self.n2, stream)
+        self.s_up.execute([self.n2, self.w1], self.a, stream)
+        self.s_up.execute([self.n2, self.w3], self.b, stream)
+        self.s_silu.execute([self.a, self.b], self.hh, stream)
+        self.s_down.execute([self.hh, self.w2], self.y, stream)
+        self.s_add.execute([self.h, self.y], self.out_p, stream)
+        if p == "head":
+            repartition(self.out_p, self.out, stream)
+        return self.out

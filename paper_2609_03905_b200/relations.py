@@ -1,0 +1,112 @@
+"""Small conveniences over the binding for callers that hold relation payloads in torch tensors:
+allocation of a payload buffer of the right size, handle lifetime, and the current stream.
+No arithmetic and no data movement happens here (packing a dense tensor into a relation is itself
+a ja_repartition from the one-block tiling)."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+_DT = {torch.float32: B.JA_F32, torch.bfloat16: B.JA_BF16}
+
+
+def equal_splits(extent: int, n: int):
+    """Near-equal intervals: interval s of n is [floor(s*E/n), floor((s+1)*E/n))."""
+    return [(s * extent) // n for s in range(n + 1)]
+
+
+def current_stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Relation:
+    """A tensor relation whose payload lives in a torch CUDA tensor (flat, 128-byte aligned)."""
+
+    def __init__(self, extents, splits, dtype=torch.bfloat16, payload: torch.Tensor | None = None, device="cuda"):
+        self.extents = [int(e) for e in extents]
+        self.splits = [[int(x) for x in s] for s in splits]
+        self.dtype = dtype
+        nbytes = B.ja_relation_bytes(self.extents, self.splits, _DT[dtype])
+        if payload is None:
+            payload = torch.zeros(nbytes // dtype.itemsize, dtype=dtype, device=device)
+        assert payload.is_cuda and payload.is_contiguous() and payload.dtype == dtype
+        assert payload.numel() * dtype.itemsize >= nbytes
+        self.payload = payload
+        self.nbytes = nbytes
+        self.handle = B.ja_relation_create(self.extents, self.splits, _DT[dtype], payload.data_ptr(),
+                                           payload.numel() * dtype.itemsize)
+
+    def view_as(self, extents, splits) -> "Relation":
+        """Another relation handle over the SAME payload (a reshape of the tensor whose block layout coincides)."""
+        return Relation(extents, splits, self.dtype, self.payload)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            B.ja_relation_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Spec:
+    def __init__(self, einsum: str, parts: dict, fn="mul", fn_params=(), agg="sum"):
+        self.einsum, self.parts = einsum, parts
+        self.handle = B.ja_spec_create(einsum, parts, fn, fn_params, agg)
+
+    def execute(self, inputs, output: Relation, stream: int | None = None):
+        B.ja_execute(self.handle, [r.handle for r in inputs], [output.handle],
+                     current_stream() if stream is None else stream)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            B.ja_spec_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def repartition(src: Relation, dst: Relation, stream: int | None = None):
+    B.ja_repartition(src.handle, dst.handle, current_stream() if stream is None else stream)
+
+
+def from_dense(dense: torch.Tensor, splits) -> Relation:
+    """Pack a dense row-major CUDA tensor into a relation: ja_repartition from the one-block tiling."""
+    dense = dense.contiguous()
+    one = Relation(list(dense.shape), [[0, e] for e in dense.shape], dense.dtype, _aligned_flat(dense))
+    dst = Relation(list(dense.shape), splits, dense.dtype)
+    repartition(one, dst)
+    torch.cuda.current_stream().synchronize()
+    one.close()
+    return dst
+
+
+def to_dense(rel: Relation) -> torch.Tensor:
+    """Recompose a relation into a dense row-major tensor: ja_repartition to the one-block tiling."""
+    one = Relation(rel.extents, [[0, e] for e in rel.extents], rel.dtype)
+    repartition(rel, one)
+    torch.cuda.current_stream().synchronize()
+    n = 1
+    for e in rel.extents:
+        n *= e
+    out = one.payload[:n].reshape(rel.extents).clone()
+    one.close()
+    return out
+
+
+def _aligned_flat(t: torch.Tensor) -> torch.Tensor:
+    flat = t.reshape(-1)
+    pad = (-flat.numel() * flat.element_size()) % 128
+    if pad or flat.data_ptr() % 128:
+        buf = torch.zeros(flat.numel() + pad // flat.element_size(), dtype=t.dtype, device=t.device)
+        buf[: flat.numel()] = flat
+        return buf
+    return flat

@@ -1,0 +1,231 @@
+"""GPU parity: every kernel of libja, called through the C ABI, against the CPU oracle on the same seeded
+inputs, element by element. Sizes here are small enough for the oracle to finish in seconds and still span
+several tiles, several blocks and ragged tails. Tolerances: relative Frobenius error 1e-5 for f32 relations,
+2e-2 for bf16 relations (f32 accumulation); bit-exact for MAX aggregation and for every relayout."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_03905_b200 as ja
+import synth_inputs as si
+from oracle import blocked, core, operators
+
+from gpu_util import TOL, check_status, download, download_bits, empty_like_tiling, np_bits, relfro, upload
+
+pytestmark = pytest.mark.gpu
+ES = blocked.equal_splits
+BF, F32 = torch.bfloat16, torch.float32
+ORC_DT = {BF: "bf16", F32: "f32"}
+
+
+def _matmul_case(M, J, N, si_, sj, sk, dtype, cfg=1, std_b=1.0):
+    A = si.normal((M, J), 0.0, 1.0, dtype, cfg, 1)
+    Bm = si.normal((J, N), 0.0, std_b, dtype, cfg, 2)
+    parts = {"i": si_, "j": sj, "k": sk}
+    spec = ja.Spec("ij,jk->ik", parts, "mul", (), "sum")
+    rA, rB = upload(A, [si_, sj]), upload(Bm, [sj, sk])
+    rC = empty_like_tiling([M, N], [si_, sk], dtype, fill=float("nan"))
+    spec.execute([rA, rB], rC)
+    got = download(rC)
+    check_status()
+    ref = operators.matmul(si.to_f64(A), si.to_f64(Bm), ORC_DT[dtype])
+    return got, ref
+
+
+# ---------------------------------------------------------------------------------------------------
+# config 1: matmul as a join-agg, f32, 256^3; decomposition invariance
+# ---------------------------------------------------------------------------------------------------
+def test_config1_matmul_f32_decompositions():
+    outs = {}
+    for grid in ((4, 4, 4), (2, 8, 4), (1, 1, 1), (4, 8, 4)):
+        got, ref = _matmul_case(256, 256, 256, ES(256, grid[0]), ES(256, grid[1]), ES(256, grid[2]), F32)
+        assert relfro(got, ref) <= TOL[F32], grid
+        outs[grid] = got
+    base = outs[(1, 1, 1)]
+    for grid, got in outs.items():  # every block decomposition of the same operator yields the same result
+        assert relfro(got, base) <= TOL[F32], grid
+
+
+def test_matmul_plain_alu_uneven_tilings():
+    got, ref = _matmul_case(100, 77, 90, [0, 33, 100], [0, 10, 50, 77], [0, 64, 65, 90], F32)
+    assert relfro(got, ref) <= TOL[F32]
+    got, ref = _matmul_case(70, 50, 45, [0, 70], [0, 17, 50], [0, 20, 45], BF)     # bf16 on irregular blocks
+    assert relfro(got, ref) <= TOL[BF]
+
+
+# ---------------------------------------------------------------------------------------------------
+# tensor-core matmul join-agg (bf16 relations, uniform blocks)
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,J,N,gi,gj,gk", [
+    (256, 256, 512, 2, 2, 2),      # 128x128 / 128x256 blocks: one full tile per output key
+    (256, 512, 256, 1, 4, 1),      # m = 4 tuples per output key, 256-row block = two row tiles
+    (384, 192, 640, 3, 3, 1),      # 64-deep contraction blocks, 640-wide block = 256+256+128 tiles
+    (256, 704, 352, 2, 2, 2),      # ragged: 352-deep blocks (5.5 k-steps), 176-wide blocks (N = 176)
+    (256, 128, 512, 4, 1, 8),      # 64-row and 64-column blocks: tiles span several output keys
+    (512, 256, 384, 2, 2, 3),      # 128-wide blocks: a 256-column tile covers two output keys (+ tail)
+    (200, 160, 136, 1, 1, 1),      # one ragged block: 200 rows (128+72), 136 columns
+])
+def test_matmul_tensor_core(M, J, N, gi, gj, gk):
+    got, ref = _matmul_case(M, J, N, ES(M, gi), ES(J, gj), ES(N, gk), BF, cfg=2, std_b=0.05)
+    assert relfro(got, ref) <= TOL[BF]
+    # the error must look like bf16 rounding of the output, not like a dropped k-step or a misplaced tile
+    assert np.abs(got - ref).max() <= 2.0 ** -7 * np.abs(ref).max() + 1e-6
+
+
+def test_matmul_tensor_core_identity_is_exact():
+    M = 256
+    A = si.normal((M, M), 0.0, 1.0, BF, 2, 3)
+    eye = torch.eye(M, dtype=BF)
+    sp = ES(M, 2)
+    spec = ja.Spec("ij,jk->ik", {"i": sp, "j": sp, "k": sp})
+    rC = empty_like_tiling([M, M], [sp, sp], BF, fill=float("nan"))
+    spec.execute([upload(A, [sp, sp]), upload(eye, [sp, sp])], rC)
+    assert np.array_equal(download(rC), si.to_f64(A))
+    rC2 = empty_like_tiling([M, M], [sp, sp], BF, fill=float("nan"))
+    spec.execute([upload(eye, [sp, sp]), upload(A, [sp, sp])], rC2)
+    assert np.array_equal(download(rC2), si.to_f64(A))
+    check_status()
+
+
+# ---------------------------------------------------------------------------------------------------
+# repartition: bit-exact block relayout
+# ---------------------------------------------------------------------------------------------------
+def test_repartition_bit_exact():
+    rng = np.random.default_rng(5)
+    cases = [([256, 256], [ES(256, 2), [0, 256]], [ES(256, 4), [0, 256]], BF),       # the paper's overlay example
+             ([512, 1024], [ES(512, 4), ES(1024, 2)], [ES(512, 4), ES(1024, 8)], BF),
+             ([96, 200], [[0, 31, 96], [0, 7, 200]], [[0, 50, 96], [0, 100, 101, 200]], BF),  # odd offsets: 2-byte path
+             ([2, 64, 4, 128], [[0, 1, 2], ES(64, 2), [0, 4], [0, 128]], [[0, 2], ES(64, 4), ES(4, 4), [0, 128]], BF),
+             ([33, 17, 9], [[0, 33], [0, 5, 17], [0, 9]], [[0, 10, 33], [0, 17], [0, 4, 9]], F32),
+             ([1000], [[0, 1000]], [ES(1000, 7)], F32)]
+    for ext, s_sp, d_sp, dt in cases:
+        if dt == BF:
+            dense = torch.from_numpy(rng.integers(0, 1 << 16, ext, dtype=np.uint16).view(np.int16)).view(BF)
+        else:
+            dense = torch.from_numpy(rng.standard_normal(ext).astype(np.float32))
+        src = upload(dense, s_sp)
+        dst = empty_like_tiling(ext, d_sp, dt)
+        ja.repartition(src, dst)
+        want = blocked.repartition(np_bits(src.payload.cpu()), ext, s_sp, d_sp)
+        assert np.array_equal(download_bits(dst), want)
+        back = empty_like_tiling(ext, s_sp, dt)
+        ja.repartition(dst, back)                                                    # round trip
+        assert np.array_equal(download_bits(back), download_bits(src))
+        one = empty_like_tiling(ext, [[0, e] for e in ext], dt)
+        ja.repartition(src, one)                                                     # one block = the dense tensor
+        assert np.array_equal(download_bits(one)[: dense.numel()], np_bits(dense).reshape(-1))
+        via = empty_like_tiling(ext, d_sp, dt)
+        ja.repartition(one, via)                                                     # via an intermediate = direct
+        assert np.array_equal(download_bits(via), want)
+        # the library's own packing helper agrees with the oracle's packing
+        assert np.array_equal(download_bits(ja.from_dense(dense.cuda(), d_sp)), want)
+        assert np.array_equal(np_bits(ja.to_dense(dst)), np_bits(dense))
+    check_status()
+
+
+# ---------------------------------------------------------------------------------------------------
+# memory-bound join-aggs
+# ---------------------------------------------------------------------------------------------------
+TILINGS_2D = [((256, 1024), ES(256, 2), ES(1024, 8)),           # 128-bit path, m = 8 column blocks per row key
+              ((64, 4096), ES(64, 1), ES(4096, 8)),              # LLaMA row length
+              ((40, 8192), ES(40, 2), ES(8192, 8)),              # 65B row length: two warps per row
+              ((37, 300), [0, 5, 37], [0, 7, 150, 300]),         # irregular splits: scalar path
+              ((9, 20000), [0, 9], ES(20000, 2))]                # long row: streaming path
+
+
+@pytest.mark.parametrize("dtype", [BF, F32])
+@pytest.mark.parametrize("shape,si_,sj", TILINGS_2D)
+def test_rmsnorm_join_aggs(shape, si_, sj, dtype):
+    X = si.normal(shape, 0.0, 2.0, dtype, 3, 1)
+    G = si.normal((shape[1],), 1.0, 0.1, dtype, 3, 2)
+    ref = operators.rmsnorm(si.to_f64(X), si.to_f64(G), 1e-5, ORC_DT[dtype])
+    rX, rG = upload(X, [si_, sj]), upload(G, [sj])
+    parts = {"i": si_, "j": sj}
+    # SUM-of-squares aggregation, then the key-aligned scale join
+    rSS = empty_like_tiling([shape[0]], [si_], F32, fill=float("nan"))
+    ja.Spec("ij->i", parts, "square", (), "sum").execute([rX], rSS)
+    assert relfro(download(rSS), ref["ss"]) <= 1e-5
+    rY = empty_like_tiling(list(shape), [si_, sj], dtype, fill=float("nan"))
+    ja.Spec("ij,i,j->ij", parts, "rms_scale", (1e-5,), "none").execute([rX, rSS, rG], rY)
+    assert relfro(download(rY), ref["y"]) <= TOL[dtype]
+    # the fused chain
+    rY2 = empty_like_tiling(list(shape), [si_, sj], dtype, fill=float("nan"))
+    ja.Spec("ij,j->ij", parts, "rmsnorm", (1e-5,), "none").execute([rX, rG], rY2)
+    assert relfro(download(rY2), ref["y"]) <= TOL[dtype]
+    check_status()
+
+
+@pytest.mark.parametrize("dtype", [BF, F32])
+@pytest.mark.parametrize("shape,sh,si_,sj", [((4, 64, 2048), ES(4, 4), ES(64, 2), ES(2048, 8)),
+                                             ((2, 17, 300), [0, 2], [0, 5, 17], [0, 7, 150, 300]),
+                                             ((1, 8, 20000), [0, 1], [0, 8], ES(20000, 2))])
+def test_softmax_join_aggs(shape, sh, si_, sj, dtype):
+    S = si.normal(shape, 0.0, 2.0, dtype, 3, 3)
+    ref = operators.softmax_rows(si.to_f64(S), ORC_DT[dtype])
+    rS = upload(S, [sh, si_, sj])
+    parts = {"h": sh, "i": si_, "j": sj}
+    stat = lambda: empty_like_tiling(list(shape[:2]), [sh, si_], F32, fill=float("nan"))
+    rM, rL = stat(), stat()
+    ja.Spec("hij->hi", parts, "ident", (), "max").execute([rS], rM)
+    assert np.array_equal(download(rM), ref["m"])                                   # MAX aggregation is exact
+    ja.Spec("hij,hi->hi", parts, "exp_sub", (), "sum").execute([rS, rM], rL)
+    assert relfro(download(rL), ref["l"]) <= 1e-5
+    rP = empty_like_tiling(list(shape), [sh, si_, sj], dtype, fill=float("nan"))
+    ja.Spec("hij,hi,hi->hij", parts, "exp_sub_div", (), "none").execute([rS, rM, rL], rP)
+    assert relfro(download(rP), ref["p"]) <= TOL[dtype]
+    rP2 = empty_like_tiling(list(shape), [sh, si_, sj], dtype, fill=float("nan"))
+    ja.Spec("hij->hij", parts, "softmax", (), "none").execute([rS], rP2)
+    assert relfro(download(rP2), ref["p"]) <= TOL[dtype]
+    check_status()
+
+
+@pytest.mark.parametrize("dtype", [BF, F32])
+def test_key_aligned_maps(dtype):
+    for shape, sp in (((256, 1376), [ES(256, 2), ES(1376, 1)]), ((50, 70), [[0, 13, 50], [0, 33, 70]])):
+        a = si.normal(shape, 0.0, 1.5, dtype, 2, 4)
+        b = si.normal(shape, 0.0, 1.0, dtype, 2, 5)
+        parts = {"i": sp[0], "j": sp[1]}
+        rA, rB = upload(a, sp), upload(b, sp)
+        rO = empty_like_tiling(list(shape), sp, dtype, fill=float("nan"))
+        ja.Spec("ij,ij->ij", parts, "silu_mul", (), "none").execute([rA, rB], rO)
+        assert relfro(download(rO), operators.silu_mul(si.to_f64(a), si.to_f64(b), ORC_DT[dtype])) <= TOL[dtype]
+        rO2 = empty_like_tiling(list(shape), sp, dtype, fill=float("nan"))
+        ja.Spec("ij,ij->ij", parts, "add", (), "none").execute([rA, rB], rO2)
+        assert np.array_equal(download(rO2), operators.add(si.to_f64(a), si.to_f64(b), ORC_DT[dtype]))  # one exact rounding
+    check_status()
+
+
+@pytest.mark.parametrize("splits", [[[0, 1, 2], ES(256, 2), ES(4, 4), [0, 128]],
+                                    [[0, 2], ES(256, 4), [0, 4], [0, 128]],
+                                    [[0, 2], [0, 100, 256], [0, 1, 4], [0, 64, 128]]])
+def test_rope(splits):
+    x = si.normal((2, 256, 4, 128), 0.0, 1.0, BF, 5, 11)
+    rX = upload(x, splits)
+    rY = empty_like_tiling(list(x.shape), splits, BF, fill=float("nan"))
+    ja.Spec("bshd->bshd", dict(zip("bshd", splits)), "rope", (1e4,), "none").execute([rX], rY)
+    assert relfro(download(rY), operators.rope(si.to_f64(x), 1e4, "bf16")) <= 4e-3
+    check_status()
+
+
+# ---------------------------------------------------------------------------------------------------
+# attention join-agg
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,S,H,qb,kb,hb,causal", [(1, 256, 2, 128, 128, 1, True), (2, 512, 2, 128, 128, 2, True),
+                                                   (1, 256, 1, 64, 64, 1, True), (1, 384, 2, 128, 64, 1, False),
+                                                   (1, 512, 1, 256, 128, 1, True)])
+def test_attention(B, S, H, qb, kb, hb, causal):
+    D = 128
+    Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (1, 2, 3))
+    spl = lambda blk: [ES(B, B), ES(S, S // blk), ES(H, H // hb), [0, D]]
+    rQ, rK, rV = upload(Q, spl(qb)), upload(K, spl(kb)), upload(V, spl(kb))
+    rO = empty_like_tiling([B, S, H, D], spl(qb), BF, fill=float("nan"))
+    parts = {"b": ES(B, B), "q": ES(S, S // qb), "h": ES(H, H // hb), "d": [0, D], "k": ES(S, S // kb)}
+    spec = ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / np.sqrt(D), 1.0 if causal else 0.0), "online_softmax")
+    spec.execute([rQ, rK, rV], rO)
+    got = download(rO)
+    check_status()
+    ref = operators.attention(si.to_f64(Q), si.to_f64(K), si.to_f64(V), causal, "bf16")
+    assert relfro(got, ref) <= TOL[BF]
+    assert np.abs(got - ref).max() <= 0.05
+    if causal:
+        assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly

@@ -1,0 +1,176 @@
+"""CPU tests of libja's host side: the library loads and exports every declared symbol, and its integer
+bookkeeping (function-spec tuples, tilings, cost counts, key tables, overlay atoms) equals, bit for bit, the
+tables the oracle builds independently from the paper's definitions. No kernel is launched here."""
+import ctypes
+import json
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2609_03905_b200 as ja
+from oracle import blocked
+
+RNG = np.random.default_rng(20260905)
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "ja.h")).read()
+    names = set(re.findall(r"\b(ja_[a-z_]+)\s*\(", hdr))
+    assert {"ja_spec_create", "ja_relation_create", "ja_execute", "ja_repartition"} <= names
+    lib = ctypes.CDLL(ja.binding.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} is declared in include/ja.h but not exported"
+    assert "sm_100a" in ja.ja_version()
+
+
+def _rand_parts(letters, lo=3, hi=40):
+    parts = {}
+    for c in letters:
+        e = int(RNG.integers(lo, hi))
+        cuts = sorted(set(RNG.integers(1, e, int(RNG.integers(0, 4))).tolist()))
+        parts[c] = [0] + cuts + [e]
+    return parts
+
+
+@pytest.mark.parametrize("einsum,fn,agg", [
+    ("ij,jk->ik", "mul", "sum"), ("ij,ij->ij", "silu_mul", "none"), ("ij->i", "square", "sum"),
+    ("hij->hi", "ident", "max"), ("hij,hi->hi", "exp_sub", "sum"), ("hij,hi,hi->hij", "exp_sub_div", "none"),
+    ("ij,i,j->ij", "rms_scale", "none"), ("bshd->bshd", "rope", "none"), ("ij,jk,kl->il", "mul", "sum"),
+])
+def test_spec_tables_match_oracle(einsum, fn, agg):
+    for _ in range(4):
+        letters = blocked.core.parse_einsum(einsum)[2]
+        parts = _rand_parts(letters)
+        ref = blocked.Spec(einsum, parts)
+        s = ja.ja_spec_create(einsum, parts, fn, (1e-5,), agg)
+        try:
+            p, n_in = ja.ja_spec_num_tuples(s)
+            assert (p, n_in) == (ref.p, len(ref.ins))
+            ink, outk = ja.ja_spec_get_tuples(s)
+            rink, routk = ref.tuples()
+            assert ink.dtype == rink.dtype and np.array_equal(ink, rink) and np.array_equal(outk, routk)
+            for operand in list(range(n_in)) + [-1]:
+                nb, splits = ja.ja_spec_operand_tiling(s, operand)
+                rnb, rsplits = ref.operand_tiling(operand)
+                assert nb == rnb and splits == [list(x) for x in rsplits]
+            assert ja.ja_spec_cost_terms(s) == ref.cost_terms()
+        finally:
+            ja.ja_spec_destroy(s)
+
+
+def test_attention_spec_band_predicate():
+    parts = {"b": [0, 1, 2], "q": blocked.equal_splits(512, 4), "h": [0, 1, 2, 3], "d": [0, 128],
+             "k": blocked.equal_splits(512, 4)}
+    es = "bqhd,bkhd,bkhd->bqhd"
+    ref = blocked.Spec(es, parts, band=("k", "q"))
+    s = ja.ja_spec_create(es, parts, "attention", (0.088, 1.0), "online_softmax")
+    ink, outk = ja.ja_spec_get_tuples(s)
+    rink, routk = ref.tuples()
+    assert np.array_equal(ink, rink) and np.array_equal(outk, routk)
+    assert ja.ja_spec_num_tuples(s)[0] == 2 * 3 * (4 * 5 // 2)          # q-blocks x k-blocks with kb <= qb
+    assert np.bincount(outk).reshape(2, 4, 3)[0, :, 0].tolist() == [1, 2, 3, 4]   # multiplicity m = qb + 1
+    ja.ja_spec_destroy(s)
+    full = ja.ja_spec_create(es, parts, "attention", (0.088, 0.0), "online_softmax")  # not causal: whole grid
+    assert ja.ja_spec_num_tuples(full)[0] == 2 * 4 * 3 * 4
+    ja.ja_spec_destroy(full)
+
+
+def test_paper_worked_examples_through_the_library(golden_dir):
+    g = json.load(open(os.path.join(golden_dir, "matmul_decomposed.json")))
+    s = ja.ja_spec_create(g["einsum"], g["four_spec"]["parts"])
+    assert ja.ja_spec_num_tuples(s)[0] == g["four_spec"]["num_function_specs"]
+    ink, outk = ja.ja_spec_get_tuples(s)
+    assert np.bincount(outk).tolist() == g["four_spec"]["multiplicity"]
+    nb, splits = ja.ja_spec_operand_tiling(s, -1)
+    types = [{"lower": [splits[0][i], 0], "upper": [splits[0][i + 1], splits[1][1]]} for i in range(nb[0])]
+    assert types == g["four_spec"]["distinct_output_types"]
+    ja.ja_spec_destroy(s)
+    s = ja.ja_spec_create(g["einsum"], g["two_spec"]["parts"])
+    assert ja.ja_spec_num_tuples(s)[0] == 2 and np.bincount(ja.ja_spec_get_tuples(s)[1]).tolist() == [2]
+    ja.ja_spec_destroy(s)
+    c = json.load(open(os.path.join(golden_dir, "cost_3d_matmul.json")))
+    for case in c["cases"]:
+        parts = {l: blocked.equal_splits(case["N"], n) for l, n in zip("ijk", (case["a"], case["b"], case["c"]))}
+        s = ja.ja_spec_create("ij,jk->ik", parts)
+        assert ja.ja_spec_cost_terms(s) == (case["join"], case["agg"])
+        ja.ja_spec_destroy(s)
+
+
+FAKE_PTR = 1 << 20  # never dereferenced on the CPU: relation creation makes no CUDA call
+
+
+def _rel(extents, splits, dtype=ja.JA_BF16, ptr=FAKE_PTR):
+    return ja.ja_relation_create(extents, splits, dtype, ptr, ja.ja_relation_bytes(extents, splits, dtype))
+
+
+def test_relation_key_table_matches_oracle():
+    for _ in range(10):
+        rank = int(RNG.integers(1, 5))
+        parts = _rand_parts("abcd"[:rank], 2, 20)
+        splits = [parts[c] for c in "abcd"[:rank]]
+        ext = [s[-1] for s in splits]
+        for dt, es in ((ja.JA_BF16, 2), (ja.JA_F32, 4)):
+            r = _rel(ext, splits, dt)
+            coords, lower, upper, offs = ja.ja_relation_get_keys(r)
+            rc, rl, ru, ro, total = blocked.relation_keys(ext, splits, es)
+            assert np.array_equal(coords, rc) and np.array_equal(lower, rl) and np.array_equal(upper, ru)
+            assert np.array_equal(offs, ro) and ja.ja_relation_bytes(ext, splits, dt) == total
+            ja.ja_relation_destroy(r)
+
+
+def test_overlay_atoms_match_oracle_and_paper(golden_dir):
+    g = json.load(open(os.path.join(golden_dir, "overlay_example.json")))
+    src = _rel(g["extents"], g["producer_splits"])
+    dst = _rel(g["extents"], g["consumer_splits"], ptr=FAKE_PTR * 2)
+    lower, upper, sb, db = ja.ja_overlay_atoms(src, dst)
+    assert len(sb) == g["num_atoms"] and sb.tolist() == g["atom_to_producer_block"] and db.tolist() == g["atom_to_consumer_block"]
+    assert sorted(set(lower[:, 0].tolist() + upper[:, 0].tolist())) == g["overlay_row_split_points"]
+    ja.ja_relation_destroy(src); ja.ja_relation_destroy(dst)
+    for _ in range(10):
+        rank = int(RNG.integers(1, 5))
+        ext = [int(RNG.integers(3, 14)) for _ in range(rank)]
+        mk = lambda: [[0] + sorted(set(RNG.integers(1, e, int(RNG.integers(0, 3))).tolist())) + [e] for e in ext]
+        s_sp, d_sp = mk(), mk()
+        src, dst = _rel(ext, s_sp), _rel(ext, d_sp, ptr=FAKE_PTR * 2)
+        lower, upper, sb, db = ja.ja_overlay_atoms(src, dst)
+        _, atoms = blocked.overlay_atoms(s_sp, d_sp)
+        assert lower.tolist() == [a[0] for a in atoms] and upper.tolist() == [a[1] for a in atoms]
+        assert sb.tolist() == [a[2] for a in atoms] and db.tolist() == [a[3] for a in atoms]
+        ja.ja_relation_destroy(src); ja.ja_relation_destroy(dst)
+
+
+def _status(fn, *a, **k):
+    with pytest.raises(ja.JaError) as e:
+        fn(*a, **k)
+    return e.value.status_name
+
+
+def test_error_codes():
+    ok = {"i": [0, 4], "j": [0, 2, 4], "k": [0, 4]}
+    assert _status(ja.ja_spec_create, "ij,jk>ik", ok) == "JA_ERR_PARSE"
+    assert _status(ja.ja_spec_create, "iJ,jk->ik", ok) == "JA_ERR_PARSE"
+    assert _status(ja.ja_spec_create, "ij,jk->iz", ok) == "JA_ERR_PARSE"
+    assert _status(ja.ja_spec_create, "ij,jk->ik", {"i": [0, 4], "j": [0, 4]}) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_spec_create, "ij,jk->ik", dict(ok, j=[0, 3, 3, 4])) == "JA_ERR_TILING"   # empty interval
+    assert _status(ja.ja_spec_create, "ij,jk->ik", dict(ok, j=[1, 2, 4])) == "JA_ERR_TILING"      # gap at 0
+    assert _status(ja.ja_spec_create, "ij,jk->ik", dict(ok, j=[0, 3, 2, 4])) == "JA_ERR_TILING"   # overlap
+    assert _status(ja.ja_spec_create, "ij,jk->ik", ok, "mul", (), "none") == "JA_ERR_TILING"      # shared output type, no (+)
+    assert _status(ja.ja_relation_create, [4, 4], [[0, 4], [0, 5]], ja.JA_BF16, FAKE_PTR, 1 << 20) == "JA_ERR_TILING"
+    assert _status(ja.ja_relation_create, [4, 4], [[0, 4], [0, 4]], ja.JA_BF16, FAKE_PTR + 2, 1 << 20) == "JA_ERR_ALIGNMENT"
+    assert _status(ja.ja_relation_create, [4, 4], [[0, 4], [0, 4]], ja.JA_BF16, FAKE_PTR, 8) == "JA_ERR_INVALID_ARG"
+    assert _status(ja.ja_relation_create, [4, 4], [[0, 4], [0, 4]], 7, FAKE_PTR, 1 << 20) == "JA_ERR_DTYPE"
+    # tiling mismatch between a relation and in_k(J) is refused before anything is enqueued
+    s = ja.ja_spec_create("ij,jk->ik", ok)
+    A = _rel([4, 4], [[0, 4], [0, 4]], ja.JA_F32)                    # j not split: differs from the spec
+    Bm = _rel([4, 4], [[0, 2, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 2)
+    C = _rel([4, 4], [[0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 3)
+    assert _status(ja.ja_execute, s, [A, Bm], [C]) == "JA_ERR_PARTITION_MISMATCH"
+    assert _status(ja.ja_execute, s, [A], [C]) == "JA_ERR_INVALID_ARG"
+    A2 = _rel([4, 5], [[0, 4], [0, 2, 5]], ja.JA_F32)
+    assert _status(ja.ja_execute, s, [A2, Bm], [C]) == "JA_ERR_SHAPE"
+    for h in (A, A2, Bm, C):
+        ja.ja_relation_destroy(h)
+    ja.ja_spec_destroy(s)
