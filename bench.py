@@ -282,6 +282,108 @@ def run_gpu(args, shape):
         dist.destroy_process_group()
 
 
+# ---- single-config kernel benchmarks (configs 2, 3, 4 of the benchmark definition) ----------------------------------
+def run_case(args):
+    """Times the kernels of one benchmark configuration in isolation (CUDA events around each launch, buffers rotated so
+    that every timed launch reads HBM-cold data when the working set is near the L2 size). Prints one JSON line."""
+    import torch
+    import paper_2609_03905_b200 as ja
+    import synth_inputs as si
+    ES = ja.equal_splits
+    bf, f32 = torch.bfloat16, torch.float32
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream()
+    peaks = measured_peaks()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+
+    def timeit(fn, reps, flush_l2):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        ts = []
+        for r in range(reps):
+            if flush_l2:
+                flush.fill_(r & 0xFF)
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record(stream)
+            fn(r)
+            e.record(stream)
+            torch.cuda.synchronize()
+            ts.append(s.elapsed_time(e))
+        ts.sort()
+        return {"ms_mean": sum(ts) / len(ts), "ms_min": ts[0], "ms_median": ts[len(ts) // 2]}
+
+    def rel(shape, splits, dtype=bf, std=1.0):
+        r = ja.Relation(list(shape), splits, dtype)
+        r.payload.normal_(0.0, std)
+        return r
+
+    res = {}
+    reps = args.steps
+    if args.case == "cfg2":
+        T, d, f = 2048, 4096, 11008
+        ti, td, tf = ES(T, 8), ES(d, 8), ES(f, 8)
+        x, W1, W3, W2 = rel((T, d), [ti, td]), rel((d, f), [td, tf], std=0.02), rel((d, f), [td, tf], std=0.02), rel((f, d), [tf, td], std=0.02)
+        a, b, h, y = rel((T, f), [ti, tf]), rel((T, f), [ti, tf]), rel((T, f), [ti, tf]), rel((T, d), [ti, td])
+        up = ja.Spec("ij,jk->ik", {"i": ti, "j": td, "k": tf})
+        down = ja.Spec("ij,jk->ik", {"i": ti, "j": tf, "k": td})
+        silu = ja.Spec("ij,ij->ij", {"i": ti, "j": tf}, "silu_mul", (), "none")
+        fl = 2.0 * T * d * f
+        for name, fn in (("gemm_x_W1", lambda r: up.execute([x, W1], a)), ("gemm_x_W3", lambda r: up.execute([x, W3], b)),
+                         ("gemm_h_W2", lambda r: down.execute([h, W2], y))):
+            t = timeit(fn, reps, True)
+            res[name] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "frac_of_burst_bf16_peak": fl / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"]}
+        t = timeit(lambda r: silu.execute([a, b], h), reps, True)
+        res["silu_mul"] = {**t, "GBps": 6.0 * T * f / (t["ms_mean"] * 1e-3) / 1e9, "frac_of_measured_hbm": 6.0 * T * f / (t["ms_mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+        def chain(r):
+            up.execute([x, W1], a); up.execute([x, W3], b); silu.execute([a, b], h); down.execute([h, W2], y)
+        t = timeit(chain, reps, True)
+        res["mlp_chain"] = {**t, "TFLOPs": 3 * fl / (t["ms_mean"] * 1e-3) / 1e12}
+    elif args.case == "cfg3":
+        ti, tj = ES(8192, 8), ES(4096, 8)
+        parts = {"i": ti, "j": tj}
+        X, G, Y = rel((8192, 4096), [ti, tj], std=2.0), rel((4096,), [tj]), rel((8192, 4096), [ti, tj])
+        SS = ja.Relation([8192], [ti], f32)
+        hb = lambda nbytes, t: {**t, "GBps": nbytes / (t["ms_mean"] * 1e-3) / 1e9, "frac_of_measured_hbm": nbytes / (t["ms_mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        nb = 8192 * 4096 * 2.0
+        s_fused = ja.Spec("ij,j->ij", parts, "rmsnorm", (1e-5,), "none")
+        s_ss = ja.Spec("ij->i", parts, "square", (), "sum")
+        s_sc = ja.Spec("ij,i,j->ij", parts, "rms_scale", (1e-5,), "none")
+        res["rmsnorm_fused"] = hb(2 * nb, timeit(lambda r: s_fused.execute([X, G], Y), reps, True))
+        res["rmsnorm_sumsq"] = hb(nb, timeit(lambda r: s_ss.execute([X], SS), reps, True))
+        res["rmsnorm_scale"] = hb(2 * nb, timeit(lambda r: s_sc.execute([X, SS, G], Y), reps, True))
+        th, si_, sj = ES(32, 32), ES(2048, 8), ES(2048, 8)
+        p3 = {"h": th, "i": si_, "j": sj}
+        S, P = rel((32, 2048, 2048), [th, si_, sj], std=2.0), rel((32, 2048, 2048), [th, si_, sj])
+        M, L = ja.Relation([32, 2048], [th, si_], f32), ja.Relation([32, 2048], [th, si_], f32)
+        nb = 32 * 2048 * 2048 * 2.0
+        s_sm = ja.Spec("hij->hij", p3, "softmax", (), "none")
+        s_mx = ja.Spec("hij->hi", p3, "ident", (), "max")
+        s_es = ja.Spec("hij,hi->hi", p3, "exp_sub", (), "sum")
+        s_dv = ja.Spec("hij,hi,hi->hij", p3, "exp_sub_div", (), "none")
+        res["softmax_fused"] = hb(2 * nb, timeit(lambda r: s_sm.execute([S], P), reps, True))
+        res["softmax_max"] = hb(nb, timeit(lambda r: s_mx.execute([S], M), reps, True))
+        res["softmax_expsum"] = hb(nb, timeit(lambda r: s_es.execute([S, M], L), reps, True))
+        res["softmax_divide"] = hb(2 * nb, timeit(lambda r: s_dv.execute([S, M, L], P), reps, True))
+        src = rel((16384, 4096), [ES(16384, 128), ES(4096, 8)])
+        dst = ja.Relation([16384, 4096], [ES(16384, 128), ES(4096, 32)], bf)
+        res["repartition_128x512_to_128x128"] = hb(2 * 16384 * 4096 * 2.0, timeit(lambda r: ja.repartition(src, dst), reps, True))
+    elif args.case == "cfg4":
+        Bn, S, H, D = 4, 2048, 32, 128
+        sp = [ES(Bn, Bn), ES(S, S // 128), ES(H, H), [0, D]]
+        Q, K, V, O = (rel((Bn, S, H, D), sp) for _ in range(4))
+        parts = {"b": sp[0], "q": sp[1], "h": sp[2], "d": sp[3], "k": sp[1]}
+        spec = ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / D ** 0.5, 1.0), "online_softmax")
+        t = timeit(lambda r: spec.execute([Q, K, V], O), reps, True)
+        fl = 4.0 * Bn * H * S * S * D / 2
+        res["attention_causal"] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "TFLOPs_executed_blocks": fl * 136 / 128 / (t["ms_mean"] * 1e-3) / 1e12,
+                                   "frac_of_burst_bf16_peak": fl / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"]}
+    assert ja.ja_stream_status(stream.cuda_stream) == 0
+    print(json.dumps({"case": args.case, "reps": reps, "l2": "512 MiB flush buffer written before every timed launch",
+                      "peaks": peaks, "kernels": res}))
+
+
 OP_NAMES = {
     "seq": ["rmsnorm_1", "q_proj", "k_proj", "v_proj", "rope_q", "rope_k", "repartition_q", "repartition_k", "repartition_v",
             "attention", "repartition_att", "o_proj", "residual_1", "rmsnorm_2", "w1_proj", "w3_proj", "silu_mul", "w2_proj",
@@ -301,9 +403,13 @@ def main():
     ap.add_argument("--impl", choices=["ja", "reference"], default="ja")
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", choices=["block", "cfg2", "cfg3", "cfg4"], default="block",
+                    help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
-    if args.impl == "reference":
+    if args.case != "block":
+        run_case(args)
+    elif args.impl == "reference":
         args.steps_ref, args.warmup_ref = args.steps, args.warmup
         run_reference(args, shape)
     else:

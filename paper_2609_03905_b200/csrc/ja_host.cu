@@ -217,6 +217,7 @@ RelView ja_view(const ja_relation* r) {
         }
     }
     v.blk_off = p;
+    v.blk_stride = r->equal_blocks ? (r->nblocks > 1 ? r->blk_off[1] - r->blk_off[0] : (int64_t)r->bytes) : 0;
     return v;
 }
 
@@ -578,8 +579,10 @@ struct ExecPlan {
     std::shared_ptr<GemmTcPlan> gemm;
     bool gemm_checked = false;
     float2* rope_table = nullptr;
+    int64_t* rope_splits = nullptr;  // split points of the collapsed (h d) index
     ~ExecPlan() {
         if (rope_table) cudaFree(rope_table);
+        if (rope_splits) cudaFree(rope_splits);
     }
 };
 
@@ -728,7 +731,22 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
             JA_CUDA(cudaMalloc((void**)&plan->rope_table, tab.size() * sizeof(float2)));
             JA_CUDA(cudaMemcpy(plan->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice));
         }
-        ra.x = ja_view(X); ra.y = ja_view(out); ra.rope_table = plan->rope_table;
+        ra.x = ja_view(X); ra.y = ja_view(out); ra.rope_table = plan->rope_table; ra.rope_d = (int)D;
+        if (X->nblk[3] == 1) {
+            // d is unsplit: a block stores, for every (b, s), its heads back to back, so (h, d) collapses into one
+            // index of extent H*d whose column blocks are whole heads -- long contiguous rows for the row kernel
+            if (!plan->rope_splits) {
+                std::vector<int64_t> sp(X->splits[2]);
+                for (int64_t& v : sp) v *= D;
+                JA_CUDA(cudaMalloc((void**)&plan->rope_splits, sp.size() * sizeof(int64_t)));
+                JA_CUDA(cudaMemcpy(plan->rope_splits, sp.data(), sp.size() * sizeof(int64_t), cudaMemcpyHostToDevice));
+            }
+            for (RelView* v : {&ra.x, &ra.y}) {
+                v->rank = 3;
+                v->extent[2] *= D; v->bs[2] *= D; v->splits[2] = plan->rope_splits;
+                v->extent[3] = 1; v->bs[3] = 1; v->nblk[3] = 1; v->splits[3] = nullptr;
+            }
+        }
         return ja_launch_row(ROW_ROPE, ra, X->dtype, stream);
     }
 

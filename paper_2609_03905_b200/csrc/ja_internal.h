@@ -24,6 +24,7 @@ struct RelView {
     const int64_t* blk_off;              // device; byte offset of every block, row-major key order
     int64_t extent[JA_MAX_RANK];
     int64_t bs[JA_MAX_RANK];             // uniform block size of dimension d, or 0 if irregular
+    int64_t blk_stride;                  // bytes between consecutive blocks when all blocks have one shape, else 0
     int32_t nblk[JA_MAX_RANK];
     int32_t rank;
     int32_t esize;
@@ -97,6 +98,7 @@ struct RowArgs {
     float eps;     // RMS_SCALE / RMSNORM
     float theta;   // ROPE
     const float2* rope_table;  // device [extent(s)][d/2] (cos, sin)
+    int rope_d;                // extent of the rotated index d (rows may hold several heads of d cells each)
 };
 ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st);
 ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,

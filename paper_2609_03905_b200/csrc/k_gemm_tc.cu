@@ -15,18 +15,31 @@
 //
 // Two accumulator stages (2 x 256 TMEM columns) let the epilogue of tile t overlap the mainloop of tile t+1.
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT, drains its copies and exits.
+//
+// The kernel exists in two forms (template parameter CG):
+//   CG = 1  one CTA per 128 x 256 tile, tcgen05.mma.cta_group::1.
+//   CG = 2  a cluster of two CTAs (two SMs) per 256 x 256 tile, tcgen05.mma.cta_group::2 issued by the leader
+//           CTA: each CTA stages its own 128 rows of A and its own half of the tile's B columns (plain TMA
+//           loads, no multicast), so every SM pulls a third less operand data per flop through L2 and can
+//           keep six stages in flight; each CTA holds the accumulator rows of its own half in its own TMEM.
 #include <cuda.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "ja_device.cuh"
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
-constexpr int B_STAGE_BYTES = BK * BN * 2;   // 32 KiB
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB: 128 rows x 64 k
 constexpr int B_CHUNK_BYTES = BK * 64 * 2;   // one 64-column box: 8 KiB
-constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
 constexpr int NUM_THREADS = 192;
+constexpr int MAX_STAGES = 6;
+template <int CG> struct Cfg {
+    static constexpr int STAGES = CG == 1 ? 4 : 6;
+    static constexpr int B_STAGE_BYTES = BK * (BN / CG) * 2;  // 32 KiB, or 16 KiB per CTA of a pair
+    static constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+};
 
 struct GemmParams {
     char* c_base;
@@ -36,8 +49,8 @@ struct GemmParams {
     int32_t nbm, nbk, nbn;     // blocks along i, j, k
     int32_t M, N;              // tensor extents along i, k
     int32_t a_box_rows;        // rows per A box (= min(bm, 128))
-    int32_t m_tiles, n_tiles;  // tile grid
-    int32_t tiles_per_mblk;    // >= 1 when bm >= 128 (tiles never leave a block), 0 when tiles span blocks
+    int32_t m_tiles, n_tiles;  // tile grid (tiles are 128*CG rows x up to 256 columns)
+    int32_t tiles_per_mblk;    // >= 1 when row tiles never leave a block, 0 when tiles are cut from global rows
     int32_t tiles_per_nblk;    // >= 1 when tiles stay inside one column block, 0 when tiles span blocks
 };
 
@@ -52,6 +65,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier that lives in another CTA of the cluster (address from mapa)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -86,28 +103,69 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa_cluster(uint32_t cta_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(cta_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// TMA tile load; `bar` is a shared::cta address (CG 1) or a shared::cluster address that may name the peer CTA's
+// barrier (CG 2). No multicast: every CTA fetches its own boxes.
+template <int CG>
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3) {
+    if (CG == 1) {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+            : "memory");
+    }
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
-// arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed
+// arrives on the mbarrier (CG 2: on the same barrier of BOTH CTAs of the pair) once every tcgen05.mma issued so far
+// by this thread has completed
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
@@ -135,27 +193,29 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr, uint32_t lbo_byte
     return d;
 }
 
+// What one CTA does for one tile: its own 128 rows, and (CG 2) its own half of the tile's columns as B operand.
 struct TileCoord {
-    int mb, r0;          // row block, first row inside it (tiles that stay inside a block)
-    int row_g0;          // first global row (tiles that span blocks)
-    int n_g0, nb, c0;    // first global column / column block and first column inside it
-    int width;           // valid columns (multiple of 8)
-    int rows;            // valid rows
+    int mb, r0;          // row block and first row inside it of THIS CTA's 128 rows
+    int row_g0;          // first global row of this CTA's rows
+    int rows;            // valid rows (0..128)
+    int n_g0, nb, c0;    // first global column of the tile / its column block / first column inside it
+    int width;           // valid columns of the tile (multiple of 8)
 };
 
-__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t) {
+template <int CG>
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int cta_rank) {
     TileCoord tc;
     const int mt = t % p.m_tiles, nt = t / p.m_tiles;
-    if (p.tiles_per_mblk > 0) {
+    if (p.tiles_per_mblk > 0) {   // CG == 1 only: row tiles stay inside a block
         tc.mb = mt / p.tiles_per_mblk;
         tc.r0 = (mt % p.tiles_per_mblk) * BM;
         tc.rows = min(BM, p.bm - tc.r0);
         tc.row_g0 = tc.mb * p.bm + tc.r0;
-    } else {
-        tc.row_g0 = mt * BM;
+    } else {                      // tiles cut from global rows (block height divides 128, or is a multiple of 128)
+        tc.row_g0 = mt * (BM * CG) + cta_rank * BM;
         tc.mb = tc.row_g0 / p.bm;
-        tc.r0 = 0;
-        tc.rows = min(BM, p.M - tc.row_g0);
+        tc.r0 = tc.row_g0 % p.bm;
+        tc.rows = max(0, min(BM, p.M - tc.row_g0));
     }
     if (p.tiles_per_nblk > 0) {
         tc.nb = nt / p.tiles_per_nblk;
@@ -171,8 +231,11 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t) {
     return tc;
 }
 
+template <int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+    constexpr int STAGES = Cfg<CG>::STAGES;
+    constexpr int B_STAGE_BYTES = Cfg<CG>::B_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
@@ -189,32 +252,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int cta_rank = CG == 2 ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), 1);
+            mbar_init(full_bar(s), 1);    // CG 2: only the leader's is used; both CTAs' copies complete_tx on it
             mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 4);
+            mbar_init(tempty_bar(a), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {  // allocate all 512 TMEM columns (two 128 x 256 fp32 accumulators)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {  // all 512 TMEM columns: two 128 x 256 fp32 accumulators (in each CTA of a pair)
+        if (CG == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int kchunks = (p.bk + BK - 1) / BK;
+    const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
     if (warp == 0) {
-        // ================= TMA producer =================
+        // ================= TMA producer (one per CTA) =================
         if (lane == 0) {
             uint32_t last_parity[STAGES];
             bool issued[STAGES];
@@ -222,57 +293,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const TileCoord tc = tile_coord(p, t);
-                const int nchunks = (tc.width + 63) / 64;
-                const uint32_t tx = A_STAGE_BYTES + nchunks * B_CHUNK_BYTES;
+            for (int t = first_tile; t < total_tiles && ok; t += tile_step) {
+                const TileCoord tc = tile_coord<CG>(p, t, cta_rank);
+                const int n_mma = (tc.width + 15) / 16 * 16;
+                const int my_cols = n_mma / CG;                    // B columns this CTA stages
+                const int my_c0 = cta_rank * my_cols;              // their offset inside the tile
+                const int nchunks = (my_cols + 63) / 64;
+                const uint32_t tx = (uint32_t)CG * (A_STAGE_BYTES + nchunks * B_CHUNK_BYTES);
                 for (int jb = 0; jb < p.nbk && ok; ++jb) {          // the tuples of this output key, ascending j
                     for (int kc = 0; kc < kchunks; ++kc) {
                         if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, p.status)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(stage), tx);
+                        uint32_t fb = full_bar(stage);
+                        if (CG == 2) fb = mapa_cluster(fb, 0);      // completion is counted on the leader's barrier
+                        if (cta_rank == 0) mbar_expect_tx(full_bar(stage), tx);
                         issued[stage] = true;
                         last_parity[stage] = phase;
                         // A: boxes of a_box_rows rows x 64 k
                         const int nboxes = BM / p.a_box_rows;
-                        for (int bx = 0; bx < nboxes; ++bx) {
-                            int mb = tc.mb + (p.tiles_per_mblk > 0 ? 0 : bx);
-                            int r0 = p.tiles_per_mblk > 0 ? tc.r0 : 0;
-                            tma_load_4d(sA + stage * A_STAGE_BYTES + bx * p.a_box_rows * 128, &tmA, full_bar(stage),
-                                        kc * BK, r0, jb, mb);
-                        }
-                        // B: one box of 64 k-rows x 64 columns per 64-column chunk of the tile
+                        for (int bx = 0; bx < nboxes; ++bx)
+                            tma_load_4d<CG>(sA + stage * A_STAGE_BYTES + bx * p.a_box_rows * 128, &tmA, fb, kc * BK,
+                                            tc.r0, jb, tc.mb + bx);
+                        // B: one box of 64 k-rows x 64 columns per 64-column chunk
                         for (int c = 0; c < nchunks; ++c) {
                             int nb, cin;
-                            if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + 64 * c; }
-                            else { int g = tc.n_g0 + 64 * c; nb = g / p.bn; cin = g % p.bn; }
-                            tma_load_4d(sB + stage * B_STAGE_BYTES + c * B_CHUNK_BYTES, &tmB, full_bar(stage), cin,
-                                        kc * BK, nb, jb);
+                            if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + my_c0 + 64 * c; }
+                            else { int g = tc.n_g0 + my_c0 + 64 * c; nb = g / p.bn; cin = g % p.bn; }
+                            tma_load_4d<CG>(sB + stage * B_STAGE_BYTES + c * B_CHUNK_BYTES, &tmB, fb, cin, kc * BK, nb, jb);
                         }
                         if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
                 }
             }
-            if (!ok) {  // drain: wait (bounded) for copies already in flight before the CTA may exit
+            // drain: wait (bounded) for copies already in flight before the CTA may exit. In a pair both CTAs' copies
+            // complete on the leader's barriers, and the peer cannot leave before the leader reaches the cluster barrier.
+            if (!ok && cta_rank == 0) {
                 for (int s = 0; s < STAGES; ++s) {
                     if (!issued[s]) continue;
                     const uint64_t t0 = global_ns();
                     while (!mbar_try_wait(full_bar(s), last_parity[s]) && global_ns() - t0 < 200000000ull) {}
                 }
             }
+            (void)issued; (void)last_parity;
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
+        // ================= MMA issuer (leader CTA only) =================
+        if (lane == 0 && cta_rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_phase[2] = {0, 0};
             int it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-                const TileCoord tc = tile_coord(p, t);
+            for (int t = first_tile; t < total_tiles && ok; t += tile_step, ++it) {
+                const TileCoord tc = tile_coord<CG>(p, t, 0);
                 const int acc = it & 1;
                 const uint32_t n_mma = (uint32_t)((tc.width + 15) / 16 * 16);
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((n_mma >> 3) << 17) | ((BM >> 4) << 24);
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((n_mma >> 3) << 17) |
+                                       ((uint32_t)((BM * CG) >> 4) << 24);
                 if (!mbar_wait(tempty_bar(acc), acc_phase[acc] ^ 1, abort_flag, p.status)) { ok = false; break; }
                 acc_phase[acc] ^= 1;
                 tc_fence_after();
@@ -290,29 +366,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             // A: K-major, 16 k = 32 bytes inside the swizzle atom; B: MN-major, 16 k-rows = 2048 bytes
                             uint64_t da = desc_sw128(a_addr + kk * 32, 16);
                             uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
-                            umma_bf16(d_tmem, da, db, idesc, accumulate);
+                            umma_bf16<CG>(d_tmem, da, db, idesc, accumulate);
                             accumulate = 1;
                         }
-                        umma_commit(empty_bar(stage));  // frees the smem stage once these MMAs have read it
+                        umma_commit<CG>(empty_bar(stage));  // frees the smem stage (in both CTAs) once these MMAs have read it
                         if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
                 }
-                if (ok) umma_commit(tfull_bar(acc));    // accumulator complete -> epilogue
+                if (ok) umma_commit<CG>(tfull_bar(acc));    // accumulator complete -> epilogue(s)
             }
         }
     } else {
-        // ================= epilogue (warps 2..5) =================
+        // ================= epilogue (warps 2..5 of every CTA) =================
         const int q = warp & 3;  // TMEM lane group this warp may access
         uint32_t acc_phase[2] = {0, 0};
         int it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            const TileCoord tc = tile_coord(p, t);
+        const uint32_t tempty0 = CG == 2 ? mapa_cluster(tempty_bar(0), 0) : tempty_bar(0);
+        const uint32_t tempty1 = CG == 2 ? mapa_cluster(tempty_bar(1), 0) : tempty_bar(1);
+        for (int t = first_tile; t < total_tiles && ok; t += tile_step, ++it) {
+            const TileCoord tc = tile_coord<CG>(p, t, cta_rank);
             const int acc = it & 1;
             if (!mbar_wait(tfull_bar(acc), acc_phase[acc], abort_flag, p.status)) { ok = false; break; }
             acc_phase[acc] ^= 1;
             tc_fence_after();
-            const int r = q * 32 + lane;                     // row of the tile held by this thread
+            const int r = q * 32 + lane;                     // row of this CTA's 128 rows held by this thread
             const int grow = tc.row_g0 + r;                  // global row
             const bool row_ok = r < tc.rows;
             int ib = 0, iin = 0;
@@ -341,15 +419,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (lane == 0) {
+                if (CG == 1) mbar_arrive(acc ? tempty1 : tempty0);
+                else mbar_arrive_cluster(acc ? tempty1 : tempty0);   // the leader's MMA thread owns the accumulators of both CTAs
+            }
         }
     }
     // ---- teardown ---------------------------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();   // nobody leaves while the peer may still signal its barriers or read its smem
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
     }
 }
 
@@ -392,6 +475,7 @@ struct GemmTcPlan {
     CUtensorMap tmA, tmB;
     GemmParams p;
     int grid;
+    int cg;   // CTAs per tile: 1 or 2
 };
 
 ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C,
@@ -413,18 +497,27 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     p.nbm = A->nblk[0]; p.nbk = A->nblk[1]; p.nbn = B->nblk[1];
     p.M = (int)A->extent[0]; p.N = (int)B->extent[1];
     p.a_box_rows = (int)std::min<int64_t>(bm, 128);
-    if (bm >= 128) { p.tiles_per_mblk = (int)((bm + BM - 1) / BM); p.m_tiles = p.tiles_per_mblk * p.nbm; }
-    else { p.tiles_per_mblk = 0; p.m_tiles = (p.M + BM - 1) / BM; }
     if (bn % 64 == 0 && bn < BN && p.nbn > 1) { p.tiles_per_nblk = 0; p.n_tiles = (p.N + BN - 1) / BN; }
     else { p.tiles_per_nblk = (int)((bn + BN - 1) / BN); p.n_tiles = p.tiles_per_nblk * p.nbn; }
+    // Two-CTA form: 256-row tiles cut from global rows; needs 128-row halves that never straddle a block and, when
+    // tiles span column blocks, column tails whose halves still start on a 64-column box boundary.
+    const char* force = getenv("JA_GEMM_CTA_GROUP");
+    bool two = (bm % 128 == 0 || 128 % bm == 0) && p.M >= 256;
+    if (p.tiles_per_nblk == 0 && (p.N % BN) % 128 != 0) two = false;
+    if (force && force[0] == '1') two = false;
+    plan->cg = two ? 2 : 1;
+    if (two || bm < 128) { p.tiles_per_mblk = 0; p.m_tiles = (p.M + BM * plan->cg - 1) / (BM * plan->cg); }
+    else { p.tiles_per_mblk = (int)((bm + BM - 1) / BM); p.m_tiles = p.tiles_per_mblk * p.nbm; }
     ja_status_t st;
     if ((st = encode_blocked_2d(A, 64, p.a_box_rows, &plan->tmA)) != JA_OK) return st;
     if ((st = encode_blocked_2d(B, 64, 64, &plan->tmB)) != JA_OK) return st;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    plan->grid = std::min(sms, p.m_tiles * p.n_tiles);
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    const int tiles = p.m_tiles * p.n_tiles;
+    plan->grid = two ? 2 * std::min(sms / 2, tiles) : std::min(sms, tiles);
+    cudaError_t e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
+                        : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES);
     if (e != cudaSuccess) return ja_cuda_fail(e, "cudaFuncSetAttribute(gemm_tc_kernel)");
     *out = plan;
     *eligible = true;
@@ -432,8 +525,25 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
 }
 
 ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
-    gemm_tc_kernel<<<plan.grid, NUM_THREADS, SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.p);
+    if (plan.cg == 2) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3((unsigned)plan.grid, 1, 1);
+        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = Cfg<2>::SMEM_BYTES;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.p));
+    } else {
+        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.p);
+        JA_CUDA(cudaGetLastError());
+    }
     ja_count_launch();
-    JA_CUDA(cudaGetLastError());
     return JA_OK;
 }

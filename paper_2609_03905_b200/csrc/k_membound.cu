@@ -8,6 +8,8 @@
 //    output key (Definition 3.7); the partial never leaves registers.
 //
 // All loads/stores are 128-bit when the tiling allows (every split of j a multiple of the vector width).
+#include <string.h>
+
 #include "ja_device.cuh"
 
 namespace {
@@ -61,39 +63,65 @@ struct alignas(sizeof(T) * VEC) Vec {
 struct RowCtx {
     int64_t lead_flat;  // flat block key over the leading dimensions
     int64_t lead_in;    // row offset inside that block (row-major over the block's leading extents)
-    int64_t pos;        // coordinate of the second index (RoPE position)
+    int pos;            // coordinate of the second index (RoPE position)
     int64_t stat_off;   // byte offset of this row's cell in a statistics relation keyed by R
 };
 
+// 32-bit coordinate arithmetic (extents are < 2^31): 64-bit division is a long software routine and would
+// dominate these memory-bound kernels. On uniform tilings every lookup is arithmetic -- no table is read.
+__device__ __forceinline__ void dim_lookup(const RelView& v, int d, int x, int* b, int* lo, int* w) {
+    if (v.bs[d]) {
+        const int bs = (int)v.bs[d];
+        const int bb = (int)((uint32_t)x / (uint32_t)bs);
+        *b = bb;
+        *lo = bb * bs;
+        *w = min(bs, (int)v.extent[d] - bb * bs);
+        return;
+    }
+    int l = 0, h = v.nblk[d] - 1;
+    while (l < h) {
+        int mid = (l + h + 1) >> 1;
+        if (v.splits[d][mid] <= (int64_t)x) l = mid;
+        else h = mid - 1;
+    }
+    *b = l;
+    *lo = (int)v.splits[d][l];
+    *w = (int)v.splits[d][l + 1] - *lo;
+}
+__device__ __forceinline__ int64_t blk_offset(const RelView& v, int64_t flat) {
+    return v.blk_stride ? flat * v.blk_stride : v.blk_off[flat];
+}
+
 __device__ __forceinline__ RowCtx row_ctx(const RelView& x, const RelView& stat, bool has_stat, int64_t row) {
     RowCtx c;
-    int64_t lead[JA_MAX_RANK] = {0, 0, 0, 0};
-    int64_t rem = row;
+    int lead[JA_MAX_RANK] = {0, 0, 0, 0};
+    uint32_t rem = (uint32_t)row;
     for (int d = x.rank - 2; d >= 0; --d) {
-        lead[d] = rem % x.extent[d];
-        rem /= x.extent[d];
+        const uint32_t e = (uint32_t)x.extent[d];
+        const uint32_t qd = rem / e;
+        lead[d] = (int)(rem - qd * e);
+        rem = qd;
     }
     c.lead_flat = 0;
     c.lead_in = 0;
     for (int d = 0; d < x.rank - 1; ++d) {
-        int b = ja_find_blk(x, d, lead[d]);
-        int64_t lo = x.splits[d][b], w = x.splits[d][b + 1] - lo;
+        int b, lo, w;
+        dim_lookup(x, d, lead[d], &b, &lo, &w);
         c.lead_flat = c.lead_flat * x.nblk[d] + b;
         c.lead_in = c.lead_in * w + (lead[d] - lo);
     }
     c.pos = lead[1];
-    c.stat_off = has_stat ? ja_elem_off(stat, lead) : 0;
+    // the statistics relation is keyed by the same leading indices with the same splits
+    c.stat_off = has_stat ? blk_offset(stat, c.lead_flat) + c.lead_in * stat.esize : 0;
     return c;
 }
 
-// byte offset of the vector starting at column `col` of the row; also the column-block index and its lower bound
-__device__ __forceinline__ int64_t vec_off(const RelView& x, const RowCtx& c, int64_t col, int* cb, int64_t* lo) {
+// byte offset of the vector starting at column `col` of the row
+__device__ __forceinline__ int64_t vec_off(const RelView& x, const RowCtx& c, int col) {
     const int last = x.rank - 1;
-    int b = ja_find_blk(x, last, col);
-    int64_t l = x.splits[last][b], w = x.splits[last][b + 1] - l;
-    *cb = b;
-    *lo = l;
-    return x.blk_off[c.lead_flat * x.nblk[last] + b] + (c.lead_in * w + (col - l)) * x.esize;
+    int b, l, w;
+    dim_lookup(x, last, col, &b, &l, &w);
+    return blk_offset(x, c.lead_flat * x.nblk[last] + b) + (c.lead_in * w + (col - l)) * x.esize;
 }
 
 template <bool IS_MAX>
@@ -132,7 +160,7 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     const int rpc = 256 / team;
     const int row_in_cta = threadIdx.x / team, lane_t = threadIdx.x % team;
     const int last = a.x.rank - 1;
-    const int64_t n = a.x.extent[last];
+    const int n = (int)a.x.extent[last];
     const int64_t row = (int64_t)blockIdx.x * rpc + row_in_cta;
     const bool live = row < n_rows;
     constexpr bool HAS_STAT = (OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM || OP == ROW_RMS_SCALE ||
@@ -140,34 +168,26 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     RowCtx ctx = row_ctx(a.x, a.s0, HAS_STAT, live ? row : 0);
 
     V raw[NV];
-    int64_t offs[NV];
     // ---- pass 0: load (resident mode) -------------------------------------------------------------------
     if (RES) {
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
-            int64_t col = ((int64_t)k * team + lane_t) * VEC;
-            offs[k] = -1;
-            if (live && col < n) {
-                int cb; int64_t lo;
-                offs[k] = vec_off(a.x, ctx, col, &cb, &lo);
-                raw[k] = *reinterpret_cast<const V*>(a.x.base + offs[k]);
-            }
+            const int col = (k * team + lane_t) * VEC;
+            if (live && col < n) raw[k] = *reinterpret_cast<const V*>(a.x.base + vec_off(a.x, ctx, col));
         }
     }
-    // iterate over this thread's vectors: f(k, col, byte offset, value)
+    // iterate over this thread's vectors: f(col, value)
     auto for_each = [&](auto f) {
         if (RES) {
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
-                int64_t col = ((int64_t)k * team + lane_t) * VEC;
-                if (offs[k] >= 0) f(col, offs[k], raw[k]);
+                const int col = (k * team + lane_t) * VEC;
+                if (live && col < n) f(col, raw[k]);
             }
         } else if (live) {
-            for (int64_t col = (int64_t)lane_t * VEC; col < n; col += (int64_t)team * VEC) {
-                int cb; int64_t lo;
-                int64_t off = vec_off(a.x, ctx, col, &cb, &lo);
-                V v = *reinterpret_cast<const V*>(a.x.base + off);
-                f(col, off, v);
+            for (int col = lane_t * VEC; col < n; col += team * VEC) {
+                V v = *reinterpret_cast<const V*>(a.x.base + vec_off(a.x, ctx, col));
+                f(col, v);
             }
         }
     };
@@ -176,7 +196,7 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     // ---- reductions ----------------------------------------------------------------------------------------
     if (OP == ROW_SUMSQ || OP == ROW_RMSNORM) {
         float s = 0.f;
-        for_each([&](int64_t, int64_t, const V& v) {
+        for_each([&](int, const V& v) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) { float f = ja_to_float(v.e[e]); s = fmaf(f, f, s); }
         });
@@ -189,7 +209,7 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     }
     if (OP == ROW_MAX || OP == ROW_SOFTMAX) {
         float mx = -INFINITY;
-        for_each([&](int64_t, int64_t, const V& v) {
+        for_each([&](int, const V& v) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) mx = fmaxf(mx, ja_to_float(v.e[e]));
         });
@@ -202,7 +222,7 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = live ? *reinterpret_cast<const float*>(a.s0.base + ctx.stat_off) : 0.f;
     if (OP == ROW_EXPSUM || OP == ROW_SOFTMAX) {
         float s = 0.f;
-        for_each([&](int64_t, int64_t, const V& v) {
+        for_each([&](int, const V& v) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) s += __expf(ja_to_float(v.e[e]) - m);
         });
@@ -219,11 +239,12 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
     }
     // ---- map + store ---------------------------------------------------------------------------------------
     const float inv_l = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : 0.f;
-    for_each([&](int64_t col, int64_t off, const V& v) {
+    for_each([&](int col, const V& v) {
         V o;
         if (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM) {
-            int cb = ja_find_blk(a.g, 0, col);
-            int64_t goff = a.g.blk_off[cb] + (col - a.g.splits[0][cb]) * a.g.esize;
+            int cb, glo, gw;
+            dim_lookup(a.g, 0, col, &cb, &glo, &gw);
+            const int64_t goff = blk_offset(a.g, cb) + (col - glo) * a.g.esize;
             V g = *reinterpret_cast<const V*>(a.g.base + goff);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(ja_to_float(v.e[e]) * rstd * ja_to_float(g.e[e]));
@@ -231,7 +252,7 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
 #pragma unroll
             for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(__expf(ja_to_float(v.e[e]) - m) * inv_l);
         } else if (OP == ROW_ROPE) {
-            const float2* tab = a.rope_table + ctx.pos * (n / 2) + col / 2;
+            const float2* tab = a.rope_table + (ctx.pos * a.rope_d + (col % a.rope_d)) / 2;
 #pragma unroll
             for (int e = 0; e + 1 < VEC; e += 2) {
                 float2 cs = tab[e / 2];
@@ -240,15 +261,224 @@ __global__ void __launch_bounds__(256) row_kernel(RowArgs a, int64_t n_rows, int
                 o.e[e + 1] = ja_from_float<T>(x0 * cs.y + x1 * cs.x);
             }
         }
-        *reinterpret_cast<V*>(a.y.base + off) = o;  // y is tiled exactly like x: same offset
+        *reinterpret_cast<V*>(a.y.base + vec_off(a.y, ctx, col)) = o;  // y is tiled exactly like x
     });
+}
+
+// ---------------------------------------------------------------------------------------------------
+// fast path: equal-sized blocks in every dimension. The payload offset of cell (row, col) separates into
+//     rowpart(row) + colpart(col),   rowpart = row-block strip + row inside the block, colpart = column block + column
+// so a thread computes colpart once for its fixed set of columns, a team computes rowpart once per row, and the
+// inner loops contain no division and no table lookup. CTAs are persistent over rows.
+// ---------------------------------------------------------------------------------------------------
+struct FastGeom {
+    int n, bsc, nbc;            // row length, column-block width, column blocks
+    int blk_elems;              // elements between consecutive blocks of x / y (equal shapes, padding included)
+    int lead_rank;              // leading dimensions (1..3)
+    int lead_ext[3], lead_bs[3], lead_nb[3];
+    int stat_blk_bytes;         // bytes between consecutive blocks of a statistics relation
+    int g_blk_bytes;            // bytes between consecutive blocks of the gain vector
+    int rope_d;
+};
+
+template <typename T, int VEC, int VPT, int OP>
+__global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowArgs a, FastGeom g, int64_t n_rows, int team) {
+    __shared__ float red[64];
+    using V = Vec<T, VEC>;
+    const int rpc = blockDim.x / team;
+    const int row_in_cta = threadIdx.x / team, lane_t = threadIdx.x % team;
+    constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
+    constexpr bool KEEP_EXP = (OP == ROW_SOFTMAX);
+
+    int colpart[VPT];
+    int gpart[HAS_G ? VPT : 1];   // byte offset of the matching cells of the gain vector
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int col = (k * team + lane_t) * VEC;
+        colpart[k] = -1;
+        if (col < g.n) {
+            const int cb = (int)((uint32_t)col / (uint32_t)g.bsc);
+            const int ci = col - cb * g.bsc;
+            colpart[k] = cb * g.blk_elems + ci;
+            if (HAS_G) gpart[k] = cb * g.g_blk_bytes + ci * (int)sizeof(T);
+        }
+    }
+    const int64_t strip = (int64_t)g.nbc * g.blk_elems;  // elements in one strip of column blocks
+
+    for (int64_t row0 = (int64_t)blockIdx.x * rpc; row0 < n_rows; row0 += (int64_t)gridDim.x * rpc) {
+        const int64_t row = row0 + row_in_cta;
+        const bool live = row < n_rows;
+        // ---- rowpart ----------------------------------------------------------------------------------------
+        uint32_t rem = (uint32_t)(live ? row : 0);
+        int lead_flat = 0, lead_in = 0, pos = 0;
+        {
+            int c[3] = {0, 0, 0};
+#pragma unroll
+            for (int d = 2; d >= 0; --d) {
+                if (d < g.lead_rank) {
+                    const uint32_t q = rem / (uint32_t)g.lead_ext[d];
+                    c[d] = (int)(rem - q * (uint32_t)g.lead_ext[d]);
+                    rem = q;
+                }
+            }
+#pragma unroll
+            for (int d = 0; d < 3; ++d) {
+                if (d < g.lead_rank) {
+                    const int b = (int)((uint32_t)c[d] / (uint32_t)g.lead_bs[d]);
+                    lead_flat = lead_flat * g.lead_nb[d] + b;
+                    lead_in = lead_in * g.lead_bs[d] + (c[d] - b * g.lead_bs[d]);
+                }
+            }
+            pos = c[1];
+        }
+        const int64_t rowpart = (int64_t)lead_flat * strip + (int64_t)lead_in * g.bsc;
+        const T* xrow = reinterpret_cast<const T*>(a.x.base) + rowpart;
+        T* yrow = reinterpret_cast<T*>(a.y.base) + rowpart;
+        const int64_t stat_off = (int64_t)lead_flat * g.stat_blk_bytes + (int64_t)lead_in * 4;
+
+        V raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k)
+            if (live && colpart[k] >= 0) raw[k] = *reinterpret_cast<const V*>(xrow + colpart[k]);
+
+        float m = 0.f, l = 0.f, rstd = 0.f;
+        float ex[KEEP_EXP ? VPT * VEC : 1];
+        if (OP == ROW_SUMSQ || OP == ROW_RMSNORM) {
+            float s = 0.f;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (live && colpart[k] >= 0) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) { float f = ja_to_float(raw[k].e[e]); s = fmaf(f, f, s); }
+                }
+            s = team_reduce<false>(s, team, red, row_in_cta, lane_t);
+            if (OP == ROW_SUMSQ) {
+                if (live && lane_t == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = s;
+                continue;
+            }
+            rstd = 1.0f / sqrtf(s / (float)g.n + a.eps);
+        }
+        if (OP == ROW_MAX || OP == ROW_SOFTMAX) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (live && colpart[k] >= 0) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) mx = fmaxf(mx, ja_to_float(raw[k].e[e]));
+                }
+            m = team_reduce<true>(mx, team, red, row_in_cta, lane_t);
+            if (OP == ROW_MAX) {
+                if (live && lane_t == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+                continue;
+            }
+        }
+        if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = live ? *reinterpret_cast<const float*>(a.s0.base + stat_off) : 0.f;
+        if (OP == ROW_EXPSUM || OP == ROW_SOFTMAX) {
+            float s = 0.f;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (live && colpart[k] >= 0) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        const float p = __expf(ja_to_float(raw[k].e[e]) - m);
+                        if (KEEP_EXP) ex[k * VEC + e] = p;
+                        s += p;
+                    }
+                }
+            l = team_reduce<false>(s, team, red, row_in_cta, lane_t);
+            if (OP == ROW_EXPSUM) {
+                if (live && lane_t == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+                continue;
+            }
+        }
+        if (OP == ROW_EXP_SUB_DIV) l = live ? *reinterpret_cast<const float*>(a.s1.base + stat_off) : 1.f;
+        if (OP == ROW_RMS_SCALE) {
+            const float ss = live ? *reinterpret_cast<const float*>(a.s0.base + stat_off) : 1.f;
+            rstd = 1.0f / sqrtf(ss / (float)g.n + a.eps);
+        }
+        const float inv_l = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : 0.f;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (!(live && colpart[k] >= 0)) continue;
+            V o;
+            if (HAS_G) {
+                const V gv = *reinterpret_cast<const V*>(a.g.base + gpart[HAS_G ? k : 0]);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e)
+                    o.e[e] = ja_from_float<T>(ja_to_float(raw[k].e[e]) * rstd * ja_to_float(gv.e[e]));
+            } else if (OP == ROW_SOFTMAX) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(ex[KEEP_EXP ? k * VEC + e : 0] * inv_l);
+            } else if (OP == ROW_EXP_SUB_DIV) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(__expf(ja_to_float(raw[k].e[e]) - m) * inv_l);
+            } else if (OP == ROW_ROPE) {
+                const int col = (k * team + lane_t) * VEC;
+                const float2* tab = a.rope_table + (pos * g.rope_d + (col % g.rope_d)) / 2;
+#pragma unroll
+                for (int e = 0; e + 1 < VEC; e += 2) {
+                    const float2 cs = tab[e / 2];
+                    const float x0 = ja_to_float(raw[k].e[e]), x1 = ja_to_float(raw[k].e[e + 1]);
+                    o.e[e] = ja_from_float<T>(x0 * cs.x - x1 * cs.y);
+                    o.e[e + 1] = ja_from_float<T>(x0 * cs.y + x1 * cs.x);
+                }
+            }
+            *reinterpret_cast<V*>(yrow + colpart[k]) = o;
+        }
+    }
+}
+
+template <typename T, int VEC, int VPT, int OP>
+void launch_fast_v(const RowArgs& a, const FastGeom& g, int64_t n_rows, int team, cudaStream_t st) {
+    // a CTA is one team when rows need several warps (its barrier then couples only the warps of one row), and four
+    // independent single-warp teams otherwise
+    const int block = team >= 64 ? team : 128;
+    const int rpc = block / team;
+    int64_t want = (n_rows + rpc - 1) / rpc;
+    const int64_t cap = (int64_t)148 * (2048 / block);
+    unsigned grid = (unsigned)(want < cap ? want : cap);
+    row_fast_kernel<T, VEC, VPT, OP><<<grid, block, 0, st>>>(a, g, n_rows, team);
+}
+
+// returns false if the shape does not fit the fast path (caller falls back to the generic kernel)
+template <typename T, int OP>
+bool launch_fast(const RowArgs& a, const FastGeom& g, int64_t n_rows, cudaStream_t st) {
+    constexpr int VEC = 16 / (int)sizeof(T);
+    // one warp per row while a lane holds at most 8 vectors (a whole row in flight per warp, no barrier);
+    // longer rows take 2, 4 or 8 warps
+    int team = 32;
+    while (team < 256 && g.n > team * VEC * 8) team *= 2;
+    const int vpt = (g.n + team * VEC - 1) / (team * VEC);
+    if (vpt <= 1) launch_fast_v<T, VEC, 1, OP>(a, g, n_rows, team, st);
+    else if (vpt <= 2) launch_fast_v<T, VEC, 2, OP>(a, g, n_rows, team, st);
+    else if (vpt <= 4) launch_fast_v<T, VEC, 4, OP>(a, g, n_rows, team, st);
+    else if (vpt <= 8) launch_fast_v<T, VEC, 8, OP>(a, g, n_rows, team, st);
+    else if (vpt <= 16) launch_fast_v<T, VEC, 16, OP>(a, g, n_rows, team, st);
+    else return false;
+    return true;
+}
+
+template <typename T>
+bool launch_fast_op(RowOp op, const RowArgs& a, const FastGeom& g, int64_t n_rows, cudaStream_t st) {
+    switch (op) {
+        case ROW_SUMSQ: return launch_fast<T, ROW_SUMSQ>(a, g, n_rows, st);
+        case ROW_MAX: return launch_fast<T, ROW_MAX>(a, g, n_rows, st);
+        case ROW_EXPSUM: return launch_fast<T, ROW_EXPSUM>(a, g, n_rows, st);
+        case ROW_RMS_SCALE: return launch_fast<T, ROW_RMS_SCALE>(a, g, n_rows, st);
+        case ROW_EXP_SUB_DIV: return launch_fast<T, ROW_EXP_SUB_DIV>(a, g, n_rows, st);
+        case ROW_RMSNORM: return launch_fast<T, ROW_RMSNORM>(a, g, n_rows, st);
+        case ROW_SOFTMAX: return launch_fast<T, ROW_SOFTMAX>(a, g, n_rows, st);
+        case ROW_ROPE: return launch_fast<T, ROW_ROPE>(a, g, n_rows, st);
+    }
+    return false;
 }
 
 template <typename T, int VEC, int OP>
 ja_status_t launch_row_t(const RowArgs& a, int64_t n_rows, int64_t n, cudaStream_t st) {
-    // team: the smallest power of two (32..256) that keeps at most 8 vectors per thread, else 16, else stream
+    // team: the smallest power of two (32..256) that keeps at most 4 vectors per thread (few registers, many
+    // resident warps), else up to 16 vectors at 256 threads, else stream
     int team = 32;
-    while (team < 256 && n > (int64_t)team * VEC * 8) team *= 2;
+    while (team < 256 && n > (int64_t)team * VEC * 4) team *= 2;
     int64_t vpt = (n + (int64_t)team * VEC - 1) / ((int64_t)team * VEC);
     const int rpc = 256 / team;
     unsigned grid = (unsigned)((n_rows + rpc - 1) / rpc);
@@ -311,9 +541,33 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
     const int64_t n = a.x.extent[last];
     int64_t n_rows = 1;
     for (int d = 0; d < last; ++d) n_rows *= a.x.extent[d];
-    // widest vector every column split allows (the host mirrors of the split tables are not kept in the view,
-    // so the caller's tiling is probed through the uniform block size when there is one)
+    if (n_rows >= (1ll << 31) || n >= (1ll << 31)) return ja_fail(JA_ERR_UNSUPPORTED, "row-structured join-agg: extents must be < 2^31");
     const int full = dt == JA_F32 ? 4 : 8;
+    const int es = dt == JA_F32 ? 4 : 2;
+    // ---- fast path: every block of x (and of g, and of the statistics relations) has the same shape --------
+    const bool has_g = (op == ROW_RMS_SCALE || op == ROW_RMSNORM);
+    const bool has_stat = (op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM || op == ROW_RMS_SCALE || op == ROW_EXP_SUB_DIV);
+    const bool has_y = !(op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM);
+    if (a.x.blk_stride != 0 && a.x.bs[last] % full == 0 && (!has_y || a.y.blk_stride == a.x.blk_stride) &&
+        (!has_g || a.g.blk_stride != 0) && (!has_stat || a.s0.blk_stride != 0) &&
+        (int64_t)a.x.nblk[last] * (a.x.blk_stride / es) < (1ll << 31)) {
+        FastGeom g;
+        memset(&g, 0, sizeof g);
+        g.n = (int)n; g.bsc = (int)a.x.bs[last]; g.nbc = a.x.nblk[last];
+        g.blk_elems = (int)(a.x.blk_stride / es);
+        g.lead_rank = last;
+        for (int d = 0; d < last; ++d) { g.lead_ext[d] = (int)a.x.extent[d]; g.lead_bs[d] = (int)a.x.bs[d]; g.lead_nb[d] = a.x.nblk[d]; }
+        g.stat_blk_bytes = has_stat ? (int)a.s0.blk_stride : 0;
+        g.g_blk_bytes = has_g ? (int)a.g.blk_stride : 0;
+        g.rope_d = a.rope_d > 0 ? a.rope_d : 2;
+        bool ok = dt == JA_F32 ? launch_fast_op<float>(op, a, g, n_rows, st) : launch_fast_op<__nv_bfloat16>(op, a, g, n_rows, st);
+        if (ok) {
+            ja_count_launch();
+            JA_CUDA(cudaGetLastError());
+            return JA_OK;
+        }
+    }
+    // ---- generic path: any tiling, key tables read on the device ----------------------------------------------
     int vec = 1;
     if (a.x.bs[last] != 0 && a.x.bs[last] % full == 0 && n % full == 0) vec = full;
     else if (op == ROW_ROPE) vec = 2;

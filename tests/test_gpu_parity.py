@@ -65,7 +65,9 @@ def test_matmul_plain_alu_uneven_tilings():
     (512, 256, 384, 2, 2, 3),      # 128-wide blocks: a 256-column tile covers two output keys (+ tail)
     (200, 160, 136, 1, 1, 1),      # one ragged block: 200 rows (128+72), 136 columns
 ])
-def test_matmul_tensor_core(M, J, N, gi, gj, gk):
+@pytest.mark.parametrize("cta_group", ["2", "1"])   # two-SM tiles where the shape allows them / one-SM tiles everywhere
+def test_matmul_tensor_core(M, J, N, gi, gj, gk, cta_group, monkeypatch):
+    monkeypatch.setenv("JA_GEMM_CTA_GROUP", cta_group)
     got, ref = _matmul_case(M, J, N, ES(M, gi), ES(J, gj), ES(N, gk), BF, cfg=2, std_b=0.05)
     assert relfro(got, ref) <= TOL[BF]
     # the error must look like bf16 rounding of the output, not like a dropped k-step or a misplaced tile
