@@ -129,3 +129,5 @@ struct AttnArgs {
     int32_t hblk;          // heads per block
 };
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);
+// tcgen05 / TMEM form; *launched stays false when the tiling does not fit it
+ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched);

@@ -8,8 +8,11 @@
 // which is the aggregation operator of the spec. O = O~/l is written once, to the key's offset in the
 // output relation. Scores and probabilities never reach HBM.
 //
-// This version feeds the tensor cores through mma.sync (m16n8k16, bf16 in, fp32 accumulate); operands are
-// staged in shared memory with cp.async under an XOR swizzle and read with ldmatrix.
+// This file holds the mma.sync form (m16n8k16, bf16 in, fp32 accumulate; operands staged in shared memory with
+// cp.async under an XOR swizzle and read with ldmatrix). It serves tilings the tensor-memory kernel cannot
+// take (64-row blocks); everything else is dispatched to the tcgen05 kernel.
+#include <stdlib.h>
+
 #include "ja_device.cuh"
 
 namespace {
@@ -238,6 +241,12 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
 }  // namespace
 
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
+    const char* legacy = getenv("JA_ATTN_MMA_SYNC");
+    if (!(legacy && legacy[0] == '1')) {
+        bool launched = false;
+        ja_status_t s = ja_launch_attention_tc(a, st, &launched);
+        if (s != JA_OK || launched) return s;
+    }
     const int QT = (a.qblk % 128 == 0) ? 128 : 64;
     dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;

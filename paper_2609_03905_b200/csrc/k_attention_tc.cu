@@ -1,0 +1,363 @@
+// Attention join-agg "bqhd,bkhd,bkhd->bqhd" (f = ATTENTION, (+) = online softmax) on the 5th-generation
+// tensor cores: both contractions of every joined tuple run as tcgen05.mma with accumulators in tensor memory.
+//
+// One CTA owns one output key tile (128 query rows of one (batch, head)) and walks the function specs that
+// share that output key -- the 128-row key/value tiles that survive the causal band predicate -- ascending.
+//
+//   warp 0      TMA producer: Q once, then K_j and V_j (two stages each), straight from the "bshd" block-key
+//               layout through rank-5 tensor maps (d, head in block, row in block, batch in block, block).
+//   warp 1      tcgen05.mma issuer (one lane):  S_j = Q K_j^T  (A, B from shared memory, both K-major)
+//                                               O'_j = P_j V_j  (A = P_j from TENSOR MEMORY, B = V_j MN-major)
+//   warps 2..5  one thread per query row: read S_j from TMEM, running max / sum in the base-2 domain, write
+//               P_j (bf16) back into the SAME TMEM columns, then fold the finished partial O'_{j-1} into the
+//               running triple held in registers:  O~ <- O~ * 2^(m_old - m_new) + O'_{j-1}.
+//
+// TMEM map (512 columns): S/P buffers at 0 and 128, partial-O buffers at 256 and 384. QK^T of step j+1 is issued
+// before the softmax of step j finishes, so the tensor pipe works while the row threads exponentiate.
+// Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT and leaves through the normal exit.
+#include "ja_device.cuh"
+#include "ja_ptx.cuh"
+
+namespace {
+
+using namespace ja_ptx;
+
+constexpr int D = 128, QT = 128, KT = 128;
+constexpr int TILE_BYTES = 128 * D * 2;      // 32 KiB: one 128 x 128 bf16 tile, stored as two 64-column halves
+constexpr int HALF_BYTES = TILE_BYTES / 2;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BYTES = 5 * TILE_BYTES + 1024 + 256;   // Q, K x2, V x2
+
+struct AttnTcParams {
+    char* o_base;
+    int32_t* status;
+    int64_t o_blk_stride;
+    int32_t B, S, H;
+    int32_t bblk, sblk, hblk;       // block extents of q / o along b, s, h
+    int32_t nsb, nhb;               // blocks along s, h (q / o)
+    int32_t k_bblk, k_sblk, k_hblk, k_nsb, k_nhb;   // same for k / v
+    int32_t causal;
+    float scale_log2e;
+};
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3,
+                                            int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void commit1(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t sQ = base, sK = base + TILE_BYTES, sV = base + 3 * TILE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 5 * TILE_BYTES);
+    const uint32_t bar0 = smem_u32(bars);
+    // barrier indices
+    enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, P_FULL = 11, O_FULL = 13, O_EMPTY = 15, NBAR = 17 };
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int n_qt = p.S / QT;
+    const int qt = n_qt - 1 - (int)blockIdx.x;   // output keys with the most surviving tuples first
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int q0 = qt * QT;
+    const int n_steps = p.causal ? (q0 + QT) / KT : p.S / KT;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NBAR; ++i) {
+            const bool row_threads_arrive = (i >= P_FULL && i < P_FULL + 2) || (i >= O_EMPTY && i < O_EMPTY + 2);
+            mbar_init(bar(i), row_threads_arrive ? 4 : 1);   // one arrival per row warp, else one commit / expect_tx
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tS[2] = {tmem_base, tmem_base + 128};
+    const uint32_t tO[2] = {tmem_base + 256, tmem_base + 384};
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            // block key and in-block coordinates of this (b, h) for q and for k / v
+            const int qb_flat_bh = (b / p.bblk) * p.nsb * p.nhb + (h / p.hblk);     // + s-block * nhb
+            const int kb_flat_bh = (b / p.k_bblk) * p.k_nsb * p.k_nhb + (h / p.k_hblk);
+            mbar_expect_tx(bar(Q_FULL), TILE_BYTES);
+            for (int half = 0; half < 2; ++half)
+                tma_load_5d(sQ + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.hblk, q0 % p.sblk, b % p.bblk,
+                            qb_flat_bh + (q0 / p.sblk) * p.nhb);
+            bool ok = true;
+            for (int j = 0; j < n_steps && ok; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1;
+                const int k0 = j * KT;
+                const int kflat = kb_flat_bh + (k0 / p.k_sblk) * p.k_nhb;
+                if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_5d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, h % p.k_hblk,
+                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_5d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, h % p.k_hblk,
+                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            // S = Q K^T: M=128, N=128, A and B K-major.  O' = P V: A from TMEM, B MN-major.
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            auto issue_qk = [&](int j) {
+                const int st = j & 1;
+                const uint32_t kaddr = sK + st * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {   // 16 d per instruction; d 0..63 in the first half, 64..127 in the second
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    umma_ss(tS[st], desc_sw128(sQ + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0);
+                }
+                commit1(bar(S_FULL + st));
+                commit1(bar(K_EMPTY + st));
+            };
+            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0);
+            }
+            for (int j = 0; j < n_steps && ok; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1;
+                if (j + 1 < n_steps) {
+                    if (!mbar_wait(bar(K_FULL + (st ^ 1)), (uint32_t)((j + 1) >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_qk(j + 1);   // overwrites the S/P buffer of step j-1: ordered behind P V of step j-1 on the tensor pipe
+                }
+                if (!mbar_wait(bar(P_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(bar(O_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t vaddr = sV + st * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)     // 16 keys per instruction: 8 TMEM columns of packed bf16 P, 2048 bytes of V
+                    umma_ts(tO[st], tS[st] + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv, kk > 0);
+                commit1(bar(O_FULL + st));
+                commit1(bar(V_EMPTY + st));
+            }
+        }
+    } else {
+        // ================= row threads: softmax and the running (O~, m, l) =================
+        const int q = warp & 3;
+        const int r = q * 32 + lane;                 // query row inside the tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        float o[D];
+#pragma unroll
+        for (int i = 0; i < D; ++i) o[i] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+        bool ok = true;
+
+        auto fold = [&](int st, float alpha) {   // O~ <- O~ * alpha + O'
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO[st] + lane_addr + c * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(v[i]));
+            }
+        };
+
+        for (int j = 0; j < n_steps && ok; ++j) {
+            const int st = j & 1;
+            const uint32_t ph = (uint32_t)(j >> 1) & 1;
+            if (!mbar_wait(bar(S_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const bool diag = p.causal && (j == n_steps - 1);
+            const int kmax = q0 + r - j * KT;        // columns c > kmax of this tile lie after the query row
+            // ---- pass 1: row maximum ----
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tS[st] + lane_addr + c * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float s = __uint_as_float(v[i]);
+                    if (diag && c * 32 + i > kmax) s = -INFINITY;
+                    mx = fmaxf(mx, s);
+                }
+            }
+            const float m_new = fmaxf(m_run, mx * p.scale_log2e);
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;           // e^(-inf - -inf) := 0
+            const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_use);
+            // ---- pass 2: P = 2^(S*scale - m), row sum, P written over S as packed bf16 ----
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tS[st] + lane_addr + c * 32, v);
+                tmem_ld_wait();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float p0 = ex2(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use));
+                    float p1 = ex2(fmaf(__uint_as_float(v[i + 1]), p.scale_log2e, -m_use));
+                    if (diag && c * 32 + i > kmax) p0 = 0.f;
+                    if (diag && c * 32 + i + 1 > kmax) p1 = 0.f;
+                    sum += p0 + p1;
+                    __nv_bfloat162 t = __floats2bfloat162_rn(p0, p1);
+                    pk[i / 2] = *reinterpret_cast<uint32_t*>(&t);
+                }
+                tmem_st16(tS[st] + lane_addr + c * 16, pk);   // columns [16c, 16c+16): S columns already consumed
+            }
+            l_run = l_run * alpha + sum;
+            m_run = m_new;
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P_FULL + st));
+            // ---- fold the partial of the previous step while the tensor pipe computes P V of this one ----
+            if (j > 0) {
+                const int ps = st ^ 1;
+                if (!mbar_wait(bar(O_FULL + ps), (uint32_t)((j - 1) >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                fold(ps, alpha_prev);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(O_EMPTY + ps));
+            }
+            alpha_prev = alpha;
+        }
+        if (ok && n_steps > 0) {
+            const int ls = (n_steps - 1) & 1;
+            if (mbar_wait(bar(O_FULL + ls), (uint32_t)((n_steps - 1) >> 1) & 1, abort_flag, p.status)) {
+                tc_fence_after();
+                fold(ls, alpha_prev);
+                // ---- O = O~ / l, one rounding, 256 contiguous bytes per row ----
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const int s_glob = q0 + r;
+                const int64_t flat = ((int64_t)(b / p.bblk) * p.nsb + s_glob / p.sblk) * p.nhb + h / p.hblk;
+                char* dst = p.o_base + flat * p.o_blk_stride +
+                            ((((int64_t)(b % p.bblk) * p.sblk + s_glob % p.sblk) * p.hblk + h % p.hblk) * D) * 2;
+#pragma unroll
+                for (int g = 0; g < 16; ++g) {
+                    uint4 ov;
+                    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
+                    *reinterpret_cast<uint4*>(dst + g * 16) = ov;
+                }
+            }
+        }
+    }
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+// "bshd" relation with equal blocks [bb, sb, hb, 128] as a rank-5 tensor: (d, h in block, s in block, b in block, block)
+ja_status_t encode_bshd(const RelView& v, CUtensorMap* tm) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const int64_t bb = v.bs[0], sb = v.bs[1], hb = v.bs[2];
+    const int64_t nblocks = (int64_t)v.nblk[0] * v.nblk[1] * v.nblk[2];
+    cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)hb, (cuuint64_t)sb, (cuuint64_t)bb, (cuuint64_t)nblocks};
+    cuuint64_t strides[4] = {(cuuint64_t)(D * 2), (cuuint64_t)(hb * D * 2), (cuuint64_t)(sb * hb * D * 2), (cuuint64_t)v.blk_stride};
+    cuuint32_t box[5] = {64, 1, 128, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, v.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (bshd) failed with code %d", (int)res);
+    return JA_OK;
+}
+
+}  // namespace
+
+// Returns JA_OK and sets *launched when the tensor-memory kernel took the job; leaves *launched false when the
+// tiling does not fit it (q and k row blocks must be multiples of 128 rows, all blocks of one shape).
+ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched) {
+    *launched = false;
+    if (a.qblk % 128 || a.kblk % 128 || !a.q.blk_stride || !a.k.blk_stride || !a.v.blk_stride || !a.o.blk_stride) return JA_OK;
+    if (a.v.blk_stride != a.k.blk_stride || a.o.blk_stride != a.q.blk_stride) return JA_OK;
+    CUtensorMap tq, tk, tv;
+    ja_status_t s;
+    if ((s = encode_bshd(a.q, &tq)) != JA_OK) return s;
+    if ((s = encode_bshd(a.k, &tk)) != JA_OK) return s;
+    if ((s = encode_bshd(a.v, &tv)) != JA_OK) return s;
+    AttnTcParams p;
+    memset(&p, 0, sizeof p);
+    p.o_base = a.o.base;
+    p.status = ja_device_status_word();
+    if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    p.o_blk_stride = a.o.blk_stride;
+    p.B = a.B; p.S = a.S; p.H = a.H;
+    p.bblk = (int)a.q.bs[0]; p.sblk = (int)a.q.bs[1]; p.hblk = (int)a.q.bs[2];
+    p.nsb = a.q.nblk[1]; p.nhb = a.q.nblk[2];
+    p.k_bblk = (int)a.k.bs[0]; p.k_sblk = (int)a.k.bs[1]; p.k_hblk = (int)a.k.bs[2];
+    p.k_nsb = a.k.nblk[1]; p.k_nhb = a.k.nblk[2];
+    p.causal = a.causal;
+    p.scale_log2e = a.scale * 1.4426950408889634f;
+    JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
+    attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+    ja_count_launch();
+    JA_CUDA(cudaGetLastError());
+    *launched = true;
+    return JA_OK;
+}
