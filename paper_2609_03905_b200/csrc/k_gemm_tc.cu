@@ -33,14 +33,18 @@ namespace {
 
 using namespace ja_ptx;
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB: 128 rows x 64 k
-constexpr int B_CHUNK_BYTES = BK * 64 * 2;   // one 64-column box: 8 KiB
+constexpr int BM = 128, BN = 256;
 constexpr int NUM_THREADS = 192;
-constexpr int MAX_STAGES = 6;
+// BK = contraction depth of one pipeline stage. TMA throughput grows with the box size (measured on this part:
+// 8 KiB boxes ~10 TB/s, 16 KiB ~12.7 TB/s aggregate), so the two-CTA form stages 128-deep chunks: every box it
+// issues (A: 128 rows x 64 k, B: 128 k x 64 columns) is 16 KiB.
 template <int CG> struct Cfg {
-    static constexpr int STAGES = CG == 1 ? 4 : 6;
-    static constexpr int B_STAGE_BYTES = BK * (BN / CG) * 2;  // 32 KiB, or 16 KiB per CTA of a pair
+    static constexpr int BK = CG == 1 ? 64 : 128;
+    static constexpr int STAGES = CG == 1 ? 4 : 3;
+    static constexpr int A_HALF_BYTES = BM * 64 * 2;                 // 128 rows x 64 k under the 128-byte swizzle
+    static constexpr int A_STAGE_BYTES = A_HALF_BYTES * (BK / 64);
+    static constexpr int B_CHUNK_BYTES = BK * 64 * 2;                // one box: BK k-rows x 64 columns
+    static constexpr int B_STAGE_BYTES = B_CHUNK_BYTES * (BN / CG / 64);
     static constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
 };
 
@@ -55,6 +59,7 @@ struct GemmParams {
     int32_t m_tiles, n_tiles;  // tile grid (tiles are 128*CG rows x up to 256 columns)
     int32_t tiles_per_mblk;    // >= 1 when row tiles never leave a block, 0 when tiles are cut from global rows
     int32_t tiles_per_nblk;    // >= 1 when tiles stay inside one column block, 0 when tiles span blocks
+    int32_t group_m;           // row tiles per rasterisation band
 };
 
 // What one CTA does for one tile: its own 128 rows, and (CG 2) its own half of the tile's columns as B operand.
@@ -69,7 +74,12 @@ struct TileCoord {
 template <int CG>
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int cta_rank) {
     TileCoord tc;
-    const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+    // banded rasterisation: tiles that run at the same time cover group_m row tiles x several column tiles, so the
+    // operand strips they stream fit in L2 together
+    const int band_sz = p.group_m * p.n_tiles;
+    const int band = t / band_sz, tin = t - band * band_sz;
+    const int rows_in_band = min(p.group_m, p.m_tiles - band * p.group_m);
+    const int mt = band * p.group_m + tin % rows_in_band, nt = tin / rows_in_band;
     if (p.tiles_per_mblk > 0) {   // CG == 1 only: row tiles stay inside a block
         tc.mb = mt / p.tiles_per_mblk;
         tc.r0 = (mt % p.tiles_per_mblk) * BM;
@@ -98,8 +108,9 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int 
 template <int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
-    constexpr int STAGES = Cfg<CG>::STAGES;
-    constexpr int B_STAGE_BYTES = Cfg<CG>::B_STAGE_BYTES;
+    constexpr int STAGES = Cfg<CG>::STAGES, BK = Cfg<CG>::BK;
+    constexpr int A_STAGE_BYTES = Cfg<CG>::A_STAGE_BYTES, A_HALF_BYTES = Cfg<CG>::A_HALF_BYTES;
+    constexpr int B_STAGE_BYTES = Cfg<CG>::B_STAGE_BYTES, B_CHUNK_BYTES = Cfg<CG>::B_CHUNK_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
@@ -145,7 +156,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tmem_base = *tmem_slot;
 
     const int total_tiles = p.m_tiles * p.n_tiles;
-    const int kchunks = (p.bk + BK - 1) / BK;
+    const int kchunks = (p.bk + Cfg<CG>::BK - 1) / Cfg<CG>::BK;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
     if (warp == 0) {
@@ -172,12 +183,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (cta_rank == 0) mbar_expect_tx(full_bar(stage), tx);
                         issued[stage] = true;
                         last_parity[stage] = phase;
-                        // A: boxes of a_box_rows rows x 64 k
+                        // A: boxes of a_box_rows rows x 64 k, one set per 64-deep half of the stage
                         const int nboxes = BM / p.a_box_rows;
-                        for (int bx = 0; bx < nboxes; ++bx)
-                            tma_load_4d<CG>(sA + stage * A_STAGE_BYTES + bx * p.a_box_rows * 128, &tmA, fb, kc * BK,
-                                            tc.r0, jb, tc.mb + bx);
-                        // B: one box of 64 k-rows x 64 columns per 64-column chunk
+                        for (int kh = 0; kh < BK / 64; ++kh)
+                            for (int bx = 0; bx < nboxes; ++bx)
+                                tma_load_4d<CG>(sA + stage * A_STAGE_BYTES + kh * A_HALF_BYTES + bx * p.a_box_rows * 128, &tmA, fb,
+                                                kc * BK + kh * 64, tc.r0, jb, tc.mb + bx);
+                        // B: one box of BK k-rows x 64 columns per 64-column chunk
                         for (int c = 0; c < nchunks; ++c) {
                             int nb, cin;
                             if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + my_c0 + 64 * c; }
@@ -227,8 +239,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint32_t a_addr = sA + stage * A_STAGE_BYTES;
                         const uint32_t b_addr = sB + stage * B_STAGE_BYTES;
                         for (int kk = 0; kk < k16; ++kk) {
-                            // A: K-major, 16 k = 32 bytes inside the swizzle atom; B: MN-major, 16 k-rows = 2048 bytes
-                            uint64_t da = desc_sw128(a_addr + kk * 32, 16);
+                            // A: K-major, 16 k = 32 bytes inside the swizzle atom, 64 k per half; B: MN-major, 16 k-rows =
+                            // 2048 bytes, 64-column groups BK*128 bytes apart
+                            uint64_t da = desc_sw128(a_addr + (kk >> 2) * A_HALF_BYTES + (kk & 3) * 32, 16);
                             uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
                             umma_bf16<CG>(d_tmem, da, db, idesc, accumulate);
                             accumulate = 1;
@@ -303,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // ---- host: tensor maps -------------------------------------------------------------------------------------
 // A relation [R, C] with equal blocks br x bc is the rank-4 tensor (c in block, r in block, col-block, row-block).
 ja_status_t encode_blocked_2d(const ja_relation* r, int box_inner, int box_rows, CUtensorMap* tm) {
+    if (box_rows > 256) return ja_fail(JA_ERR_INVALID_ARG, "TMA box too tall");
     EncodeTiledFn enc = get_encode();
     if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     const int64_t br = r->bs[0], bc = r->bs[1];
@@ -349,8 +363,11 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     else { p.tiles_per_nblk = (int)((bn + BN - 1) / BN); p.n_tiles = p.tiles_per_nblk * p.nbn; }
     // Two-CTA form: 256-row tiles cut from global rows; needs 128-row halves that never straddle a block and, when
     // tiles span column blocks, column tails whose halves still start on a 64-column box boundary.
+    const char* gm = getenv("JA_GEMM_GROUP_M");
+    p.group_m = gm ? atoi(gm) : 8;
+    if (p.group_m < 1) p.group_m = 1;
     const char* force = getenv("JA_GEMM_CTA_GROUP");
-    bool two = (bm % 128 == 0 || 128 % bm == 0) && p.M >= 256;
+    bool two = (bm % 128 == 0 || 128 % bm == 0) && p.M >= 256 && bk >= Cfg<2>::BK;
     if (p.tiles_per_nblk == 0 && (p.N % BN) % 128 != 0) two = false;
     if (force && force[0] == '1') two = false;
     plan->cg = two ? 2 : 1;
@@ -358,7 +375,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     else { p.tiles_per_mblk = (int)((bm + BM - 1) / BM); p.m_tiles = p.tiles_per_mblk * p.nbm; }
     ja_status_t st;
     if ((st = encode_blocked_2d(A, 64, p.a_box_rows, &plan->tmA)) != JA_OK) return st;
-    if ((st = encode_blocked_2d(B, 64, 64, &plan->tmB)) != JA_OK) return st;
+    if ((st = encode_blocked_2d(B, 64, two ? Cfg<2>::BK : Cfg<1>::BK, &plan->tmB)) != JA_OK) return st;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
