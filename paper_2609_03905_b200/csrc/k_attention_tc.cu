@@ -15,6 +15,8 @@
 // TMEM map (512 columns): S/P buffers at 0 and 128, partial-O buffers at 256 and 384. QK^T of step j+1 is issued
 // before the softmax of step j finishes, so the tensor pipe works while the row threads exponentiate.
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT and leaves through the normal exit.
+#include <stdlib.h>
+
 #include "ja_device.cuh"
 #include "ja_ptx.cuh"
 
@@ -75,6 +77,27 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
           "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+          "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2(float x) {
@@ -311,6 +334,300 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 }
 
+// ---- row-thread arithmetic: 3-input max and packed f32x2 math keep the instruction count per score low ----
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// maximum of one row of scores (128 fp32 bit patterns); MASK: columns > kmax lie after the query row
+template <bool MASK>
+__device__ __forceinline__ float row_max128(const uint32_t (&v)[128], int kmax) {
+    if (MASK) {
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; ++i) mx = fmaxf(mx, i > kmax ? -INFINITY : __uint_as_float(v[i]));
+        return mx;
+    }
+    float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]), m2 = __uint_as_float(v[2]), m3 = __uint_as_float(v[3]);
+#pragma unroll
+    for (int i = 4; i + 7 < 128; i += 8) {
+        m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+        m2 = max3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+        m3 = max3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+    }
+    m0 = max3(m0, __uint_as_float(v[124]), __uint_as_float(v[125]));
+    m1 = max3(m1, __uint_as_float(v[126]), __uint_as_float(v[127]));
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// P = 2^(S*scale - m) as packed bf16 written over S in tensor memory; returns the row sum
+template <bool MASK>
+__device__ __forceinline__ float row_exp_store128(const uint32_t (&v)[128], int kmax, float scale, float m_used, uint32_t t_dst) {
+    const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
+    uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+            const int col = c * 16 + i;
+            float p0, p1;
+            unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
+            if (MASK) {
+                if (col > kmax) p0 = 0.f;
+                if (col + 1 > kmax) p1 = 0.f;
+            }
+            if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
+            else sum_b = add2(sum_b, pack2(p0, p1));
+            __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
+            pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
+        }
+        tmem_st8(t_dst + c * 8, pk);
+    }
+    float a0, a1, b0, b1;
+    unpack2(sum_a, a0, a1);
+    unpack2(sum_b, b0, b1);
+    return (a0 + a1) + (b0 + b1);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Two query tiles per CTA. The CTA owns 256 query rows of one (batch, head) as two independent 128-row output
+// key tiles A and B that share every K_j / V_j tile it loads. While the row threads of one tile exponentiate,
+// the tensor pipe works on the other tile, and each scheduler holds two row warps.
+//   TMEM: S/P of A at 0, S/P of B at 128, O~ of A at 256, O~ of B at 384 (fp32, 128 columns each).
+//   O~ is ACCUMULATED IN TENSOR MEMORY by the P V products (accumulate flag), not in registers. The running
+//   maximum used as the exponent offset is only raised when a row's new maximum exceeds it by more than 2^8
+//   (P stays <= 256, exact in the final O~/l); only then is the row's O~ rescaled in TMEM by its row thread.
+//   warp 0 TMA, warp 1 MMA issuer, warps 2..5 rows of A, warps 6..9 rows of B.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int NUM_THREADS2 = 320;
+constexpr int SMEM_BYTES2 = 6 * TILE_BYTES + 1024 + 256;   // Q_A, Q_B, K x2, V x2
+
+__global__ void __launch_bounds__(NUM_THREADS2, 1)
+attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t sQ = base, sK = base + 2 * TILE_BYTES, sV = base + 4 * TILE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * TILE_BYTES);
+    const uint32_t bar0 = smem_u32(bars);
+    enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, P_FULL = 11, O_FULL = 13, NBAR = 15 };
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int n_pairs = p.S / (2 * QT);
+    const int pr = n_pairs - 1 - (int)blockIdx.x;     // heaviest output keys first
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int q0 = pr * 2 * QT;                       // first row of tile A; tile B starts at q0 + 128
+    const int n_steps_a = p.causal ? (q0 + QT) / KT : p.S / KT;
+    const int n_steps_b = p.causal ? (q0 + 2 * QT) / KT : p.S / KT;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2) ? 4 : 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            const int qb_flat_bh = (b / p.bblk) * p.nsb * p.nhb + (h / p.hblk);
+            const int kb_flat_bh = (b / p.k_bblk) * p.k_nsb * p.k_nhb + (h / p.k_hblk);
+            mbar_expect_tx(bar(Q_FULL), 2 * TILE_BYTES);
+            for (int t = 0; t < 2; ++t)
+                for (int half = 0; half < 2; ++half) {
+                    const int qs = q0 + t * QT;
+                    tma_load_5d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.hblk, qs % p.sblk,
+                                b % p.bblk, qb_flat_bh + (qs / p.sblk) * p.nhb);
+                }
+            bool ok = true;
+            for (int j = 0; j < n_steps_b && ok; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1;
+                const int k0 = j * KT;
+                const int kflat = kb_flat_bh + (k0 / p.k_sblk) * p.k_nhb;
+                if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_5d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, h % p.k_hblk,
+                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_5d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, h % p.k_hblk,
+                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            auto issue_qk = [&](int t, int j) {          // S_t = Q_t K_j^T
+                const uint32_t kaddr = sK + (j & 1) * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    umma_ss(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0);
+                }
+                commit1(bar(S_FULL + t));
+            };
+            auto issue_pv = [&](int t, int j) {          // O~_t (+)= P_t V_j
+                const uint32_t vaddr = sV + (j & 1) * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
+                            (j > 0 || kk > 0) ? 1u : 0u);
+                commit1(bar(O_FULL + t));
+            };
+            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0);
+                issue_qk(1, 0);
+                commit1(bar(K_EMPTY + 0));                // K_0 consumed
+            }
+            for (int j = 0; j < n_steps_b && ok; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1;
+                const bool more = j + 1 < n_steps_b;
+                if (more) {
+                    if (!mbar_wait(bar(K_FULL + (st ^ 1)), (uint32_t)((j + 1) >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                }
+                if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
+                for (int t = 0; t < 2 && ok; ++t) {
+                    const int n_t = t == 0 ? n_steps_a : n_steps_b;
+                    if (j < n_t) {
+                        if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_pv(t, j);
+                    }
+                    if (j + 1 < n_t) issue_qk(t, j + 1);   // ordered behind P V of this tile on the tensor pipe
+                }
+                if (!ok) break;
+                commit1(bar(V_EMPTY + st));               // V_j consumed by both tiles
+                // K_{j+1} consumed by the QK products issued above (both tiles, or tile B alone on its last step)
+                if (more) commit1(bar(K_EMPTY + (st ^ 1)));
+            }
+        }
+    } else {
+        // ================= row threads =================
+        const int t = (warp - 2) >> 2;               // tile: 0 = A, 1 = B
+        const int q = warp & 3;                      // TMEM lane group of this warp (warps 2..5 -> 2,3,0,1; 6..9 -> 2,3,0,1)
+        const int r = q * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const uint32_t tS = tmem_base + t * 128 + lane_addr, tO = tmem_base + 256 + t * 128 + lane_addr;
+        const int n_t = t == 0 ? n_steps_a : n_steps_b;
+        const int qrow = q0 + t * QT + r;            // sequence position of this row
+        float m_used = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_t && ok; ++j) {
+            if (!mbar_wait(bar(S_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const bool diag = p.causal && (j == n_t - 1);
+            const int kmax = qrow - j * KT;
+            uint32_t v[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
+            tmem_ld_wait();
+            const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
+            const float m_new = mx * p.scale_log2e;       // finite: key 0 of the first tile is never masked
+            // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
+            float alpha = 1.f;
+            bool need = false;
+            if (j == 0) m_used = m_new;
+            else if (m_new > m_used + 8.f) { alpha = ex2(m_used - m_new); m_used = m_new; need = true; }
+            if (__any_sync(0xffffffffu, need)) {
+                // O~ of this tile holds the products up to step j-1: wait for them, then scale this row in place
+                if (!mbar_wait(bar(O_FULL + t), (uint32_t)(j - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll 1
+                for (int c = 0; c < 16; ++c) {   // rare path: small chunks keep the register footprint of the hot path low
+                    uint32_t o[8];
+                    tmem_ld8(tO + c * 8, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st8(tO + c * 8, o);
+                }
+                tmem_st_wait();
+                l_run *= alpha;
+            }
+            const float sum = diag ? row_exp_store128<true>(v, kmax, p.scale_log2e, m_used, tS)
+                                   : row_exp_store128<false>(v, kmax, p.scale_log2e, m_used, tS);
+            l_run += sum;
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P_FULL + t));
+        }
+        if (ok && n_t > 0) {
+            if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
+                tc_fence_after();
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const int64_t flat = ((int64_t)(b / p.bblk) * p.nsb + qrow / p.sblk) * p.nhb + h / p.hblk;
+                char* dst = p.o_base + flat * p.o_blk_stride +
+                            ((((int64_t)(b % p.bblk) * p.sblk + qrow % p.sblk) * p.hblk + h % p.hblk) * D) * 2;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 ov;
+                        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 64 + g * 16) = ov;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
 // "bshd" relation with equal blocks [bb, sb, hb, 128] as a rank-5 tensor: (d, h in block, s in block, b in block, block)
 ja_status_t encode_bshd(const RelView& v, CUtensorMap* tm) {
     EncodeTiledFn enc = get_encode();
@@ -353,9 +670,16 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
     p.k_nsb = a.k.nblk[1]; p.k_nhb = a.k.nblk[2];
     p.causal = a.causal;
     p.scale_log2e = a.scale * 1.4426950408889634f;
-    JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
-    attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+    const char* one = getenv("JA_ATTN_ONE_TILE");
+    if (a.S % (2 * QT) == 0 && !(one && one[0] == '1')) {
+        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
+        dim3 grid((unsigned)(a.S / (2 * QT)), (unsigned)a.H, (unsigned)a.B);
+        attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
+    } else {
+        JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
+        attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+    }
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
     *launched = true;

@@ -8,6 +8,7 @@
 //    output key (Definition 3.7); the partial never leaves registers.
 //
 // All loads/stores are 128-bit when the tiling allows (every split of j a multiple of the vector width).
+#include <stdlib.h>
 #include <string.h>
 
 #include "ja_device.cuh"
@@ -282,7 +283,7 @@ struct FastGeom {
 };
 
 template <typename T, int VEC, int VPT, int OP>
-__global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowArgs a, FastGeom g, int64_t n_rows, int team) {
+__global__ void __launch_bounds__(256, (VPT <= 4 ? 3 : 1)) row_fast_kernel(RowArgs a, FastGeom g, int64_t n_rows, int team) {
     __shared__ float red[64];
     using V = Vec<T, VEC>;
     const int rpc = blockDim.x / team;
@@ -305,41 +306,58 @@ __global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowAr
     }
     const int64_t strip = (int64_t)g.nbc * g.blk_elems;  // elements in one strip of column blocks
 
-    for (int64_t row0 = (int64_t)blockIdx.x * rpc; row0 < n_rows; row0 += (int64_t)gridDim.x * rpc) {
-        const int64_t row = row0 + row_in_cta;
-        const bool live = row < n_rows;
-        // ---- rowpart ----------------------------------------------------------------------------------------
-        uint32_t rem = (uint32_t)(live ? row : 0);
-        int lead_flat = 0, lead_in = 0, pos = 0;
-        {
-            int c[3] = {0, 0, 0};
+    // rowpart, statistics offset and position of one row
+    struct RowGeom { int64_t rowpart, stat_off; int pos; bool live; };
+    auto geom = [&](int64_t row) {
+        RowGeom rg;
+        rg.live = row < n_rows;
+        uint32_t rem = (uint32_t)(rg.live ? row : 0);
+        int lead_flat = 0, lead_in = 0;
+        int c[3] = {0, 0, 0};
 #pragma unroll
-            for (int d = 2; d >= 0; --d) {
-                if (d < g.lead_rank) {
-                    const uint32_t q = rem / (uint32_t)g.lead_ext[d];
-                    c[d] = (int)(rem - q * (uint32_t)g.lead_ext[d]);
-                    rem = q;
-                }
+        for (int d = 2; d >= 0; --d) {
+            if (d < g.lead_rank) {
+                const uint32_t q = rem / (uint32_t)g.lead_ext[d];
+                c[d] = (int)(rem - q * (uint32_t)g.lead_ext[d]);
+                rem = q;
             }
-#pragma unroll
-            for (int d = 0; d < 3; ++d) {
-                if (d < g.lead_rank) {
-                    const int b = (int)((uint32_t)c[d] / (uint32_t)g.lead_bs[d]);
-                    lead_flat = lead_flat * g.lead_nb[d] + b;
-                    lead_in = lead_in * g.lead_bs[d] + (c[d] - b * g.lead_bs[d]);
-                }
-            }
-            pos = c[1];
         }
-        const int64_t rowpart = (int64_t)lead_flat * strip + (int64_t)lead_in * g.bsc;
-        const T* xrow = reinterpret_cast<const T*>(a.x.base) + rowpart;
-        T* yrow = reinterpret_cast<T*>(a.y.base) + rowpart;
-        const int64_t stat_off = (int64_t)lead_flat * g.stat_blk_bytes + (int64_t)lead_in * 4;
+#pragma unroll
+        for (int d = 0; d < 3; ++d) {
+            if (d < g.lead_rank) {
+                const int b = (int)((uint32_t)c[d] / (uint32_t)g.lead_bs[d]);
+                lead_flat = lead_flat * g.lead_nb[d] + b;
+                lead_in = lead_in * g.lead_bs[d] + (c[d] - b * g.lead_bs[d]);
+            }
+        }
+        rg.pos = c[1];
+        rg.rowpart = (int64_t)lead_flat * strip + (int64_t)lead_in * g.bsc;
+        rg.stat_off = (int64_t)lead_flat * g.stat_blk_bytes + (int64_t)lead_in * 4;
+        return rg;
+    };
 
-        V raw[VPT];
+    // software pipeline over rows: the loads of the next row are in flight while this row is reduced and written
+    const int64_t row_step = (int64_t)gridDim.x * rpc;
+    RowGeom cur = geom((int64_t)blockIdx.x * rpc + row_in_cta);
+    V raw[VPT], nxt[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k)
+        if (cur.live && colpart[k] >= 0) raw[k] = *reinterpret_cast<const V*>(reinterpret_cast<const T*>(a.x.base) + cur.rowpart + colpart[k]);
+
+    for (int64_t row0 = (int64_t)blockIdx.x * rpc; row0 < n_rows; row0 += row_step) {
+        const bool live = cur.live;
+        const int pos = cur.pos;
+        const int64_t stat_off = cur.stat_off;
+        T* yrow = reinterpret_cast<T*>(a.y.base) + cur.rowpart;
+        RowGeom nx = geom(row0 + row_step + row_in_cta);
 #pragma unroll
         for (int k = 0; k < VPT; ++k)
-            if (live && colpart[k] >= 0) raw[k] = *reinterpret_cast<const V*>(xrow + colpart[k]);
+            if (nx.live && colpart[k] >= 0) nxt[k] = *reinterpret_cast<const V*>(reinterpret_cast<const T*>(a.x.base) + nx.rowpart + colpart[k]);
+        auto advance = [&]() {
+#pragma unroll
+            for (int k = 0; k < VPT; ++k) raw[k] = nxt[k];
+            cur = nx;
+        };
 
         float m = 0.f, l = 0.f, rstd = 0.f;
         float ex[KEEP_EXP ? VPT * VEC : 1];
@@ -354,6 +372,7 @@ __global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowAr
             s = team_reduce<false>(s, team, red, row_in_cta, lane_t);
             if (OP == ROW_SUMSQ) {
                 if (live && lane_t == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = s;
+                advance();
                 continue;
             }
             rstd = 1.0f / sqrtf(s / (float)g.n + a.eps);
@@ -369,6 +388,7 @@ __global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowAr
             m = team_reduce<true>(mx, team, red, row_in_cta, lane_t);
             if (OP == ROW_MAX) {
                 if (live && lane_t == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+                advance();
                 continue;
             }
         }
@@ -388,6 +408,7 @@ __global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowAr
             l = team_reduce<false>(s, team, red, row_in_cta, lane_t);
             if (OP == ROW_EXPSUM) {
                 if (live && lane_t == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+                advance();
                 continue;
             }
         }
@@ -425,6 +446,7 @@ __global__ void __launch_bounds__(256, (VPT <= 8 ? 3 : 1)) row_fast_kernel(RowAr
             }
             *reinterpret_cast<V*>(yrow + colpart[k]) = o;
         }
+        advance();
     }
 }
 
@@ -435,8 +457,14 @@ void launch_fast_v(const RowArgs& a, const FastGeom& g, int64_t n_rows, int team
     const int block = team >= 64 ? team : 128;
     const int rpc = block / team;
     int64_t want = (n_rows + rpc - 1) / rpc;
-    const int64_t cap = (int64_t)148 * (2048 / block);
-    unsigned grid = (unsigned)(want < cap ? want : cap);
+    // persistent: exactly as many CTAs as are resident at once
+    static int resident = 0;   // per template instance
+    if (resident == 0) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_fast_kernel<T, VEC, VPT, OP>, block, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+        resident = per_sm * 148;
+    }
+    unsigned grid = (unsigned)(want < resident ? want : resident);
     row_fast_kernel<T, VEC, VPT, OP><<<grid, block, 0, st>>>(a, g, n_rows, team);
 }
 
@@ -444,10 +472,13 @@ void launch_fast_v(const RowArgs& a, const FastGeom& g, int64_t n_rows, int team
 template <typename T, int OP>
 bool launch_fast(const RowArgs& a, const FastGeom& g, int64_t n_rows, cudaStream_t st) {
     constexpr int VEC = 16 / (int)sizeof(T);
-    // one warp per row while a lane holds at most 8 vectors (a whole row in flight per warp, no barrier);
-    // longer rows take 2, 4 or 8 warps
+    // few vectors per thread (two register sets: the row being processed and the prefetched next row);
+    // rows longer than one warp's share take 2, 4 or 8 warps
+    // measured on B200: maps that write a row back run best with 2 vectors per thread, pure reductions with 4
+    constexpr bool REDUCE_ONLY = (OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM);
     int team = 32;
-    while (team < 256 && g.n > team * VEC * 8) team *= 2;
+    while (team < 256 && g.n > team * VEC * (REDUCE_ONLY ? 4 : 2)) team *= 2;
+    if (const char* e = getenv("JA_ROW_TEAM")) { int t = atoi(e); if (t >= 32 && t <= 256 && (t & (t - 1)) == 0) team = t; }
     const int vpt = (g.n + team * VEC - 1) / (team * VEC);
     if (vpt <= 1) launch_fast_v<T, VEC, 1, OP>(a, g, n_rows, team, st);
     else if (vpt <= 2) launch_fast_v<T, VEC, 2, OP>(a, g, n_rows, team, st);

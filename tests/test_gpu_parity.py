@@ -216,9 +216,10 @@ def test_rope(splits):
                                                    (1, 256, 1, 64, 64, 1, True), (1, 384, 2, 128, 64, 1, False),
                                                    (1, 512, 1, 256, 128, 1, True), (2, 1024, 3, 128, 256, 3, True),
                                                    (1, 640, 2, 128, 128, 1, False)])
-@pytest.mark.parametrize("form", ["tcgen05", "mma_sync"])
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles", "tcgen05_one_tile", "mma_sync"])
 def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
     monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
+    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
     D = 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (1, 2, 3))
     spl = lambda blk: [ES(B, B), ES(S, S // blk), ES(H, H // hb), [0, D]]
