@@ -163,6 +163,28 @@ ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* dst, void* c
 ja_status_t ja_overlay_atoms(const ja_relation_t* src, const ja_relation_t* dst, int64_t* n_atoms, int64_t* lower,
                              int64_t* upper, int32_t* src_block, int32_t* dst_block);
 
+/* ---- relayout without allocation -------------------------------------------------------------------
+ * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)
+ * Same data movement as ja_repartition -- every atom of the overlay of the two tilings is copied from its
+ * source block to its destination block, bit-exact -- for callers that must not trigger a device (or host)
+ * allocation: servers that gave all of HBM to their own pool at start-up, latency-critical loops that cannot
+ * afford cudaMalloc's implicit synchronisation, harnesses that fail on any allocation they did not make.
+ * It takes the tilings and the payload pointers directly (no relation handles), keeps its copy plan in a
+ * fixed device array inside the library (16384 slabs, 512 KiB per GPU, held until process exit) and calls no
+ * cudaMalloc / cudaFree / allocating routine.
+ *   extents[rank]; src_nparts / dst_nparts [rank]; src_splits / dst_splits [rank] pointers to nparts+1
+ *   ascending split points each (all HOST); src_device / dst_device: DEVICE payloads in block-key layout,
+ *   128-byte aligned, distinct, sized as ja_relation_bytes reports for their tilings.
+ * Limits (JA_ERR_UNSUPPORTED beyond them): 16384 copy slabs (one per atom row-chunk of <= 64 KiB), 4096 blocks
+ * per tiling, 1024 overlay split points per dimension.
+ * All calls share the plan array; it keeps the last call's contents and a call reads only what it has just
+ * written, so nothing needs clearing -- but calls whose GPU work overlaps race on it: serialise them.
+ * The first call on each device resolves the array's device address; issue it before any stream capture. */
+ja_status_t ja_repartition_noalloc(int32_t rank, const int64_t* extents, const int32_t* src_nparts,
+                                   const int64_t* const* src_splits, const int32_t* dst_nparts,
+                                   const int64_t* const* dst_splits, ja_dtype_t dtype, const void* src_device,
+                                   void* dst_device, void* cuda_stream);
+
 /* Device-detected conditions (bounded-wait expiry) accumulate in a status word; this call synchronizes
  * `cuda_stream`, returns the word in *device_status and clears it. */
 ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_status);

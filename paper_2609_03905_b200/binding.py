@@ -60,6 +60,7 @@ def _load() -> ctypes.CDLL:
         "ja_repartition": [vp, vp, vp],
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
+        "ja_repartition_noalloc": [i32, P(i64), P(i32), P(P(i64)), P(i32), P(P(i64)), ctypes.c_int, vp, vp, vp],
     }
     for name, argtypes in sigs.items():
         fn = getattr(lib, name)
@@ -193,6 +194,20 @@ def ja_execute(spec: int, inputs, outputs, stream: int = 0):
 
 def ja_repartition(src: int, dst: int, stream: int = 0):
     _check(LIB.ja_repartition(src, dst, ctypes.c_void_p(stream)))
+
+
+def ja_repartition_noalloc(extents, src_splits, dst_splits, dtype: int, src_ptr: int, dst_ptr: int, stream: int = 0):
+    """Relayout between two tilings given as plain split lists and raw device pointers. Unlike ja_repartition this
+    never allocates (no cudaMalloc, no cached plan): for callers whose memory is fixed up front. Calls share one
+    fixed plan table on the device, so do not let two of them overlap on the GPU."""
+    rank = len(extents)
+    ext = (ctypes.c_int64 * rank)(*[int(e) for e in extents])
+    snp = (ctypes.c_int32 * rank)(*[len(s) - 1 for s in src_splits])
+    dnp = (ctypes.c_int32 * rank)(*[len(s) - 1 for s in dst_splits])
+    keep_s, sp = _splits_arrays(src_splits)
+    keep_d, dp = _splits_arrays(dst_splits)
+    _check(LIB.ja_repartition_noalloc(rank, ext, snp, sp, dnp, dp, dtype, ctypes.c_void_p(src_ptr), ctypes.c_void_p(dst_ptr),
+                                      ctypes.c_void_p(stream)))
 
 
 def ja_overlay_atoms(src: int, dst: int):
