@@ -283,7 +283,7 @@ struct FastGeom {
 };
 
 template <typename T, int VEC, int VPT, int OP>
-__global__ void __launch_bounds__(256, (VPT <= 4 ? 3 : 1)) row_fast_kernel(RowArgs a, FastGeom g, int64_t n_rows, int team) {
+__global__ void __launch_bounds__(256, (VPT <= 2 ? 4 : (VPT <= 4 ? 3 : 1))) row_fast_kernel(RowArgs a, FastGeom g, int64_t n_rows, int team) {
     __shared__ float red[64];
     using V = Vec<T, VEC>;
     const int rpc = blockDim.x / team;
