@@ -203,24 +203,60 @@ def run_gpu(args, shape):
     ms_total = t_start.elapsed_time(t_end)
     assert ja.ja_stream_status(stream.cuda_stream) == 0, "device status word set during the timed region"
 
-    # ---- end to end: H2D of the step's input, pack, block, unpack, D2H of the result ------------------------------
+    # ---- end to end: every step copies its input from pinned host memory, packs it into the block's input relation
+    # (ja_repartition), runs the block, recomposes the output (ja_repartition) and copies it back to the host. Steps are
+    # independent, so the copies of neighbouring steps overlap the compute of this one: H2D on one stream, kernels on the
+    # caller's stream, D2H on a third, two staging buffers each, ordered by events.
+    x_devs = [x_dev, torch.empty_like(x_dev)]
+    x_denses = [x_dense, ja.Relation([T, hidden], [[0, T], [0, hidden]], bf, x_devs[1].reshape(-1))]
+    out_denses = [out_dense, ja.Relation([T, hidden], [[0, T], [0, hidden]], bf)]
+    out_hosts = [out_host, torch.empty((T, hidden), dtype=bf).pin_memory()]
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(2)]         # H2D of buffer b finished
+    ev_packed = [torch.cuda.Event() for _ in range(2)]     # buffer b consumed by the pack relayout
+    ev_out = [torch.cuda.Event() for _ in range(2)]        # output buffer b written
+    ev_d2h = [torch.cuda.Event() for _ in range(2)]        # output buffer b copied to the host
+    step_no = [0]
+
     def e2e_step():
-        x_dev.copy_(x_host, non_blocking=True)
-        ja.repartition(x_dense, blk.x)
+        i = step_no[0]
+        b = i & 1
+        step_no[0] += 1
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(ev_packed[b])
+            x_devs[b].copy_(x_host, non_blocking=True)
+            ev_in[b].record(s_in)
+        stream.wait_event(ev_in[b])
+        ja.repartition(x_denses[b], blk.x)
+        ev_packed[b].record(stream)
         blk.forward()
-        ja.repartition(blk.out, out_dense)
-        out_host.copy_(out_dense.payload[: T * hidden].view(T, hidden), non_blocking=True)
+        if i >= 2:
+            stream.wait_event(ev_d2h[b])
+        ja.repartition(blk.out, out_denses[b])
+        ev_out[b].record(stream)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_out[b])
+            out_hosts[b].copy_(out_denses[b].payload[: T * hidden].view(T, hidden), non_blocking=True)
+            ev_d2h[b].record(s_out)
+
+    def e2e_drain():
+        stream.wait_stream(s_in)
+        stream.wait_stream(s_out)
 
     for _ in range(min(args.warmup, 3)):
         e2e_step()
+    e2e_drain()
     sync_all()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
         e2e_step()
+    e2e_drain()
     e1.record(stream)
     sync_all()
     ms_e2e = e0.elapsed_time(e1)
+    assert torch.equal(out_hosts[0], out_hosts[1]), "end-to-end outputs of consecutive steps differ"
 
     times = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
     if world > 1:

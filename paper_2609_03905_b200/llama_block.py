@@ -26,7 +26,8 @@ from .relations import Relation, Spec, equal_splits as ES, from_dense, repartiti
 
 class LlamaBlock:
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
-                 theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8):
+                 theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8,
+                 ffn_blocks: int | None = None):
         assert plan in ("seq", "head")
         assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
         assert seq % token_block == 0
@@ -39,7 +40,11 @@ class LlamaBlock:
         io_c = ES(hidden, col_blocks)                    # column tiling of the block's input / output
         head_c = ES(hidden, n_heads)                     # one head per column block
         act_c = io_c if plan == "seq" else head_c        # column tiling of the plan's [T, hidden] activations
-        ffn_c = ES(ffn, col_blocks)
+        # the FFN index is cut into 256-wide blocks when it divides evenly (11008 = 43 x 256, 22016 = 86 x 256): every
+        # output tile of the up-projections is then a whole block, with no ragged tail tile per block
+        if ffn_blocks is None:
+            ffn_blocks = ffn // 256 if ffn % 256 == 0 else col_blocks
+        ffn_c = ES(ffn, ffn_blocks)
         self.t_sp, self.io_c, self.head_c, self.act_c, self.ffn_c = t_sp, io_c, head_c, act_c, ffn_c
         qkv_c = io_c if plan == "seq" else head_c        # tiling q, k, v are produced in
 
