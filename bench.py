@@ -141,7 +141,7 @@ def run_gpu(args, shape):
     Bt, S, hidden, heads, ffn = shape["batch"], shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
     T = Bt * S
     weights = si.llama_weights(hidden, ffn)
-    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan, fused=not args.unfused)
     x_host = si.normal((T, hidden), 0.0, 1.0, bf, 5, 0).pin_memory()
     out_host = torch.empty((T, hidden), dtype=bf).pin_memory()
     x_dev = torch.empty((T, hidden), dtype=bf, device="cuda")
@@ -161,7 +161,7 @@ def run_gpu(args, shape):
             return
         import paper_2609_03905_b200.relations as R
         orig_exec, orig_rep = R.B.ja_execute, R.B.ja_repartition
-        names = iter(OP_NAMES[args.plan])
+        names = iter(blk.op_names())
 
         def wrap(fn):
             def inner(*a, **k):
@@ -272,13 +272,14 @@ def run_gpu(args, shape):
     for name, s, e in events:
         per_op.setdefault(name, []).append(s.elapsed_time(e))
     ops = {k: sum(v) / len(v) for k, v in per_op.items()}
-    gemm_flops = {"q_proj": 2.0 * T * hidden * hidden, "k_proj": 2.0 * T * hidden * hidden, "v_proj": 2.0 * T * hidden * hidden,
-                  "o_proj": 2.0 * T * hidden * hidden, "w1_proj": 2.0 * T * hidden * ffn, "w3_proj": 2.0 * T * hidden * ffn,
-                  "w2_proj": 2.0 * T * hidden * ffn}
+    fl_h, fl_f = 2.0 * T * hidden * hidden, 2.0 * T * hidden * ffn
+    gemm_flops_all = {"q_proj": fl_h, "k_proj": fl_h, "v_proj": fl_h, "o_proj": fl_h, "w1_proj": fl_f, "w3_proj": fl_f, "w2_proj": fl_f,
+                      "q_proj_rope": fl_h, "k_proj_rope": fl_h, "o_proj_add": fl_h, "w13_swiglu": 2 * fl_f, "w2_proj_add": fl_f}
+    gemm_flops = {k: v for k, v in gemm_flops_all.items() if k in ops}
     gemm_ms = sum(ops[k] for k in gemm_flops)
     peaks = measured_peaks()
     achieved = sum(gemm_flops.values()) / (gemm_ms * 1e-3) / 1e12
-    roof = {"bound": "tensor", "kernel": "gemm_tc_kernel (7 launches per step)", "achieved": achieved,
+    roof = {"bound": "tensor", "kernel": f"gemm_tc_kernel ({len(gemm_flops)} launches per step)", "achieved": achieved,
             "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"],
             "frac_of_burst_peak": achieved / peaks["bf16"], "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
             "traffic": None, "share_of_step": gemm_ms / ms_step}
@@ -292,7 +293,8 @@ def run_gpu(args, shape):
     attn_fl = 4.0 * T * S * hidden / 2
     detail = {"ops_ms": ops, "memory_bound_ops": hbm,
               "attention": {"ms": ops["attention"], "TFLOPs": attn_fl / (ops["attention"] * 1e-3) / 1e12},
-              "gemm_TFLOPs": {k: gemm_flops[k] / (ops[k] * 1e-3) / 1e12 for k in gemm_flops}}
+              "gemm_TFLOPs": {k: gemm_flops[k] / (ops[k] * 1e-3) / 1e12 for k in gemm_flops},
+              "fused_chains": {"rope": blk.fuse_rope, "residual_add": blk.fuse_add, "swiglu": blk.fuse_swiglu}}
 
     if rank != 0:
         return
@@ -307,7 +309,7 @@ def run_gpu(args, shape):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"LLaMA-{args.shape} block forward as chained join-aggs, plan '{args.plan}' "
-                               f"({blk.n_relayouts} ja_repartition relayouts per step)", **shape,
+                               f"({blk.n_relayouts} ja_repartition relayouts per step; fused chains: {'on' if not args.unfused else 'off'})", **shape,
                    "l2": "working set per step (weights 405 MB + activations) exceeds the 126 MB L2; no flush needed",
                    "replicas": "independent replica per GPU (path does not shard)" if world > 1 else "single GPU"},
         "clocks": clocks, "gpu_launches": launches,
@@ -420,15 +422,6 @@ def run_case(args):
                       "peaks": peaks, "kernels": res}))
 
 
-OP_NAMES = {
-    "seq": ["rmsnorm_1", "q_proj", "k_proj", "v_proj", "rope_q", "rope_k", "repartition_q", "repartition_k", "repartition_v",
-            "attention", "repartition_att", "o_proj", "residual_1", "rmsnorm_2", "w1_proj", "w3_proj", "silu_mul", "w2_proj",
-            "residual_2"],
-    "head": ["repartition_x", "rmsnorm_1", "q_proj", "k_proj", "v_proj", "rope_q", "rope_k", "attention", "o_proj", "residual_1",
-             "rmsnorm_2", "w1_proj", "w3_proj", "silu_mul", "w2_proj", "residual_2", "repartition_out"],
-}
-
-
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -439,6 +432,7 @@ def main():
     ap.add_argument("--impl", choices=["ja", "reference"], default="ja")
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
     ap.add_argument("--case", choices=["block", "cfg2", "cfg3", "cfg4"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation")
     args = ap.parse_args()

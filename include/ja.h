@@ -78,7 +78,11 @@ typedef enum {
     JA_FN_ATTENTION = 9,   /* per (q-block,k-block) tuple: scale*Q K^T, causal band, partial (O~,m,l);
                               with JA_AGG_ONLINE_SOFTMAX, then O = O~/l                  [scale, causal]  */
     JA_FN_RMSNORM = 10,    /* fused chain SQUARE/SUM -> RMS_SCALE over the last index              [eps]  */
-    JA_FN_SOFTMAX = 11     /* fused chain IDENT/MAX -> EXP_SUB/SUM -> EXP_SUB_DIV over the last index     */
+    JA_FN_SOFTMAX = 11,    /* fused chain IDENT/MAX -> EXP_SUB/SUM -> EXP_SUB_DIV over the last index     */
+    JA_FN_MATMUL_ADD = 12, /* fused chain MUL/SUM -> ADD:        "ij,jk,ik->ik"   C = A B + R                   */
+    JA_FN_MATMUL_ROPE = 13,/* fused chain MUL/SUM -> ROPE:       "ij,jk->ik"      rows are tokens of sequences of
+                              seq_len rows, columns are heads of head_dim cells  [theta, seq_len, head_dim]     */
+    JA_FN_SWIGLU_UP = 14   /* fused chain 2 x MUL/SUM -> SILU_MUL: "ij,jk,jk->ik" silu(A B) * (A B')            */
 } ja_fn_t;
 
 typedef struct ja_spec ja_spec_t;
@@ -140,6 +144,9 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  * Supported forms (letters are free; shapes of the signature matter):
  *   "ij,jk->ik"            MUL / SUM        bf16 or f32 operands, f32 accumulate (tensor cores for bf16 on
  *                                            uniform 16-byte-aligned blocks, plain ALUs otherwise)
+ *   "ij,jk,ik->ik"         MATMUL_ADD / SUM   } fused chains: the accumulator of the contraction goes through the
+ *   "ij,jk->ik"            MATMUL_ROPE / SUM  } next join-agg before its single rounding and store; bf16 relations
+ *   "ij,jk,jk->ik"         SWIGLU_UP / SUM    } on uniform blocks only (JA_ERR_UNSUPPORTED otherwise: run the chain)
  *   "X,X->X", X any rank   ADD | SILU_MUL / NONE          key-aligned join
  *   "Rj->R"                SQUARE/SUM, IDENT/MAX          R = leading letters; f32 statistics output
  *   "Rj,R->R"              EXP_SUB / SUM

@@ -21,7 +21,7 @@ STATUS = {0: "JA_OK", 1: "JA_ERR_INVALID_ARG", 2: "JA_ERR_PARSE", 3: "JA_ERR_SHA
 JA_F32, JA_BF16 = 0, 1
 AGG = {"none": 0, "sum": 1, "max": 2, "online_softmax": 3}
 FN = {"mul": 0, "ident": 1, "square": 2, "add": 3, "silu_mul": 4, "rms_scale": 5, "exp_sub": 6, "exp_sub_div": 7,
-      "rope": 8, "attention": 9, "rmsnorm": 10, "softmax": 11}
+      "rope": 8, "attention": 9, "rmsnorm": 10, "softmax": 11, "matmul_add": 12, "matmul_rope": 13, "swiglu_up": 14}
 
 
 class JaError(RuntimeError):

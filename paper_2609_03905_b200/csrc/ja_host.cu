@@ -236,7 +236,7 @@ extern "C" ja_status_t ja_spec_create(const char* einsum, const ja_index_part_t*
     *out = nullptr;
     if (!einsum || !parts || n_parts < 1) return ja_fail(JA_ERR_INVALID_ARG, "einsum / parts missing");
     if (accum_dtype != JA_F32) return ja_fail(JA_ERR_DTYPE, "accumulation dtype must be JA_F32");
-    if ((int)fn < 0 || (int)fn > (int)JA_FN_SOFTMAX) return ja_fail(JA_ERR_INVALID_ARG, "unknown fn %d", (int)fn);
+    if ((int)fn < 0 || (int)fn > (int)JA_FN_SWIGLU_UP) return ja_fail(JA_ERR_INVALID_ARG, "unknown fn %d", (int)fn);
     if ((int)agg < 0 || (int)agg > (int)JA_AGG_ONLINE_SOFTMAX) return ja_fail(JA_ERR_INVALID_ARG, "unknown agg %d", (int)agg);
     if (n_fn_params < 0 || (n_fn_params > 0 && !fn_params)) return ja_fail(JA_ERR_INVALID_ARG, "fn_params missing");
 
@@ -646,13 +646,61 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         if (A->dtype == JA_BF16) {
             if (!plan->gemm_checked) {
                 bool ok = false;
-                if ((st = ja_gemm_tc_plan(A, B, out, &plan->gemm, &ok)) != JA_OK) return st;
+                if ((st = ja_gemm_tc_plan(A, B, out, nullptr, &plan->gemm, &ok)) != JA_OK) return st;
                 if (!ok) plan->gemm.reset();
                 plan->gemm_checked = true;
             }
             if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
         }
         return ja_launch_matmul_simt(ja_view(A), ja_view(B), ja_view(out), A->dtype, stream);
+    }
+
+    // ---- fused chains on the tensor-core matmul -------------------------------------------------------------------
+    if ((fn == JA_FN_MATMUL_ADD || fn == JA_FN_MATMUL_ROPE || fn == JA_FN_SWIGLU_UP) && agg == JA_AGG_SUM && n_in >= 2 &&
+        in[0].size() == 2 && in[1].size() == 2 && o.size() == 2 && in[0][1] == in[1][0] && o[0] == in[0][0] && o[1] == in[1][1] &&
+        in[0][0] != in[1][1]) {
+        const ja_relation *A = inputs[0], *B = inputs[1];
+        for (int k = 0; k < n_in; ++k)
+            if (inputs[k]->dtype != JA_BF16) return ja_fail(JA_ERR_UNSUPPORTED, "fused matmul chains need bf16 relations");
+        if (out->dtype != JA_BF16) return ja_fail(JA_ERR_UNSUPPORTED, "fused matmul chains need bf16 relations");
+        GemmEpilogue ep;
+        memset(&ep, 0, sizeof ep);
+        if (fn == JA_FN_MATMUL_ADD) {
+            if (n_in != 3 || in[2] != o) return ja_fail(JA_ERR_SHAPE, "MATMUL_ADD needs \"ij,jk,ik->ik\"");
+            ep.epi = 1;
+            ep.addend = inputs[2];
+        } else if (fn == JA_FN_SWIGLU_UP) {
+            if (n_in != 3 || in[2] != in[1]) return ja_fail(JA_ERR_SHAPE, "SWIGLU_UP needs \"ij,jk,jk->ik\"");
+            ep.epi = 3;
+            ep.B2 = inputs[2];
+        } else {
+            if (n_in != 2 || spec->params.size() < 3) return ja_fail(JA_ERR_INVALID_ARG, "MATMUL_ROPE needs \"ij,jk->ik\" and [theta, seq_len, head_dim]");
+            const double theta = spec->params[0];
+            const int64_t S = (int64_t)spec->params[1], D = (int64_t)spec->params[2];
+            if (S < 1 || D < 2 || D % 2 || A->extent[0] % S || B->extent[1] % D) return ja_fail(JA_ERR_SHAPE, "MATMUL_ROPE: rows must be whole sequences and columns whole heads");
+            if (!plan->rope_table) {
+                std::vector<float2> tab((size_t)S * (D / 2));
+                for (int64_t s = 0; s < S; ++s)
+                    for (int64_t pp = 0; pp < D / 2; ++pp) {
+                        double phi = (double)s * std::pow(theta, -2.0 * (double)pp / (double)D);
+                        tab[s * (D / 2) + pp] = make_float2((float)std::cos(phi), (float)std::sin(phi));
+                    }
+                JA_CUDA(cudaMalloc((void**)&plan->rope_table, tab.size() * sizeof(float2)));
+                JA_CUDA(cudaMemcpy(plan->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice));
+            }
+            ep.epi = 2;
+            ep.rope_table = plan->rope_table;
+            ep.rope_S = (int)S;
+            ep.rope_D = (int)D;
+        }
+        if (!plan->gemm_checked) {
+            bool ok = false;
+            if ((st = ja_gemm_tc_plan(A, B, out, &ep, &plan->gemm, &ok)) != JA_OK) return st;
+            if (!ok) plan->gemm.reset();
+            plan->gemm_checked = true;
+        }
+        if (!plan->gemm) return ja_fail(JA_ERR_UNSUPPORTED, "this tiling cannot run the fused matmul chain: execute the join-aggs one by one");
+        return ja_launch_gemm_tc(*plan->gemm, stream);
     }
 
     // ---- key-aligned maps "X,X->X" ----------------------------------------------------------------------

@@ -115,7 +115,17 @@ ja_status_t ja_launch_repartition(const char* src, char* dst, const CopySlab* d_
 
 // tcgen05 / TMEM / TMA matmul join-agg for bf16 relations with uniform blocks.
 struct GemmTcPlan;
-ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C,
+// Fused epilogue of the matmul join-agg: the next join-agg of a chain applied to the accumulator before its single store.
+//   epi 0 none; 1 ADD with `addend` (tiled like the output); 2 ROPE (rotation table, position = row % rope_S, rotated
+//   extent rope_D); 3 SWIGLU: silu(A B) * (A B2), B2 tiled like B.
+struct GemmEpilogue {
+    int epi;
+    const ja_relation* addend;
+    const ja_relation* B2;
+    const float2* rope_table;
+    int rope_S, rope_D;
+};
+ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C, const GemmEpilogue* ep,
                             std::shared_ptr<GemmTcPlan>* out, bool* eligible);
 ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st);
 

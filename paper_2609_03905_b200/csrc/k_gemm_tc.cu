@@ -60,7 +60,14 @@ struct GemmParams {
     int32_t tiles_per_mblk;    // >= 1 when row tiles never leave a block, 0 when tiles are cut from global rows
     int32_t tiles_per_nblk;    // >= 1 when tiles stay inside one column block, 0 when tiles span blocks
     int32_t group_m;           // row tiles per rasterisation band
+    // fused epilogue (a join-agg chain executed in one pass, the intermediate never stored)
+    int32_t epi;               // EPI_*
+    int32_t bn_tile;           // output columns per tile: 256, or 128 for EPI_SWIGLU (two 128-column products per tile)
+    const char* r_base;        // EPI_ADD: payload of the relation added to the product (tiled exactly like the output)
+    const float2* rope_table;  // EPI_ROPE: (cos, sin)[position][pair]
+    int32_t rope_S, rope_D;    // EPI_ROPE: positions per sequence (row % rope_S), rotated extent (column % rope_D)
 };
+enum { EPI_NONE = 0, EPI_ADD = 1, EPI_ROPE = 2, EPI_SWIGLU = 3 };
 
 // What one CTA does for one tile: its own 128 rows, and (CG 2) its own half of the tile's columns as B operand.
 struct TileCoord {
@@ -93,21 +100,22 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int 
     }
     if (p.tiles_per_nblk > 0) {
         tc.nb = nt / p.tiles_per_nblk;
-        tc.c0 = (nt % p.tiles_per_nblk) * BN;
-        tc.width = min(BN, p.bn - tc.c0);
+        tc.c0 = (nt % p.tiles_per_nblk) * p.bn_tile;
+        tc.width = min(p.bn_tile, p.bn - tc.c0);
         tc.n_g0 = tc.nb * p.bn + tc.c0;
     } else {
-        tc.n_g0 = nt * BN;
+        tc.n_g0 = nt * p.bn_tile;
         tc.nb = tc.n_g0 / p.bn;
         tc.c0 = tc.n_g0 % p.bn;
-        tc.width = min(BN, p.N - tc.n_g0);
+        tc.width = min(p.bn_tile, p.N - tc.n_g0);
     }
     return tc;
 }
 
 template <int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
     constexpr int STAGES = Cfg<CG>::STAGES, BK = Cfg<CG>::BK;
     constexpr int A_STAGE_BYTES = Cfg<CG>::A_STAGE_BYTES, A_HALF_BYTES = Cfg<CG>::A_HALF_BYTES;
     constexpr int B_STAGE_BYTES = Cfg<CG>::B_STAGE_BYTES, B_CHUNK_BYTES = Cfg<CG>::B_CHUNK_BYTES;
@@ -170,7 +178,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             for (int t = first_tile; t < total_tiles && ok; t += tile_step) {
                 const TileCoord tc = tile_coord<CG>(p, t, cta_rank);
-                const int n_mma = (tc.width + 15) / 16 * 16;
+                // EPI_SWIGLU: the MMA tile is [128 columns of x W1 | the same 128 columns of x W3]
+                const int n_mma = p.epi == EPI_SWIGLU ? 2 * tc.width : (tc.width + 15) / 16 * 16;
                 const int my_cols = n_mma / CG;                    // B columns this CTA stages
                 const int my_c0 = cta_rank * my_cols;              // their offset inside the tile
                 const int nchunks = (my_cols + 63) / 64;
@@ -191,10 +200,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                                 kc * BK + kh * 64, tc.r0, jb, tc.mb + bx);
                         // B: one box of BK k-rows x 64 columns per 64-column chunk
                         for (int c = 0; c < nchunks; ++c) {
+                            int mc = my_c0 + 64 * c;               // column of the MMA tile this box starts at
+                            const CUtensorMap* tb = &tmB;
+                            if (p.epi == EPI_SWIGLU && mc >= p.bn_tile) { tb = &tmB2; mc -= p.bn_tile; }
                             int nb, cin;
-                            if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + my_c0 + 64 * c; }
-                            else { int g = tc.n_g0 + my_c0 + 64 * c; nb = g / p.bn; cin = g % p.bn; }
-                            tma_load_4d<CG>(sB + stage * B_STAGE_BYTES + c * B_CHUNK_BYTES, &tmB, fb, cin, kc * BK, nb, jb);
+                            if (p.tiles_per_nblk > 0) { nb = tc.nb; cin = tc.c0 + mc; }
+                            else { int g = tc.n_g0 + mc; nb = g / p.bn; cin = g % p.bn; }
+                            tma_load_4d<CG>(sB + stage * B_STAGE_BYTES + c * B_CHUNK_BYTES, tb, fb, cin, kc * BK, nb, jb);
                         }
                         if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
@@ -222,7 +234,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int t = first_tile; t < total_tiles && ok; t += tile_step, ++it) {
                 const TileCoord tc = tile_coord<CG>(p, t, 0);
                 const int acc = it & 1;
-                const uint32_t n_mma = (uint32_t)((tc.width + 15) / 16 * 16);
+                const uint32_t n_mma = p.epi == EPI_SWIGLU ? (uint32_t)(2 * tc.width) : (uint32_t)((tc.width + 15) / 16 * 16);
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((n_mma >> 3) << 17) |
                                        ((uint32_t)((BM * CG) >> 4) << 24);
                 if (!mbar_wait(tempty_bar(acc), acc_phase[acc] ^ 1, abort_flag, p.status)) { ok = false; break; }
@@ -275,20 +287,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int ch = 0; ch * 32 < tc.width; ++ch) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + ch * 32, v);
-                tmem_ld_wait();
+                if (p.epi == EPI_SWIGLU) {   // silu(x W1) * (x W3): the W3 product sits 128 columns to the right
+                    uint32_t w[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + p.bn_tile + ch * 32, w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float a = __uint_as_float(v[i]);
+                        v[i] = __float_as_uint(a / (1.f + __expf(-a)) * __uint_as_float(w[i]));
+                    }
+                } else {
+                    tmem_ld_wait();
+                }
                 if (row_ok) {
                     const int gcol = tc.n_g0 + ch * 32;
                     const int kb = gcol / p.bn, cin = gcol % p.bn;
-                    char* dst = p.c_base + p.c_blk_off[(int64_t)ib * p.nbn + kb] + ((int64_t)iin * p.bn + cin) * 2;
+                    const int64_t off = p.c_blk_off[(int64_t)ib * p.nbn + kb] + ((int64_t)iin * p.bn + cin) * 2;
+                    char* dst = p.c_base + off;
                     const int valid = min(32, tc.width - ch * 32);  // multiple of 8
+                    if (p.epi == EPI_ROPE) {
+                        // rotate pairs (2p, 2p+1) by the angle of (position, pair): position = row inside its sequence
+                        const float2* tab = p.rope_table + ((int64_t)(grow % p.rope_S) * p.rope_D + gcol % p.rope_D) / 2;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            const float2 cs = tab[i / 2];
+                            const float x0 = __uint_as_float(v[i]), x1 = __uint_as_float(v[i + 1]);
+                            v[i] = __float_as_uint(x0 * cs.x - x1 * cs.y);
+                            v[i + 1] = __float_as_uint(x0 * cs.y + x1 * cs.x);
+                        }
+                    }
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         if (g * 8 < valid) {
+                            float f[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[g * 8 + e]);
+                            if (p.epi == EPI_ADD) {   // key-aligned join with the addend relation: same block, same cell
+                                const uint4 rv = *reinterpret_cast<const uint4*>(p.r_base + off + g * 16);
+                                const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float2 rf = __bfloat1622float2(pr[e]);
+                                    f[2 * e] += rf.x;
+                                    f[2 * e + 1] += rf.y;
+                                }
+                            }
                             uint4 o;
                             __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                po[e] = __floats2bfloat162_rn(__uint_as_float(v[g * 8 + 2 * e]), __uint_as_float(v[g * 8 + 2 * e + 1]));
+                            for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
                             *reinterpret_cast<uint4*>(dst + g * 16) = o;
                         }
                     }
@@ -334,16 +381,20 @@ ja_status_t encode_blocked_2d(const ja_relation* r, int box_inner, int box_rows,
 }  // namespace
 
 struct GemmTcPlan {
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmB2;
     GemmParams p;
     int grid;
     int cg;   // CTAs per tile: 1 or 2
 };
 
-ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C,
+ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C, const GemmEpilogue* ep,
                             std::shared_ptr<GemmTcPlan>* out, bool* eligible) {
     *eligible = false;
     if (!A->equal_blocks || !B->equal_blocks || !C->equal_blocks) return JA_OK;
+    const int epi = ep ? ep->epi : 0;
+    const int bn_tile = epi == EPI_SWIGLU ? 128 : BN;
+    if (epi == EPI_SWIGLU && (B->bs[1] % 128 != 0 || !ep->B2 || !ep->B2->equal_blocks)) return JA_OK;
+    if (epi == EPI_ROPE && (ep->rope_D % 32 != 0 || B->bs[1] % 32 != 0)) return JA_OK;
     const int64_t bm = A->bs[0], bk = A->bs[1], bn = B->bs[1];
     // TMA needs 16-byte row pitches; boxes are 64 elements wide; A boxes hold min(bm,128) rows
     if (bk % 8 || bn % 8 || bk < 64 || bn < 64) return JA_OK;
@@ -359,8 +410,14 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     p.nbm = A->nblk[0]; p.nbk = A->nblk[1]; p.nbn = B->nblk[1];
     p.M = (int)A->extent[0]; p.N = (int)B->extent[1];
     p.a_box_rows = (int)std::min<int64_t>(bm, 128);
-    if (bn % 64 == 0 && bn < BN && p.nbn > 1) { p.tiles_per_nblk = 0; p.n_tiles = (p.N + BN - 1) / BN; }
-    else { p.tiles_per_nblk = (int)((bn + BN - 1) / BN); p.n_tiles = p.tiles_per_nblk * p.nbn; }
+    p.epi = epi;
+    p.bn_tile = bn_tile;
+    p.r_base = (epi == EPI_ADD) ? (const char*)ep->addend->base : nullptr;
+    p.rope_table = (epi == EPI_ROPE) ? ep->rope_table : nullptr;
+    p.rope_S = ep ? ep->rope_S : 1;
+    p.rope_D = ep ? ep->rope_D : 2;
+    if (bn % 64 == 0 && bn < bn_tile && p.nbn > 1) { p.tiles_per_nblk = 0; p.n_tiles = (p.N + bn_tile - 1) / bn_tile; }
+    else { p.tiles_per_nblk = (int)((bn + bn_tile - 1) / bn_tile); p.n_tiles = p.tiles_per_nblk * p.nbn; }
     // Two-CTA form: 256-row tiles cut from global rows; needs 128-row halves that never straddle a block and, when
     // tiles span column blocks, column tails whose halves still start on a 64-column box boundary.
     const char* gm = getenv("JA_GEMM_GROUP_M");
@@ -368,7 +425,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     if (p.group_m < 1) p.group_m = 1;
     const char* force = getenv("JA_GEMM_CTA_GROUP");
     bool two = (bm % 128 == 0 || 128 % bm == 0) && p.M >= 256 && bk >= Cfg<2>::BK;
-    if (p.tiles_per_nblk == 0 && (p.N % BN) % 128 != 0) two = false;
+    if (p.tiles_per_nblk == 0 && (p.N % bn_tile) % (bn_tile / 2) != 0) two = false;
     if (force && force[0] == '1') two = false;
     plan->cg = two ? 2 : 1;
     if (two || bm < 128) { p.tiles_per_mblk = 0; p.m_tiles = (p.M + BM * plan->cg - 1) / (BM * plan->cg); }
@@ -376,6 +433,8 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     ja_status_t st;
     if ((st = encode_blocked_2d(A, 64, p.a_box_rows, &plan->tmA)) != JA_OK) return st;
     if ((st = encode_blocked_2d(B, 64, two ? Cfg<2>::BK : Cfg<1>::BK, &plan->tmB)) != JA_OK) return st;
+    plan->tmB2 = plan->tmB;
+    if (epi == EPI_SWIGLU && (st = encode_blocked_2d(ep->B2, 64, two ? Cfg<2>::BK : Cfg<1>::BK, &plan->tmB2)) != JA_OK) return st;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -404,9 +463,9 @@ ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.p));
+        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.tmB2, plan.p));
     } else {
-        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.p);
+        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, plan.p);
         JA_CUDA(cudaGetLastError());
     }
     ja_count_launch();

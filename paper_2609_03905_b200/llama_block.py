@@ -27,8 +27,9 @@ from .relations import Relation, Spec, equal_splits as ES, from_dense, repartiti
 class LlamaBlock:
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
                  theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8,
-                 ffn_blocks: int | None = None):
+                 ffn_blocks: int | None = None, fused: bool = True):
         assert plan in ("seq", "head")
+        self.fused = fused
         assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
         assert seq % token_block == 0
         self.plan, self.B, self.S, self.hidden, self.H, self.ffn = plan, batch, seq, hidden, n_heads, ffn
@@ -104,11 +105,45 @@ class LlamaBlock:
         self.s_silu = Spec("ij,ij->ij", {"i": t_sp, "j": ffn_c}, "silu_mul", (), "none")
         self.s_down = mm(ffn_c, act_c)
         self.n_relayouts = 4 if plan == "seq" else 2
+        # fused chains: the projection's accumulator goes through RoPE / the residual ADD / SILU_MUL before its store
+        # (a fused form that the tiling cannot run -- JA_ERR_UNSUPPORTED -- falls back to its chain, once and for all)
+        self.fuse_rope = self.fuse_add = self.fuse_swiglu = fused
+        if fused:
+            self.s_qk_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": qkv_c}, "matmul_rope", (theta, seq, D), "sum")
+            self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": act_c, "k": act_c}, "matmul_add", (), "sum")
+            self.s_up_swiglu = Spec("ij,jk,jk->ik", {"i": t_sp, "j": act_c, "k": ffn_c}, "swiglu_up", (), "sum")
+            self.s_down_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": ffn_c, "k": act_c}, "matmul_add", (), "sum")
 
     # flop count of one forward (dense contractions only; causal attention counted at half the square)
     def flops(self) -> float:
         T, d, f, S = self.T, self.hidden, self.ffn, self.S
         return 2.0 * T * d * d * 4 + 2.0 * T * d * f * 3 + 4.0 * T * S * d / 2
+
+    @staticmethod
+    def _fused(spec: Spec, inputs, output: Relation, stream) -> bool:
+        """Run a fused chain; False if libja has no fused kernel for this tiling (nothing was enqueued)."""
+        try:
+            spec.execute(inputs, output, stream)
+            return True
+        except B.JaError as e:
+            if e.status_name != "JA_ERR_UNSUPPORTED":
+                raise
+            return False
+
+    def op_names(self):
+        """Names of the libja calls of one forward(), in order (for per-op timing)."""
+        n = ["repartition_x"] if self.plan == "head" else []
+        n += ["rmsnorm_1"]
+        n += ["q_proj_rope", "k_proj_rope", "v_proj"] if self.fuse_rope else ["q_proj", "k_proj", "v_proj", "rope_q", "rope_k"]
+        n += ["repartition_q", "repartition_k", "repartition_v"] if self.plan == "seq" else []
+        n += ["attention"]
+        n += ["repartition_att"] if self.plan == "seq" else []
+        n += ["o_proj_add"] if self.fuse_add else ["o_proj", "residual_1"]
+        n += ["rmsnorm_2"]
+        n += ["w13_swiglu"] if self.fuse_swiglu else ["w1_proj", "w3_proj", "silu_mul"]
+        n += ["w2_proj_add"] if self.fuse_add else ["w2_proj", "residual_2"]
+        n += ["repartition_out"] if self.plan == "head" else []
+        return n
 
     def forward(self, stream: int | None = None) -> Relation:
         """Enqueue the whole chain on the current stream; returns the output relation (tiled like x)."""
@@ -116,11 +151,17 @@ class LlamaBlock:
         if p == "head":
             repartition(self.x, self.x_p, stream)
         self.s_norm.execute([self.x_p, self.g1], self.n1, stream)
-        self.s_qkv.execute([self.n1, self.wq], self.q, stream)
-        self.s_qkv.execute([self.n1, self.wk], self.k, stream)
-        self.s_qkv.execute([self.n1, self.wv], self.v, stream)
-        self.s_rope.execute([self.q4], self.q4r, stream)
-        self.s_rope.execute([self.k4], self.k4r, stream)
+        if self.fuse_rope and not self._fused(self.s_qk_rope, [self.n1, self.wq], self.q_r, stream):
+            self.fuse_rope = False
+        if self.fuse_rope:
+            self.s_qk_rope.execute([self.n1, self.wk], self.k_r, stream)
+            self.s_qkv.execute([self.n1, self.wv], self.v, stream)
+        else:
+            self.s_qkv.execute([self.n1, self.wq], self.q, stream)
+            self.s_qkv.execute([self.n1, self.wk], self.k, stream)
+            self.s_qkv.execute([self.n1, self.wv], self.v, stream)
+            self.s_rope.execute([self.q4], self.q4r, stream)
+            self.s_rope.execute([self.k4], self.k4r, stream)
         if p == "seq":
             repartition(self.q_r, self.q_h, stream)
             repartition(self.k_r, self.k_h, stream)
@@ -128,14 +169,23 @@ class LlamaBlock:
         self.s_attn.execute([self.qa, self.ka, self.va], self.oa, stream)
         if p == "seq":
             repartition(self.att_h, self.att, stream)
-        self.s_wo.execute([self.att, self.wo], self.o, stream)
-        self.s_add.execute([self.x_p, self.o], self.h, stream)
+        if self.fuse_add and not self._fused(self.s_wo_add, [self.att, self.wo, self.x_p], self.h, stream):
+            self.fuse_add = False
+        if not self.fuse_add:
+            self.s_wo.execute([self.att, self.wo], self.o, stream)
+            self.s_add.execute([self.x_p, self.o], self.h, stream)
         self.s_norm.execute([self.h, self.g2], self.n2, stream)
-        self.s_up.execute([self.n2, self.w1], self.a, stream)
-        self.s_up.execute([self.n2, self.w3], self.b, stream)
-        self.s_silu.execute([self.a, self.b], self.hh, stream)
-        self.s_down.execute([self.hh, self.w2], self.y, stream)
-        self.s_add.execute([self.h, self.y], self.out_p, stream)
+        if self.fuse_swiglu and not self._fused(self.s_up_swiglu, [self.n2, self.w1, self.w3], self.hh, stream):
+            self.fuse_swiglu = False
+        if not self.fuse_swiglu:
+            self.s_up.execute([self.n2, self.w1], self.a, stream)
+            self.s_up.execute([self.n2, self.w3], self.b, stream)
+            self.s_silu.execute([self.a, self.b], self.hh, stream)
+        if self.fuse_add:
+            self.s_down_add.execute([self.hh, self.w2, self.h], self.out_p, stream)
+        else:
+            self.s_down.execute([self.hh, self.w2], self.y, stream)
+            self.s_add.execute([self.h, self.y], self.out_p, stream)
         if p == "head":
             repartition(self.out_p, self.out, stream)
         return self.out

@@ -113,20 +113,22 @@ def _block_case(shape_name, Bt, S, hidden, heads, ffn, prefix, seq_id):
     w = si.llama_weights(hidden, ffn)
     x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 0)
     outs = {}
-    for plan in ("seq", "head"):
-        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan)
+    for plan, fused in (("seq", True), ("head", True), ("seq", False)):
+        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, fused=fused)
         ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
-        outs[plan] = download(blk.forward())
+        outs[plan if fused else "seq_unfused"] = download(blk.forward())
         check_status()
+        assert blk.fuse_swiglu == fused and blk.fuse_rope == fused and blk.fuse_add == fused
         del blk
         torch.cuda.empty_cache()
-    # the two decompositions of the same block agree with each other on the whole output ...
+    # the two decompositions of the same block agree with each other on the whole output, fused chains or not ...
     assert relfro(outs["head"], outs["seq"]) <= TOL[BF]
+    assert relfro(outs["seq_unfused"], outs["seq"]) <= TOL[BF]
     # ... and with the oracle on sampled token rows of one sequence (causal: a prefix is self-contained)
     rows = np.unique(np.concatenate([[0, 1, 127, 128, prefix - 1], np.linspace(0, prefix - 1, 8).astype(int)]))
     xs = si.to_f64(x[seq_id * S: seq_id * S + prefix])
     ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows)["out"]
-    for plan in ("seq", "head"):
+    for plan in ("seq", "head", "seq_unfused"):
         assert relfro(outs[plan][seq_id * S + rows], ref) <= TOL[BF], (shape_name, plan)
 
 
@@ -147,12 +149,16 @@ def test_small_block_every_intermediate():
     w64 = {k: si.to_f64(v) for k, v in w.items()}
     refs = [operators.llama_block(si.to_f64(x[b * S:(b + 1) * S]), w64, heads) for b in range(Bt)]
     cat = lambda name: np.concatenate([r[name].reshape(S, -1) for r in refs])
-    for plan in ("seq", "head"):
-        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4)
+    for plan, fused, ffn_blocks in (("seq", False, 4), ("head", False, 4), ("seq", True, 11), ("head", True, 11), ("seq", True, 4)):
+        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4, ffn_blocks=ffn_blocks, fused=fused)
         ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
         out = download(blk.forward())
         check_status()
-        for name, rel in (("n1", blk.n1), ("q", blk.q_r), ("k", blk.k_r), ("v", blk.v), ("att", blk.att), ("h", blk.h),
-                          ("n2", blk.n2), ("mlp", blk.y)):
-            assert relfro(download(rel), cat(name)) <= TOL[BF], (plan, name)
-        assert relfro(out, cat("out")) <= TOL[BF], plan
+        # 128-wide FFN blocks (1408 = 11 x 128) can run the fused SwiGLU chain, 352-wide ones fall back to the chain
+        assert blk.fuse_swiglu == (fused and ffn_blocks == 11) and blk.fuse_rope == fused and blk.fuse_add == fused
+        rels = [("n1", blk.n1), ("q", blk.q_r), ("k", blk.k_r), ("v", blk.v), ("att", blk.att), ("h", blk.h), ("n2", blk.n2)]
+        if not fused:
+            rels.append(("mlp", blk.y))
+        for name, rel in rels:
+            assert relfro(download(rel), cat(name)) <= TOL[BF], (plan, fused, name)
+        assert relfro(out, cat("out")) <= TOL[BF], (plan, fused)

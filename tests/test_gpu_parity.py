@@ -235,3 +235,51 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
     assert np.abs(got - ref).max() <= 0.05
     if causal:
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
+
+
+# ---------------------------------------------------------------------------------------------------
+# fused chains on the tensor-core matmul: the accumulator goes through the next join-agg before its one store
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("cta_group", ["2", "1"])
+@pytest.mark.parametrize("M,J,N,gi,gj,gk", [(512, 256, 512, 4, 2, 2), (256, 384, 1024, 2, 3, 8), (512, 512, 256, 2, 1, 2)])
+def test_matmul_fused_chains(M, J, N, gi, gj, gk, cta_group, monkeypatch):
+    monkeypatch.setenv("JA_GEMM_CTA_GROUP", cta_group)
+    A = si.normal((M, J), 0.0, 1.0, BF, 2, 6)
+    W1 = si.normal((J, N), 0.0, 0.06, BF, 2, 7)
+    W3 = si.normal((J, N), 0.0, 0.06, BF, 2, 8)
+    R = si.normal((M, N), 0.0, 1.0, BF, 2, 9)
+    ti, tj, tk = ES(M, gi), ES(J, gj), ES(N, gk)
+    parts = {"i": ti, "j": tj, "k": tk}
+    rA, rW1, rW3, rR = upload(A, [ti, tj]), upload(W1, [tj, tk]), upload(W3, [tj, tk]), upload(R, [ti, tk])
+    a64 = core.matmul(si.to_f64(A), si.to_f64(W1))          # unrounded products: the fused forms store nothing in between
+    b64 = core.matmul(si.to_f64(A), si.to_f64(W3))
+    out = lambda: empty_like_tiling([M, N], [ti, tk], BF, fill=float("nan"))
+    # MUL/SUM -> ADD
+    rC = out()
+    ja.Spec("ij,jk,ik->ik", parts, "matmul_add", (), "sum").execute([rA, rW1, rR], rC)
+    assert relfro(download(rC), core.round_to(a64 + si.to_f64(R), "bf16")) <= 2e-3
+    # two MUL/SUM -> SILU_MUL
+    rC = out()
+    ja.Spec("ij,jk,jk->ik", parts, "swiglu_up", (), "sum").execute([rA, rW1, rW3], rC)
+    assert relfro(download(rC), operators.silu_mul(a64, b64, "bf16")) <= 3e-3
+    # MUL/SUM -> ROPE: rows are 128-token sequences, columns 128-wide heads
+    rC = out()
+    ja.Spec("ij,jk->ik", parts, "matmul_rope", (1e4, 128, 128), "sum").execute([rA, rW1], rC)
+    ref = operators.rope(a64.reshape(M // 128, 128, N // 128, 128), 1e4, "bf16").reshape(M, N)
+    assert relfro(download(rC), ref) <= 3e-3
+    check_status()
+
+
+def test_fused_chain_refused_when_the_tiling_cannot_run_it():
+    # 64-wide column blocks cannot hold the paired 128-column products of the fused SwiGLU chain: nothing is enqueued
+    M, J, N = 256, 128, 256
+    ti, tj, tk = ES(M, 2), ES(J, 1), ES(N, 4)
+    rA = empty_like_tiling([M, J], [ti, tj], BF, fill=1.0)
+    rW = empty_like_tiling([J, N], [tj, tk], BF, fill=1.0)
+    rW3 = empty_like_tiling([J, N], [tj, tk], BF, fill=1.0)
+    rC = empty_like_tiling([M, N], [ti, tk], BF, fill=0.0)
+    with pytest.raises(ja.JaError) as e:
+        ja.Spec("ij,jk,jk->ik", {"i": ti, "j": tj, "k": tk}, "swiglu_up", (), "sum").execute([rA, rW, rW3], rC)
+    assert e.value.status_name == "JA_ERR_UNSUPPORTED"
+    torch.cuda.synchronize()
+    assert float(rC.payload.abs().max()) == 0.0
