@@ -282,7 +282,14 @@ def run_gpu(args, shape):
     roof = {"bound": "tensor", "kernel": f"gemm_tc_kernel ({len(gemm_flops)} launches per step)", "achieved": achieved,
             "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"],
             "frac_of_burst_peak": achieved / peaks["bf16"], "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
-            "traffic": None, "share_of_step": gemm_ms / ms_step}
+            "traffic": None, "share_of_step": gemm_ms / ms_step,
+            "algorithmic_flops_per_launch": sum(gemm_flops.values()) / len(gemm_flops)}
+    # DRAM bytes per launch of this kernel (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches of one step)
+    # from the ncu capture summarised in profiles/gemm_tc_kernel_dram_traffic_llama7b_block.md; it holds for the workload it
+    # was taken on only
+    if args.shape == "7b" and args.plan == "seq" and not args.unfused:
+        roof["traffic"] = 1.037e9
+        roof["traffic_unit"] = "bytes per launch (ncu, 7b / seq / fused; operands once + output would be 0.456e9)"
     mem_bytes = {"rmsnorm_1": 4.0 * T * hidden, "rmsnorm_2": 4.0 * T * hidden, "rope_q": 4.0 * T * hidden, "rope_k": 4.0 * T * hidden,
                  "residual_1": 6.0 * T * hidden, "residual_2": 6.0 * T * hidden, "silu_mul": 6.0 * T * ffn}
     for k in ops:
