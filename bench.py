@@ -88,6 +88,19 @@ def run_reference(args, shape):
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+# ---- replicas: the path does not shard, so N GPUs run N independent replicas ------------------------------------------
+def replica_aggregate(ms_values, flops_per_replica_step, steps, world, device="cpu"):
+    """Whole-job throughput of `world` independent replicas: every rank contributes its device-timed milliseconds for
+    `steps` steps; the job time is the MAX over ranks; the job did world x steps x flops. Returns (ms maxima, TFLOP/s)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(ms_values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = t.tolist()
+    return ms, [world * flops_per_replica_step / (m / steps * 1e-3) / 1e12 for m in ms]
+
+
 # ---- GPU leg ---------------------------------------------------------------------------------------------------
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -258,14 +271,9 @@ def run_gpu(args, shape):
     ms_e2e = e0.elapsed_time(e1)
     assert torch.equal(out_hosts[0], out_hosts[1]), "end-to-end outputs of consecutive steps differ"
 
-    times = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = times.tolist()
     fl = block_flops(Bt, S, hidden, ffn)
+    (ms_total, ms_e2e), (value, e2e_val) = replica_aggregate([ms_total, ms_e2e], fl, args.steps, world, device="cuda")
     ms_step = ms_total / args.steps
-    value = world * fl / (ms_step * 1e-3) / 1e12
-    e2e_val = world * fl / (ms_e2e / args.steps * 1e-3) / 1e12
 
     # ---- per-op breakdown and the roofline of the dominant kernel -----------------------------------------------------
     per_op = {}
@@ -365,7 +373,15 @@ def run_case(args):
 
     res = {}
     reps = args.steps
-    if args.case == "cfg2":
+    if args.case == "cfg1":
+        for grid in ((4, 4, 4), (2, 8, 4)):
+            ti, tj, tk = (ES(256, g) for g in grid)
+            A, Bm, C = rel((256, 256), [ti, tj], f32), rel((256, 256), [tj, tk], f32), rel((256, 256), [ti, tk], f32)
+            sp = ja.Spec("ij,jk->ik", {"i": ti, "j": tj, "k": tk})
+            t = timeit(lambda r: sp.execute([A, Bm], C), reps, False)
+            res["matmul_f32_256_grid_%dx%dx%d" % grid] = {**t, "GFLOPs": 2.0 * 256 ** 3 / (t["ms_mean"] * 1e-3) / 1e9,
+                                                          "note": "plain fp32 ALUs; launch-latency bound at this size"}
+    elif args.case == "cfg2":
         T, d, f = 2048, 4096, 11008
         ti, td, tf = ES(T, 8), ES(d, 8), ES(f, 8)
         x, W1, W3, W2 = rel((T, d), [ti, td]), rel((d, f), [td, tf], std=0.02), rel((d, f), [td, tf], std=0.02), rel((f, d), [tf, td], std=0.02)
@@ -440,7 +456,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg2", "cfg3", "cfg4"], default="block",
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
