@@ -440,6 +440,24 @@ def run_case(args):
         fl = 4.0 * Bn * H * S * S * D / 2
         res["attention_causal"] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "TFLOPs_executed_blocks": fl * 136 / 128 / (t["ms_mean"] * 1e-3) / 1e12,
                                    "frac_of_burst_bf16_peak": fl / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"]}
+    elif args.case == "gqa":
+        # Example 3.10: 32 query heads on 8 key/value heads, sequence index 4096 holding sequences that end at 1024, 2560, 4096
+        Bn, S, Hq, Hkv, D, grp = 8, 4096, 32, 8, 128, 4
+        ends = [1024, 2560, 4096]
+        gs = list(range(Hkv + 1))
+        hs = [grp * v for v in gs]
+        fl_packed = 4.0 * Bn * Hq * D * sum((b - a) ** 2 for a, b in zip([0] + ends[:-1], ends)) / 2
+        for name, s_split, prm_ends, fl in (("gqa_packed_cut_at_ends", [0] + ends, ends, fl_packed),
+                                            ("gqa_packed_128_row_blocks", ES(S, S // 128), ends, fl_packed),
+                                            ("gqa_one_sequence", ES(S, S // 128), [], 4.0 * Bn * Hq * S * S * D / 2)):
+            q_sp, k_sp = [ES(Bn, Bn), s_split, hs, [0, D]], [ES(Bn, Bn), s_split, gs, [0, D]]
+            Q, O = rel((Bn, S, Hq, D), q_sp), rel((Bn, S, Hq, D), q_sp)
+            K, V = rel((Bn, S, Hkv, D), k_sp), rel((Bn, S, Hkv, D), k_sp)
+            parts = {"b": q_sp[0], "q": s_split, "h": hs, "d": [0, D], "k": s_split, "g": gs}
+            spec = ja.Spec("bqhd,bkgd,bkgd->bqhd", parts, "attention", (1.0 / D ** 0.5, 1.0) + tuple(map(float, prm_ends)), "online_softmax")
+            t = timeit(lambda r: spec.execute([Q, K, V], O), reps, True)
+            res[name] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "frac_of_burst_bf16_peak": fl / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"],
+                         "tuples": ja.ja_spec_num_tuples(spec.handle)[0]}
     assert ja.ja_stream_status(stream.cuda_stream) == 0
     print(json.dumps({"case": args.case, "reps": reps, "l2": "512 MiB flush buffer written before every timed launch",
                       "peaks": peaks, "kernels": res}))
@@ -456,8 +474,9 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4"], default="block",
-                    help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation")
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa"], default="block",
+                    help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "
+                         "gqa = grouped-query attention over packed sequences")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
     if args.case != "block":

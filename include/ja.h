@@ -76,7 +76,12 @@ typedef enum {
     JA_FN_ROPE = 8,        /* rotate pairs (2p,2p+1) of the last index by t*theta^(-2p/d), t = value of the
                               second index of "bshd"                                             [theta]  */
     JA_FN_ATTENTION = 9,   /* per (q-block,k-block) tuple: scale*Q K^T, causal band, partial (O~,m,l);
-                              with JA_AGG_ONLINE_SOFTMAX, then O = O~/l                  [scale, causal]  */
+                              with JA_AGG_ONLINE_SOFTMAX, then O = O~/l.   [scale, causal, end_1 .. end_n]
+                              Example 3.10: "bqhd,bkgd,bkgd->bqhd" is grouped-query attention, query head h joins
+                              key/value head h / (extent(h)/extent(g)) and the split of h must be the split of g
+                              scaled by that factor (else JA_ERR_TILING); end_1 < .. < end_n = extent(q), n <= 16,
+                              are the ends of sequences packed along q and k: every end must be a split point of
+                              q and of k (else JA_ERR_TILING) and only blocks of one sequence are joined          */
     JA_FN_RMSNORM = 10,    /* fused chain SQUARE/SUM -> RMS_SCALE over the last index              [eps]  */
     JA_FN_SOFTMAX = 11,    /* fused chain IDENT/MAX -> EXP_SUB/SUM -> EXP_SUB_DIV over the last index     */
     JA_FN_MATMUL_ADD = 12, /* fused chain MUL/SUM -> ADD:        "ij,jk,ik->ik"   C = A B + R                   */

@@ -43,10 +43,16 @@ def check_splits(extent: int, splits) -> None:
 class Spec:
     """The join-agg spec J for one interval decomposition (Definition 3.6 / Section 3.3)."""
 
-    def __init__(self, einsum: str, parts: dict, band=None):
+    def __init__(self, einsum: str, parts: dict, band=None, induced=None, segments=None):
         """band = (k_letter, q_letter): the selection k <= q lifted to blocks -- a cell of the interval grid is
         a function specification only if some key position of its k interval is <= some query position of its
-        q interval (attention with the key index split inside a sequence)."""
+        q interval (attention with the key index split inside a sequence).
+        induced = (h_letter, g_letter, group): h is not shardable by itself (Example 3.10, grouped-query attention):
+        its intervals are those of g scaled by `group`, and a function specification pairs interval m of g with
+        interval m of h only.
+        segments = (k_letter, q_letter, ends): packed sequences ending at `ends` (Example 3.10): attention never
+        crosses a sequence boundary, so a cell is a function specification only if its q and k intervals lie in
+        the same sequence; both indices may be split at sequence ends (and, in the extended form, inside)."""
         self.einsum = einsum
         self.ins, self.out, self.letters = core.parse_einsum(einsum)
         self.parts = {c: list(parts[c]) for c in self.letters}
@@ -60,6 +66,21 @@ class Spec:
             ik, iq = self.letters.index(band[0]), self.letters.index(band[1])
             self.cells = [c for c in self.cells
                           if self.parts[band[0]][c[ik]] <= self.parts[band[1]][c[iq] + 1] - 1]
+        if induced is not None:
+            h, g, group = induced
+            if self.parts[h] != [group * x for x in self.parts[g]]:
+                raise ValueError(f"intervals of '{h}' must be those of '{g}' scaled by {group}")
+            ih, ig = self.letters.index(h), self.letters.index(g)
+            self.cells = [c for c in self.cells if c[ih] == c[ig]]
+        if segments is not None:
+            kl, ql, ends = segments
+            for l in (kl, ql):
+                if any(e not in self.parts[l] for e in ends):
+                    raise ValueError(f"index '{l}' may only be cut so that every sequence end is a split point")
+            seq_of = lambda x: sum(1 for e in ends if e <= x)   # sequence that position x belongs to
+            ik, iq = self.letters.index(kl), self.letters.index(ql)
+            self.cells = [c for c in self.cells
+                          if seq_of(self.parts[kl][c[ik]]) == seq_of(self.parts[ql][c[iq]])]
         self.p = len(self.cells)
 
     # -- per-operand helpers (operand = index into self.ins, or -1 for the output) --------------

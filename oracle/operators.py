@@ -76,6 +76,27 @@ def attention(Q, K, V, causal=True, out_dtype="bf16", scale=None, qpos=None):
     return rnd(core.attention(Q, K, V, scale, causal, qpos), out_dtype)
 
 
+def attention_gqa_packed(Q, K, V, group=1, ends=None, causal=True, out_dtype="bf16", scale=None):
+    """Grouped-query attention over packed sequences (Example 3.10). Q[b,s,hq,d], K,V[b,s,hkv,d] with hq = group*hkv:
+    query heads [group*m, group*(m+1)) attend key/value head m; the sequence index holds independent sequences ending
+    at `ends`, and attention never crosses a sequence boundary. Built from the plain definition above, one
+    (sequence, query head) at a time."""
+    Q, K, V = (np.asarray(t, dtype=np.float64) for t in (Q, K, V))
+    B, S, Hq, D = Q.shape
+    assert K.shape[2] * group == Hq
+    ends = [S] if ends is None else list(ends)
+    assert ends[-1] == S
+    scale = 1.0 / math.sqrt(D) if scale is None else scale
+    O = np.empty_like(Q)
+    s0 = 0
+    for s1 in ends:
+        for h in range(Hq):
+            g = h // group
+            O[:, s0:s1, h:h + 1] = core.attention(Q[:, s0:s1, h:h + 1], K[:, s0:s1, g:g + 1], V[:, s0:s1, g:g + 1], scale, causal)
+        s0 = s1
+    return rnd(O, out_dtype)
+
+
 def attention_as_join_aggs(Q, K, V, causal=True, scale=None):
     """The same operator as an explicit chain of scalar-keyed join-aggs (small shapes): scores =
     join on d + SUM; the causal band is a selection k <= q; MAX and exp/SUM aggregations over k;

@@ -313,18 +313,54 @@ extern "C" ja_status_t ja_spec_create(const char* einsum, const ja_index_part_t*
         p *= nb[l];
         if (p > (int64_t)1 << 26) return ja_fail(JA_ERR_UNSUPPORTED, "more than 2^26 function specs");
     }
-    // band predicate of attention: a (q-block, k-block) pair is a tuple only if some k <= some q
-    int band_q = -1, band_k = -1;
-    if (fn == JA_FN_ATTENTION && s->params.size() >= 2 && s->params[1] != 0.0 && s->ins.size() == 3 &&
-        s->ins[0].size() == 4 && s->ins[1].size() == 4) {
-        band_q = letter_pos(s->letters, s->ins[0][1]);
-        band_k = letter_pos(s->letters, s->ins[1][1]);
+    // Attention (Example 3.10). Three selections remove cells of the interval grid:
+    //   band      causal attention: a (q-block, k-block) pair is a tuple only if some k <= some q;
+    //   induced   grouped-query attention "bqhd,bkgd,bkgd->bqhd": h is not shardable by itself, its intervals are
+    //             those of g scaled by group = extent(h)/extent(g), and interval m of g pairs with interval m of h;
+    //   segments  packed sequences ending at params[2..]: q and k may be cut so that every sequence end is a split
+    //             point, and a pair of blocks is a tuple only if both lie in the same sequence.
+    int band_q = -1, band_k = -1, ind_h = -1, ind_g = -1, seg_q = -1, seg_k = -1;
+    std::vector<int64_t> ends;
+    if (fn == JA_FN_ATTENTION && s->ins.size() == 3 && s->ins[0].size() == 4 && s->ins[1].size() == 4) {
+        const int lq = letter_pos(s->letters, s->ins[0][1]), lk = letter_pos(s->letters, s->ins[1][1]);
+        if (s->params.size() >= 2 && s->params[1] != 0.0) { band_q = lq; band_k = lk; }
+        if (s->ins[1][2] != s->ins[0][2]) {
+            ind_h = letter_pos(s->letters, s->ins[0][2]);
+            ind_g = letter_pos(s->letters, s->ins[1][2]);
+            const int64_t eh = s->parts[ind_h].back(), eg = s->parts[ind_g].back();
+            if (eh % eg) return ja_fail(JA_ERR_SHAPE, "query heads (%lld) must be a multiple of key/value heads (%lld)", (long long)eh, (long long)eg);
+            const int64_t group = eh / eg;
+            bool same = s->parts[ind_h].size() == s->parts[ind_g].size();
+            for (size_t i = 0; same && i < s->parts[ind_g].size(); ++i) same = s->parts[ind_h][i] == group * s->parts[ind_g][i];
+            if (!same)
+                return ja_fail(JA_ERR_TILING, "index '%c' is not shardable by itself: its intervals must be those of '%c' scaled by %lld",
+                               s->ins[0][2], s->ins[1][2], (long long)group);
+        }
+        for (size_t i = 2; i < s->params.size(); ++i) ends.push_back((int64_t)s->params[i]);
+        if (!ends.empty()) {
+            if (s->parts[lq].back() != s->parts[lk].back()) return ja_fail(JA_ERR_SHAPE, "packed sequences need equal query and key extents");
+            if (ends.size() > JA_MAX_SEQ) return ja_fail(JA_ERR_UNSUPPORTED, "more than %d packed sequences", JA_MAX_SEQ);
+            for (size_t i = 0; i < ends.size(); ++i) {
+                if ((double)ends[i] != s->params[2 + i] || ends[i] <= (i ? ends[i - 1] : 0))
+                    return ja_fail(JA_ERR_INVALID_ARG, "sequence ends must be ascending positive integers");
+                for (int l : {lq, lk})
+                    if (!std::binary_search(s->parts[l].begin(), s->parts[l].end(), ends[i]))
+                        return ja_fail(JA_ERR_TILING, "index '%c' may only be cut so that every sequence end (%lld) is a split point",
+                                       s->letters[l], (long long)ends[i]);
+            }
+            if (ends.back() != s->parts[lq].back()) return ja_fail(JA_ERR_INVALID_ARG, "the last sequence must end at the extent of the sequence index");
+            seg_q = lq;
+            seg_k = lk;
+        }
     }
+    auto seq_of = [&](int64_t x) { return (int)(std::upper_bound(ends.begin(), ends.end(), x) - ends.begin()); };
     const int n_in = (int)s->ins.size();
     std::vector<int32_t> cell(L, 0);
     for (int64_t t = 0; t < p; ++t) {
         bool keep = true;
         if (band_q >= 0) keep = s->parts[band_k][cell[band_k]] <= s->parts[band_q][cell[band_q] + 1] - 1;
+        if (keep && ind_h >= 0) keep = cell[ind_h] == cell[ind_g];
+        if (keep && seg_q >= 0) keep = seq_of(s->parts[seg_k][cell[seg_k]]) == seq_of(s->parts[seg_q][cell[seg_q]]);
         if (keep) {
             for (int k = 0; k <= n_in; ++k) {
                 const std::string& term = (k < n_in) ? s->ins[k] : s->out;
@@ -586,6 +622,24 @@ struct ExecPlan {
     }
 };
 
+// True when a "bshd" relation has uniform blocks along b and h, an unsplit d, and every block starts where the closed
+// form used by the tensor-memory attention kernel puts it: blocks in key order, each a dense run of rows of
+// hblk * extent(d) cells, so block (bb, sb, hb) starts (bb*bblk*S + bblk*start(sb)) * nhb + hb*bblk*rows(sb) rows in.
+static bool bshd_rows_layout(const ja_relation* r) {
+    if (r->rank != 4 || !r->bs[0] || !r->bs[2] || r->nblk[3] != 1) return false;
+    const int64_t S = r->extent[1], bblk = r->bs[0], hblk = r->bs[2], nhb = r->nblk[2];
+    const int64_t row_bytes = hblk * r->extent[3] * r->esize;
+    if (r->extent[0] * S * nhb >= ((int64_t)1 << 31)) return false;
+    for (int32_t bb = 0; bb < r->nblk[0]; ++bb)
+        for (int32_t sb = 0; sb < r->nblk[1]; ++sb)
+            for (int32_t hb = 0; hb < r->nblk[2]; ++hb) {
+                const int64_t start = r->splits[1][sb], rows = r->splits[1][sb + 1] - start;
+                const int64_t want = ((bb * bblk * S + bblk * start) * nhb + hb * bblk * rows) * row_bytes;
+                if (r->blk_off[((int64_t)bb * r->nblk[1] + sb) * r->nblk[2] + hb] != want) return false;
+            }
+    return true;
+}
+
 static ja_status_t check_tiling(const ja_spec* s, int operand, const ja_relation* r) {
     const std::string& term = spec_term(s, operand);
     if (!r) return ja_fail(JA_ERR_INVALID_ARG, "relation for operand %d is NULL", operand);
@@ -798,23 +852,38 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         return ja_launch_row(ROW_ROPE, ra, X->dtype, stream);
     }
 
-    // ---- attention: "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX --------------------------------------
+    // ---- attention: "bqhd,bkhd,bkhd->bqhd" (or "bqhd,bkgd,bkgd->bqhd", grouped-query) ATTENTION / ONLINE_SOFTMAX ----
     if (fn == JA_FN_ATTENTION && agg == JA_AGG_ONLINE_SOFTMAX && n_in == 3 && x.size() == 4 && in[1].size() == 4 &&
-        in[1] == in[2] && o == x && in[1][0] == x[0] && in[1][2] == x[2] && in[1][3] == x[3] && in[1][1] != x[1]) {
+        in[1] == in[2] && o == x && in[1][0] == x[0] && in[1][3] == x[3] && in[1][1] != x[1] && in[1][2] != x[1] &&
+        in[1][2] != x[0] && in[1][2] != x[3]) {
         const ja_relation *Q = inputs[0], *K = inputs[1], *V = inputs[2];
         if (Q->dtype != JA_BF16 || K->dtype != JA_BF16 || V->dtype != JA_BF16 || out->dtype != JA_BF16)
             return ja_fail(JA_ERR_DTYPE, "attention relations must be bf16");
         if (Q->extent[3] != 128 || Q->nblk[3] != 1) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs an unsplit last index of extent 128");
         if (Q->extent[1] != K->extent[1]) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs equal query and key extents");
-        if (!Q->equal_blocks || !K->equal_blocks) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs uniform blocks");
         AttnArgs aa;
         memset(&aa, 0, sizeof aa);
         aa.q = ja_view(Q); aa.k = ja_view(K); aa.v = ja_view(V); aa.o = ja_view(out);
         aa.B = (int32_t)Q->extent[0]; aa.S = (int32_t)Q->extent[1]; aa.H = (int32_t)Q->extent[2]; aa.D = 128;
-        aa.qblk = (int32_t)Q->bs[1]; aa.kblk = (int32_t)K->bs[1]; aa.hblk = (int32_t)Q->bs[2];
-        if (aa.qblk % 64 || aa.kblk % 64) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs q/k blocks that are multiples of 64 rows");
+        aa.group = (int32_t)(Q->extent[2] / K->extent[2]);
+        int64_t g = Q->extent[1];
+        for (int64_t v : Q->splits[1]) g = std::__gcd(g, v);
+        for (int64_t v : K->splits[1]) g = std::__gcd(g, v);
+        aa.n_ends = spec->params.size() > 2 ? (int32_t)spec->params.size() - 2 : 0;
+        for (int i = 0; i < aa.n_ends; ++i) {
+            aa.ends[i] = (int32_t)spec->params[2 + i];
+            g = std::__gcd(g, (int64_t)aa.ends[i]);
+        }
+        aa.align = (int32_t)g;
+        if (aa.align % 64) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs q/k split points and sequence ends that are multiples of 64 rows");
         aa.scale = spec->params.size() >= 1 ? (float)spec->params[0] : 0.08838834764831845f;
         aa.causal = spec->params.size() >= 2 ? (spec->params[1] != 0.0) : 1;
+        std::vector<int32_t> qs(Q->splits[1].begin(), Q->splits[1].end()), ks(K->splits[1].begin(), K->splits[1].end());
+        aa.q_split = qs.data();
+        aa.k_split = ks.data();
+        aa.rows_layout = bshd_rows_layout(Q) && bshd_rows_layout(K) && bshd_rows_layout(V) && bshd_rows_layout(out) &&
+                         V->splits[1] == K->splits[1] && V->bs[0] == K->bs[0] && V->bs[2] == K->bs[2] &&
+                         out->splits[1] == Q->splits[1] && out->bs[0] == Q->bs[0] && out->bs[2] == Q->bs[2];
         return ja_launch_attention(aa, stream);
     }
 

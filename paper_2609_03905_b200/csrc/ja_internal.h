@@ -14,6 +14,7 @@
 #define JA_MAX_RANK 4
 #define JA_MAX_IN 4
 #define JA_ALIGN 128
+#define JA_MAX_SEQ 16      // packed sequences per attention spec
 
 // ---- device-side view of a tensor relation (passed to kernels by value) -------------------------
 // Key table on the device: per-dimension split points and per-block byte offsets. A kernel turns a
@@ -134,9 +135,16 @@ struct AttnArgs {
     RelView q, k, v, o;
     float scale;
     int causal;
-    int32_t B, S, H, D;
-    int32_t qblk, kblk;    // rows per q block / k block (uniform)
-    int32_t hblk;          // heads per block
+    int32_t B, S, H, D;    // H = query heads
+    int32_t group;         // query heads per key/value head (grouped-query attention); 1 otherwise
+    int32_t align;         // greatest common divisor of every q / k split point and sequence end
+    int32_t n_ends;        // packed sequences: ends[0..n_ends) ascending, ends[n_ends-1] == S; 0 = one sequence
+    int32_t ends[JA_MAX_SEQ];
+    // host copies of the sequence split points of q (= o) and k (= v), nblk[1] + 1 entries each, and whether all four
+    // payloads follow the closed-form block order the tensor-memory kernel addresses by (uniform b and h blocks)
+    const int32_t* q_split;
+    const int32_t* k_split;
+    bool rows_layout;
 };
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);
 // tcgen05 / TMEM form; *launched stays false when the tiling does not fit it

@@ -8,6 +8,9 @@
 // which is the aggregation operator of the spec. O = O~/l is written once, to the key's offset in the
 // output relation. Scores and probabilities never reach HBM.
 //
+// Grouped-query attention: query head h joins key/value head h / group. Packed sequences: an output key tile
+// joins only key/value tiles of its own sequence [s0, s1) (Example 3.10).
+//
 // This file holds the mma.sync form (m16n8k16, bf16 in, fp32 accumulate; operands staged in shared memory with
 // cp.async under an XOR swizzle and read with ldmatrix). It serves tilings the tensor-memory kernel cannot
 // take (64-row blocks); everything else is dispatched to the tcgen05 kernel.
@@ -74,6 +77,12 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest output keys (most surviving tuples) first
     const int h = blockIdx.y, b = blockIdx.z;
     const int q0 = qt * QT;
+    const int hk = h / a.group;                  // key/value head joined with this query head
+    int s0 = 0, s1 = a.S;                        // the packed sequence this tile lies in (no tile straddles an end)
+    for (int i = 0; i < a.n_ends; ++i) {
+        if (a.ends[i] <= q0) s0 = a.ends[i];
+        else { s1 = a.ends[i]; break; }
+    }
 
     // ---- stage Q, read its A fragments ---------------------------------------------------------------------
     {
@@ -85,15 +94,15 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
         }
         cp_async_commit();
     }
-    // number of 64-row key steps this output key joins with: keys [0, q0 + QT) when causal
-    const int k_end = a.causal ? min(a.S, q0 + QT) : a.S;
-    const int n_steps = (k_end + KT - 1) / KT;
+    // number of 64-row key steps this output key joins with: keys [s0, q0 + QT) when causal, else [s0, s1)
+    const int k_end = a.causal ? min(s1, q0 + QT) : s1;
+    const int n_steps = (k_end - s0 + KT - 1) / KT;
 
     auto load_kv = [&](int step, int buf) {
-        const int k0 = step * KT;  // a 64-row step never straddles a key block (64 divides kblk)
+        const int k0 = s0 + step * KT;  // a 64-row step never straddles a key block (64 divides every split point)
         int64_t pk, pv;
-        const char* kp = row_ptr(a.k, b, k0, h, &pk);
-        const char* vp = row_ptr(a.v, b, k0, h, &pv);
+        const char* kp = row_ptr(a.k, b, k0, hk, &pk);
+        const char* vp = row_ptr(a.v, b, k0, hk, &pv);
         const uint32_t dk = smem_u32(sK) + buf * KT * ROW_BYTES, dv = smem_u32(sV) + buf * KT * ROW_BYTES;
         for (int i = tid; i < KT * 16; i += NT) {
             int r = i / 16, c = i % 16;
@@ -148,7 +157,7 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
             }
         }
         // ---- scale, causal band inside the diagonal block, row max ---------------------------------------------
-        const int k0 = step * KT;
+        const int k0 = s0 + step * KT;
         const bool diag = a.causal && (k0 + KT - 1 > q0 + warp * 16);
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
@@ -247,7 +256,7 @@ ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
         ja_status_t s = ja_launch_attention_tc(a, st, &launched);
         if (s != JA_OK || launched) return s;
     }
-    const int QT = (a.qblk % 128 == 0) ? 128 : 64;
+    const int QT = (a.align % 128 == 0) ? 128 : 64;
     dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
     if (QT == 128) {

@@ -5,7 +5,9 @@
 // share that output key -- the 128-row key/value tiles that survive the causal band predicate -- ascending.
 //
 //   warp 0      TMA producer: Q once, then K_j and V_j (two stages each), straight from the "bshd" block-key
-//               layout through rank-5 tensor maps (d, head in block, row in block, batch in block, block).
+//               layout through rank-3 tensor maps (d, head in block, row): with uniform blocks along b and h every
+//               block is a run of rows of hblk x 128 cells, and the rows of consecutive blocks follow one another,
+//               so one map serves any split of the sequence index (uniform or at packed-sequence ends).
 //   warp 1      tcgen05.mma issuer (one lane):  S_j = Q K_j^T  (A, B from shared memory, both K-major)
 //                                               O'_j = P_j V_j  (A = P_j from TENSOR MEMORY, B = V_j MN-major)
 //   warps 2..5  one thread per query row: read S_j from TMEM, running max / sum in the base-2 domain, write
@@ -14,6 +16,8 @@
 //
 // TMEM map (512 columns): S/P buffers at 0 and 128, partial-O buffers at 256 and 384. QK^T of step j+1 is issued
 // before the softmax of step j finishes, so the tensor pipe works while the row threads exponentiate.
+// Grouped-query attention: query head h joins key/value head h / group. Packed sequences (Example 3.10): an output
+// key tile joins only the key/value tiles of its own sequence [s0, s1), so the walk starts at s0.
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT and leaves through the normal exit.
 #include <stdlib.h>
 
@@ -30,23 +34,60 @@ constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BYTES = 5 * TILE_BYTES + 1024 + 256;   // Q, K x2, V x2
 
+constexpr int MAX_SB = 64;   // sequence blocks of an irregular split held in the kernel parameters
+
+// Tiling of one "bshd" relation: uniform blocks along b and h, any split of s, d unsplit.
+struct SeqGeom {
+    int32_t bblk, hblk, nhb;     // batch rows per block, heads per block, blocks along h
+    int32_t sblk;                // uniform rows per s block, or 0: split[] holds the nsb + 1 split points
+    int32_t nsb;
+    int32_t split[MAX_SB + 1];
+};
+
 struct AttnTcParams {
     char* o_base;
     int32_t* status;
-    int64_t o_blk_stride;
     int32_t B, S, H;
-    int32_t bblk, sblk, hblk;       // block extents of q / o along b, s, h
-    int32_t nsb, nhb;               // blocks along s, h (q / o)
-    int32_t k_bblk, k_sblk, k_hblk, k_nsb, k_nhb;   // same for k / v
+    int32_t group;               // query heads per key/value head
     int32_t causal;
+    int32_t n_ends;              // packed sequences; 0 = one sequence [0, S)
     float scale_log2e;
+    int32_t ends[JA_MAX_SEQ];
+    SeqGeom q, k;                // o is tiled like q, v like k
 };
 
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3,
-                                            int c4) {
+// Row coordinate of cell (b, s, h, :) in the rank-3 view (d, head in block, row). Block (bb, sb, hb) starts
+// 128 * hblk * [ (bb*bblk*S + bblk*start(sb)) * nhb + hb*bblk*rows(sb) ] elements into the payload (blocks are stored
+// in key order, each dense), and inside it the row is (b in block) * rows(sb) + (s - start(sb)).
+__device__ __forceinline__ int seq_row(const SeqGeom& g, int S, int b, int s, int h) {
+    int start, rows;
+    if (g.sblk) {
+        start = (s / g.sblk) * g.sblk;
+        rows = g.sblk;
+    } else {
+        int sb = 0;
+        while (sb + 1 < g.nsb && g.split[sb + 1] <= s) ++sb;
+        start = g.split[sb];
+        rows = g.split[sb + 1] - start;
+    }
+    const int bb = b / g.bblk, hb = h / g.hblk;
+    return ((bb * g.bblk * S + g.bblk * start) * g.nhb + hb * g.bblk * rows) + (b - bb * g.bblk) * rows + (s - start);
+}
+
+// the packed sequence [s0, s1) that holds position q0
+__device__ __forceinline__ void sequence_of(const AttnTcParams& p, int q0, int& s0, int& s1) {
+    s0 = 0;
+    s1 = p.S;
+    for (int i = 0; i < p.n_ends; ++i) {
+        if (p.ends[i] <= q0) s0 = p.ends[i];
+        else { s1 = p.ends[i]; break; }
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
     asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 
@@ -108,7 +149,7 @@ __device__ __forceinline__ float ex2(float x) {
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                    const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -127,7 +168,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int qt = n_qt - 1 - (int)blockIdx.x;   // output keys with the most surviving tuples first
     const int h = blockIdx.y, b = blockIdx.z;
     const int q0 = qt * QT;
-    const int n_steps = p.causal ? (q0 + QT) / KT : p.S / KT;
+    int s0, s1;
+    sequence_of(p, q0, s0, s1);
+    const int n_steps = p.causal ? (q0 + QT - s0) / KT : (s1 - s0) / KT;   // key tiles [s0 + j*KT, ...) joined with this tile
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBAR; ++i) {
@@ -151,29 +194,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            // block key and in-block coordinates of this (b, h) for q and for k / v
-            const int qb_flat_bh = (b / p.bblk) * p.nsb * p.nhb + (h / p.hblk);     // + s-block * nhb
-            const int kb_flat_bh = (b / p.k_bblk) * p.k_nsb * p.k_nhb + (h / p.k_hblk);
+            const int hk = h / p.group;
+            const int qrow = seq_row(p.q, p.S, b, q0, h);
             mbar_expect_tx(bar(Q_FULL), TILE_BYTES);
             for (int half = 0; half < 2; ++half)
-                tma_load_5d(sQ + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.hblk, q0 % p.sblk, b % p.bblk,
-                            qb_flat_bh + (q0 / p.sblk) * p.nhb);
+                tma_load_3d(sQ + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow);
             bool ok = true;
             for (int j = 0; j < n_steps && ok; ++j) {
                 const int st = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1;
-                const int k0 = j * KT;
-                const int kflat = kb_flat_bh + (k0 / p.k_sblk) * p.k_nhb;
+                const int krow = seq_row(p.k, p.S, b, s0 + j * KT, hk);
                 if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
                 mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_5d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, h % p.k_hblk,
-                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                    tma_load_3d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, hk % p.k.hblk, krow);
                 if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
                 mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_5d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, h % p.k_hblk,
-                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                    tma_load_3d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, hk % p.k.hblk, krow);
             }
         }
     } else if (warp == 1) {
@@ -247,7 +285,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (!mbar_wait(bar(S_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
             const bool diag = p.causal && (j == n_steps - 1);
-            const int kmax = q0 + r - j * KT;        // columns c > kmax of this tile lie after the query row
+            const int kmax = q0 + r - (s0 + j * KT); // columns c > kmax of this tile lie after the query row
             // ---- pass 1: row maximum ----
             float mx = -INFINITY;
 #pragma unroll
@@ -310,10 +348,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 fold(ls, alpha_prev);
                 // ---- O = O~ / l, one rounding, 256 contiguous bytes per row ----
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const int s_glob = q0 + r;
-                const int64_t flat = ((int64_t)(b / p.bblk) * p.nsb + s_glob / p.sblk) * p.nhb + h / p.hblk;
-                char* dst = p.o_base + flat * p.o_blk_stride +
-                            ((((int64_t)(b % p.bblk) * p.sblk + s_glob % p.sblk) * p.hblk + h % p.hblk) * D) * 2;
+                char* dst = p.o_base + ((int64_t)seq_row(p.q, p.S, b, q0 + r, h) * p.q.hblk + h % p.q.hblk) * (D * 2);
 #pragma unroll
                 for (int g = 0; g < 16; ++g) {
                     uint4 ov;
@@ -426,7 +461,7 @@ constexpr int SMEM_BYTES2 = 6 * TILE_BYTES + 1024 + 256;   // Q_A, Q_B, K x2, V 
 
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -444,8 +479,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const int pr = n_pairs - 1 - (int)blockIdx.x;     // heaviest output keys first
     const int h = blockIdx.y, b = blockIdx.z;
     const int q0 = pr * 2 * QT;                       // first row of tile A; tile B starts at q0 + 128
-    const int n_steps_a = p.causal ? (q0 + QT) / KT : p.S / KT;
-    const int n_steps_b = p.causal ? (q0 + 2 * QT) / KT : p.S / KT;
+    int s0, s1;                                       // both tiles lie in one packed sequence (ends are multiples of 256)
+    sequence_of(p, q0, s0, s1);
+    const int n_steps_a = p.causal ? (q0 + QT - s0) / KT : (s1 - s0) / KT;
+    const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2) ? 4 : 1);
@@ -464,31 +501,26 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            const int qb_flat_bh = (b / p.bblk) * p.nsb * p.nhb + (h / p.hblk);
-            const int kb_flat_bh = (b / p.k_bblk) * p.k_nsb * p.k_nhb + (h / p.k_hblk);
+            const int hk = h / p.group;
             mbar_expect_tx(bar(Q_FULL), 2 * TILE_BYTES);
-            for (int t = 0; t < 2; ++t)
-                for (int half = 0; half < 2; ++half) {
-                    const int qs = q0 + t * QT;
-                    tma_load_5d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.hblk, qs % p.sblk,
-                                b % p.bblk, qb_flat_bh + (qs / p.sblk) * p.nhb);
-                }
+            for (int t = 0; t < 2; ++t) {
+                const int qrow_t = seq_row(p.q, p.S, b, q0 + t * QT, h);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow_t);
+            }
             bool ok = true;
             for (int j = 0; j < n_steps_b && ok; ++j) {
                 const int st = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1;
-                const int k0 = j * KT;
-                const int kflat = kb_flat_bh + (k0 / p.k_sblk) * p.k_nhb;
+                const int krow = seq_row(p.k, p.S, b, s0 + j * KT, hk);
                 if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
                 mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_5d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, h % p.k_hblk,
-                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                    tma_load_3d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, hk % p.k.hblk, krow);
                 if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
                 mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_5d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, h % p.k_hblk,
-                                k0 % p.k_sblk, b % p.k_bblk, kflat);
+                    tma_load_3d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, hk % p.k.hblk, krow);
             }
         }
     } else if (warp == 1) {
@@ -559,13 +591,13 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (!mbar_wait(bar(S_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
             const bool diag = p.causal && (j == n_t - 1);
-            const int kmax = qrow - j * KT;
+            const int kmax = qrow - (s0 + j * KT);
             uint32_t v[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
             tmem_ld_wait();
             const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
-            const float m_new = mx * p.scale_log2e;       // finite: key 0 of the first tile is never masked
+            const float m_new = mx * p.scale_log2e;       // finite: the first key of the sequence is never masked
             // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
             float alpha = 1.f;
             bool need = false;
@@ -599,9 +631,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
                 tc_fence_after();
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const int64_t flat = ((int64_t)(b / p.bblk) * p.nsb + qrow / p.sblk) * p.nhb + h / p.hblk;
-                char* dst = p.o_base + flat * p.o_blk_stride +
-                            ((((int64_t)(b % p.bblk) * p.sblk + qrow % p.sblk) * p.hblk + h % p.hblk) * D) * 2;
+                char* dst = p.o_base + ((int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk) * (D * 2);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -628,50 +658,67 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
 }
 
-// "bshd" relation with equal blocks [bb, sb, hb, 128] as a rank-5 tensor: (d, h in block, s in block, b in block, block)
-ja_status_t encode_bshd(const RelView& v, CUtensorMap* tm) {
+// "bshd" relation with uniform blocks along b and h as a rank-3 tensor (d, head in block, row of hblk x 128 cells)
+ja_status_t encode_rows(const RelView& v, CUtensorMap* tm) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-    const int64_t bb = v.bs[0], sb = v.bs[1], hb = v.bs[2];
-    const int64_t nblocks = (int64_t)v.nblk[0] * v.nblk[1] * v.nblk[2];
-    cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)hb, (cuuint64_t)sb, (cuuint64_t)bb, (cuuint64_t)nblocks};
-    cuuint64_t strides[4] = {(cuuint64_t)(D * 2), (cuuint64_t)(hb * D * 2), (cuuint64_t)(sb * hb * D * 2), (cuuint64_t)v.blk_stride};
-    cuuint32_t box[5] = {64, 1, 128, 1, 1};
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, v.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const int64_t hb = v.bs[2];
+    const int64_t rows = v.extent[0] * v.extent[1] * v.nblk[2];
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)hb, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)(D * 2), (cuuint64_t)(hb * D * 2)};
+    cuuint32_t box[3] = {64, 1, 128};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (bshd) failed with code %d", (int)res);
+    if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (bshd rows) failed with code %d", (int)res);
     return JA_OK;
+}
+
+bool fill_geom(const RelView& v, const int32_t* host_split, SeqGeom* g) {
+    if (!v.bs[0] || !v.bs[2] || v.nblk[3] != 1) return false;
+    g->bblk = (int32_t)v.bs[0];
+    g->hblk = (int32_t)v.bs[2];
+    g->nhb = v.nblk[2];
+    g->sblk = (int32_t)v.bs[1];
+    g->nsb = v.nblk[1];
+    if (!g->sblk) {
+        if (g->nsb > MAX_SB || !host_split) return false;
+        for (int i = 0; i <= g->nsb; ++i) g->split[i] = host_split[i];
+    }
+    return true;
 }
 
 }  // namespace
 
 // Returns JA_OK and sets *launched when the tensor-memory kernel took the job; leaves *launched false when the
-// tiling does not fit it (q and k row blocks must be multiples of 128 rows, all blocks of one shape).
+// tiling does not fit it (every q / k split point and sequence end must be a multiple of 128 rows, blocks uniform
+// along b and h, at most MAX_SB sequence blocks when they are irregular).
 ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched) {
     *launched = false;
-    if (a.qblk % 128 || a.kblk % 128 || !a.q.blk_stride || !a.k.blk_stride || !a.v.blk_stride || !a.o.blk_stride) return JA_OK;
-    if (a.v.blk_stride != a.k.blk_stride || a.o.blk_stride != a.q.blk_stride) return JA_OK;
-    CUtensorMap tq, tk, tv;
-    ja_status_t s;
-    if ((s = encode_bshd(a.q, &tq)) != JA_OK) return s;
-    if ((s = encode_bshd(a.k, &tk)) != JA_OK) return s;
-    if ((s = encode_bshd(a.v, &tv)) != JA_OK) return s;
+    if (a.align % 128 || !a.rows_layout) return JA_OK;
     AttnTcParams p;
     memset(&p, 0, sizeof p);
+    if (!fill_geom(a.q, a.q_split, &p.q) || !fill_geom(a.k, a.k_split, &p.k)) return JA_OK;
+    CUtensorMap tq, tk, tv;
+    ja_status_t s;
+    if ((s = encode_rows(a.q, &tq)) != JA_OK) return s;
+    if ((s = encode_rows(a.k, &tk)) != JA_OK) return s;
+    if ((s = encode_rows(a.v, &tv)) != JA_OK) return s;
     p.o_base = a.o.base;
     p.status = ja_device_status_word();
     if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
-    p.o_blk_stride = a.o.blk_stride;
     p.B = a.B; p.S = a.S; p.H = a.H;
-    p.bblk = (int)a.q.bs[0]; p.sblk = (int)a.q.bs[1]; p.hblk = (int)a.q.bs[2];
-    p.nsb = a.q.nblk[1]; p.nhb = a.q.nblk[2];
-    p.k_bblk = (int)a.k.bs[0]; p.k_sblk = (int)a.k.bs[1]; p.k_hblk = (int)a.k.bs[2];
-    p.k_nsb = a.k.nblk[1]; p.k_nhb = a.k.nblk[2];
+    p.group = a.group;
     p.causal = a.causal;
+    p.n_ends = a.n_ends;
+    bool pair_ok = a.S % (2 * QT) == 0;
+    for (int i = 0; i < a.n_ends; ++i) {
+        p.ends[i] = a.ends[i];
+        if (a.ends[i] % (2 * QT)) pair_ok = false;
+    }
     p.scale_log2e = a.scale * 1.4426950408889634f;
     const char* one = getenv("JA_ATTN_ONE_TILE");
-    if (a.S % (2 * QT) == 0 && !(one && one[0] == '1')) {
+    if (pair_ok && !(one && one[0] == '1')) {
         JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
         dim3 grid((unsigned)(a.S / (2 * QT)), (unsigned)a.H, (unsigned)a.B);
         attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);

@@ -109,6 +109,37 @@ def test_config4_attention_full_size():
         assert relfro(got[b:b + 1, rows, h:h + 1], ref) <= TOL[BF], (b, h)
 
 
+def test_grouped_query_attention_packed_sequences_full_size():
+    """Example 3.10 at its own sizes: 32 query heads on 8 key/value heads (cut into unit intervals, so the query heads
+    fall into intervals of 4), a sequence index of 4096 holding three sequences that end at 1024, 2560 and 4096 and cut
+    only there. Checked on sampled (batch, head, row) triples, each against the oracle's attention over its own sequence."""
+    B, S, Hq, Hkv, D, grp = 2, 4096, 32, 8, 128, 4
+    ends = [1024, 2560, 4096]
+    Q = si.normal((B, S, Hq, D), 0.0, 1.0, BF, 4, 11)
+    K, V = (si.normal((B, S, Hkv, D), 0.0, 1.0, BF, 4, o) for o in (12, 13))
+    g_split = list(range(Hkv + 1))
+    h_split = [grp * x for x in g_split]
+    q_sp = [ES(B, B), [0] + ends, h_split, [0, D]]
+    k_sp = [ES(B, B), [0] + ends, g_split, [0, D]]
+    rQ, rK, rV = upload(Q, q_sp), upload(K, k_sp), upload(V, k_sp)
+    rO = empty_like_tiling([B, S, Hq, D], q_sp, BF, fill=float("nan"))
+    parts = {"b": q_sp[0], "q": q_sp[1], "h": h_split, "d": [0, D], "k": q_sp[1], "g": g_split}
+    spec = ja.Spec("bqhd,bkgd,bkgd->bqhd", parts, "attention", (1.0 / np.sqrt(D), 1.0) + tuple(map(float, ends)), "online_softmax")
+    assert ja.ja_spec_num_tuples(spec.handle)[0] == B * 3 * Hkv          # pure join and recompose: one tuple per output key
+    spec.execute([rQ, rK, rV], rO)
+    got = download(rO)
+    check_status()
+    assert not np.isnan(got).any()
+    for s0, s1 in zip([0] + ends[:-1], ends):
+        rows = np.array([s0, s0 + 1, s0 + 127, s0 + 128, s0 + 700, s1 - 129, s1 - 1])
+        for b, h in ((0, 0), (1, 13), (1, 31)):
+            g = h // grp
+            ref = operators.attention(si.to_f64(Q[b:b + 1, rows, h:h + 1]), si.to_f64(K[b:b + 1, s0:s1, g:g + 1]),
+                                      si.to_f64(V[b:b + 1, s0:s1, g:g + 1]), True, "bf16", qpos=rows - s0)
+            assert relfro(got[b:b + 1, rows, h:h + 1], ref) <= TOL[BF], (s0, b, h)
+        assert np.array_equal(got[:, s0], np.repeat(si.to_f64(V)[:, s0], grp, axis=1))
+
+
 def _block_case(shape_name, Bt, S, hidden, heads, ffn, prefix, seq_id):
     w = si.llama_weights(hidden, ffn)
     x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 0)

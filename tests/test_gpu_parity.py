@@ -237,6 +237,46 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
 
 
+# grouped-query attention over packed sequences (Example 3.10): query head h joins key/value head h // group and
+# no tuple crosses a sequence end. `cut` says where the sequence index is split: "ends" = at the sequence ends only
+# (irregular blocks), an integer = uniform blocks of that many rows (every end is then a split point).
+@pytest.mark.parametrize("B,S,Hq,Hkv,gblk,ends,cut,causal", [
+    (1, 512, 4, 2, 1, [128, 384, 512], 128, True),          # ends at odd multiples of 128: one-tile kernel
+    (2, 1024, 8, 2, 1, [256, 768, 1024], "ends", True),     # the paper's cut: blocks of 256, 512, 256 rows
+    (1, 1024, 4, 4, 2, [512, 1024], "ends", False),         # group 1, two heads per block, not causal
+    (1, 512, 2, 1, 1, [64, 320, 512], 64, True),            # 64-row granularity: mma.sync form
+    (2, 768, 6, 2, 2, [768], 256, True),                    # one sequence, grouped heads only
+    (1, 1280, 4, 1, 1, [256, 384, 1280], "ends", True),     # blocks of 256, 128, 896 rows
+])
+@pytest.mark.parametrize("form", ["default", "tcgen05_one_tile", "mma_sync"])
+def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut, causal, form, monkeypatch):
+    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
+    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
+    D, grp = 128, Hq // Hkv
+    Q = si.normal((B, S, Hq, D), 0.0, 1.0, BF, 4, 11)
+    K, V = (si.normal((B, S, Hkv, D), 0.0, 1.0, BF, 4, o) for o in (12, 13))
+    s_split = [0] + ends if cut == "ends" else ES(S, S // cut)
+    g_split = ES(Hkv, Hkv // gblk)
+    h_split = [grp * x for x in g_split]
+    q_sp = [ES(B, B), s_split, h_split, [0, D]]
+    k_sp = [ES(B, B), s_split, g_split, [0, D]]
+    rQ, rK, rV = upload(Q, q_sp), upload(K, k_sp), upload(V, k_sp)
+    rO = empty_like_tiling([B, S, Hq, D], q_sp, BF, fill=float("nan"))
+    parts = {"b": q_sp[0], "q": s_split, "h": h_split, "d": [0, D], "k": s_split, "g": g_split}
+    prm = (1.0 / np.sqrt(D), 1.0 if causal else 0.0) + tuple(float(e) for e in ends)
+    spec = ja.Spec("bqhd,bkgd,bkgd->bqhd" if grp > 1 else "bqhd,bkhd,bkhd->bqhd",
+                   parts if grp > 1 else {k: v for k, v in parts.items() if k != "g"}, "attention", prm, "online_softmax")
+    spec.execute([rQ, rK, rV], rO)
+    got = download(rO)
+    check_status()
+    ref = operators.attention_gqa_packed(si.to_f64(Q), si.to_f64(K), si.to_f64(V), grp, ends, causal, "bf16")
+    assert relfro(got, ref) <= TOL[BF]
+    assert np.abs(got - ref).max() <= 0.05
+    if causal:   # the first row of every sequence joins with its own key only: O = V exactly
+        for s0 in [0] + ends[:-1]:
+            assert np.array_equal(got[:, s0], np.repeat(si.to_f64(V)[:, s0], grp, axis=1))
+
+
 # ---------------------------------------------------------------------------------------------------
 # fused chains on the tensor-core matmul: the accumulator goes through the next join-agg before its one store
 # ---------------------------------------------------------------------------------------------------

@@ -78,6 +78,48 @@ def test_attention_spec_band_predicate():
     ja.ja_spec_destroy(full)
 
 
+def test_attention_spec_grouped_heads_and_packed_sequences(golden_dir):
+    """Example 3.10: heads_q inherits its split from heads_kv; the sequence is cut at sequence ends only."""
+    g = json.load(open(os.path.join(golden_dir, "gqa_packed_example.json")))
+    Hq, Hkv, grp, S, ends = g["heads_q"], g["heads_kv"], g["group"], g["sequence_extent"], g["sequence_ends"]
+    es = "bqhd,bkgd,bkgd->bqhd"
+    parts = {"b": [0, 1], "q": [0, S], "h": [grp * m for m in range(Hkv + 1)], "d": [0, 128], "k": [0, S],
+             "g": list(range(Hkv + 1))}
+    s = ja.ja_spec_create(es, parts, "attention", (0.088, 1.0), "online_softmax")
+    assert ja.ja_spec_num_tuples(s)[0] == g["num_function_specs_when_heads_kv_is_cut_into_unit_intervals"]
+    ink, outk = ja.ja_spec_get_tuples(s)
+    rink, routk = blocked.Spec(es, parts, band=("k", "q"), induced=("h", "g", grp)).tuples()
+    assert np.array_equal(ink, rink) and np.array_equal(outk, routk)
+    assert ink[:, 0].tolist() == ink[:, 1].tolist() == list(range(Hkv))     # m-th spec: q-head block m with kv head m
+    ja.ja_spec_destroy(s)
+    with pytest.raises(ja.JaError):      # heads_q is not shardable by itself
+        ja.ja_spec_create(es, dict(parts, h=[0, 16, 32]), "attention", (0.088, 1.0), "online_softmax")
+    # cut at the sequence ends: 3 sequences x 8 heads, no aggregation (every output key has one tuple)
+    parts2 = dict(parts, q=[0] + ends, k=[0] + ends)
+    prm = (0.088, 1.0) + tuple(float(e) for e in ends)
+    s = ja.ja_spec_create(es, parts2, "attention", prm, "online_softmax")
+    assert ja.ja_spec_num_tuples(s)[0] == g["num_function_specs_when_sequence_is_cut_at_its_ends_and_heads_kv_into_unit_intervals"]
+    ink, outk = ja.ja_spec_get_tuples(s)
+    ref = blocked.Spec(es, parts2, band=("k", "q"), induced=("h", "g", grp), segments=("k", "q", ends))
+    rink, routk = ref.tuples()
+    assert np.array_equal(ink, rink) and np.array_equal(outk, routk)
+    assert np.bincount(outk).tolist() == [1] * 24
+    ja.ja_spec_destroy(s)
+    # finer cuts inside sequences (every end still a split point): band and same-sequence selections together
+    parts3 = dict(parts, q=blocked.equal_splits(S, 8), k=blocked.equal_splits(S, 16))
+    for causal in (1.0, 0.0):
+        s = ja.ja_spec_create(es, parts3, "attention", (0.088, causal) + prm[2:], "online_softmax")
+        ref = blocked.Spec(es, parts3, band=("k", "q") if causal else None, induced=("h", "g", grp), segments=("k", "q", ends))
+        ink, outk = ja.ja_spec_get_tuples(s)
+        rink, routk = ref.tuples()
+        assert np.array_equal(ink, rink) and np.array_equal(outk, routk)
+        ja.ja_spec_destroy(s)
+    with pytest.raises(ja.JaError):      # a cut that skips a sequence end
+        ja.ja_spec_create(es, dict(parts, q=[0, 2048, S], k=[0, 2048, S]), "attention", prm, "online_softmax")
+    with pytest.raises(ja.JaError):      # ends must ascend and finish at the extent
+        ja.ja_spec_create(es, parts2, "attention", (0.088, 1.0, 2560.0, 1024.0, 4096.0), "online_softmax")
+
+
 def test_paper_worked_examples_through_the_library(golden_dir):
     g = json.load(open(os.path.join(golden_dir, "matmul_decomposed.json")))
     s = ja.ja_spec_create(g["einsum"], g["four_spec"]["parts"])

@@ -384,3 +384,51 @@ def test_llama_block_composition():
     # with storage rounding the result stays within bf16 distance of the unrounded one
     b16 = operators.llama_block(x, w, H, 1e4, 1e-5, dtype="bf16")["out"]
     assert np.linalg.norm(b16 - full["out"]) / np.linalg.norm(full["out"]) < 2e-2
+
+
+# ---------------------------------------------------------------------------------------------------
+# grouped-query attention and packed sequences (Example 3.10)
+# ---------------------------------------------------------------------------------------------------
+def test_gqa_packed_spec_example(golden_dir):
+    g = _golden(golden_dir, "gqa_packed_example.json")
+    Hq, Hkv, grp, S = g["heads_q"], g["heads_kv"], g["group"], g["sequence_extent"]
+    es = "bqhd,bkgd,bkgd->bqhd"
+    parts = {"b": [0, 1], "q": [0, S], "h": [grp * m for m in range(Hkv + 1)], "d": [0, 128], "k": [0, S],
+             "g": list(range(Hkv + 1))}
+    spec = blocked.Spec(es, parts, induced=("h", "g", grp))
+    assert spec.p == g["num_function_specs_when_heads_kv_is_cut_into_unit_intervals"]
+    for cell in spec.cells:   # the m-th specification: key/value head m, query heads [4m, 4(m+1))
+        m = cell[spec.letters.index("g")]
+        lo, hi = spec.bounds(spec.block_coords(cell, 0), 0)
+        assert [lo[2], hi[2]] == [grp * m, grp * (m + 1)]
+        if str(m) in g["query_head_interval_of_kv_head"]:
+            assert [lo[2], hi[2]] == g["query_head_interval_of_kv_head"][str(m)]
+    with pytest.raises(ValueError):   # heads_q is not shardable on its own
+        blocked.Spec(es, dict(parts, h=[0, 16, 32]), induced=("h", "g", grp))
+    ends = g["sequence_ends"]
+    parts2 = dict(parts, q=[0] + ends, k=[0] + ends)
+    spec2 = blocked.Spec(es, parts2, induced=("h", "g", grp), segments=("k", "q", ends), band=("k", "q"))
+    assert spec2.p == g["num_function_specs_when_sequence_is_cut_at_its_ends_and_heads_kv_into_unit_intervals"]
+    assert (spec2.multiplicity() == 1).all()     # pure join + recompose: no aggregation (as the paper notes)
+    with pytest.raises(ValueError):   # a cut that is not at a sequence end and removes an end is refused
+        blocked.Spec(es, dict(parts, q=[0, 2048, S], k=[0, 2048, S]), induced=("h", "g", grp), segments=("k", "q", ends))
+
+
+def test_gqa_packed_attention_against_library():
+    B, S, Hq, Hkv, D = 1, 24, 4, 2, 8
+    ends = [5, 16, 24]
+    Q = RNG.standard_normal((B, S, Hq, D))
+    K, V = RNG.standard_normal((B, S, Hkv, D)), RNG.standard_normal((B, S, Hkv, D))
+    got = operators.attention_gqa_packed(Q, K, V, group=2, ends=ends, causal=True, out_dtype=None)
+    # torch: repeat the kv heads, block-diagonal causal mask
+    t = lambda a: torch.from_numpy(a).permute(0, 2, 1, 3)
+    seq = np.searchsorted(np.array(ends), np.arange(S), side="right")
+    mask = torch.from_numpy((seq[:, None] == seq[None, :]) & (np.arange(S)[None, :] <= np.arange(S)[:, None]))
+    want = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K).repeat_interleave(2, dim=1), t(V).repeat_interleave(2, dim=1),
+                                                            attn_mask=mask).permute(0, 2, 1, 3).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    # one sequence, group 1 reduces to plain attention
+    np.testing.assert_array_equal(operators.attention_gqa_packed(Q, Q, Q, 1, None, True, None), operators.attention(Q, Q, Q, True, None))
+    # the first row of every sequence sees only itself
+    for s0 in [0] + ends[:-1]:
+        np.testing.assert_allclose(got[:, s0], V[:, s0].repeat(2, axis=1), rtol=1e-14)
