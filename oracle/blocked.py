@@ -254,3 +254,69 @@ def t2_join_agg(einsum: str, parts: dict, inputs, fn="mul", agg="sum", params=()
         out[tuple(slice(l, h) for l, h in zip(lo, hi))] = blk
     assert not np.isnan(out).any(), "output types do not tile the output (tiling condition)"
     return out
+
+
+# ---------------------------------------------------------------------------------------------------
+# Producers compiled "through their join" and the aggregating relayout that consumes them
+# (Section 5.1: the unaggregated partial blocks of a producer stay where they were computed and the
+# consumer aggregates them as it brings them where they are needed; Section 5.3: decompose every
+# copy into atoms, (+)-aggregate the m copies of each atom, recompose the consumer's blocks).
+# ---------------------------------------------------------------------------------------------------
+def join_partials(einsum: str, parts: dict, inputs, fn="mul", agg="sum", params=(), dtype=None):
+    """Step (1) of Definition 3.7 alone.  Returns the dense tensor P[c, out...]: for every output type,
+    copy c is the output of the c-th function specification (ascending F) that has this output type.
+    Every output type must have the same multiplicity m.  Each partial block is rounded once to
+    `dtype` (its store); the per-specification reduction over the indices inside the block uses `agg`."""
+    spec = Spec(einsum, parts)
+    mult = spec.multiplicity()
+    m = int(mult.reshape(-1)[0])
+    if not (mult == m).all():
+        raise ValueError("output types have different multiplicities")
+    arrs = [np.asarray(a, dtype=np.float64) for a in inputs]
+    out = np.full([m] + [spec.extent[c] for c in spec.out], np.nan)
+    seen = {}
+    for cell in spec.cells:
+        proj = []
+        for k in range(len(spec.ins)):
+            lo, hi = spec.bounds(spec.block_coords(cell, k), k)
+            proj.append(arrs[k][tuple(slice(l, h) for l, h in zip(lo, hi))])
+        ext = {c: spec.parts[c][x + 1] - spec.parts[c][x] for c, x in zip(spec.letters, cell)}
+        part = core.join_agg(einsum, proj, fn=fn, agg=agg, params=params, extents=ext)
+        okey = spec.block_coords(cell, -1)
+        c = seen.get(okey, 0)
+        seen[okey] = c + 1
+        lo, hi = spec.bounds(okey, -1)
+        out[(c,) + tuple(slice(l, h) for l, h in zip(lo, hi))] = part
+    assert not np.isnan(out).any()
+    return core.round_to(out, dtype) if dtype in ("f32", "bf16") else out
+
+
+def partial_splits(m: int, splits):
+    """Tiling of a partial relation: the copy index in front, cut into its m unit intervals."""
+    return [list(range(m + 1))] + [list(s) for s in splits]
+
+
+def aggregate_repartition(partials: np.ndarray, src_splits, dst_splits, agg="sum", dtype=None) -> np.ndarray:
+    """Section 5.3 on one processor.  `partials` is the dense fp64 tensor P[c, x...] of a partial
+    relation whose blocks are (copy c) x (block of src_splits).  decompose: every copy of every
+    producer block is sliced into the atoms of the overlay of src_splits and dst_splits; aggregate:
+    the m copies of an atom are (+)-combined in ascending copy order; recompose: the aggregated atoms
+    of a consumer block are concatenated.  One rounding to `dtype` at the consumer's store.  Returns
+    the dense tensor (the caller packs it with dst_splits)."""
+    P = np.asarray(partials, dtype=np.float64)
+    m = P.shape[0]
+    out = np.full(P.shape[1:], np.nan)
+    _, atoms = overlay_atoms(src_splits, dst_splits)
+    for lo, hi, _sb, _db in atoms:
+        sl = tuple(slice(l, h) for l, h in zip(lo, hi))
+        acc = P[(0,) + sl].copy()
+        for c in range(1, m):
+            if agg == "sum":
+                acc = acc + P[(c,) + sl]
+            elif agg == "max":
+                acc = np.maximum(acc, P[(c,) + sl])
+            else:
+                raise ValueError("an atom has several copies but there is no aggregation")
+        out[sl] = acc
+    assert not np.isnan(out).any()
+    return core.round_to(out, dtype) if dtype in ("f32", "bf16") else out

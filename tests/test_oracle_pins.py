@@ -432,3 +432,63 @@ def test_gqa_packed_attention_against_library():
     # the first row of every sequence sees only itself
     for s0 in [0] + ends[:-1]:
         np.testing.assert_allclose(got[:, s0], V[:, s0].repeat(2, axis=1), rtol=1e-14)
+
+
+# ---------------------------------------------------------------------------------------------------
+# producers compiled through their join + the aggregating relayout (Sections 5.1, 5.3)
+# ---------------------------------------------------------------------------------------------------
+def test_preamble_example_atoms_and_aggregates(golden_dir):
+    g = _golden(golden_dir, "preamble_example.json")
+    ext, src, dst = g["extents"], g["producer_splits"], g["consumer_splits"]
+    # label every cell of copy X of atom j with j and of copy Y with 10 j: OUT must hold 11 j in consumer block j-1
+    P = np.zeros([g["copies_per_block"]] + ext)
+    for name, info in g["in"].items():
+        for j in info["atoms"]:
+            r0, r1 = g["atom_rows"][str(j)]
+            P[info["copy"], r0:r1] = j * (1 if name == "X" else 10)
+    out = blocked.aggregate_repartition(P, src, dst, "sum")
+    payload = blocked.pack(out, dst)
+    _, lower, upper, offsets, _ = blocked.relation_keys(ext, dst, 8)
+    for req in g["out"]:
+        j = int(req["sum_of"][0][1:])
+        assert req["sum_of"] == [f"X{j}", f"Y{j}"]
+        b = req["consumer_block"]
+        n = int(np.prod(upper[b] - lower[b]))
+        blk = payload[offsets[b] // 8: offsets[b] // 8 + n]
+        assert (blk == 11 * j).all() and [int(lower[b][0]), int(upper[b][0])] == g["atom_rows"][str(j)]
+
+
+def test_join_partials_sum_to_the_aggregated_output():
+    A, B = RNG.standard_normal((24, 30)), RNG.standard_normal((30, 20))
+    parts = {"i": [0, 8, 24], "j": [0, 10, 20, 30], "k": [0, 5, 20]}
+    P = blocked.join_partials("ij,jk->ik", parts, [A, B])
+    assert P.shape == (3, 24, 20)
+    np.testing.assert_allclose(P.sum(axis=0), A @ B, rtol=1e-12, atol=1e-12)       # plain definition
+    for c, (j0, j1) in enumerate(zip(parts["j"], parts["j"][1:])):                 # copy c = contracted block c
+        np.testing.assert_allclose(P[c], A[:, j0:j1] @ B[j0:j1], rtol=1e-12, atol=1e-12)
+    src = [parts["i"], parts["k"]]
+    for dst in (src, [[0, 24], [0, 20]], [[0, 3, 12, 24], [0, 7, 11, 20]]):
+        out = blocked.aggregate_repartition(P, src, dst, "sum")
+        # same (+) order as Definition 3.7's aggregate step: bit-equal to the one-shot implementation
+        np.testing.assert_array_equal(out, blocked.t2_join_agg("ij,jk->ik", parts, [A, B]))
+    with pytest.raises(ValueError):    # several copies of an atom and no aggregation operator
+        blocked.aggregate_repartition(P, src, src, "none")
+
+
+def test_aggregate_repartition_against_dense_reduction_and_plain_repartition():
+    ext = [20, 12]
+    src, dst = [[0, 7, 20], [0, 4, 12]], [[0, 5, 10, 20], [0, 12]]
+    P = RNG.standard_normal([4] + ext)
+    # brute force through an independent route: pack copies, unpack to dense, reduce with numpy
+    payload = blocked.pack(P, blocked.partial_splits(4, src))
+    dense = blocked.unpack(payload, [4] + ext, blocked.partial_splits(4, src))
+    np.testing.assert_array_equal(dense, P)
+    np.testing.assert_array_equal(blocked.aggregate_repartition(P, src, dst, "max"), dense.max(axis=0))
+    np.testing.assert_allclose(blocked.aggregate_repartition(P, src, dst, "sum"), dense.sum(axis=0), rtol=1e-13, atol=1e-13)
+    # ascending copy order, one rounding at the store
+    s = ((P[0] + P[1]) + P[2]) + P[3]
+    np.testing.assert_array_equal(blocked.aggregate_repartition(P, src, dst, "sum", "bf16"), core.round_to(s, "bf16"))
+    # one copy: the aggregating relayout is the plain relayout, bit for bit
+    one = blocked.pack(P[:1], blocked.partial_splits(1, src))
+    got = blocked.pack(blocked.aggregate_repartition(P[:1], src, dst, "none"), dst)
+    np.testing.assert_array_equal(got, blocked.repartition(one, ext, src, dst))
