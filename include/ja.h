@@ -159,7 +159,8 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  *   "Rj,R,R->Rj"           EXP_SUB_DIV / NONE
  *   "Rj,j->Rj"             RMSNORM / NONE   (fused)       "Rj->Rj"  SOFTMAX / NONE (fused)
  *   "bshd->bshd"           ROPE / NONE
- *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128
+ *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128; q / k split points and sequence
+ *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends multiples of 64 rows (tensor memory kernels: 128)
  * The first call for a given (spec, relations) tuple builds and caches tables on the device (a few
  * synchronous cudaMalloc / cudaMemcpy); later calls only launch. */
 ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,
@@ -174,6 +175,27 @@ ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* dst, void* c
  * flat source block, flat destination block.  Pass NULL arrays to query the count only. */
 ja_status_t ja_overlay_atoms(const ja_relation_t* src, const ja_relation_t* dst, int64_t* n_atoms, int64_t* lower,
                              int64_t* upper, int32_t* src_block, int32_t* dst_block);
+
+/* ---- a producer executed through its join, and the aggregating relayout that consumes it (Sections 5.1, 5.3) ----
+ * ja_execute_join runs step (1) of Definition 3.7 alone: the concrete operator of every function spec, nothing
+ * aggregated across specs. `partials` receives the unaggregated blocks as a PARTIAL RELATION: a relation of rank
+ * rank(out)+1 whose leading index is the copy index c, extent m = the number of function specs per output type
+ * (it must be the same for all of them), cut into its m unit intervals; the other indices are those of the output,
+ * tiled as out(J). Block (c, key) holds the output of the c-th function spec (ascending F) with output type `key`.
+ * Supported: "ij,jk->ik" MUL/SUM -- copy c is A[:, block c] B[block c, :]. bf16 operands on uniform blocks: tensor
+ * cores, partial relation bf16 (one rounding per copy) or f32 (the accumulator as it is); otherwise plain ALUs and a
+ * partial relation of the operands' dtype. Errors as ja_execute; JA_ERR_UNSUPPORTED for other forms.
+ *
+ * ja_repartition_agg is the one-processor image of an exchange program: every atom of the overlay of the partial
+ * relation's tiling (copy index dropped) and dst's tiling has m copies; they are (+)-combined in ascending copy
+ * order in f32 (agg = JA_AGG_SUM or JA_AGG_MAX; JA_AGG_NONE only when m == 1, a plain relayout) and stored once,
+ * rounded once, in dst's block. partials may be f32 or bf16, dst f32 or bf16, independently. partials is borrowed and
+ * unchanged. Asynchronous on `cuda_stream`; the first call per (partials, dst) pair builds and caches the copy plan
+ * (one synchronous cudaMalloc + cudaMemcpy). Errors: JA_ERR_SHAPE, JA_ERR_TILING (copy index not cut into unit
+ * intervals), JA_ERR_INVALID_ARG (aggregation missing; dst aliases partials). */
+ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,
+                            ja_relation_t* partials, void* cuda_stream);
+ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_t agg, ja_relation_t* dst, void* cuda_stream);
 
 /* ---- relayout without allocation -------------------------------------------------------------------
  * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)

@@ -4,4 +4,5 @@
 """
 from . import binding  # noqa: F401  (raises if libja.so is absent and cannot be built)
 from .binding import *  # noqa: F401,F403
-from .relations import Relation, Spec, equal_splits, from_dense, repartition, to_dense  # noqa: F401
+from .relations import (Relation, Spec, equal_splits, from_dense, partial_relation, repartition,  # noqa: F401
+                        repartition_agg, to_dense)

@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
         "ja_relation_get_keys": [vp, vp, vp, vp, vp],
         "ja_execute": [vp, P(vp), i32, P(vp), i32, vp],
         "ja_repartition": [vp, vp, vp],
+        "ja_execute_join": [vp, P(vp), i32, vp, vp],
+        "ja_repartition_agg": [vp, ctypes.c_int, vp, vp],
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
         "ja_repartition_noalloc": [i32, P(i64), P(i32), P(P(i64)), P(i32), P(P(i64)), ctypes.c_int, vp, vp, vp],
@@ -194,6 +196,17 @@ def ja_execute(spec: int, inputs, outputs, stream: int = 0):
 
 def ja_repartition(src: int, dst: int, stream: int = 0):
     _check(LIB.ja_repartition(src, dst, ctypes.c_void_p(stream)))
+
+
+def ja_execute_join(spec: int, inputs, partials: int, stream: int = 0):
+    """Join only: every function spec's output goes, unaggregated, to its copy of the partial relation."""
+    ins = (ctypes.c_void_p * len(inputs))(*inputs)
+    _check(LIB.ja_execute_join(spec, ins, len(inputs), partials, ctypes.c_void_p(stream)))
+
+
+def ja_repartition_agg(partials: int, agg, dst: int, stream: int = 0):
+    """Aggregating relayout: the m copies of every atom are combined and stored in dst's tiling."""
+    _check(LIB.ja_repartition_agg(partials, AGG[agg] if isinstance(agg, str) else int(agg), dst, ctypes.c_void_p(stream)))
 
 
 def ja_repartition_noalloc(extents, src_splits, dst_splits, dtype: int, src_ptr: int, dst_ptr: int, stream: int = 0):

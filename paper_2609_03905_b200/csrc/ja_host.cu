@@ -4,6 +4,7 @@
 // happens on the host.
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -547,6 +548,48 @@ static int64_t in_block_offset(const ja_relation* r, int32_t b, const int64_t* x
     return off;
 }
 
+// Cuts every atom of the overlay of src and dst into 2-D slabs: (rows of the second-to-last dimension) x (contiguous run
+// of the last dimension), one per assignment of the outer dimensions, at most 64 KiB of source bytes each. Offsets and
+// pitches are in bytes of the respective relation (their element sizes may differ); row_bytes counts source bytes.
+// src_or / dst_or: OR of every quantity that limits the access width on that side.
+static void plan_slabs(const ja_relation* src, const ja_relation* dst, std::vector<CopySlab>* slabs, int64_t* src_or, int64_t* dst_or) {
+    std::vector<Atom> atoms;
+    build_atoms(src, dst, &atoms);
+    const int r = src->rank, es = src->esize, ed = dst->esize;
+    const int64_t slab_bytes = 64 * 1024;
+    for (const Atom& at : atoms) {
+        int64_t rows = r >= 2 ? at.hi[r - 2] - at.lo[r - 2] : 1;
+        int64_t row_bytes = (at.hi[r - 1] - at.lo[r - 1]) * es;
+        int64_t outer = 1;
+        for (int d = 0; d + 2 < r; ++d) outer *= at.hi[d] - at.lo[d];
+        int64_t rows_per = std::max<int64_t>(1, slab_bytes / row_bytes);
+        for (int64_t o = 0; o < outer; ++o) {
+            int64_t x[JA_MAX_RANK];
+            int64_t rem = o;
+            for (int d = r - 3; d >= 0; --d) {
+                int64_t e = at.hi[d] - at.lo[d];
+                x[d] = at.lo[d] + rem % e;
+                rem /= e;
+            }
+            for (int64_t r0 = 0; r0 < rows; r0 += rows_per) {
+                if (r >= 2) x[r - 2] = at.lo[r - 2] + r0;
+                x[r - 1] = at.lo[r - 1];
+                int64_t sw = 0, dw = 0;
+                CopySlab s;
+                s.src_off = src->blk_off[at.sb] + in_block_offset(src, at.sb, x, &sw) * es;
+                s.dst_off = dst->blk_off[at.db] + in_block_offset(dst, at.db, x, &dw) * ed;
+                s.rows = (int32_t)std::min(rows_per, rows - r0);
+                s.row_bytes = (int32_t)row_bytes;
+                s.src_pitch = (int32_t)(sw * es);
+                s.dst_pitch = (int32_t)(dw * ed);
+                *src_or |= s.src_off | s.row_bytes | s.src_pitch;
+                *dst_or |= s.dst_off | s.dst_pitch;
+                slabs->push_back(s);
+            }
+        }
+    }
+}
+
 extern "C" ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* dst, void* cuda_stream) {
     ja_status_t st = check_same_tensor(src, dst);
     if (st != JA_OK) return st;
@@ -558,43 +601,11 @@ extern "C" ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* d
         if (it != g_repart_plans.end()) plan = it->second;
     }
     if (!plan) {
-        std::vector<Atom> atoms;
-        build_atoms(src, dst, &atoms);
-        const int r = src->rank, es = src->esize;
+        const int es = src->esize;
         std::vector<CopySlab> slabs;
-        int64_t all_or = 0;  // OR of every quantity that limits the vector width
-        for (const Atom& at : atoms) {
-            // a slab = (rows of the second-to-last dimension) x (contiguous run of the last dimension),
-            // one per assignment of the outer dimensions
-            int64_t rows = r >= 2 ? at.hi[r - 2] - at.lo[r - 2] : 1;
-            int64_t row_bytes = (at.hi[r - 1] - at.lo[r - 1]) * es;
-            int64_t outer = 1;
-            for (int d = 0; d + 2 < r; ++d) outer *= at.hi[d] - at.lo[d];
-            int64_t rows_per = std::max<int64_t>(1, (64 * 1024) / row_bytes);
-            for (int64_t o = 0; o < outer; ++o) {
-                int64_t x[JA_MAX_RANK];
-                int64_t rem = o;
-                for (int d = r - 3; d >= 0; --d) {
-                    int64_t e = at.hi[d] - at.lo[d];
-                    x[d] = at.lo[d] + rem % e;
-                    rem /= e;
-                }
-                for (int64_t r0 = 0; r0 < rows; r0 += rows_per) {
-                    if (r >= 2) x[r - 2] = at.lo[r - 2] + r0;
-                    x[r - 1] = at.lo[r - 1];
-                    int64_t sw = 0, dw = 0;
-                    CopySlab s;
-                    s.src_off = src->blk_off[at.sb] + in_block_offset(src, at.sb, x, &sw) * es;
-                    s.dst_off = dst->blk_off[at.db] + in_block_offset(dst, at.db, x, &dw) * es;
-                    s.rows = (int32_t)std::min(rows_per, rows - r0);
-                    s.row_bytes = (int32_t)row_bytes;
-                    s.src_pitch = (int32_t)(sw * es);
-                    s.dst_pitch = (int32_t)(dw * es);
-                    all_or |= s.src_off | s.dst_off | s.row_bytes | s.src_pitch | s.dst_pitch;
-                    slabs.push_back(s);
-                }
-            }
-        }
+        int64_t src_or = 0, dst_or = 0;
+        plan_slabs(src, dst, &slabs, &src_or, &dst_or);
+        const int64_t all_or = src_or | dst_or;
         plan.reset(new RepartPlan());
         plan->vec_bytes = 16;
         while (plan->vec_bytes > es && (all_or % plan->vec_bytes) != 0) plan->vec_bytes /= 2;
@@ -606,6 +617,74 @@ extern "C" ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* d
     }
     return ja_launch_repartition((const char*)src->base, (char*)dst->base, plan->d_slabs, plan->n_slabs,
                                  plan->vec_bytes, (cudaStream_t)cuda_stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// aggregating relayout (Sections 5.1, 5.3): m unaggregated copies of every producer block -> aggregated consumer blocks
+// ---------------------------------------------------------------------------------------------------
+static std::map<std::vector<uint64_t>, std::shared_ptr<RepartPlan>> g_repart_agg_plans;
+
+// partials must be [c, x...] with the copy index c cut into its unit intervals and x... the tensor of `like`
+static ja_status_t check_partial_relation(const ja_relation* partials, const ja_relation* like, int like_rank, const int64_t* like_extent) {
+    if (!partials) return ja_fail(JA_ERR_INVALID_ARG, "partial relation is NULL");
+    if (partials->rank != like_rank + 1)
+        return ja_fail(JA_ERR_SHAPE, "a partial relation has the copy index in front: rank %d expected, got %d", like_rank + 1, partials->rank);
+    if (partials->nblk[0] != partials->extent[0])
+        return ja_fail(JA_ERR_TILING, "the copy index of a partial relation must be cut into unit intervals");
+    for (int d = 0; d < like_rank; ++d)
+        if (partials->extent[d + 1] != like_extent[d]) return ja_fail(JA_ERR_SHAPE, "extent of dimension %d differs", d);
+    (void)like;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_t agg, ja_relation_t* dst, void* cuda_stream) {
+    if (!dst) return ja_fail(JA_ERR_INVALID_ARG, "relation is NULL");
+    ja_status_t st = check_partial_relation(partials, dst, dst->rank, dst->extent);
+    if (st != JA_OK) return st;
+    const int m = (int)partials->extent[0];
+    if (agg != JA_AGG_SUM && agg != JA_AGG_MAX && !(agg == JA_AGG_NONE && m == 1))
+        return ja_fail(JA_ERR_INVALID_ARG, "%d copies of every atom need SUM or MAX aggregation", m);
+    if (partials->base == dst->base) return ja_fail(JA_ERR_INVALID_ARG, "repartition in place is not supported");
+    std::shared_ptr<RepartPlan> plan;
+    const std::vector<uint64_t> key = {partials->id, dst->id};
+    {
+        std::lock_guard<std::mutex> lk(g_repart_mu);
+        auto it = g_repart_agg_plans.find(key);
+        if (it != g_repart_agg_plans.end()) plan = it->second;
+    }
+    const int64_t ntrail = partials->nblocks / m;
+    const int64_t copy_stride = m > 1 ? partials->blk_off[ntrail] - partials->blk_off[0] : 0;
+    if (!plan) {
+        // copy 0 of the partial relation seen as a relation over the consumer's tensor
+        ja_relation view;
+        view.rank = dst->rank;
+        view.esize = partials->esize;
+        view.dtype = partials->dtype;
+        for (int d = 0; d < dst->rank; ++d) {
+            view.extent[d] = partials->extent[d + 1];
+            view.nblk[d] = partials->nblk[d + 1];
+            view.splits[d] = partials->splits[d + 1];
+        }
+        view.blk_off.assign(partials->blk_off.begin(), partials->blk_off.begin() + ntrail);
+        for (int c = 1; c < m; ++c)   // every copy has the block structure of copy 0, copy_stride bytes further on
+            for (int64_t b = 0; b < ntrail; ++b)
+                if (partials->blk_off[c * ntrail + b] != view.blk_off[b] + c * copy_stride)
+                    return ja_fail(JA_ERR_UNSUPPORTED, "copies of the partial relation are not equally spaced");
+        std::vector<CopySlab> slabs;
+        int64_t src_or = copy_stride, dst_or = 0;
+        plan_slabs(&view, dst, &slabs, &src_or, &dst_or);
+        const int vec = partials->esize == 4 ? 4 : 8;                       // cells per 16-byte source access
+        const int dst_access = std::min(16, vec * dst->esize);
+        plan.reset(new RepartPlan());
+        plan->vec_bytes = (src_or % 16 == 0 && dst_or % dst_access == 0) ? vec : 1;   // here: cells per access
+        plan->n_slabs = (int64_t)slabs.size();
+        JA_CUDA(cudaMalloc((void**)&plan->d_slabs, std::max<size_t>(1, slabs.size()) * sizeof(CopySlab)));
+        JA_CUDA(cudaMemcpy(plan->d_slabs, slabs.data(), slabs.size() * sizeof(CopySlab), cudaMemcpyHostToDevice));
+        std::lock_guard<std::mutex> lk(g_repart_mu);
+        g_repart_agg_plans[key] = plan;
+    }
+    return ja_launch_repartition_agg((const char*)partials->base, (char*)dst->base, plan->d_slabs, plan->n_slabs, m, copy_stride,
+                                     partials->dtype, dst->dtype, agg, plan->vec_bytes, (cudaStream_t)cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -889,4 +968,68 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
 
     return ja_fail(JA_ERR_UNSUPPORTED, "no kernel for einsum '%s' with fn %d / agg %d", spec->einsum.c_str(), (int)fn,
                    (int)agg);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// ja_execute_join: step (1) of Definition 3.7 alone (Section 5.1: a producer compiled through its join)
+// ---------------------------------------------------------------------------------------------------
+extern "C" ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,
+                                       ja_relation_t* partials, void* cuda_stream) {
+    if (!spec || !inputs || !partials) return ja_fail(JA_ERR_INVALID_ARG, "spec / inputs / partials is NULL");
+    const int n_in = (int)spec->ins.size();
+    if (n_inputs != n_in) return ja_fail(JA_ERR_INVALID_ARG, "spec has %d operands, %d relations given", n_in, n_inputs);
+    ja_status_t st;
+    for (int k = 0; k < n_in; ++k)
+        if ((st = check_tiling(spec, k, inputs[k])) != JA_OK) return st;
+    // multiplicity of every output type: the number of function specs that share it
+    int64_t n_out = 1;
+    for (char c : spec->out) n_out *= (int64_t)spec->parts[letter_pos(spec->letters, c)].size() - 1;
+    std::vector<int32_t> mult((size_t)n_out, 0);
+    for (int32_t k : spec->out_keys) ++mult[k];
+    const int32_t m = mult.empty() ? 0 : mult[0];
+    for (int32_t v : mult)
+        if (v != m) return ja_fail(JA_ERR_UNSUPPORTED, "output types have different multiplicities: no rectangular partial relation");
+    // partials: [c, out...], c cut into m unit intervals, the rest tiled as out(J)
+    const int orank = (int)spec->out.size();
+    int64_t oext[JA_MAX_RANK] = {0, 0, 0, 0};
+    for (int d = 0; d < orank; ++d) oext[d] = spec->parts[letter_pos(spec->letters, spec->out[d])].back();
+    if ((st = check_partial_relation(partials, nullptr, orank, oext)) != JA_OK) return st;
+    if (partials->extent[0] != m)
+        return ja_fail(JA_ERR_SHAPE, "every output type has %d function specs, the partial relation holds %lld copies", m, (long long)partials->extent[0]);
+    for (int d = 0; d < orank; ++d)
+        if (partials->splits[d + 1] != spec->parts[letter_pos(spec->letters, spec->out[d])])
+            return ja_fail(JA_ERR_PARTITION_MISMATCH, "the partial relation is not tiled as out(J) along index '%c'", spec->out[d]);
+    for (int k = 0; k < n_in; ++k)
+        if (inputs[k]->base == partials->base) return ja_fail(JA_ERR_INVALID_ARG, "output aliases input %d", k);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const std::vector<std::string>& in = spec->ins;
+    const std::string& o = spec->out;
+    for (int k = 0; k < n_in; ++k)
+        if ((st = ja_relation_to_device(inputs[k])) != JA_OK) return st;
+    if ((st = ja_relation_to_device(partials)) != JA_OK) return st;
+
+    if (spec->fn == JA_FN_MUL && spec->agg == JA_AGG_SUM && n_in == 2 && in[0].size() == 2 && in[1].size() == 2 && o.size() == 2 &&
+        in[0][1] == in[1][0] && o[0] == in[0][0] && o[1] == in[1][1] && in[0][0] != in[1][1]) {
+        const ja_relation *A = inputs[0], *B = inputs[1];
+        if (A->dtype != B->dtype) return ja_fail(JA_ERR_DTYPE, "matmul operands must share one dtype");
+        std::vector<uint64_t> key = {A->id, B->id, partials->id, ~(uint64_t)0};
+        std::shared_ptr<ExecPlan>& plan = spec->plans[key];
+        if (!plan) plan.reset(new ExecPlan());
+        if (A->dtype == JA_BF16) {
+            if (!plan->gemm_checked) {
+                bool ok = false;
+                GemmEpilogue ep;
+                memset(&ep, 0, sizeof ep);
+                ep.partials = 1;
+                if ((st = ja_gemm_tc_plan(A, B, partials, &ep, &plan->gemm, &ok)) != JA_OK) return st;
+                if (!ok) plan->gemm.reset();
+                plan->gemm_checked = true;
+            }
+            if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
+        }
+        if (partials->dtype != A->dtype) return ja_fail(JA_ERR_UNSUPPORTED, "this tiling needs a partial relation of the operands' dtype");
+        return ja_launch_matmul_simt(ja_view(A), ja_view(B), ja_view(partials), A->dtype, stream, true);
+    }
+    return ja_fail(JA_ERR_UNSUPPORTED, "join-only execution has no kernel for einsum '%s' with fn %d / agg %d", spec->einsum.c_str(),
+                   (int)spec->fn, (int)spec->agg);
 }

@@ -84,7 +84,7 @@ void ja_count_launch(int n = 1);
 // ---- kernel launchers (one per .cu file) ------------------------------------------------------------
 // Plain-ALU tiled matmul join-agg over arbitrary tilings (f32 or bf16 operands, f32 accumulate).
 ja_status_t ja_launch_matmul_simt(const RelView& A, const RelView& B, const RelView& C, ja_dtype_t dt,
-                                  cudaStream_t st);
+                                  cudaStream_t st, bool partials = false);
 
 // Memory-bound join-aggs: flat key-aligned maps and row-structured maps / reductions.
 enum RowOp {
@@ -102,6 +102,8 @@ struct RowArgs {
     int rope_d;                // extent of the rotated index d (rows may hold several heads of d cells each)
 };
 ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st);
+// bulk-copy pipelined form for uniform tilings; *launched stays false when the shape does not fit it
+ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched);
 ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,
                            cudaStream_t st);
 
@@ -113,6 +115,12 @@ struct CopySlab {
 };
 ja_status_t ja_launch_repartition(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int vec_bytes,
                                   cudaStream_t st);
+// Aggregating relayout: every slab is read from n_copies copies of the source, copy_stride bytes apart, (+)-combined
+// in ascending copy order in f32 and stored once. Slab sizes are in SOURCE bytes; destination offsets / pitches in
+// destination bytes. vec = cells per access (8 / 4 for 16-byte accesses of bf16 / f32 sources, or 1).
+ja_status_t ja_launch_repartition_agg(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int n_copies,
+                                      int64_t copy_stride, ja_dtype_t src_dt, ja_dtype_t dst_dt, ja_agg_t agg, int vec,
+                                      cudaStream_t st);
 
 // tcgen05 / TMEM / TMA matmul join-agg for bf16 relations with uniform blocks.
 struct GemmTcPlan;
@@ -125,6 +133,7 @@ struct GemmEpilogue {
     const ja_relation* B2;
     const float2* rope_table;
     int rope_S, rope_D;
+    int partials;   // join only: C is a partial relation [c, i, k] holding one copy per contracted block, nothing is summed across blocks
 };
 ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja_relation* C, const GemmEpilogue* ep,
                             std::shared_ptr<GemmTcPlan>* out, bool* eligible);

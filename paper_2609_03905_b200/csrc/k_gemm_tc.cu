@@ -63,6 +63,9 @@ struct GemmParams {
     // fused epilogue (a join-agg chain executed in one pass, the intermediate never stored)
     int32_t epi;               // EPI_*
     int32_t bn_tile;           // output columns per tile: 256, or 128 for EPI_SWIGLU (two 128-column products per tile)
+    int32_t n_copies;          // 1: SUM over all contracted blocks (aggregated output). nbk: join only -- tile (c, ., .) covers the
+                               // single contracted block c and is stored to copy c of a partial relation [c, i, k]
+    int32_t c_esize;           // bytes per output cell: 2 (bf16) or 4 (f32, partial relations only)
     const char* r_base;        // EPI_ADD: payload of the relation added to the product (tiled exactly like the output)
     const float2* rope_table;  // EPI_ROPE: (cos, sin)[position][pair]
     int32_t rope_S, rope_D;    // EPI_ROPE: positions per sequence (row % rope_S), rotated extent (column % rope_D)
@@ -76,11 +79,19 @@ struct TileCoord {
     int rows;            // valid rows (0..128)
     int n_g0, nb, c0;    // first global column of the tile / its column block / first column inside it
     int width;           // valid columns of the tile (multiple of 8)
+    int jb0, jb1;        // contracted blocks [jb0, jb1) accumulated into this tile
+    int copy;            // copy index of a partial relation (0 for an aggregated output)
 };
 
 template <int CG>
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int cta_rank) {
     TileCoord tc;
+    // join-only form: copies are the slowest tile coordinate, so tiles in flight share one contracted block
+    const int per_copy = p.m_tiles * p.n_tiles;
+    tc.copy = t / per_copy;
+    t -= tc.copy * per_copy;
+    tc.jb0 = p.n_copies > 1 ? tc.copy : 0;
+    tc.jb1 = p.n_copies > 1 ? tc.copy + 1 : p.nbk;
     // banded rasterisation: tiles that run at the same time cover group_m row tiles x several column tiles, so the
     // operand strips they stream fit in L2 together
     const int band_sz = p.group_m * p.n_tiles;
@@ -163,7 +174,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = p.m_tiles * p.n_tiles * p.n_copies;
     const int kchunks = (p.bk + Cfg<CG>::BK - 1) / Cfg<CG>::BK;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
@@ -184,7 +195,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int my_c0 = cta_rank * my_cols;              // their offset inside the tile
                 const int nchunks = (my_cols + 63) / 64;
                 const uint32_t tx = (uint32_t)CG * (A_STAGE_BYTES + nchunks * B_CHUNK_BYTES);
-                for (int jb = 0; jb < p.nbk && ok; ++jb) {          // the tuples of this output key, ascending j
+                for (int jb = tc.jb0; jb < tc.jb1 && ok; ++jb) {    // the tuples of this output key, ascending j
                     for (int kc = 0; kc < kchunks; ++kc) {
                         if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                         uint32_t fb = full_bar(stage);
@@ -242,7 +253,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 uint32_t accumulate = 0;
-                for (int jb = 0; jb < p.nbk && ok; ++jb) {
+                for (int jb = tc.jb0; jb < tc.jb1 && ok; ++jb) {
                     for (int kc = 0; kc < kchunks; ++kc) {
                         if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
@@ -302,9 +313,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (row_ok) {
                     const int gcol = tc.n_g0 + ch * 32;
                     const int kb = gcol / p.bn, cin = gcol % p.bn;
-                    const int64_t off = p.c_blk_off[(int64_t)ib * p.nbn + kb] + ((int64_t)iin * p.bn + cin) * 2;
+                    const int64_t off = p.c_blk_off[((int64_t)tc.copy * p.nbm + ib) * p.nbn + kb] + ((int64_t)iin * p.bn + cin) * p.c_esize;
                     char* dst = p.c_base + off;
                     const int valid = min(32, tc.width - ch * 32);  // multiple of 8
+                    if (p.c_esize == 4) {   // partial relation kept in f32: the accumulator is stored as it is
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (g * 4 < valid)
+                                *reinterpret_cast<uint4*>(dst + g * 16) = make_uint4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+                        continue;
+                    }
                     if (p.epi == EPI_ROPE) {
                         // rotate pairs (2p, 2p+1) by the angle of (position, pair): position = row inside its sequence
                         const float2* tab = p.rope_table + ((int64_t)(grow % p.rope_S) * p.rope_D + gcol % p.rope_D) / 2;
@@ -412,6 +430,9 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     p.a_box_rows = (int)std::min<int64_t>(bm, 128);
     p.epi = epi;
     p.bn_tile = bn_tile;
+    p.n_copies = (ep && ep->partials) ? p.nbk : 1;
+    p.c_esize = C->esize;
+    if (p.c_esize == 4 && !(ep && ep->partials)) return JA_OK;
     p.r_base = (epi == EPI_ADD) ? (const char*)ep->addend->base : nullptr;
     p.rope_table = (epi == EPI_ROPE) ? ep->rope_table : nullptr;
     p.rope_S = ep ? ep->rope_S : 1;
@@ -438,7 +459,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int tiles = p.m_tiles * p.n_tiles;
+    const int tiles = p.m_tiles * p.n_tiles * p.n_copies;
     plan->grid = two ? 2 * std::min(sms / 2, tiles) : std::min(sms, tiles);
     cudaError_t e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
                         : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES);

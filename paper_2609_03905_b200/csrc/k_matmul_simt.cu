@@ -4,6 +4,8 @@
 // aggregation over the function specs that share an output type (Definition 3.7, Example 3.8).
 // Used for f32 relations (tf32 tensor-core math cannot meet a 1e-5 bound) and as the fallback for
 // bf16 relations whose blocks the tensor-core path cannot address.
+// Join-only form (partials != 0): grid.z enumerates the contracted blocks; CTA (., ., c) multiplies block c alone and
+// stores copy c of the partial relation C[c, i, k] -- nothing is summed across function specs.
 #include "ja_device.cuh"
 
 namespace {
@@ -11,7 +13,7 @@ namespace {
 constexpr int TM = 64, TN = 64, TK = 16;
 
 template <typename T>
-__global__ void __launch_bounds__(256) matmul_simt_kernel(RelView A, RelView B, RelView C) {
+__global__ void __launch_bounds__(256) matmul_simt_kernel(RelView A, RelView B, RelView C, int partials) {
     __shared__ float As[TK][TM + 4];
     __shared__ float Bs[TK][TN + 4];
     const int tid = threadIdx.x;
@@ -24,7 +26,8 @@ __global__ void __launch_bounds__(256) matmul_simt_kernel(RelView A, RelView B, 
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
-    for (int jb = 0; jb < A.nblk[1]; ++jb) {  // the tuples of this output key, ascending
+    const int jb_lo = partials ? (int)blockIdx.z : 0, jb_hi = partials ? (int)blockIdx.z + 1 : A.nblk[1];
+    for (int jb = jb_lo; jb < jb_hi; ++jb) {  // the tuples of this output key, ascending
         const int64_t jlo = A.splits[1][jb], jhi = A.splits[1][jb + 1];
         for (int64_t j0 = jlo; j0 < jhi; j0 += TK) {
             for (int e = tid; e < TM * TK; e += 256) {
@@ -62,17 +65,21 @@ __global__ void __launch_bounds__(256) matmul_simt_kernel(RelView A, RelView B, 
     for (int u = 0; u < 4; ++u)
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-            int64_t x[2] = {i0 + tr * 4 + u, k0 + tc * 4 + w};
-            if (x[0] < M && x[1] < N) *(T*)(C.base + ja_elem_off(C, x)) = ja_from_float<T>(acc[u][w]);
+            int64_t x[3] = {i0 + tr * 4 + u, k0 + tc * 4 + w, 0};
+            if (x[0] < M && x[1] < N) {
+                if (partials) { x[2] = x[1]; x[1] = x[0]; x[0] = blockIdx.z; }
+                *(T*)(C.base + ja_elem_off(C, x)) = ja_from_float<T>(acc[u][w]);
+            }
         }
 }
 
 }  // namespace
 
-ja_status_t ja_launch_matmul_simt(const RelView& A, const RelView& B, const RelView& C, ja_dtype_t dt, cudaStream_t st) {
-    dim3 grid((unsigned)((B.extent[1] + TN - 1) / TN), (unsigned)((A.extent[0] + TM - 1) / TM));
-    if (dt == JA_F32) matmul_simt_kernel<float><<<grid, 256, 0, st>>>(A, B, C);
-    else matmul_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(A, B, C);
+ja_status_t ja_launch_matmul_simt(const RelView& A, const RelView& B, const RelView& C, ja_dtype_t dt, cudaStream_t st,
+                                  bool partials) {
+    dim3 grid((unsigned)((B.extent[1] + TN - 1) / TN), (unsigned)((A.extent[0] + TM - 1) / TM), partials ? (unsigned)A.nblk[1] : 1u);
+    if (dt == JA_F32) matmul_simt_kernel<float><<<grid, 256, 0, st>>>(A, B, C, partials ? 1 : 0);
+    else matmul_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(A, B, C, partials ? 1 : 0);
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
     return JA_OK;

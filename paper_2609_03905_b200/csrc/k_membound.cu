@@ -575,6 +575,12 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
     if (n_rows >= (1ll << 31) || n >= (1ll << 31)) return ja_fail(JA_ERR_UNSUPPORTED, "row-structured join-agg: extents must be < 2^31");
     const int full = dt == JA_F32 ? 4 : 8;
     const int es = dt == JA_F32 ? 4 : 2;
+    // ---- uniform tilings: bulk-copy pipeline through shared memory ---------------------------------------------
+    {
+        bool launched = false;
+        ja_status_t s = ja_launch_row_tma(op, a, dt, st, &launched);
+        if (s != JA_OK || launched) return s;
+    }
     // ---- fast path: every block of x (and of g, and of the statistics relations) has the same shape --------
     const bool has_g = (op == ROW_RMS_SCALE || op == ROW_RMSNORM);
     const bool has_stat = (op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM || op == ROW_RMS_SCALE || op == ROW_EXP_SUB_DIV);

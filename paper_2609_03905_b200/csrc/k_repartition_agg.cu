@@ -1,0 +1,120 @@
+// Aggregating relayout (Sections 5.1 and 5.3): a producer that was executed through its join only leaves, for every
+// output block, m unaggregated copies. The consumer needs every block of ITS tiling fully aggregated. The overlay of
+// the two tilings gives atoms; each atom is cut into 2-D slabs exactly as in the plain relayout, and for every cell of
+// a slab the m copies are read ("decompose"), (+)-combined in ascending copy order in f32 ("aggregate") and stored
+// once, rounded once, at the cell's place in the consumer's block ("recompose"). One pass, no staging buffer.
+// HBM-bound: m source cells read and one destination cell written per cell.
+#include "ja_device.cuh"
+
+namespace {
+
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int N = 4; };            // 16 bytes
+template <> struct VecOf<__nv_bfloat16> { static constexpr int N = 8; };    // 16 bytes
+
+template <typename TS, int VEC> __device__ __forceinline__ void load_cells(const char* p, float* f) {
+    if (VEC == 1) {
+        f[0] = ja_to_float(*reinterpret_cast<const TS*>(p));
+    } else {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+        if (sizeof(TS) == 4) {
+            f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+        } else {
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 t = __bfloat1622float2(h[e]);
+                f[2 * e] = t.x;
+                f[2 * e + 1] = t.y;
+            }
+        }
+    }
+}
+
+template <typename TD, int VEC> __device__ __forceinline__ void store_cells(char* p, const float* f) {
+    if (VEC == 1) {
+        *reinterpret_cast<TD*>(p) = ja_from_float<TD>(f[0]);
+    } else if (sizeof(TD) == 4) {
+#pragma unroll
+        for (int e = 0; e < VEC; e += 4) *reinterpret_cast<float4*>(p + e * 4) = make_float4(f[e], f[e + 1], f[e + 2], f[e + 3]);
+    } else if (VEC == 8) {
+        uint4 o;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+        *reinterpret_cast<uint4*>(p) = o;
+    } else {   // 4 bf16 cells
+        uint2 o;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+        h[0] = __floats2bfloat162_rn(f[0], f[1]);
+        h[1] = __floats2bfloat162_rn(f[2], f[3]);
+        *reinterpret_cast<uint2*>(p) = o;
+    }
+}
+
+template <bool IS_MAX> __device__ __forceinline__ float combine(float a, float b) { return IS_MAX ? fmaxf(a, b) : a + b; }
+
+template <typename TS, typename TD, int VEC, bool IS_MAX>
+__global__ void __launch_bounds__(256) repartition_agg_kernel(const char* __restrict__ src, char* __restrict__ dst,
+                                                              const CopySlab* __restrict__ slabs, int64_t n_slabs, int n_copies,
+                                                              int64_t copy_stride) {
+    for (int64_t s = blockIdx.x; s < n_slabs; s += gridDim.x) {
+        const CopySlab sl = slabs[s];
+        const int vpr = sl.row_bytes / (int)(VEC * sizeof(TS));  // accesses per row
+        const int total = vpr * sl.rows;
+        for (int i = threadIdx.x; i < total; i += 256) {
+            const int r = i / vpr, c = i - r * vpr;
+            const char* sp = src + sl.src_off + (int64_t)r * sl.src_pitch + (int64_t)c * (VEC * sizeof(TS));
+            float acc[VEC];
+            load_cells<TS, VEC>(sp, acc);
+            int cc = 1;
+            for (; cc + 3 < n_copies; cc += 4) {   // four copies in flight, combined in ascending order
+                float t0[VEC], t1[VEC], t2[VEC], t3[VEC];
+                load_cells<TS, VEC>(sp + (int64_t)cc * copy_stride, t0);
+                load_cells<TS, VEC>(sp + (int64_t)(cc + 1) * copy_stride, t1);
+                load_cells<TS, VEC>(sp + (int64_t)(cc + 2) * copy_stride, t2);
+                load_cells<TS, VEC>(sp + (int64_t)(cc + 3) * copy_stride, t3);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e)
+                    acc[e] = combine<IS_MAX>(combine<IS_MAX>(combine<IS_MAX>(combine<IS_MAX>(acc[e], t0[e]), t1[e]), t2[e]), t3[e]);
+            }
+            for (; cc < n_copies; ++cc) {
+                float t[VEC];
+                load_cells<TS, VEC>(sp + (int64_t)cc * copy_stride, t);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] = combine<IS_MAX>(acc[e], t[e]);
+            }
+            store_cells<TD, VEC>(dst + sl.dst_off + (int64_t)r * sl.dst_pitch + (int64_t)c * (VEC * sizeof(TD)), acc);
+        }
+    }
+}
+
+template <typename TS, typename TD>
+void launch(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int n_copies, int64_t copy_stride, bool is_max,
+            bool vec, unsigned grid, cudaStream_t st) {
+    constexpr int V = VecOf<TS>::N;
+    if (vec) {
+        if (is_max) repartition_agg_kernel<TS, TD, V, true><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+        else repartition_agg_kernel<TS, TD, V, false><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+    } else {
+        if (is_max) repartition_agg_kernel<TS, TD, 1, true><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+        else repartition_agg_kernel<TS, TD, 1, false><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+    }
+}
+
+}  // namespace
+
+ja_status_t ja_launch_repartition_agg(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int n_copies,
+                                      int64_t copy_stride, ja_dtype_t src_dt, ja_dtype_t dst_dt, ja_agg_t agg, int vec,
+                                      cudaStream_t st) {
+    if (n_slabs == 0) return JA_OK;
+    const unsigned grid = (unsigned)(n_slabs < (int64_t)148 * 64 ? n_slabs : (int64_t)148 * 64);
+    const bool is_max = agg == JA_AGG_MAX, v = vec > 1;
+    if (src_dt == JA_F32 && dst_dt == JA_F32) launch<float, float>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
+    else if (src_dt == JA_F32) launch<float, __nv_bfloat16>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
+    else if (dst_dt == JA_F32) launch<__nv_bfloat16, float>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
+    else launch<__nv_bfloat16, __nv_bfloat16>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
+    ja_count_launch();
+    JA_CUDA(cudaGetLastError());
+    return JA_OK;
+}

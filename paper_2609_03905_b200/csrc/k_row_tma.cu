@@ -1,0 +1,551 @@
+// Row-structured join-aggs ("Rj..." forms) on uniform tilings, staged through shared memory by bulk asynchronous
+// copies. These operators move a few bytes per flop, so the only thing that matters is how many bytes are in flight:
+// a thread that loads its cells into registers, reduces and stores keeps a few hundred bytes in flight; a ring of
+// shared-memory stages filled by cp.async.bulk keeps 100-200 KiB in flight per SM with one issuing thread.
+//
+// Layout fact used: inside a block the cells of consecutive rows of one column block are contiguous, so the R rows of
+// a work unit are nbc contiguous segments (one per column block) -- nbc bulk copies in, nbc bulk copies out.
+//
+//   warps 0..7  consumers: warp w owns rows w, w+8, ... of the stage. It walks the row's column blocks in ascending
+//               order -- for the reductions (SQUARE/SUM, IDENT/MAX, EXP_SUB/SUM) that walk is the aggregation over the
+//               function specs that share the row's output key -- and, for the maps, writes the result over the input
+//               in shared memory.
+//   warp 8      loader: one thread issues the bulk loads of a unit into a free stage (mbarrier complete_tx).
+//   warp 9      storer (maps only): when the eight consumer warps are done with a stage, one thread issues the bulk
+//               stores of the stage and frees it once the copies have read shared memory.
+// Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT, waits (bounded) for its loads in flight
+// and leaves through the normal exit.
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include "ja_device.cuh"
+#include "ja_ptx.cuh"
+
+namespace {
+
+using namespace ja_ptx;
+
+constexpr int CONSUMER_WARPS = 8;
+constexpr int NUM_THREADS = (CONSUMER_WARPS + 2) * 32;
+constexpr int MAX_STAGES = 6;
+
+struct RowTmaGeom {
+    int n, bsc, nbc;             // row length, column-block width, column blocks (cells)
+    int rows_per_blk;            // rows (flattened leading coordinates) inside one block
+    int chunks_per_blk;          // work units per strip of nbc blocks
+    int R;                       // rows per unit (the last unit of a block may hold fewer)
+    int stages;
+    int64_t n_units;
+    int64_t blk_bytes;           // bytes between consecutive blocks of x / y
+    int seg_bytes;               // shared-memory bytes of one column-block segment of a stage: R * bsc * sizeof(T)
+    int stage_bytes;             // nbc * seg_bytes
+    int stat_blk_bytes;          // bytes between consecutive blocks of a statistics relation
+    int g_blk_bytes;             // bytes between consecutive blocks of the gain vector
+    float eps;
+};
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <typename T, int VEC> struct alignas(sizeof(T) * VEC) RVec { T e[VEC]; };
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ---- one row, any cell type: plain scalar arithmetic --------------------------------------------------------
+template <typename T, int OP, int VPL>
+__device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL],
+                                            const uint8_t* g_s, int64_t stat_off, int lane) {
+    constexpr int VEC = 16 / (int)sizeof(T);
+    using V = RVec<T, VEC>;
+    constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
+    constexpr bool HAS_Y = !(OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM);
+    constexpr bool KEEP_EXP = (OP == ROW_SOFTMAX);
+    float m = 0.f, l = 0.f, rstd = 0.f;
+    float ex[KEEP_EXP ? VPL * VEC : 1];
+    if (OP == ROW_SUMSQ || OP == ROW_RMSNORM) {
+        float sacc = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const V v = *reinterpret_cast<const V*>(rowp + off[k]);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { const float f = ja_to_float(v.e[e]); sacc = fmaf(f, f, sacc); }
+            }
+        sacc = warp_sum(sacc);
+        if (OP == ROW_SUMSQ) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
+            return;
+        }
+        rstd = 1.0f / sqrtf(sacc / (float)g.n + g.eps);
+    }
+    if (OP == ROW_MAX || OP == ROW_SOFTMAX) {
+        float mx = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const V v = *reinterpret_cast<const V*>(rowp + off[k]);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) mx = fmaxf(mx, ja_to_float(v.e[e]));
+            }
+        m = warp_max(mx);
+        if (OP == ROW_MAX) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+            return;
+        }
+    }
+    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+    if (OP == ROW_EXPSUM || OP == ROW_SOFTMAX) {
+        float sacc = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const V v = *reinterpret_cast<const V*>(rowp + off[k]);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    const float p = __expf(ja_to_float(v.e[e]) - m);
+                    if (KEEP_EXP) ex[k * VEC + e] = p;
+                    sacc += p;
+                }
+            }
+        l = warp_sum(sacc);
+        if (OP == ROW_EXPSUM) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+            return;
+        }
+    }
+    if (OP == ROW_EXP_SUB_DIV) l = *reinterpret_cast<const float*>(a.s1.base + stat_off);
+    if (OP == ROW_RMS_SCALE) {
+        const float ss = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+        rstd = 1.0f / sqrtf(ss / (float)g.n + g.eps);
+    }
+    const float inv_l = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : 0.f;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        if (off[k] < 0) continue;
+        V o;
+        if (HAS_G) {
+            const V v = *reinterpret_cast<const V*>(rowp + off[k]);
+            const V gv = *reinterpret_cast<const V*>(g_s + (size_t)(lane + 32 * k) * 16);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(ja_to_float(v.e[e]) * rstd * ja_to_float(gv.e[e]));
+        } else if (OP == ROW_SOFTMAX) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(ex[KEEP_EXP ? k * VEC + e : 0] * inv_l);
+        } else if (OP == ROW_EXP_SUB_DIV) {
+            const V v = *reinterpret_cast<const V*>(rowp + off[k]);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(__expf(ja_to_float(v.e[e]) - m) * inv_l);
+        }
+        if (HAS_Y) *reinterpret_cast<V*>(rowp + off[k]) = o;
+    }
+}
+
+// ---- one row of bf16 cells: the same arithmetic with few instructions per cell -----------------------------------
+// bf16 -> f32 is a shift or a mask; MAX runs on packed bf16 pairs (exact); products, sums and the exponent argument
+// run on packed f32 pairs. exp(x - m) is ex2(x log2e - m log2e), one multiply-add and one special-function op.
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t x, uint64_t y, uint64_t z) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(x), "l"(y), "l"(z));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t x, uint64_t y) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(x), "l"(y));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t x, uint64_t y) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(x), "l"(y));
+    return d;
+}
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint64_t widen(uint32_t w) { return pk2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)); }
+__device__ __forceinline__ uint32_t narrow(uint64_t v) {   // two f32 -> packed bf16, round to nearest even
+    float lo, hi;
+    upk2(v, lo, hi);
+    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&t);
+}
+
+template <int OP, int VPL>
+__device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL], const uint8_t* g_s,
+                                         int64_t stat_off, int lane) {
+    constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
+    constexpr bool KEEP_EXP = (OP == ROW_SOFTMAX);
+    constexpr float LOG2E = 1.4426950408889634f;
+    float m = 0.f, l = 0.f, rstd = 0.f;
+    uint64_t ex[KEEP_EXP ? VPL * 4 : 1];
+    if (OP == ROW_SUMSQ || OP == ROW_RMSNORM) {
+        uint64_t acc0 = pk2(0.f, 0.f), acc1 = pk2(0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
+                const uint64_t f0 = widen(v.x), f1 = widen(v.y), f2 = widen(v.z), f3 = widen(v.w);
+                acc0 = fma2(f0, f0, acc0);
+                acc1 = fma2(f1, f1, acc1);
+                acc0 = fma2(f2, f2, acc0);
+                acc1 = fma2(f3, f3, acc1);
+            }
+        float s0, s1, s2, s3;
+        upk2(acc0, s0, s1);
+        upk2(acc1, s2, s3);
+        const float sacc = warp_sum((s0 + s1) + (s2 + s3));
+        if (OP == ROW_SUMSQ) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
+            return;
+        }
+        rstd = 1.0f / sqrtf(sacc / (float)g.n + g.eps);
+    }
+    if (OP == ROW_MAX || OP == ROW_SOFTMAX) {
+        __nv_bfloat162 mx = __float2bfloat162_rn(-INFINITY);
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+                mx = __hmax2(__hmax2(mx, h[0]), __hmax2(h[1], __hmax2(h[2], h[3])));
+            }
+        const float2 mf = __bfloat1622float2(mx);
+        m = warp_max(fmaxf(mf.x, mf.y));
+        if (OP == ROW_MAX) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+            return;
+        }
+    }
+    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+    const uint64_t sc2 = pk2(LOG2E, LOG2E), nm2 = pk2(-m * LOG2E, -m * LOG2E);
+    auto exp_pair = [&](uint32_t w) {
+        float t0, t1;
+        upk2(fma2(widen(w), sc2, nm2), t0, t1);
+        return pk2(ex2f(t0), ex2f(t1));
+    };
+    if (OP == ROW_EXPSUM || OP == ROW_SOFTMAX) {
+        uint64_t acc0 = pk2(0.f, 0.f), acc1 = pk2(0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (off[k] >= 0) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
+                const uint64_t e0 = exp_pair(v.x), e1 = exp_pair(v.y), e2 = exp_pair(v.z), e3 = exp_pair(v.w);
+                if (KEEP_EXP) { ex[k * 4] = e0; ex[k * 4 + 1] = e1; ex[k * 4 + 2] = e2; ex[k * 4 + 3] = e3; }
+                acc0 = add2(acc0, e0);
+                acc1 = add2(acc1, e1);
+                acc0 = add2(acc0, e2);
+                acc1 = add2(acc1, e3);
+            }
+        float s0, s1, s2, s3;
+        upk2(acc0, s0, s1);
+        upk2(acc1, s2, s3);
+        l = warp_sum((s0 + s1) + (s2 + s3));
+        if (OP == ROW_EXPSUM) {
+            if (lane == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+            return;
+        }
+    }
+    if (OP == ROW_EXP_SUB_DIV) l = *reinterpret_cast<const float*>(a.s1.base + stat_off);
+    if (OP == ROW_RMS_SCALE) {
+        const float ss = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+        rstd = 1.0f / sqrtf(ss / (float)g.n + g.eps);
+    }
+    const float scale = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : rstd;
+    const uint64_t scale2 = pk2(scale, scale);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        if (off[k] < 0) continue;
+        uint4 o;
+        if (HAS_G) {
+            const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
+            const uint4 gv = *reinterpret_cast<const uint4*>(g_s + (size_t)(lane + 32 * k) * 16);
+            o.x = narrow(mul2(mul2(widen(v.x), scale2), widen(gv.x)));
+            o.y = narrow(mul2(mul2(widen(v.y), scale2), widen(gv.y)));
+            o.z = narrow(mul2(mul2(widen(v.z), scale2), widen(gv.z)));
+            o.w = narrow(mul2(mul2(widen(v.w), scale2), widen(gv.w)));
+        } else if (OP == ROW_SOFTMAX) {
+            o.x = narrow(mul2(ex[KEEP_EXP ? k * 4 : 0], scale2));
+            o.y = narrow(mul2(ex[KEEP_EXP ? k * 4 + 1 : 0], scale2));
+            o.z = narrow(mul2(ex[KEEP_EXP ? k * 4 + 2 : 0], scale2));
+            o.w = narrow(mul2(ex[KEEP_EXP ? k * 4 + 3 : 0], scale2));
+        } else {   // ROW_EXP_SUB_DIV
+            const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
+            o.x = narrow(mul2(exp_pair(v.x), scale2));
+            o.y = narrow(mul2(exp_pair(v.y), scale2));
+            o.z = narrow(mul2(exp_pair(v.z), scale2));
+            o.w = narrow(mul2(exp_pair(v.w), scale2));
+        }
+        *reinterpret_cast<uint4*>(rowp + off[k]) = o;
+    }
+}
+
+// VPL = 16-byte vectors per lane covering one row (lane + 32 k, k < VPL)
+// CTAs per SM: two, so that sixteen consumer warps share an SM's issue slots and special-function unit; one for the
+// softmax of very long rows, whose exponentials fill the register file
+template <typename T, int OP, int VPL> constexpr int ctas_per_sm() { return (OP == ROW_SOFTMAX && VPL * sizeof(T) >= 32) ? 1 : 2; }
+
+template <typename T, int OP, int VPL>
+__global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_tma_kernel(RowArgs a, RowTmaGeom g, int32_t* status) {
+    constexpr int VEC = 16 / (int)sizeof(T);
+    using V = RVec<T, VEC>;
+    constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
+    constexpr bool HAS_Y = !(OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM);
+    extern __shared__ __align__(128) uint8_t smem[];
+    // [stages][nbc][R][bsc] cells, then the gain vector [n], then the barriers
+    const uint32_t s_stage0 = smem_u32(smem);
+    uint8_t* g_s = smem + (size_t)g.stages * g.stage_bytes;
+    const size_t g_bytes = HAS_G ? ((size_t)g.n * sizeof(T) + 127) / 128 * 128 : 0;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(g_s + g_bytes);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto done_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };       // consumers -> storer
+    auto free_bar = [&](int s) { return bar0 + 8u * (2 * MAX_STAGES + s); };   // storer (or consumers) -> loader
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 3 * MAX_STAGES);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(done_bar(s), CONSUMER_WARPS);
+            mbar_init(free_bar(s), HAS_Y ? 1 : CONSUMER_WARPS);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (HAS_G && warp < CONSUMER_WARPS) {   // the gain vector, dense, once per CTA; the loader is already fetching rows meanwhile
+        for (int v = threadIdx.x; v * VEC < g.n; v += CONSUMER_WARPS * 32) {
+            const int col = v * VEC, cb = col / g.bsc, ci = col - cb * g.bsc;
+            *reinterpret_cast<V*>(g_s + (size_t)col * sizeof(T)) =
+                *reinterpret_cast<const V*>(a.g.base + (int64_t)cb * g.g_blk_bytes + (int64_t)ci * sizeof(T));
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(CONSUMER_WARPS * 32) : "memory");
+    }
+
+    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int row_seg_bytes = g.bsc * (int)sizeof(T);   // bytes of one row inside one column-block segment
+
+    // unit -> (strip of blocks, first row inside the block, rows)
+    auto unit_geom = [&](int64_t u, int64_t* lb, int* r0, int* rows) {
+        *lb = u / g.chunks_per_blk;
+        const int ch = (int)(u - *lb * g.chunks_per_blk);
+        *r0 = ch * g.R;
+        *rows = min(g.R, g.rows_per_blk - *r0);
+    };
+
+    if (warp == CONSUMER_WARPS) {
+        // ================= loader =================
+        if (lane == 0) {
+            bool ok = true;
+            int64_t i = 0;
+            for (int64_t u = first; u < g.n_units && ok; u += step, ++i) {
+                const int s = (int)(i % g.stages);
+                const uint32_t ph = (uint32_t)(i / g.stages) & 1;
+                if (i >= g.stages && !mbar_wait(free_bar(s), ph ^ 1, abort_flag, status)) { ok = false; break; }
+                int64_t lb;
+                int r0, rows;
+                unit_geom(u, &lb, &r0, &rows);
+                const uint32_t bytes = (uint32_t)(rows * row_seg_bytes);
+                mbar_expect_tx(full_bar(s), bytes * (uint32_t)g.nbc);
+                const char* src = a.x.base + lb * g.nbc * g.blk_bytes + (int64_t)r0 * row_seg_bytes;
+                const uint32_t dst = s_stage0 + (uint32_t)s * g.stage_bytes;
+                for (int cb = 0; cb < g.nbc; ++cb) bulk_load(dst + cb * g.seg_bytes, src + cb * g.blk_bytes, bytes, full_bar(s));
+            }
+            if (!ok) {   // loads already issued still write shared memory: wait (bounded) for them before leaving
+                for (int64_t j = i > g.stages ? i - g.stages : 0; j < i; ++j) {
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(full_bar((int)(j % g.stages)), (uint32_t)(j / g.stages) & 1) && global_ns() - t0 < 200000000ull) {}
+                }
+            }
+        }
+    } else if (warp == CONSUMER_WARPS + 1) {
+        // ================= storer =================
+        if (HAS_Y && lane == 0) {
+            bool ok = true;
+            int64_t i = 0;
+            for (int64_t u = first; u < g.n_units && ok; u += step, ++i) {
+                const int s = (int)(i % g.stages);
+                const uint32_t ph = (uint32_t)(i / g.stages) & 1;
+                if (!mbar_wait(done_bar(s), ph, abort_flag, status)) { ok = false; break; }
+                int64_t lb;
+                int r0, rows;
+                unit_geom(u, &lb, &r0, &rows);
+                const uint32_t bytes = (uint32_t)(rows * row_seg_bytes);
+                char* dstp = a.y.base + lb * g.nbc * g.blk_bytes + (int64_t)r0 * row_seg_bytes;
+                const uint32_t src = s_stage0 + (uint32_t)s * g.stage_bytes;
+                for (int cb = 0; cb < g.nbc; ++cb) bulk_store(dstp + cb * g.blk_bytes, src + cb * g.seg_bytes, bytes);
+                bulk_commit();
+                bulk_wait_read0();                 // the copies have read the stage: it may be refilled
+                mbar_arrive(free_bar(s));
+            }
+            bulk_wait0();
+        }
+    } else {
+        // ================= consumers =================
+        int off[VPL];   // byte offset of this lane's k-th vector inside a row of the stage (column block + column), or -1
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int col = (lane + 32 * k) * VEC;
+            off[k] = -1;
+            if (col < g.n) {
+                const int cb = col / g.bsc, ci = col - cb * g.bsc;
+                off[k] = cb * g.seg_bytes + ci * (int)sizeof(T);
+            }
+        }
+        bool ok = true;
+        int64_t i = 0;
+        for (int64_t u = first; u < g.n_units && ok; u += step, ++i) {
+            const int s = (int)(i % g.stages);
+            const uint32_t ph = (uint32_t)(i / g.stages) & 1;
+            if (!mbar_wait(full_bar(s), ph, abort_flag, status)) { ok = false; break; }
+            int64_t lb;
+            int r0, rows;
+            unit_geom(u, &lb, &r0, &rows);
+            uint8_t* stage = smem + (size_t)s * g.stage_bytes;
+            for (int r = warp; r < rows; r += CONSUMER_WARPS) {
+                uint8_t* rowp = stage + (size_t)r * row_seg_bytes;
+                const int64_t stat_off = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
+                if constexpr (sizeof(T) == 2) row_bf16<OP, VPL>(a, g, rowp, off, g_s, stat_off, lane);
+                else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, lane);
+            }
+            if (HAS_Y) fence_async_smem();    // this thread's writes to the stage become visible to the bulk stores
+            __syncwarp();
+            if (lane == 0) mbar_arrive(HAS_Y ? done_bar(s) : free_bar(s));
+        }
+    }
+}
+
+template <typename T, int OP, int VPL>
+ja_status_t launch_v(const RowArgs& a, RowTmaGeom g, int g_bytes, int sms, int32_t* status, cudaStream_t st, bool* launched) {
+    constexpr int CTAS = ctas_per_sm<T, OP, VPL>();
+    const int budget = (CTAS == 2 ? 100 : 200) * 1024 - g_bytes;
+    g.stages = (int)std::min<int64_t>(MAX_STAGES, budget / g.stage_bytes);
+    if (g.stages < 2) { *launched = false; return JA_OK; }
+    static bool configured = false;   // per template instance
+    if (!configured) {
+        JA_CUDA(cudaFuncSetAttribute(row_tma_kernel<T, OP, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024 + 1024));
+        configured = true;
+    }
+    const int smem_bytes = g.stages * g.stage_bytes + g_bytes + (3 * MAX_STAGES + 2) * 8;
+    const unsigned grid = (unsigned)std::min<int64_t>(g.n_units, (int64_t)sms * CTAS);
+    row_tma_kernel<T, OP, VPL><<<grid, NUM_THREADS, smem_bytes, st>>>(a, g, status);
+    return JA_OK;
+}
+
+template <typename T, int OP>
+ja_status_t launch_op(const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms, int32_t* status, cudaStream_t st,
+                      bool* launched) {
+    *launched = true;
+    if (vpl <= 1) return launch_v<T, OP, 1>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 2) return launch_v<T, OP, 2>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 4) return launch_v<T, OP, 4>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 8) return launch_v<T, OP, 8>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 16) return launch_v<T, OP, 16>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 32 && OP != ROW_SOFTMAX) return launch_v<T, OP, (OP != ROW_SOFTMAX ? 32 : 16)>(a, g, g_bytes, sms, status, st, launched);
+    *launched = false;
+    return JA_OK;
+}
+
+template <typename T>
+ja_status_t launch_t(RowOp op, const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms, int32_t* status,
+                     cudaStream_t st, bool* launched) {
+    switch (op) {
+        case ROW_SUMSQ: return launch_op<T, ROW_SUMSQ>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_MAX: return launch_op<T, ROW_MAX>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_EXPSUM: return launch_op<T, ROW_EXPSUM>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_RMS_SCALE: return launch_op<T, ROW_RMS_SCALE>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_EXP_SUB_DIV: return launch_op<T, ROW_EXP_SUB_DIV>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_RMSNORM: return launch_op<T, ROW_RMSNORM>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_SOFTMAX: return launch_op<T, ROW_SOFTMAX>(a, g, vpl, g_bytes, sms, status, st, launched);
+        default: break;
+    }
+    *launched = false;
+    return JA_OK;
+}
+
+}  // namespace
+
+// Sets *launched when this form took the job; leaves it false (and launches nothing) when the shape does not fit:
+// blocks of different shapes, rows longer than 32 vectors per lane, column blocks that are not whole 16-byte vectors,
+// RoPE (its rotation needs the row's coordinates).
+ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched) {
+    *launched = false;
+    if (op == ROW_ROPE) return JA_OK;
+    const char* off_env = getenv("JA_ROW_TMA");
+    if (off_env && off_env[0] == '0') return JA_OK;
+    const int last = a.x.rank - 1;
+    const int es = dt == JA_F32 ? 4 : 2, vec = 16 / es;
+    const bool has_g = (op == ROW_RMS_SCALE || op == ROW_RMSNORM);
+    const bool has_stat = (op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM || op == ROW_RMS_SCALE || op == ROW_EXP_SUB_DIV);
+    const bool two_stats = (op == ROW_EXPSUM || op == ROW_EXP_SUB_DIV);
+    const bool has_y = !(op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM);
+    if (!a.x.blk_stride || a.x.bs[last] % vec != 0) return JA_OK;
+    if (has_y && a.y.blk_stride != a.x.blk_stride) return JA_OK;
+    if (has_g && !a.g.blk_stride) return JA_OK;
+    if (has_stat && !a.s0.blk_stride) return JA_OK;
+    if (two_stats && a.s1.blk_stride != a.s0.blk_stride) return JA_OK;
+    RowTmaGeom g;
+    memset(&g, 0, sizeof g);
+    const int64_t n = a.x.extent[last];
+    g.n = (int)n;
+    g.bsc = (int)a.x.bs[last];
+    g.nbc = a.x.nblk[last];
+    int64_t rows_per_blk = 1, n_lead = 1;
+    for (int d = 0; d < last; ++d) { rows_per_blk *= a.x.bs[d]; n_lead *= a.x.nblk[d]; }
+    if (rows_per_blk >= (1 << 30) || n >= (1 << 24)) return JA_OK;
+    g.rows_per_blk = (int)rows_per_blk;
+    g.blk_bytes = a.x.blk_stride;
+    const int64_t row_bytes = n * es;
+    const int vpl = (int)((n + vec * 32 - 1) / (vec * 32));
+    if (vpl > 32 || (vpl > 16 && op == ROW_SOFTMAX)) return JA_OK;
+    // rows per unit: the largest power of two (at most 32, at most a block holds) that keeps a stage within 32 KiB
+    int R = 1;
+    while (R < 32 && (int64_t)R * 2 * row_bytes <= 32 * 1024 && R * 2 <= rows_per_blk) R *= 2;
+    g.R = R;
+    g.chunks_per_blk = (int)((rows_per_blk + R - 1) / R);
+    g.n_units = n_lead * g.chunks_per_blk;
+    g.seg_bytes = R * g.bsc * es;
+    g.stage_bytes = g.nbc * g.seg_bytes;
+    const int g_bytes = has_g ? (int)((row_bytes + 127) / 128 * 128) : 0;
+    g.stat_blk_bytes = has_stat ? (int)a.s0.blk_stride : 0;
+    g.g_blk_bytes = has_g ? (int)a.g.blk_stride : 0;
+    g.eps = a.eps;
+    int32_t* status = ja_device_status_word();
+    if (!status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    ja_status_t s = dt == JA_F32 ? launch_t<float>(op, a, g, vpl, g_bytes, sms, status, st, launched)
+                                 : launch_t<__nv_bfloat16>(op, a, g, vpl, g_bytes, sms, status, st, launched);
+    if (s != JA_OK || !*launched) return s;
+    ja_count_launch();
+    JA_CUDA(cudaGetLastError());
+    return JA_OK;
+}

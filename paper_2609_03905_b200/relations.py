@@ -62,6 +62,9 @@ class Spec:
         B.ja_execute(self.handle, [r.handle for r in inputs], [output.handle],
                      current_stream() if stream is None else stream)
 
+    def execute_join(self, inputs, partials: Relation, stream: int | None = None):
+        B.ja_execute_join(self.handle, [r.handle for r in inputs], partials.handle, current_stream() if stream is None else stream)
+
     def close(self):
         if getattr(self, "handle", None):
             B.ja_spec_destroy(self.handle)
@@ -76,6 +79,15 @@ class Spec:
 
 def repartition(src: Relation, dst: Relation, stream: int | None = None):
     B.ja_repartition(src.handle, dst.handle, current_stream() if stream is None else stream)
+
+
+def repartition_agg(partials: Relation, agg: str, dst: Relation, stream: int | None = None):
+    B.ja_repartition_agg(partials.handle, agg, dst.handle, current_stream() if stream is None else stream)
+
+
+def partial_relation(copies: int, extents, splits, dtype) -> Relation:
+    """Empty partial relation [c, x...]: the copy index in front, cut into its unit intervals."""
+    return Relation([copies] + list(extents), [list(range(copies + 1))] + [list(s) for s in splits], dtype)
 
 
 def from_dense(dense: torch.Tensor, splits) -> Relation:

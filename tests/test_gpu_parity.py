@@ -323,3 +323,73 @@ def test_fused_chain_refused_when_the_tiling_cannot_run_it():
     assert e.value.status_name == "JA_ERR_UNSUPPORTED"
     torch.cuda.synchronize()
     assert float(rC.payload.abs().max()) == 0.0
+
+
+# ---------------------------------------------------------------------------------------------------
+# a producer executed through its join + the aggregating relayout that consumes it (Sections 5.1, 5.3)
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,J,N,gi,gj,gk,dtype,pdtype", [
+    (256, 512, 256, 2, 2, 1, BF, BF),          # the four-specification matmul of Example 3.8
+    (512, 1024, 768, 2, 4, 3, BF, F32),        # tensor cores, accumulators kept in f32
+    (256, 768, 512, 1, 3, 2, BF, BF),
+    (96, 80, 72, 2, 5, 3, F32, F32),           # plain ALUs, ragged blocks
+    (100, 90, 56, 3, 2, 2, BF, BF),            # bf16 on a tiling the tensor-core path cannot address
+])
+def test_join_only_matmul_partials(M, J, N, gi, gj, gk, dtype, pdtype):
+    A = si.normal((M, J), 0.0, 1.0, dtype, 2, 21)
+    Bm = si.normal((J, N), 0.0, 1.0, dtype, 2, 22)
+    parts = {"i": ES(M, gi), "j": ES(J, gj), "k": ES(N, gk)}
+    spec = ja.Spec("ij,jk->ik", parts)
+    rA, rB = upload(A, [parts["i"], parts["j"]]), upload(Bm, [parts["j"], parts["k"]])
+    rP = ja.partial_relation(gj, [M, N], [parts["i"], parts["k"]], pdtype)
+    rP.payload.fill_(float("nan"))
+    spec.execute_join([rA, rB], rP)
+    got = download(rP)
+    check_status()
+    ref = blocked.join_partials("ij,jk->ik", parts, [si.to_f64(A), si.to_f64(Bm)], dtype=ORC_DT[pdtype])
+    assert got.shape == (gj, M, N)
+    for c in range(gj):
+        assert relfro(got[c], ref[c]) <= TOL[pdtype], c
+    # and the consumer's side: aggregate the copies into a different tiling
+    dst_sp = [ES(M, 4), ES(N, 2)]
+    rC = empty_like_tiling([M, N], dst_sp, dtype, fill=float("nan"))
+    ja.repartition_agg(rP, "sum", rC)
+    out = download(rC)
+    check_status()
+    want = blocked.aggregate_repartition(got, [parts["i"], parts["k"]], dst_sp, "sum", ORC_DT[dtype])
+    if dtype == F32:
+        assert relfro(out, want) <= 1e-6     # f32 additions in the oracle's order; the oracle adds in fp64 and rounds once
+    else:
+        assert np.mean(out != want) < 2e-3 and relfro(out, want) <= 1e-3   # double rounding f64->f32->bf16 flips rare ties
+    assert relfro(out, operators.matmul(si.to_f64(A), si.to_f64(Bm), ORC_DT[dtype])) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("sdt,ddt", [(BF, BF), (F32, F32), (F32, BF), (BF, F32)])
+@pytest.mark.parametrize("agg", ["sum", "max"])
+@pytest.mark.parametrize("m,ext,src,dst", [
+    (2, [256, 256], [[0, 128, 256], [0, 256]], [[0, 64, 128, 192, 256], [0, 256]]),       # the preamble example
+    (5, [300, 200], [ES(300, 3), ES(200, 2)], [ES(300, 2), ES(200, 5)]),
+    (3, [64, 40, 24], [ES(64, 2), ES(40, 1), ES(24, 3)], [ES(64, 4), ES(40, 5), ES(24, 1)]),
+    (7, [33, 17], [[0, 10, 33], [0, 17]], [[0, 33], [0, 5, 17]]),                          # odd sizes: scalar accesses
+    (1, [128, 96], [ES(128, 2), ES(96, 3)], [ES(128, 4), ES(96, 1)]),                      # one copy: a plain relayout
+])
+def test_aggregating_relayout(m, ext, src, dst, agg, sdt, ddt):
+    P = si.normal([m] + ext, 0.0, 1.0, sdt, 3, 31)
+    rP = upload(P, blocked.partial_splits(m, src))
+    rD = empty_like_tiling(ext, dst, ddt, fill=float("nan"))
+    before = download_bits(rP).copy()
+    ja.repartition_agg(rP, agg if m > 1 else "none", rD)
+    got = download(rD)
+    check_status()
+    assert np.array_equal(download_bits(rP), before)                      # partials are borrowed, unchanged
+    P64 = si.to_f64(P)
+    if agg == "max" or m == 1:
+        want = blocked.aggregate_repartition(P64, src, dst, agg, ORC_DT[ddt])
+        assert np.array_equal(got, want)                                  # MAX and plain relayout: bit-exact
+    else:
+        # the kernel adds in f32 in ascending copy order; restate that order in f32, then one rounding
+        acc = P64[0].astype(np.float32)
+        for c in range(1, m):
+            acc = acc + P64[c].astype(np.float32)
+        assert np.array_equal(got, core.round_to(acc.astype(np.float64), ORC_DT[ddt]))
+        assert relfro(got, blocked.aggregate_repartition(P64, src, dst, "sum", ORC_DT[ddt])) <= TOL[ddt]

@@ -216,3 +216,32 @@ def test_error_codes():
     for h in (A, A2, Bm, C):
         ja.ja_relation_destroy(h)
     ja.ja_spec_destroy(s)
+
+
+def test_partial_relation_argument_checks():
+    """Join-only execution and the aggregating relayout refuse malformed partial relations before any CUDA call."""
+    parts = {"i": [0, 4], "j": [0, 2, 4], "k": [0, 4]}
+    s = ja.ja_spec_create("ij,jk->ik", parts)
+    A = _rel([4, 4], [[0, 4], [0, 2, 4]], ja.JA_F32)
+    Bm = _rel([4, 4], [[0, 2, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 2)
+    C = _rel([4, 4], [[0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 3)
+    P_rank = _rel([4, 4], [[0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 4)                                 # no copy index
+    P_m3 = _rel([3, 4, 4], [[0, 1, 2, 3], [0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 5)                  # multiplicity is 2
+    P_coarse = _rel([2, 4, 4], [[0, 2], [0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 6)                    # copies share a block
+    P_tiled = _rel([2, 4, 4], [[0, 1, 2], [0, 2, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 7)               # not out(J)
+    P_shape = _rel([2, 4, 6], [[0, 1, 2], [0, 4], [0, 6]], ja.JA_F32, FAKE_PTR * 8)
+    P_ok = _rel([2, 4, 4], [[0, 1, 2], [0, 4], [0, 4]], ja.JA_F32, FAKE_PTR * 9)
+    assert _status(ja.ja_execute_join, s, [A, Bm], P_rank) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_execute_join, s, [A, Bm], P_m3) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_execute_join, s, [A, Bm], P_coarse) == "JA_ERR_TILING"
+    assert _status(ja.ja_execute_join, s, [A, Bm], P_tiled) == "JA_ERR_PARTITION_MISMATCH"
+    assert _status(ja.ja_execute_join, s, [A, Bm], P_shape) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_execute_join, s, [A], P_ok) == "JA_ERR_INVALID_ARG"
+    assert _status(ja.ja_repartition_agg, P_rank, "sum", C) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_repartition_agg, P_coarse, "sum", C) == "JA_ERR_TILING"
+    assert _status(ja.ja_repartition_agg, P_shape, "sum", C) == "JA_ERR_SHAPE"
+    assert _status(ja.ja_repartition_agg, P_ok, "none", C) == "JA_ERR_INVALID_ARG"      # two copies, no (+)
+    assert _status(ja.ja_repartition_agg, P_ok, "online_softmax", C) == "JA_ERR_INVALID_ARG"
+    for h in (A, Bm, C, P_rank, P_m3, P_coarse, P_tiled, P_shape, P_ok):
+        ja.ja_relation_destroy(h)
+    ja.ja_spec_destroy(s)
