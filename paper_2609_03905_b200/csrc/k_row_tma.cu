@@ -3,15 +3,17 @@
 // a thread that loads its cells into registers, reduces and stores keeps a few hundred bytes in flight; a ring of
 // shared-memory stages filled by cp.async.bulk keeps 100-200 KiB in flight per SM with one issuing thread.
 //
-// Layout fact used: inside a block the cells of consecutive rows of one column block are contiguous, so the R rows of
-// a work unit are nbc contiguous segments (one per column block) -- nbc bulk copies in, nbc bulk copies out.
+// A relation with uniform blocks is a rank-4 tensor (column in block, row in block, column block, strip of blocks), so
+// one tiled TMA copy fetches the R rows of a work unit out of ALL the column blocks they cross (boxes are at most 256
+// cells wide: a unit is bsc/bw copies in and as many out). Few, large copies matter: this part's TMA unit spends
+// about 0.1 us per copy whatever its size.
 //
 //   warps 0..7  consumers: warp w owns rows w, w+8, ... of the stage. It walks the row's column blocks in ascending
 //               order -- for the reductions (SQUARE/SUM, IDENT/MAX, EXP_SUB/SUM) that walk is the aggregation over the
 //               function specs that share the row's output key -- and, for the maps, writes the result over the input
 //               in shared memory.
-//   warp 8      loader: one thread issues the bulk loads of a unit into a free stage (mbarrier complete_tx).
-//   warp 9      storer (maps only): when the eight consumer warps are done with a stage, one thread issues the bulk
+//   warp 8      loader: one thread issues the TMA loads of a unit into a free stage (mbarrier complete_tx).
+//   warp 9      storer (maps only): when the eight consumer warps are done with a stage, one thread issues the TMA
 //               stores of the stage and frees it once the copies have read shared memory.
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT, waits (bounded) for its loads in flight
 // and leaves through the normal exit.
@@ -37,21 +39,21 @@ struct RowTmaGeom {
     int chunks_per_blk;          // work units per strip of nbc blocks
     int R;                       // rows per unit (the last unit of a block may hold fewer)
     int stages;
+    int wpr;                     // consumer warps per row (1, 2, 4 or 8); R * wpr >= 8 whenever wpr > 1
     int64_t n_units;
     int64_t blk_bytes;           // bytes between consecutive blocks of x / y
-    int seg_bytes;               // shared-memory bytes of one column-block segment of a stage: R * bsc * sizeof(T)
-    int stage_bytes;             // nbc * seg_bytes
+    int bw, nh;                  // TMA box width in cells (divides bsc, at most 256) and boxes per unit: bsc / bw
+    int seg_bytes;               // shared-memory bytes of one column block inside a box: R * bw * sizeof(T)
+    int half_bytes;              // one box: nbc * seg_bytes
+    int stage_bytes;             // nh * half_bytes
     int stat_blk_bytes;          // bytes between consecutive blocks of a statistics relation
     int g_blk_bytes;             // bytes between consecutive blocks of the gain vector
     float eps;
 };
 
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -71,10 +73,39 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+// A row is owned by a team of wpr warps (1, 2, 4 or 8): long rows are split so that all eight consumer warps work on the
+// few rows a stage can hold. A team reduction is a warp reduction, one partial per warp in shared memory, an mbarrier
+// (bounded wait) and a sum / max over the partials in a fixed order, so every warp of the team gets the same bits.
+struct Team {
+    int wpr, sub;            // warps per row; this warp's index inside its team
+    float* red;              // [2][8] partials of this team (two buffers: consecutive reductions alternate)
+    uint32_t bar;            // the team's mbarrier (count wpr)
+    uint32_t count;          // reductions done so far by this warp
+    volatile int* abort_flag;
+    int32_t* status;
+    bool ok;
+};
+
+template <bool IS_MAX>
+__device__ __forceinline__ float team_reduce(Team& t, float v, int lane) {
+    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    if (t.wpr == 1) return v;
+    float* buf = t.red + (t.count & 1) * 8;
+    if (lane == 0) {
+        buf[t.sub] = v;
+        mbar_arrive(t.bar);
+    }
+    if (!mbar_wait(t.bar, t.count & 1, t.abort_flag, t.status)) t.ok = false;
+    ++t.count;
+    float r = buf[0];
+    for (int i = 1; i < t.wpr; ++i) r = IS_MAX ? fmaxf(r, buf[i]) : r + buf[i];
+    return r;
+}
+
 // ---- one row, any cell type: plain scalar arithmetic --------------------------------------------------------
 template <typename T, int OP, int VPL>
 __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL],
-                                            const uint8_t* g_s, int64_t stat_off, int lane) {
+                                            const uint8_t* g_s, int64_t stat_off, int lane, Team& team) {
     constexpr int VEC = 16 / (int)sizeof(T);
     using V = RVec<T, VEC>;
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
@@ -91,9 +122,9 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) { const float f = ja_to_float(v.e[e]); sacc = fmaf(f, f, sacc); }
             }
-        sacc = warp_sum(sacc);
+        sacc = team_reduce<false>(team, sacc, lane);
         if (OP == ROW_SUMSQ) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
             return;
         }
         rstd = 1.0f / sqrtf(sacc / (float)g.n + g.eps);
@@ -107,9 +138,9 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) mx = fmaxf(mx, ja_to_float(v.e[e]));
             }
-        m = warp_max(mx);
+        m = team_reduce<true>(team, mx, lane);
         if (OP == ROW_MAX) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
             return;
         }
     }
@@ -127,9 +158,9 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
                     sacc += p;
                 }
             }
-        l = warp_sum(sacc);
+        l = team_reduce<false>(team, sacc, lane);
         if (OP == ROW_EXPSUM) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
             return;
         }
     }
@@ -145,7 +176,7 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
         V o;
         if (HAS_G) {
             const V v = *reinterpret_cast<const V*>(rowp + off[k]);
-            const V gv = *reinterpret_cast<const V*>(g_s + (size_t)(lane + 32 * k) * 16);
+            const V gv = *reinterpret_cast<const V*>(g_s + (size_t)((k * team.wpr + team.sub) * 32 + lane) * 16);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) o.e[e] = ja_from_float<T>(ja_to_float(v.e[e]) * rstd * ja_to_float(gv.e[e]));
         } else if (OP == ROW_SOFTMAX) {
@@ -199,7 +230,7 @@ __device__ __forceinline__ uint32_t narrow(uint64_t v) {   // two f32 -> packed 
 
 template <int OP, int VPL>
 __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL], const uint8_t* g_s,
-                                         int64_t stat_off, int lane) {
+                                         int64_t stat_off, int lane, Team& team) {
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
     constexpr bool KEEP_EXP = (OP == ROW_SOFTMAX);
     constexpr float LOG2E = 1.4426950408889634f;
@@ -220,9 +251,9 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         float s0, s1, s2, s3;
         upk2(acc0, s0, s1);
         upk2(acc1, s2, s3);
-        const float sacc = warp_sum((s0 + s1) + (s2 + s3));
+        const float sacc = team_reduce<false>(team, (s0 + s1) + (s2 + s3), lane);
         if (OP == ROW_SUMSQ) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = sacc;
             return;
         }
         rstd = 1.0f / sqrtf(sacc / (float)g.n + g.eps);
@@ -237,9 +268,9 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
                 mx = __hmax2(__hmax2(mx, h[0]), __hmax2(h[1], __hmax2(h[2], h[3])));
             }
         const float2 mf = __bfloat1622float2(mx);
-        m = warp_max(fmaxf(mf.x, mf.y));
+        m = team_reduce<true>(team, fmaxf(mf.x, mf.y), lane);
         if (OP == ROW_MAX) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s0.base + stat_off) = m;
             return;
         }
     }
@@ -266,9 +297,9 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         float s0, s1, s2, s3;
         upk2(acc0, s0, s1);
         upk2(acc1, s2, s3);
-        l = warp_sum((s0 + s1) + (s2 + s3));
+        l = team_reduce<false>(team, (s0 + s1) + (s2 + s3), lane);
         if (OP == ROW_EXPSUM) {
-            if (lane == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
+            if (lane == 0 && team.sub == 0) *reinterpret_cast<float*>(a.s1.base + stat_off) = l;
             return;
         }
     }
@@ -285,7 +316,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         uint4 o;
         if (HAS_G) {
             const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
-            const uint4 gv = *reinterpret_cast<const uint4*>(g_s + (size_t)(lane + 32 * k) * 16);
+            const uint4 gv = *reinterpret_cast<const uint4*>(g_s + (size_t)((k * team.wpr + team.sub) * 32 + lane) * 16);
             o.x = narrow(mul2(mul2(widen(v.x), scale2), widen(gv.x)));
             o.y = narrow(mul2(mul2(widen(v.y), scale2), widen(gv.y)));
             o.z = narrow(mul2(mul2(widen(v.z), scale2), widen(gv.z)));
@@ -312,14 +343,17 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
 template <typename T, int OP, int VPL> constexpr int ctas_per_sm() { return (OP == ROW_SOFTMAX && VPL * sizeof(T) >= 32) ? 1 : 2; }
 
 template <typename T, int OP, int VPL>
-__global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_tma_kernel(RowArgs a, RowTmaGeom g, int32_t* status) {
+__global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_tma_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, RowArgs a, RowTmaGeom g,
+               int32_t* status) {
     constexpr int VEC = 16 / (int)sizeof(T);
     using V = RVec<T, VEC>;
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
     constexpr bool HAS_Y = !(OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM);
-    extern __shared__ __align__(128) uint8_t smem[];
-    // [stages][nbc][R][bsc] cells, then the gain vector [n], then the barriers
-    const uint32_t s_stage0 = smem_u32(smem);
+    extern __shared__ uint8_t smem_raw[];
+    // [stages][nh][nbc][R][bw] cells, then the gain vector [n], then the barriers
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t s_stage0 = (raw + 127u) & ~127u;
+    uint8_t* smem = smem_raw + (s_stage0 - raw);
     uint8_t* g_s = smem + (size_t)g.stages * g.stage_bytes;
     const size_t g_bytes = HAS_G ? ((size_t)g.n * sizeof(T) + 127) / 128 * 128 : 0;
     uint64_t* bars = reinterpret_cast<uint64_t*>(g_s + g_bytes);
@@ -327,7 +361,9 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto done_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };       // consumers -> storer
     auto free_bar = [&](int s) { return bar0 + 8u * (2 * MAX_STAGES + s); };   // storer (or consumers) -> loader
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 3 * MAX_STAGES);
+    auto team_bar = [&](int t) { return bar0 + 8u * (3 * MAX_STAGES + t); };
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 3 * MAX_STAGES + CONSUMER_WARPS);
+    float* red_all = reinterpret_cast<float*>(bars + 3 * MAX_STAGES + CONSUMER_WARPS + 1);   // [8 teams][2][8]
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     if (threadIdx.x == 0) {
@@ -336,6 +372,7 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
             mbar_init(done_bar(s), CONSUMER_WARPS);
             mbar_init(free_bar(s), HAS_Y ? 1 : CONSUMER_WARPS);
         }
+        for (int t = 0; t < CONSUMER_WARPS; ++t) mbar_init(team_bar(t), (uint32_t)g.wpr);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -350,7 +387,7 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
     }
 
     const int64_t first = blockIdx.x, step = gridDim.x;
-    const int row_seg_bytes = g.bsc * (int)sizeof(T);   // bytes of one row inside one column-block segment
+    const int row_seg_bytes = g.bw * (int)sizeof(T);    // bytes of one row inside one column block of a box
 
     // unit -> (strip of blocks, first row inside the block, rows)
     auto unit_geom = [&](int64_t u, int64_t* lb, int* r0, int* rows) {
@@ -372,11 +409,9 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
                 int64_t lb;
                 int r0, rows;
                 unit_geom(u, &lb, &r0, &rows);
-                const uint32_t bytes = (uint32_t)(rows * row_seg_bytes);
-                mbar_expect_tx(full_bar(s), bytes * (uint32_t)g.nbc);
-                const char* src = a.x.base + lb * g.nbc * g.blk_bytes + (int64_t)r0 * row_seg_bytes;
+                mbar_expect_tx(full_bar(s), (uint32_t)g.stage_bytes);   // whole boxes: rows past the block's end arrive as zeros
                 const uint32_t dst = s_stage0 + (uint32_t)s * g.stage_bytes;
-                for (int cb = 0; cb < g.nbc; ++cb) bulk_load(dst + cb * g.seg_bytes, src + cb * g.blk_bytes, bytes, full_bar(s));
+                for (int h = 0; h < g.nh; ++h) tma_load_4d<1>(dst + h * g.half_bytes, &tmX, full_bar(s), h * g.bw, r0, 0, (int)lb);
             }
             if (!ok) {   // loads already issued still write shared memory: wait (bounded) for them before leaving
                 for (int64_t j = i > g.stages ? i - g.stages : 0; j < i; ++j) {
@@ -397,10 +432,8 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
                 int64_t lb;
                 int r0, rows;
                 unit_geom(u, &lb, &r0, &rows);
-                const uint32_t bytes = (uint32_t)(rows * row_seg_bytes);
-                char* dstp = a.y.base + lb * g.nbc * g.blk_bytes + (int64_t)r0 * row_seg_bytes;
                 const uint32_t src = s_stage0 + (uint32_t)s * g.stage_bytes;
-                for (int cb = 0; cb < g.nbc; ++cb) bulk_store(dstp + cb * g.blk_bytes, src + cb * g.seg_bytes, bytes);
+                for (int h = 0; h < g.nh; ++h) tma_store_4d(&tmY, src + h * g.half_bytes, h * g.bw, r0, 0, (int)lb);   // rows past the block's end are clipped
                 bulk_commit();
                 bulk_wait_read0();                 // the copies have read the stage: it may be refilled
                 mbar_arrive(free_bar(s));
@@ -412,29 +445,39 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
         int off[VPL];   // byte offset of this lane's k-th vector inside a row of the stage (column block + column), or -1
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            const int col = (lane + 32 * k) * VEC;
+            const int col = ((k * g.wpr + warp % g.wpr) * 32 + lane) * VEC;
             off[k] = -1;
             if (col < g.n) {
-                const int cb = col / g.bsc, ci = col - cb * g.bsc;
-                off[k] = cb * g.seg_bytes + ci * (int)sizeof(T);
+                const int cb = col / g.bsc, ci = col - cb * g.bsc, h = ci / g.bw;
+                off[k] = h * g.half_bytes + cb * g.seg_bytes + (ci - h * g.bw) * (int)sizeof(T);
             }
         }
-        bool ok = true;
+        Team team;
+        team.wpr = g.wpr;
+        team.sub = warp % g.wpr;
+        const int tid = warp / g.wpr, n_teams = CONSUMER_WARPS / g.wpr;
+        team.red = red_all + tid * 16;
+        team.bar = team_bar(tid);
+        team.count = 0;
+        team.abort_flag = abort_flag;
+        team.status = status;
+        team.ok = true;
         int64_t i = 0;
-        for (int64_t u = first; u < g.n_units && ok; u += step, ++i) {
+        for (int64_t u = first; u < g.n_units && team.ok; u += step, ++i) {
             const int s = (int)(i % g.stages);
             const uint32_t ph = (uint32_t)(i / g.stages) & 1;
-            if (!mbar_wait(full_bar(s), ph, abort_flag, status)) { ok = false; break; }
+            if (!mbar_wait(full_bar(s), ph, abort_flag, status)) { team.ok = false; break; }
             int64_t lb;
             int r0, rows;
             unit_geom(u, &lb, &r0, &rows);
             uint8_t* stage = smem + (size_t)s * g.stage_bytes;
-            for (int r = warp; r < rows; r += CONSUMER_WARPS) {
+            for (int r = tid; r < rows && team.ok; r += n_teams) {
                 uint8_t* rowp = stage + (size_t)r * row_seg_bytes;
                 const int64_t stat_off = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
-                if constexpr (sizeof(T) == 2) row_bf16<OP, VPL>(a, g, rowp, off, g_s, stat_off, lane);
-                else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, lane);
+                if constexpr (sizeof(T) == 2) row_bf16<OP, VPL>(a, g, rowp, off, g_s, stat_off, lane, team);
+                else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, lane, team);
             }
+            if (!team.ok) break;
             if (HAS_Y) fence_async_smem();    // this thread's writes to the stage become visible to the bulk stores
             __syncwarp();
             if (lane == 0) mbar_arrive(HAS_Y ? done_bar(s) : free_bar(s));
@@ -442,51 +485,70 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
     }
 }
 
+struct RowMaps { CUtensorMap x, y; };
+
 template <typename T, int OP, int VPL>
-ja_status_t launch_v(const RowArgs& a, RowTmaGeom g, int g_bytes, int sms, int32_t* status, cudaStream_t st, bool* launched) {
+ja_status_t launch_v(const RowMaps& tm, const RowArgs& a, RowTmaGeom g, int g_bytes, int sms, int32_t* status, cudaStream_t st,
+                     bool* launched) {
     constexpr int CTAS = ctas_per_sm<T, OP, VPL>();
-    const int budget = (CTAS == 2 ? 100 : 200) * 1024 - g_bytes;
+    const int budget = (CTAS == 2 ? 110 : 220) * 1024 - g_bytes;
     g.stages = (int)std::min<int64_t>(MAX_STAGES, budget / g.stage_bytes);
     if (g.stages < 2) { *launched = false; return JA_OK; }
     static bool configured = false;   // per template instance
     if (!configured) {
-        JA_CUDA(cudaFuncSetAttribute(row_tma_kernel<T, OP, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024 + 1024));
+        JA_CUDA(cudaFuncSetAttribute(row_tma_kernel<T, OP, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
         configured = true;
     }
-    const int smem_bytes = g.stages * g.stage_bytes + g_bytes + (3 * MAX_STAGES + 2) * 8;
+    const int smem_bytes = g.stages * g.stage_bytes + g_bytes + (3 * MAX_STAGES + CONSUMER_WARPS + 2) * 8 + CONSUMER_WARPS * 16 * 4 + 128;
     const unsigned grid = (unsigned)std::min<int64_t>(g.n_units, (int64_t)sms * CTAS);
-    row_tma_kernel<T, OP, VPL><<<grid, NUM_THREADS, smem_bytes, st>>>(a, g, status);
+    row_tma_kernel<T, OP, VPL><<<grid, NUM_THREADS, smem_bytes, st>>>(tm.x, tm.y, a, g, status);
     return JA_OK;
 }
 
 template <typename T, int OP>
-ja_status_t launch_op(const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms, int32_t* status, cudaStream_t st,
-                      bool* launched) {
+ja_status_t launch_op(const RowMaps& tm, const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms, int32_t* status,
+                      cudaStream_t st, bool* launched) {
     *launched = true;
-    if (vpl <= 1) return launch_v<T, OP, 1>(a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 2) return launch_v<T, OP, 2>(a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 4) return launch_v<T, OP, 4>(a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 8) return launch_v<T, OP, 8>(a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 16) return launch_v<T, OP, 16>(a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 32 && OP != ROW_SOFTMAX) return launch_v<T, OP, (OP != ROW_SOFTMAX ? 32 : 16)>(a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 1) return launch_v<T, OP, 1>(tm, a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 2) return launch_v<T, OP, 2>(tm, a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 4) return launch_v<T, OP, 4>(tm, a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 8) return launch_v<T, OP, 8>(tm, a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 16) return launch_v<T, OP, 16>(tm, a, g, g_bytes, sms, status, st, launched);
+    if (vpl <= 32 && OP != ROW_SOFTMAX) return launch_v<T, OP, (OP != ROW_SOFTMAX ? 32 : 16)>(tm, a, g, g_bytes, sms, status, st, launched);
     *launched = false;
     return JA_OK;
 }
 
 template <typename T>
-ja_status_t launch_t(RowOp op, const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms, int32_t* status,
-                     cudaStream_t st, bool* launched) {
+ja_status_t launch_t(RowOp op, const RowMaps& tm, const RowArgs& a, const RowTmaGeom& g, int vpl, int g_bytes, int sms,
+                     int32_t* status, cudaStream_t st, bool* launched) {
     switch (op) {
-        case ROW_SUMSQ: return launch_op<T, ROW_SUMSQ>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_MAX: return launch_op<T, ROW_MAX>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_EXPSUM: return launch_op<T, ROW_EXPSUM>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_RMS_SCALE: return launch_op<T, ROW_RMS_SCALE>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_EXP_SUB_DIV: return launch_op<T, ROW_EXP_SUB_DIV>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_RMSNORM: return launch_op<T, ROW_RMSNORM>(a, g, vpl, g_bytes, sms, status, st, launched);
-        case ROW_SOFTMAX: return launch_op<T, ROW_SOFTMAX>(a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_SUMSQ: return launch_op<T, ROW_SUMSQ>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_MAX: return launch_op<T, ROW_MAX>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_EXPSUM: return launch_op<T, ROW_EXPSUM>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_RMS_SCALE: return launch_op<T, ROW_RMS_SCALE>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_EXP_SUB_DIV: return launch_op<T, ROW_EXP_SUB_DIV>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_RMSNORM: return launch_op<T, ROW_RMSNORM>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
+        case ROW_SOFTMAX: return launch_op<T, ROW_SOFTMAX>(tm, a, g, vpl, g_bytes, sms, status, st, launched);
         default: break;
     }
     *launched = false;
+    return JA_OK;
+}
+
+// x / y with uniform blocks as the rank-4 tensor (column in block, row in block, column block, strip), box (bw, R, nbc, 1)
+ja_status_t encode_rows4(const RelView& v, const RowTmaGeom& g, int64_t n_lead, ja_dtype_t dt, CUtensorMap* tm) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const int es = dt == JA_F32 ? 4 : 2;
+    cuuint64_t dims[4] = {(cuuint64_t)g.bsc, (cuuint64_t)g.rows_per_blk, (cuuint64_t)g.nbc, (cuuint64_t)n_lead};
+    cuuint64_t strides[3] = {(cuuint64_t)g.bsc * es, (cuuint64_t)g.blk_bytes, (cuuint64_t)g.blk_bytes * g.nbc};
+    cuuint32_t box[4] = {(cuuint32_t)g.bw, (cuuint32_t)g.R, (cuuint32_t)g.nbc, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult res = enc(tm, dt == JA_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, v.base, dims, strides, box,
+                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (row strips) failed with code %d", (int)res);
     return JA_OK;
 }
 
@@ -494,7 +556,7 @@ ja_status_t launch_t(RowOp op, const RowArgs& a, const RowTmaGeom& g, int vpl, i
 
 // Sets *launched when this form took the job; leaves it false (and launches nothing) when the shape does not fit:
 // blocks of different shapes, rows longer than 32 vectors per lane, column blocks that are not whole 16-byte vectors,
-// RoPE (its rotation needs the row's coordinates).
+// more than 256 column blocks, RoPE (its rotation needs the row's coordinates).
 ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched) {
     *launched = false;
     if (op == ROW_ROPE) return JA_OK;
@@ -506,7 +568,7 @@ ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStr
     const bool has_stat = (op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM || op == ROW_RMS_SCALE || op == ROW_EXP_SUB_DIV);
     const bool two_stats = (op == ROW_EXPSUM || op == ROW_EXP_SUB_DIV);
     const bool has_y = !(op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM);
-    if (!a.x.blk_stride || a.x.bs[last] % vec != 0) return JA_OK;
+    if (!a.x.blk_stride || a.x.bs[last] % vec != 0 || a.x.nblk[last] > 256) return JA_OK;
     if (has_y && a.y.blk_stride != a.x.blk_stride) return JA_OK;
     if (has_g && !a.g.blk_stride) return JA_OK;
     if (has_stat && !a.s0.blk_stride) return JA_OK;
@@ -519,31 +581,50 @@ ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStr
     g.nbc = a.x.nblk[last];
     int64_t rows_per_blk = 1, n_lead = 1;
     for (int d = 0; d < last; ++d) { rows_per_blk *= a.x.bs[d]; n_lead *= a.x.nblk[d]; }
-    if (rows_per_blk >= (1 << 30) || n >= (1 << 24)) return JA_OK;
+    if (rows_per_blk >= (1 << 30) || n >= (1 << 24) || n_lead >= ((int64_t)1 << 31)) return JA_OK;
     g.rows_per_blk = (int)rows_per_blk;
     g.blk_bytes = a.x.blk_stride;
     const int64_t row_bytes = n * es;
-    const int vpl = (int)((n + vec * 32 - 1) / (vec * 32));
-    if (vpl > 32 || (vpl > 16 && op == ROW_SOFTMAX)) return JA_OK;
+    if ((n + vec * 32 - 1) / (vec * 32) > 256) return JA_OK;
+    // box width: the widest divisor of the column-block width that is a whole number of 128-byte lines and at most 256 cells
+    g.bw = 0;
+    for (int w = std::min(g.bsc, 256); w >= 128 / es; --w)
+        if (g.bsc % w == 0 && (w * es) % 128 == 0) { g.bw = w; break; }
+    if (!g.bw) return JA_OK;
+    g.nh = g.bsc / g.bw;
     // rows per unit: the largest power of two (at most 32, at most a block holds) that keeps a stage within 32 KiB
     int R = 1;
     while (R < 32 && (int64_t)R * 2 * row_bytes <= 32 * 1024 && R * 2 <= rows_per_blk) R *= 2;
     g.R = R;
+    // all eight consumer warps work: a stage of fewer than eight rows gives every row to a team of warps
+    g.wpr = 1;
+    while (g.wpr < CONSUMER_WARPS && R * g.wpr < CONSUMER_WARPS && n > (int64_t)g.wpr * vec * 32) g.wpr *= 2;
+    const int vpl = (int)((n + (int64_t)vec * 32 * g.wpr - 1) / ((int64_t)vec * 32 * g.wpr));
+    if (vpl > 32 || (vpl > 16 && op == ROW_SOFTMAX)) return JA_OK;
     g.chunks_per_blk = (int)((rows_per_blk + R - 1) / R);
     g.n_units = n_lead * g.chunks_per_blk;
-    g.seg_bytes = R * g.bsc * es;
-    g.stage_bytes = g.nbc * g.seg_bytes;
+    g.seg_bytes = R * g.bw * es;
+    g.half_bytes = g.nbc * g.seg_bytes;
+    g.stage_bytes = g.nh * g.half_bytes;
     const int g_bytes = has_g ? (int)((row_bytes + 127) / 128 * 128) : 0;
     g.stat_blk_bytes = has_stat ? (int)a.s0.blk_stride : 0;
     g.g_blk_bytes = has_g ? (int)a.g.blk_stride : 0;
     g.eps = a.eps;
     int32_t* status = ja_device_status_word();
     if (!status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    ja_status_t s = dt == JA_F32 ? launch_t<float>(op, a, g, vpl, g_bytes, sms, status, st, launched)
-                                 : launch_t<__nv_bfloat16>(op, a, g, vpl, g_bytes, sms, status, st, launched);
+    RowMaps tm;
+    ja_status_t s = encode_rows4(a.x, g, n_lead, dt, &tm.x);
+    if (s != JA_OK) return s;
+    tm.y = tm.x;
+    if (has_y && (s = encode_rows4(a.y, g, n_lead, dt, &tm.y)) != JA_OK) return s;
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
+    }
+    s = dt == JA_F32 ? launch_t<float>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched)
+                     : launch_t<__nv_bfloat16>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched);
     if (s != JA_OK || !*launched) return s;
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
