@@ -197,6 +197,32 @@ ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_t* const* i
                             ja_relation_t* partials, void* cuda_stream);
 ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_t agg, ja_relation_t* dst, void* cuda_stream);
 
+/* ---- logical optimization (Section 4.2, Algorithm 1; cost proxy of Section 4.3) -------------------------------
+ * Chooses one join-agg spec per abstract operator of a computation TREE (every node but the last is consumed by
+ * exactly one later node; the last node produces the result) for p processors = p function specs per operator.
+ * A spec is the vector of interval counts of the operator's letters, in order of first appearance (near-equal
+ * intervals, Section 3.3); specs(Op) are all count vectors whose product is p (fixed letters keep one interval).
+ * Cost(J, T_1..T_n) = repartition (the cells of operand k when its producer's output tiling differs from in_k(J);
+ * nothing for inputs of the computation) + join (the cells of every input block of every function spec) +
+ * aggregation ((m-1) x the cells of every distinct output type). The dynamic program keeps, per operator and per
+ * output tiling, the cheapest spec and the producers' tilings that achieved it, and walks back from the root.
+ * All arrays are HOST memory; no CUDA call is made.
+ *   counts   out, [n_nodes][JA_PLAN_MAX_LETTERS]: interval count per letter of the chosen spec (0 beyond the letters)
+ *   total_cost  out (may be NULL): the minimum of the summed Cost
+ * ja_plan_cost evaluates the summed Cost of a given assignment (same layout of `counts`).
+ * Errors: JA_ERR_PARSE, JA_ERR_SHAPE (operand / producer mismatch), JA_ERR_INVALID_ARG (not a tree in topological
+ * order), JA_ERR_UNSUPPORTED (a node consumed twice: cut the graph first, Section 4.4; more than 8 letters),
+ * JA_ERR_TILING (no decomposition into p function specs). */
+#define JA_PLAN_MAX_LETTERS 8
+typedef struct {
+    const char* einsum;       /* signature of the abstract operator, as for ja_spec_create */
+    const int64_t* extents;   /* one per distinct letter, in order of first appearance */
+    const int32_t* producers; /* one per operand: index of the node that produces it (smaller than this node's), or -1 */
+    uint32_t fixed_letters;   /* bit l set: the l-th letter is not shardable */
+} ja_plan_node_t;
+ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
+ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost);
+
 /* ---- relayout without allocation -------------------------------------------------------------------
  * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)
  * Same data movement as ja_repartition -- every atom of the overlay of the two tilings is copied from its

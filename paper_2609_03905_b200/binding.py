@@ -31,6 +31,11 @@ class JaError(RuntimeError):
         self.status_name = STATUS.get(status, str(status))
 
 
+class ja_plan_node_t(ctypes.Structure):
+    _fields_ = [("einsum", ctypes.c_char_p), ("extents", ctypes.POINTER(ctypes.c_int64)),
+                ("producers", ctypes.POINTER(ctypes.c_int32)), ("fixed_letters", ctypes.c_uint32)]
+
+
 class ja_index_part_t(ctypes.Structure):
     _fields_ = [("name", ctypes.c_char), ("extent", ctypes.c_int64), ("nparts", ctypes.c_int32),
                 ("splits", ctypes.POINTER(ctypes.c_int64))]
@@ -59,6 +64,8 @@ def _load() -> ctypes.CDLL:
         "ja_execute": [vp, P(vp), i32, P(vp), i32, vp],
         "ja_repartition": [vp, vp, vp],
         "ja_execute_join": [vp, P(vp), i32, vp, vp],
+        "ja_plan_optimize": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
+        "ja_plan_cost": [P(ja_plan_node_t), i32, P(i32), P(i64)],
         "ja_repartition_agg": [vp, ctypes.c_int, vp, vp],
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
@@ -207,6 +214,49 @@ def ja_execute_join(spec: int, inputs, partials: int, stream: int = 0):
 def ja_repartition_agg(partials: int, agg, dst: int, stream: int = 0):
     """Aggregating relayout: the m copies of every atom are combined and stored in dst's tiling."""
     _check(LIB.ja_repartition_agg(partials, AGG[agg] if isinstance(agg, str) else int(agg), dst, ctypes.c_void_p(stream)))
+
+
+JA_PLAN_MAX_LETTERS = 8
+
+
+def _plan_nodes(ops):
+    """ops: [{"einsum": str, "extents": {letter: n}, "inputs": [producer index | None, ...], "fixed": set of letters}]"""
+    keep = []
+    arr = (ja_plan_node_t * len(ops))()
+    for i, op in enumerate(ops):
+        lhs = op["einsum"].replace(" ", "").split("->")[0]
+        letters = []
+        for c in lhs.replace(",", ""):
+            if c not in letters:
+                letters.append(c)
+        ext = (ctypes.c_int64 * len(letters))(*[op["extents"][c] for c in letters])
+        prod = (ctypes.c_int32 * len(op["inputs"]))(*[-1 if q is None else q for q in op["inputs"]])
+        fixed = sum(1 << letters.index(c) for c in op.get("fixed", ()))
+        keep += [ext, prod]
+        arr[i] = ja_plan_node_t(op["einsum"].encode(), ext, prod, fixed)
+        op["_letters"] = letters
+    return arr, keep
+
+
+def ja_plan_optimize(ops, p: int):
+    """Algorithm 1 on a computation tree. Returns (total cost, [{letter: intervals} per operator])."""
+    arr, keep = _plan_nodes(ops)
+    counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
+    total = ctypes.c_int64()
+    _check(LIB.ja_plan_optimize(arr, len(ops), p, counts, ctypes.byref(total)))
+    plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
+    return total.value, plan
+
+
+def ja_plan_cost(ops, plan) -> int:
+    arr, keep = _plan_nodes(ops)
+    counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
+    for i, op in enumerate(ops):
+        for l, c in enumerate(op["_letters"]):
+            counts[i * JA_PLAN_MAX_LETTERS + l] = plan[i][c]
+    total = ctypes.c_int64()
+    _check(LIB.ja_plan_cost(arr, len(ops), counts, ctypes.byref(total)))
+    return total.value
 
 
 def ja_repartition_noalloc(extents, src_splits, dst_splits, dtype: int, src_ptr: int, dst_ptr: int, stream: int = 0):

@@ -1,0 +1,243 @@
+// Logical optimization (Section 4): one join-agg spec per abstract operator of a computation tree, chosen by the
+// dynamic program Opt(Op, T) of Section 4.2 / Algorithm 1 under the communication proxy of Section 4.3. Host code only.
+//
+// A spec of an operator is the vector of interval counts of its letters (near-equal intervals, Section 3.3); the
+// tiling it induces on an operand is the sub-vector of that operand's letters. Sub-costs in closed form:
+//   join         sum over operands k of  card(T_k) * prod of the counts of the letters ABSENT from operand k
+//                (every cell of operand k is part of one input block per cell of the grid over the absent letters)
+//   aggregation  (m - 1) * card(T_out),  m = prod of the counts of the letters absent from the output
+//   repartition  card(T_k) when operand k comes from a producer whose output tiling differs from in_k(J)
+#include <string.h>
+
+#include <map>
+#include <string>
+#include <vector>
+
+#include "ja_internal.h"
+
+namespace {
+
+struct Op {
+    std::vector<std::string> ins;
+    std::string out, letters;
+    std::vector<int64_t> extent;      // per letter
+    std::vector<int32_t> producers;   // per operand, -1 = input of the computation
+    uint32_t fixed = 0;
+};
+typedef std::vector<int32_t> Counts;   // per letter (a spec) or per index of a tensor (a tiling)
+
+int pos(const std::string& s, char c) {
+    size_t p = s.find(c);
+    return p == std::string::npos ? -1 : (int)p;
+}
+
+ja_status_t parse_op(const ja_plan_node_t& n, int index, Op* op) {
+    if (!n.einsum || !n.extents) return ja_fail(JA_ERR_INVALID_ARG, "node %d: einsum / extents missing", index);
+    std::string e;
+    for (const char* c = n.einsum; *c; ++c)
+        if (*c != ' ') e.push_back(*c);
+    size_t arrow = e.find("->");
+    if (arrow == std::string::npos) return ja_fail(JA_ERR_PARSE, "node %d: einsum '%s' needs '->'", index, n.einsum);
+    std::string lhs = e.substr(0, arrow);
+    op->out = e.substr(arrow + 2);
+    size_t p0 = 0;
+    while (true) {
+        size_t comma = lhs.find(',', p0);
+        op->ins.push_back(lhs.substr(p0, comma == std::string::npos ? std::string::npos : comma - p0));
+        if (comma == std::string::npos) break;
+        p0 = comma + 1;
+    }
+    for (const std::string& t : op->ins)
+        for (char c : t) {
+            if (c < 'a' || c > 'z') return ja_fail(JA_ERR_PARSE, "node %d: bad character '%c'", index, c);
+            if (pos(op->letters, c) < 0) op->letters.push_back(c);
+        }
+    if (op->letters.size() > JA_PLAN_MAX_LETTERS) return ja_fail(JA_ERR_UNSUPPORTED, "node %d: more than %d letters", index, JA_PLAN_MAX_LETTERS);
+    for (char c : op->out)
+        if (pos(op->letters, c) < 0) return ja_fail(JA_ERR_PARSE, "node %d: output letter '%c' appears in no input", index, c);
+    op->extent.assign(n.extents, n.extents + op->letters.size());
+    for (int64_t x : op->extent)
+        if (x < 1) return ja_fail(JA_ERR_SHAPE, "node %d: extents must be positive", index);
+    if (!n.producers) return ja_fail(JA_ERR_INVALID_ARG, "node %d: producers missing", index);
+    op->producers.assign(n.producers, n.producers + op->ins.size());
+    for (int32_t q : op->producers)
+        if (q < -1 || q >= index) return ja_fail(JA_ERR_INVALID_ARG, "node %d: a producer must be an earlier node or -1", index);
+    op->fixed = n.fixed_letters;
+    return JA_OK;
+}
+
+int64_t card(const Op& op, const std::string& term) {
+    int64_t n = 1;
+    for (char c : term) n *= op.extent[pos(op.letters, c)];
+    return n;
+}
+Counts tiling(const Op& op, const Counts& spec, const std::string& term) {
+    Counts t;
+    for (char c : term) t.push_back(spec[pos(op.letters, c)]);
+    return t;
+}
+int64_t absent_product(const Op& op, const Counts& spec, const std::string& term) {
+    int64_t m = 1;
+    for (size_t l = 0; l < op.letters.size(); ++l)
+        if (pos(term, op.letters[l]) < 0) m *= spec[l];
+    return m;
+}
+// Cost(J, T_1..T_n); Ts[k] == nullptr for an input of the computation
+int64_t cost(const Op& op, const Counts& spec, const std::vector<const Counts*>& Ts) {
+    int64_t total = (absent_product(op, spec, op.out) - 1) * card(op, op.out);
+    for (size_t k = 0; k < op.ins.size(); ++k) {
+        total += card(op, op.ins[k]) * absent_product(op, spec, op.ins[k]);
+        if (Ts[k] && *Ts[k] != tiling(op, spec, op.ins[k])) total += card(op, op.ins[k]);
+    }
+    return total;
+}
+// specs(Op): interval counts whose product is p, lexicographic over the letters in order of first appearance
+void enum_specs(const Op& op, int32_t p, size_t l, Counts* cur, std::vector<Counts>* out) {
+    if (l == op.letters.size()) {
+        if (p == 1) out->push_back(*cur);
+        return;
+    }
+    if (op.fixed & (1u << l)) {
+        cur->push_back(1);
+        enum_specs(op, p, l + 1, cur, out);
+        cur->pop_back();
+        return;
+    }
+    for (int32_t c = 1; c <= p; ++c) {
+        if (p % c || (int64_t)c > op.extent[l]) continue;
+        cur->push_back(c);
+        enum_specs(op, p / c, l + 1, cur, out);
+        cur->pop_back();
+    }
+}
+
+struct Choice {
+    Counts spec;
+    std::vector<Counts> in_tilings;   // chosen T_k per operand (empty for inputs of the computation)
+};
+
+ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, std::vector<Op>* ops) {
+    if (!nodes || n_nodes < 1) return ja_fail(JA_ERR_INVALID_ARG, "no nodes");
+    ops->resize(n_nodes);
+    std::vector<int> consumers(n_nodes, 0);
+    for (int32_t i = 0; i < n_nodes; ++i) {
+        ja_status_t st = parse_op(nodes[i], i, &(*ops)[i]);
+        if (st != JA_OK) return st;
+        const Op& op = (*ops)[i];
+        for (size_t k = 0; k < op.ins.size(); ++k) {
+            const int32_t q = op.producers[k];
+            if (q < 0) continue;
+            const Op& pr = (*ops)[q];
+            if (pr.out.size() != op.ins[k].size()) return ja_fail(JA_ERR_SHAPE, "node %d operand %zu: rank differs from its producer's output", i, k);
+            for (size_t d = 0; d < pr.out.size(); ++d)
+                if (pr.extent[pos(pr.letters, pr.out[d])] != op.extent[pos(op.letters, op.ins[k][d])])
+                    return ja_fail(JA_ERR_SHAPE, "node %d operand %zu: extent %zu differs from its producer's output", i, k, d);
+            if (++consumers[q] > 1) return ja_fail(JA_ERR_UNSUPPORTED, "node %d is consumed twice: cut the graph into trees first (Section 4.4)", q);
+        }
+    }
+    for (int32_t i = 0; i + 1 < n_nodes; ++i)
+        if (consumers[i] != 1) return ja_fail(JA_ERR_INVALID_ARG, "node %d is not consumed: the last node must be the root of a tree", i);
+    return JA_OK;
+}
+
+}  // namespace
+
+extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost) {
+    if (p < 1 || !counts) return ja_fail(JA_ERR_INVALID_ARG, "p must be positive and counts non-NULL");
+    std::vector<Op> ops;
+    ja_status_t st = parse_all(nodes, n_nodes, &ops);
+    if (st != JA_OK) return st;
+    // cand[Op] in insertion order, Opt[Op, T], choice[Op, T]
+    std::vector<std::vector<Counts>> cand(n_nodes);
+    std::vector<std::map<Counts, int64_t>> opt(n_nodes);
+    std::vector<std::map<Counts, Choice>> choice(n_nodes);
+    for (int32_t i = 0; i < n_nodes; ++i) {
+        const Op& op = ops[i];
+        std::vector<Counts> specs;
+        Counts cur;
+        enum_specs(op, p, 0, &cur, &specs);
+        if (specs.empty()) return ja_fail(JA_ERR_TILING, "node %d has no decomposition into %d function specs", i, p);
+        const size_t n = op.ins.size();
+        for (const Counts& J : specs) {
+            // B(J): minimum over the producers' candidate tilings (odometer over cand lists; inputs have one entry)
+            std::vector<size_t> idx(n, 0);
+            int64_t best = -1;
+            std::vector<size_t> best_idx;
+            while (true) {
+                std::vector<const Counts*> Ts(n, nullptr);
+                int64_t b = 0;
+                for (size_t k = 0; k < n; ++k) {
+                    const int32_t q = op.producers[k];
+                    if (q < 0) continue;
+                    Ts[k] = &cand[q][idx[k]];
+                    b += opt[q][*Ts[k]];
+                }
+                b += cost(op, J, Ts);
+                if (best < 0 || b < best) { best = b; best_idx = idx; }
+                int k = (int)n - 1;
+                for (; k >= 0; --k) {
+                    const int32_t q = op.producers[k];
+                    const size_t lim = q < 0 ? 1 : cand[q].size();
+                    if (++idx[k] < lim) break;
+                    idx[k] = 0;
+                }
+                if (k < 0) break;
+            }
+            const Counts T = tiling(op, J, op.out);
+            auto it = opt[i].find(T);
+            if (it == opt[i].end() || best < it->second) {
+                if (it == opt[i].end()) cand[i].push_back(T);
+                opt[i][T] = best;
+                Choice c;
+                c.spec = J;
+                c.in_tilings.resize(n);
+                for (size_t k = 0; k < n; ++k)
+                    if (op.producers[k] >= 0) c.in_tilings[k] = cand[op.producers[k]][best_idx[k]];
+                choice[i][T] = c;
+            }
+        }
+    }
+    const int32_t root = n_nodes - 1;
+    const Counts* T_star = nullptr;
+    for (const Counts& T : cand[root])
+        if (!T_star || opt[root][T] < opt[root][*T_star]) T_star = &T;
+    if (total_cost) *total_cost = opt[root][*T_star];
+    // Assign: walk back from the root
+    memset(counts, 0, sizeof(int32_t) * (size_t)n_nodes * JA_PLAN_MAX_LETTERS);
+    std::vector<std::pair<int32_t, Counts>> stack;
+    stack.push_back({root, *T_star});
+    while (!stack.empty()) {
+        const int32_t i = stack.back().first;
+        const Counts T = stack.back().second;
+        stack.pop_back();
+        const Choice& c = choice[i][T];
+        for (size_t l = 0; l < c.spec.size(); ++l) counts[(size_t)i * JA_PLAN_MAX_LETTERS + l] = c.spec[l];
+        for (size_t k = 0; k < ops[i].ins.size(); ++k)
+            if (ops[i].producers[k] >= 0) stack.push_back({ops[i].producers[k], c.in_tilings[k]});
+    }
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost) {
+    if (!counts || !total_cost) return ja_fail(JA_ERR_INVALID_ARG, "counts / total_cost is NULL");
+    std::vector<Op> ops;
+    ja_status_t st = parse_all(nodes, n_nodes, &ops);
+    if (st != JA_OK) return st;
+    std::vector<Counts> spec(n_nodes), out_tiling(n_nodes);
+    int64_t total = 0;
+    for (int32_t i = 0; i < n_nodes; ++i) {
+        const Op& op = ops[i];
+        for (size_t l = 0; l < op.letters.size(); ++l) {
+            const int32_t c = counts[(size_t)i * JA_PLAN_MAX_LETTERS + l];
+            if (c < 1 || c > op.extent[l]) return ja_fail(JA_ERR_TILING, "node %d letter '%c': %d intervals", i, op.letters[l], c);
+            spec[i].push_back(c);
+        }
+        out_tiling[i] = tiling(op, spec[i], op.out);
+        std::vector<const Counts*> Ts(op.ins.size(), nullptr);
+        for (size_t k = 0; k < op.ins.size(); ++k)
+            if (op.producers[k] >= 0) Ts[k] = &out_tiling[op.producers[k]];
+        total += cost(op, spec[i], Ts);
+    }
+    *total_cost = total;
+    return JA_OK;
+}

@@ -245,3 +245,43 @@ def test_partial_relation_argument_checks():
     for h in (A, Bm, C, P_rank, P_m3, P_coarse, P_tiled, P_shape, P_ok):
         ja.ja_relation_destroy(h)
     ja.ja_spec_destroy(s)
+
+
+def _mlp_tree(T, d, f):
+    return [{"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+            {"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+            {"einsum": "ik,ik->ik", "extents": {"i": T, "k": f}, "inputs": [0, 1]},
+            {"einsum": "ik,kl->il", "extents": {"i": T, "k": f, "l": d}, "inputs": [2, None]}]
+
+
+def test_logical_optimizer_matches_oracle(golden_dir):
+    """ja_plan_optimize / ja_plan_cost (closed-form sub-costs) against the oracle's Algorithm 1 and its explicit
+    per-function-spec cost count: total costs are integers and must be equal; the returned plan must cost what it claims."""
+    from oracle import optimizer
+    g = json.load(open(os.path.join(golden_dir, "optimizer_example.json")))
+    for c in g["three_d"]:
+        N, p, q = c["N"], c["p"], c["q"]
+        op = {"einsum": "ij,jk->ik", "extents": {"i": N, "j": N, "k": N}, "inputs": [None, None]}
+        total, plan = ja.ja_plan_optimize([op], p)
+        assert total == (3 * q - 1) * N * N and plan == [{"i": q, "j": q, "k": q}]
+    ch = g["chain"]
+    for pc in ch["plan_costs"]:
+        assert ja.ja_plan_cost(ch["ops"], pc["plan"]) == pc["cost"]
+    assert ja.ja_plan_optimize(ch["ops"], ch["p"])[0] == ch["optimum"]
+    rng = np.random.default_rng(5)
+    trees = [(_mlp_tree(8, 6, 12), 4), (_mlp_tree(2048, 4096, 11008), 8), (_mlp_tree(100, 36, 50), 12),
+             ([{"einsum": "bqhd,bkhd->bhqk", "extents": {"b": 2, "q": 8, "h": 4, "d": 4, "k": 8}, "inputs": [None, None], "fixed": {"d"}},
+               {"einsum": "bhqk,bkhd->bqhd", "extents": {"b": 2, "h": 4, "q": 8, "k": 8, "d": 4}, "inputs": [0, None], "fixed": {"d"}}], 4)]
+    for ops, p in trees:
+        want, want_plan = optimizer.optimize_tree(ops, p)
+        got, plan = ja.ja_plan_optimize(ops, p)
+        assert got == want
+        assert ja.ja_plan_cost(ops, plan) == got == optimizer.plan_cost(ops, plan)
+        for _ in range(5):   # random assignments cost the same on both sides and never less than the optimum
+            rp = [optimizer.specs(op, p)[int(rng.integers(len(optimizer.specs(op, p))))] for op in ops]
+            c = ja.ja_plan_cost(ops, rp)
+            assert c == optimizer.plan_cost(ops, rp) and c >= got
+    with pytest.raises(ja.JaError):   # a node consumed twice is not a tree
+        ja.ja_plan_optimize([ch["ops"][0], {"einsum": "ik,ik->ik", "extents": {"i": 4, "k": 4}, "inputs": [0, 0]}], 2)
+    with pytest.raises(ja.JaError):   # producer / operand shapes must agree
+        ja.ja_plan_optimize([ch["ops"][0], {"einsum": "ik->i", "extents": {"i": 4, "k": 5}, "inputs": [0]}], 2)

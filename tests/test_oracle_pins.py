@@ -492,3 +492,46 @@ def test_aggregate_repartition_against_dense_reduction_and_plain_repartition():
     one = blocked.pack(P[:1], blocked.partial_splits(1, src))
     got = blocked.pack(blocked.aggregate_repartition(P[:1], src, dst, "none"), dst)
     np.testing.assert_array_equal(got, blocked.repartition(one, ext, src, dst))
+
+
+# ---------------------------------------------------------------------------------------------------
+# logical optimization (Section 4): Algorithm 1 against the paper's 3D matmul, a hand-costed chain and exhaustive search
+# ---------------------------------------------------------------------------------------------------
+def _mlp_tree(T, d, f):
+    return [{"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+            {"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+            {"einsum": "ik,ik->ik", "extents": {"i": T, "k": f}, "inputs": [0, 1]},
+            {"einsum": "ik,kl->il", "extents": {"i": T, "k": f, "l": d}, "inputs": [2, None]}]
+
+
+def test_optimizer_recovers_3d_matmul_and_hand_costed_chain(golden_dir):
+    from oracle import optimizer
+    g = _golden(golden_dir, "optimizer_example.json")
+    for c in g["three_d"]:
+        N, p, q = c["N"], c["p"], c["q"]
+        op = {"einsum": "ij,jk->ik", "extents": {"i": N, "j": N, "k": N}, "inputs": [None, None]}
+        for J in optimizer.specs(op, p):
+            assert optimizer.cost(op, J, [None, None]) == (J["i"] + J["j"] + J["k"] - 1) * N * N
+        total, plan = optimizer.optimize_tree([op], p)
+        assert total == (3 * q - 1) * N * N and plan == [{"i": q, "j": q, "k": q}]
+    ch = g["chain"]
+    for pc in ch["plan_costs"]:
+        assert optimizer.plan_cost(ch["ops"], pc["plan"]) == pc["cost"]
+    total, plan = optimizer.optimize_tree(ch["ops"], ch["p"])
+    assert total == ch["optimum"] and plan == ch["plan_costs"][0]["plan"]
+
+
+def test_optimizer_dynamic_program_equals_exhaustive_search():
+    from oracle import optimizer
+    trees = [(_mlp_tree(8, 6, 12), 4),
+             ([{"einsum": "ij,jk->ik", "extents": {"i": 6, "j": 9, "k": 4}, "inputs": [None, None]},
+               {"einsum": "ik,kl->il", "extents": {"i": 6, "k": 4, "l": 10}, "inputs": [0, None]},
+               {"einsum": "il->i", "extents": {"i": 6, "l": 10}, "inputs": [1]}], 6),
+             ([{"einsum": "bqhd,bkhd->bhqk", "extents": {"b": 2, "q": 8, "h": 4, "d": 4, "k": 8}, "inputs": [None, None], "fixed": {"d"}},
+               {"einsum": "bhqk,bkhd->bqhd", "extents": {"b": 2, "h": 4, "q": 8, "k": 8, "d": 4}, "inputs": [0, None], "fixed": {"d"}}], 4)]
+    for ops, p in trees:
+        dp_cost, dp_plan = optimizer.optimize_tree(ops, p)
+        ex_cost, _ = optimizer.exhaustive(ops, p)
+        assert dp_cost == ex_cost == optimizer.plan_cost(ops, dp_plan)
+        for op, J in zip(ops, dp_plan):
+            assert int(np.prod(list(J.values()))) == p and all(J[c] == 1 for c in op.get("fixed", ()))
