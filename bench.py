@@ -24,13 +24,18 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 SHAPES = {"7b": dict(batch=8, seq=2048, hidden=4096, heads=32, ffn=11008),
-          "65b": dict(batch=1, seq=4096, hidden=8192, heads=64, ffn=22016)}
+          "65b": dict(batch=1, seq=4096, hidden=8192, heads=64, ffn=22016),
+          # the paper's own block (Section 7): grouped-query attention, 32 query heads on 8 key/value heads, FFN 14336
+          "paper_b8_1k": dict(batch=8, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336),
+          "paper_1x8k": dict(batch=1, seq=8192, hidden=4096, heads=32, kv_heads=8, ffn=14336),
+          "paper_b128_1k": dict(batch=128, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336)}
 METRIC = "join-agg TFLOP/s, LLaMA-block forward on 1 B200"
 
 
-def block_flops(batch, seq, hidden, ffn):
+def block_flops(batch, seq, hidden, ffn, heads=None, kv_heads=None):
     T = batch * seq
-    return 2.0 * T * hidden * hidden * 4 + 2.0 * T * hidden * ffn * 3 + 4.0 * T * seq * hidden / 2
+    kv_hidden = hidden if not kv_heads else hidden // heads * kv_heads
+    return 2.0 * T * hidden * (2 * hidden + 2 * kv_hidden) + 2.0 * T * hidden * ffn * 3 + 4.0 * T * seq * hidden / 2
 
 
 def measured_peaks():
@@ -53,13 +58,15 @@ def oracle_sample(shape, rows_n=16, prefix=None):
     from oracle import core, operators
     import torch
     S, hidden, heads, ffn = prefix or shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
-    w = {k: si.to_f64(v) for k, v in si.llama_weights(hidden, ffn).items()}
+    kvh = shape.get("kv_heads") or heads
+    kv_hidden = hidden // heads * kvh
+    w = {k: si.to_f64(v) for k, v in si.llama_weights(hidden, ffn, kv_hidden=kv_hidden).items()}
     x = si.to_f64(si.normal((S, hidden), 0.0, 1.0, torch.bfloat16, 5, 0))
     rows = np.linspace(0, S - 1, rows_n).astype(np.int64)
     t0 = time.perf_counter()
-    operators.llama_block(x, w, heads, 1e4, 1e-5, rows=rows)
+    operators.llama_block(x, w, heads, 1e4, 1e-5, rows=rows, n_kv_heads=kvh)
     dt = time.perf_counter() - t0
-    fl = 2.0 * S * hidden * hidden * 2 + 2.0 * rows_n * hidden * hidden * 2 + 2.0 * rows_n * hidden * ffn * 3 \
+    fl = 2.0 * S * hidden * kv_hidden * 2 + 2.0 * rows_n * hidden * hidden * 2 + 2.0 * rows_n * hidden * ffn * 3 \
         + 4.0 * float(np.sum(rows + 1)) * hidden
     return fl, dt, core.num_threads()
 
@@ -153,8 +160,9 @@ def run_gpu(args, shape):
     bf = torch.bfloat16
     Bt, S, hidden, heads, ffn = shape["batch"], shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
     T = Bt * S
-    weights = si.llama_weights(hidden, ffn)
-    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan, fused=not args.unfused)
+    kvh = shape.get("kv_heads") or heads
+    weights = si.llama_weights(hidden, ffn, kv_hidden=hidden // heads * kvh)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan, fused=not args.unfused, n_kv_heads=kvh)
     x_host = si.normal((T, hidden), 0.0, 1.0, bf, 5, 0).pin_memory()
     out_host = torch.empty((T, hidden), dtype=bf).pin_memory()
     x_dev = torch.empty((T, hidden), dtype=bf, device="cuda")
@@ -271,7 +279,7 @@ def run_gpu(args, shape):
     ms_e2e = e0.elapsed_time(e1)
     assert torch.equal(out_hosts[0], out_hosts[1]), "end-to-end outputs of consecutive steps differ"
 
-    fl = block_flops(Bt, S, hidden, ffn)
+    fl = block_flops(Bt, S, hidden, ffn, heads, shape.get("kv_heads"))
     (ms_total, ms_e2e), (value, e2e_val) = replica_aggregate([ms_total, ms_e2e], fl, args.steps, world, device="cuda")
     ms_step = ms_total / args.steps
 
@@ -280,9 +288,10 @@ def run_gpu(args, shape):
     for name, s, e in events:
         per_op.setdefault(name, []).append(s.elapsed_time(e))
     ops = {k: sum(v) / len(v) for k, v in per_op.items()}
-    fl_h, fl_f = 2.0 * T * hidden * hidden, 2.0 * T * hidden * ffn
-    gemm_flops_all = {"q_proj": fl_h, "k_proj": fl_h, "v_proj": fl_h, "o_proj": fl_h, "w1_proj": fl_f, "w3_proj": fl_f, "w2_proj": fl_f,
-                      "q_proj_rope": fl_h, "k_proj_rope": fl_h, "o_proj_add": fl_h, "w13_swiglu": 2 * fl_f, "w2_proj_add": fl_f}
+    kv_hidden = hidden // heads * kvh
+    fl_h, fl_f, fl_kv = 2.0 * T * hidden * hidden, 2.0 * T * hidden * ffn, 2.0 * T * hidden * kv_hidden
+    gemm_flops_all = {"q_proj": fl_h, "k_proj": fl_kv, "v_proj": fl_kv, "o_proj": fl_h, "w1_proj": fl_f, "w3_proj": fl_f, "w2_proj": fl_f,
+                      "q_proj_rope": fl_h, "k_proj_rope": fl_kv, "o_proj_add": fl_h, "w13_swiglu": 2 * fl_f, "w2_proj_add": fl_f}
     gemm_flops = {k: v for k, v in gemm_flops_all.items() if k in ops}
     gemm_ms = sum(ops[k] for k in gemm_flops)
     peaks = measured_peaks()
@@ -298,11 +307,11 @@ def run_gpu(args, shape):
     if args.shape == "7b" and args.plan == "seq" and not args.unfused:
         roof["traffic"] = 1.037e9
         roof["traffic_unit"] = "bytes per launch (ncu, 7b / seq / fused; operands once + output would be 0.456e9)"
-    mem_bytes = {"rmsnorm_1": 4.0 * T * hidden, "rmsnorm_2": 4.0 * T * hidden, "rope_q": 4.0 * T * hidden, "rope_k": 4.0 * T * hidden,
+    mem_bytes = {"rmsnorm_1": 4.0 * T * hidden, "rmsnorm_2": 4.0 * T * hidden, "rope_q": 4.0 * T * hidden, "rope_k": 4.0 * T * kv_hidden,
                  "residual_1": 6.0 * T * hidden, "residual_2": 6.0 * T * hidden, "silu_mul": 6.0 * T * ffn}
     for k in ops:
         if k.startswith("repartition"):
-            mem_bytes[k] = 4.0 * T * hidden
+            mem_bytes[k] = 4.0 * T * (kv_hidden if k in ("repartition_k", "repartition_v") else hidden)
     hbm = {k: {"ms": ops[k], "GBps": mem_bytes[k] / (ops[k] * 1e-3) / 1e9, "frac_of_measured_hbm": mem_bytes[k] / (ops[k] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
            for k in mem_bytes if k in ops}
     attn_fl = 4.0 * T * S * hidden / 2
@@ -482,6 +491,96 @@ def run_case(args):
             es = 4 if pdt == f32 else 2
             res["aggregating_relayout_" + tag] = hb((m * es + 2.0) * T * d, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
             del h, W2, P, y, spec
+    elif args.case == "opt":
+        # logical optimization (Algorithm 1) of the SwiGLU MLP tree of config 2, then the chosen plan and three hand
+        # plans executed as join-aggs (a relayout wherever a producer's tiling differs from what its consumer's spec needs)
+        import time
+        T, d, f = 2048, 4096, 11008
+        ops = [{"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+               {"einsum": "ij,jk->ik", "extents": {"i": T, "j": d, "k": f}, "inputs": [None, None]},
+               {"einsum": "ik,ik->ik", "extents": {"i": T, "k": f}, "inputs": [0, 1]},
+               {"einsum": "ik,kl->il", "extents": {"i": T, "k": f, "l": d}, "inputs": [2, None]}]
+
+        def run_plan(plan):
+            t_up = [ES(T, plan[0]["i"]), ES(d, plan[0]["j"]), ES(f, plan[0]["k"])]
+            t_up3 = [ES(T, plan[1]["i"]), ES(d, plan[1]["j"]), ES(f, plan[1]["k"])]
+            t_act = [ES(T, plan[2]["i"]), ES(f, plan[2]["k"])]
+            t_dn = [ES(T, plan[3]["i"]), ES(f, plan[3]["k"]), ES(d, plan[3]["l"])]
+            x1, W1 = rel((T, d), t_up[:2]), rel((d, f), t_up[1:], std=0.02)
+            x3, W3 = rel((T, d), t_up3[:2]), rel((d, f), t_up3[1:], std=0.02)
+            a, b = rel((T, f), [t_up[0], t_up[2]]), rel((T, f), [t_up3[0], t_up3[2]])
+            a2 = a if [t_up[0], t_up[2]] == t_act else rel((T, f), t_act)
+            b2 = b if [t_up3[0], t_up3[2]] == t_act else rel((T, f), t_act)
+            h = rel((T, f), t_act)
+            h2 = h if t_act == t_dn[:2] else rel((T, f), t_dn[:2])
+            W2, y = rel((f, d), t_dn[1:], std=0.02), rel((T, d), [t_dn[0], t_dn[2]])
+            s1 = ja.Spec("ij,jk->ik", dict(zip("ijk", t_up)))
+            s3 = ja.Spec("ij,jk->ik", dict(zip("ijk", t_up3)))
+            sa = ja.Spec("ik,ik->ik", dict(zip("ik", t_act)), "silu_mul", (), "none")
+            s2 = ja.Spec("ik,kl->il", dict(zip("ikl", t_dn)))
+
+            def chain(r):
+                s1.execute([x1, W1], a); s3.execute([x3, W3], b)
+                if a2 is not a: ja.repartition(a, a2)
+                if b2 is not b: ja.repartition(b, b2)
+                sa.execute([a2, b2], h)
+                if h2 is not h: ja.repartition(h, h2)
+                s2.execute([h2, W2], y)
+            return timeit(chain, reps, True), (a2 is not a) + (b2 is not b) + (h2 is not h)
+
+        for p_ in (8, 64):
+            t0 = time.perf_counter()
+            best_cost, best = ja.ja_plan_optimize(ops, p_)
+            opt_ms = (time.perf_counter() - t0) * 1e3
+            q = round(p_ ** (1 / 3))
+            hand = {"optimizer": best,
+                    "rows_only": [{"i": p_, "j": 1, "k": 1}, {"i": p_, "j": 1, "k": 1}, {"i": p_, "k": 1}, {"i": p_, "k": 1, "l": 1}],
+                    "contracted_only": [{"i": 1, "j": p_, "k": 1}, {"i": 1, "j": p_, "k": 1}, {"i": 1, "k": p_}, {"i": 1, "k": p_, "l": 1}],
+                    "cube": [{"i": q, "j": q, "k": q}, {"i": q, "j": q, "k": q}, {"i": q, "k": p_ // q}, {"i": q, "k": q, "l": q}]}
+            for name, plan in hand.items():
+                t, n_rep = run_plan(plan)
+                res["p%d_%s" % (p_, name)] = {**t, "proxy_cost_cells": ja.ja_plan_cost(ops, plan), "relayouts": n_rep,
+                                              "TFLOPs": 6.0 * T * d * f / (t["ms_mean"] * 1e-3) / 1e12, "plan": plan}
+            res["p%d_optimizer_host_ms" % p_] = {"ms_mean": opt_ms, "ms_min": opt_ms, "ms_median": opt_ms, "cost": best_cost}
+    elif args.case == "chains":
+        # Section 7, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
+        # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)
+        def right(lo, hi):   # M_lo (M_lo+1 (... M_hi))
+            return lo if lo == hi else (lo, right(lo + 1, hi))
+
+        chains = {
+            "A": ([10240] + [16384, 6144] * 4 + [10240], ((0, 1), (((2, 3), ((4, 5), (6, 7))), 8))),
+            "B": ([9216, 20480, 5120, 20480, 5120, 9216], ((0, 1), ((2, 3), 4))),
+            "C": ([10240, 12288, 32768, 2048], (0, (1, 2))),
+            "D": ([24576, 1536] + [20480] * 6 + [1536, 24576], (0, (right(1, 7), 8))),
+            "E": ([49152, 1024] + [20480] * 10 + [1024, 49152], (0, (right(1, 11), 12))),
+        }
+        blk = lambda n: ES(n, n // 512)
+
+        for name, (dims, tree) in chains.items():
+            mats = [rel((dims[i], dims[i + 1]), [blk(dims[i]), blk(dims[i + 1])], std=dims[i] ** -0.5) for i in range(len(dims) - 1)]
+            steps, flops = [], [0.0]
+
+            def build(t):   # allocates the intermediates and the specs once; returns (relation, rows, cols)
+                if isinstance(t, int):
+                    return mats[t], dims[t], dims[t + 1]
+                (A, m, j), (Bm, j2, n) = build(t[0]), build(t[1])
+                out = ja.Relation([m, n], [blk(m), blk(n)], bf)
+                steps.append((ja.Spec("ij,jk->ik", {"i": blk(m), "j": blk(j), "k": blk(n)}), A, Bm, out))
+                flops[0] += 2.0 * m * j * n
+                return out, m, n
+
+            build(tree)
+
+            def run(r):
+                for sp, A, Bm, out in steps:
+                    sp.execute([A, Bm], out)
+            t = timeit(run, reps, True)
+            res["chain_" + name] = {**t, "multiplies": len(steps), "TFLOPs": flops[0] / (t["ms_mean"] * 1e-3) / 1e12,
+                                    "frac_of_burst_bf16_peak": flops[0] / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"],
+                                    "mean_multiply_vs_8192_cubed": flops[0] / 2 / len(steps) / 8192.0 ** 3}
+            del mats, steps
+            torch.cuda.empty_cache()
     assert ja.ja_stream_status(stream.cuda_stream) == 0
     print(json.dumps({"case": args.case, "reps": reps, "l2": "512 MiB flush buffer written, then a 256 MiB buffer read (clean lines), before every timed launch",
                       "peaks": peaks, "kernels": res}))
@@ -498,9 +597,10 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg"], default="block",
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "chains"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "
-                         "gqa = grouped-query attention over packed sequences; agg = join-only matmul + aggregating relayout")
+                         "gqa = grouped-query attention over packed sequences; agg = join-only matmul + aggregating relayout; "
+                         "opt = logical optimizer's plan for the MLP tree against hand plans; chains = the five matrix chains")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
     if args.case != "block":

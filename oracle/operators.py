@@ -183,22 +183,29 @@ def add(x, y, out_dtype="bf16"):
 
 
 # ---- LLaMA block --------------------------------------------------------------------------------
-def llama_block(x, w, n_heads, theta=1e4, eps=1e-5, rows=None, dtype="bf16"):
+def llama_block(x, w, n_heads, theta=1e4, eps=1e-5, rows=None, dtype="bf16", n_kv_heads=None):
     """Pre-norm transformer block forward for ONE sequence x[S, hidden] (sequences of a batch are
-    independent).  w: dict with wq, wk, wv, wo [hidden, hidden], w1, w3 [hidden, ffn], w2 [ffn, hidden],
-    g1, g2 [hidden]; all weights are [in, out].  rows: optional subset of token positions for which the
-    block output is wanted; K and V are always computed for the whole sequence."""
+    independent).  w: dict with wq, wo [hidden, hidden], wk, wv [hidden, n_kv_heads * d_head], w1, w3 [hidden, ffn],
+    w2 [ffn, hidden], g1, g2 [hidden]; all weights are [in, out].  rows: optional subset of token positions for
+    which the block output is wanted; K and V are always computed for the whole sequence.  With n_kv_heads <
+    n_heads the attention is grouped-query (Example 3.10): query head h joins key/value head h // group."""
     x = np.asarray(x, dtype=np.float64)
     S, hidden = x.shape
     d = hidden // n_heads
+    n_kv = n_heads if n_kv_heads is None else n_kv_heads
+    group = n_heads // n_kv
     rows = np.arange(S) if rows is None else np.asarray(rows)
     n1 = rmsnorm(x, w["g1"], eps, dtype)["y"]
     k = matmul(n1, w["wk"], dtype)
     v = matmul(n1, w["wv"], dtype)
     q = matmul(n1[rows], w["wq"], dtype)
-    k = rope(k.reshape(1, S, n_heads, d), theta, dtype)
+    k = rope(k.reshape(1, S, n_kv, d), theta, dtype)
     q = rope(q.reshape(1, len(rows), n_heads, d), theta, dtype, pos=rows)
-    att = attention(q, k, v.reshape(1, S, n_heads, d), causal=True, out_dtype=dtype, qpos=rows)
+    v4 = v.reshape(1, S, n_kv, d)
+    att = np.empty((1, len(rows), n_heads, d))
+    for hq in range(n_heads):     # plain definition, one query head at a time against its key/value head
+        g = hq // group
+        att[:, :, hq:hq + 1] = attention(q[:, :, hq:hq + 1], k[:, :, g:g + 1], v4[:, :, g:g + 1], causal=True, out_dtype=dtype, qpos=rows)
     att = att.reshape(len(rows), hidden)
     h = add(x[rows], matmul(att, w["wo"], dtype), dtype)
     n2 = rmsnorm(h, w["g2"], eps, dtype)["y"]

@@ -27,19 +27,24 @@ from .relations import Relation, Spec, equal_splits as ES, from_dense, repartiti
 class LlamaBlock:
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
                  theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8,
-                 ffn_blocks: int | None = None, fused: bool = True):
+                 ffn_blocks: int | None = None, fused: bool = True, n_kv_heads: int | None = None):
         assert plan in ("seq", "head")
         self.fused = fused
         assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
         assert seq % token_block == 0
         self.plan, self.B, self.S, self.hidden, self.H, self.ffn = plan, batch, seq, hidden, n_heads, ffn
+        n_kv = n_heads if n_kv_heads is None else n_kv_heads       # grouped-query attention (Example 3.10) when smaller
+        assert n_heads % n_kv == 0
+        self.n_kv, self.kv_hidden = n_kv, n_kv * (hidden // n_heads)
+        kv_hidden = self.kv_hidden
         T = batch * seq
         self.T = T
         bf = torch.bfloat16
         D = hidden // n_heads
         t_sp = ES(T, T // token_block)
         io_c = ES(hidden, col_blocks)                    # column tiling of the block's input / output
-        head_c = ES(hidden, n_heads)                     # one head per column block
+        head_c = ES(hidden, n_kv)                        # one key/value head's group of query heads per column block
+        kvhead_c = ES(kv_hidden, n_kv)                   # one key/value head per column block
         act_c = io_c if plan == "seq" else head_c        # column tiling of the plan's [T, hidden] activations
         # the FFN index is cut into 256-wide blocks when it divides evenly (11008 = 43 x 256, 22016 = 86 x 256): every
         # output tile of the up-projections is then a whole block, with no ragged tail tile per block
@@ -47,20 +52,25 @@ class LlamaBlock:
             ffn_blocks = ffn // 256 if ffn % 256 == 0 else col_blocks
         ffn_c = ES(ffn, ffn_blocks)
         self.t_sp, self.io_c, self.head_c, self.act_c, self.ffn_c = t_sp, io_c, head_c, act_c, ffn_c
-        qkv_c = io_c if plan == "seq" else head_c        # tiling q, k, v are produced in
+        qkv_c = io_c if plan == "seq" else head_c        # tiling q is produced in
+        # tiling k, v are produced in: column blocks hold whole heads, so the narrower key/value relations may get fewer blocks
+        kv_c = ES(kv_hidden, min(col_blocks, n_kv)) if plan == "seq" else kvhead_c
 
         def act(cols=act_c):
             return Relation([T, hidden], [t_sp, cols], bf)
+
+        def kv(cols=kv_c):
+            return Relation([T, kv_hidden], [t_sp, cols], bf)
 
         # ---- relations -------------------------------------------------------------------------------
         self.x = Relation([T, hidden], [t_sp, io_c], bf)                 # block input (filled by the caller)
         self.out = Relation([T, hidden], [t_sp, io_c], bf)               # block output
         self.x_p = self.x if plan == "seq" else act()                    # input in the plan's tiling
         self.n1, self.h, self.n2, self.o, self.y = act(), act(), act(), act(), act()
-        self.q, self.k, self.v = act(qkv_c), act(qkv_c), act(qkv_c)
-        self.q_r, self.k_r = act(qkv_c), act(qkv_c)                      # after RoPE
+        self.q, self.k, self.v = act(qkv_c), kv(), kv()
+        self.q_r, self.k_r = act(qkv_c), kv()                            # after RoPE
         if plan == "seq":
-            self.q_h, self.k_h, self.v_h, self.att_h = act(head_c), act(head_c), act(head_c), act(head_c)
+            self.q_h, self.k_h, self.v_h, self.att_h = act(head_c), kv(kvhead_c), kv(kvhead_c), act(head_c)
             self.att = act()
         else:
             self.q_h, self.k_h, self.v_h = self.q_r, self.k_r, self.v
@@ -71,7 +81,8 @@ class LlamaBlock:
         self.hh = Relation([T, ffn], [t_sp, ffn_c], bf)
         # weights [in, out]: rows tiled like the activation they contract with, columns like the result
         w = {n: weights[n].to("cuda", bf) for n in weights}
-        self.wq, self.wk, self.wv = (from_dense(w[n], [act_c, qkv_c]) for n in ("wq", "wk", "wv"))
+        self.wq = from_dense(w["wq"], [act_c, qkv_c])
+        self.wk, self.wv = (from_dense(w[n], [act_c, kv_c]) for n in ("wk", "wv"))
         self.wo = from_dense(w["wo"], [act_c if plan == "seq" else head_c, act_c])
         self.w1, self.w3 = from_dense(w["w1"], [act_c, ffn_c]), from_dense(w["w3"], [act_c, ffn_c])
         self.w2 = from_dense(w["w2"], [ffn_c, act_c])
@@ -81,13 +92,14 @@ class LlamaBlock:
         # and whole-head column blocks IS the layout of [b, s, h, d] with blocks [1, 128, heads/block, 128])
         b_sp, s_sp = ES(batch, batch), ES(seq, seq // token_block)
 
-        def v4(rel: Relation, cols):
-            hb = ES(n_heads, len(cols) - 1)
-            return rel.view_as([batch, seq, n_heads, D], [b_sp, s_sp, hb, [0, D]])
+        def v4(rel: Relation, cols, heads=n_heads):
+            hb = ES(heads, len(cols) - 1)
+            return rel.view_as([batch, seq, heads, D], [b_sp, s_sp, hb, [0, D]])
 
-        self.q4, self.k4 = v4(self.q, qkv_c), v4(self.k, qkv_c)
-        self.q4r, self.k4r = v4(self.q_r, qkv_c), v4(self.k_r, qkv_c)
-        self.qa, self.ka, self.va, self.oa = (v4(r, head_c) for r in (self.q_h, self.k_h, self.v_h, self.att_h))
+        self.q4, self.k4 = v4(self.q, qkv_c), v4(self.k, kv_c, n_kv)
+        self.q4r, self.k4r = v4(self.q_r, qkv_c), v4(self.k_r, kv_c, n_kv)
+        self.qa, self.oa = v4(self.q_h, head_c), v4(self.att_h, head_c)
+        self.ka, self.va = v4(self.k_h, kvhead_c, n_kv), v4(self.v_h, kvhead_c, n_kv)
 
         # ---- specs -------------------------------------------------------------------------------------
         def mm(jc, kc):
@@ -95,10 +107,17 @@ class LlamaBlock:
 
         self.s_norm = Spec("ij,j->ij", {"i": t_sp, "j": act_c}, "rmsnorm", (eps,), "none")
         self.s_qkv = mm(act_c, qkv_c)
+        self.s_kv = mm(act_c, kv_c)
         self.s_rope = Spec("bshd->bshd", {"b": b_sp, "s": s_sp, "h": ES(n_heads, len(qkv_c) - 1), "d": [0, D]}, "rope",
                            (theta,), "none")
-        self.s_attn = Spec("bqhd,bkhd,bkhd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_heads), "d": [0, D], "k": s_sp},
-                           "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
+        self.s_rope_k = Spec("bshd->bshd", {"b": b_sp, "s": s_sp, "h": ES(n_kv, len(kv_c) - 1), "d": [0, D]}, "rope",
+                             (theta,), "none")
+        if n_kv == n_heads:
+            self.s_attn = Spec("bqhd,bkhd,bkhd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_heads), "d": [0, D], "k": s_sp},
+                               "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
+        else:   # query heads inherit their split from the key/value heads: intervals of n_heads / n_kv heads
+            self.s_attn = Spec("bqhd,bkgd,bkgd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_kv), "d": [0, D], "k": s_sp,
+                                                         "g": ES(n_kv, n_kv)}, "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
         self.s_wo = mm(act_c if plan == "seq" else head_c, act_c)
         self.s_add = Spec("ij,ij->ij", {"i": t_sp, "j": act_c}, "add", (), "none")
         self.s_up = mm(act_c, ffn_c)
@@ -110,6 +129,7 @@ class LlamaBlock:
         self.fuse_rope = self.fuse_add = self.fuse_swiglu = fused
         if fused:
             self.s_qk_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": qkv_c}, "matmul_rope", (theta, seq, D), "sum")
+            self.s_k_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": kv_c}, "matmul_rope", (theta, seq, D), "sum")
             self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": act_c, "k": act_c}, "matmul_add", (), "sum")
             self.s_up_swiglu = Spec("ij,jk,jk->ik", {"i": t_sp, "j": act_c, "k": ffn_c}, "swiglu_up", (), "sum")
             self.s_down_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": ffn_c, "k": act_c}, "matmul_add", (), "sum")
@@ -117,7 +137,7 @@ class LlamaBlock:
     # flop count of one forward (dense contractions only; causal attention counted at half the square)
     def flops(self) -> float:
         T, d, f, S = self.T, self.hidden, self.ffn, self.S
-        return 2.0 * T * d * d * 4 + 2.0 * T * d * f * 3 + 4.0 * T * S * d / 2
+        return 2.0 * T * d * (2 * d + 2 * self.kv_hidden) + 2.0 * T * d * f * 3 + 4.0 * T * S * d / 2
 
     @staticmethod
     def _fused(spec: Spec, inputs, output: Relation, stream) -> bool:
@@ -154,14 +174,14 @@ class LlamaBlock:
         if self.fuse_rope and not self._fused(self.s_qk_rope, [self.n1, self.wq], self.q_r, stream):
             self.fuse_rope = False
         if self.fuse_rope:
-            self.s_qk_rope.execute([self.n1, self.wk], self.k_r, stream)
-            self.s_qkv.execute([self.n1, self.wv], self.v, stream)
+            self.s_k_rope.execute([self.n1, self.wk], self.k_r, stream)
+            self.s_kv.execute([self.n1, self.wv], self.v, stream)
         else:
             self.s_qkv.execute([self.n1, self.wq], self.q, stream)
-            self.s_qkv.execute([self.n1, self.wk], self.k, stream)
-            self.s_qkv.execute([self.n1, self.wv], self.v, stream)
+            self.s_kv.execute([self.n1, self.wk], self.k, stream)
+            self.s_kv.execute([self.n1, self.wv], self.v, stream)
             self.s_rope.execute([self.q4], self.q4r, stream)
-            self.s_rope.execute([self.k4], self.k4r, stream)
+            self.s_rope_k.execute([self.k4], self.k4r, stream)
         if p == "seq":
             repartition(self.q_r, self.q_h, stream)
             repartition(self.k_r, self.k_h, stream)

@@ -25,11 +25,13 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu").to(torch.float64).numpy()
 
 
-def llama_weights(hidden: int, ffn: int, config: int = 5, dtype=torch.bfloat16, first_ordinal: int = 1):
-    """Random-init block weights, all [in, out]: N(0, 0.02); norm gains N(1, 0.1)."""
+def llama_weights(hidden: int, ffn: int, config: int = 5, dtype=torch.bfloat16, first_ordinal: int = 1, kv_hidden: int | None = None):
+    """Random-init block weights, all [in, out]: N(0, 0.02); norm gains N(1, 0.1). kv_hidden = width of the key / value
+    projections (n_kv_heads * d_head; = hidden unless the block is grouped-query)."""
     o = first_ordinal
     w = {}
-    for name, shape in (("wq", (hidden, hidden)), ("wk", (hidden, hidden)), ("wv", (hidden, hidden)),
+    kvh = hidden if kv_hidden is None else kv_hidden
+    for name, shape in (("wq", (hidden, hidden)), ("wk", (hidden, kvh)), ("wv", (hidden, kvh)),
                         ("wo", (hidden, hidden)), ("w1", (hidden, ffn)), ("w3", (hidden, ffn)),
                         ("w2", (ffn, hidden))):
         w[name] = normal(shape, 0.0, 0.02, dtype, config, o)

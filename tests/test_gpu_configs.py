@@ -9,7 +9,7 @@ import torch
 
 import paper_2609_03905_b200 as ja
 import synth_inputs as si
-from oracle import blocked, operators
+from oracle import blocked, core, operators
 from paper_2609_03905_b200.llama_block import LlamaBlock
 
 from gpu_util import TOL, check_status, download, empty_like_tiling, relfro, upload
@@ -193,3 +193,85 @@ def test_small_block_every_intermediate():
         for name, rel in rels:
             assert relfro(download(rel), cat(name)) <= TOL[BF], (plan, fused, name)
         assert relfro(out, cat("out")) <= TOL[BF], (plan, fused)
+
+
+# ---------------------------------------------------------------------------------------------------
+# the paper's own workloads (Section 7): the grouped-query block and the matrix chains
+# ---------------------------------------------------------------------------------------------------
+def test_small_grouped_query_block_every_intermediate():
+    """4 query heads on 2 key/value heads: each intermediate relation against the oracle, both decompositions."""
+    Bt, S, hidden, heads, kvh, ffn = 2, 256, 512, 4, 2, 1408
+    w = si.llama_weights(hidden, ffn, config=5, first_ordinal=41, kv_hidden=kvh * 128)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 40)
+    w64 = {k: si.to_f64(v) for k, v in w.items()}
+    refs = [operators.llama_block(si.to_f64(x[b * S:(b + 1) * S]), w64, heads, n_kv_heads=kvh) for b in range(Bt)]
+    cat = lambda name: np.concatenate([r[name].reshape(S, -1) for r in refs])
+    for plan, fused in (("seq", False), ("head", False), ("seq", True), ("head", True)):
+        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4, ffn_blocks=11, fused=fused, n_kv_heads=kvh)
+        ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
+        out = download(blk.forward())
+        check_status()
+        for name, rel in (("n1", blk.n1), ("q", blk.q_r), ("k", blk.k_r), ("v", blk.v), ("att", blk.att), ("h", blk.h), ("n2", blk.n2)):
+            assert relfro(download(rel), cat(name)) <= TOL[BF], (plan, fused, name)
+        assert relfro(out, cat("out")) <= TOL[BF], (plan, fused)
+
+
+def test_paper_block_shape_grouped_query_sampled():
+    """Hidden 4096, 32 query heads on 8 key/value heads of 128, FFN 14336 (Section 7), eight sequences of 1K tokens;
+    sampled token rows of one sequence against the oracle."""
+    Bt, S, hidden, heads, kvh, ffn = 8, 1024, 4096, 32, 8, 14336
+    w = si.llama_weights(hidden, ffn, config=5, first_ordinal=61, kv_hidden=kvh * 128)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 60)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan="seq", n_kv_heads=kvh)
+    ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
+    out = download(blk.forward())
+    check_status()
+    assert blk.fuse_swiglu and blk.fuse_rope and blk.fuse_add
+    seq_id, prefix = 5, 512
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, prefix - 1], np.linspace(0, prefix - 1, 6).astype(int)]))
+    xs = si.to_f64(x[seq_id * S: seq_id * S + prefix])
+    ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows, n_kv_heads=kvh)["out"]
+    assert relfro(out[seq_id * S + rows], ref) <= TOL[BF]
+
+
+def _chain_eval(dims, tree, mats, mm):
+    """tree: nested pairs of matrix indices, e.g. (0, (1, 2)); mm(A, B) multiplies two operands."""
+    if isinstance(tree, int):
+        return mats[tree]
+    return mm(_chain_eval(dims, tree[0], mats, mm), _chain_eval(dims, tree[1], mats, mm))
+
+
+CHAINS = {   # Section 7: fixed parenthesizations; dimensions divided by `div` keep the structure at oracle-sized cost
+    "A": ([10240] + [16384, 6144] * 4 + [10240], ((0, 1), (((2, 3), ((4, 5), (6, 7))), 8))),
+    "B": ([9216, 20480, 5120, 20480, 5120, 9216], ((0, 1), ((2, 3), 4))),
+    "C": ([10240, 12288, 32768, 2048], (0, (1, 2))),
+    "D": ([24576, 1536] + [20480] * 6 + [1536, 24576], (0, ((1, (2, (3, (4, (5, (6, 7)))))), 8))),
+}
+
+
+@pytest.mark.parametrize("name,div", [("A", 32), ("B", 32), ("C", 16), ("D", 32)])
+def test_matrix_chain_reduced(name, div):
+    """The chain's own parenthesization as a sequence of matmul join-aggs; every intermediate is stored in bf16, and the
+    oracle rounds at the same store points. Whole result compared."""
+    dims, tree = CHAINS[name]
+    dims = [d // div for d in dims]
+    mats = [si.normal((dims[i], dims[i + 1]), 0.0, dims[i] ** -0.5, BF, 6, 10 * ord(name) + i) for i in range(len(dims) - 1)]
+
+    def blocks(n):
+        return ES(n, max(1, n // 128))
+
+    def gpu_mm(A, Bm):
+        (ra, sa), (rb, sb) = A, Bm
+        M, J, N = ra.extents[0], ra.extents[1], rb.extents[1]
+        out = empty_like_tiling([M, N], [sa[0], sb[1]], BF, fill=float("nan"))
+        ja.Spec("ij,jk->ik", {"i": sa[0], "j": sa[1], "k": sb[1]}).execute([ra, rb], out)
+        return out, [sa[0], sb[1]]
+
+    rels = []
+    for m in mats:
+        sp = [blocks(m.shape[0]), blocks(m.shape[1])]
+        rels.append((upload(m, sp), sp))
+    got = download(_chain_eval(dims, tree, rels, gpu_mm)[0])
+    check_status()
+    ref = _chain_eval(dims, tree, [si.to_f64(m) for m in mats], lambda A, Bm: core.round_to(A @ Bm, "bf16"))
+    assert relfro(got, ref) <= TOL[BF]
