@@ -74,8 +74,8 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     const int g = lane / 4, t4 = lane % 4;
 
     const int n_qt = a.S / QT;
-    const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest output keys (most surviving tuples) first
-    const int h = blockIdx.y, b = blockIdx.z;
+    const int qt = n_qt - 1 - (int)blockIdx.z;   // heaviest output keys (most surviving tuples) first, across all (batch, head)
+    const int h = blockIdx.x, b = blockIdx.y;
     const int q0 = qt * QT;
     const int hk = h / a.group;                  // key/value head joined with this query head
     int s0 = 0, s1 = a.S;                        // the packed sequence this tile lies in (no tile straddles an end)
@@ -257,7 +257,7 @@ ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
         if (s != JA_OK || launched) return s;
     }
     const int QT = (a.align % 128 == 0) ? 128 : 64;
-    dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
+    dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / QT));
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
     if (QT == 128) {
         JA_CUDA(cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

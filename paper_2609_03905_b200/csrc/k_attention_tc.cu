@@ -21,6 +21,10 @@
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT and leaves through the normal exit.
 #include <stdlib.h>
 
+#include <algorithm>
+#include <utility>
+#include <vector>
+
 #include "ja_device.cuh"
 #include "ja_ptx.cuh"
 
@@ -35,6 +39,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BYTES = 5 * TILE_BYTES + 1024 + 256;   // Q, K x2, V x2
 
 constexpr int MAX_SB = 64;   // sequence blocks of an irregular split held in the kernel parameters
+constexpr int MAX_ORDER = 512;   // query tiles (pairs) whose launch order is held in the kernel parameters
 
 // Tiling of one "bshd" relation: uniform blocks along b and h, any split of s, d unsplit.
 struct SeqGeom {
@@ -54,6 +59,8 @@ struct AttnTcParams {
     float scale_log2e;
     int32_t ends[JA_MAX_SEQ];
     SeqGeom q, k;                // o is tiled like q, v like k
+    int32_t n_order;             // > 0: order[z] = the query tile (pair) that CTAs with blockIdx.z == z own, heaviest first
+    uint16_t order[MAX_ORDER];
 };
 
 // Row coordinate of cell (b, s, h, :) in the rank-3 view (d, head in block, row). Block (bb, sb, hb) starts
@@ -165,8 +172,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n_qt = p.S / QT;
-    const int qt = n_qt - 1 - (int)blockIdx.x;   // output keys with the most surviving tuples first
-    const int h = blockIdx.y, b = blockIdx.z;
+    // CTAs are handed to SMs in order of blockIdx.x, then .y, then .z: with the tile index slowest, every (batch, head)
+    // starts its output key with the most surviving tuples before any lighter one starts (longest work first)
+    const int qt = p.n_order ? (int)p.order[blockIdx.z] : n_qt - 1 - (int)blockIdx.z;
+    const int h = blockIdx.x, b = blockIdx.y;
     const int q0 = qt * QT;
     int s0, s1;
     sequence_of(p, q0, s0, s1);
@@ -476,8 +485,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n_pairs = p.S / (2 * QT);
-    const int pr = n_pairs - 1 - (int)blockIdx.x;     // heaviest output keys first
-    const int h = blockIdx.y, b = blockIdx.z;
+    const int pr = p.n_order ? (int)p.order[blockIdx.z] : n_pairs - 1 - (int)blockIdx.z;   // heaviest output keys first, across all (batch, head)
+    const int h = blockIdx.x, b = blockIdx.y;
     const int q0 = pr * 2 * QT;                       // first row of tile A; tile B starts at q0 + 128
     int s0, s1;                                       // both tiles lie in one packed sequence (ends are multiples of 256)
     sequence_of(p, q0, s0, s1);
@@ -718,13 +727,31 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
     }
     p.scale_log2e = a.scale * 1.4426950408889634f;
     const char* one = getenv("JA_ATTN_ONE_TILE");
-    if (pair_ok && !(one && one[0] == '1')) {
+    const bool two_tiles = pair_ok && !(one && one[0] == '1');
+    // packed sequences: the work of a tile is its distance from the start of its own sequence, not its index
+    const int rows_per_cta = two_tiles ? 2 * QT : QT, n_cta_tiles = a.S / rows_per_cta;
+    if (a.n_ends > 1 && n_cta_tiles <= MAX_ORDER) {
+        std::vector<std::pair<int, int>> w(n_cta_tiles);   // (-steps, tile)
+        for (int t = 0; t < n_cta_tiles; ++t) {
+            const int q0 = t * rows_per_cta;
+            int s0 = 0, s1 = a.S;
+            for (int i = 0; i < a.n_ends; ++i) {
+                if (a.ends[i] <= q0) s0 = a.ends[i];
+                else { s1 = a.ends[i]; break; }
+            }
+            w[t] = {-(a.causal ? q0 + rows_per_cta - s0 : s1 - s0), t};
+        }
+        std::sort(w.begin(), w.end());
+        p.n_order = n_cta_tiles;
+        for (int t = 0; t < n_cta_tiles; ++t) p.order[t] = (uint16_t)w[t].second;
+    }
+    if (two_tiles) {
         JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
-        dim3 grid((unsigned)(a.S / (2 * QT)), (unsigned)a.H, (unsigned)a.B);
+        dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / (2 * QT)));
         attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        dim3 grid((unsigned)(a.S / QT), (unsigned)a.H, (unsigned)a.B);
+        dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / QT));
         attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
     }
     ja_count_launch();
