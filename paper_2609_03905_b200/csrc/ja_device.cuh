@@ -40,3 +40,20 @@ __device__ __forceinline__ float ja_to_float(__nv_bfloat16 x) { return __bfloat1
 template <typename T> __device__ __forceinline__ T ja_from_float(float x);
 template <> __device__ __forceinline__ float ja_from_float<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 ja_from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Launch order of the attention CTAs (CTAs are handed to SMs in order of blockIdx.x). One CTA = one query tile (or pair
+// of tiles) of one (batch, head). (batch, head) pairs are taken in sections of `sect` consecutive pairs and inside a
+// section all pairs run their heaviest tile first, then the next one, and so on. One section holding every pair is
+// "longest work first" (short tail; used when tiles differ in weight); sections that fill the GPU once keep the CTAs
+// that run together on few (batch, head) pairs, whose K / V tiles are then re-used through L2 (used for equal tiles).
+// Returns the slot of the tile in heaviest-first order and the flat (batch, head) index.
+__device__ __forceinline__ void ja_attn_decode_cta(int cta, int n_tiles, int n_bh, int sect, int* slot, int* bh) {
+    const int per_section = sect * n_tiles;
+    const int sec = cta / per_section;
+    const int first_bh = sec * sect;
+    const int g = min(sect, n_bh - first_bh);       // the last section may hold fewer pairs
+    const int local = cta - sec * per_section;
+    *slot = local / g;
+    *bh = first_bh + local % g;
+}
+

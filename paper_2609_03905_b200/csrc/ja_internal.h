@@ -149,6 +149,7 @@ struct AttnArgs {
     int32_t align;         // greatest common divisor of every q / k split point and sequence end
     int32_t n_ends;        // packed sequences: ends[0..n_ends) ascending, ends[n_ends-1] == S; 0 = one sequence
     int32_t ends[JA_MAX_SEQ];
+    int32_t sect;          // (batch, head) pairs per launch-order section (set by the launcher)
     // host copies of the sequence split points of q (= o) and k (= v), nblk[1] + 1 entries each, and whether all four
     // payloads follow the closed-form block order the tensor-memory kernel addresses by (uniform b and h blocks)
     const int32_t* q_split;

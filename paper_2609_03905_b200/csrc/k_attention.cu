@@ -16,6 +16,8 @@
 // take (64-row blocks); everything else is dispatched to the tcgen05 kernel.
 #include <stdlib.h>
 
+#include <algorithm>
+
 #include "ja_device.cuh"
 
 namespace {
@@ -74,8 +76,10 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     const int g = lane / 4, t4 = lane % 4;
 
     const int n_qt = a.S / QT;
-    const int qt = n_qt - 1 - (int)blockIdx.z;   // heaviest output keys (most surviving tuples) first, across all (batch, head)
-    const int h = blockIdx.x, b = blockIdx.y;
+    int slot, bh;
+    ja_attn_decode_cta((int)blockIdx.x, n_qt, a.H * a.B, a.sect, &slot, &bh);
+    const int qt = n_qt - 1 - slot;              // heaviest output keys (most surviving tuples) first
+    const int h = bh % a.H, b = bh / a.H;
     const int q0 = qt * QT;
     const int hk = h / a.group;                  // key/value head joined with this query head
     int s0 = 0, s1 = a.S;                        // the packed sequence this tile lies in (no tile straddles an end)
@@ -257,14 +261,16 @@ ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
         if (s != JA_OK || launched) return s;
     }
     const int QT = (a.align % 128 == 0) ? 128 : 64;
-    dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / QT));
+    AttnArgs a2 = a;
+    a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (148 + a.S / QT - 1) / (a.S / QT)));
+    dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
     if (QT == 128) {
         JA_CUDA(cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attention_kernel<128><<<grid, 256, smem, st>>>(a);
+        attention_kernel<128><<<grid, 256, smem, st>>>(a2);
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attention_kernel<64><<<grid, 128, smem, st>>>(a);
+        attention_kernel<64><<<grid, 128, smem, st>>>(a2);
     }
     ja_count_launch();
     JA_CUDA(cudaGetLastError());

@@ -59,7 +59,8 @@ struct AttnTcParams {
     float scale_log2e;
     int32_t ends[JA_MAX_SEQ];
     SeqGeom q, k;                // o is tiled like q, v like k
-    int32_t n_order;             // > 0: order[z] = the query tile (pair) that CTAs with blockIdx.z == z own, heaviest first
+    int32_t sect;                // (batch, head) pairs per launch-order section (ja_attn_decode_cta)
+    int32_t n_order;             // > 0: order[slot] = the query tile (pair) in heaviest-first slot `slot`
     uint16_t order[MAX_ORDER];
 };
 
@@ -172,10 +173,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n_qt = p.S / QT;
-    // CTAs are handed to SMs in order of blockIdx.x, then .y, then .z: with the tile index slowest, every (batch, head)
-    // starts its output key with the most surviving tuples before any lighter one starts (longest work first)
-    const int qt = p.n_order ? (int)p.order[blockIdx.z] : n_qt - 1 - (int)blockIdx.z;
-    const int h = blockIdx.x, b = blockIdx.y;
+    int slot, bh;
+    ja_attn_decode_cta((int)blockIdx.x, n_qt, p.H * p.B, p.sect, &slot, &bh);
+    const int qt = p.n_order ? (int)p.order[slot] : n_qt - 1 - slot;   // output keys with the most surviving tuples first
+    const int h = bh % p.H, b = bh / p.H;
     const int q0 = qt * QT;
     int s0, s1;
     sequence_of(p, q0, s0, s1);
@@ -485,8 +486,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n_pairs = p.S / (2 * QT);
-    const int pr = p.n_order ? (int)p.order[blockIdx.z] : n_pairs - 1 - (int)blockIdx.z;   // heaviest output keys first, across all (batch, head)
-    const int h = blockIdx.x, b = blockIdx.y;
+    int slot, bh;
+    ja_attn_decode_cta((int)blockIdx.x, n_pairs, p.H * p.B, p.sect, &slot, &bh);
+    const int pr = p.n_order ? (int)p.order[slot] : n_pairs - 1 - slot;   // heaviest output keys first
+    const int h = bh % p.H, b = bh / p.H;
     const int q0 = pr * 2 * QT;                       // first row of tile A; tile B starts at q0 + 128
     int s0, s1;                                       // both tiles lie in one packed sequence (ends are multiples of 256)
     sequence_of(p, q0, s0, s1);
@@ -745,13 +748,24 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
         p.n_order = n_cta_tiles;
         for (int t = 0; t < n_cta_tiles; ++t) p.order[t] = (uint16_t)w[t].second;
     }
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
+    }
+    // tiles of different weight (causal band, packed sequences): one section, i.e. heaviest first across all (batch, head)
+    // pairs -- measured better than any sectioning (balance beats L2 re-use); equal tiles: sections that fill the GPU once
+    p.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::max(1, (sms + n_cta_tiles - 1) / n_cta_tiles);
+    if (const char* se = getenv("JA_ATTN_SECTION")) p.sect = std::max(1, atoi(se));
+    p.sect = std::min(p.sect, a.H * a.B);
     if (two_tiles) {
         JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
-        dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / (2 * QT)));
+        dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / (2 * QT))), 1, 1);
         attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        dim3 grid((unsigned)a.H, (unsigned)a.B, (unsigned)(a.S / QT));
+        dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
         attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
     }
     ja_count_launch();
