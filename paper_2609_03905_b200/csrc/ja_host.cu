@@ -9,6 +9,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <iterator>
 #include <cmath>
 #include <mutex>
 
@@ -151,8 +152,11 @@ extern "C" ja_status_t ja_relation_create(int32_t rank, const int64_t* extents, 
     return JA_OK;
 }
 
+static void forget_relayout_plans(uint64_t relation_id);
+
 extern "C" ja_status_t ja_relation_destroy(ja_relation_t* rel) {
     if (!rel) return JA_OK;
+    forget_relayout_plans(rel->id);   // cached copy plans of relayouts from / to this relation (device tables) go with it
     if (rel->d_tables) cudaFree(rel->d_tables);
     delete rel;
     return JA_OK;
@@ -623,6 +627,14 @@ extern "C" ja_status_t ja_repartition(const ja_relation_t* src, ja_relation_t* d
 // aggregating relayout (Sections 5.1, 5.3): m unaggregated copies of every producer block -> aggregated consumer blocks
 // ---------------------------------------------------------------------------------------------------
 static std::map<std::vector<uint64_t>, std::shared_ptr<RepartPlan>> g_repart_agg_plans;
+
+static void forget_relayout_plans(uint64_t relation_id) {
+    std::lock_guard<std::mutex> lk(g_repart_mu);
+    for (auto it = g_repart_plans.begin(); it != g_repart_plans.end();)
+        it = (it->first.first == relation_id || it->first.second == relation_id) ? g_repart_plans.erase(it) : std::next(it);
+    for (auto it = g_repart_agg_plans.begin(); it != g_repart_agg_plans.end();)
+        it = (it->first[0] == relation_id || it->first[1] == relation_id) ? g_repart_agg_plans.erase(it) : std::next(it);
+}
 
 // partials must be [c, x...] with the copy index c cut into its unit intervals and x... the tensor of `like`
 static ja_status_t check_partial_relation(const ja_relation* partials, const ja_relation* like, int like_rank, const int64_t* like_extent) {
