@@ -161,6 +161,9 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  *   "bshd->bshd"           ROPE / NONE
  *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128; q / k split points and sequence
  *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends multiples of 64 rows (tensor memory kernels: 128)
+ * n_outputs is 1, except for ATTENTION where it may be 2: outputs[1] then receives lse[b, q, h] = log of the softmax
+ * denominator of every query row (f32, tiled like the first three indices of outputs[0]) -- with it two results over
+ * disjoint key ranges combine by the online-softmax aggregation: O = w1 O1 + w2 O2, w_i = exp(lse_i - lse).
  * The first call for a given (spec, relations) tuple builds and caches tables on the device (a few
  * synchronous cudaMalloc / cudaMemcpy); later calls only launch. */
 ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,

@@ -76,6 +76,21 @@ def attention(Q, K, V, causal=True, out_dtype="bf16", scale=None, qpos=None):
     return rnd(core.attention(Q, K, V, scale, causal, qpos), out_dtype)
 
 
+def attention_lse(Q, K, causal=True, scale=None, qpos=None):
+    """Second output of the attention join-agg: lse[b,q,h] = log sum_k exp(scale * <Q[b,q,h,:], K[b,k,h,:]>) over the
+    keys the query joins with (k <= q when causal).  With it two partial results over disjoint key ranges combine as
+    O = w1 O1 + w2 O2, w_i = exp(lse_i - lse), lse = log(exp(lse_1) + exp(lse_2)) -- the online-softmax aggregation
+    written for normalised partials.  Plain numpy route (independent of the C engine); statistics are stored in f32."""
+    Q, K = np.asarray(Q, dtype=np.float64), np.asarray(K, dtype=np.float64)
+    scale = 1.0 / math.sqrt(Q.shape[-1]) if scale is None else scale
+    s = scale * np.einsum("bqhd,bkhd->bqhk", Q, K)
+    if causal:
+        pos = np.arange(Q.shape[1]) if qpos is None else np.asarray(qpos)
+        s = np.where(np.arange(K.shape[1])[None, None, None, :] <= pos[None, :, None, None], s, -np.inf)
+    m = s.max(axis=-1)
+    return rnd(m + np.log(np.exp(s - m[..., None]).sum(axis=-1)), "f32")
+
+
 def attention_gqa_packed(Q, K, V, group=1, ends=None, causal=True, out_dtype="bf16", scale=None):
     """Grouped-query attention over packed sequences (Example 3.10). Q[b,s,hq,d], K,V[b,s,hkv,d] with hq = group*hkv:
     query heads [group*m, group*(m+1)) attend key/value head m; the sequence index holds independent sequences ending

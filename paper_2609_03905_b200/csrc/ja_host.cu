@@ -758,7 +758,8 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
     if (!spec || !inputs || !outputs) return ja_fail(JA_ERR_INVALID_ARG, "spec / inputs / outputs is NULL");
     const int n_in = (int)spec->ins.size();
     if (n_inputs != n_in) return ja_fail(JA_ERR_INVALID_ARG, "spec has %d operands, %d relations given", n_in, n_inputs);
-    if (n_outputs != 1) return ja_fail(JA_ERR_UNSUPPORTED, "exactly one output relation is supported");
+    if (n_outputs != 1 && !(n_outputs == 2 && spec->fn == JA_FN_ATTENTION))
+        return ja_fail(JA_ERR_UNSUPPORTED, "one output relation, or two for ATTENTION (O and the log of the softmax denominator)");
     ja_status_t st;
     for (int k = 0; k < n_in; ++k)
         if ((st = check_tiling(spec, k, inputs[k])) != JA_OK) return st;
@@ -955,6 +956,26 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         AttnArgs aa;
         memset(&aa, 0, sizeof aa);
         aa.q = ja_view(Q); aa.k = ja_view(K); aa.v = ja_view(V); aa.o = ja_view(out);
+        if (n_outputs == 2) {   // second output: lse[b, q, h], f32, tiled like the (b, q, h) indices of the output
+            ja_relation* L = outputs[1];
+            if (!L || L->rank != 3 || L->dtype != JA_F32) return ja_fail(JA_ERR_DTYPE, "the second attention output is an f32 relation over (b, q, h)");
+            for (int d = 0; d < 3; ++d)
+                if (L->extent[d] != out->extent[d] || L->splits[d] != out->splits[d])
+                    return ja_fail(JA_ERR_PARTITION_MISMATCH, "the second attention output must be tiled like the first along its three indices");
+            if ((st = ja_relation_to_device(L)) != JA_OK) return st;
+            aa.lse = ja_view(L);
+            // same closed form as bshd_rows_layout, for cells of 4 bytes and no last index
+            bool okl = L->bs[0] && L->bs[2];
+            const int64_t S = L->extent[1], bblk = L->bs[0], hblk = L->bs[2], nhb = L->nblk[2];
+            for (int32_t bb = 0; okl && bb < L->nblk[0]; ++bb)
+                for (int32_t sb = 0; okl && sb < L->nblk[1]; ++sb)
+                    for (int32_t hb = 0; okl && hb < L->nblk[2]; ++hb) {
+                        const int64_t start = L->splits[1][sb], rows = L->splits[1][sb + 1] - start;
+                        okl = L->blk_off[((int64_t)bb * L->nblk[1] + sb) * L->nblk[2] + hb] ==
+                              ((bb * bblk * S + bblk * start) * nhb + hb * bblk * rows) * hblk * 4;
+                    }
+            aa.lse_rows_layout = okl;
+        }
         aa.B = (int32_t)Q->extent[0]; aa.S = (int32_t)Q->extent[1]; aa.H = (int32_t)Q->extent[2]; aa.D = 128;
         aa.group = (int32_t)(Q->extent[2] / K->extent[2]);
         int64_t g = Q->extent[1];
@@ -972,7 +993,7 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         std::vector<int32_t> qs(Q->splits[1].begin(), Q->splits[1].end()), ks(K->splits[1].begin(), K->splits[1].end());
         aa.q_split = qs.data();
         aa.k_split = ks.data();
-        aa.rows_layout = bshd_rows_layout(Q) && bshd_rows_layout(K) && bshd_rows_layout(V) && bshd_rows_layout(out) &&
+        aa.rows_layout = (n_outputs == 1 || aa.lse_rows_layout) && bshd_rows_layout(Q) && bshd_rows_layout(K) && bshd_rows_layout(V) && bshd_rows_layout(out) &&
                          V->splits[1] == K->splits[1] && V->bs[0] == K->bs[0] && V->bs[2] == K->bs[2] &&
                          out->splits[1] == Q->splits[1] && out->bs[0] == Q->bs[0] && out->bs[2] == Q->bs[2];
         return ja_launch_attention(aa, stream);

@@ -142,6 +142,8 @@ ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st);
 // Attention join-agg (QK^T join, online-softmax aggregation, PV).
 struct AttnArgs {
     RelView q, k, v, o;
+    RelView lse;           // optional second output [b, q, h] f32: log of the softmax denominator; base == nullptr if absent
+    bool lse_rows_layout;  // lse blocks follow the closed-form order of q's (b, s, h) blocks (tensor-memory kernels)
     float scale;
     int causal;
     int32_t B, S, H, D;    // H = query heads

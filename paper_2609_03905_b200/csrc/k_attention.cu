@@ -231,6 +231,13 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
     }
     const float inv0 = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f, inv1 = l_run[1] > 0.f ? 1.f / l_run[1] : 0.f;
+    if (a.lse.base && t4 == 0) {   // second output: log of the softmax denominator (scores were kept in base 2)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int64_t x[3] = {b, row0 + 8 * r, h};
+            *reinterpret_cast<float*>(a.lse.base + ja_elem_off(a.lse, x)) = (m_run[r] + log2f(l_run[r])) * 0.6931471805599453f;
+        }
+    }
     {
         const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
 #pragma unroll

@@ -51,6 +51,7 @@ struct SeqGeom {
 
 struct AttnTcParams {
     char* o_base;
+    float* lse_base;             // optional second output (nullptr if absent), addressed like o without the last index
     int32_t* status;
     int32_t B, S, H;
     int32_t group;               // query heads per key/value head
@@ -358,7 +359,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 fold(ls, alpha_prev);
                 // ---- O = O~ / l, one rounding, 256 contiguous bytes per row ----
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                char* dst = p.o_base + ((int64_t)seq_row(p.q, p.S, b, q0 + r, h) * p.q.hblk + h % p.q.hblk) * (D * 2);
+                const int64_t cell = (int64_t)seq_row(p.q, p.S, b, q0 + r, h) * p.q.hblk + h % p.q.hblk;
+                char* dst = p.o_base + cell * (D * 2);
+                if (p.lse_base) p.lse_base[cell] = (m_run + log2f(l_run)) * 0.6931471805599453f;   // scores were kept in base 2
 #pragma unroll
                 for (int g = 0; g < 16; ++g) {
                     uint4 ov;
@@ -643,7 +646,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
                 tc_fence_after();
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                char* dst = p.o_base + ((int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk) * (D * 2);
+                const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
+                char* dst = p.o_base + cell * (D * 2);
+                if (p.lse_base) p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -717,6 +722,7 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
     if ((s = encode_rows(a.k, &tk)) != JA_OK) return s;
     if ((s = encode_rows(a.v, &tv)) != JA_OK) return s;
     p.o_base = a.o.base;
+    p.lse_base = reinterpret_cast<float*>(a.lse.base);
     p.status = ja_device_status_word();
     if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
     p.B = a.B; p.S = a.S; p.H = a.H;

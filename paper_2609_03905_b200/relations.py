@@ -58,8 +58,10 @@ class Spec:
         self.einsum, self.parts = einsum, parts
         self.handle = B.ja_spec_create(einsum, parts, fn, fn_params, agg)
 
-    def execute(self, inputs, output: Relation, stream: int | None = None):
-        B.ja_execute(self.handle, [r.handle for r in inputs], [output.handle],
+    def execute(self, inputs, output, stream: int | None = None):
+        """output: one relation, or a list of relations for multi-output specs (attention: [O, lse])."""
+        outs = output if isinstance(output, (list, tuple)) else [output]
+        B.ja_execute(self.handle, [r.handle for r in inputs], [r.handle for r in outs],
                      current_stream() if stream is None else stream)
 
     def execute_join(self, inputs, partials: Relation, stream: int | None = None):

@@ -237,6 +237,30 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
 
 
+@pytest.mark.parametrize("form", ["default", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("causal,S,hb", [(True, 512, 1), (False, 384, 2), (True, 256, 2)])
+def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
+    """n_outputs = 2: the log of the softmax denominator beside O, and the combine it exists for."""
+    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
+    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
+    B, H, D = 2, 4, 128
+    Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (21, 22, 23))
+    sp = [ES(B, B), ES(S, S // 128), ES(H, H // hb), [0, D]]
+    rQ, rK, rV = upload(Q, sp), upload(K, sp), upload(V, sp)
+    rO = empty_like_tiling([B, S, H, D], sp, BF, fill=float("nan"))
+    rL = empty_like_tiling([B, S, H], sp[:3], F32, fill=float("nan"))
+    parts = {"b": sp[0], "q": sp[1], "h": sp[2], "d": sp[3], "k": sp[1]}
+    spec = ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / np.sqrt(D), 1.0 if causal else 0.0), "online_softmax")
+    spec.execute([rQ, rK, rV], [rO, rL])
+    got_o, got_l = download(rO), download(rL)
+    check_status()
+    assert relfro(got_o, operators.attention(si.to_f64(Q), si.to_f64(K), si.to_f64(V), causal, "bf16")) <= TOL[BF]
+    ref_l = operators.attention_lse(si.to_f64(Q), si.to_f64(K), causal)
+    assert np.abs(got_l - ref_l).max() <= 2e-3        # absolute: lse is a logarithm; 2e-3 = a relative 2e-3 on the denominator
+    with pytest.raises(ja.JaError):                   # the second output must be tiled like the first
+        spec.execute([rQ, rK, rV], [rO, empty_like_tiling([B, S, H], [sp[0], ES(S, 1), sp[2]], F32)])
+
+
 # grouped-query attention over packed sequences (Example 3.10): query head h joins key/value head h // group and
 # no tuple crosses a sequence end. `cut` says where the sequence index is split: "ends" = at the sequence ends only
 # (irregular blocks), an integer = uniform blocks of that many rows (every end is then a split point).

@@ -535,3 +535,26 @@ def test_optimizer_dynamic_program_equals_exhaustive_search():
         assert dp_cost == ex_cost == optimizer.plan_cost(ops, dp_plan)
         for op, J in zip(ops, dp_plan):
             assert int(np.prod(list(J.values()))) == p and all(J[c] == 1 for c in op.get("fixed", ()))
+
+
+def test_attention_lse_combines_partial_results():
+    """The second attention output pins itself against the first: attention over two disjoint key ranges, combined with
+    weights exp(lse_i - lse), must equal attention over all keys (the O side comes from the C engine, lse from numpy)."""
+    B, S, H, D = 2, 24, 3, 8
+    Q, K, V = (RNG.standard_normal((B, S, H, D)) for _ in range(3))
+    lse = operators.attention_lse(Q, K, causal=False).astype(np.float64)
+    want = operators.attention(Q, K, V, causal=False, out_dtype=None)
+    parts = []
+    for k0, k1 in ((0, 10), (10, 24)):
+        parts.append((operators.attention(Q, K[:, k0:k1], V[:, k0:k1], causal=False, out_dtype=None),
+                      operators.attention_lse(Q, K[:, k0:k1], causal=False).astype(np.float64)))
+    tot = np.log(sum(np.exp(l) for _, l in parts))
+    np.testing.assert_allclose(tot, lse, rtol=1e-6, atol=1e-6)                      # f32-rounded statistics
+    got = sum(o * np.exp(l - tot)[..., None] for o, l in parts)
+    np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-6)
+    # causal: the first row joins one key, so lse is that single score; closed form
+    lc = operators.attention_lse(Q, K, causal=True).astype(np.float64)
+    np.testing.assert_allclose(lc[:, 0], np.einsum("bhd,bhd->bh", Q[:, 0], K[:, 0]) / np.sqrt(D), rtol=1e-6, atol=1e-6)
+    # all keys equal: lse = score + log(number of keys)
+    K1 = np.repeat(K[:, :1], S, axis=1)
+    np.testing.assert_allclose(operators.attention_lse(Q, K1, causal=False), np.einsum("bqhd,bhd->bqh", Q, K[:, 0]) / np.sqrt(D) + np.log(S), rtol=1e-6, atol=1e-6)
