@@ -53,6 +53,32 @@ def test_matmul_plain_alu_uneven_tilings():
     assert relfro(got, ref) <= TOL[BF]
 
 
+def test_degenerate_tilings_scalar_keys_and_single_block():
+    """The two ends of the decomposition space: every sub-tensor one scalar (the classical relational form: key = cell,
+    p = 12 * 10 * 9 function specs, m = 10 tuples per output key) and one block per relation (p = 1, no aggregation)."""
+    unit = lambda n: list(range(n + 1))
+    for dt in (F32, BF):
+        got, ref = _matmul_case(12, 10, 9, unit(12), unit(10), unit(9), dt)
+        assert relfro(got, ref) <= TOL[dt]
+        got1, ref1 = _matmul_case(12, 10, 9, [0, 12], [0, 10], [0, 9], dt)
+        assert relfro(got1, ref1) <= TOL[dt] and relfro(got, got1) <= TOL[dt]
+    # relayout between the two ends, bit-exact both ways
+    x = si.normal((12, 9), 0.0, 1.0, F32, 1, 7)
+    one, cells = [[0, 12], [0, 9]], [unit(12), unit(9)]
+    r1 = upload(x, one)
+    rc = empty_like_tiling([12, 9], cells, F32)
+    ja.repartition(r1, rc)
+    assert np.array_equal(download_bits(rc), blocked.pack(np_bits(x), cells))
+    back = empty_like_tiling([12, 9], one, F32)
+    ja.repartition(rc, back)
+    assert np.array_equal(download_bits(back), download_bits(r1))
+    # a row-structured join-agg over scalar blocks (sum of squares: m = 9 tuples per row key)
+    ss = ja.Relation([12], [unit(12)], F32)
+    ja.Spec("ij->i", {"i": unit(12), "j": unit(9)}, "square", (), "sum").execute([rc], ss)
+    assert relfro(download(ss), operators.sumsq_rows(si.to_f64(x))) <= TOL[F32]
+    check_status()
+
+
 # ---------------------------------------------------------------------------------------------------
 # tensor-core matmul join-agg (bf16 relations, uniform blocks)
 # ---------------------------------------------------------------------------------------------------
