@@ -225,6 +225,14 @@ typedef struct {
 } ja_plan_node_t;
 ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
 ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost);
+/* Outputs with several consumers (Section 4.4): the graph (nodes in topological order; a node may be consumed any number
+ * of times) is cut at every edge out of a multiply consumed tensor; the resulting trees are optimised with Algorithm 1
+ * one at a time, largest first (ties: smaller root first), each subject to the specs already fixed: an operand produced
+ * in an already-optimised tree enters like an input of the computation whose tiling is fixed (Cost charges the repartition
+ * on a mismatch); an operand produced in a tree still to come enters like a free input; the root of a tree is chosen with
+ * the repartition charges of its already-planned consumers added. total_cost is the summed Cost of the assembled plan
+ * (what ja_plan_cost returns for it). On a tree the result equals ja_plan_optimize. */
+ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
 
 /* ---- relayout without allocation -------------------------------------------------------------------
  * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)

@@ -132,3 +132,89 @@ def exhaustive(ops, p: int):
         if best is None or c < best:
             best, best_plan = c, list(plan)
     return best, best_plan
+
+
+# ---------------------------------------------------------------------------------------------------
+# Outputs with several consumers (Section 4.4): the graph is cut at every edge out of a multiply
+# consumed tensor and the resulting trees are optimised one at a time, largest first, each subject
+# to the specs already fixed.
+# ---------------------------------------------------------------------------------------------------
+def cut_into_trees(ops):
+    """Returns [(root, sorted member nodes)], largest tree first (ties: smaller root first).  Roots are the
+    operators whose output is not consumed exactly once; a tree is its root plus every producer reachable
+    through singly-consumed outputs."""
+    consumers = [0] * len(ops)
+    for op in ops:
+        for q in op["inputs"]:
+            if q is not None:
+                consumers[q] += 1
+    trees = []
+    for root in range(len(ops)):
+        if consumers[root] == 1:
+            continue
+        members, stack = [], [root]
+        while stack:
+            i = stack.pop()
+            members.append(i)
+            stack += [q for q in ops[i]["inputs"] if q is not None and consumers[q] == 1]
+        trees.append((root, sorted(members)))
+    trees.sort(key=lambda t: (-len(t[1]), t[0]))
+    return trees
+
+
+def optimize_graph(ops, p: int):
+    """Section 4.4.  An operand produced in a tree that is already optimised enters like an input whose tiling
+    is fixed (Cost charges the repartition when in_k(J) differs from it); an operand produced in a tree not
+    yet optimised enters like an input of the computation.  When the root of a tree feeds consumers whose
+    specs are already fixed, the root's tiling is chosen with their repartition charges added (the paper only
+    says 'subject to the specs already fixed'; this is the reading taken).
+    Returns (plan_cost of the assembled plan, plan)."""
+    plan = [None] * len(ops)
+    for root, members in cut_into_trees(ops):
+        inside = set(members)
+        cand, opt, choice = {}, {}, {}
+        for idx in members:                     # members are sorted = topological
+            op = ops[idx]
+            cand[idx] = []
+            for J in specs(op, p):
+                lists = []
+                for q in op["inputs"]:
+                    if q is None or (q not in inside and plan[q] is None):
+                        lists.append([None])
+                    elif q in inside:
+                        lists.append(cand[q])
+                    else:
+                        lists.append([tiling_of(ops[q], plan[q], -1)])
+                best, best_T = None, None
+                for Ts in itertools.product(*lists):
+                    b = cost(op, J, Ts) + sum(opt[(q, T)] for q, T in zip(op["inputs"], Ts) if q is not None and q in inside)
+                    if best is None or b < best:
+                        best, best_T = b, Ts
+                T = tiling_of(op, J, -1)
+                if T not in cand[idx] or best < opt[(idx, T)]:
+                    if T not in cand[idx]:
+                        cand[idx].append(T)
+                    opt[(idx, T)] = best
+                    choice[(idx, T)] = (J, best_T)
+
+        def consumer_charge(T):
+            c = 0
+            for j, op in enumerate(ops):
+                if plan[j] is None:
+                    continue
+                for k, q in enumerate(op["inputs"]):
+                    if q == root and tiling_of(op, plan[j], k) != T:
+                        c += card(op, k)
+            return c
+
+        T_star = min(cand[root], key=lambda T: opt[(root, T)] + consumer_charge(T))
+
+        def assign(idx, T):
+            J, Ts = choice[(idx, T)]
+            plan[idx] = J
+            for q, Tq in zip(ops[idx]["inputs"], Ts):
+                if q is not None and q in inside:
+                    assign(q, Tq)
+
+        assign(root, T_star)
+    return plan_cost(ops, plan), plan

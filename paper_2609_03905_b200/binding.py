@@ -66,6 +66,7 @@ def _load() -> ctypes.CDLL:
         "ja_execute_join": [vp, P(vp), i32, vp, vp],
         "ja_plan_optimize": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_plan_cost": [P(ja_plan_node_t), i32, P(i32), P(i64)],
+        "ja_plan_optimize_graph": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_repartition_agg": [vp, ctypes.c_int, vp, vp],
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
@@ -244,6 +245,16 @@ def ja_plan_optimize(ops, p: int):
     counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
     total = ctypes.c_int64()
     _check(LIB.ja_plan_optimize(arr, len(ops), p, counts, ctypes.byref(total)))
+    plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
+    return total.value, plan
+
+
+def ja_plan_optimize_graph(ops, p: int):
+    """Section 4.4: a graph with multiply consumed tensors, cut into trees and optimised tree by tree."""
+    arr, keep = _plan_nodes(ops)
+    counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
+    total = ctypes.c_int64()
+    _check(LIB.ja_plan_optimize_graph(arr, len(ops), p, counts, ctypes.byref(total)))
     plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
     return total.value, plan
 

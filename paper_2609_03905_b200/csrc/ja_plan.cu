@@ -9,6 +9,7 @@
 //   repartition  card(T_k) when operand k comes from a producer whose output tiling differs from in_k(J)
 #include <string.h>
 
+#include <algorithm>
 #include <map>
 #include <string>
 #include <vector>
@@ -113,13 +114,14 @@ void enum_specs(const Op& op, int32_t p, size_t l, Counts* cur, std::vector<Coun
 
 struct Choice {
     Counts spec;
-    std::vector<Counts> in_tilings;   // chosen T_k per operand (empty for inputs of the computation)
+    std::vector<Counts> in_tilings;   // chosen T_k per operand produced inside the tree (empty otherwise)
 };
 
-ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, std::vector<Op>* ops) {
+// allow_sharing = false: every node but the last must be consumed exactly once (a tree, Section 4.2)
+ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, bool allow_sharing, std::vector<Op>* ops, std::vector<int>* consumers) {
     if (!nodes || n_nodes < 1) return ja_fail(JA_ERR_INVALID_ARG, "no nodes");
     ops->resize(n_nodes);
-    std::vector<int> consumers(n_nodes, 0);
+    consumers->assign(n_nodes, 0);
     for (int32_t i = 0; i < n_nodes; ++i) {
         ja_status_t st = parse_op(nodes[i], i, &(*ops)[i]);
         if (st != JA_OK) return st;
@@ -132,34 +134,43 @@ ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, std::vector<
             for (size_t d = 0; d < pr.out.size(); ++d)
                 if (pr.extent[pos(pr.letters, pr.out[d])] != op.extent[pos(op.letters, op.ins[k][d])])
                     return ja_fail(JA_ERR_SHAPE, "node %d operand %zu: extent %zu differs from its producer's output", i, k, d);
-            if (++consumers[q] > 1) return ja_fail(JA_ERR_UNSUPPORTED, "node %d is consumed twice: cut the graph into trees first (Section 4.4)", q);
+            if (++(*consumers)[q] > 1 && !allow_sharing)
+                return ja_fail(JA_ERR_UNSUPPORTED, "node %d is consumed twice: use ja_plan_optimize_graph, which cuts the graph into trees (Section 4.4)", q);
         }
     }
-    for (int32_t i = 0; i + 1 < n_nodes; ++i)
-        if (consumers[i] != 1) return ja_fail(JA_ERR_INVALID_ARG, "node %d is not consumed: the last node must be the root of a tree", i);
+    if (!allow_sharing)
+        for (int32_t i = 0; i + 1 < n_nodes; ++i)
+            if ((*consumers)[i] != 1) return ja_fail(JA_ERR_INVALID_ARG, "node %d is not consumed: the last node must be the root of a tree", i);
     return JA_OK;
 }
 
-}  // namespace
-
-extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost) {
-    if (p < 1 || !counts) return ja_fail(JA_ERR_INVALID_ARG, "p must be positive and counts non-NULL");
-    std::vector<Op> ops;
-    ja_status_t st = parse_all(nodes, n_nodes, &ops);
-    if (st != JA_OK) return st;
-    // cand[Op] in insertion order, Opt[Op, T], choice[Op, T]
-    std::vector<std::vector<Counts>> cand(n_nodes);
-    std::vector<std::map<Counts, int64_t>> opt(n_nodes);
-    std::vector<std::map<Counts, Choice>> choice(n_nodes);
-    for (int32_t i = 0; i < n_nodes; ++i) {
+// Algorithm 1 on the tree `members` (ascending = topological) rooted at `root`. An operand produced outside the tree by a
+// node that already has a spec enters with that node's output tiling fixed (Cost charges the repartition on a mismatch);
+// any other outside operand enters like an input of the computation. If `charge_consumers`, the root's tiling is chosen
+// with the repartition charges of its already-planned consumers added. Fills plan[] for the members.
+ja_status_t optimize_tree(const std::vector<Op>& ops, const std::vector<int32_t>& members, int32_t root, int32_t p,
+                          bool charge_consumers, std::vector<Counts>* plan, int64_t* tree_cost) {
+    std::vector<char> inside(ops.size(), 0);
+    for (int32_t i : members) inside[i] = 1;
+    std::map<int32_t, std::vector<Counts>> cand;
+    std::map<int32_t, std::map<Counts, int64_t>> opt;
+    std::map<int32_t, std::map<Counts, Choice>> choice;
+    for (int32_t i : members) {
         const Op& op = ops[i];
         std::vector<Counts> specs;
         Counts cur;
         enum_specs(op, p, 0, &cur, &specs);
         if (specs.empty()) return ja_fail(JA_ERR_TILING, "node %d has no decomposition into %d function specs", i, p);
         const size_t n = op.ins.size();
+        std::vector<Counts> fixed(n);               // tiling of an operand whose producer is planned outside the tree
+        std::vector<int> kind(n, 0);                // 0 free, 1 produced inside the tree, 2 fixed
+        for (size_t k = 0; k < n; ++k) {
+            const int32_t q = op.producers[k];
+            if (q < 0) continue;
+            if (inside[q]) kind[k] = 1;
+            else if (!(*plan)[q].empty()) { kind[k] = 2; fixed[k] = tiling(ops[q], (*plan)[q], ops[q].out); }
+        }
         for (const Counts& J : specs) {
-            // B(J): minimum over the producers' candidate tilings (odometer over cand lists; inputs have one entry)
             std::vector<size_t> idx(n, 0);
             int64_t best = -1;
             std::vector<size_t> best_idx;
@@ -167,17 +178,18 @@ extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_n
                 std::vector<const Counts*> Ts(n, nullptr);
                 int64_t b = 0;
                 for (size_t k = 0; k < n; ++k) {
-                    const int32_t q = op.producers[k];
-                    if (q < 0) continue;
-                    Ts[k] = &cand[q][idx[k]];
-                    b += opt[q][*Ts[k]];
+                    if (kind[k] == 1) {
+                        Ts[k] = &cand[op.producers[k]][idx[k]];
+                        b += opt[op.producers[k]][*Ts[k]];
+                    } else if (kind[k] == 2) {
+                        Ts[k] = &fixed[k];
+                    }
                 }
                 b += cost(op, J, Ts);
                 if (best < 0 || b < best) { best = b; best_idx = idx; }
                 int k = (int)n - 1;
                 for (; k >= 0; --k) {
-                    const int32_t q = op.producers[k];
-                    const size_t lim = q < 0 ? 1 : cand[q].size();
+                    const size_t lim = kind[k] == 1 ? cand[op.producers[k]].size() : 1;
                     if (++idx[k] < lim) break;
                     idx[k] = 0;
                 }
@@ -192,18 +204,28 @@ extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_n
                 c.spec = J;
                 c.in_tilings.resize(n);
                 for (size_t k = 0; k < n; ++k)
-                    if (op.producers[k] >= 0) c.in_tilings[k] = cand[op.producers[k]][best_idx[k]];
+                    if (kind[k] == 1) c.in_tilings[k] = cand[op.producers[k]][best_idx[k]];
                 choice[i][T] = c;
             }
         }
     }
-    const int32_t root = n_nodes - 1;
+    auto consumer_charge = [&](const Counts& T) {
+        int64_t c = 0;
+        if (!charge_consumers) return c;
+        for (size_t j = 0; j < ops.size(); ++j) {
+            if ((*plan)[j].empty()) continue;
+            for (size_t k = 0; k < ops[j].ins.size(); ++k)
+                if (ops[j].producers[k] == root && tiling(ops[j], (*plan)[j], ops[j].ins[k]) != T) c += card(ops[j], ops[j].ins[k]);
+        }
+        return c;
+    };
     const Counts* T_star = nullptr;
-    for (const Counts& T : cand[root])
-        if (!T_star || opt[root][T] < opt[root][*T_star]) T_star = &T;
-    if (total_cost) *total_cost = opt[root][*T_star];
-    // Assign: walk back from the root
-    memset(counts, 0, sizeof(int32_t) * (size_t)n_nodes * JA_PLAN_MAX_LETTERS);
+    int64_t best_total = -1;
+    for (const Counts& T : cand[root]) {
+        const int64_t v = opt[root][T] + consumer_charge(T);
+        if (!T_star || v < best_total) { T_star = &T; best_total = v; }
+    }
+    if (tree_cost) *tree_cost = opt[root][*T_star];
     std::vector<std::pair<int32_t, Counts>> stack;
     stack.push_back({root, *T_star});
     while (!stack.empty()) {
@@ -211,33 +233,97 @@ extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_n
         const Counts T = stack.back().second;
         stack.pop_back();
         const Choice& c = choice[i][T];
-        for (size_t l = 0; l < c.spec.size(); ++l) counts[(size_t)i * JA_PLAN_MAX_LETTERS + l] = c.spec[l];
+        (*plan)[i] = c.spec;
         for (size_t k = 0; k < ops[i].ins.size(); ++k)
-            if (ops[i].producers[k] >= 0) stack.push_back({ops[i].producers[k], c.in_tilings[k]});
+            if (ops[i].producers[k] >= 0 && inside[ops[i].producers[k]]) stack.push_back({ops[i].producers[k], c.in_tilings[k]});
     }
+    return JA_OK;
+}
+
+void write_counts(const std::vector<Counts>& plan, int32_t* counts) {
+    memset(counts, 0, sizeof(int32_t) * plan.size() * JA_PLAN_MAX_LETTERS);
+    for (size_t i = 0; i < plan.size(); ++i)
+        for (size_t l = 0; l < plan[i].size(); ++l) counts[i * JA_PLAN_MAX_LETTERS + l] = plan[i][l];
+}
+
+int64_t assembled_cost(const std::vector<Op>& ops, const std::vector<Counts>& plan) {
+    int64_t total = 0;
+    for (size_t i = 0; i < ops.size(); ++i) {
+        std::vector<Counts> outs(ops[i].ins.size());
+        std::vector<const Counts*> Ts(ops[i].ins.size(), nullptr);
+        for (size_t k = 0; k < ops[i].ins.size(); ++k)
+            if (ops[i].producers[k] >= 0) {
+                outs[k] = tiling(ops[ops[i].producers[k]], plan[ops[i].producers[k]], ops[ops[i].producers[k]].out);
+                Ts[k] = &outs[k];
+            }
+        total += cost(ops[i], plan[i], Ts);
+    }
+    return total;
+}
+
+}  // namespace
+
+extern "C" ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost) {
+    if (p < 1 || !counts) return ja_fail(JA_ERR_INVALID_ARG, "p must be positive and counts non-NULL");
+    std::vector<Op> ops;
+    std::vector<int> consumers;
+    ja_status_t st = parse_all(nodes, n_nodes, false, &ops, &consumers);
+    if (st != JA_OK) return st;
+    std::vector<int32_t> members(n_nodes);
+    for (int32_t i = 0; i < n_nodes; ++i) members[i] = i;
+    std::vector<Counts> plan(n_nodes);
+    if ((st = optimize_tree(ops, members, n_nodes - 1, p, false, &plan, total_cost)) != JA_OK) return st;
+    write_counts(plan, counts);
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost) {
+    if (p < 1 || !counts) return ja_fail(JA_ERR_INVALID_ARG, "p must be positive and counts non-NULL");
+    std::vector<Op> ops;
+    std::vector<int> consumers;
+    ja_status_t st = parse_all(nodes, n_nodes, true, &ops, &consumers);
+    if (st != JA_OK) return st;
+    // cut at every edge out of a multiply consumed tensor: roots are the nodes not consumed exactly once
+    std::vector<std::pair<int32_t, std::vector<int32_t>>> trees;
+    for (int32_t root = 0; root < n_nodes; ++root) {
+        if (consumers[root] == 1) continue;
+        std::vector<int32_t> members, stack(1, root);
+        while (!stack.empty()) {
+            const int32_t i = stack.back();
+            stack.pop_back();
+            members.push_back(i);
+            for (int32_t q : ops[i].producers)
+                if (q >= 0 && consumers[q] == 1) stack.push_back(q);
+        }
+        std::sort(members.begin(), members.end());
+        trees.push_back({root, members});
+    }
+    std::stable_sort(trees.begin(), trees.end(), [](const std::pair<int32_t, std::vector<int32_t>>& a, const std::pair<int32_t, std::vector<int32_t>>& b) {
+        return a.second.size() != b.second.size() ? a.second.size() > b.second.size() : a.first < b.first;
+    });
+    std::vector<Counts> plan(n_nodes);
+    for (const auto& t : trees)
+        if ((st = optimize_tree(ops, t.second, t.first, p, true, &plan, nullptr)) != JA_OK) return st;
+    write_counts(plan, counts);
+    if (total_cost) *total_cost = assembled_cost(ops, plan);
     return JA_OK;
 }
 
 extern "C" ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost) {
     if (!counts || !total_cost) return ja_fail(JA_ERR_INVALID_ARG, "counts / total_cost is NULL");
     std::vector<Op> ops;
-    ja_status_t st = parse_all(nodes, n_nodes, &ops);
+    std::vector<int> consumers;
+    ja_status_t st = parse_all(nodes, n_nodes, true, &ops, &consumers);
     if (st != JA_OK) return st;
-    std::vector<Counts> spec(n_nodes), out_tiling(n_nodes);
-    int64_t total = 0;
+    std::vector<Counts> plan(n_nodes);
     for (int32_t i = 0; i < n_nodes; ++i) {
         const Op& op = ops[i];
         for (size_t l = 0; l < op.letters.size(); ++l) {
             const int32_t c = counts[(size_t)i * JA_PLAN_MAX_LETTERS + l];
             if (c < 1 || c > op.extent[l]) return ja_fail(JA_ERR_TILING, "node %d letter '%c': %d intervals", i, op.letters[l], c);
-            spec[i].push_back(c);
+            plan[i].push_back(c);
         }
-        out_tiling[i] = tiling(op, spec[i], op.out);
-        std::vector<const Counts*> Ts(op.ins.size(), nullptr);
-        for (size_t k = 0; k < op.ins.size(); ++k)
-            if (op.producers[k] >= 0) Ts[k] = &out_tiling[op.producers[k]];
-        total += cost(op, spec[i], Ts);
     }
-    *total_cost = total;
+    *total_cost = assembled_cost(ops, plan);
     return JA_OK;
 }

@@ -285,3 +285,16 @@ def test_logical_optimizer_matches_oracle(golden_dir):
         ja.ja_plan_optimize([ch["ops"][0], {"einsum": "ik,ik->ik", "extents": {"i": 4, "k": 4}, "inputs": [0, 0]}], 2)
     with pytest.raises(ja.JaError):   # producer / operand shapes must agree
         ja.ja_plan_optimize([ch["ops"][0], {"einsum": "ik->i", "extents": {"i": 4, "k": 5}, "inputs": [0]}], 2)
+
+
+def test_logical_optimizer_on_graphs_with_shared_tensors():
+    """Section 4.4 through the library against the oracle: same trees, same order, same assembled cost."""
+    from oracle import optimizer
+    from test_oracle_pins import _block_graph
+    for dims, p in (((16, 8, 12), 2), ((16, 8, 12), 4), ((64, 32, 48), 8)):
+        ops = _block_graph(*dims)
+        want, want_plan = optimizer.optimize_graph(ops, p)
+        got, plan = ja.ja_plan_optimize_graph(ops, p)
+        assert got == want == optimizer.plan_cost(ops, plan) == ja.ja_plan_cost(ops, plan)
+    tree = _mlp_tree(100, 36, 50)
+    assert ja.ja_plan_optimize_graph(tree, 12)[0] == ja.ja_plan_optimize(tree, 12)[0]

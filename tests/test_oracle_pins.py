@@ -558,3 +558,44 @@ def test_attention_lse_combines_partial_results():
     # all keys equal: lse = score + log(number of keys)
     K1 = np.repeat(K[:, :1], S, axis=1)
     np.testing.assert_allclose(operators.attention_lse(Q, K1, causal=False), np.einsum("bqhd,bhd->bqh", Q, K[:, 0]) / np.sqrt(D) + np.log(S), rtol=1e-6, atol=1e-6)
+
+
+def _block_graph(T=16, d=8, f=12, S=4):
+    """The operators of a transformer block as a DAG with multiply consumed tensors (x, n1, h): small extents."""
+    E = lambda **k: k
+    return [
+        {"einsum": "ij,j->ij", "extents": E(i=T, j=d), "inputs": [None, None]},                       # 0 n1 = norm(x)
+        {"einsum": "ij,jk->ik", "extents": E(i=T, j=d, k=d), "inputs": [0, None]},                    # 1 q
+        {"einsum": "ij,jk->ik", "extents": E(i=T, j=d, k=d), "inputs": [0, None]},                    # 2 k
+        {"einsum": "ij,jk->ik", "extents": E(i=T, j=d, k=d), "inputs": [0, None]},                    # 3 v
+        {"einsum": "ik,ik,ik->ik", "extents": E(i=T, k=d), "inputs": [1, 2, 3]},                      # 4 att (row-local stand-in)
+        {"einsum": "ik,kl,il->il", "extents": E(i=T, k=d, l=d), "inputs": [4, None, None]},           # 5 h = x + att Wo
+        {"einsum": "ij,j->ij", "extents": E(i=T, j=d), "inputs": [5, None]},                          # 6 n2
+        {"einsum": "ij,jk->ik", "extents": E(i=T, j=d, k=f), "inputs": [6, None]},                    # 7 a
+        {"einsum": "ij,jk->ik", "extents": E(i=T, j=d, k=f), "inputs": [6, None]},                    # 8 b
+        {"einsum": "ik,ik->ik", "extents": E(i=T, k=f), "inputs": [7, 8]},                            # 9 silu(a) b
+        {"einsum": "ik,kl,il->il", "extents": E(i=T, k=f, l=d), "inputs": [9, None, 5]},              # 10 out = h + . W2
+    ]
+
+
+def test_optimizer_graph_cut_into_trees():
+    from oracle import optimizer
+    ops = _block_graph()
+    trees = optimizer.cut_into_trees(ops)
+    # multiply consumed: n1 (0), h (5), n2 (6); final: 10
+    assert sorted(r for r, _ in trees) == [0, 5, 6, 10]
+    assert dict(trees)[5] == [1, 2, 3, 4, 5] and dict(trees)[10] == [7, 8, 9, 10] and dict(trees)[0] == [0] and dict(trees)[6] == [6]
+    assert [r for r, _ in trees] == [5, 10, 0, 6]                        # largest first, ties by root
+    for p in (2, 4):
+        total, plan = optimizer.optimize_graph(ops, p)
+        assert total == optimizer.plan_cost(ops, plan)
+        # the tree optimised last cannot be improved with everything else fixed (its root's consumers included)
+        last_root, members = trees[-1]
+        for alt in itertools.product(*[optimizer.specs(ops[i], p) for i in members]):
+            trial = list(plan)
+            for i, J in zip(members, alt):
+                trial[i] = J
+            assert optimizer.plan_cost(ops, trial) >= total
+    # on a tree the graph procedure is Algorithm 1
+    tree = _mlp_tree(8, 6, 12)
+    assert optimizer.optimize_graph(tree, 4)[0] == optimizer.optimize_tree(tree, 4)[0]
