@@ -171,29 +171,24 @@ ja_status_t optimize_tree(const std::vector<Op>& ops, const std::vector<int32_t>
             else if (!(*plan)[q].empty()) { kind[k] = 2; fixed[k] = tiling(ops[q], (*plan)[q], ops[q].out); }
         }
         for (const Counts& J : specs) {
-            std::vector<size_t> idx(n, 0);
-            int64_t best = -1;
-            std::vector<size_t> best_idx;
-            while (true) {
-                std::vector<const Counts*> Ts(n, nullptr);
-                int64_t b = 0;
-                for (size_t k = 0; k < n; ++k) {
-                    if (kind[k] == 1) {
-                        Ts[k] = &cand[op.producers[k]][idx[k]];
-                        b += opt[op.producers[k]][*Ts[k]];
-                    } else if (kind[k] == 2) {
-                        Ts[k] = &fixed[k];
+            // B(J). Cost is a sum over operands (join and repartition terms) plus the aggregation term, so the minimum over
+            // the producers' candidate tilings separates: each operand picks its own cheapest (Opt + repartition charge).
+            std::vector<const Counts*> none(n, nullptr);
+            int64_t best = cost(op, J, none);
+            std::vector<size_t> best_idx(n, 0);
+            for (size_t k = 0; k < n; ++k) {
+                const Counts need = tiling(op, J, op.ins[k]);
+                if (kind[k] == 2) {
+                    if (fixed[k] != need) best += card(op, op.ins[k]);
+                } else if (kind[k] == 1) {
+                    const std::vector<Counts>& cs = cand[op.producers[k]];
+                    int64_t bk = -1;
+                    for (size_t c = 0; c < cs.size(); ++c) {
+                        const int64_t v = opt[op.producers[k]][cs[c]] + (cs[c] != need ? card(op, op.ins[k]) : 0);
+                        if (bk < 0 || v < bk) { bk = v; best_idx[k] = c; }
                     }
+                    best += bk;
                 }
-                b += cost(op, J, Ts);
-                if (best < 0 || b < best) { best = b; best_idx = idx; }
-                int k = (int)n - 1;
-                for (; k >= 0; --k) {
-                    const size_t lim = kind[k] == 1 ? cand[op.producers[k]].size() : 1;
-                    if (++idx[k] < lim) break;
-                    idx[k] = 0;
-                }
-                if (k < 0) break;
             }
             const Counts T = tiling(op, J, op.out);
             auto it = opt[i].find(T);
