@@ -224,6 +224,23 @@ def run_gpu(args, shape):
     ms_total = t_start.elapsed_time(t_end)
     assert ja.ja_stream_status(stream.cuda_stream) == 0, "device status word set during the timed region"
 
+    # ---- the same K steps replayed from one CUDA graph of the chain (no per-op events inside a graph, so the per-op
+    # breakdown and the roofline above come from the eager region) ------------------------------------------------
+    graph = blk.capture()
+    sync_all()
+    for _ in range(3):
+        graph.replay()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    g0.record(stream)
+    for _ in range(args.steps):
+        graph.replay()
+    g1.record(stream)
+    sync_all()
+    ms_graph = g0.elapsed_time(g1)
+    assert ja.ja_stream_status(stream.cuda_stream) == 0, "device status word set during graph replay"
+    del graph
+
     # ---- end to end: every step copies its input from pinned host memory, packs it into the block's input relation
     # (ja_repartition), runs the block, recomposes the output (ja_repartition) and copies it back to the host. Steps are
     # independent, so the copies of neighbouring steps overlap the compute of this one: H2D on one stream, kernels on the
@@ -280,7 +297,7 @@ def run_gpu(args, shape):
     assert torch.equal(out_hosts[0], out_hosts[1]), "end-to-end outputs of consecutive steps differ"
 
     fl = block_flops(Bt, S, hidden, ffn, heads, shape.get("kv_heads"))
-    (ms_total, ms_e2e), (value, e2e_val) = replica_aggregate([ms_total, ms_e2e], fl, args.steps, world, device="cuda")
+    (ms_total, ms_e2e, ms_graph), (value, e2e_val, graph_val) = replica_aggregate([ms_total, ms_e2e, ms_graph], fl, args.steps, world, device="cuda")
     ms_step = ms_total / args.steps
 
     # ---- per-op breakdown and the roofline of the dominant kernel -----------------------------------------------------
@@ -339,6 +356,8 @@ def run_gpu(args, shape):
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "ms_per_step": ms_e2e / args.steps,
                 "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": out_host.numel() * 2},
+        "cuda_graph_replay": {"value": graph_val, "unit": "TFLOP/s", "ms_per_step": ms_graph / args.steps,
+                              "note": "the same steps replayed from one CUDA graph of the chain, timed after the eager region"},
         "roofline": roof, "cpu_baseline": cpu, "detail": detail}))
     if world > 1:
         dist.destroy_process_group()

@@ -165,6 +165,15 @@ class LlamaBlock:
         n += ["repartition_out"] if self.plan == "head" else []
         return n
 
+    def capture(self):
+        """The whole chain as one CUDA graph (the paper builds one graph per plan): returns a torch.cuda.CUDAGraph whose
+        replay() re-runs forward() on the relations of this block. Call forward() once before, so that every plan and
+        device table the library caches exists (creating them allocates, which a capture does not allow)."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.forward()
+        return g
+
     def forward(self, stream: int | None = None) -> Relation:
         """Enqueue the whole chain on the current stream; returns the output relation (tiled like x)."""
         p = self.plan

@@ -12,7 +12,7 @@ import synth_inputs as si
 from oracle import blocked, core, operators
 from paper_2609_03905_b200.llama_block import LlamaBlock
 
-from gpu_util import TOL, check_status, download, empty_like_tiling, relfro, upload
+from gpu_util import TOL, check_status, download, empty_like_tiling, np_bits, relfro, upload
 
 pytestmark = pytest.mark.gpu
 ES = blocked.equal_splits
@@ -198,6 +198,23 @@ def test_small_block_every_intermediate():
 # ---------------------------------------------------------------------------------------------------
 # the paper's own workloads (Section 7): the grouped-query block and the matrix chains
 # ---------------------------------------------------------------------------------------------------
+def test_block_replayed_from_a_cuda_graph():
+    """The chain captured into one CUDA graph replays to the same bits as the eager launches."""
+    Bt, S, hidden, heads, ffn = 2, 256, 512, 4, 1408
+    w = si.llama_weights(hidden, ffn, config=5, first_ordinal=21)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 20)
+    for plan in ("seq", "head"):
+        blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4, ffn_blocks=11)
+        ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
+        eager = np_bits(blk.forward().payload.cpu()).copy()
+        graph = blk.capture()
+        blk.out.payload.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(np_bits(blk.out.payload.cpu()), eager)
+        check_status()
+
+
 def test_small_grouped_query_block_every_intermediate():
     """4 query heads on 2 key/value heads: each intermediate relation against the oracle, both decompositions."""
     Bt, S, hidden, heads, kvh, ffn = 2, 256, 512, 4, 2, 1408
