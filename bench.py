@@ -610,7 +610,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--plan", choices=["seq", "head"], default="seq")
+    ap.add_argument("--plan", choices=["seq", "head", "mixed"], default="seq")
     ap.add_argument("--shape", choices=list(SHAPES), default="7b")
     ap.add_argument("--impl", choices=["ja", "reference"], default="ja")
     ap.add_argument("--ref-rows", type=int, default=16)

@@ -13,6 +13,9 @@ blocks x 8 column blocks):
   "head"  head-blocked: x is re-tiled once to 128 x 128 blocks (one head per column block); all projections
           contract over 32 (64) head-sized blocks and emit head-sized blocks, so attention needs no
           relayout; the block output is re-tiled back at the end.
+  "mixed" sequence-blocked activations, but the q / k / v projections EMIT head-sized column blocks (out(J) of a
+          join-agg spec is free to differ from the tiling of its inputs) and the output projection contracts over
+          them: no relayout anywhere inside the block.
 """
 from __future__ import annotations
 
@@ -28,7 +31,7 @@ class LlamaBlock:
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
                  theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8,
                  ffn_blocks: int | None = None, fused: bool = True, n_kv_heads: int | None = None):
-        assert plan in ("seq", "head")
+        assert plan in ("seq", "head", "mixed")
         self.fused = fused
         assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
         assert seq % token_block == 0
@@ -45,7 +48,7 @@ class LlamaBlock:
         io_c = ES(hidden, col_blocks)                    # column tiling of the block's input / output
         head_c = ES(hidden, n_kv)                        # one key/value head's group of query heads per column block
         kvhead_c = ES(kv_hidden, n_kv)                   # one key/value head per column block
-        act_c = io_c if plan == "seq" else head_c        # column tiling of the plan's [T, hidden] activations
+        act_c = head_c if plan == "head" else io_c       # column tiling of the plan's [T, hidden] activations
         # the FFN index is cut into 256-wide blocks when it divides evenly (11008 = 43 x 256, 22016 = 86 x 256): every
         # output tile of the up-projections is then a whole block, with no ragged tail tile per block
         if ffn_blocks is None:
@@ -65,7 +68,7 @@ class LlamaBlock:
         # ---- relations -------------------------------------------------------------------------------
         self.x = Relation([T, hidden], [t_sp, io_c], bf)                 # block input (filled by the caller)
         self.out = Relation([T, hidden], [t_sp, io_c], bf)               # block output
-        self.x_p = self.x if plan == "seq" else act()                    # input in the plan's tiling
+        self.x_p = act() if plan == "head" else self.x                   # input in the plan's tiling
         self.n1, self.h, self.n2, self.o, self.y = act(), act(), act(), act(), act()
         self.q, self.k, self.v = act(qkv_c), kv(), kv()
         self.q_r, self.k_r = act(qkv_c), kv()                            # after RoPE
@@ -74,8 +77,8 @@ class LlamaBlock:
             self.att = act()
         else:
             self.q_h, self.k_h, self.v_h = self.q_r, self.k_r, self.v
-            self.att_h = self.att = act()
-        self.out_p = self.out if plan == "seq" else act()
+            self.att_h = self.att = act(head_c)
+        self.out_p = act() if plan == "head" else self.out
         self.a = Relation([T, ffn], [t_sp, ffn_c], bf)
         self.b = Relation([T, ffn], [t_sp, ffn_c], bf)
         self.hh = Relation([T, ffn], [t_sp, ffn_c], bf)
@@ -83,7 +86,7 @@ class LlamaBlock:
         w = {n: weights[n].to("cuda", bf) for n in weights}
         self.wq = from_dense(w["wq"], [act_c, qkv_c])
         self.wk, self.wv = (from_dense(w[n], [act_c, kv_c]) for n in ("wk", "wv"))
-        self.wo = from_dense(w["wo"], [act_c if plan == "seq" else head_c, act_c])
+        self.wo = from_dense(w["wo"], [io_c if plan == "seq" else head_c, act_c])
         self.w1, self.w3 = from_dense(w["w1"], [act_c, ffn_c]), from_dense(w["w3"], [act_c, ffn_c])
         self.w2 = from_dense(w["w2"], [ffn_c, act_c])
         self.g1, self.g2 = from_dense(w["g1"], [act_c]), from_dense(w["g2"], [act_c])
@@ -118,19 +121,19 @@ class LlamaBlock:
         else:   # query heads inherit their split from the key/value heads: intervals of n_heads / n_kv heads
             self.s_attn = Spec("bqhd,bkgd,bkgd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_kv), "d": [0, D], "k": s_sp,
                                                          "g": ES(n_kv, n_kv)}, "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
-        self.s_wo = mm(act_c if plan == "seq" else head_c, act_c)
+        self.s_wo = mm(io_c if plan == "seq" else head_c, act_c)
         self.s_add = Spec("ij,ij->ij", {"i": t_sp, "j": act_c}, "add", (), "none")
         self.s_up = mm(act_c, ffn_c)
         self.s_silu = Spec("ij,ij->ij", {"i": t_sp, "j": ffn_c}, "silu_mul", (), "none")
         self.s_down = mm(ffn_c, act_c)
-        self.n_relayouts = 4 if plan == "seq" else 2
+        self.n_relayouts = {"seq": 4, "head": 2, "mixed": 0}[plan]
         # fused chains: the projection's accumulator goes through RoPE / the residual ADD / SILU_MUL before its store
         # (a fused form that the tiling cannot run -- JA_ERR_UNSUPPORTED -- falls back to its chain, once and for all)
         self.fuse_rope = self.fuse_add = self.fuse_swiglu = fused
         if fused:
             self.s_qk_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": qkv_c}, "matmul_rope", (theta, seq, D), "sum")
             self.s_k_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": kv_c}, "matmul_rope", (theta, seq, D), "sum")
-            self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": act_c, "k": act_c}, "matmul_add", (), "sum")
+            self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": io_c if plan == "seq" else head_c, "k": act_c}, "matmul_add", (), "sum")
             self.s_up_swiglu = Spec("ij,jk,jk->ik", {"i": t_sp, "j": act_c, "k": ffn_c}, "swiglu_up", (), "sum")
             self.s_down_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": ffn_c, "k": act_c}, "matmul_add", (), "sum")
 

@@ -144,7 +144,7 @@ def _block_case(shape_name, Bt, S, hidden, heads, ffn, prefix, seq_id):
     w = si.llama_weights(hidden, ffn)
     x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 0)
     outs = {}
-    for plan, fused in (("seq", True), ("head", True), ("seq", False)):
+    for plan, fused in (("seq", True), ("head", True), ("seq", False), ("mixed", True)):
         blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, fused=fused)
         ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
         outs[plan if fused else "seq_unfused"] = download(blk.forward())
@@ -154,12 +154,13 @@ def _block_case(shape_name, Bt, S, hidden, heads, ffn, prefix, seq_id):
         torch.cuda.empty_cache()
     # the two decompositions of the same block agree with each other on the whole output, fused chains or not ...
     assert relfro(outs["head"], outs["seq"]) <= TOL[BF]
+    assert relfro(outs["mixed"], outs["seq"]) <= TOL[BF]
     assert relfro(outs["seq_unfused"], outs["seq"]) <= TOL[BF]
     # ... and with the oracle on sampled token rows of one sequence (causal: a prefix is self-contained)
     rows = np.unique(np.concatenate([[0, 1, 127, 128, prefix - 1], np.linspace(0, prefix - 1, 8).astype(int)]))
     xs = si.to_f64(x[seq_id * S: seq_id * S + prefix])
     ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows)["out"]
-    for plan in ("seq", "head", "seq_unfused"):
+    for plan in ("seq", "head", "seq_unfused", "mixed"):
         assert relfro(outs[plan][seq_id * S + rows], ref) <= TOL[BF], (shape_name, plan)
 
 
@@ -180,7 +181,8 @@ def test_small_block_every_intermediate():
     w64 = {k: si.to_f64(v) for k, v in w.items()}
     refs = [operators.llama_block(si.to_f64(x[b * S:(b + 1) * S]), w64, heads) for b in range(Bt)]
     cat = lambda name: np.concatenate([r[name].reshape(S, -1) for r in refs])
-    for plan, fused, ffn_blocks in (("seq", False, 4), ("head", False, 4), ("seq", True, 11), ("head", True, 11), ("seq", True, 4)):
+    for plan, fused, ffn_blocks in (("seq", False, 4), ("head", False, 4), ("seq", True, 11), ("head", True, 11), ("seq", True, 4),
+                                    ("mixed", True, 11), ("mixed", False, 4)):
         blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4, ffn_blocks=ffn_blocks, fused=fused)
         ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
         out = download(blk.forward())
@@ -223,7 +225,7 @@ def test_small_grouped_query_block_every_intermediate():
     w64 = {k: si.to_f64(v) for k, v in w.items()}
     refs = [operators.llama_block(si.to_f64(x[b * S:(b + 1) * S]), w64, heads, n_kv_heads=kvh) for b in range(Bt)]
     cat = lambda name: np.concatenate([r[name].reshape(S, -1) for r in refs])
-    for plan, fused in (("seq", False), ("head", False), ("seq", True), ("head", True)):
+    for plan, fused in (("seq", False), ("head", False), ("seq", True), ("head", True), ("mixed", True)):
         blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan=plan, col_blocks=4, ffn_blocks=11, fused=fused, n_kv_heads=kvh)
         ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
         out = download(blk.forward())
