@@ -13,9 +13,10 @@ blocks x 8 column blocks):
   "head"  head-blocked: x is re-tiled once to 128 x 128 blocks (one head per column block); all projections
           contract over 32 (64) head-sized blocks and emit head-sized blocks, so attention needs no
           relayout; the block output is re-tiled back at the end.
-  "mixed" sequence-blocked activations, but the q / k / v projections EMIT head-sized column blocks (out(J) of a
-          join-agg spec is free to differ from the tiling of its inputs) and the output projection contracts over
-          them: no relayout anywhere inside the block.
+  "mixed" sequence-blocked everywhere, attention included: its spec cuts the head index into as many intervals as the
+          activations have column blocks (several heads per block), so q, k, v are consumed in the tiling their
+          projections emit and the attention output in the tiling the output projection contracts over: no relayout
+          anywhere inside the block.
 """
 from __future__ import annotations
 
@@ -55,9 +56,13 @@ class LlamaBlock:
             ffn_blocks = ffn // 256 if ffn % 256 == 0 else col_blocks
         ffn_c = ES(ffn, ffn_blocks)
         self.t_sp, self.io_c, self.head_c, self.act_c, self.ffn_c = t_sp, io_c, head_c, act_c, ffn_c
-        qkv_c = io_c if plan == "seq" else head_c        # tiling q is produced in
-        # tiling k, v are produced in: column blocks hold whole heads, so the narrower key/value relations may get fewer blocks
-        kv_c = ES(kv_hidden, min(col_blocks, n_kv)) if plan == "seq" else kvhead_c
+        # tilings q and k, v are produced in: column blocks hold whole heads, so the narrower key/value relations may get
+        # fewer blocks; plan "mixed" feeds them to attention as they are, so there q is cut like k, v (grouped heads)
+        n_kvb = min(col_blocks, n_kv)
+        qkv_c = {"seq": io_c, "head": head_c, "mixed": ES(hidden, n_kvb)}[plan]
+        kv_c = kvhead_c if plan == "head" else ES(kv_hidden, n_kvb)
+        att_c = head_c if plan != "mixed" else qkv_c     # tiling attention reads q from and writes its output in
+        kvatt_c = kvhead_c if plan != "mixed" else kv_c
 
         def act(cols=act_c):
             return Relation([T, hidden], [t_sp, cols], bf)
@@ -77,7 +82,7 @@ class LlamaBlock:
             self.att = act()
         else:
             self.q_h, self.k_h, self.v_h = self.q_r, self.k_r, self.v
-            self.att_h = self.att = act(head_c)
+            self.att_h = self.att = act(att_c)
         self.out_p = act() if plan == "head" else self.out
         self.a = Relation([T, ffn], [t_sp, ffn_c], bf)
         self.b = Relation([T, ffn], [t_sp, ffn_c], bf)
@@ -86,7 +91,7 @@ class LlamaBlock:
         w = {n: weights[n].to("cuda", bf) for n in weights}
         self.wq = from_dense(w["wq"], [act_c, qkv_c])
         self.wk, self.wv = (from_dense(w[n], [act_c, kv_c]) for n in ("wk", "wv"))
-        self.wo = from_dense(w["wo"], [io_c if plan == "seq" else head_c, act_c])
+        self.wo = from_dense(w["wo"], [io_c if plan == "seq" else att_c, act_c])
         self.w1, self.w3 = from_dense(w["w1"], [act_c, ffn_c]), from_dense(w["w3"], [act_c, ffn_c])
         self.w2 = from_dense(w["w2"], [ffn_c, act_c])
         self.g1, self.g2 = from_dense(w["g1"], [act_c]), from_dense(w["g2"], [act_c])
@@ -101,8 +106,8 @@ class LlamaBlock:
 
         self.q4, self.k4 = v4(self.q, qkv_c), v4(self.k, kv_c, n_kv)
         self.q4r, self.k4r = v4(self.q_r, qkv_c), v4(self.k_r, kv_c, n_kv)
-        self.qa, self.oa = v4(self.q_h, head_c), v4(self.att_h, head_c)
-        self.ka, self.va = v4(self.k_h, kvhead_c, n_kv), v4(self.v_h, kvhead_c, n_kv)
+        self.qa, self.oa = v4(self.q_h, att_c), v4(self.att_h, att_c)
+        self.ka, self.va = v4(self.k_h, kvatt_c, n_kv), v4(self.v_h, kvatt_c, n_kv)
 
         # ---- specs -------------------------------------------------------------------------------------
         def mm(jc, kc):
@@ -115,13 +120,14 @@ class LlamaBlock:
                            (theta,), "none")
         self.s_rope_k = Spec("bshd->bshd", {"b": b_sp, "s": s_sp, "h": ES(n_kv, len(kv_c) - 1), "d": [0, D]}, "rope",
                              (theta,), "none")
+        n_hb = len(att_c) - 1                             # intervals of the head index in the attention spec
         if n_kv == n_heads:
-            self.s_attn = Spec("bqhd,bkhd,bkhd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_heads), "d": [0, D], "k": s_sp},
+            self.s_attn = Spec("bqhd,bkhd,bkhd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_hb), "d": [0, D], "k": s_sp},
                                "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
-        else:   # query heads inherit their split from the key/value heads: intervals of n_heads / n_kv heads
-            self.s_attn = Spec("bqhd,bkgd,bkgd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_kv), "d": [0, D], "k": s_sp,
-                                                         "g": ES(n_kv, n_kv)}, "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
-        self.s_wo = mm(io_c if plan == "seq" else head_c, act_c)
+        else:   # query heads inherit their split from the key/value heads: intervals of n_heads / n_kv heads per key/value head
+            self.s_attn = Spec("bqhd,bkgd,bkgd->bqhd", {"b": b_sp, "q": s_sp, "h": ES(n_heads, n_hb), "d": [0, D], "k": s_sp,
+                                                         "g": ES(n_kv, n_hb)}, "attention", (1.0 / math.sqrt(D), 1.0), "online_softmax")
+        self.s_wo = mm(io_c if plan == "seq" else att_c, act_c)
         self.s_add = Spec("ij,ij->ij", {"i": t_sp, "j": act_c}, "add", (), "none")
         self.s_up = mm(act_c, ffn_c)
         self.s_silu = Spec("ij,ij->ij", {"i": t_sp, "j": ffn_c}, "silu_mul", (), "none")
@@ -133,7 +139,7 @@ class LlamaBlock:
         if fused:
             self.s_qk_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": qkv_c}, "matmul_rope", (theta, seq, D), "sum")
             self.s_k_rope = Spec("ij,jk->ik", {"i": t_sp, "j": act_c, "k": kv_c}, "matmul_rope", (theta, seq, D), "sum")
-            self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": io_c if plan == "seq" else head_c, "k": act_c}, "matmul_add", (), "sum")
+            self.s_wo_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": io_c if plan == "seq" else att_c, "k": act_c}, "matmul_add", (), "sum")
             self.s_up_swiglu = Spec("ij,jk,jk->ik", {"i": t_sp, "j": act_c, "k": ffn_c}, "swiglu_up", (), "sum")
             self.s_down_add = Spec("ij,jk,ik->ik", {"i": t_sp, "j": ffn_c, "k": act_c}, "matmul_add", (), "sum")
 
