@@ -25,7 +25,7 @@ sys.path.insert(0, ROOT)
 
 SHAPES = {"7b": dict(batch=8, seq=2048, hidden=4096, heads=32, ffn=11008),
           "65b": dict(batch=1, seq=4096, hidden=8192, heads=64, ffn=22016),
-          # the paper's own block (Section 7): grouped-query attention, 32 query heads on 8 key/value heads, FFN 14336
+          # the paper's own block (Section 6): grouped-query attention, 32 query heads on 8 key/value heads, FFN 14336
           "paper_b8_1k": dict(batch=8, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336),
           "paper_1x8k": dict(batch=1, seq=8192, hidden=4096, heads=32, kv_heads=8, ffn=14336),
           "paper_b128_1k": dict(batch=128, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336)}
@@ -562,7 +562,7 @@ def run_case(args):
                                               "TFLOPs": 6.0 * T * d * f / (t["ms_mean"] * 1e-3) / 1e12, "plan": plan}
             res["p%d_optimizer_host_ms" % p_] = {"ms_mean": opt_ms, "ms_min": opt_ms, "ms_median": opt_ms, "cost": best_cost}
     elif args.case == "chains":
-        # Section 7, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
+        # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
         # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)
         def right(lo, hi):   # M_lo (M_lo+1 (... M_hi))
             return lo if lo == hi else (lo, right(lo + 1, hi))

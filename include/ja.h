@@ -214,7 +214,7 @@ ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_t agg, ja_r
  *   total_cost  out (may be NULL): the minimum of the summed Cost
  * ja_plan_cost evaluates the summed Cost of a given assignment (same layout of `counts`).
  * Errors: JA_ERR_PARSE, JA_ERR_SHAPE (operand / producer mismatch), JA_ERR_INVALID_ARG (not a tree in topological
- * order), JA_ERR_UNSUPPORTED (a node consumed twice: cut the graph first, Section 4.4; more than 8 letters),
+ * order), JA_ERR_UNSUPPORTED (a node consumed twice: ja_plan_optimize_graph handles that, Section 4.5; more than 8 letters),
  * JA_ERR_TILING (no decomposition into p function specs). */
 #define JA_PLAN_MAX_LETTERS 8
 typedef struct {
@@ -225,7 +225,7 @@ typedef struct {
 } ja_plan_node_t;
 ja_status_t ja_plan_optimize(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
 ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost);
-/* Outputs with several consumers (Section 4.4): the graph (nodes in topological order; a node may be consumed any number
+/* Outputs with several consumers (Section 4.5): the graph (nodes in topological order; a node may be consumed any number
  * of times) is cut at every edge out of a multiply consumed tensor; the resulting trees are optimised with Algorithm 1
  * one at a time, largest first (ties: smaller root first), each subject to the specs already fixed: an operand produced
  * in an already-optimised tree enters like an input of the computation whose tiling is fixed (Cost charges the repartition

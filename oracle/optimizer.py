@@ -135,7 +135,7 @@ def exhaustive(ops, p: int):
 
 
 # ---------------------------------------------------------------------------------------------------
-# Outputs with several consumers (Section 4.4): the graph is cut at every edge out of a multiply
+# Outputs with several consumers (Section 4.5): the graph is cut at every edge out of a multiply
 # consumed tensor and the resulting trees are optimised one at a time, largest first, each subject
 # to the specs already fixed.
 # ---------------------------------------------------------------------------------------------------
@@ -163,7 +163,7 @@ def cut_into_trees(ops):
 
 
 def optimize_graph(ops, p: int):
-    """Section 4.4.  An operand produced in a tree that is already optimised enters like an input whose tiling
+    """Section 4.5.  An operand produced in a tree that is already optimised enters like an input whose tiling
     is fixed (Cost charges the repartition when in_k(J) differs from it); an operand produced in a tree not
     yet optimised enters like an input of the computation.  When the root of a tree feeds consumers whose
     specs are already fixed, the root's tiling is chosen with their repartition charges added (the paper only

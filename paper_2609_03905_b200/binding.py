@@ -250,7 +250,7 @@ def ja_plan_optimize(ops, p: int):
 
 
 def ja_plan_optimize_graph(ops, p: int):
-    """Section 4.4: a graph with multiply consumed tensors, cut into trees and optimised tree by tree."""
+    """Section 4.5: a graph with multiply consumed tensors, cut into trees and optimised tree by tree."""
     arr, keep = _plan_nodes(ops)
     counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
     total = ctypes.c_int64()

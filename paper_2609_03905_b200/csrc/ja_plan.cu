@@ -135,7 +135,7 @@ ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, bool allow_s
                 if (pr.extent[pos(pr.letters, pr.out[d])] != op.extent[pos(op.letters, op.ins[k][d])])
                     return ja_fail(JA_ERR_SHAPE, "node %d operand %zu: extent %zu differs from its producer's output", i, k, d);
             if (++(*consumers)[q] > 1 && !allow_sharing)
-                return ja_fail(JA_ERR_UNSUPPORTED, "node %d is consumed twice: use ja_plan_optimize_graph, which cuts the graph into trees (Section 4.4)", q);
+                return ja_fail(JA_ERR_UNSUPPORTED, "node %d is consumed twice: use ja_plan_optimize_graph, which cuts the graph into trees (Section 4.5)", q);
         }
     }
     if (!allow_sharing)

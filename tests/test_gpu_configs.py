@@ -198,7 +198,7 @@ def test_small_block_every_intermediate():
 
 
 # ---------------------------------------------------------------------------------------------------
-# the paper's own workloads (Section 7): the grouped-query block and the matrix chains
+# the paper's own workloads (Section 6): the grouped-query block and the matrix chains
 # ---------------------------------------------------------------------------------------------------
 def test_block_replayed_from_a_cuda_graph():
     """The chain captured into one CUDA graph replays to the same bits as the eager launches."""
@@ -236,7 +236,7 @@ def test_small_grouped_query_block_every_intermediate():
 
 
 def test_paper_block_shape_grouped_query_sampled():
-    """Hidden 4096, 32 query heads on 8 key/value heads of 128, FFN 14336 (Section 7), eight sequences of 1K tokens;
+    """Hidden 4096, 32 query heads on 8 key/value heads of 128, FFN 14336 (Section 6), eight sequences of 1K tokens;
     sampled token rows of one sequence against the oracle."""
     Bt, S, hidden, heads, kvh, ffn = 8, 1024, 4096, 32, 8, 14336
     w = si.llama_weights(hidden, ffn, config=5, first_ordinal=61, kv_hidden=kvh * 128)
@@ -260,7 +260,7 @@ def _chain_eval(dims, tree, mats, mm):
     return mm(_chain_eval(dims, tree[0], mats, mm), _chain_eval(dims, tree[1], mats, mm))
 
 
-CHAINS = {   # Section 7: fixed parenthesizations; dimensions divided by `div` keep the structure at oracle-sized cost
+CHAINS = {   # Section 6: fixed parenthesizations; dimensions divided by `div` keep the structure at oracle-sized cost
     "A": ([10240] + [16384, 6144] * 4 + [10240], ((0, 1), (((2, 3), ((4, 5), (6, 7))), 8))),
     "B": ([9216, 20480, 5120, 20480, 5120, 9216], ((0, 1), ((2, 3), 4))),
     "C": ([10240, 12288, 32768, 2048], (0, (1, 2))),

@@ -288,7 +288,7 @@ def test_logical_optimizer_matches_oracle(golden_dir):
 
 
 def test_logical_optimizer_on_graphs_with_shared_tensors():
-    """Section 4.4 through the library against the oracle: same trees, same order, same assembled cost."""
+    """Section 4.5 through the library against the oracle: same trees, same order, same assembled cost."""
     from oracle import optimizer
     from test_oracle_pins import _block_graph
     for dims, p in (((16, 8, 12), 2), ((16, 8, 12), 4), ((64, 32, 48), 8)):
