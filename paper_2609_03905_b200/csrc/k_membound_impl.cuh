@@ -8,6 +8,8 @@
 //    output key (Definition 3.7); the partial never leaves registers.
 //
 // All loads/stores are 128-bit when the tiling allows (every split of j a multiple of the vector width).
+#pragma once
+
 #include <stdlib.h>
 #include <string.h>
 
@@ -547,27 +549,9 @@ ja_status_t launch_row_op(RowOp op, const RowArgs& a, int vec, int64_t n_rows, i
     return ja_fail(JA_ERR_INVALID_ARG, "unknown row op");
 }
 
-}  // namespace
-
-ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,
-                           cudaStream_t st) {
-    // payload sizes are multiples of 128 bytes, so whole 16-byte vectors cover them exactly
-    const int64_t n_vec = n_elems * (dt == JA_F32 ? 4 : 2) / 16;
-    int64_t want = (n_vec + 255) / 256;
-    unsigned grid = (unsigned)(want < (int64_t)148 * 32 ? (want > 0 ? want : 1) : (int64_t)148 * 32);
-    if (dt == JA_BF16) {
-        if (fn == JA_FN_ADD) flat_bf16_kernel<JA_FN_ADD><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
-        else flat_bf16_kernel<JA_FN_SILU_MUL><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
-    } else {
-        if (fn == JA_FN_ADD) flat_f32_kernel<JA_FN_ADD><<<grid, 256, 0, st>>>((const float4*)a, (const float4*)b, (float4*)out, n_vec);
-        else flat_f32_kernel<JA_FN_SILU_MUL><<<grid, 256, 0, st>>>((const float4*)a, (const float4*)b, (float4*)out, n_vec);
-    }
-    ja_count_launch();
-    JA_CUDA(cudaGetLastError());
-    return JA_OK;
-}
-
-ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st) {
+template <typename T>
+ja_status_t launch_row_typed(RowOp op, const RowArgs& a, cudaStream_t st) {
+    const ja_dtype_t dt = sizeof(T) == 4 ? JA_F32 : JA_BF16;
     const int last = a.x.rank - 1;
     const int64_t n = a.x.extent[last];
     int64_t n_rows = 1;
@@ -575,12 +559,6 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
     if (n_rows >= (1ll << 31) || n >= (1ll << 31)) return ja_fail(JA_ERR_UNSUPPORTED, "row-structured join-agg: extents must be < 2^31");
     const int full = dt == JA_F32 ? 4 : 8;
     const int es = dt == JA_F32 ? 4 : 2;
-    // ---- uniform tilings: bulk-copy pipeline through shared memory ---------------------------------------------
-    {
-        bool launched = false;
-        ja_status_t s = ja_launch_row_tma(op, a, dt, st, &launched);
-        if (s != JA_OK || launched) return s;
-    }
     // ---- fast path: every block of x (and of g, and of the statistics relations) has the same shape --------
     const bool has_g = (op == ROW_RMS_SCALE || op == ROW_RMSNORM);
     const bool has_stat = (op == ROW_SUMSQ || op == ROW_MAX || op == ROW_EXPSUM || op == ROW_RMS_SCALE || op == ROW_EXP_SUB_DIV);
@@ -597,7 +575,7 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
         g.stat_blk_bytes = has_stat ? (int)a.s0.blk_stride : 0;
         g.g_blk_bytes = has_g ? (int)a.g.blk_stride : 0;
         g.rope_d = a.rope_d > 0 ? a.rope_d : 2;
-        bool ok = dt == JA_F32 ? launch_fast_op<float>(op, a, g, n_rows, st) : launch_fast_op<__nv_bfloat16>(op, a, g, n_rows, st);
+        bool ok = launch_fast_op<T>(op, a, g, n_rows, st);
         if (ok) {
             ja_count_launch();
             JA_CUDA(cudaGetLastError());
@@ -608,6 +586,7 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
     int vec = 1;
     if (a.x.bs[last] != 0 && a.x.bs[last] % full == 0 && n % full == 0) vec = full;
     else if (op == ROW_ROPE) vec = 2;
-    return dt == JA_F32 ? launch_row_op<float>(op, a, vec, n_rows, n, st)
-                        : launch_row_op<__nv_bfloat16>(op, a, vec, n_rows, n, st);
+    return launch_row_op<T>(op, a, vec, n_rows, n, st);
 }
+
+}  // namespace

@@ -17,6 +17,8 @@
 //               stores of the stage and frees it once the copies have read shared memory.
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT, waits (bounded) for its loads in flight
 // and leaves through the normal exit.
+#pragma once
+
 #include <stdlib.h>
 #include <string.h>
 
@@ -514,7 +516,6 @@ ja_status_t launch_op(const RowMaps& tm, const RowArgs& a, const RowTmaGeom& g, 
     if (vpl <= 4) return launch_v<T, OP, 4>(tm, a, g, g_bytes, sms, status, st, launched);
     if (vpl <= 8) return launch_v<T, OP, 8>(tm, a, g, g_bytes, sms, status, st, launched);
     if (vpl <= 16) return launch_v<T, OP, 16>(tm, a, g, g_bytes, sms, status, st, launched);
-    if (vpl <= 32 && OP != ROW_SOFTMAX) return launch_v<T, OP, (OP != ROW_SOFTMAX ? 32 : 16)>(tm, a, g, g_bytes, sms, status, st, launched);
     *launched = false;
     return JA_OK;
 }
@@ -552,12 +553,12 @@ ja_status_t encode_rows4(const RelView& v, const RowTmaGeom& g, int64_t n_lead, 
     return JA_OK;
 }
 
-}  // namespace
-
 // Sets *launched when this form took the job; leaves it false (and launches nothing) when the shape does not fit:
-// blocks of different shapes, rows longer than 32 vectors per lane, column blocks that are not whole 16-byte vectors,
+// blocks of different shapes, rows longer than 16 vectors per lane of a warp team, column blocks that are not whole 16-byte vectors,
 // more than 256 column blocks, RoPE (its rotation needs the row's coordinates).
-ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched) {
+template <typename T>
+ja_status_t row_tma_launch(RowOp op, const RowArgs& a, cudaStream_t st, bool* launched) {
+    const ja_dtype_t dt = sizeof(T) == 4 ? JA_F32 : JA_BF16;
     *launched = false;
     if (op == ROW_ROPE) return JA_OK;
     const char* off_env = getenv("JA_ROW_TMA");
@@ -600,7 +601,7 @@ ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStr
     g.wpr = 1;
     while (g.wpr < CONSUMER_WARPS && R * g.wpr < CONSUMER_WARPS && n > (int64_t)g.wpr * vec * 32) g.wpr *= 2;
     const int vpl = (int)((n + (int64_t)vec * 32 * g.wpr - 1) / ((int64_t)vec * 32 * g.wpr));
-    if (vpl > 32 || (vpl > 16 && op == ROW_SOFTMAX)) return JA_OK;
+    if (vpl > 16) return JA_OK;
     g.chunks_per_blk = (int)((rows_per_blk + R - 1) / R);
     g.n_units = n_lead * g.chunks_per_blk;
     g.seg_bytes = R * g.bw * es;
@@ -623,10 +624,11 @@ ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStr
         cudaGetDevice(&dev);
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
     }
-    s = dt == JA_F32 ? launch_t<float>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched)
-                     : launch_t<__nv_bfloat16>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched);
+    s = launch_t<T>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched);
     if (s != JA_OK || !*launched) return s;
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
     return JA_OK;
 }
+
+}  // namespace
