@@ -28,7 +28,9 @@ SHAPES = {"7b": dict(batch=8, seq=2048, hidden=4096, heads=32, ffn=11008),
           # the paper's own block (Section 6): grouped-query attention, 32 query heads on 8 key/value heads, FFN 14336
           "paper_b8_1k": dict(batch=8, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336),
           "paper_1x8k": dict(batch=1, seq=8192, hidden=4096, heads=32, kv_heads=8, ffn=14336),
-          "paper_b128_1k": dict(batch=128, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336)}
+          "paper_b128_1k": dict(batch=128, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336),
+          "paper_1x1k": dict(batch=1, seq=1024, hidden=4096, heads=32, kv_heads=8, ffn=14336),
+          "paper_1x128k": dict(batch=1, seq=131072, hidden=4096, heads=32, kv_heads=8, ffn=14336)}
 METRIC = "join-agg TFLOP/s, LLaMA-block forward on 1 B200"
 
 
