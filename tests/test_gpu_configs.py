@@ -253,6 +253,35 @@ def test_paper_block_shape_grouped_query_sampled():
     assert relfro(out[seq_id * S + rows], ref) <= TOL[BF]
 
 
+def test_join_only_and_aggregating_relayout_full_size():
+    """The down projection of the 7B block executed through its join (m = 4 unaggregated copies per output block) and
+    aggregated into the consumer's tiling, at full size; sampled rows against the oracle."""
+    T, f, d, m = 16384, 11008, 4096, 4
+    h = si.normal((T, f), 0.0, 1.0, BF, 2, 51)
+    W2 = si.normal((f, d), 0.0, 0.02, BF, 2, 52)
+    ti, tf, td = ES(T, 16), ES(f, m), ES(d, 8)
+    rh, rW = upload(h, [ti, tf]), upload(W2, [tf, td])
+    rP = ja.partial_relation(m, [T, d], [ti, td], BF)
+    spec = ja.Spec("ij,jk->ik", {"i": ti, "j": tf, "k": td})
+    spec.execute_join([rh, rW], rP)
+    dst_sp = [ES(T, 128), ES(d, 8)]
+    rY = empty_like_tiling([T, d], dst_sp, BF, fill=float("nan"))
+    ja.repartition_agg(rP, "sum", rY)
+    P, Y = download(rP), download(rY)
+    check_status()
+    assert not np.isnan(Y).any()
+    rows = np.array([0, 1, 127, 128, 1023, 1024, 5000, 9999, 16383])
+    h64, W64 = si.to_f64(h[rows]), si.to_f64(W2)
+    for c in range(m):
+        j0, j1 = tf[c], tf[c + 1]
+        ref = core.round_to(h64[:, j0:j1] @ W64[j0:j1], "bf16")
+        assert relfro(P[c][rows], ref) <= TOL[BF], c
+    # the aggregate of the library's own copies, in the oracle's arithmetic (fp64 sum in ascending copy order, one rounding)
+    want = core.round_to(((P[0][rows] + P[1][rows]) + P[2][rows]) + P[3][rows], "bf16")
+    assert np.mean(Y[rows] != want) < 2e-3 and relfro(Y[rows], want) <= 1e-3
+    assert relfro(Y[rows], core.round_to(h64 @ W64, "bf16")) <= TOL[BF]
+
+
 def _chain_eval(dims, tree, mats, mm):
     """tree: nested pairs of matrix indices, e.g. (0, (1, 2)); mm(A, B) multiplies two operands."""
     if isinstance(tree, int):
