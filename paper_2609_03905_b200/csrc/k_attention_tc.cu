@@ -118,6 +118,37 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same three, executed by a whole converged warp with one lane (pred != 0) issuing: every operand is then warp-uniform, which
+// lets the compiler keep descriptors and addresses in uniform registers instead of moving them there before every instruction.
+__device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate, uint32_t pred) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate, uint32_t pred) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void commit1_w(uint32_t bar, uint32_t pred) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar), "r"(pred) : "memory");
+}
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.b32 %0, 1, 0, q;\n\t}" : "=r"(pred));
+    return pred;
+}
 __device__ __forceinline__ void commit1(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -459,6 +490,49 @@ __device__ __forceinline__ float row_exp_store128(const uint32_t (&v)[128], int 
     return (a0 + a1) + (b0 + b1);
 }
 
+// One half (64 keys) of P = 2^(S*scale - m) written as packed bf16 over S; returns the half's row sum. HALF 0 also returns the
+// maximum of all 128 raw scores, computed alongside (two max3 per pair of exponentials).
+template <int HALF>
+__device__ __forceinline__ float row_exp_store_half(const uint32_t (&v)[128], float scale, float m_used, uint32_t t_dst, float& mx_out) {
+    const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
+    uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
+    float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]), m2 = __uint_as_float(v[2]), m3 = __uint_as_float(v[3]);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+            const int col = HALF * 64 + c * 16 + i;
+            float p0, p1;
+            unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
+            if (HALF == 0) {   // pair number q = (c*16+i)/2 in 0..31 covers scores 4q .. 4q+3 (scores 0..3 seed the four maxima)
+                const int q4 = (c * 16 + i) * 2;
+                if (q4 >= 4) {
+                    if (i & 2) {
+                        m2 = max3(m2, __uint_as_float(v[q4]), __uint_as_float(v[q4 + 1]));
+                        m3 = max3(m3, __uint_as_float(v[q4 + 2]), __uint_as_float(v[q4 + 3]));
+                    } else {
+                        m0 = max3(m0, __uint_as_float(v[q4]), __uint_as_float(v[q4 + 1]));
+                        m1 = max3(m1, __uint_as_float(v[q4 + 2]), __uint_as_float(v[q4 + 3]));
+                    }
+                }
+            }
+            if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
+            else sum_b = add2(sum_b, pack2(p0, p1));
+            __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
+            pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
+        }
+        tmem_st8(t_dst + HALF * 32 + c * 8, pk);
+    }
+    if (HALF == 0) mx_out = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    float a0, a1, b0, b1;
+    unpack2(sum_a, a0, a1);
+    unpack2(sum_b, b0, b1);
+    return (a0 + a1) + (b0 + b1);
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Two query tiles per CTA. The CTA owns 256 query rows of one (batch, head) as two independent 128-row output
 // key tiles A and B that share every K_j / V_j tile it loads. While the row threads of one tile exponentiate,
@@ -467,10 +541,18 @@ __device__ __forceinline__ float row_exp_store128(const uint32_t (&v)[128], int 
 //   O~ is ACCUMULATED IN TENSOR MEMORY by the P V products (accumulate flag), not in registers. The running
 //   maximum used as the exponent offset is only raised when a row's new maximum exceeds it by more than 2^8
 //   (P stays <= 256, exact in the final O~/l); only then is the row's O~ rescaled in TMEM by its row thread.
-//   warp 0 TMA, warp 1 MMA issuer, warps 2..5 rows of A, warps 6..9 rows of B.
+//   Past the first key tile the row threads exponentiate against the offset in use WHILE they reduce the tile's
+//   maximum (the max3 instructions run in the shadow of the ex2 pipe) and hand the first 64 keys of P to the tensor
+//   pipe before they start on the other 64; a warp in which some row outgrew its offset redoes the tile.
+//   warp 0 TMA (K / V tiles through one ring of five slots), warp 1 MMA issuer, warps 2..5 rows of A, 6..9 rows of B.
+//   The MMA warp runs its loop converged, one elected lane issuing: addresses and descriptors are then warp-uniform
+//   values, and the steady state is straight-line code (measured on this part: a branch between two tcgen05.mma
+//   instructions, or operands that have to be moved to uniform registers first, cost the issuing thread ~40 cycles
+//   per instruction, against 64 cycles of tensor-pipe time for M128 N128 K16).
 // ---------------------------------------------------------------------------------------------------------
 constexpr int NUM_THREADS2 = 320;
-constexpr int SMEM_BYTES2 = 6 * TILE_BYTES + 1024 + 256;   // Q_A, Q_B, K x2, V x2
+constexpr int KV_RING = 5;                                  // K / V tiles in shared memory: two in use, three in flight
+constexpr int SMEM_BYTES2 = (2 + KV_RING) * TILE_BYTES + 1024 + 256;   // Q_A, Q_B, ring of K / V tiles
 
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -479,15 +561,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t sQ = base, sK = base + 2 * TILE_BYTES, sV = base + 4 * TILE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * TILE_BYTES);
+    const uint32_t sQ = base, sKV = base + 2 * TILE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + KV_RING) * TILE_BYTES);
     const uint32_t bar0 = smem_u32(bars);
-    enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, P_FULL = 11, O_FULL = 13, NBAR = 15 };
+    // K / V tiles go through one ring in the order K_0 V_0 K_1 V_1 ...: tile number 2j is K_j, 2j+1 is V_j
+    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + KV_RING, S_FULL = 1 + 2 * KV_RING, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4, P_HALF = S_FULL + 6, NBAR = S_FULL + 8 };
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;   // warp-uniform by construction
     const int n_pairs = p.S / (2 * QT);
     int slot, bh;
     ja_attn_decode_cta((int)blockIdx.x, n_pairs, p.H * p.B, p.sect, &slot, &bh);
@@ -500,7 +583,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2) ? 4 : 1);
+        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), ((i >= P_FULL && i < P_FULL + 2) || (i >= P_HALF && i < P_HALF + 2)) ? 4 : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -511,7 +594,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -523,72 +606,100 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 for (int half = 0; half < 2; ++half)
                     tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow_t);
             }
-            bool ok = true;
-            for (int j = 0; j < n_steps_b && ok; ++j) {
-                const int st = j & 1;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1;
-                const int krow = seq_row(p.k, p.S, b, s0 + j * KT, hk);
-                if (!mbar_wait(bar(K_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                mbar_expect_tx(bar(K_FULL + st), TILE_BYTES);
+            int sl = 0;
+            uint32_t ph = 0;
+            for (int li = 0; li < 2 * n_steps_b; ++li) {
+                const int krow = seq_row(p.k, p.S, b, s0 + (li >> 1) * KT, hk);
+                if (!mbar_wait(bar(KV_EMPTY + sl), ph ^ 1, abort_flag, p.status)) break;
+                mbar_expect_tx(bar(KV_FULL + sl), TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sK + st * TILE_BYTES + half * HALF_BYTES, &tmK, bar(K_FULL + st), half * 64, hk % p.k.hblk, krow);
-                if (!mbar_wait(bar(V_EMPTY + st), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                mbar_expect_tx(bar(V_FULL + st), TILE_BYTES);
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sV + st * TILE_BYTES + half * HALF_BYTES, &tmV, bar(V_FULL + st), half * 64, hk % p.k.hblk, krow);
+                    tma_load_3d(sKV + sl * TILE_BYTES + half * HALF_BYTES, (li & 1) ? &tmV : &tmK, bar(KV_FULL + sl), half * 64, hk % p.k.hblk, krow);
+                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
+        // ================= MMA issuer: the whole warp runs the loop, one elected lane issues =================
+        {
+            const uint32_t leader = elect_one();
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
-            auto issue_qk = [&](int t, int j) {          // S_t = Q_t K_j^T
-                const uint32_t kaddr = sK + (j & 1) * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
+            auto issue_qk = [&](int t, int ksl) {        // S_t = Q_t K^T with the K tile in ring slot ksl
+                const uint32_t kaddr = sKV + ksl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma_ss(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0);
+                    umma_ss_w(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
                 }
-                commit1(bar(S_FULL + t));
+                commit1_w(bar(S_FULL + t), leader);
             };
-            auto issue_pv = [&](int t, int j) {          // O~_t (+)= P_t V_j
-                const uint32_t vaddr = sV + (j & 1) * TILE_BYTES;
+            // O~_t (+)= P_t V_j with V_j in ring slot vsl, in two halves of 64 keys: the row threads release the first half of
+            // P while they still exponentiate the second
+            auto issue_pv = [&](int t, int j, int vsl) -> bool {
+                const uint32_t vaddr = sKV + vsl * TILE_BYTES;
+                if (!mbar_wait(bar(P_HALF + t), (uint32_t)j & 1, abort_flag, p.status)) return false;
+                tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
-                            (j > 0 || kk > 0) ? 1u : 0u);
-                commit1(bar(O_FULL + t));
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_ts_w(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
+                              (j > 0 || kk > 0) ? 1u : 0u, leader);
+                if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 4; kk < 8; ++kk)
+                    umma_ts_w(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv, 1u, leader);
+                commit1_w(bar(O_FULL + t), leader);
+                return true;
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
-            if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(KV_FULL + 0), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
                 issue_qk(0, 0);
                 issue_qk(1, 0);
-                commit1(bar(K_EMPTY + 0));                // K_0 consumed
+                commit1_w(bar(KV_EMPTY + 0), leader);               // K_0 consumed
             }
-            for (int j = 0; j < n_steps_b && ok; ++j) {
-                const int st = j & 1;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1;
+            int sl = 1;                                   // ring slot and phase of tile number 2j+1 = V_j
+            uint32_t ph = 0;
+            int j = 0;
+            // steady state: both tiles do P V_j and Q K_{j+1}^T. Straight-line body: every branch between two tcgen05.mma
+            // instructions costs the issuing warp tens of cycles in which the tensor pipe drains.
+            const int n_common = min(n_steps_a, n_steps_b) - 1;
+            for (; j < n_common && ok; ++j) {
+                const int vsl = sl;
+                const uint32_t vph = ph;
+                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
+                const int ksl = sl;
+                const uint32_t kph = ph;
+                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
+                ok = mbar_wait(bar(KV_FULL + vsl), vph, abort_flag, p.status) && mbar_wait(bar(KV_FULL + ksl), kph, abort_flag, p.status) &&
+                     issue_pv(0, j, vsl);
+                if (!ok) break;
+                issue_qk(0, ksl);
+                ok = issue_pv(1, j, vsl);
+                if (!ok) break;
+                issue_qk(1, ksl);
+                commit1_w(bar(KV_EMPTY + vsl), leader);
+                commit1_w(bar(KV_EMPTY + ksl), leader);
+            }
+            for (; j < n_steps_b && ok; ++j) {            // the last steps: a tile may have run out of key tiles
                 const bool more = j + 1 < n_steps_b;
+                const int vsl = sl;
+                if (!mbar_wait(bar(KV_FULL + vsl), ph, abort_flag, p.status)) { ok = false; break; }
+                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
+                const int ksl = sl;                       // tile number 2j+2 = K_{j+1}
                 if (more) {
-                    if (!mbar_wait(bar(K_FULL + (st ^ 1)), (uint32_t)((j + 1) >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    if (!mbar_wait(bar(KV_FULL + ksl), ph, abort_flag, p.status)) { ok = false; break; }
+                    if (++sl == KV_RING) { sl = 0; ph ^= 1; }
                 }
-                if (!mbar_wait(bar(V_FULL + st), ph, abort_flag, p.status)) { ok = false; break; }
                 for (int t = 0; t < 2 && ok; ++t) {
                     const int n_t = t == 0 ? n_steps_a : n_steps_b;
-                    if (j < n_t) {
-                        if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
-                        tc_fence_after();
-                        issue_pv(t, j);
-                    }
-                    if (j + 1 < n_t) issue_qk(t, j + 1);   // ordered behind P V of this tile on the tensor pipe
+                    if (j < n_t && !issue_pv(t, j, vsl)) { ok = false; break; }
+                    if (j + 1 < n_t) issue_qk(t, ksl);     // ordered behind P V of this tile on the tensor pipe
                 }
                 if (!ok) break;
-                commit1(bar(V_EMPTY + st));               // V_j consumed by both tiles
+                commit1_w(bar(KV_EMPTY + vsl), leader);             // V_j consumed by both tiles
                 // K_{j+1} consumed by the QK products issued above (both tiles, or tile B alone on its last step)
-                if (more) commit1(bar(K_EMPTY + (st ^ 1)));
+                if (more) commit1_w(bar(KV_EMPTY + ksl), leader);
             }
         }
     } else {
@@ -611,6 +722,28 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
             tmem_ld_wait();
+            if (j > 0 && !diag) {
+                // Speculative step: exponentiate against the offset in use while the row maximum of this tile is still being
+                // computed (the max3 instructions run in the shadow of the ex2 pipe). The first 64 keys of P are released to
+                // the tensor pipe as soon as they are stored, unless some row of the warp outgrew its offset (below).
+                float mx;
+                const float sum0 = row_exp_store_half<0>(v, p.scale_log2e, m_used, tS, mx);
+                const bool need = mx * p.scale_log2e > m_used + 8.f;
+                if (!__any_sync(0xffffffffu, need)) {
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(P_HALF + t));
+                    float unused;
+                    l_run += sum0 + row_exp_store_half<1>(v, p.scale_log2e, m_used, tS, unused);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(P_FULL + t));
+                    continue;
+                }
+                // rare: redo the whole tile with the raised offset (the general path below; S is still in registers)
+            }
             const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
             const float m_new = mx * p.scale_log2e;       // finite: the first key of the sequence is never masked
             // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
@@ -640,7 +773,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(P_FULL + t));
+            if (lane == 0) {
+                mbar_arrive(bar(P_HALF + t));
+                mbar_arrive(bar(P_FULL + t));
+            }
         }
         if (ok && n_t > 0) {
             if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
