@@ -110,6 +110,51 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
             : "memory");
     }
 }
+// The same instruction executed by a whole converged warp in which one lane (pred != 0) issues. Every operand is then a
+// warp-uniform value that the compiler can keep in uniform registers; issued from a single diverged lane the operands have to be
+// moved there before every instruction, which costs the issuing thread tens of cycles per tcgen05.mma.
+template <int CG>
+__device__ __forceinline__ void umma_bf16_w(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate, uint32_t pred) {
+    if (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "setp.ne.b32 q, %5, 0;\n\t"
+            "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "setp.ne.b32 q, %5, 0;\n\t"
+            "@q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred)
+            : "memory");
+    }
+}
+template <int CG>
+__device__ __forceinline__ void umma_commit_w(uint32_t bar, uint32_t pred) {
+    if (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred q;\n\t"
+            "setp.ne.b32 q, %1, 0;\n\t"
+            "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar), "r"(pred) : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile(
+            "{\n\t.reg .pred q;\n\t"
+            "setp.ne.b32 q, %2, 0;\n\t"
+            "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+            ::"r"(bar), "h"(mask), "r"(pred) : "memory");
+    }
+}
+// 1 in exactly one lane of a converged warp
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.b32 %0, 1, 0, q;\n\t}" : "=r"(pred));
+    return pred;
+}
 // arrives on the mbarrier (CG 2: on the same barrier of BOTH CTAs of the pair) once every tcgen05.mma issued so far
 // by this thread has completed
 template <int CG>

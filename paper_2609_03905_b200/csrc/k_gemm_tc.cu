@@ -145,7 +145,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;   // warp-uniform by construction
     const int cta_rank = CG == 2 ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -172,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     if (CG == 2) cluster_sync_all();   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
     const int total_tiles = p.m_tiles * p.n_tiles * p.n_copies;
     const int kchunks = (p.bk + Cfg<CG>::BK - 1) / Cfg<CG>::BK;
@@ -235,8 +235,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             (void)issued; (void)last_parity;
         }
     } else if (warp == 1) {
-        // ================= MMA issuer (leader CTA only) =================
-        if (lane == 0 && cta_rank == 0) {
+        // ================= MMA issuer (leader CTA only): the whole warp runs the loop, one elected lane issues =================
+        if (cta_rank == 0) {
+            const uint32_t leader = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_phase[2] = {0, 0};
@@ -261,19 +262,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int k16 = (kvalid + 15) / 16;
                         const uint32_t a_addr = sA + stage * A_STAGE_BYTES;
                         const uint32_t b_addr = sB + stage * B_STAGE_BYTES;
-                        for (int kk = 0; kk < k16; ++kk) {
-                            // A: K-major, 16 k = 32 bytes inside the swizzle atom, 64 k per half; B: MN-major, 16 k-rows =
-                            // 2048 bytes, 64-column groups BK*128 bytes apart
-                            uint64_t da = desc_sw128(a_addr + (kk >> 2) * A_HALF_BYTES + (kk & 3) * 32, 16);
-                            uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
-                            umma_bf16<CG>(d_tmem, da, db, idesc, accumulate);
-                            accumulate = 1;
+                        // A: K-major, 16 k = 32 bytes inside the swizzle atom, 64 k per half; B: MN-major, 16 k-rows =
+                        // 2048 bytes, 64-column groups BK*128 bytes apart
+                        if (k16 == BK / 16) {   // a full stage: straight-line code, no branch between two tcgen05.mma
+#pragma unroll
+                            for (int kk = 0; kk < BK / 16; ++kk) {
+                                const uint64_t da = desc_sw128(a_addr + (kk >> 2) * A_HALF_BYTES + (kk & 3) * 32, 16);
+                                const uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
+                                umma_bf16_w<CG>(d_tmem, da, db, idesc, kk > 0 ? 1u : accumulate, leader);
+                            }
+                        } else {
+                            for (int kk = 0; kk < k16; ++kk) {
+                                const uint64_t da = desc_sw128(a_addr + (kk >> 2) * A_HALF_BYTES + (kk & 3) * 32, 16);
+                                const uint64_t db = desc_sw128(b_addr + kk * 2048, BK * 128);
+                                umma_bf16_w<CG>(d_tmem, da, db, idesc, kk > 0 ? 1u : accumulate, leader);
+                            }
                         }
-                        umma_commit<CG>(empty_bar(stage));  // frees the smem stage (in both CTAs) once these MMAs have read it
+                        accumulate = 1;
+                        umma_commit_w<CG>(empty_bar(stage), leader);  // frees the smem stage (in both CTAs) once these MMAs have read it
                         if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
                 }
-                if (ok) umma_commit<CG>(tfull_bar(acc));    // accumulator complete -> epilogue(s)
+                if (ok) umma_commit_w<CG>(tfull_bar(acc), leader);    // accumulator complete -> epilogue(s)
             }
         }
     } else {
