@@ -263,6 +263,38 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
 
 
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
+    """Keys whose magnitude grows from one 128-row key tile to the next: the running row maximum then outgrows the exponent
+    offset in use by more than the 2^8 head-room at almost every key tile, so the kernels take their offset-raising path
+    (rescale of the accumulated output, and in the two-tile form the redo of a tile that was exponentiated against the
+    old offset) instead of the common one that N(0,1) inputs exercise."""
+    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
+    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
+    B, S, H, D = 1, 1024, 2, 128
+    Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (31, 32, 33))
+    growth = 1.0 + 3.0 * (np.arange(S) // 128)              # score spread x1, x4, x7, ... per key tile
+    K = (si.to_f64(K) * growth[None, :, None, None]).astype(np.float32)
+    K = torch.from_numpy(K).to(torch.bfloat16)
+    sp = [ES(B, B), ES(S, S // 128), ES(H, H), [0, D]]
+    rQ, rK, rV = upload(Q, sp), upload(K, sp), upload(V, sp)
+    rO = empty_like_tiling([B, S, H, D], sp, BF, fill=float("nan"))
+    rL = empty_like_tiling([B, S, H], sp[:3], F32, fill=float("nan"))
+    parts = {"b": sp[0], "q": sp[1], "h": sp[2], "d": sp[3], "k": sp[1]}
+    spec = ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / np.sqrt(D), 1.0 if causal else 0.0), "online_softmax")
+    spec.execute([rQ, rK, rV], [rO, rL])
+    got, got_l = download(rO), download(rL)
+    check_status()
+    ref = operators.attention(si.to_f64(Q), si.to_f64(K), si.to_f64(V), causal, "bf16")
+    assert relfro(got, ref) <= TOL[BF]
+    ref_l = operators.attention_lse(si.to_f64(Q), si.to_f64(K), causal)
+    assert np.abs(got_l - ref_l).max() <= 2e-3 * max(1.0, np.abs(ref_l).max())
+    # the case does what it is for: the row maximum of the last key tile exceeds that of the first by far more than 8 / log2(e)
+    s = np.einsum("qd,kd->qk", si.to_f64(Q)[0, :, 0], si.to_f64(K)[0, :, 0]) / np.sqrt(D)
+    assert np.median(s[:, -128:].max(1) - s[:, :128].max(1)) > 20.0
+
+
 @pytest.mark.parametrize("form", ["default", "tcgen05_one_tile", "mma_sync"])
 @pytest.mark.parametrize("causal,S,hb", [(True, 512, 1), (False, 384, 2), (True, 256, 2)])
 def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
