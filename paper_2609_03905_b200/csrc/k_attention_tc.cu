@@ -806,6 +806,275 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Two query tiles per CTA with P handed to the P V product through SHARED memory. In the kernel above P overwrites S in
+// tensor memory, so the next Q K^T of a tile cannot start before its P V has read P: per tile the row softmax and the two
+// contractions form one serial chain, and the tensor pipe waits for the row threads about a third of the time. Here the
+// row threads copy S into registers and release the S columns at once, the next Q K^T of the tile runs WHILE they
+// exponentiate, and P goes to a 128-byte-swizzled K-major tile in shared memory (the layout TMA gives Q), read by the P V
+// product as a shared-memory A operand. Shared memory: Q_A, Q_B, P_A, P_B and THREE K / V slots that K_0, K_1, V_0, K_2,
+// V_1, ... pass through in the order the products consume them (7 tiles = 224 KiB).
+// ---------------------------------------------------------------------------------------------------------
+constexpr int SMEM_BYTES3 = 7 * TILE_BYTES + 1024 + 256;
+
+__global__ void __launch_bounds__(NUM_THREADS2, 1)
+attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t sQ = base, sKV = base + 2 * TILE_BYTES, sP = base + 5 * TILE_BYTES;
+    uint8_t* pP = smem + 5 * TILE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 7 * TILE_BYTES);
+    const uint32_t bar0 = smem_u32(bars);
+    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 4, S_FULL = 7, S_FREE = 9, P_FULL = 11, P_EMPTY = 13, O_FULL = 15, NBAR = 17 };
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
+    const int n_pairs = p.S / (2 * QT);
+    int slot, bh;
+    ja_attn_decode_cta((int)blockIdx.x, n_pairs, p.H * p.B, p.sect, &slot, &bh);
+    const int pr = p.n_order ? (int)p.order[slot] : n_pairs - 1 - slot;
+    const int h = bh % p.H, b = bh / p.H;
+    const int q0 = pr * 2 * QT;
+    int s0, s1;
+    sequence_of(p, q0, s0, s1);
+    const int n_steps_a = p.causal ? (q0 + QT - s0) / KT : (s1 - s0) / KT;
+    const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NBAR; ++i) {
+            const bool row_warps_arrive = (i >= S_FREE && i < S_FREE + 2) || (i >= P_FULL && i < P_FULL + 2);
+            mbar_init(bar(i), row_warps_arrive ? 4 : 1);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+
+    // K / V tiles in the order the products consume them: K_0, then for every step j: K_{j+1} (if any), V_j
+    // load index li -> slot li % 3, phase (li / 3) & 1
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            const int hk = h / p.group;
+            mbar_expect_tx(bar(Q_FULL), 2 * TILE_BYTES);
+            for (int t = 0; t < 2; ++t) {
+                const int qrow_t = seq_row(p.q, p.S, b, q0 + t * QT, h);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow_t);
+            }
+            bool ok = true;
+            int li = 0;
+            auto load = [&](const CUtensorMap* tm, int j) {
+                const int sl = li % 3;
+                const uint32_t ph = (uint32_t)(li / 3) & 1;
+                if (!mbar_wait(bar(KV_EMPTY + sl), ph ^ 1, abort_flag, p.status)) { ok = false; return; }
+                const int krow = seq_row(p.k, p.S, b, s0 + j * KT, hk);
+                mbar_expect_tx(bar(KV_FULL + sl), TILE_BYTES);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(sKV + sl * TILE_BYTES + half * HALF_BYTES, tm, bar(KV_FULL + sl), half * 64, hk % p.k.hblk, krow);
+                ++li;
+            };
+            load(&tmK, 0);
+            for (int j = 0; j < n_steps_b && ok; ++j) {
+                if (j + 1 < n_steps_b) load(&tmK, j + 1);
+                if (ok) load(&tmV, j);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        {
+            const uint32_t leader = elect_one();
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            auto issue_qk = [&](int t, int sl) {          // S_t = Q_t K^T, K in slot sl
+                const uint32_t kaddr = sKV + sl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    umma_ss_w(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
+                }
+                commit1_w(bar(S_FULL + t), leader);
+            };
+            auto issue_pv = [&](int t, int sl, bool first) {   // O~_t (+)= P_t V, P in shared memory (K-major), V in slot sl (MN-major)
+                const uint32_t vaddr = sKV + sl * TILE_BYTES, paddr = sP + t * TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    umma_ss_w(tmem_base + 256 + t * 128, desc_sw128(paddr + off, 16), desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
+                              (!first || kk > 0) ? 1u : 0u, leader);
+                }
+                commit1_w(bar(P_EMPTY + t), leader);
+                commit1_w(bar(O_FULL + t), leader);
+            };
+            int li = 0;
+            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(KV_FULL + 0), 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0);
+                issue_qk(1, 0);
+                commit1_w(bar(KV_EMPTY + 0), leader);
+                li = 1;
+            }
+            for (int j = 0; j < n_steps_b && ok; ++j) {
+                if (j + 1 < n_steps_b) {
+                    const int sl = li % 3;
+                    if (!mbar_wait(bar(KV_FULL + sl), (uint32_t)(li / 3) & 1, abort_flag, p.status)) { ok = false; break; }
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        const int n_t = t == 0 ? n_steps_a : n_steps_b;
+                        if (j + 1 < n_t) {
+                            // the row threads have copied S_t of step j into registers: its columns may be overwritten
+                            if (!mbar_wait(bar(S_FREE + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
+                            tc_fence_after();
+                            issue_qk(t, sl);
+                        }
+                    }
+                    if (!ok) break;
+                    commit1_w(bar(KV_EMPTY + sl), leader);
+                    ++li;
+                }
+                const int sl = li % 3;
+                if (!mbar_wait(bar(KV_FULL + sl), (uint32_t)(li / 3) & 1, abort_flag, p.status)) { ok = false; break; }
+                for (int t = 0; t < 2 && ok; ++t) {
+                    const int n_t = t == 0 ? n_steps_a : n_steps_b;
+                    if (j < n_t) {
+                        if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_pv(t, sl, j == 0);
+                    }
+                }
+                if (!ok) break;
+                commit1_w(bar(KV_EMPTY + sl), leader);
+                ++li;
+            }
+        }
+    } else {
+        // ================= row threads =================
+        const int t = (warp - 2) >> 2;
+        const int q = warp & 3;
+        const int r = q * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const uint32_t tS = tmem_base + t * 128 + lane_addr, tO = tmem_base + 256 + t * 128 + lane_addr;
+        const int n_t = t == 0 ? n_steps_a : n_steps_b;
+        const int qrow = q0 + t * QT + r;
+        uint8_t* prow = pP + t * TILE_BYTES + r * 128;     // this row inside each 64-key half of the P tile
+        const int sw = r & 7;                              // 128-byte swizzle: 16-byte chunk c of row r lives at chunk c ^ (r & 7)
+        float m_used = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_t && ok; ++j) {
+            if (!mbar_wait(bar(S_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const bool diag = p.causal && (j == n_t - 1);
+            const int kmax = qrow - (s0 + j * KT);
+            uint32_t v[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(S_FREE + t));   // S_t is in registers: the next Q K^T of this tile may run
+            const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
+            const float m_new = mx * p.scale_log2e;
+            float alpha = 1.f;
+            bool need = false;
+            if (j == 0) m_used = m_new;
+            else if (m_new > m_used + 8.f) { alpha = ex2(m_used - m_new); m_used = m_new; need = true; }
+            // P V of step j-1 has finished: it no longer reads the P tile, and O~ holds the products up to step j-1
+            if (j > 0 && !mbar_wait(bar(P_EMPTY + t), (uint32_t)(j - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+            if (__any_sync(0xffffffffu, need)) {
+                tc_fence_after();
+#pragma unroll 1
+                for (int c = 0; c < 16; ++c) {
+                    uint32_t o[8];
+                    tmem_ld8(tO + c * 8, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st8(tO + c * 8, o);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                l_run *= alpha;
+            }
+            // P = 2^(S*scale - m) as bf16 into the swizzled K-major tile; row sum in f32
+            {
+                const uint64_t sc2 = pack2(p.scale_log2e, p.scale_log2e), nm2 = pack2(-m_used, -m_used);
+                uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {          // 16 chunks of 8 keys = 16 bytes of bf16
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int i = 0; i < 8; i += 2) {
+                        const int col = c * 8 + i;
+                        float p0, p1;
+                        unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
+                        p0 = ex2(p0);
+                        p1 = ex2(p1);
+                        if (diag) {
+                            if (col > kmax) p0 = 0.f;
+                            if (col + 1 > kmax) p1 = 0.f;
+                        }
+                        if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
+                        else sum_b = add2(sum_b, pack2(p0, p1));
+                        __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
+                        pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
+                    }
+                    *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+                float a0, a1, b0, b1;
+                unpack2(sum_a, a0, a1);
+                unpack2(sum_b, b0, b1);
+                l_run += (a0 + a1) + (b0 + b1);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads P through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P_FULL + t));
+        }
+        if (ok && n_t > 0) {
+            if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
+                tc_fence_after();
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
+                char* dst = p.o_base + cell * (D * 2);
+                if (p.lse_base) p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 ov;
+                        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 64 + g * 16) = ov;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
 // "bshd" relation with uniform blocks along b and h as a rank-3 tensor (d, head in block, row of hblk x 128 cells)
 ja_status_t encode_rows(const RelView& v, CUtensorMap* tm) {
     EncodeTiledFn enc = get_encode();
@@ -897,9 +1166,20 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
     if (const char* se = getenv("JA_ATTN_SECTION")) p.sect = std::max(1, atoi(se));
     p.sect = std::min(p.sect, a.H * a.B);
     if (two_tiles) {
-        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
         dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / (2 * QT))), 1, 1);
-        attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
+        // Two forms of the two-tile kernel (both verified against the oracle; JA_ATTN_P_SMEM = 0 / 1 forces one). P through
+        // shared memory takes the next Q K^T of a tile off the chain softmax -> P V -> Q K^T, which pays where work items are
+        // short or uneven (causal band, packed sequences: 5-7 % faster at 1K-2K rows per sequence, equal beyond 8K); with
+        // equal items (not causal, one sequence) P in tensor memory is as fast or faster (10 % at 2K rows).
+        const char* v3 = getenv("JA_ATTN_P_SMEM");
+        const bool p_smem = v3 ? v3[0] == '1' : (a.causal || a.n_ends > 1);
+        if (p_smem) {
+            JA_CUDA(cudaFuncSetAttribute(attention_tc3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
+            attention_tc3_kernel<<<grid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, p);
+        } else {
+            JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
+            attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
+        }
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
