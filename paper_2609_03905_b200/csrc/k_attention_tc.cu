@@ -100,26 +100,10 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 
+// tcgen05.mma and tcgen05.commit as executed by a whole converged warp with one lane (pred != 0) issuing: every operand is then
+// warp-uniform, which lets the compiler keep descriptors and addresses in uniform registers instead of moving them there before
+// every instruction.
 // D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// The same three, executed by a whole converged warp with one lane (pred != 0) issuing: every operand is then warp-uniform, which
-// lets the compiler keep descriptors and addresses in uniform registers instead of moving them there before every instruction.
 __device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate, uint32_t pred) {
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
@@ -129,6 +113,7 @@ __device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint64_t a_desc, uint
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred)
         : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void umma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate, uint32_t pred) {
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
@@ -144,24 +129,11 @@ __device__ __forceinline__ void commit1_w(uint32_t bar, uint32_t pred) {
         "setp.ne.b32 q, %1, 0;\n\t"
         "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar), "r"(pred) : "memory");
 }
-__device__ __forceinline__ void commit1(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
           "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
-          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
-          "r"(r[30]), "r"(r[31])
         : "memory");
 }
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
@@ -198,7 +170,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;   // warp-uniform by construction
     const int n_qt = p.S / QT;
     int slot, bh;
     ja_attn_decode_cta((int)blockIdx.x, n_qt, p.H * p.B, p.sect, &slot, &bh);
@@ -224,7 +196,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
     const uint32_t tS[2] = {tmem_base, tmem_base + 128};
     const uint32_t tO[2] = {tmem_base + 256, tmem_base + 384};
 
@@ -252,8 +224,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
+        // ================= MMA issuer: the whole warp runs the loop, one elected lane issues =================
+        {
+            const uint32_t leader = elect_one();
             // S = Q K^T: M=128, N=128, A and B K-major.  O' = P V: A from TMEM, B MN-major.
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
@@ -263,10 +236,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {   // 16 d per instruction; d 0..63 in the first half, 64..127 in the second
                     const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma_ss(tS[st], desc_sw128(sQ + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0);
+                    umma_ss_w(tS[st], desc_sw128(sQ + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
                 }
-                commit1(bar(S_FULL + st));
-                commit1(bar(K_EMPTY + st));
+                commit1_w(bar(S_FULL + st), leader);
+                commit1_w(bar(K_EMPTY + st), leader);
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
             if (ok) ok = mbar_wait(bar(K_FULL + 0), 0, abort_flag, p.status);
@@ -289,9 +262,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const uint32_t vaddr = sV + st * TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)     // 16 keys per instruction: 8 TMEM columns of packed bf16 P, 2048 bytes of V
-                    umma_ts(tO[st], tS[st] + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv, kk > 0);
-                commit1(bar(O_FULL + st));
-                commit1(bar(V_EMPTY + st));
+                    umma_ts_w(tO[st], tS[st] + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv, kk > 0, leader);
+                commit1_w(bar(O_FULL + st), leader);
+                commit1_w(bar(V_EMPTY + st), leader);
             }
         }
     } else {
