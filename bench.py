@@ -563,6 +563,36 @@ def run_case(args):
                 res["p%d_%s" % (p_, name)] = {**t, "proxy_cost_cells": ja.ja_plan_cost(ops, plan), "relayouts": n_rep,
                                               "TFLOPs": 6.0 * T * d * f / (t["ms_mean"] * 1e-3) / 1e12, "plan": plan}
             res["p%d_optimizer_host_ms" % p_] = {"ms_mean": opt_ms, "ms_min": opt_ms, "ms_median": opt_ms, "cost": best_cost}
+        # Section 6 ablation in miniature: 20 plans drawn at random (one spec per operator, uniformly from specs(Op) for p = 8,
+        # seeded), their proxy cost and measured chain time against the optimizer's plan
+        import random
+
+        def all_specs(op, p_):
+            letters = []
+            for term in op["einsum"].replace("->", ",").split(","):
+                letters += [c for c in term if c not in letters]
+            out = []
+
+            def rec(i, rest, acc):
+                if i == len(letters):
+                    if rest == 1: out.append(dict(zip(letters, acc)))
+                    return
+                for c_ in range(1, rest + 1):
+                    if rest % c_ == 0: rec(i + 1, rest // c_, acc + [c_])
+            rec(0, p_, [])
+            return out
+
+        rng = random.Random(3905)
+        cand = [all_specs(op, 8) for op in ops]
+        draws = []
+        for n_ in range(20):
+            plan = [rng.choice(c_) for c_ in cand]
+            t, n_rep = run_plan(plan)
+            draws.append({"ms": t["ms_median"], "proxy_cost_cells": ja.ja_plan_cost(ops, plan), "relayouts": n_rep, "plan": plan})
+        ms_sorted = sorted(d_["ms"] for d_ in draws)
+        res["p8_random_20"] = {"ms_mean": sum(ms_sorted) / 20, "ms_min": ms_sorted[0], "ms_median": 0.5 * (ms_sorted[9] + ms_sorted[10]),
+                               "ms_max": ms_sorted[-1], "proxy_cost_cells_median": sorted(d_["proxy_cost_cells"] for d_ in draws)[10],
+                               "proxy_cost_cells_min": min(d_["proxy_cost_cells"] for d_ in draws), "draws": draws}
     elif args.case == "chains":
         # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
         # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)
