@@ -60,6 +60,7 @@ struct GemmParams {
     int32_t tiles_per_mblk;    // >= 1 when row tiles never leave a block, 0 when tiles are cut from global rows
     int32_t tiles_per_nblk;    // >= 1 when tiles stay inside one column block, 0 when tiles span blocks
     int32_t group_m;           // row tiles per rasterisation band
+    int32_t heavy_first;       // 1: full-width tiles are scheduled before the narrow last tile of every column block (see tile_of_iter)
     // fused epilogue (a join-agg chain executed in one pass, the intermediate never stored)
     int32_t epi;               // EPI_*
     int32_t bn_tile;           // output columns per tile: 256, or 128 for EPI_SWIGLU (two 128-column products per tile)
@@ -92,12 +93,23 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int 
     t -= tc.copy * per_copy;
     tc.jb0 = p.n_copies > 1 ? tc.copy : 0;
     tc.jb1 = p.n_copies > 1 ? tc.copy + 1 : p.nbk;
+    // heavy-first schedule: t counts the full-width tiles of all column blocks first, then the narrow last tiles
+    int n_tiles_v = p.n_tiles;
+    bool narrow = false;
+    if (p.heavy_first) {
+        const int full_tiles = p.m_tiles * p.nbn * (p.tiles_per_nblk - 1);
+        narrow = t >= full_tiles;
+        if (narrow) t -= full_tiles;
+        n_tiles_v = narrow ? p.nbn : p.nbn * (p.tiles_per_nblk - 1);
+    }
     // banded rasterisation: tiles that run at the same time cover group_m row tiles x several column tiles, so the
     // operand strips they stream fit in L2 together
-    const int band_sz = p.group_m * p.n_tiles;
+    const int band_sz = p.group_m * n_tiles_v;
     const int band = t / band_sz, tin = t - band * band_sz;
     const int rows_in_band = min(p.group_m, p.m_tiles - band * p.group_m);
-    const int mt = band * p.group_m + tin % rows_in_band, nt = tin / rows_in_band;
+    const int mt = band * p.group_m + tin % rows_in_band;
+    int nt = tin / rows_in_band;
+    if (p.heavy_first) nt = narrow ? nt * p.tiles_per_nblk + p.tiles_per_nblk - 1 : (nt / (p.tiles_per_nblk - 1)) * p.tiles_per_nblk + nt % (p.tiles_per_nblk - 1);
     if (p.tiles_per_mblk > 0) {   // CG == 1 only: row tiles stay inside a block
         tc.mb = mt / p.tiles_per_mblk;
         tc.r0 = (mt % p.tiles_per_mblk) * BM;
@@ -121,6 +133,14 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int t, int 
         tc.width = min(p.bn_tile, p.N - tc.n_g0);
     }
     return tc;
+}
+
+// Which tile a CTA group works on in its i-th round, or -1 when it has none left. Plain round-robin, or -- with the heavy-first
+// order, where tiles come sorted by weight -- round-robin that reverses direction every round, so that the groups that got an
+// extra full tile in the last full-width round are the last to be handed narrow ones.
+__device__ __forceinline__ int tile_of_iter(const GemmParams& p, int i, int first, int step, int total) {
+    const int t = i * step + ((p.heavy_first && (i & 1)) ? step - 1 - first : first);
+    return t < total ? t : -1;
 }
 
 template <int CG>
@@ -187,7 +207,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int t = first_tile; t < total_tiles && ok; t += tile_step) {
+            for (int it = 0; ok; ++it) {
+                const int t = tile_of_iter(p, it, first_tile, tile_step, total_tiles);
+                if (t < 0) break;
                 const TileCoord tc = tile_coord<CG>(p, t, cta_rank);
                 // EPI_SWIGLU: the MMA tile is [128 columns of x W1 | the same 128 columns of x W3]
                 const int n_mma = p.epi == EPI_SWIGLU ? 2 * tc.width : (tc.width + 15) / 16 * 16;
@@ -241,9 +263,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_phase[2] = {0, 0};
-            int it = 0;
             bool ok = true;
-            for (int t = first_tile; t < total_tiles && ok; t += tile_step, ++it) {
+            for (int it = 0; ok; ++it) {
+                const int t = tile_of_iter(p, it, first_tile, tile_step, total_tiles);
+                if (t < 0) break;
                 const TileCoord tc = tile_coord<CG>(p, t, 0);
                 const int acc = it & 1;
                 const uint32_t n_mma = p.epi == EPI_SWIGLU ? (uint32_t)(2 * tc.width) : (uint32_t)((tc.width + 15) / 16 * 16);
@@ -290,11 +313,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ================= epilogue (warps 2..5 of every CTA) =================
         const int q = warp & 3;  // TMEM lane group this warp may access
         uint32_t acc_phase[2] = {0, 0};
-        int it = 0;
         bool ok = true;
         const uint32_t tempty0 = CG == 2 ? mapa_cluster(tempty_bar(0), 0) : tempty_bar(0);
         const uint32_t tempty1 = CG == 2 ? mapa_cluster(tempty_bar(1), 0) : tempty_bar(1);
-        for (int t = first_tile; t < total_tiles && ok; t += tile_step, ++it) {
+        for (int it = 0; ok; ++it) {
+            const int t = tile_of_iter(p, it, first_tile, tile_step, total_tiles);
+            if (t < 0) break;
             const TileCoord tc = tile_coord<CG>(p, t, cta_rank);
             const int acc = it & 1;
             if (!mbar_wait(tfull_bar(acc), acc_phase[acc], abort_flag, p.status)) { ok = false; break; }
@@ -451,6 +475,11 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     else { p.tiles_per_nblk = (int)((bn + bn_tile - 1) / bn_tile); p.n_tiles = p.tiles_per_nblk * p.nbn; }
     // Two-CTA form: 256-row tiles cut from global rows; needs 128-row halves that never straddle a block and, when
     // tiles span column blocks, column tails whose halves still start on a 64-column box boundary.
+    // narrow last tile in every column block (block width not a multiple of the tile width): schedule it after the full tiles
+    {
+        const char* hf = getenv("JA_GEMM_HEAVY_FIRST");
+        p.heavy_first = (p.n_copies == 1 && p.tiles_per_nblk > 1 && bn % bn_tile != 0 && !(hf && hf[0] == '0')) ? 1 : 0;
+    }
     const char* gm = getenv("JA_GEMM_GROUP_M");
     p.group_m = gm ? atoi(gm) : 8;
     if (p.group_m < 1) p.group_m = 1;
