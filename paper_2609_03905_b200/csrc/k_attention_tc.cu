@@ -100,6 +100,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 
+// TMA store of one box from shared memory (bulk-group completion)
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+
 // tcgen05.mma and tcgen05.commit as executed by a whole converged warp with one lane (pred != 0) issuing: every operand is then
 // warp-uniform, which lets the compiler keep descriptors and addresses in uniform registers instead of moving them there before
 // every instruction.
@@ -792,7 +799,8 @@ constexpr int SMEM_BYTES3 = 7 * TILE_BYTES + 1024 + 256;
 
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
 attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                     const __grid_constant__ AttnTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -801,7 +809,7 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint8_t* pP = smem + 5 * TILE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 7 * TILE_BYTES);
     const uint32_t bar0 = smem_u32(bars);
-    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 4, S_FULL = 7, S_FREE = 9, P_FULL = 11, P_EMPTY = 13, O_FULL = 15, NBAR = 17 };
+    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 4, S_FULL = 7, S_FREE = 9, P_FULL = 11, P_EMPTY = 13, O_FULL = 15, O_STAGED = 17, NBAR = 19 };
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -820,7 +828,7 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBAR; ++i) {
-            const bool row_warps_arrive = (i >= S_FREE && i < S_FREE + 2) || (i >= P_FULL && i < P_FULL + 2);
+            const bool row_warps_arrive = (i >= S_FREE && i < S_FREE + 2) || (i >= P_FULL && i < P_FULL + 2) || i >= O_STAGED;
             mbar_init(bar(i), row_warps_arrive ? 4 : 1);
         }
         *abort_flag = 0;
@@ -1016,12 +1024,16 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (lane == 0) mbar_arrive(bar(P_FULL + t));
         }
         if (ok && n_t > 0) {
+            // O = O~ / l goes out through the tile's P buffer (its last P V has read it once O_FULL fires): every row thread
+            // writes its 256 bytes in the swizzled layout of the tensor map, and one thread hands the tile to two TMA stores --
+            // 16-byte stores from 32 lanes to 32 different rows would write half-filled sectors.
             if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
                 tc_fence_after();
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
-                char* dst = p.o_base + cell * (D * 2);
-                if (p.lse_base) p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+                if (p.lse_base) {
+                    const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
+                    p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
+                }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -1034,8 +1046,19 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
                             po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 64 + g * 16) = ov;
+                        const int cc = c * 4 + g;                      // 16-byte chunk 0..15 of the row
+                        *reinterpret_cast<uint4*>(prow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) = ov;
                     }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(O_STAGED + t));
+                if (q == 0 && lane == 0 && mbar_wait(bar(O_STAGED + t), 0, abort_flag, p.status)) {
+                    const int orow = seq_row(p.q, p.S, b, q0 + t * QT, h);
+                    for (int half = 0; half < 2; ++half)
+                        tma_store_3d(&tmO, sP + t * TILE_BYTES + half * HALF_BYTES, half * 64, h % p.q.hblk, orow);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
                 }
             }
         }
@@ -1148,8 +1171,10 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
         const char* v3 = getenv("JA_ATTN_P_SMEM");
         const bool p_smem = v3 ? v3[0] == '1' : (a.causal || a.n_ends > 1);
         if (p_smem) {
+            CUtensorMap to;
+            if ((s = encode_rows(a.o, &to)) != JA_OK) return s;
             JA_CUDA(cudaFuncSetAttribute(attention_tc3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
-            attention_tc3_kernel<<<grid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, p);
+            attention_tc3_kernel<<<grid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
         } else {
             JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
             attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
