@@ -531,7 +531,8 @@ constexpr int SMEM_BYTES2 = (2 + KV_RING) * TILE_BYTES + 1024 + 256;   // Q_A, Q
 
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                     const __grid_constant__ AttnTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -540,7 +541,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + KV_RING) * TILE_BYTES);
     const uint32_t bar0 = smem_u32(bars);
     // K / V tiles go through one ring in the order K_0 V_0 K_1 V_1 ...: tile number 2j is K_j, 2j+1 is V_j
-    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + KV_RING, S_FULL = 1 + 2 * KV_RING, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4, P_HALF = S_FULL + 6, NBAR = S_FULL + 8 };
+    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + KV_RING, S_FULL = 1 + 2 * KV_RING, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4, P_HALF = S_FULL + 6, O_STAGED = S_FULL + 8, NBAR = S_FULL + 10 };
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -558,7 +559,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), ((i >= P_FULL && i < P_FULL + 2) || (i >= P_HALF && i < P_HALF + 2)) ? 4 : 1);
+        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), ((i >= P_FULL && i < P_FULL + 2) || (i >= P_HALF && i < P_HALF + 2) || i >= O_STAGED) ? 4 : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -754,12 +755,17 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             }
         }
         if (ok && n_t > 0) {
+            // O = O~ / l goes out through the tile's Q buffer (dead since the tile's last Q K^T): every row thread writes its
+            // 256 bytes in the swizzled layout of the tensor map, and one thread hands the tile to two TMA stores
             if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
                 tc_fence_after();
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
-                char* dst = p.o_base + cell * (D * 2);
-                if (p.lse_base) p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
+                if (p.lse_base) {
+                    const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
+                    p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
+                }
+                uint8_t* orow = smem + t * TILE_BYTES + r * 128;
+                const int sw = r & 7;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -772,8 +778,19 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
                             po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 64 + g * 16) = ov;
+                        const int cc = c * 4 + g;                      // 16-byte chunk 0..15 of the row
+                        *reinterpret_cast<uint4*>(orow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) = ov;
                     }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(O_STAGED + t));
+                if (q == 0 && lane == 0 && mbar_wait(bar(O_STAGED + t), 0, abort_flag, p.status)) {
+                    const int orow0 = seq_row(p.q, p.S, b, q0 + t * QT, h);
+                    for (int half = 0; half < 2; ++half)
+                        tma_store_3d(&tmO, sQ + t * TILE_BYTES + half * HALF_BYTES, half * 64, h % p.q.hblk, orow0);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
                 }
             }
         }
@@ -1168,16 +1185,16 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
         // short or uneven (causal band, packed sequences: 5-7 % faster at 1K-2K rows per sequence, equal beyond 8K); with
         // equal items (not causal, one sequence) the two forms measure the same, and P in tensor memory executes a third
         // fewer instructions.
+        CUtensorMap to;
+        if ((s = encode_rows(a.o, &to)) != JA_OK) return s;
         const char* v3 = getenv("JA_ATTN_P_SMEM");
         const bool p_smem = v3 ? v3[0] == '1' : (a.causal || a.n_ends > 1);
         if (p_smem) {
-            CUtensorMap to;
-            if ((s = encode_rows(a.o, &to)) != JA_OK) return s;
             JA_CUDA(cudaFuncSetAttribute(attention_tc3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
             attention_tc3_kernel<<<grid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
         } else {
             JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
-            attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, p);
+            attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);
         }
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
