@@ -242,11 +242,12 @@ def test_rope(splits):
                                                    (1, 256, 1, 64, 64, 1, True), (1, 384, 2, 128, 64, 1, False),
                                                    (1, 512, 1, 256, 128, 1, True), (2, 1024, 3, 128, 256, 3, True),
                                                    (1, 640, 2, 128, 128, 1, False)])
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
 def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
     monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
     monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form == "tcgen05_two_tiles_p_smem" else "0")
+    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
+    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
     D = 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (1, 2, 3))
     spl = lambda blk: [ES(B, B), ES(S, S // blk), ES(H, H // hb), [0, D]]
@@ -264,7 +265,7 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
 
 
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
 @pytest.mark.parametrize("causal", [False, True])
 def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
     """Keys whose magnitude grows from one 128-row key tile to the next: the running row maximum then outgrows the exponent
@@ -273,7 +274,8 @@ def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
     old offset) instead of the common one that N(0,1) inputs exercise."""
     monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
     monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form == "tcgen05_two_tiles_p_smem" else "0")
+    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
+    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
     B, S, H, D = 1, 1024, 2, 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (31, 32, 33))
     growth = 1.0 + 3.0 * (np.arange(S) // 128)              # score spread x1, x4, x7, ... per key tile
@@ -297,13 +299,14 @@ def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
     assert np.median(s[:, -128:].max(1) - s[:, :128].max(1)) > 20.0
 
 
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
 @pytest.mark.parametrize("causal,S,hb", [(True, 512, 1), (False, 384, 2), (True, 256, 2)])
 def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
     """n_outputs = 2: the log of the softmax denominator beside O, and the combine it exists for."""
     monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
     monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form == "tcgen05_two_tiles_p_smem" else "0")
+    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
+    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
     B, H, D = 2, 4, 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (21, 22, 23))
     sp = [ES(B, B), ES(S, S // 128), ES(H, H // hb), [0, D]]
@@ -333,11 +336,12 @@ def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
     (2, 768, 6, 2, 2, [768], 256, True),                    # one sequence, grouped heads only
     (1, 1280, 4, 1, 1, [256, 384, 1280], "ends", True),     # blocks of 256, 128, 896 rows
 ])
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
 def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut, causal, form, monkeypatch):
     monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
     monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form == "tcgen05_two_tiles_p_smem" else "0")
+    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
+    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
     D, grp = 128, Hq // Hkv
     Q = si.normal((B, S, Hq, D), 0.0, 1.0, BF, 4, 11)
     K, V = (si.normal((B, S, Hkv, D), 0.0, 1.0, BF, 4, o) for o in (12, 13))
