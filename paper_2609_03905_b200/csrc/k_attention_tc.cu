@@ -21,6 +21,8 @@
 // Every mbarrier wait is bounded; on expiry the CTA records JA_ERR_TIMEOUT and leaves through the normal exit.
 #include <stdlib.h>
 
+#include <atomic>
+
 #include <algorithm>
 #include <utility>
 #include <vector>
@@ -61,6 +63,7 @@ struct AttnTcParams {
     int32_t ends[JA_MAX_SEQ];
     SeqGeom q, k;                // o is tiled like q, v like k
     int32_t sect;                // (batch, head) pairs per launch-order section (ja_attn_decode_cta)
+    int32_t* queue;              // persistent form: {next item, CTAs finished} of this launch, both zero before and after it
     int32_t n_order;             // > 0: order[slot] = the query tile (pair) in heaviest-first slot `slot`
     uint16_t order[MAX_ORDER];
 };
@@ -1090,19 +1093,25 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
 // ---------------------------------------------------------------------------------------------------------
 // The shared-memory form above, persistent over work items. One work item = the pair of query tiles of one (batch, head);
-// one CTA per SM walks items in an order known to all its roles (heaviest items first; rounds alternate direction, so that
-// every CTA's share of the work is about the same). Barriers and tensor memory are set up once. The producer runs ahead
+// one CTA per SM takes items, heaviest first, from a counter in global memory (its producer thread claims the next item and
+// hands its number to the other roles through a two-entry queue in shared memory), so CTAs that drew short items simply take
+// more of them. Barriers and tensor memory are set up once. The producer runs ahead
 // into the next item as soon as the Q buffers are free (after the item's last Q K^T, about one key step before its end),
 // so the next item's Q and first K tile load, and its first Q K^T products run, while the row threads finish the last
 // softmax, normalise and store this item's output. Barrier phases follow running counters (items; key steps per tile).
 // ---------------------------------------------------------------------------------------------------------
+// {next item, CTAs finished} pairs for launches of the persistent kernel: a launch takes the next pair of the ring, and its
+// last CTA zeroes the pair again, so a pair is ready for reuse (also by a replay of a captured launch) as soon as its kernel
+// has finished. 256 launches would have to be in flight at once for two of them to share a pair.
+constexpr int ATTN_QUEUES = 256;
+__device__ int32_t g_attn_queues[2 * ATTN_QUEUES];
+
 struct AttnItem {
     int q0, h, b, s0, n_a, n_b;
 };
-// item of CTA `cta` in round `round`; false past the end
-__device__ __forceinline__ bool attn_item(const AttnTcParams& p, int cta, int n_ctas, int round, AttnItem* it) {
+// item number `rank` in heaviest-first order; false past the end
+__device__ __forceinline__ bool attn_item(const AttnTcParams& p, int rank, AttnItem* it) {
     const int hb = p.H * p.B, n_pairs = p.S / (2 * QT);
-    const int rank = round * n_ctas + ((round & 1) ? n_ctas - 1 - cta : cta);
     if (rank >= n_pairs * hb) return false;
     const int pidx = rank / hb, r = rank - pidx * hb;
     const int pr = p.n_order ? (int)p.order[pidx] : n_pairs - 1 - pidx;   // heaviest pairs of all (batch, head) first
@@ -1129,19 +1138,28 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 7 * TILE_BYTES);
     const uint32_t bar0 = smem_u32(bars);
     enum { Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 5, S_FULL = 8, S_FREE = 10, P_FULL = 12, P_EMPTY = 14, O_FULL = 16,
-           O_STAGED = 18, O_READ = 20, P_STORED = 22, NBAR = 24 };
+           O_STAGED = 18, O_READ = 20, P_STORED = 22, ITEM_FULL = 24, ITEM_EMPTY = 26, NBAR = 28 };
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* item_rank = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [2]: the item numbers in flight
 
     const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
-    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    // consumers of the item queue (MMA warp, row warps): wait for entry k, read it, release it
+    auto next_item = [&](int k, AttnItem* it) -> bool {
+        const int e = k & 1;
+        if (!mbar_wait(bar(ITEM_FULL + e), (uint32_t)(k >> 1) & 1, abort_flag, p.status)) return false;
+        const int rank = item_rank[e];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(ITEM_EMPTY + e));
+        return attn_item(p, rank, it);
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBAR; ++i) {
             const bool row_warps_arrive = (i >= S_FREE && i < S_FREE + 2) || (i >= P_FULL && i < P_FULL + 2) ||
                                           (i >= O_STAGED && i < O_STAGED + 2) || (i >= O_READ && i < O_READ + 2);
-            mbar_init(bar(i), row_warps_arrive ? 4 : 1);
+            mbar_init(bar(i), row_warps_arrive ? 4 : (i >= ITEM_EMPTY && i < ITEM_EMPTY + 2) ? 9 : 1);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1161,7 +1179,15 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             int li = 0;                       // K / V tiles loaded so far: ring slot li % 3, phase (li / 3) & 1
             bool ok = true;
             AttnItem it;
-            for (int item = 0; ok && attn_item(p, cta, n_ctas, item, &it); ++item) {
+            for (int item = 0; ok; ++item) {
+                // claim the next item and publish its number (entry item & 1 of the queue, free once all nine consumer warps
+                // have read what it held two items ago)
+                const int e = item & 1;
+                if (item >= 2 && !mbar_wait(bar(ITEM_EMPTY + e), (uint32_t)((item >> 1) - 1) & 1, abort_flag, p.status)) break;
+                const int rank = atomicAdd(p.queue, 1);
+                item_rank[e] = rank;
+                mbar_arrive(bar(ITEM_FULL + e));
+                if (!attn_item(p, rank, &it)) break;
                 const int hk = it.h / p.group;
                 // the Q buffers are free once the previous item's last Q K^T has read them
                 if (item > 0 && !mbar_wait(bar(Q_EMPTY), (uint32_t)(item - 1) & 1, abort_flag, p.status)) break;
@@ -1186,6 +1212,13 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     if (j + 1 < it.n_b) load(&tmK, j + 1);
                     if (ok) load(&tmV, j);
                 }
+            }
+            // the last CTA to get here leaves the counter pair as it found it
+            __threadfence();
+            if (atomicAdd(p.queue + 1, 1) == (int)gridDim.x - 1) {
+                p.queue[0] = 0;
+                p.queue[1] = 0;
+                __threadfence();
             }
         }
     } else if (warp == 1) {
@@ -1217,7 +1250,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         int cs[2] = {0, 0};                   // key steps of each tile in all items so far
         bool ok = true;
         AttnItem it;
-        for (int item = 0; ok && attn_item(p, cta, n_ctas, item, &it); ++item) {
+        for (int item = 0; ok && next_item(item, &it); ++item) {
             const int n_of[2] = {it.n_a, it.n_b};
             ok = mbar_wait(bar(Q_FULL), (uint32_t)item & 1, abort_flag, p.status);
             {
@@ -1280,7 +1313,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         int cs = 0;                                        // key steps of this tile in all items so far
         bool ok = true;
         AttnItem it;
-        for (int item = 0; ok && attn_item(p, cta, n_ctas, item, &it); ++item) {
+        for (int item = 0; ok && next_item(item, &it); ++item) {
             const int n_t = t == 0 ? it.n_a : it.n_b;
             const int qrow = it.q0 + t * QT + r;
             float m_used = -INFINITY, l_run = 0.f;
@@ -1522,6 +1555,13 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
             }
             const char* pe = getenv("JA_ATTN_PERSISTENT");
             if (pe ? pe[0] == '1' : longest <= 4096) {
+                static int32_t* queues = nullptr;
+                static std::atomic<unsigned> next_queue{0};
+                if (!queues && cudaGetSymbolAddress((void**)&queues, g_attn_queues) != cudaSuccess) {
+                    queues = nullptr;
+                    return ja_fail(JA_ERR_CUDA, "cannot resolve the attention work queues");
+                }
+                p.queue = queues + 2 * (next_queue.fetch_add(1) % ATTN_QUEUES);
                 JA_CUDA(cudaFuncSetAttribute(attention_tc3p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
                 dim3 pgrid((unsigned)std::min<int64_t>((int64_t)a.H * a.B * (a.S / (2 * QT)), sms), 1, 1);
                 attention_tc3p_kernel<<<pgrid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
