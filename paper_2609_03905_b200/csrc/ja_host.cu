@@ -60,6 +60,7 @@ extern "C" ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_s
     if (v != 0) {
         int zero = 0;
         JA_CUDA(cudaMemcpy(w, &zero, sizeof zero, cudaMemcpyHostToDevice));
+        ja_attention_reset_queues();
     }
     return JA_OK;
 }

@@ -161,3 +161,4 @@ struct AttnArgs {
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);
 // tcgen05 / TMEM form; *launched stays false when the tiling does not fit it
 ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched);
+void ja_attention_reset_queues();   // zeroes the work counters of the persistent attention kernel (after a device-side failure)

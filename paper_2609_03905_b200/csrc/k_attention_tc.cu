@@ -1475,6 +1475,13 @@ bool fill_geom(const RelView& v, const int32_t* host_split, SeqGeom* g) {
 
 }  // namespace
 
+// After a device-side failure (a bounded wait that expired) a persistent launch may have left its work counter non-zero:
+// put every counter pair back to zero. Called by ja_stream_status when it reports such a failure; the stream is idle then.
+void ja_attention_reset_queues() {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_attn_queues) == cudaSuccess && q) cudaMemset(q, 0, sizeof(int32_t) * 2 * ATTN_QUEUES);
+}
+
 // Returns JA_OK and sets *launched when the tensor-memory kernel took the job; leaves *launched false when the
 // tiling does not fit it (every q / k split point and sequence end must be a multiple of 128 rows, blocks uniform
 // along b and h, at most MAX_SB sequence blocks when they are irregular).
