@@ -1102,7 +1102,8 @@ attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 // ---------------------------------------------------------------------------------------------------------
 // {next item, CTAs finished} pairs for launches of the persistent kernel: a launch takes the next pair of the ring, and its
 // last CTA zeroes the pair again, so a pair is ready for reuse (also by a replay of a captured launch) as soon as its kernel
-// has finished. 256 launches would have to be in flight at once for two of them to share a pair.
+// has finished. 128 launches would have to be in flight at once (or 128 captured launches alive in graphs that replay
+// concurrently) for two of them to share a pair.
 constexpr int ATTN_QUEUES = 256;
 __device__ int32_t g_attn_queues[2 * ATTN_QUEUES];
 
@@ -1568,7 +1569,14 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
                     queues = nullptr;
                     return ja_fail(JA_ERR_CUDA, "cannot resolve the attention work queues");
                 }
-                p.queue = queues + 2 * (next_queue.fetch_add(1) % ATTN_QUEUES);
+                // launches recorded into a CUDA graph keep their pair for as long as the graph lives: they draw from the upper half
+                // of the ring, launches that run at once from the lower half, so a replay never shares a pair with an eager launch
+                static std::atomic<unsigned> next_captured{0};
+                cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+                if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
+                const unsigned half = ATTN_QUEUES / 2;
+                const unsigned slot = cap == cudaStreamCaptureStatusActive ? half + next_captured.fetch_add(1) % half : next_queue.fetch_add(1) % half;
+                p.queue = queues + 2 * slot;
                 JA_CUDA(cudaFuncSetAttribute(attention_tc3p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
                 dim3 pgrid((unsigned)std::min<int64_t>((int64_t)a.H * a.B * (a.S / (2 * QT)), sms), 1, 1);
                 attention_tc3p_kernel<<<pgrid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
