@@ -112,38 +112,68 @@ def replica_aggregate(ms_values, flops_per_replica_step, steps, world, device="c
 
 # ---- GPU leg ---------------------------------------------------------------------------------------------------
 class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """nvidia-smi polled every 20 ms in a child process that is started well before the timed region (its start-up takes longer
+    than a short region lasts); every sample carries nvidia-smi's own timestamp, and only those that fall inside the region
+    marked by mark_start() / mark_end() are reported."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.proc = None
+        self.t0 = self.t1 = None
+        self.lines = []
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            import threading
+            self.reader = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)   # keeps the pipe drained
+            self.reader.start()
         except Exception:
             self.proc = None
+
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
 
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        import datetime
+        time.sleep(0.05)
         self.proc.terminate()
-        out, _ = self.proc.communicate(timeout=10)
-        sm, mx, reasons = [], [], set()
-        for line in out.strip().splitlines():
+        self.reader.join(timeout=10)
+        rows = []
+        for line in list(self.lines):
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), f[4:8]))
             except ValueError:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+        t0 = self.t0 if self.t0 is not None else 0.0
+        t1 = self.t1 if self.t1 is not None else float("inf")
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        note = None
+        if not inside and rows:   # a region shorter than the polling period: the samples nearest to it
+            mid = 0.5 * (t0 + min(t1, t0 + 3600.0))
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:3]
+            note = "no sample fell inside the timed region; the three nearest are reported"
+        sm = [r[1] for r in inside]
+        mx = [r[2] for r in inside]
+        reasons = set()
+        for r in inside:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        busy = [s for s in sm if s > 300] or sm
-        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        res = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+               "reasons": sorted(reasons), "samples": len(sm)}
+        if note:
+            res["note"] = note
+        return res
 
 
 def run_gpu(args, shape):
@@ -159,6 +189,7 @@ def run_gpu(args, shape):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    sampler = ClockSampler(local) if rank == 0 else None   # started during set-up so that it is polling long before the timed region
     bf = torch.bfloat16
     Bt, S, hidden, heads, ffn = shape["batch"], shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
     T = Bt * S
@@ -212,15 +243,18 @@ def run_gpu(args, shape):
     assert ja.ja_stream_status(stream.cuda_stream) == 0, "device status word set during warm-up"
 
     # ---- timed region: K steps, inputs resident in HBM ---------------------------------------------------------
-    sampler = ClockSampler(local) if rank == 0 else None
     launches0 = ja.ja_launch_count()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
+    if sampler:
+        sampler.mark_start()
     t_start.record(stream)
     for _ in range(args.steps):
         timed_forward(True)
     t_end.record(stream)
     sync_all()
+    if sampler:
+        sampler.mark_end()
     launches = ja.ja_launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     ms_total = t_start.elapsed_time(t_end)
