@@ -230,7 +230,9 @@ __device__ __forceinline__ uint32_t narrow(uint64_t v) {   // two f32 -> packed 
     return *reinterpret_cast<const uint32_t*>(&t);
 }
 
-template <int OP, int VPL>
+// FULL: every lane owns VPL valid vectors of the row (the row length is exactly VPL * warps-per-row * 32 vectors), so the walk
+// over them is straight-line code that the compiler can interleave; otherwise each vector is guarded.
+template <int OP, int VPL, bool FULL>
 __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL], const uint8_t* g_s,
                                          int64_t stat_off, int lane, Team& team) {
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
@@ -242,7 +244,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         uint64_t acc0 = pk2(0.f, 0.f), acc1 = pk2(0.f, 0.f);
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
-            if (off[k] >= 0) {
+            if (FULL || off[k] >= 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
                 const uint64_t f0 = widen(v.x), f1 = widen(v.y), f2 = widen(v.z), f3 = widen(v.w);
                 acc0 = fma2(f0, f0, acc0);
@@ -264,7 +266,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         __nv_bfloat162 mx = __float2bfloat162_rn(-INFINITY);
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
-            if (off[k] >= 0) {
+            if (FULL || off[k] >= 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
                 const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
                 mx = __hmax2(__hmax2(mx, h[0]), __hmax2(h[1], __hmax2(h[2], h[3])));
@@ -287,7 +289,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
         uint64_t acc0 = pk2(0.f, 0.f), acc1 = pk2(0.f, 0.f);
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
-            if (off[k] >= 0) {
+            if (FULL || off[k] >= 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
                 const uint64_t e0 = exp_pair(v.x), e1 = exp_pair(v.y), e2 = exp_pair(v.z), e3 = exp_pair(v.w);
                 if (KEEP_EXP) { ex[k * 4] = e0; ex[k * 4 + 1] = e1; ex[k * 4 + 2] = e2; ex[k * 4 + 3] = e3; }
@@ -314,7 +316,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
     const uint64_t scale2 = pk2(scale, scale);
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
-        if (off[k] < 0) continue;
+        if (!FULL && off[k] < 0) continue;
         uint4 o;
         if (HAS_G) {
             const uint4 v = *reinterpret_cast<const uint4*>(rowp + off[k]);
@@ -445,6 +447,7 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
     } else {
         // ================= consumers =================
         int off[VPL];   // byte offset of this lane's k-th vector inside a row of the stage (column block + column), or -1
+        const bool full_rows = (int64_t)VPL * g.wpr * 32 * VEC == (int64_t)g.n;   // no lane has a vector past the end of the row
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int col = ((k * g.wpr + warp % g.wpr) * 32 + lane) * VEC;
@@ -476,7 +479,10 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
             for (int r = tid; r < rows && team.ok; r += n_teams) {
                 uint8_t* rowp = stage + (size_t)r * row_seg_bytes;
                 const int64_t stat_off = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
-                if constexpr (sizeof(T) == 2) row_bf16<OP, VPL>(a, g, rowp, off, g_s, stat_off, lane, team);
+                if constexpr (sizeof(T) == 2) {
+                    if (full_rows) row_bf16<OP, VPL, true>(a, g, rowp, off, g_s, stat_off, lane, team);
+                    else row_bf16<OP, VPL, false>(a, g, rowp, off, g_s, stat_off, lane, team);
+                }
                 else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, lane, team);
             }
             if (!team.ok) break;
