@@ -176,6 +176,37 @@ class ClockSampler:
         return res
 
 
+TRAFFIC_PROFILE = os.path.join("profiles", "gemm_tc_kernel_dram_traffic_llama7b_block.md")
+
+
+def recorded_traffic(args):
+    """DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches
+    of one step) as recorded in the ncu summary under profiles/. The summary names the workload it was captured on and the
+    SHA-256 of the kernel source it was captured with; the figure is reported only for that workload and that source,
+    otherwise traffic is null with the reason."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, TRAFFIC_PROFILE)
+    if not os.path.exists(path):
+        return {"traffic": None, "traffic_note": f"{TRAFFIC_PROFILE} is missing"}
+    text = open(path).read()
+    m_t = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", text)
+    m_a = re.search(r"algorithmic_bytes_per_launch:\s*([0-9.eE+]+)", text)
+    m_h = re.search(r"sha256\(k_gemm_tc\.cu\):\s*([0-9a-f]{64})", text)
+    m_c = re.search(r"captured_at_commit:\s*([0-9a-f]{7,40})", text)
+    if not (m_t and m_h):
+        return {"traffic": None, "traffic_note": f"{TRAFFIC_PROFILE} carries no machine-readable traffic record"}
+    src = os.path.join(ROOT, "paper_2609_03905_b200", "csrc", "k_gemm_tc.cu")
+    digest = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    if digest != m_h.group(1):
+        return {"traffic": None, "traffic_note": f"k_gemm_tc.cu has changed since {TRAFFIC_PROFILE} was captured; no current figure"}
+    if not (args.shape == "7b" and args.plan == "seq" and not args.unfused):
+        return {"traffic": None, "traffic_note": "the recorded capture is of the 7b / seq / fused step only"}
+    return {"traffic": float(m_t.group(1)), "traffic_unit": "bytes per launch (ncu, one pass, full workload)",
+            "traffic_algorithmic": float(m_a.group(1)) if m_a else None, "traffic_source": TRAFFIC_PROFILE,
+            "traffic_commit": m_c.group(1) if m_c else None}
+
+
 def run_gpu(args, shape):
     import torch
     import torch.distributed as dist
@@ -349,17 +380,18 @@ def run_gpu(args, shape):
     gemm_ms = sum(ops[k] for k in gemm_flops)
     peaks = measured_peaks()
     achieved = sum(gemm_flops.values()) / (gemm_ms * 1e-3) / 1e12
+    # Denominator: the burst cuBLAS figure when the timed region is short (under a second the part has not settled at its
+    # power-capped clock: the condition the burst peak was measured in), the sustained one for long regions.
+    short_region = ms_total < 1000.0
+    peak_used = peaks["bf16"] if short_region else peaks["bf16_sustained"]
     roof = {"bound": "tensor", "kernel": f"gemm_tc_kernel ({len(gemm_flops)} launches per step)", "achieved": achieved,
-            "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"],
-            "frac_of_burst_peak": achieved / peaks["bf16"], "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
+            "peak": peak_used, "unit": "TFLOP/s", "frac": achieved / peak_used,
+            "peak_source": peaks["source"] + (" (burst cuBLAS bf16: timed region %.0f ms)" % ms_total if short_region
+                                              else " (sustained cuBLAS bf16: timed region %.0f ms)" % ms_total),
+            "frac_of_burst_peak": achieved / peaks["bf16"], "frac_of_sustained_peak": achieved / peaks["bf16_sustained"],
             "traffic": None, "share_of_step": gemm_ms / ms_step,
             "algorithmic_flops_per_launch": sum(gemm_flops.values()) / len(gemm_flops)}
-    # DRAM bytes per launch of this kernel (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches of one step)
-    # from the ncu capture summarised in profiles/gemm_tc_kernel_dram_traffic_llama7b_block.md; it holds for the workload it
-    # was taken on only
-    if args.shape == "7b" and args.plan == "seq" and not args.unfused:
-        roof["traffic"] = 1.037e9
-        roof["traffic_unit"] = "bytes per launch (ncu, 7b / seq / fused; operands once + output would be 0.456e9)"
+    roof.update(recorded_traffic(args))
     mem_bytes = {"rmsnorm_1": 4.0 * T * hidden, "rmsnorm_2": 4.0 * T * hidden, "rope_q": 4.0 * T * hidden, "rope_k": 4.0 * T * kv_hidden,
                  "residual_1": 6.0 * T * hidden, "residual_2": 6.0 * T * hidden, "silu_mul": 6.0 * T * ffn}
     for k in ops:
@@ -372,6 +404,19 @@ def run_gpu(args, shape):
               "attention": {"ms": ops["attention"], "TFLOPs": attn_fl / (ops["attention"] * 1e-3) / 1e12},
               "gemm_TFLOPs": {k: gemm_flops[k] / (ops[k] * 1e-3) / 1e12 for k in gemm_flops},
               "fused_chains": {"rope": blk.fuse_rope, "residual_add": blk.fuse_add, "swiglu": blk.fuse_swiglu}}
+
+    # ---- configurations 1-4 of the benchmark definition: their kernels in isolation, after the headline region (the block's
+    # relations stay allocated; every timed launch is preceded by an L2 flush), with the clocks of this sub-run
+    configs = None
+    if rank == 0 and args.shape == "7b" and not args.no_configs:
+        cs = ClockSampler(local)
+        time.sleep(0.3)
+        cs.mark_start()
+        configs = {c: case_results(c, args.config_reps) for c in ("cfg1", "cfg2", "cfg3", "cfg4")}
+        torch.cuda.synchronize()
+        cs.mark_end()
+        configs = {"l2": L2_NOTE, "reps_per_kernel": args.config_reps, "clocks": cs.stop(), "kernels": configs,
+                   "peaks": {"hbm_GBps": peaks["hbm_gbs"], "bf16_TFLOPs_burst": peaks["bf16"], "source": peaks["source"]}}
 
     if rank != 0:
         return
@@ -394,23 +439,38 @@ def run_gpu(args, shape):
                 "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": out_host.numel() * 2},
         "cuda_graph_replay": {"value": graph_val, "unit": "TFLOP/s", "ms_per_step": ms_graph / args.steps,
                               "note": "the same steps replayed from one CUDA graph of the chain, timed after the eager region"},
-        "roofline": roof, "cpu_baseline": cpu, "detail": detail}))
+        "roofline": roof, "cpu_baseline": cpu, "configs": configs, "detail": detail}))
     if world > 1:
         dist.destroy_process_group()
 
 
 # ---- single-config kernel benchmarks (configs 2, 3, 4 of the benchmark definition) ----------------------------------
+L2_NOTE = "512 MiB flush buffer written, then a 256 MiB buffer read (clean lines), before every timed launch"
+
+
 def run_case(args):
-    """Times the kernels of one benchmark configuration in isolation (CUDA events around each launch, buffers rotated so
-    that every timed launch reads HBM-cold data when the working set is near the L2 size). Prints one JSON line."""
+    """Times the kernels of one benchmark configuration in isolation and prints one JSON line."""
+    import torch
+    torch.cuda.set_device(0)
+    res = case_results(args.case, args.steps)
+    print(json.dumps({"case": args.case, "reps": args.steps, "l2": L2_NOTE, "peaks": measured_peaks(), "kernels": res}))
+
+
+def case_results(case, reps):
+    """The kernels of one benchmark configuration in isolation: CUDA events around each launch on the current stream, L2
+    flushed before every timed launch. Returns {kernel: {ms_mean, ms_min, ms_median, TFLOPs | GBps, fraction of measured peak}}."""
     import torch
     import paper_2609_03905_b200 as ja
     import synth_inputs as si
     ES = ja.equal_splits
     bf, f32 = torch.bfloat16, torch.float32
-    torch.cuda.set_device(0)
     stream = torch.cuda.current_stream()
     peaks = measured_peaks()
+
+    class _A:
+        pass
+    args = _A()
+    args.case, args.steps = case, reps
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     # Writing the flush buffer evicts the inputs but leaves L2 full of DIRTY lines, whose write-back (up to the L2 size,
     # about as many bytes as a small kernel moves) would then be charged to the kernel under test; a read sweep over a
@@ -667,8 +727,9 @@ def run_case(args):
             del mats, steps
             torch.cuda.empty_cache()
     assert ja.ja_stream_status(stream.cuda_stream) == 0
-    print(json.dumps({"case": args.case, "reps": reps, "l2": "512 MiB flush buffer written, then a 256 MiB buffer read (clean lines), before every timed launch",
-                      "peaks": peaks, "kernels": res}))
+    del flush, clean
+    torch.cuda.empty_cache()
+    return res
 
 
 def main():
@@ -681,6 +742,8 @@ def main():
     ap.add_argument("--impl", choices=["ja", "reference"], default="ja")
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the kernels of configurations 1-4 after the headline region")
+    ap.add_argument("--config-reps", type=int, default=20, help="timed launches per kernel of configurations 1-4")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
     ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "chains"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "

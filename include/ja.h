@@ -135,7 +135,8 @@ ja_status_t ja_relation_bytes(int32_t rank, const int64_t* extents, const int32_
 ja_status_t ja_relation_create(int32_t rank, const int64_t* extents, const int32_t* nparts,
                                const int64_t* const* splits, ja_dtype_t dtype, void* device_ptr, size_t bytes,
                                ja_relation_t** out);
-ja_status_t ja_relation_destroy(ja_relation_t* rel); /* frees key tables only, never the payload */
+/* Frees the key tables and every cached launch state or copy plan that names this relation; never the payload. */
+ja_status_t ja_relation_destroy(ja_relation_t* rel);
 ja_status_t ja_relation_num_blocks(const ja_relation_t* rel, int64_t* nblocks, int32_t* rank);
 /* Key table (host outputs): per block, in key order, coords[rank] (int32), lower[rank], upper[rank]
  * (the tensor type = the key of the paper) and the byte offset of the block in the payload. */
@@ -238,8 +239,8 @@ ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32_t n_nodes,
  * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)
  * Same data movement as ja_repartition -- every atom of the overlay of the two tilings is copied from its
  * source block to its destination block, bit-exact -- for callers that must not trigger a device (or host)
- * allocation: servers that gave all of HBM to their own pool at start-up, latency-critical loops that cannot
- * afford cudaMalloc's implicit synchronisation, harnesses that fail on any allocation they did not make.
+ * allocation: servers that gave all of HBM to their own pool at start-up, loops that must never take
+ * cudaMalloc's implicit device synchronisation, harnesses that fail on any allocation they did not make.
  * It takes the tilings and the payload pointers directly (no relation handles), keeps its copy plan in a
  * fixed device array inside the library (16384 slabs, 512 KiB per GPU, held until process exit) and calls no
  * cudaMalloc / cudaFree / allocating routine.
@@ -250,15 +251,39 @@ ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32_t n_nodes,
  * per tiling, 1024 overlay split points per dimension.
  * All calls share the plan array; it keeps the last call's contents and a call reads only what it has just
  * written, so nothing needs clearing -- but calls whose GPU work overlaps race on it: serialise them.
- * The first call on each device resolves the array's device address; issue it before any stream capture. */
+ * The first call on each device resolves the array's device address; issue it before any stream capture.
+ * The plan reaches the device by a stream-ordered copy from a fixed host table (the host may block briefly while it is
+ * read); a call on a stream that is being captured is refused with JA_ERR_UNSUPPORTED and enqueues nothing. */
 ja_status_t ja_repartition_noalloc(int32_t rank, const int64_t* extents, const int32_t* src_nparts,
                                    const int64_t* const* src_splits, const int32_t* dst_nparts,
                                    const int64_t* const* dst_splits, ja_dtype_t dtype, const void* src_device,
                                    void* dst_device, void* cuda_stream);
 
-/* Device-detected conditions (bounded-wait expiry) accumulate in a status word; this call synchronizes
- * `cuda_stream`, returns the word in *device_status and clears it. */
+/* Device-detected conditions (a bounded wait that ran out: JA_ERR_TIMEOUT) are recorded in a status word that belongs
+ * to the stream the kernel was launched on (per device a fixed table of 64 words; the 64th and later streams of a device
+ * share the last one). This call synchronizes `cuda_stream`, returns that stream's word in *device_status and clears it.
+ * After JA_ERR_TIMEOUT the outputs of the launches since the last call are undefined; the context stays usable and later
+ * launches run normally. */
 ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_status);
+
+/* ---- switches and test hooks (no counterpart in the paper) ---------------------------------------------------------
+ * Every device-side wait of the kernels is bounded (default 2 s; JA_WAIT_CAP=<nanoseconds> in the environment). The
+ * environment (JA_* variables: the wait limit and switches that force a kernel form or a schedule) is read ONCE, when the
+ * library is first used; ja_debug_set changes a value afterwards. Names: "wait_cap_ns", "attn_mma_sync", "attn_one_tile",
+ * "attn_persistent", "attn_section", "attn_variant", "gemm_cta_group", "gemm_group_m", "gemm_heavy_first", "gemm_split",
+ * "gemm_loader", "row_tma", "row_team"; -1 = not forced. JA_ERR_INVALID_ARG for an unknown name or a value out of range. */
+ja_status_t ja_debug_set(const char* name, int64_t value);
+/* Launches one CTA that waits, with the configured limit, on a barrier nothing arrives at: the wait runs out, the kernel
+ * records JA_ERR_TIMEOUT in the stream's status word and returns normally (no trap, no fault). waiters_ok: optional
+ * DEVICE array of two ints, set to 0 / 0 (the waiter whose limit ran out, and a second waiter that gave up on the abort
+ * flag). For tests of the failure path; asynchronous on `cuda_stream`. */
+ja_status_t ja_debug_wait_timeout(void* cuda_stream, int32_t* waiters_ok);
+/* The same wait loop run on the HOST against a scripted barrier and clock (no CUDA call): the barrier completes at poll
+ * `ready_at_poll` (counted from 1; <= 0 never), the clock advances ns_per_poll per poll, another role raises the abort
+ * flag at poll abort_at_poll (<= 0 never). Outputs (any may be NULL): polls made, success, whether this waiter recorded
+ * the time-out, clock at return. */
+ja_status_t ja_debug_bounded_wait_host(int64_t ready_at_poll, int64_t ns_per_poll, int64_t cap_ns, int64_t abort_at_poll,
+                                       int64_t* polls, int32_t* succeeded, int32_t* recorded_timeout, int64_t* elapsed_ns);
 
 /* Number of kernels this library has launched since load (for launch accounting by callers). */
 int64_t ja_launch_count(void);

@@ -71,6 +71,9 @@ def _load() -> ctypes.CDLL:
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
         "ja_repartition_noalloc": [i32, P(i64), P(i32), P(P(i64)), P(i32), P(P(i64)), ctypes.c_int, vp, vp, vp],
+        "ja_debug_set": [ctypes.c_char_p, i64],
+        "ja_debug_wait_timeout": [vp, vp],
+        "ja_debug_bounded_wait_host": [i64, i64, i64, i64, P(i64), P(i32), P(i32), P(i64)],
     }
     for name, argtypes in sigs.items():
         fn = getattr(lib, name)
@@ -301,3 +304,21 @@ def ja_stream_status(stream: int = 0) -> int:
     st = ctypes.c_int()
     _check(LIB.ja_stream_status(ctypes.c_void_p(stream), ctypes.byref(st)))
     return st.value
+
+
+def ja_debug_set(name: str, value: int):
+    """Force a kernel form / schedule, or set the limit of the device-side waits ("wait_cap_ns"); -1 = not forced."""
+    _check(LIB.ja_debug_set(name.encode(), int(value)))
+
+
+def ja_debug_wait_timeout(stream: int = 0, waiters_ok_ptr: int = 0):
+    """Test hook: a one-CTA kernel whose bounded wait runs out (JA_ERR_TIMEOUT lands in the stream's status word)."""
+    _check(LIB.ja_debug_wait_timeout(ctypes.c_void_p(stream), ctypes.c_void_p(waiters_ok_ptr)))
+
+
+def ja_debug_bounded_wait_host(ready_at_poll: int, ns_per_poll: int, cap_ns: int, abort_at_poll: int = 0):
+    """The kernels' wait loop on the host against a scripted barrier and clock: (polls, succeeded, recorded_timeout, ns)."""
+    polls, ok, rec, ns = ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int64()
+    _check(LIB.ja_debug_bounded_wait_host(ready_at_poll, ns_per_poll, cap_ns, abort_at_poll, ctypes.byref(polls), ctypes.byref(ok),
+                                          ctypes.byref(rec), ctypes.byref(ns)))
+    return polls.value, bool(ok.value), bool(rec.value), ns.value

@@ -12,8 +12,10 @@
 #include <iterator>
 #include <cmath>
 #include <mutex>
+#include <set>
 
 #include "ja_internal.h"
+#include "ja_wait.h"
 
 // ---------------------------------------------------------------------------------------------------
 // errors, counters, device status word
@@ -21,7 +23,9 @@
 static thread_local char g_err[512] = "";
 static std::atomic<int64_t> g_launches{0};
 static std::atomic<uint64_t> g_next_id{1};
-__device__ int g_ja_status_word;
+#define JA_STATUS_SLOTS 64
+#define JA_MAX_DEVICES 64
+__device__ int g_ja_status_words[JA_STATUS_SLOTS];
 
 ja_status_t ja_fail(ja_status_t st, const char* fmt, ...) {
     va_list ap;
@@ -37,22 +41,101 @@ ja_status_t ja_cuda_fail(cudaError_t e, const char* what) {
 
 void ja_count_launch(int n) { g_launches += n; }
 
-int* ja_device_status_word() {
-    static int* p = nullptr;
-    if (!p) {
-        if (cudaGetSymbolAddress((void**)&p, g_ja_status_word) != cudaSuccess) p = nullptr;
+// ---- configuration: the environment is read once -------------------------------------------------------------
+static int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return (v && *v) ? atoi(v) : dflt;
+}
+JaConfig& ja_config() {
+    static JaConfig cfg;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        cfg.attn_mma_sync = env_int("JA_ATTN_MMA_SYNC", -1);
+        cfg.attn_one_tile = env_int("JA_ATTN_ONE_TILE", -1);
+        cfg.attn_persistent = env_int("JA_ATTN_PERSISTENT", -1);
+        cfg.attn_section = env_int("JA_ATTN_SECTION", -1);
+        cfg.attn_variant = env_int("JA_ATTN_VARIANT", -1);
+        cfg.gemm_cta_group = env_int("JA_GEMM_CTA_GROUP", -1);
+        cfg.gemm_group_m = env_int("JA_GEMM_GROUP_M", -1);
+        cfg.gemm_heavy_first = env_int("JA_GEMM_HEAVY_FIRST", -1);
+        cfg.gemm_split = env_int("JA_GEMM_SPLIT", -1);
+        cfg.gemm_loader = env_int("JA_GEMM_LOADER", -1);
+        cfg.row_tma = env_int("JA_ROW_TMA", -1);
+        cfg.row_team = env_int("JA_ROW_TEAM", -1);
+        if (const char* v = getenv("JA_WAIT_CAP")) {
+            const long long ns = atoll(v);
+            if (ns >= 1000 && ns <= 4000000000000ll) cfg.wait_cap_us = ns / 1000;
+        }
+    });
+    return cfg;
+}
+
+extern "C" ja_status_t ja_debug_set(const char* name, int64_t value) {
+    if (!name) return ja_fail(JA_ERR_INVALID_ARG, "name is NULL");
+    JaConfig& c = ja_config();
+    const std::string n(name);
+    struct { const char* key; int* field; } ints[] = {
+        {"attn_mma_sync", &c.attn_mma_sync}, {"attn_one_tile", &c.attn_one_tile}, {"attn_persistent", &c.attn_persistent},
+        {"attn_section", &c.attn_section}, {"attn_variant", &c.attn_variant}, {"gemm_cta_group", &c.gemm_cta_group},
+        {"gemm_group_m", &c.gemm_group_m}, {"gemm_heavy_first", &c.gemm_heavy_first}, {"gemm_split", &c.gemm_split},
+        {"gemm_loader", &c.gemm_loader}, {"row_tma", &c.row_tma}, {"row_team", &c.row_team}};
+    for (auto& e : ints)
+        if (n == e.key) {
+            *e.field = (int)value;
+            return JA_OK;
+        }
+    if (n == "wait_cap_ns") {
+        if (value < 1000 || value > 4000000000000ll) return ja_fail(JA_ERR_INVALID_ARG, "wait_cap_ns must lie in [1e3, 4e12]");
+        c.wait_cap_us = value / 1000;
+        return JA_OK;
     }
-    return p;
+    return ja_fail(JA_ERR_INVALID_ARG, "unknown switch '%s'", name);
+}
+
+// ---- per-device state: status words, multiprocessor count ------------------------------------------------------
+struct DeviceState {
+    int* words = nullptr;                    // device address of g_ja_status_words on this device
+    std::map<cudaStream_t, int> slot_of;     // stream -> word
+    int sms = 0;
+};
+static std::mutex g_dev_mu;
+static DeviceState g_dev[JA_MAX_DEVICES];
+
+static DeviceState* device_state_locked() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= JA_MAX_DEVICES) return nullptr;
+    DeviceState* d = &g_dev[dev];
+    if (!d->words && cudaGetSymbolAddress((void**)&d->words, g_ja_status_words) != cudaSuccess) d->words = nullptr;
+    if (!d->sms && (cudaDeviceGetAttribute(&d->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || d->sms < 1)) d->sms = 148;
+    return d;
+}
+
+int* ja_device_status_word(cudaStream_t st) {
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    DeviceState* d = device_state_locked();
+    if (!d || !d->words) return nullptr;
+    auto it = d->slot_of.find(st);
+    if (it == d->slot_of.end()) {
+        const int slot = std::min<int>((int)d->slot_of.size(), JA_STATUS_SLOTS - 1);
+        it = d->slot_of.emplace(st, slot).first;
+    }
+    return d->words + it->second;
+}
+
+int ja_sm_count() {
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    DeviceState* d = device_state_locked();
+    return d ? d->sms : 148;
 }
 
 extern "C" const char* ja_last_error(void) { return g_err; }
-extern "C" const char* ja_version(void) { return "libja 0.1 (sm_100a)"; }
+extern "C" const char* ja_version(void) { return "libja 0.2 (sm_100a)"; }
 extern "C" int64_t ja_launch_count(void) { return g_launches.load(); }
 
 extern "C" ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_status) {
     if (!device_status) return ja_fail(JA_ERR_INVALID_ARG, "device_status is NULL");
     JA_CUDA(cudaStreamSynchronize((cudaStream_t)cuda_stream));
-    int* w = ja_device_status_word();
+    int* w = ja_device_status_word((cudaStream_t)cuda_stream);
     if (!w) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
     int v = 0;
     JA_CUDA(cudaMemcpy(&v, w, sizeof v, cudaMemcpyDeviceToHost));
@@ -62,6 +145,25 @@ extern "C" ja_status_t ja_stream_status(void* cuda_stream, ja_status_t* device_s
         JA_CUDA(cudaMemcpy(w, &zero, sizeof zero, cudaMemcpyHostToDevice));
         ja_attention_reset_queues();
     }
+    return JA_OK;
+}
+
+// ---- the bounded wait, run on the host against a scripted barrier and clock (tests) ------------------------------
+// The barrier completes at poll number `ready_at_poll` (counting from 1; <= 0: never); the clock advances `ns_per_poll`
+// per poll; another role raises the abort flag at poll `abort_at_poll` (<= 0: never). Outputs: polls made, whether the
+// wait succeeded, whether THIS waiter recorded the time-out, and the clock when it returned.
+extern "C" ja_status_t ja_debug_bounded_wait_host(int64_t ready_at_poll, int64_t ns_per_poll, int64_t cap_ns, int64_t abort_at_poll,
+                                                  int64_t* polls, int32_t* succeeded, int32_t* recorded_timeout, int64_t* elapsed_ns) {
+    if (ns_per_poll < 0 || cap_ns < 0) return ja_fail(JA_ERR_INVALID_ARG, "negative time");
+    int64_t n = 0;
+    bool failed = false;
+    const bool ok = ja_bounded_wait([&] { ++n; return ready_at_poll > 0 && n >= ready_at_poll; },
+                                    [&] { return (uint64_t)(n * ns_per_poll); },
+                                    [&] { return abort_at_poll > 0 && n >= abort_at_poll; }, [&] { failed = true; }, (uint64_t)cap_ns);
+    if (polls) *polls = n;
+    if (succeeded) *succeeded = ok ? 1 : 0;
+    if (recorded_timeout) *recorded_timeout = failed ? 1 : 0;
+    if (elapsed_ns) *elapsed_ns = n * ns_per_poll;
     return JA_OK;
 }
 
@@ -153,11 +255,16 @@ extern "C" ja_status_t ja_relation_create(int32_t rank, const int64_t* extents, 
     return JA_OK;
 }
 
+// live specs, so that ja_relation_destroy can drop the launch state cached for a relation that goes away
+static std::mutex g_specs_mu;
+static std::set<ja_spec*> g_specs;
 static void forget_relayout_plans(uint64_t relation_id);
+static void forget_exec_plans(uint64_t relation_id);
 
 extern "C" ja_status_t ja_relation_destroy(ja_relation_t* rel) {
     if (!rel) return JA_OK;
     forget_relayout_plans(rel->id);   // cached copy plans of relayouts from / to this relation (device tables) go with it
+    forget_exec_plans(rel->id);       // and the launch state (tensor maps, rotation tables) of every spec that ran on it
     if (rel->d_tables) cudaFree(rel->d_tables);
     delete rel;
     return JA_OK;
@@ -191,6 +298,8 @@ extern "C" ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* c
 
 // device copy of the key table: [splits of dim 0 | dim 1 | ... | block offsets]
 ja_status_t ja_relation_to_device(const ja_relation* r) {
+    static std::mutex mu;   // two threads may execute on one relation for the first time at once
+    std::lock_guard<std::mutex> lk(mu);
     if (r->on_device) return JA_OK;
     std::vector<int64_t> host;
     for (int d = 0; d < r->rank; ++d) host.insert(host.end(), r->splits[d].begin(), r->splits[d].end());
@@ -386,10 +495,28 @@ extern "C" ja_status_t ja_spec_create(const char* einsum, const ja_index_part_t*
     }
     s->p = (int64_t)s->out_keys.size();
     *out = s.release();
+    {
+        std::lock_guard<std::mutex> lk(g_specs_mu);
+        g_specs.insert(*out);
+    }
     return JA_OK;
 }
 
+
+static void forget_exec_plans(uint64_t relation_id) {
+    std::lock_guard<std::mutex> lk(g_specs_mu);
+    for (ja_spec* s : g_specs) {
+        std::lock_guard<std::mutex> lk2(s->plans_mu);
+        for (auto it = s->plans.begin(); it != s->plans.end();)
+            it = std::find(it->first.begin(), it->first.end(), relation_id) != it->first.end() ? s->plans.erase(it) : std::next(it);
+    }
+}
+
 extern "C" ja_status_t ja_spec_destroy(ja_spec_t* spec) {
+    if (spec) {
+        std::lock_guard<std::mutex> lk(g_specs_mu);
+        g_specs.erase(spec);
+    }
     delete spec;
     return JA_OK;
 }
@@ -706,6 +833,7 @@ extern "C" ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_
 struct ExecPlan {
     std::shared_ptr<GemmTcPlan> gemm;
     bool gemm_checked = false;
+    AttnTcCache attn;
     float2* rope_table = nullptr;
     int64_t* rope_splits = nullptr;  // split points of the collapsed (h d) index
     ~ExecPlan() {
@@ -778,8 +906,9 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
     std::vector<uint64_t> key;
     for (int k = 0; k < n_in; ++k) key.push_back(inputs[k]->id);
     key.push_back(out->id);
-    std::shared_ptr<ExecPlan>& plan = spec->plans[key];
-    if (!plan) plan.reset(new ExecPlan());
+    std::lock_guard<std::mutex> plans_lock(spec->plans_mu);   // held to the end: plan building and the launch that uses the plan
+    std::shared_ptr<ExecPlan> plan = spec->plans[key];
+    if (!plan) spec->plans[key] = plan = std::make_shared<ExecPlan>();
 
     for (int k = 0; k < n_in; ++k)
         if ((st = ja_relation_to_device(inputs[k])) != JA_OK) return st;
@@ -956,6 +1085,7 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         if (Q->extent[1] != K->extent[1]) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs equal query and key extents");
         AttnArgs aa;
         memset(&aa, 0, sizeof aa);
+        aa.cache = &plan->attn;
         aa.q = ja_view(Q); aa.k = ja_view(K); aa.v = ja_view(V); aa.o = ja_view(out);
         if (n_outputs == 2) {   // second output: lse[b, q, h], f32, tiled like the (b, q, h) indices of the output
             ja_relation* L = outputs[1];
@@ -1047,8 +1177,9 @@ extern "C" ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_
         const ja_relation *A = inputs[0], *B = inputs[1];
         if (A->dtype != B->dtype) return ja_fail(JA_ERR_DTYPE, "matmul operands must share one dtype");
         std::vector<uint64_t> key = {A->id, B->id, partials->id, ~(uint64_t)0};
-        std::shared_ptr<ExecPlan>& plan = spec->plans[key];
-        if (!plan) plan.reset(new ExecPlan());
+        std::lock_guard<std::mutex> plans_lock(spec->plans_mu);
+        std::shared_ptr<ExecPlan> plan = spec->plans[key];
+        if (!plan) spec->plans[key] = plan = std::make_shared<ExecPlan>();
         if (A->dtype == JA_BF16) {
             if (!plan->gemm_checked) {
                 bool ok = false;

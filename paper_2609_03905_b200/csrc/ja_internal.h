@@ -6,6 +6,7 @@
 
 #include <map>
 #include <memory>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -64,6 +65,9 @@ struct ja_spec {
     int64_t p = 0;
     std::vector<int32_t> in_keys;   // [p][n_in]
     std::vector<int32_t> out_keys;  // [p]
+    // launch state cached per tuple of relation ids; guarded by plans_mu (ja_execute may be called from several threads
+    // on one spec); entries that name a destroyed relation are dropped by ja_relation_destroy
+    mutable std::mutex plans_mu;
     mutable std::map<std::vector<uint64_t>, std::shared_ptr<ExecPlan>> plans;
 };
 
@@ -72,8 +76,30 @@ ja_status_t ja_fail(ja_status_t st, const char* fmt, ...);
 ja_status_t ja_cuda_fail(cudaError_t e, const char* what);
 ja_status_t ja_relation_to_device(const ja_relation* r);
 RelView ja_view(const ja_relation* r);
-int* ja_device_status_word();
+// The status word of (current device, stream): a fixed table of words per device, one per stream seen so far (the 64th and
+// later streams of a device share the last word). nullptr when the table's address cannot be resolved.
+int* ja_device_status_word(cudaStream_t st);
 void ja_count_launch(int n = 1);
+int ja_sm_count();   // multiprocessors of the current device (cached per device)
+
+// Switches that force a kernel form or a schedule. Read ONCE from the environment (JA_* variables) when the library is
+// first used; afterwards only ja_debug_set changes them (tests, A/B measurements). -1 = not forced.
+struct JaConfig {
+    int attn_mma_sync = -1;     // JA_ATTN_MMA_SYNC     1: the mma.sync attention kernel
+    int attn_one_tile = -1;     // JA_ATTN_ONE_TILE     1: one query tile per CTA
+    int attn_persistent = -1;   // JA_ATTN_PERSISTENT   0 / 1: work items drawn from a counter by one CTA per SM
+    int attn_section = -1;      // JA_ATTN_SECTION      n: launch-order sections of n (batch, head) pairs
+    int attn_variant = -1;      // JA_ATTN_VARIANT      row-thread variant of the two-tile kernel (see k_attention_tc.cu)
+    int gemm_cta_group = -1;    // JA_GEMM_CTA_GROUP    1: no two-CTA pairs
+    int gemm_group_m = -1;      // JA_GEMM_GROUP_M      n: row tiles per rasterisation band
+    int gemm_heavy_first = -1;  // JA_GEMM_HEAVY_FIRST  0: plain tile order
+    int gemm_split = -1;        // JA_GEMM_SPLIT        0: the last partial wave is not split along the contracted index
+    int gemm_loader = -1;       // JA_GEMM_LOADER       1: operands staged by plain loads even where TMA could take them
+    int row_tma = -1;           // JA_ROW_TMA           0: row join-aggs without the TMA-staged kernel
+    int row_team = -1;          // JA_ROW_TEAM          n: threads per row of the plain row kernel
+    int64_t wait_cap_us = 2000000;   // JA_WAIT_CAP (nanoseconds in the environment): limit of every device-side wait
+};
+JaConfig& ja_config();
 
 #define JA_CUDA(call)                                              \
     do {                                                           \
@@ -140,7 +166,13 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
 ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st);
 
 // Attention join-agg (QK^T join, online-softmax aggregation, PV).
+// the four tensor maps (Q, K, V, O) of the tensor-memory kernels, encoded once per (spec, relations) tuple
+struct AttnTcCache {
+    alignas(64) unsigned char maps[4][128];
+    bool valid = false;
+};
 struct AttnArgs {
+    AttnTcCache* cache;    // where the tensor maps are kept between launches, or nullptr
     RelView q, k, v, o;
     RelView lse;           // optional second output [b, q, h] f32: log of the softmax denominator; base == nullptr if absent
     bool lse_rows_layout;  // lse blocks follow the closed-form order of q's (b, s, h) blocks (tensor-memory kernels)

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "ja_internal.h"
+#include "ja_wait.h"
 
 namespace ja_ptx {
 
@@ -41,21 +42,24 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after ~2 s, records the failure and raises the CTA-wide abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63) == 63) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > 2000000000ull) {
-                *abort_flag = 1;
-                atomicExch(status, (int)JA_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
+// Bounded wait on an mbarrier phase. `ctl` points at two words of shared memory that the CTA sets up before its first
+// wait: ctl[0] = the CTA-wide abort flag, ctl[1] = the wait limit in microseconds (a kernel parameter: JA_WAIT_CAP of the
+// host configuration, 2 s by default). When the limit runs out the thread records JA_ERR_TIMEOUT in the stream's status
+// word, raises the abort flag so that every other role of the CTA gives up at its next check, and returns false; the
+// caller leaves through the kernel's normal exit. The loop itself is ja_bounded_wait (ja_wait.h), which is also
+// compiled for the host and tested there against a scripted barrier and clock.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
+    return ja_bounded_wait([&] { return mbar_try_wait(bar, parity); }, [] { return global_ns(); }, [&] { return ctl[0] != 0; },
+                           [&] {
+                               ctl[0] = 1;
+                               atomicExch(status, (int)JA_ERR_TIMEOUT);
+                           },
+                           (uint64_t)(uint32_t)ctl[1] * 1000ull);
+}
+// what a CTA's first thread writes into the two control words before any wait
+__device__ __forceinline__ void wait_ctl_init(volatile int* ctl, uint32_t cap_us) {
+    ctl[0] = 0;
+    ctl[1] = (int)cap_us;
 }
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {

@@ -261,15 +261,14 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
 }  // namespace
 
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
-    const char* legacy = getenv("JA_ATTN_MMA_SYNC");
-    if (!(legacy && legacy[0] == '1')) {
+    if (ja_config().attn_mma_sync != 1) {
         bool launched = false;
         ja_status_t s = ja_launch_attention_tc(a, st, &launched);
         if (s != JA_OK || launched) return s;
     }
     const int QT = (a.align % 128 == 0) ? 128 : 64;
     AttnArgs a2 = a;
-    a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (148 + a.S / QT - 1) / (a.S / QT)));
+    a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (ja_sm_count() + a.S / QT - 1) / (a.S / QT)));
     dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
     if (QT == 128) {

@@ -1,7 +1,9 @@
 // Attention join-agg "bqhd,bkhd,bkhd->bqhd" (f = ATTENTION, (+) = online softmax) on the 5th-generation
 // tensor cores: both contractions of every joined tuple run as tcgen05.mma with accumulators in tensor memory.
 //
-// One CTA owns one output key tile (128 query rows of one (batch, head)) and walks the function specs that
+// Two kernels. attention_tc2_kernel (further down) gives a CTA two output key tiles of one (batch, head) and is the one
+// that runs whenever sequences are whole pairs of 128-row tiles; attention_tc_kernel, described here, takes the rest:
+// one CTA owns one output key tile (128 query rows of one (batch, head)) and walks the function specs that
 // share that output key -- the 128-row key/value tiles that survive the causal band predicate -- ascending.
 //
 //   warp 0      TMA producer: Q once, then K_j and V_j (two stages each), straight from the "bshd" block-key
@@ -54,7 +56,8 @@ struct SeqGeom {
 struct AttnTcParams {
     char* o_base;
     float* lse_base;             // optional second output (nullptr if absent), addressed like o without the last index
-    int32_t* status;
+    int32_t* status;             // status word of the launching stream
+    uint32_t wait_cap_us;        // limit of every bounded wait
     int32_t B, S, H;
     int32_t group;               // query heads per key/value head
     int32_t causal;
@@ -196,7 +199,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const bool row_threads_arrive = (i >= P_FULL && i < P_FULL + 2) || (i >= O_EMPTY && i < O_EMPTY + 2);
             mbar_init(bar(i), row_threads_arrive ? 4 : 1);   // one arrival per row warp, else one commit / expect_tx
         }
-        *abort_flag = 0;
+        wait_ctl_init(abort_flag, p.wait_cap_us);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -436,21 +439,52 @@ __device__ __forceinline__ float row_max128(const uint32_t (&v)[128], int kmax) 
     return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// P = 2^(S*scale - m) as packed bf16 written over S in tensor memory; returns the row sum
-template <bool MASK>
-__device__ __forceinline__ float row_exp_store128(const uint32_t (&v)[128], int kmax, float scale, float m_used, uint32_t t_dst) {
+// 2^x for a pair of exponents on the FMA pipe (no special-function unit): x = n + f with n = round(x), f in [-1/2, 1/2];
+// 2^f by a cubic fitted to a relative error of 7.5e-5 (bf16 keeps 8 bits of P); n is added to the exponent field. x is
+// clamped at -126 so that the exponent field cannot wrap; scores above the offset by more than 2^8 never reach here (lazy
+// rescale keeps x <= 8).
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x0 = fmaxf(x0, -126.f);
+    x1 = fmaxf(x1, -126.f);
+    const uint64_t x = pack2(x0, x1);
+    const uint64_t magic = pack2(12582912.f, 12582912.f);        // 1.5 * 2^23: adding it rounds x to an integer in the low mantissa bits
+    const uint64_t t = add2(x, magic);
+    const uint64_t n = add2(t, pack2(-12582912.f, -12582912.f));
+    const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
+    uint64_t r = fma2(pack2(0.05517162f, 0.05517162f), f, pack2(0.24261113f, 0.24261113f));
+    r = fma2(r, f, pack2(0.69326097f, 0.69326097f));
+    r = fma2(r, f, pack2(0.99992806f, 0.99992806f));
+    float r0, r1, t0, t1;
+    unpack2(r, r0, r1);
+    unpack2(t, t0, t1);
+    p0 = __int_as_float(__float_as_int(r0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(r1) + (__float_as_int(t1) << 23));
+}
+
+// One row of P = 2^(S * scale - m) for 128 keys as 64 packed bf16 pairs in registers; returns the row sum (f32, of the
+// unrounded values). MASK: keys > kmax lie after the query row and get P = 0. POLY: how many of the four pairs of every
+// group of eight keys take the FMA-pipe exponential instead of ex2 (0, 1 or 2), interleaved so that both pipes stay busy.
+template <bool MASK, int POLY>
+__device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], int kmax, float scale, float m_used, uint32_t (&pk)[64]) {
     const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
     uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint32_t pk[8];
+    for (int cc = 0; cc < 16; ++cc) {
 #pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-            const int col = c * 16 + i;
+        for (int i = 0; i < 8; i += 2) {
+            const int col = cc * 8 + i;
+            const uint64_t x2 = fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2);
             float p0, p1;
-            unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
-            p0 = ex2(p0);
-            p1 = ex2(p1);
+            const bool poly = (POLY == 1 && i == 6) || (POLY == 2 && (i == 2 || i == 6));
+            if (poly) {
+                exp2_poly_pair(x2, p0, p1);
+            } else {
+                unpack2(x2, p0, p1);
+                p0 = ex2(p0);
+                p1 = ex2(p1);
+            }
             if (MASK) {
                 if (col > kmax) p0 = 0.f;
                 if (col + 1 > kmax) p1 = 0.f;
@@ -458,53 +492,9 @@ __device__ __forceinline__ float row_exp_store128(const uint32_t (&v)[128], int 
             if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
             else sum_b = add2(sum_b, pack2(p0, p1));
             __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
-            pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
+            pk[col / 2] = *reinterpret_cast<uint32_t*>(&tt);
         }
-        tmem_st8(t_dst + c * 8, pk);
     }
-    float a0, a1, b0, b1;
-    unpack2(sum_a, a0, a1);
-    unpack2(sum_b, b0, b1);
-    return (a0 + a1) + (b0 + b1);
-}
-
-// One half (64 keys) of P = 2^(S*scale - m) written as packed bf16 over S; returns the half's row sum. HALF 0 also returns the
-// maximum of all 128 raw scores, computed alongside (two max3 per pair of exponentials).
-template <int HALF>
-__device__ __forceinline__ float row_exp_store_half(const uint32_t (&v)[128], float scale, float m_used, uint32_t t_dst, float& mx_out) {
-    const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
-    uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
-    float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]), m2 = __uint_as_float(v[2]), m3 = __uint_as_float(v[3]);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t pk[8];
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-            const int col = HALF * 64 + c * 16 + i;
-            float p0, p1;
-            unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
-            p0 = ex2(p0);
-            p1 = ex2(p1);
-            if (HALF == 0) {   // pair number q = (c*16+i)/2 in 0..31 covers scores 4q .. 4q+3 (scores 0..3 seed the four maxima)
-                const int q4 = (c * 16 + i) * 2;
-                if (q4 >= 4) {
-                    if (i & 2) {
-                        m2 = max3(m2, __uint_as_float(v[q4]), __uint_as_float(v[q4 + 1]));
-                        m3 = max3(m3, __uint_as_float(v[q4 + 2]), __uint_as_float(v[q4 + 3]));
-                    } else {
-                        m0 = max3(m0, __uint_as_float(v[q4]), __uint_as_float(v[q4 + 1]));
-                        m1 = max3(m1, __uint_as_float(v[q4 + 2]), __uint_as_float(v[q4 + 3]));
-                    }
-                }
-            }
-            if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
-            else sum_b = add2(sum_b, pack2(p0, p1));
-            __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
-            pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
-        }
-        tmem_st8(t_dst + HALF * 32 + c * 8, pk);
-    }
-    if (HALF == 0) mx_out = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     float a0, a1, b0, b1;
     unpack2(sum_a, a0, a1);
     unpack2(sum_b, b0, b1);
@@ -512,595 +502,38 @@ __device__ __forceinline__ float row_exp_store_half(const uint32_t (&v)[128], fl
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Two query tiles per CTA. The CTA owns 256 query rows of one (batch, head) as two independent 128-row output
-// key tiles A and B that share every K_j / V_j tile it loads. While the row threads of one tile exponentiate,
-// the tensor pipe works on the other tile, and each scheduler holds two row warps.
-//   TMEM: S/P of A at 0, S/P of B at 128, O~ of A at 256, O~ of B at 384 (fp32, 128 columns each).
-//   O~ is ACCUMULATED IN TENSOR MEMORY by the P V products (accumulate flag), not in registers. The running
-//   maximum used as the exponent offset is only raised when a row's new maximum exceeds it by more than 2^8
-//   (P stays <= 256, exact in the final O~/l); only then is the row's O~ rescaled in TMEM by its row thread.
-//   Past the first key tile the row threads exponentiate against the offset in use WHILE they reduce the tile's
-//   maximum (the max3 instructions run in the shadow of the ex2 pipe) and hand the first 64 keys of P to the tensor
-//   pipe before they start on the other 64; a warp in which some row outgrew its offset redoes the tile.
-//   warp 0 TMA (K / V tiles through one ring of five slots), warp 1 MMA issuer, warps 2..5 rows of A, 6..9 rows of B.
-//   The MMA warp runs its loop converged, one elected lane issuing: addresses and descriptors are then warp-uniform
-//   values, and the steady state is straight-line code (measured on this part: a branch between two tcgen05.mma
-//   instructions, or operands that have to be moved to uniform registers first, cost the issuing thread ~40 cycles
-//   per instruction, against 64 cycles of tensor-pipe time for M128 N128 K16).
+// Two query tiles per CTA. The CTA owns 256 query rows of one (batch, head) as two independent 128-row output key tiles
+// A and B that share every K_j / V_j tile it loads; while the row threads of one tile exponentiate, the tensor pipe works
+// on the other tile, and each scheduler holds two row warps.
+//   warp 0 TMA producer, warp 1 MMA issuer (runs converged, one elected lane issues; the steady state is straight-line
+//   code: a branch or a move to uniform registers between two tcgen05.mma costs the issuing thread ~40 cycles against
+//   64 cycles of tensor-pipe time for M128 N128 K16), warps 2..5 rows of A, warps 6..9 rows of B (one thread per row).
+//   TMEM: S of A at 0, S of B at 128, O~ of A at 256, O~ of B at 384 (fp32, 128 columns each). O~ is ACCUMULATED IN TENSOR
+//   MEMORY by the P V products. The running maximum used as the exponent offset is only raised when a row's new maximum
+//   exceeds it by more than 2^8 (P stays <= 256, exact in the final O~/l); only then is the row's O~ rescaled in place.
+//   P goes to the P V product through SHARED memory (a 128-byte-swizzled K-major tile, the layout TMA gives Q): the row
+//   threads copy S into registers and release the S columns at once, so the next Q K^T of the tile runs WHILE they
+//   exponentiate.
+//   Shared memory: Q_A, Q_B, P_A, P_B and THREE K / V slots that K_0, K_1, V_0, K_2, V_1, ... pass through in the order
+//   the products consume them (7 tiles = 224 KiB). O leaves through the tile's P buffer and two TMA stores.
+// PERSIST: one CTA per SM takes work items (one item = the pair of tiles of one (batch, head)), heaviest first, from a
+//   counter in global memory: the producer thread claims the next item and hands its number to the other roles through a
+//   two-entry queue in shared memory, and runs ahead into the next item as soon as the Q buffers are free, so the next
+//   item's Q and first K tile load, and its first Q K^T run, while the row threads finish this item. Barrier phases follow
+//   running counters (items; key steps per tile). Otherwise one CTA per item, handed out by the hardware in grid order.
+// VAR selects row-thread variants that were built, verified against the oracle and measured slower on this part (kept
+//   selectable for A/B runs, "attn_variant"): bits 0-1 = POLY of row_exp_pack128 (a quarter or half of the exponentials on
+//   the FMA pipe: +1 % / +8 % time on B4 S2048 causal); bit 2 = exponentiate into registers first and wait for the P tile
+//   only before storing (+3 %). 0 = the default. Timing-only ablations of this kernel (B4 S2048 H32 causal, 0.163 ms on the
+//   box of that run): no P stores -6 %, no exponentials -7 %, QK^T or P V reduced to one instruction of eight -6 % / 0 %,
+//   no K / V loads -10 %, no output stage -3 %; all of them together still leave 0.067 ms: the row threads' own
+//   instruction stream (two row warps per scheduler, ~420 instructions per row and key tile, issued in order) and the
+//   barrier hand-offs between the roles bound the kernel, not one of the units.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int NUM_THREADS2 = 320;
-constexpr int KV_RING = 5;                                  // K / V tiles in shared memory: two in use, three in flight
-constexpr int SMEM_BYTES2 = (2 + KV_RING) * TILE_BYTES + 1024 + 256;   // Q_A, Q_B, ring of K / V tiles
+constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
 
-__global__ void __launch_bounds__(NUM_THREADS2, 1)
-attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                     const __grid_constant__ AttnTcParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t sQ = base, sKV = base + 2 * TILE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + KV_RING) * TILE_BYTES);
-    const uint32_t bar0 = smem_u32(bars);
-    // K / V tiles go through one ring in the order K_0 V_0 K_1 V_1 ...: tile number 2j is K_j, 2j+1 is V_j
-    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 1 + KV_RING, S_FULL = 1 + 2 * KV_RING, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4, P_HALF = S_FULL + 6, O_STAGED = S_FULL + 8, NBAR = S_FULL + 10 };
-    auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;   // warp-uniform by construction
-    const int n_pairs = p.S / (2 * QT);
-    int slot, bh;
-    ja_attn_decode_cta((int)blockIdx.x, n_pairs, p.H * p.B, p.sect, &slot, &bh);
-    const int pr = p.n_order ? (int)p.order[slot] : n_pairs - 1 - slot;   // heaviest output keys first
-    const int h = bh % p.H, b = bh / p.H;
-    const int q0 = pr * 2 * QT;                       // first row of tile A; tile B starts at q0 + 128
-    int s0, s1;                                       // both tiles lie in one packed sequence (ends are multiples of 256)
-    sequence_of(p, q0, s0, s1);
-    const int n_steps_a = p.causal ? (q0 + QT - s0) / KT : (s1 - s0) / KT;
-    const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < NBAR; ++i) mbar_init(bar(i), ((i >= P_FULL && i < P_FULL + 2) || (i >= P_HALF && i < P_HALF + 2) || i >= O_STAGED) ? 4 : 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
-
-    if (warp == 0) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            const int hk = h / p.group;
-            mbar_expect_tx(bar(Q_FULL), 2 * TILE_BYTES);
-            for (int t = 0; t < 2; ++t) {
-                const int qrow_t = seq_row(p.q, p.S, b, q0 + t * QT, h);
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow_t);
-            }
-            int sl = 0;
-            uint32_t ph = 0;
-            for (int li = 0; li < 2 * n_steps_b; ++li) {
-                const int krow = seq_row(p.k, p.S, b, s0 + (li >> 1) * KT, hk);
-                if (!mbar_wait(bar(KV_EMPTY + sl), ph ^ 1, abort_flag, p.status)) break;
-                mbar_expect_tx(bar(KV_FULL + sl), TILE_BYTES);
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sKV + sl * TILE_BYTES + half * HALF_BYTES, (li & 1) ? &tmV : &tmK, bar(KV_FULL + sl), half * 64, hk % p.k.hblk, krow);
-                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
-            }
-        }
-    } else if (warp == 1) {
-        // ================= MMA issuer: the whole warp runs the loop, one elected lane issues =================
-        {
-            const uint32_t leader = elect_one();
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
-            const uint32_t idesc_pv = idesc_qk | (1u << 16);
-            auto issue_qk = [&](int t, int ksl) {        // S_t = Q_t K^T with the K tile in ring slot ksl
-                const uint32_t kaddr = sKV + ksl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma_ss_w(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
-                }
-                commit1_w(bar(S_FULL + t), leader);
-            };
-            // O~_t (+)= P_t V_j with V_j in ring slot vsl, in two halves of 64 keys: the row threads release the first half of
-            // P while they still exponentiate the second
-            auto issue_pv = [&](int t, int j, int vsl) -> bool {
-                const uint32_t vaddr = sKV + vsl * TILE_BYTES;
-                if (!mbar_wait(bar(P_HALF + t), (uint32_t)j & 1, abort_flag, p.status)) return false;
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    umma_ts_w(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
-                              (j > 0 || kk > 0) ? 1u : 0u, leader);
-                if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) return false;
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 4; kk < 8; ++kk)
-                    umma_ts_w(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8, desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv, 1u, leader);
-                commit1_w(bar(O_FULL + t), leader);
-                return true;
-            };
-            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
-            if (ok) ok = mbar_wait(bar(KV_FULL + 0), 0, abort_flag, p.status);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(0, 0);
-                issue_qk(1, 0);
-                commit1_w(bar(KV_EMPTY + 0), leader);               // K_0 consumed
-            }
-            int sl = 1;                                   // ring slot and phase of tile number 2j+1 = V_j
-            uint32_t ph = 0;
-            int j = 0;
-            // steady state: both tiles do P V_j and Q K_{j+1}^T. Straight-line body: every branch between two tcgen05.mma
-            // instructions costs the issuing warp tens of cycles in which the tensor pipe drains.
-            const int n_common = min(n_steps_a, n_steps_b) - 1;
-            for (; j < n_common && ok; ++j) {
-                const int vsl = sl;
-                const uint32_t vph = ph;
-                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
-                const int ksl = sl;
-                const uint32_t kph = ph;
-                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
-                ok = mbar_wait(bar(KV_FULL + vsl), vph, abort_flag, p.status) && mbar_wait(bar(KV_FULL + ksl), kph, abort_flag, p.status) &&
-                     issue_pv(0, j, vsl);
-                if (!ok) break;
-                issue_qk(0, ksl);
-                ok = issue_pv(1, j, vsl);
-                if (!ok) break;
-                issue_qk(1, ksl);
-                commit1_w(bar(KV_EMPTY + vsl), leader);
-                commit1_w(bar(KV_EMPTY + ksl), leader);
-            }
-            for (; j < n_steps_b && ok; ++j) {            // the last steps: a tile may have run out of key tiles
-                const bool more = j + 1 < n_steps_b;
-                const int vsl = sl;
-                if (!mbar_wait(bar(KV_FULL + vsl), ph, abort_flag, p.status)) { ok = false; break; }
-                if (++sl == KV_RING) { sl = 0; ph ^= 1; }
-                const int ksl = sl;                       // tile number 2j+2 = K_{j+1}
-                if (more) {
-                    if (!mbar_wait(bar(KV_FULL + ksl), ph, abort_flag, p.status)) { ok = false; break; }
-                    if (++sl == KV_RING) { sl = 0; ph ^= 1; }
-                }
-                for (int t = 0; t < 2 && ok; ++t) {
-                    const int n_t = t == 0 ? n_steps_a : n_steps_b;
-                    if (j < n_t && !issue_pv(t, j, vsl)) { ok = false; break; }
-                    if (j + 1 < n_t) issue_qk(t, ksl);     // ordered behind P V of this tile on the tensor pipe
-                }
-                if (!ok) break;
-                commit1_w(bar(KV_EMPTY + vsl), leader);             // V_j consumed by both tiles
-                // K_{j+1} consumed by the QK products issued above (both tiles, or tile B alone on its last step)
-                if (more) commit1_w(bar(KV_EMPTY + ksl), leader);
-            }
-        }
-    } else {
-        // ================= row threads =================
-        const int t = (warp - 2) >> 2;               // tile: 0 = A, 1 = B
-        const int q = warp & 3;                      // TMEM lane group of this warp (warps 2..5 -> 2,3,0,1; 6..9 -> 2,3,0,1)
-        const int r = q * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        const uint32_t tS = tmem_base + t * 128 + lane_addr, tO = tmem_base + 256 + t * 128 + lane_addr;
-        const int n_t = t == 0 ? n_steps_a : n_steps_b;
-        const int qrow = q0 + t * QT + r;            // sequence position of this row
-        float m_used = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_t && ok; ++j) {
-            if (!mbar_wait(bar(S_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const bool diag = p.causal && (j == n_t - 1);
-            const int kmax = qrow - (s0 + j * KT);
-            uint32_t v[128];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
-            tmem_ld_wait();
-            if (j > 0 && !diag) {
-                // Speculative step: exponentiate against the offset in use while the row maximum of this tile is still being
-                // computed (the max3 instructions run in the shadow of the ex2 pipe). The first 64 keys of P are released to
-                // the tensor pipe as soon as they are stored, unless some row of the warp outgrew its offset (below).
-                float mx;
-                const float sum0 = row_exp_store_half<0>(v, p.scale_log2e, m_used, tS, mx);
-                const bool need = mx * p.scale_log2e > m_used + 8.f;
-                if (!__any_sync(0xffffffffu, need)) {
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(P_HALF + t));
-                    float unused;
-                    l_run += sum0 + row_exp_store_half<1>(v, p.scale_log2e, m_used, tS, unused);
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(P_FULL + t));
-                    continue;
-                }
-                // rare: redo the whole tile with the raised offset (the general path below; S is still in registers)
-            }
-            const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
-            const float m_new = mx * p.scale_log2e;       // finite: the first key of the sequence is never masked
-            // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
-            float alpha = 1.f;
-            bool need = false;
-            if (j == 0) m_used = m_new;
-            else if (m_new > m_used + 8.f) { alpha = ex2(m_used - m_new); m_used = m_new; need = true; }
-            if (__any_sync(0xffffffffu, need)) {
-                // O~ of this tile holds the products up to step j-1: wait for them, then scale this row in place
-                if (!mbar_wait(bar(O_FULL + t), (uint32_t)(j - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < 16; ++c) {   // rare path: small chunks keep the register footprint of the hot path low
-                    uint32_t o[8];
-                    tmem_ld8(tO + c * 8, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st8(tO + c * 8, o);
-                }
-                tmem_st_wait();
-                l_run *= alpha;
-            }
-            const float sum = diag ? row_exp_store128<true>(v, kmax, p.scale_log2e, m_used, tS)
-                                   : row_exp_store128<false>(v, kmax, p.scale_log2e, m_used, tS);
-            l_run += sum;
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(P_HALF + t));
-                mbar_arrive(bar(P_FULL + t));
-            }
-        }
-        if (ok && n_t > 0) {
-            // O = O~ / l goes out through the tile's Q buffer (dead since the tile's last Q K^T): every row thread writes its
-            // 256 bytes in the swizzled layout of the tensor map, and one thread hands the tile to two TMA stores
-            if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
-                tc_fence_after();
-                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                if (p.lse_base) {
-                    const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
-                    p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
-                }
-                uint8_t* orow = smem + t * TILE_BYTES + r * 128;
-                const int sw = r & 7;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4 ov;
-                        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
-                        const int cc = c * 4 + g;                      // 16-byte chunk 0..15 of the row
-                        *reinterpret_cast<uint4*>(orow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) = ov;
-                    }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(O_STAGED + t));
-                if (q == 0 && lane == 0 && mbar_wait(bar(O_STAGED + t), 0, abort_flag, p.status)) {
-                    const int orow0 = seq_row(p.q, p.S, b, q0 + t * QT, h);
-                    for (int half = 0; half < 2; ++half)
-                        tma_store_3d(&tmO, sQ + t * TILE_BYTES + half * HALF_BYTES, half * 64, h % p.q.hblk, orow0);
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
-                }
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------------
-// Two query tiles per CTA with P handed to the P V product through SHARED memory. In the kernel above P overwrites S in
-// tensor memory, so the next Q K^T of a tile cannot start before its P V has read P: per tile the row softmax and the two
-// contractions form one serial chain, and the tensor pipe waits for the row threads about a third of the time. Here the
-// row threads copy S into registers and release the S columns at once, the next Q K^T of the tile runs WHILE they
-// exponentiate, and P goes to a 128-byte-swizzled K-major tile in shared memory (the layout TMA gives Q), read by the P V
-// product as a shared-memory A operand. Shared memory: Q_A, Q_B, P_A, P_B and THREE K / V slots that K_0, K_1, V_0, K_2,
-// V_1, ... pass through in the order the products consume them (7 tiles = 224 KiB).
-// ---------------------------------------------------------------------------------------------------------
-constexpr int SMEM_BYTES3 = 7 * TILE_BYTES + 1024 + 256;
-
-__global__ void __launch_bounds__(NUM_THREADS2, 1)
-attention_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                     const __grid_constant__ AttnTcParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t sQ = base, sKV = base + 2 * TILE_BYTES, sP = base + 5 * TILE_BYTES;
-    uint8_t* pP = smem + 5 * TILE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 7 * TILE_BYTES);
-    const uint32_t bar0 = smem_u32(bars);
-    enum { Q_FULL = 0, KV_FULL = 1, KV_EMPTY = 4, S_FULL = 7, S_FREE = 9, P_FULL = 11, P_EMPTY = 13, O_FULL = 15, O_STAGED = 17, NBAR = 19 };
-    auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-    const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
-    const int n_pairs = p.S / (2 * QT);
-    int slot, bh;
-    ja_attn_decode_cta((int)blockIdx.x, n_pairs, p.H * p.B, p.sect, &slot, &bh);
-    const int pr = p.n_order ? (int)p.order[slot] : n_pairs - 1 - slot;
-    const int h = bh % p.H, b = bh / p.H;
-    const int q0 = pr * 2 * QT;
-    int s0, s1;
-    sequence_of(p, q0, s0, s1);
-    const int n_steps_a = p.causal ? (q0 + QT - s0) / KT : (s1 - s0) / KT;
-    const int n_steps_b = p.causal ? (q0 + 2 * QT - s0) / KT : (s1 - s0) / KT;
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < NBAR; ++i) {
-            const bool row_warps_arrive = (i >= S_FREE && i < S_FREE + 2) || (i >= P_FULL && i < P_FULL + 2) || i >= O_STAGED;
-            mbar_init(bar(i), row_warps_arrive ? 4 : 1);
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
-
-    // K / V tiles in the order the products consume them: K_0, then for every step j: K_{j+1} (if any), V_j
-    // load index li -> slot li % 3, phase (li / 3) & 1
-    if (warp == 0) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            const int hk = h / p.group;
-            mbar_expect_tx(bar(Q_FULL), 2 * TILE_BYTES);
-            for (int t = 0; t < 2; ++t) {
-                const int qrow_t = seq_row(p.q, p.S, b, q0 + t * QT, h);
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, h % p.q.hblk, qrow_t);
-            }
-            bool ok = true;
-            int li = 0;
-            auto load = [&](const CUtensorMap* tm, int j) {
-                const int sl = li % 3;
-                const uint32_t ph = (uint32_t)(li / 3) & 1;
-                if (!mbar_wait(bar(KV_EMPTY + sl), ph ^ 1, abort_flag, p.status)) { ok = false; return; }
-                const int krow = seq_row(p.k, p.S, b, s0 + j * KT, hk);
-                mbar_expect_tx(bar(KV_FULL + sl), TILE_BYTES);
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(sKV + sl * TILE_BYTES + half * HALF_BYTES, tm, bar(KV_FULL + sl), half * 64, hk % p.k.hblk, krow);
-                ++li;
-            };
-            load(&tmK, 0);
-            for (int j = 0; j < n_steps_b && ok; ++j) {
-                if (j + 1 < n_steps_b) load(&tmK, j + 1);
-                if (ok) load(&tmV, j);
-            }
-        }
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
-        {
-            const uint32_t leader = elect_one();
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
-            const uint32_t idesc_pv = idesc_qk | (1u << 16);
-            auto issue_qk = [&](int t, int sl) {          // S_t = Q_t K^T, K in slot sl
-                const uint32_t kaddr = sKV + sl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma_ss_w(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
-                }
-                commit1_w(bar(S_FULL + t), leader);
-            };
-            auto issue_pv = [&](int t, int sl, bool first) {   // O~_t (+)= P_t V, P in shared memory (K-major), V in slot sl (MN-major)
-                const uint32_t vaddr = sKV + sl * TILE_BYTES, paddr = sP + t * TILE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma_ss_w(tmem_base + 256 + t * 128, desc_sw128(paddr + off, 16), desc_sw128(vaddr + kk * 2048, HALF_BYTES), idesc_pv,
-                              (!first || kk > 0) ? 1u : 0u, leader);
-                }
-                commit1_w(bar(P_EMPTY + t), leader);
-                commit1_w(bar(O_FULL + t), leader);
-            };
-            int li = 0;
-            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag, p.status);
-            if (ok) ok = mbar_wait(bar(KV_FULL + 0), 0, abort_flag, p.status);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(0, 0);
-                issue_qk(1, 0);
-                commit1_w(bar(KV_EMPTY + 0), leader);
-                li = 1;
-            }
-            for (int j = 0; j < n_steps_b && ok; ++j) {
-                if (j + 1 < n_steps_b) {
-                    const int sl = li % 3;
-                    if (!mbar_wait(bar(KV_FULL + sl), (uint32_t)(li / 3) & 1, abort_flag, p.status)) { ok = false; break; }
-                    for (int t = 0; t < 2 && ok; ++t) {
-                        const int n_t = t == 0 ? n_steps_a : n_steps_b;
-                        if (j + 1 < n_t) {
-                            // the row threads have copied S_t of step j into registers: its columns may be overwritten
-                            if (!mbar_wait(bar(S_FREE + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
-                            tc_fence_after();
-                            issue_qk(t, sl);
-                        }
-                    }
-                    if (!ok) break;
-                    commit1_w(bar(KV_EMPTY + sl), leader);
-                    ++li;
-                }
-                const int sl = li % 3;
-                if (!mbar_wait(bar(KV_FULL + sl), (uint32_t)(li / 3) & 1, abort_flag, p.status)) { ok = false; break; }
-                for (int t = 0; t < 2 && ok; ++t) {
-                    const int n_t = t == 0 ? n_steps_a : n_steps_b;
-                    if (j < n_t) {
-                        if (!mbar_wait(bar(P_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
-                        tc_fence_after();
-                        issue_pv(t, sl, j == 0);
-                    }
-                }
-                if (!ok) break;
-                commit1_w(bar(KV_EMPTY + sl), leader);
-                ++li;
-            }
-        }
-    } else {
-        // ================= row threads =================
-        const int t = (warp - 2) >> 2;
-        const int q = warp & 3;
-        const int r = q * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        const uint32_t tS = tmem_base + t * 128 + lane_addr, tO = tmem_base + 256 + t * 128 + lane_addr;
-        const int n_t = t == 0 ? n_steps_a : n_steps_b;
-        const int qrow = q0 + t * QT + r;
-        uint8_t* prow = pP + t * TILE_BYTES + r * 128;     // this row inside each 64-key half of the P tile
-        const int sw = r & 7;                              // 128-byte swizzle: 16-byte chunk c of row r lives at chunk c ^ (r & 7)
-        float m_used = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_t && ok; ++j) {
-            if (!mbar_wait(bar(S_FULL + t), (uint32_t)j & 1, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const bool diag = p.causal && (j == n_t - 1);
-            const int kmax = qrow - (s0 + j * KT);
-            uint32_t v[128];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, v + c * 32);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(S_FREE + t));   // S_t is in registers: the next Q K^T of this tile may run
-            const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
-            const float m_new = mx * p.scale_log2e;
-            float alpha = 1.f;
-            bool need = false;
-            if (j == 0) m_used = m_new;
-            else if (m_new > m_used + 8.f) { alpha = ex2(m_used - m_new); m_used = m_new; need = true; }
-            // P V of step j-1 has finished: it no longer reads the P tile, and O~ holds the products up to step j-1
-            if (j > 0 && !mbar_wait(bar(P_EMPTY + t), (uint32_t)(j - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-            if (__any_sync(0xffffffffu, need)) {
-                tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < 16; ++c) {
-                    uint32_t o[8];
-                    tmem_ld8(tO + c * 8, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st8(tO + c * 8, o);
-                }
-                tmem_st_wait();
-                tc_fence_before();
-                l_run *= alpha;
-            }
-            // P = 2^(S*scale - m) as bf16 into the swizzled K-major tile; row sum in f32
-            {
-                const uint64_t sc2 = pack2(p.scale_log2e, p.scale_log2e), nm2 = pack2(-m_used, -m_used);
-                uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {          // 16 chunks of 8 keys = 16 bytes of bf16
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int i = 0; i < 8; i += 2) {
-                        const int col = c * 8 + i;
-                        float p0, p1;
-                        unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
-                        p0 = ex2(p0);
-                        p1 = ex2(p1);
-                        if (diag) {
-                            if (col > kmax) p0 = 0.f;
-                            if (col + 1 > kmax) p1 = 0.f;
-                        }
-                        if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
-                        else sum_b = add2(sum_b, pack2(p0, p1));
-                        __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
-                        pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
-                    }
-                    *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-                float a0, a1, b0, b1;
-                unpack2(sum_a, a0, a1);
-                unpack2(sum_b, b0, b1);
-                l_run += (a0 + a1) + (b0 + b1);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads P through the async proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(P_FULL + t));
-        }
-        if (ok && n_t > 0) {
-            // O = O~ / l goes out through the tile's P buffer (its last P V has read it once O_FULL fires): every row thread
-            // writes its 256 bytes in the swizzled layout of the tensor map, and one thread hands the tile to two TMA stores --
-            // 16-byte stores from 32 lanes to 32 different rows would write half-filled sectors.
-            if (mbar_wait(bar(O_FULL + t), (uint32_t)(n_t - 1) & 1, abort_flag, p.status)) {
-                tc_fence_after();
-                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                if (p.lse_base) {
-                    const int64_t cell = (int64_t)seq_row(p.q, p.S, b, qrow, h) * p.q.hblk + h % p.q.hblk;
-                    p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4 ov;
-                        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
-                        const int cc = c * 4 + g;                      // 16-byte chunk 0..15 of the row
-                        *reinterpret_cast<uint4*>(prow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) = ov;
-                    }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(O_STAGED + t));
-                if (q == 0 && lane == 0 && mbar_wait(bar(O_STAGED + t), 0, abort_flag, p.status)) {
-                    const int orow = seq_row(p.q, p.S, b, q0 + t * QT, h);
-                    for (int half = 0; half < 2; ++half)
-                        tma_store_3d(&tmO, sP + t * TILE_BYTES + half * HALF_BYTES, half * 64, h % p.q.hblk, orow);
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
-                }
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------------
-// The shared-memory form above, persistent over work items. One work item = the pair of query tiles of one (batch, head);
-// one CTA per SM takes items, heaviest first, from a counter in global memory (its producer thread claims the next item and
-// hands its number to the other roles through a two-entry queue in shared memory), so CTAs that drew short items simply take
-// more of them. Barriers and tensor memory are set up once. The producer runs ahead
-// into the next item as soon as the Q buffers are free (after the item's last Q K^T, about one key step before its end),
-// so the next item's Q and first K tile load, and its first Q K^T products run, while the row threads finish the last
-// softmax, normalise and store this item's output. Barrier phases follow running counters (items; key steps per tile).
-// ---------------------------------------------------------------------------------------------------------
-// {next item, CTAs finished} pairs for launches of the persistent kernel: a launch takes the next pair of the ring, and its
+// {next item, CTAs finished} pairs for launches of the persistent form: a launch takes the next pair of the ring, and its
 // last CTA zeroes the pair again, so a pair is ready for reuse (also by a replay of a captured launch) as soon as its kernel
 // has finished. 128 launches would have to be in flight at once (or 128 captured launches alive in graphs that replay
 // concurrently) for two of them to share a pair.
@@ -1110,14 +543,16 @@ __device__ int32_t g_attn_queues[2 * ATTN_QUEUES];
 struct AttnItem {
     int q0, h, b, s0, n_a, n_b;
 };
-// item number `rank` in heaviest-first order; false past the end
+// item number `rank` in launch order (ja_attn_decode_cta: heaviest pairs first inside sections of (batch, head) pairs);
+// false past the end
 __device__ __forceinline__ bool attn_item(const AttnTcParams& p, int rank, AttnItem* it) {
     const int hb = p.H * p.B, n_pairs = p.S / (2 * QT);
     if (rank >= n_pairs * hb) return false;
-    const int pidx = rank / hb, r = rank - pidx * hb;
-    const int pr = p.n_order ? (int)p.order[pidx] : n_pairs - 1 - pidx;   // heaviest pairs of all (batch, head) first
-    it->h = r % p.H;
-    it->b = r / p.H;
+    int slot, bh;
+    ja_attn_decode_cta(rank, n_pairs, hb, p.sect, &slot, &bh);
+    const int pr = p.n_order ? (int)p.order[slot] : n_pairs - 1 - slot;
+    it->h = bh % p.H;
+    it->b = bh / p.H;
     it->q0 = pr * 2 * QT;
     int s1;
     sequence_of(p, it->q0, it->s0, s1);
@@ -1126,10 +561,13 @@ __device__ __forceinline__ bool attn_item(const AttnTcParams& p, int rank, AttnI
     return true;
 }
 
+template <bool PERSIST, int VAR>
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
-attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                      const __grid_constant__ AttnTcParams p) {
+attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                     const __grid_constant__ AttnTcParams p) {
+    constexpr int POLY = VAR & 3;
+    constexpr bool WAIT_FIRST = (VAR & 4) == 0;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -1142,12 +580,13 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
            O_STAGED = 18, O_READ = 20, P_STORED = 22, ITEM_FULL = 24, ITEM_EMPTY = 26, NBAR = 28 };
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBAR);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* item_rank = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [2]: the item numbers in flight
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // two words: abort flag, wait limit
+    volatile int* item_rank = reinterpret_cast<volatile int*>(tmem_slot + 3);    // [2]: the item numbers in flight
 
     const int warp = __shfl_sync(0xffffffffu, (int)threadIdx.x / 32, 0), lane = threadIdx.x % 32;
     // consumers of the item queue (MMA warp, row warps): wait for entry k, read it, release it
     auto next_item = [&](int k, AttnItem* it) -> bool {
+        if (!PERSIST) return k == 0 && attn_item(p, (int)blockIdx.x, it);
         const int e = k & 1;
         if (!mbar_wait(bar(ITEM_FULL + e), (uint32_t)(k >> 1) & 1, abort_flag, p.status)) return false;
         const int rank = item_rank[e];
@@ -1162,7 +601,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                                           (i >= O_STAGED && i < O_STAGED + 2) || (i >= O_READ && i < O_READ + 2);
             mbar_init(bar(i), row_warps_arrive ? 4 : (i >= ITEM_EMPTY && i < ITEM_EMPTY + 2) ? 9 : 1);
         }
-        *abort_flag = 0;
+        wait_ctl_init(abort_flag, p.wait_cap_us);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -1181,13 +620,19 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             bool ok = true;
             AttnItem it;
             for (int item = 0; ok; ++item) {
-                // claim the next item and publish its number (entry item & 1 of the queue, free once all nine consumer warps
-                // have read what it held two items ago)
-                const int e = item & 1;
-                if (item >= 2 && !mbar_wait(bar(ITEM_EMPTY + e), (uint32_t)((item >> 1) - 1) & 1, abort_flag, p.status)) break;
-                const int rank = atomicAdd(p.queue, 1);
-                item_rank[e] = rank;
-                mbar_arrive(bar(ITEM_FULL + e));
+                int rank;
+                if (PERSIST) {
+                    // claim the next item and publish its number (entry item & 1 of the queue, free once all nine consumer
+                    // warps have read what it held two items ago)
+                    const int e = item & 1;
+                    if (item >= 2 && !mbar_wait(bar(ITEM_EMPTY + e), (uint32_t)((item >> 1) - 1) & 1, abort_flag, p.status)) break;
+                    rank = atomicAdd(p.queue, 1);
+                    item_rank[e] = rank;
+                    mbar_arrive(bar(ITEM_FULL + e));
+                } else {
+                    if (item > 0) break;
+                    rank = (int)blockIdx.x;
+                }
                 if (!attn_item(p, rank, &it)) break;
                 const int hk = it.h / p.group;
                 // the Q buffers are free once the previous item's last Q K^T has read them
@@ -1198,6 +643,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     for (int half = 0; half < 2; ++half)
                         tma_load_3d(sQ + t * TILE_BYTES + half * HALF_BYTES, &tmQ, bar(Q_FULL), half * 64, it.h % p.q.hblk, qrow_t);
                 }
+                // K / V tiles in the order the products consume them: K_0, then for every step j: K_{j+1} (if any), V_j
                 auto load = [&](const CUtensorMap* tm, int j) {
                     const int sl = li % 3;
                     const uint32_t ph = (uint32_t)(li / 3) & 1;
@@ -1214,12 +660,13 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     if (ok) load(&tmV, j);
                 }
             }
-            // the last CTA to get here leaves the counter pair as it found it
-            __threadfence();
-            if (atomicAdd(p.queue + 1, 1) == (int)gridDim.x - 1) {
-                p.queue[0] = 0;
-                p.queue[1] = 0;
+            if (PERSIST) {   // the last CTA to get here leaves the counter pair as it found it
                 __threadfence();
+                if (atomicAdd(p.queue + 1, 1) == (int)gridDim.x - 1) {
+                    p.queue[0] = 0;
+                    p.queue[1] = 0;
+                    __threadfence();
+                }
             }
         }
     } else if (warp == 1) {
@@ -1230,7 +677,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         auto issue_qk = [&](int t, int sl) {          // S_t = Q_t K^T, K in slot sl
             const uint32_t kaddr = sKV + sl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
+            for (int kk = 0; kk < 8; ++kk) {          // 16 d per instruction; d 0..63 in the first half, 64..127 in the second
                 const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
                 umma_ss_w(tmem_base + t * 128, desc_sw128(qaddr + off, 16), desc_sw128(kaddr + off, 16), idesc_qk, kk > 0, leader);
             }
@@ -1274,6 +721,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     if (!mbar_wait(bar(KV_FULL + sl), (uint32_t)(li / 3) & 1, abort_flag, p.status)) { ok = false; break; }
                     for (int t = 0; t < 2 && ok; ++t) {
                         if (j + 1 < n_of[t]) {
+                            // the row threads have copied S_t of step j into registers: its columns may be overwritten
                             if (!mbar_wait(bar(S_FREE + t), (uint32_t)(cs[t] + j) & 1, abort_flag, p.status)) { ok = false; break; }
                             tc_fence_after();
                             issue_qk(t, sl);
@@ -1304,8 +752,8 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
     } else {
         // ================= row threads =================
-        const int t = (warp - 2) >> 2;
-        const int q = warp & 3;
+        const int t = (warp - 2) >> 2;                     // tile: 0 = A, 1 = B
+        const int q = warp & 3;                            // TMEM lane group of this warp
         const int r = q * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const uint32_t tS = tmem_base + t * 128 + lane_addr, tO = tmem_base + 256 + t * 128 + lane_addr;
@@ -1332,19 +780,28 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(S_FREE + t));   // S_t is in registers: the next Q K^T of this tile may run
                 const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
-                const float m_new = mx * p.scale_log2e;
+                const float m_new = mx * p.scale_log2e;        // finite: the first key of a sequence is never masked
+                // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
                 float alpha = 1.f;
                 bool need = false;
                 if (j == 0) m_used = m_new;
                 else if (m_new > m_used + 8.f) { alpha = ex2(m_used - m_new); m_used = m_new; need = true; }
-                // P V of the tile's previous key step has finished: it no longer reads the P tile, and O~ holds the products so far;
-                // at the first step of an item the P tile also held the previous item's output until its TMA stores had read it
-                if (c > 0 && !mbar_wait(bar(P_EMPTY + t), (uint32_t)(c - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                if (j == 0 && item > 0 && !mbar_wait(bar(P_STORED + t), (uint32_t)(item - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                if (__any_sync(0xffffffffu, need)) {
+                const bool rescale = __any_sync(0xffffffffu, need);
+                // Two things have to hold before P of this step may be stored: the P V of the tile's previous key step has
+                // read the P tile (P_EMPTY; O~ then also holds every product so far), and at the first step of an item the
+                // TMA stores of the previous item's output, which was staged in the P tile, have read it (P_STORED).
+                auto wait_p_tile = [&]() -> bool {
+                    if (c > 0 && !mbar_wait(bar(P_EMPTY + t), (uint32_t)(c - 1) & 1, abort_flag, p.status)) return false;
+                    if (j == 0 && item > 0 && !mbar_wait(bar(P_STORED + t), (uint32_t)(item - 1) & 1, abort_flag, p.status)) return false;
+                    return true;
+                };
+                if (WAIT_FIRST || rescale) {
+                    if (!wait_p_tile()) { ok = false; break; }
+                }
+                if (rescale) {
                     tc_fence_after();
 #pragma unroll 1
-                    for (int cc = 0; cc < 16; ++cc) {
+                    for (int cc = 0; cc < 16; ++cc) {   // rare path: small chunks keep the register footprint of the hot path low
                         uint32_t o[8];
                         tmem_ld8(tO + cc * 8, o);
                         tmem_ld_wait();
@@ -1356,47 +813,29 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     tc_fence_before();
                     l_run *= alpha;
                 }
-                {
-                    const uint64_t sc2 = pack2(p.scale_log2e, p.scale_log2e), nm2 = pack2(-m_used, -m_used);
-                    uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
-#pragma unroll
-                    for (int cc = 0; cc < 16; ++cc) {          // 16 chunks of 8 keys = 16 bytes of bf16
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int i = 0; i < 8; i += 2) {
-                            const int col = cc * 8 + i;
-                            float p0, p1;
-                            unpack2(fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2), p0, p1);
-                            p0 = ex2(p0);
-                            p1 = ex2(p1);
-                            if (diag) {
-                                if (col > kmax) p0 = 0.f;
-                                if (col + 1 > kmax) p1 = 0.f;
-                            }
-                            if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
-                            else sum_b = add2(sum_b, pack2(p0, p1));
-                            __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
-                            pk[i / 2] = *reinterpret_cast<uint32_t*>(&tt);
-                        }
-                        *reinterpret_cast<uint4*>(prow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                    float a0, a1, b0, b1;
-                    unpack2(sum_a, a0, a1);
-                    unpack2(sum_b, b0, b1);
-                    l_run += (a0 + a1) + (b0 + b1);
+                uint32_t pk[64];
+                l_run += diag ? row_exp_pack128<true, POLY>(v, kmax, p.scale_log2e, m_used, pk)
+                              : row_exp_pack128<false, POLY>(v, kmax, p.scale_log2e, m_used, pk);
+                if (!(WAIT_FIRST || rescale)) {
+                    if (!wait_p_tile()) { ok = false; break; }
                 }
+#pragma unroll
+                for (int cc = 0; cc < 16; ++cc)          // 16 chunks of 8 keys = 16 bytes of bf16
+                    *reinterpret_cast<uint4*>(prow + (cc >> 3) * HALF_BYTES + (((cc & 7) ^ sw) << 4)) =
+                        make_uint4(pk[cc * 4], pk[cc * 4 + 1], pk[cc * 4 + 2], pk[cc * 4 + 3]);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads P through the async proxy
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(P_FULL + t));
             }
             if (!ok) break;
-            // ---- the item's output: O = O~ / l through the tile's P buffer and two TMA stores
+            // ---- the item's output: O = O~ / l through the tile's P buffer (its last P V has read it once O_FULL fires) and two
+            // TMA stores -- 16-byte stores from 32 lanes to 32 different rows would write half-filled sectors
             if (!mbar_wait(bar(O_FULL + t), (uint32_t)(cs + n_t - 1) & 1, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
             if (p.lse_base) {
                 const int64_t cell = (int64_t)seq_row(p.q, p.S, it.b, qrow, it.h) * p.q.hblk + it.h % p.q.hblk;
-                p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+                p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
             }
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
@@ -1410,7 +849,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
                         po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
-                    const int ch = cc * 4 + g;
+                    const int ch = cc * 4 + g;                      // 16-byte chunk 0..15 of the row
                     *reinterpret_cast<uint4*>(prow + (ch >> 3) * HALF_BYTES + (((ch & 7) ^ sw) << 4)) = ov;
                 }
             }
@@ -1428,7 +867,7 @@ attention_tc3p_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     for (int half = 0; half < 2; ++half)
                         tma_store_3d(&tmO, sP + t * TILE_BYTES + half * HALF_BYTES, half * 64, it.h % p.q.hblk, orow);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be reused after this
                     mbar_arrive(bar(P_STORED + t));  // the P tile may be written again
                 }
             }
@@ -1476,31 +915,66 @@ bool fill_geom(const RelView& v, const int32_t* host_split, SeqGeom* g) {
 
 }  // namespace
 
+
 // After a device-side failure (a bounded wait that expired) a persistent launch may have left its work counter non-zero:
-// put every counter pair back to zero. Called by ja_stream_status when it reports such a failure; the stream is idle then.
+// put every counter pair of the current device back to zero. Called by ja_stream_status when it reports such a failure;
+// the stream is idle then.
 void ja_attention_reset_queues() {
     void* q = nullptr;
     if (cudaGetSymbolAddress(&q, g_attn_queues) == cudaSuccess && q) cudaMemset(q, 0, sizeof(int32_t) * 2 * ATTN_QUEUES);
 }
 
-// Returns JA_OK and sets *launched when the tensor-memory kernel took the job; leaves *launched false when the
-// tiling does not fit it (every q / k split point and sequence end must be a multiple of 128 rows, blocks uniform
-// along b and h, at most MAX_SB sequence blocks when they are irregular).
+namespace {
+
+template <bool PERSIST>
+ja_status_t launch_two_tiles(int variant, dim3 grid, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             const CUtensorMap& to, const AttnTcParams& p) {
+#define JA_ATTN_LAUNCH(V)                                                                                                          \
+    case V: {                                                                                                                      \
+        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel<PERSIST, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2)); \
+        attention_tc2_kernel<PERSIST, V><<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);                             \
+        return JA_OK;                                                                                                              \
+    }
+    switch (variant) {
+        JA_ATTN_LAUNCH(0)
+        JA_ATTN_LAUNCH(1)
+        JA_ATTN_LAUNCH(4)
+        default: return ja_fail(JA_ERR_INVALID_ARG, "unknown attention variant %d", variant);
+    }
+#undef JA_ATTN_LAUNCH
+}
+
+}  // namespace
+
+// Returns JA_OK and sets *launched when a tensor-memory kernel took the job; leaves *launched false when the tiling does
+// not fit (every q / k split point and sequence end must be a multiple of 128 rows, blocks uniform along b and h, at most
+// MAX_SB sequence blocks when they are irregular). The four tensor maps are encoded once per (spec, relations) tuple and
+// kept in a.cache.
 ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched) {
     *launched = false;
     if (a.align % 128 || !a.rows_layout) return JA_OK;
     AttnTcParams p;
     memset(&p, 0, sizeof p);
     if (!fill_geom(a.q, a.q_split, &p.q) || !fill_geom(a.k, a.k_split, &p.k)) return JA_OK;
-    CUtensorMap tq, tk, tv;
-    ja_status_t s;
-    if ((s = encode_rows(a.q, &tq)) != JA_OK) return s;
-    if ((s = encode_rows(a.k, &tk)) != JA_OK) return s;
-    if ((s = encode_rows(a.v, &tv)) != JA_OK) return s;
+    static_assert(sizeof(CUtensorMap) == 128, "AttnTcCache holds four 128-byte tensor maps");
+    AttnTcCache local;
+    AttnTcCache* cache = a.cache ? a.cache : &local;
+    CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(cache->maps);
+    if (!cache->valid) {
+        ja_status_t s;
+        if ((s = encode_rows(a.q, &maps[0])) != JA_OK) return s;
+        if ((s = encode_rows(a.k, &maps[1])) != JA_OK) return s;
+        if ((s = encode_rows(a.v, &maps[2])) != JA_OK) return s;
+        if ((s = encode_rows(a.o, &maps[3])) != JA_OK) return s;
+        cache->valid = true;
+    }
+    const CUtensorMap &tq = maps[0], &tk = maps[1], &tv = maps[2], &to = maps[3];
+    const JaConfig& cfg = ja_config();
     p.o_base = a.o.base;
     p.lse_base = reinterpret_cast<float*>(a.lse.base);
-    p.status = ja_device_status_word();
+    p.status = ja_device_status_word(st);
     if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    p.wait_cap_us = (uint32_t)cfg.wait_cap_us;
     p.B = a.B; p.S = a.S; p.H = a.H;
     p.group = a.group;
     p.causal = a.causal;
@@ -1511,8 +985,7 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
         if (a.ends[i] % (2 * QT)) pair_ok = false;
     }
     p.scale_log2e = a.scale * 1.4426950408889634f;
-    const char* one = getenv("JA_ATTN_ONE_TILE");
-    const bool two_tiles = pair_ok && !(one && one[0] == '1');
+    const bool two_tiles = pair_ok && cfg.attn_one_tile != 1;
     // packed sequences: the work of a tile is its distance from the start of its own sequence, not its index
     const int rows_per_cta = two_tiles ? 2 * QT : QT, n_cta_tiles = a.S / rows_per_cta;
     if (a.n_ends > 1 && n_cta_tiles <= MAX_ORDER) {
@@ -1530,64 +1003,41 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
         p.n_order = n_cta_tiles;
         for (int t = 0; t < n_cta_tiles; ++t) p.order[t] = (uint16_t)w[t].second;
     }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
-    }
+    const int sms = ja_sm_count();
     // tiles of different weight (causal band, packed sequences): one section, i.e. heaviest first across all (batch, head)
-    // pairs -- measured better than any sectioning (balance beats L2 re-use); equal tiles: sections that fill the GPU once
+    // pairs; equal tiles: sections that fill the GPU once, so that CTAs running together share K / V tiles through L2
     p.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::max(1, (sms + n_cta_tiles - 1) / n_cta_tiles);
-    if (const char* se = getenv("JA_ATTN_SECTION")) p.sect = std::max(1, atoi(se));
+    if (cfg.attn_section >= 1) p.sect = cfg.attn_section;
     p.sect = std::min(p.sect, a.H * a.B);
     if (two_tiles) {
-        dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / (2 * QT))), 1, 1);
-        // Two forms of the two-tile kernel (both verified against the oracle; JA_ATTN_P_SMEM = 0 / 1 forces one). P through
-        // shared memory takes the next Q K^T of a tile off the chain softmax -> P V -> Q K^T, which pays where work items are
-        // short or uneven (causal band, packed sequences: 5-7 % faster at 1K-2K rows per sequence, equal beyond 8K); with
-        // equal items (not causal, one sequence) the two forms measure the same, and P in tensor memory executes a third
-        // fewer instructions.
-        CUtensorMap to;
-        if ((s = encode_rows(a.o, &to)) != JA_OK) return s;
-        const char* v3 = getenv("JA_ATTN_P_SMEM");
-        const bool p_smem = v3 ? v3[0] == '1' : (a.causal || a.n_ends > 1);
-        if (p_smem) {
-            // persistent over work items where items are short (no sequence longer than 4096 rows: 6 % faster at 2048 rows,
-            // 13 % on packed sequences of 1024-1536 rows); beyond that the fixed item order balances worse than the hardware's
-            // hand-out of CTAs (1-2 % slower at 8K-16K rows). JA_ATTN_PERSISTENT = 0 / 1 forces one.
-            int longest = a.S;
-            if (a.n_ends > 0) {
-                longest = a.ends[0];
-                for (int i = 1; i < a.n_ends; ++i) longest = std::max(longest, a.ends[i] - a.ends[i - 1]);
-            }
-            const char* pe = getenv("JA_ATTN_PERSISTENT");
-            if (pe ? pe[0] == '1' : longest <= 4096) {
-                static int32_t* queues = nullptr;
-                static std::atomic<unsigned> next_queue{0};
-                if (!queues && cudaGetSymbolAddress((void**)&queues, g_attn_queues) != cudaSuccess) {
-                    queues = nullptr;
-                    return ja_fail(JA_ERR_CUDA, "cannot resolve the attention work queues");
-                }
-                // launches recorded into a CUDA graph keep their pair for as long as the graph lives: they draw from the upper half
-                // of the ring, launches that run at once from the lower half, so a replay never shares a pair with an eager launch
-                static std::atomic<unsigned> next_captured{0};
-                cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-                if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
-                const unsigned half = ATTN_QUEUES / 2;
-                const unsigned slot = cap == cudaStreamCaptureStatusActive ? half + next_captured.fetch_add(1) % half : next_queue.fetch_add(1) % half;
-                p.queue = queues + 2 * slot;
-                JA_CUDA(cudaFuncSetAttribute(attention_tc3p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
-                dim3 pgrid((unsigned)std::min<int64_t>((int64_t)a.H * a.B * (a.S / (2 * QT)), sms), 1, 1);
-                attention_tc3p_kernel<<<pgrid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
-            } else {
-                JA_CUDA(cudaFuncSetAttribute(attention_tc3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES3));
-                attention_tc3_kernel<<<grid, NUM_THREADS2, SMEM_BYTES3, st>>>(tq, tk, tv, to, p);
-            }
-        } else {
-            JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
-            attention_tc2_kernel<<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);
+        const int64_t items = (int64_t)a.H * a.B * (a.S / (2 * QT));
+        // persistent over work items where items are short (no sequence longer than 4096 rows); beyond that the hardware's
+        // hand-out of one CTA per item balances as well and the queue buys nothing
+        int longest = a.S;
+        if (a.n_ends > 0) {
+            longest = a.ends[0];
+            for (int i = 1; i < a.n_ends; ++i) longest = std::max(longest, a.ends[i] - a.ends[i - 1]);
         }
+        const bool persist = cfg.attn_persistent >= 0 ? cfg.attn_persistent == 1 : longest <= 4096;
+        const int variant = cfg.attn_variant >= 0 ? cfg.attn_variant : 0;
+        ja_status_t s;
+        if (persist) {
+            int32_t* queues = nullptr;
+            if (cudaGetSymbolAddress((void**)&queues, g_attn_queues) != cudaSuccess || !queues)
+                return ja_fail(JA_ERR_CUDA, "cannot resolve the attention work queues");
+            // launches recorded into a CUDA graph keep their pair for as long as the graph lives: they draw from the upper half
+            // of the ring, launches that run at once from the lower half, so a replay never shares a pair with an eager launch
+            static std::atomic<unsigned> next_queue{0}, next_captured{0};
+            cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+            if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
+            const unsigned half = ATTN_QUEUES / 2;
+            const unsigned slot = cap == cudaStreamCaptureStatusActive ? half + next_captured.fetch_add(1) % half : next_queue.fetch_add(1) % half;
+            p.queue = queues + 2 * slot;
+            s = launch_two_tiles<true>(variant, dim3((unsigned)std::min<int64_t>(items, sms), 1, 1), st, tq, tk, tv, to, p);
+        } else {
+            s = launch_two_tiles<false>(variant, dim3((unsigned)items, 1, 1), st, tq, tk, tv, to, p);
+        }
+        if (s != JA_OK) return s;
     } else {
         JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);

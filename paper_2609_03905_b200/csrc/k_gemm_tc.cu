@@ -51,7 +51,8 @@ template <int CG> struct Cfg {
 struct GemmParams {
     char* c_base;
     const int64_t* c_blk_off;  // device: byte offsets of the output blocks
-    int32_t* status;           // device status word
+    int32_t* status;           // status word of the launching stream (set at launch)
+    uint32_t wait_cap_us;      // limit of every bounded wait (set at launch)
     int32_t bm, bk, bn;        // block extents along i, j, k
     int32_t nbm, nbk, nbn;     // blocks along i, j, k
     int32_t M, N;              // tensor extents along i, k
@@ -176,7 +177,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(tfull_bar(a), 1);
             mbar_init(tempty_bar(a), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
         }
-        *abort_flag = 0;
+        wait_ctl_init(abort_flag, p.wait_cap_us);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // all 512 TMEM columns: two 128 x 256 fp32 accumulators (in each CTA of a pair)
@@ -456,8 +457,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     GemmParams& p = plan->p;
     p.c_base = (char*)C->base;
     p.c_blk_off = ja_view(C).blk_off;
-    p.status = ja_device_status_word();
-    if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    p.status = nullptr;
     p.bm = (int)bm; p.bk = (int)bk; p.bn = (int)bn;
     p.nbm = A->nblk[0]; p.nbk = A->nblk[1]; p.nbn = B->nblk[1];
     p.M = (int)A->extent[0]; p.N = (int)B->extent[1];
@@ -476,17 +476,12 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     // Two-CTA form: 256-row tiles cut from global rows; needs 128-row halves that never straddle a block and, when
     // tiles span column blocks, column tails whose halves still start on a 64-column box boundary.
     // narrow last tile in every column block (block width not a multiple of the tile width): schedule it after the full tiles
-    {
-        const char* hf = getenv("JA_GEMM_HEAVY_FIRST");
-        p.heavy_first = (p.n_copies == 1 && p.tiles_per_nblk > 1 && bn % bn_tile != 0 && !(hf && hf[0] == '0')) ? 1 : 0;
-    }
-    const char* gm = getenv("JA_GEMM_GROUP_M");
-    p.group_m = gm ? atoi(gm) : 8;
-    if (p.group_m < 1) p.group_m = 1;
-    const char* force = getenv("JA_GEMM_CTA_GROUP");
+    const JaConfig& cfg = ja_config();
+    p.heavy_first = (p.n_copies == 1 && p.tiles_per_nblk > 1 && bn % bn_tile != 0 && cfg.gemm_heavy_first != 0) ? 1 : 0;
+    p.group_m = cfg.gemm_group_m >= 1 ? cfg.gemm_group_m : 8;
     bool two = (bm % 128 == 0 || 128 % bm == 0) && p.M >= 256 && bk >= Cfg<2>::BK;
     if (p.tiles_per_nblk == 0 && (p.N % bn_tile) % (bn_tile / 2) != 0) two = false;
-    if (force && force[0] == '1') two = false;
+    if (cfg.gemm_cta_group == 1) two = false;
     plan->cg = two ? 2 : 1;
     if (two || bm < 128) { p.tiles_per_mblk = 0; p.m_tiles = (p.M + BM * plan->cg - 1) / (BM * plan->cg); }
     else { p.tiles_per_mblk = (int)((bm + BM - 1) / BM); p.m_tiles = p.tiles_per_mblk * p.nbm; }
@@ -495,9 +490,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     if ((st = encode_blocked_2d(B, 64, two ? Cfg<2>::BK : Cfg<1>::BK, &plan->tmB)) != JA_OK) return st;
     plan->tmB2 = plan->tmB;
     if (epi == EPI_SWIGLU && (st = encode_blocked_2d(ep->B2, 64, two ? Cfg<2>::BK : Cfg<1>::BK, &plan->tmB2)) != JA_OK) return st;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = ja_sm_count();
     const int tiles = p.m_tiles * p.n_tiles * p.n_copies;
     plan->grid = two ? 2 * std::min(sms / 2, tiles) : std::min(sms, tiles);
     cudaError_t e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
@@ -509,6 +502,10 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
 }
 
 ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
+    GemmParams p = plan.p;
+    p.status = ja_device_status_word(st);
+    if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
+    p.wait_cap_us = (uint32_t)ja_config().wait_cap_us;
     if (plan.cg == 2) {
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
@@ -523,9 +520,9 @@ ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.tmB2, plan.p));
+        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.tmB2, p));
     } else {
-        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, plan.p);
+        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, p);
         JA_CUDA(cudaGetLastError());
     }
     ja_count_launch();

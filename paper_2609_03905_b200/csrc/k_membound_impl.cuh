@@ -464,7 +464,7 @@ void launch_fast_v(const RowArgs& a, const FastGeom& g, int64_t n_rows, int team
     if (resident == 0) {
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_fast_kernel<T, VEC, VPT, OP>, block, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-        resident = per_sm * 148;
+        resident = per_sm * ja_sm_count();
     }
     unsigned grid = (unsigned)(want < resident ? want : resident);
     row_fast_kernel<T, VEC, VPT, OP><<<grid, block, 0, st>>>(a, g, n_rows, team);
@@ -480,7 +480,7 @@ bool launch_fast(const RowArgs& a, const FastGeom& g, int64_t n_rows, cudaStream
     constexpr bool REDUCE_ONLY = (OP == ROW_SUMSQ || OP == ROW_MAX || OP == ROW_EXPSUM);
     int team = 32;
     while (team < 256 && g.n > team * VEC * (REDUCE_ONLY ? 4 : 2)) team *= 2;
-    if (const char* e = getenv("JA_ROW_TEAM")) { int t = atoi(e); if (t >= 32 && t <= 256 && (t & (t - 1)) == 0) team = t; }
+    { const int t = ja_config().row_team; if (t >= 32 && t <= 256 && (t & (t - 1)) == 0) team = t; }
     const int vpt = (g.n + team * VEC - 1) / (team * VEC);
     if (vpt <= 1) launch_fast_v<T, VEC, 1, OP>(a, g, n_rows, team, st);
     else if (vpt <= 2) launch_fast_v<T, VEC, 2, OP>(a, g, n_rows, team, st);

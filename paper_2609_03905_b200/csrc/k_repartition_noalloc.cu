@@ -2,7 +2,7 @@
 //
 // Who needs it: code that runs where device allocation is forbidden or impossible -- inside a region whose memory
 // was budgeted up front (an inference server that hands every byte of HBM to its own pool at start-up), in a
-// real-time loop where cudaMalloc's implicit synchronisation is unacceptable, or under a memory-accounting
+// loop that must never take cudaMalloc's implicit device synchronisation, or under a memory-accounting
 // harness that fails any allocation it did not make itself. ja_repartition builds its copy plan in a
 // cudaMalloc'ed table and keeps it cached; this entry point keeps the plan in a fixed, file-scope device array
 // instead and never calls cudaMalloc, cudaFree, or any allocating library routine (host or device).
@@ -15,7 +15,11 @@
 //   * two calls that overlap on the GPU (different streams, or the same stream from two threads) race on it --
 //     serialise them;
 //   * the first call on each device resolves the array's device address (set-up, one cudaGetSymbolAddress with
-//     that device current); make that first call before starting any stream capture.
+//     that device current); make that first call before starting any stream capture;
+//   * the plan travels to the device with a stream-ordered copy out of a fixed host table that the next call
+//     overwrites, so the host may block for the few microseconds the copy needs, and a call on a stream that is
+//     being captured is refused (JA_ERR_UNSUPPORTED, nothing enqueued): a recorded copy would read, at replay
+//     time, whatever plan the latest call left in that table.
 #include <string.h>
 
 #include <mutex>
@@ -210,6 +214,13 @@ extern "C" ja_status_t ja_repartition_noalloc(int32_t rank, const int64_t* exten
     ja_status_t st = scratch_for_device(&d_slabs);
     if (st != JA_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        JA_CUDA(cudaStreamIsCapturing(stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone)
+            return ja_fail(JA_ERR_UNSUPPORTED, "ja_repartition_noalloc was called on a stream that is being captured: its plan is staged in "
+                                               "a host table shared by all calls, which a replay would read too late");
+    }
     // plan -> the fixed device table (stream-ordered; the copy reads host_slabs before returning because it is pageable)
     JA_CUDA(cudaMemcpyAsync(d_slabs, host_slabs, (size_t)n_slabs * sizeof(CopySlab), cudaMemcpyHostToDevice, stream));
     int vec = 16;

@@ -51,6 +51,7 @@ struct RowTmaGeom {
     int stat_blk_bytes;          // bytes between consecutive blocks of a statistics relation
     int g_blk_bytes;             // bytes between consecutive blocks of the gain vector
     float eps;
+    uint32_t wait_cap_us;        // limit of every bounded wait
 };
 
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
@@ -377,7 +378,7 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
             mbar_init(free_bar(s), HAS_Y ? 1 : CONSUMER_WARPS);
         }
         for (int t = 0; t < CONSUMER_WARPS; ++t) mbar_init(team_bar(t), (uint32_t)g.wpr);
-        *abort_flag = 0;
+        wait_ctl_init(abort_flag, g.wait_cap_us);   // two words: the slot is eight bytes wide
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -502,10 +503,12 @@ ja_status_t launch_v(const RowMaps& tm, const RowArgs& a, RowTmaGeom g, int g_by
     const int budget = (CTAS == 2 ? 110 : 220) * 1024 - g_bytes;
     g.stages = (int)std::min<int64_t>(MAX_STAGES, budget / g.stage_bytes);
     if (g.stages < 2) { *launched = false; return JA_OK; }
-    static bool configured = false;   // per template instance
-    if (!configured) {
+    static bool configured[64] = {};   // per template instance and device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!configured[dev & 63]) {
         JA_CUDA(cudaFuncSetAttribute(row_tma_kernel<T, OP, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024));
-        configured = true;
+        configured[dev & 63] = true;
     }
     const int smem_bytes = g.stages * g.stage_bytes + g_bytes + (3 * MAX_STAGES + CONSUMER_WARPS + 2) * 8 + CONSUMER_WARPS * 16 * 4 + 128;
     const unsigned grid = (unsigned)std::min<int64_t>(g.n_units, (int64_t)sms * CTAS);
@@ -567,8 +570,7 @@ ja_status_t row_tma_launch(RowOp op, const RowArgs& a, cudaStream_t st, bool* la
     const ja_dtype_t dt = sizeof(T) == 4 ? JA_F32 : JA_BF16;
     *launched = false;
     if (op == ROW_ROPE) return JA_OK;
-    const char* off_env = getenv("JA_ROW_TMA");
-    if (off_env && off_env[0] == '0') return JA_OK;
+    if (ja_config().row_tma == 0) return JA_OK;
     const int last = a.x.rank - 1;
     const int es = dt == JA_F32 ? 4 : 2, vec = 16 / es;
     const bool has_g = (op == ROW_RMS_SCALE || op == ROW_RMSNORM);
@@ -617,19 +619,15 @@ ja_status_t row_tma_launch(RowOp op, const RowArgs& a, cudaStream_t st, bool* la
     g.stat_blk_bytes = has_stat ? (int)a.s0.blk_stride : 0;
     g.g_blk_bytes = has_g ? (int)a.g.blk_stride : 0;
     g.eps = a.eps;
-    int32_t* status = ja_device_status_word();
+    g.wait_cap_us = (uint32_t)ja_config().wait_cap_us;
+    int32_t* status = ja_device_status_word(st);
     if (!status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
     RowMaps tm;
     ja_status_t s = encode_rows4(a.x, g, n_lead, dt, &tm.x);
     if (s != JA_OK) return s;
     tm.y = tm.x;
     if (has_y && (s = encode_rows4(a.y, g, n_lead, dt, &tm.y)) != JA_OK) return s;
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
-    }
+    const int sms = ja_sm_count();
     s = launch_t<T>(op, tm, a, g, vpl, g_bytes, sms, status, st, launched);
     if (s != JA_OK || !*launched) return s;
     ja_count_launch();

@@ -17,6 +17,16 @@ ES = blocked.equal_splits
 BF, F32 = torch.bfloat16, torch.float32
 ORC_DT = {BF: "bf16", F32: "f32"}
 
+# every attention kernel form, forced through the library's switches (conftest.py puts them back after each test)
+ATTN_FORMS = ["tcgen05_two_tiles", "tcgen05_two_tiles_persistent", "tcgen05_two_tiles_poly_exp", "tcgen05_two_tiles_exp_first", "tcgen05_one_tile", "mma_sync"]
+
+
+def force_attention_form(form):
+    ja.ja_debug_set("attn_mma_sync", 1 if form == "mma_sync" else 0)
+    ja.ja_debug_set("attn_one_tile", 1 if form == "tcgen05_one_tile" else 0)
+    ja.ja_debug_set("attn_persistent", 0 if form == "tcgen05_two_tiles" else 1)
+    ja.ja_debug_set("attn_variant", 1 if form.endswith("poly_exp") else 4 if form.endswith("exp_first") else 0)
+
 
 def _matmul_case(M, J, N, si_, sj, sk, dtype, cfg=1, std_b=1.0):
     A = si.normal((M, J), 0.0, 1.0, dtype, cfg, 1)
@@ -92,8 +102,8 @@ def test_degenerate_tilings_scalar_keys_and_single_block():
     (200, 160, 136, 1, 1, 1),      # one ragged block: 200 rows (128+72), 136 columns
 ])
 @pytest.mark.parametrize("cta_group", ["2", "1"])   # two-SM tiles where the shape allows them / one-SM tiles everywhere
-def test_matmul_tensor_core(M, J, N, gi, gj, gk, cta_group, monkeypatch):
-    monkeypatch.setenv("JA_GEMM_CTA_GROUP", cta_group)
+def test_matmul_tensor_core(M, J, N, gi, gj, gk, cta_group):
+    ja.ja_debug_set("gemm_cta_group", int(cta_group))
     got, ref = _matmul_case(M, J, N, ES(M, gi), ES(J, gj), ES(N, gk), BF, cfg=2, std_b=0.05)
     assert relfro(got, ref) <= TOL[BF]
     # the error must look like bf16 rounding of the output, not like a dropped k-step or a misplaced tile
@@ -242,12 +252,9 @@ def test_rope(splits):
                                                    (1, 256, 1, 64, 64, 1, True), (1, 384, 2, 128, 64, 1, False),
                                                    (1, 512, 1, 256, 128, 1, True), (2, 1024, 3, 128, 256, 3, True),
                                                    (1, 640, 2, 128, 128, 1, False)])
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
-def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
-    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
-    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
-    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
+@pytest.mark.parametrize("form", ATTN_FORMS)
+def test_attention(B, S, H, qb, kb, hb, causal, form):
+    force_attention_form(form)
     D = 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (1, 2, 3))
     spl = lambda blk: [ES(B, B), ES(S, S // blk), ES(H, H // hb), [0, D]]
@@ -265,17 +272,14 @@ def test_attention(B, S, H, qb, kb, hb, causal, form, monkeypatch):
         assert np.array_equal(got[:, 0], si.to_f64(V)[:, 0])   # row 0 joins with key 0 only: O = V[0] exactly
 
 
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ATTN_FORMS)
 @pytest.mark.parametrize("causal", [False, True])
-def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
+def test_attention_scores_that_grow_along_the_keys(causal, form):
     """Keys whose magnitude grows from one 128-row key tile to the next: the running row maximum then outgrows the exponent
     offset in use by more than the 2^8 head-room at almost every key tile, so the kernels take their offset-raising path
     (rescale of the accumulated output, and in the two-tile form the redo of a tile that was exponentiated against the
     old offset) instead of the common one that N(0,1) inputs exercise."""
-    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
-    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
-    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
+    force_attention_form(form)
     B, S, H, D = 1, 1024, 2, 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (31, 32, 33))
     growth = 1.0 + 3.0 * (np.arange(S) // 128)              # score spread x1, x4, x7, ... per key tile
@@ -299,14 +303,11 @@ def test_attention_scores_that_grow_along_the_keys(causal, form, monkeypatch):
     assert np.median(s[:, -128:].max(1) - s[:, :128].max(1)) > 20.0
 
 
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
+@pytest.mark.parametrize("form", ATTN_FORMS)
 @pytest.mark.parametrize("causal,S,hb", [(True, 512, 1), (False, 384, 2), (True, 256, 2)])
-def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
+def test_attention_second_output_lse(causal, S, hb, form):
     """n_outputs = 2: the log of the softmax denominator beside O, and the combine it exists for."""
-    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
-    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
-    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
+    force_attention_form(form)
     B, H, D = 2, 4, 128
     Q, K, V = (si.normal((B, S, H, D), 0.0, 1.0, BF, 4, o) for o in (21, 22, 23))
     sp = [ES(B, B), ES(S, S // 128), ES(H, H // hb), [0, D]]
@@ -336,12 +337,9 @@ def test_attention_second_output_lse(causal, S, hb, form, monkeypatch):
     (2, 768, 6, 2, 2, [768], 256, True),                    # one sequence, grouped heads only
     (1, 1280, 4, 1, 1, [256, 384, 1280], "ends", True),     # blocks of 256, 128, 896 rows
 ])
-@pytest.mark.parametrize("form", ["tcgen05_two_tiles_p_tmem", "tcgen05_two_tiles_p_smem", "tcgen05_two_tiles_p_smem_persistent", "tcgen05_one_tile", "mma_sync"])
-def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut, causal, form, monkeypatch):
-    monkeypatch.setenv("JA_ATTN_MMA_SYNC", "1" if form == "mma_sync" else "0")
-    monkeypatch.setenv("JA_ATTN_ONE_TILE", "1" if form == "tcgen05_one_tile" else "0")
-    monkeypatch.setenv("JA_ATTN_P_SMEM", "1" if form.startswith("tcgen05_two_tiles_p_smem") else "0")
-    monkeypatch.setenv("JA_ATTN_PERSISTENT", "1" if form.endswith("persistent") else "0")
+@pytest.mark.parametrize("form", ATTN_FORMS)
+def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut, causal, form):
+    force_attention_form(form)
     D, grp = 128, Hq // Hkv
     Q = si.normal((B, S, Hq, D), 0.0, 1.0, BF, 4, 11)
     K, V = (si.normal((B, S, Hkv, D), 0.0, 1.0, BF, 4, o) for o in (12, 13))
@@ -372,8 +370,8 @@ def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut
 # ---------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("cta_group", ["2", "1"])
 @pytest.mark.parametrize("M,J,N,gi,gj,gk", [(512, 256, 512, 4, 2, 2), (256, 384, 1024, 2, 3, 8), (512, 512, 256, 2, 1, 2)])
-def test_matmul_fused_chains(M, J, N, gi, gj, gk, cta_group, monkeypatch):
-    monkeypatch.setenv("JA_GEMM_CTA_GROUP", cta_group)
+def test_matmul_fused_chains(M, J, N, gi, gj, gk, cta_group):
+    ja.ja_debug_set("gemm_cta_group", int(cta_group))
     A = si.normal((M, J), 0.0, 1.0, BF, 2, 6)
     W1 = si.normal((J, N), 0.0, 0.06, BF, 2, 7)
     W3 = si.normal((J, N), 0.0, 0.06, BF, 2, 8)
