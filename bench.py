@@ -687,6 +687,46 @@ def case_results(case, reps):
         res["p8_random_20"] = {"ms_mean": sum(ms_sorted) / 20, "ms_min": ms_sorted[0], "ms_median": 0.5 * (ms_sorted[9] + ms_sorted[10]),
                                "ms_max": ms_sorted[-1], "proxy_cost_cells_median": sorted(d_["proxy_cost_cells"] for d_ in draws)[10],
                                "proxy_cost_cells_min": min(d_["proxy_cost_cells"] for d_ in draws), "draws": draws}
+    elif args.case == "optblock":
+        # Section 4 on the whole block: the optimizer's plans for p = 8 and p = 64 function specs per operator
+        # (ja_plan_optimize_graph on the eleven-operator graph, three multiply consumed tensors) executed by PlannedBlock -- a
+        # ja_repartition per repartition charge of the plan -- beside the three hand decompositions of LlamaBlock written as
+        # interval counts of the same graph, so that the proxy cost (cells) and the measured time stand side by side.
+        import time
+        from paper_2609_03905_b200.llama_block import LlamaBlock
+        from paper_2609_03905_b200.planned_block import PlannedBlock, block_graph, plan_repartition_charges
+        shape = SHAPES["7b"]
+        Bt, S, hidden, heads, ffn = shape["batch"], shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
+        ops = block_graph(Bt, S, hidden, heads, ffn)
+        weights = si.llama_weights(hidden, ffn)
+        fl = block_flops(Bt, S, hidden, ffn)
+        sb, fb = S // 128, ffn // 256      # the hand plans cut tokens into 128-row blocks and the FFN index into 256-wide ones
+
+        def hand_counts(e_c, h_proj, h_att, wo_h):
+            tok = {"b": Bt, "s": sb}
+            return [{**tok, "e": e_c}] + [{**tok, "e": e_c, "h": h_proj, "d": 1}] * 3 + \
+                   [{"b": Bt, "q": sb, "h": h_att, "d": 1, "k": sb}, {**tok, "h": wo_h, "d": 1, "e": e_c}, {**tok, "e": e_c},
+                    {**tok, "e": e_c, "f": fb}, {**tok, "e": e_c, "f": fb}, {**tok, "f": fb}, {**tok, "f": fb, "e": e_c}]
+        hands = {"seq": hand_counts(8, 8, heads, 8), "head": hand_counts(heads, heads, heads, heads), "mixed": hand_counts(8, 8, 8, 8)}
+        for name, counts in hands.items():
+            blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=name)
+            t = timeit(lambda r: blk.forward(), reps, True)
+            res["hand_" + name] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "proxy_cost_cells": ja.ja_plan_cost(ops, counts),
+                                   "repartition_charges": plan_repartition_charges(ops, counts)[0], "relayouts_executed": blk.n_relayouts,
+                                   "function_specs_per_matmul": "tokens x %d column blocks" % (len(blk.act_c) - 1)}
+            del blk
+            torch.cuda.empty_cache()
+        for p_ in (8, 64):
+            t0 = time.perf_counter()
+            cost, plan = ja.ja_plan_optimize_graph(ops, p_)
+            opt_ms = (time.perf_counter() - t0) * 1e3
+            blk = PlannedBlock(Bt, S, hidden, heads, ffn, weights, plan)
+            t = timeit(lambda r: blk.forward(), reps, True)
+            res["optimizer_p%d" % p_] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "proxy_cost_cells": cost,
+                                         "repartition_charges": plan_repartition_charges(ops, plan)[0], "relayouts_executed": blk.n_relayouts,
+                                         "optimizer_host_ms": opt_ms, "launches": len(blk.steps), "plan": plan}
+            del blk
+            torch.cuda.empty_cache()
     elif args.case == "chains":
         # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
         # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)
@@ -745,10 +785,11 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="skip the kernels of configurations 1-4 after the headline region")
     ap.add_argument("--config-reps", type=int, default=20, help="timed launches per kernel of configurations 1-4")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "chains"], default="block",
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "
                          "gqa = grouped-query attention over packed sequences; agg = join-only matmul + aggregating relayout; "
-                         "opt = logical optimizer's plan for the MLP tree against hand plans; chains = the five matrix chains")
+                         "opt = logical optimizer's plan for the MLP tree against hand plans; optblock = the optimizer's plans for the whole "
+                         "7B block against the hand decompositions; chains = the five matrix chains")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
     if args.case != "block":

@@ -294,10 +294,12 @@ CHAINS = {   # Section 6: fixed parenthesizations; dimensions divided by `div` k
     "B": ([9216, 20480, 5120, 20480, 5120, 9216], ((0, 1), ((2, 3), 4))),
     "C": ([10240, 12288, 32768, 2048], (0, (1, 2))),
     "D": ([24576, 1536] + [20480] * 6 + [1536, 24576], (0, ((1, (2, (3, (4, (5, (6, 7)))))), 8))),
+    # thirteen matrices with 1024-wide necks: at 1/32 the necks are 32 cells wide, narrower than any tensor-core tile
+    "E": ([49152, 1024] + [20480] * 10 + [1024, 49152], (0, ((1, (2, (3, (4, (5, (6, (7, (8, (9, (10, 11)))))))))), 12))),
 }
 
 
-@pytest.mark.parametrize("name,div", [("A", 32), ("B", 32), ("C", 16), ("D", 32)])
+@pytest.mark.parametrize("name,div", [("A", 32), ("B", 32), ("C", 16), ("D", 32), ("E", 32), ("E", 8)])
 def test_matrix_chain_reduced(name, div):
     """The chain's own parenthesization as a sequence of matmul join-aggs; every intermediate is stored in bf16, and the
     oracle rounds at the same store points. Whole result compared."""
@@ -323,3 +325,83 @@ def test_matrix_chain_reduced(name, div):
     check_status()
     ref = _chain_eval(dims, tree, [si.to_f64(m) for m in mats], lambda A, Bm: core.round_to(A @ Bm, "bf16"))
     assert relfro(got, ref) <= TOL[BF]
+
+
+# ---------------------------------------------------------------------------------------------------
+# whole-output checks at full size (every tile of the launch, not sampled rows)
+# ---------------------------------------------------------------------------------------------------
+def _freivalds(got_bits_rel, A, Bm, R=None, n_vec=3, seed=77):
+    """C = A B (+ R) checked on EVERY row through random projections: for random sign vectors v the oracle side is the
+    fp64 product A (B v) (+ R v), O(n^2); the GPU side is C v from the stored bf16 output. Each stored cell carries one
+    RNE rounding to bf16 (relative error uniform in +-2^-9, standard deviation 2^-9 / sqrt(3)), independent between
+    cells, so row i of C v differs from the exact value by a sum of N such terms: standard deviation
+    2^-9 / sqrt(3) * sqrt(sum_j C_ij^2). The bound is six of those. A tile that is wrong in any visible way (stale,
+    missing one 128-deep chunk of the contraction, shifted by one block) moves its rows by tens of such deviations."""
+    rel = got_bits_rel
+    M, N = rel.extents
+    C = download(rel)                                    # fp64 dense, via the oracle's unpacking
+    rng = np.random.default_rng(seed)
+    A64, B64 = si.to_f64(A), si.to_f64(Bm)
+    R64 = si.to_f64(R) if R is not None else None
+    sigma = (2.0 ** -9) / np.sqrt(3.0) * np.sqrt((C * C).sum(axis=1))
+    worst = 0.0
+    for _ in range(n_vec):
+        v = rng.choice([-1.0, 1.0], size=N)
+        want = A64 @ (B64 @ v)
+        if R64 is not None:
+            want = want + R64 @ v
+        dev = np.abs(C @ v - want) / np.maximum(sigma, 1e-30)
+        worst = max(worst, float(dev.max()))
+        assert dev.max() <= 6.0, f"row {int(dev.argmax())} is {dev.max():.1f} rounding deviations off"
+        # and the same through the columns: u C against (u A) B, so that a defect confined to some columns shows in them
+        u = rng.choice([-1.0, 1.0], size=M)
+        want_c = (u @ A64) @ B64
+        if R64 is not None:
+            want_c = want_c + u @ R64
+        sigma_c = (2.0 ** -9) / np.sqrt(3.0) * np.sqrt((C * C).sum(axis=0))
+        dev_c = np.abs(u @ C - want_c) / np.maximum(sigma_c, 1e-30)
+        assert dev_c.max() <= 6.0, f"column {int(dev_c.argmax())} is {dev_c.max():.1f} rounding deviations off"
+    return worst
+
+
+@pytest.mark.parametrize("which", ["up_projection_ragged_blocks", "down_projection_add", "block_up_projection_256_wide"])
+def test_full_size_matmul_every_tile_by_random_projection(which):
+    """The tensor-core matmul launches of configurations 2 and 5 at full size, whole output: the banded / heavy-first tile
+    schedules, ragged 1376-wide blocks and the fused residual add are all in play; every output row and column is
+    checked (sampled-row tests cannot see a defect confined to a late row band of one schedule)."""
+    if which == "up_projection_ragged_blocks":          # config 2: x [2048, 4096] W1 [4096, 11008], 8 x 8 x 8
+        M, J, N, gi, gj, gk = 2048, 4096, 11008, 8, 8, 8
+    elif which == "down_projection_add":                # config 5: h [16384, 11008] W2 [11008, 4096] + residual, block tilings
+        M, J, N, gi, gj, gk = 16384, 11008, 4096, 128, 43, 8
+    else:                                               # config 5: n2 [16384, 4096] W1 [4096, 11008], 256-wide FFN blocks
+        M, J, N, gi, gj, gk = 16384, 4096, 11008, 128, 8, 43
+    A = si.normal((M, J), 0.0, 1.0, BF, 9, 1)
+    Bm = si.normal((J, N), 0.0, 0.02, BF, 9, 2)
+    ti, tj, tk = ES(M, gi), ES(J, gj), ES(N, gk)
+    rA, rB = upload(A, [ti, tj]), upload(Bm, [tj, tk])
+    rC = empty_like_tiling([M, N], [ti, tk], BF, fill=float("nan"))
+    if which == "down_projection_add":
+        R = si.normal((M, N), 0.0, 1.0, BF, 9, 3)
+        rR = upload(R, [ti, tk])
+        ja.Spec("ij,jk,ik->ik", {"i": ti, "j": tj, "k": tk}, "matmul_add", (), "sum").execute([rA, rB, rR], rC)
+    else:
+        R = None
+        ja.Spec("ij,jk->ik", {"i": ti, "j": tj, "k": tk}).execute([rA, rB], rC)
+    check_status()
+    _freivalds(rC, A, Bm, R)
+
+
+def test_config5_llama_7b_block_second_sampled_sequence():
+    """The 7B block once more on another sequence of the batch (sequence 2, first 256 tokens), so that the sampled-row
+    check does not rest on one sequence's tiles alone."""
+    Bt, S, hidden, heads, ffn, prefix, seq_id = 8, 2048, 4096, 32, 11008, 256, 2
+    w = si.llama_weights(hidden, ffn)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 0)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan="seq", fused=True)
+    ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
+    out = download(blk.forward())
+    check_status()
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, prefix - 1], np.linspace(0, prefix - 1, 6).astype(int)]))
+    xs = si.to_f64(x[seq_id * S: seq_id * S + prefix])
+    ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows)["out"]
+    assert relfro(out[seq_id * S + rows], ref) <= TOL[BF]
