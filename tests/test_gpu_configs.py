@@ -333,17 +333,20 @@ def test_matrix_chain_reduced(name, div):
 def _freivalds(got_bits_rel, A, Bm, R=None, n_vec=3, seed=77):
     """C = A B (+ R) checked on EVERY row through random projections: for random sign vectors v the oracle side is the
     fp64 product A (B v) (+ R v), O(n^2); the GPU side is C v from the stored bf16 output. Each stored cell carries one
-    RNE rounding to bf16 (relative error uniform in +-2^-9, standard deviation 2^-9 / sqrt(3)), independent between
-    cells, so row i of C v differs from the exact value by a sum of N such terms: standard deviation
-    2^-9 / sqrt(3) * sqrt(sum_j C_ij^2). The bound is six of those. A tile that is wrong in any visible way (stale,
-    missing one 128-deep chunk of the contraction, shifted by one block) moves its rows by tens of such deviations."""
+    RNE rounding to bf16: an absolute error uniform in +-ulp/2 with ulp = 2^(floor(log2 |c|) - 7), standard deviation
+    ulp / sqrt(12), independent between cells, so row i of C v differs from the exact value by a sum of N such terms with
+    standard deviation sqrt(sum_j ulp_ij^2 / 12). The bound is six of those (about 50 000 rows and columns are looked at;
+    a six-sigma excursion of a sum of thousands of bounded terms has probability 2e-9 each). A tile that is wrong in any
+    visible way (stale, missing one 128-deep chunk of the contraction, shifted by one block) moves its rows by tens of
+    such deviations."""
     rel = got_bits_rel
     M, N = rel.extents
     C = download(rel)                                    # fp64 dense, via the oracle's unpacking
     rng = np.random.default_rng(seed)
     A64, B64 = si.to_f64(A), si.to_f64(Bm)
     R64 = si.to_f64(R) if R is not None else None
-    sigma = (2.0 ** -9) / np.sqrt(3.0) * np.sqrt((C * C).sum(axis=1))
+    ulp2 = np.exp2(2.0 * (np.floor(np.log2(np.maximum(np.abs(C), 1e-30))) - 7.0)) / 12.0     # variance of one cell's rounding
+    sigma = np.sqrt(ulp2.sum(axis=1))
     worst = 0.0
     for _ in range(n_vec):
         v = rng.choice([-1.0, 1.0], size=N)
@@ -358,7 +361,7 @@ def _freivalds(got_bits_rel, A, Bm, R=None, n_vec=3, seed=77):
         want_c = (u @ A64) @ B64
         if R64 is not None:
             want_c = want_c + u @ R64
-        sigma_c = (2.0 ** -9) / np.sqrt(3.0) * np.sqrt((C * C).sum(axis=0))
+        sigma_c = np.sqrt(ulp2.sum(axis=0))
         dev_c = np.abs(u @ C - want_c) / np.maximum(sigma_c, 1e-30)
         assert dev_c.max() <= 6.0, f"column {int(dev_c.argmax())} is {dev_c.max():.1f} rounding deviations off"
     return worst
