@@ -928,7 +928,7 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
             }
             if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
         }
-        return ja_launch_matmul_simt(ja_view(A), ja_view(B), ja_view(out), A->dtype, stream);
+        return ja_launch_matmul_simt(A, B, out, stream);
     }
 
     // ---- fused chains on the tensor-core matmul -------------------------------------------------------------------
@@ -1193,7 +1193,7 @@ extern "C" ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_
             if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
         }
         if (partials->dtype != A->dtype) return ja_fail(JA_ERR_UNSUPPORTED, "this tiling needs a partial relation of the operands' dtype");
-        return ja_launch_matmul_simt(ja_view(A), ja_view(B), ja_view(partials), A->dtype, stream, true);
+        return ja_launch_matmul_simt(A, B, partials, stream, true);
     }
     return ja_fail(JA_ERR_UNSUPPORTED, "join-only execution has no kernel for einsum '%s' with fn %d / agg %d", spec->einsum.c_str(),
                    (int)spec->fn, (int)spec->agg);

@@ -108,9 +108,10 @@ JaConfig& ja_config();
     } while (0)
 
 // ---- kernel launchers (one per .cu file) ------------------------------------------------------------
-// Plain-ALU tiled matmul join-agg over arbitrary tilings (f32 or bf16 operands, f32 accumulate).
-ja_status_t ja_launch_matmul_simt(const RelView& A, const RelView& B, const RelView& C, ja_dtype_t dt,
-                                  cudaStream_t st, bool partials = false);
+// Plain-ALU tiled matmul join-agg over arbitrary tilings (f32 or bf16 operands, f32 accumulate). The key tables of the
+// three relations must be on the device (ja_relation_to_device).
+ja_status_t ja_launch_matmul_simt(const ja_relation* A, const ja_relation* B, const ja_relation* C, cudaStream_t st,
+                                  bool partials = false);
 
 // Memory-bound join-aggs: flat key-aligned maps and row-structured maps / reductions.
 enum RowOp {
