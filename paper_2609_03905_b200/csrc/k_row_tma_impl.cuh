@@ -108,7 +108,7 @@ __device__ __forceinline__ float team_reduce(Team& t, float v, int lane) {
 // ---- one row, any cell type: plain scalar arithmetic --------------------------------------------------------
 template <typename T, int OP, int VPL>
 __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL],
-                                            const uint8_t* g_s, int64_t stat_off, int lane, Team& team) {
+                                            const uint8_t* g_s, int64_t stat_off, float pre0, float pre1, int lane, Team& team) {
     constexpr int VEC = 16 / (int)sizeof(T);
     using V = RVec<T, VEC>;
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
@@ -147,7 +147,7 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
             return;
         }
     }
-    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = pre0;
     if (OP == ROW_EXPSUM || OP == ROW_SOFTMAX) {
         float sacc = 0.f;
 #pragma unroll
@@ -167,9 +167,9 @@ __device__ __forceinline__ void row_generic(const RowArgs& a, const RowTmaGeom& 
             return;
         }
     }
-    if (OP == ROW_EXP_SUB_DIV) l = *reinterpret_cast<const float*>(a.s1.base + stat_off);
+    if (OP == ROW_EXP_SUB_DIV) l = pre1;
     if (OP == ROW_RMS_SCALE) {
-        const float ss = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+        const float ss = pre0;
         rstd = 1.0f / sqrtf(ss / (float)g.n + g.eps);
     }
     const float inv_l = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : 0.f;
@@ -235,7 +235,7 @@ __device__ __forceinline__ uint32_t narrow(uint64_t v) {   // two f32 -> packed 
 // over them is straight-line code that the compiler can interleave; otherwise each vector is guarded.
 template <int OP, int VPL, bool FULL>
 __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, uint8_t* rowp, const int (&off)[VPL], const uint8_t* g_s,
-                                         int64_t stat_off, int lane, Team& team) {
+                                         int64_t stat_off, float pre0, float pre1, int lane, Team& team) {
     constexpr bool HAS_G = (OP == ROW_RMS_SCALE || OP == ROW_RMSNORM);
     constexpr bool KEEP_EXP = (OP == ROW_SOFTMAX);
     constexpr float LOG2E = 1.4426950408889634f;
@@ -279,7 +279,7 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
             return;
         }
     }
-    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+    if (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV) m = pre0;
     const uint64_t sc2 = pk2(LOG2E, LOG2E), nm2 = pk2(-m * LOG2E, -m * LOG2E);
     auto exp_pair = [&](uint32_t w) {
         float t0, t1;
@@ -308,9 +308,9 @@ __device__ __forceinline__ void row_bf16(const RowArgs& a, const RowTmaGeom& g, 
             return;
         }
     }
-    if (OP == ROW_EXP_SUB_DIV) l = *reinterpret_cast<const float*>(a.s1.base + stat_off);
+    if (OP == ROW_EXP_SUB_DIV) l = pre1;
     if (OP == ROW_RMS_SCALE) {
-        const float ss = *reinterpret_cast<const float*>(a.s0.base + stat_off);
+        const float ss = pre0;
         rstd = 1.0f / sqrtf(ss / (float)g.n + g.eps);
     }
     const float scale = (OP == ROW_SOFTMAX || OP == ROW_EXP_SUB_DIV) ? 1.0f / l : rstd;
@@ -468,23 +468,56 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
         team.abort_flag = abort_flag;
         team.status = status;
         team.ok = true;
+        // Input statistics of a row (m for EXP_SUB, m and l for EXP_SUB_DIV, the sum of squares for RMS_SCALE) are loaded one
+        // unit AHEAD: a row's arithmetic cannot start without them, and a load issued when the row's turn comes is a cold
+        // global access in front of every row. (On the 268 MB exp-SUM join-agg this measured the same as loading them in
+        // place, 65 us: that kernel is bound by its warps' own dependent instruction chains -- one CTA per SM takes 94 us,
+        // two 65 us, three, with two stages each instead of three, 72 us.)
+        constexpr bool PRE0 = (OP == ROW_EXPSUM || OP == ROW_EXP_SUB_DIV || OP == ROW_RMS_SCALE), PRE1 = (OP == ROW_EXP_SUB_DIV);
+        constexpr int MAXR = 4;   // rows of one unit that one team handles: at most 32 rows per unit over 8 teams
+        float nxt0[MAXR], nxt1[MAXR];
+        auto prefetch_stats = [&](int64_t u) {
+#pragma unroll
+            for (int q = 0; q < MAXR; ++q) { nxt0[q] = 0.f; nxt1[q] = 0.f; }
+            if (!PRE0 || u >= g.n_units) return;
+            int64_t lb;
+            int r0, rows;
+            unit_geom(u, &lb, &r0, &rows);
+#pragma unroll
+            for (int q = 0; q < MAXR; ++q) {
+                const int r = tid + q * n_teams;
+                if (r < rows) {
+                    const int64_t so = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
+                    nxt0[q] = *reinterpret_cast<const float*>(a.s0.base + so);
+                    if (PRE1) nxt1[q] = *reinterpret_cast<const float*>(a.s1.base + so);
+                }
+            }
+        };
+        prefetch_stats(first);
         int64_t i = 0;
         for (int64_t u = first; u < g.n_units && team.ok; u += step, ++i) {
             const int s = (int)(i % g.stages);
             const uint32_t ph = (uint32_t)(i / g.stages) & 1;
+            float cur0[MAXR], cur1[MAXR];
+#pragma unroll
+            for (int q = 0; q < MAXR; ++q) { cur0[q] = nxt0[q]; cur1[q] = nxt1[q]; }
+            prefetch_stats(u + step);
             if (!mbar_wait(full_bar(s), ph, abort_flag, status)) { team.ok = false; break; }
             int64_t lb;
             int r0, rows;
             unit_geom(u, &lb, &r0, &rows);
             uint8_t* stage = smem + (size_t)s * g.stage_bytes;
-            for (int r = tid; r < rows && team.ok; r += n_teams) {
+#pragma unroll
+            for (int q = 0; q < MAXR; ++q) {
+                const int r = tid + q * n_teams;
+                if (r >= rows || !team.ok) break;
                 uint8_t* rowp = stage + (size_t)r * row_seg_bytes;
                 const int64_t stat_off = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
                 if constexpr (sizeof(T) == 2) {
-                    if (full_rows) row_bf16<OP, VPL, true>(a, g, rowp, off, g_s, stat_off, lane, team);
-                    else row_bf16<OP, VPL, false>(a, g, rowp, off, g_s, stat_off, lane, team);
+                    if (full_rows) row_bf16<OP, VPL, true>(a, g, rowp, off, g_s, stat_off, cur0[q], cur1[q], lane, team);
+                    else row_bf16<OP, VPL, false>(a, g, rowp, off, g_s, stat_off, cur0[q], cur1[q], lane, team);
                 }
-                else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, lane, team);
+                else row_generic<T, OP, VPL>(a, g, rowp, off, g_s, stat_off, cur0[q], cur1[q], lane, team);
             }
             if (!team.ok) break;
             if (HAS_Y) fence_async_smem();    // this thread's writes to the stage become visible to the bulk stores
