@@ -528,7 +528,8 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], int k
 //   box of that run): no P stores -6 %, no exponentials -7 %, QK^T or P V reduced to one instruction of eight -6 % / 0 %,
 //   no K / V loads -10 %, no output stage -3 %; all of them together still leave 0.067 ms: the row threads' own
 //   instruction stream (two row warps per scheduler, ~420 instructions per row and key tile, issued in order) and the
-//   barrier hand-offs between the roles bound the kernel, not one of the units.
+//   barrier hand-offs between the roles bound the kernel, not one of the units. Also measured and not kept: on the diagonal
+//   tile, skipping the keys that no row of a warp may see (half of that tile's exponentials on average): 2-3 % SLOWER.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int NUM_THREADS2 = 320;
 constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
