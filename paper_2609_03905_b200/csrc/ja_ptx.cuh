@@ -48,13 +48,19 @@ __device__ __forceinline__ uint64_t global_ns() {
 // word, raises the abort flag so that every other role of the CTA gives up at its next check, and returns false; the
 // caller leaves through the kernel's normal exit. The loop itself is ja_bounded_wait (ja_wait.h), which is also
 // compiled for the host and tested there against a scripted barrier and clock.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
+// The polling loop is kept out of line: a kernel has dozens of wait sites, and their code competes with the hot loops for the
+// instruction cache (measured on the attention kernel: instruction-fetch stalls were a tenth of its time).
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
     return ja_bounded_wait([&] { return mbar_try_wait(bar, parity); }, [] { return global_ns(); }, [&] { return ctl[0] != 0; },
                            [&] {
                                ctl[0] = 1;
                                atomicExch(status, (int)JA_ERR_TIMEOUT);
                            },
                            (uint64_t)(uint32_t)ctl[1] * 1000ull);
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, ctl, status);
 }
 // what a CTA's first thread writes into the two control words before any wait
 __device__ __forceinline__ void wait_ctl_init(volatile int* ctl, uint32_t cap_us) {

@@ -310,7 +310,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const bool diag = p.causal && (j == n_steps - 1);
             const int kmax = q0 + r - (s0 + j * KT); // columns c > kmax of this tile lie after the query row
             // ---- pass 1: row maximum ----
-            float mx = -INFINITY;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains, not one of 128 links
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t v[32];
@@ -320,9 +320,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int i = 0; i < 32; ++i) {
                     float s = __uint_as_float(v[i]);
                     if (diag && c * 32 + i > kmax) s = -INFINITY;
-                    mx = fmaxf(mx, s);
+                    mx4[i & 3] = fmaxf(mx4[i & 3], s);
                 }
             }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_run, mx * p.scale_log2e);
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;           // e^(-inf - -inf) := 0
             const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_use);
@@ -417,15 +418,8 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     return d;
 }
 
-// maximum of one row of scores (128 fp32 bit patterns); MASK: columns > kmax lie after the query row
-template <bool MASK>
-__device__ __forceinline__ float row_max128(const uint32_t (&v)[128], int kmax) {
-    if (MASK) {
-        float mx = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 128; ++i) mx = fmaxf(mx, i > kmax ? -INFINITY : __uint_as_float(v[i]));
-        return mx;
-    }
+// maximum of one row of scores (128 fp32 bit patterns): four chains of 3-input maxima
+__device__ __forceinline__ float row_max128(const uint32_t (&v)[128]) {
     float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]), m2 = __uint_as_float(v[2]), m3 = __uint_as_float(v[3]);
 #pragma unroll
     for (int i = 4; i + 7 < 128; i += 8) {
@@ -464,10 +458,11 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 }
 
 // One row of P = 2^(S * scale - m) for 128 keys as 64 packed bf16 pairs in registers; returns the row sum (f32, of the
-// unrounded values). MASK: keys > kmax lie after the query row and get P = 0. POLY: how many of the four pairs of every
-// group of eight keys take the FMA-pipe exponential instead of ex2 (0, 1 or 2), interleaved so that both pipes stay busy.
-template <bool MASK, int POLY>
-__device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], int kmax, float scale, float m_used, uint32_t (&pk)[64]) {
+// unrounded values); a score of -inf (a masked key) gives exactly 0. POLY: which pairs of every group of eight keys take the
+// FMA-pipe exponential instead of ex2 -- 0 none, 1 one of four, 2 two of four, 3 one of eight -- interleaved so that both
+// pipes stay busy.
+template <int POLY>
+__device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float scale, float m_used, uint32_t (&pk)[64]) {
     const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
     uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
 #pragma unroll
@@ -477,17 +472,13 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], int k
             const int col = cc * 8 + i;
             const uint64_t x2 = fma2(pack2(__uint_as_float(v[col]), __uint_as_float(v[col + 1])), sc2, nm2);
             float p0, p1;
-            const bool poly = (POLY == 1 && i == 6) || (POLY == 2 && (i == 2 || i == 6));
+            const bool poly = (POLY == 1 && i == 6) || (POLY == 2 && (i == 2 || i == 6)) || (POLY == 3 && i == 6 && (cc & 1));
             if (poly) {
                 exp2_poly_pair(x2, p0, p1);
             } else {
                 unpack2(x2, p0, p1);
                 p0 = ex2(p0);
                 p1 = ex2(p1);
-            }
-            if (MASK) {
-                if (col > kmax) p0 = 0.f;
-                if (col + 1 > kmax) p1 = 0.f;
             }
             if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
             else sum_b = add2(sum_b, pack2(p0, p1));
@@ -521,16 +512,16 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], int k
 //   two-entry queue in shared memory, and runs ahead into the next item as soon as the Q buffers are free, so the next
 //   item's Q and first K tile load, and its first Q K^T run, while the row threads finish this item. Barrier phases follow
 //   running counters (items; key steps per tile). Otherwise one CTA per item, handed out by the hardware in grid order.
-// VAR selects row-thread variants that were built, verified against the oracle and measured slower on this part (kept
-//   selectable for A/B runs, "attn_variant"): bits 0-1 = POLY of row_exp_pack128 (a quarter or half of the exponentials on
-//   the FMA pipe: +1 % / +8 % time on B4 S2048 causal); bit 2 = exponentiate into registers first and wait for the P tile
-//   only before storing (+3 %). 0 = the default. Timing-only ablations of this kernel (B4 S2048 H32 causal, 0.163 ms on the
-//   box of that run): no P stores -6 %, no exponentials -7 %, QK^T or P V reduced to one instruction of eight -6 % / 0 %,
-//   no K / V loads -10 %, no output stage -3 %; all of them together still leave 0.067 ms: the row threads' own
-//   instruction stream (two row warps per scheduler, ~420 instructions per row and key tile, issued in order) and the
-//   barrier hand-offs between the roles bound the kernel, not one of the units. Also measured and not kept: on the diagonal
-//   tile, skipping the keys that no row of a warp may see (half of that tile's exponentials on average): 2-3 % SLOWER.
-// ---------------------------------------------------------------------------------------------------------
+// VAR selects row-thread variants ("attn_variant"; all verified against the oracle): bits 0-1 = POLY of row_exp_pack128, bit 2 =
+//   exponentiate into registers first and wait for the P tile only before storing. Default 1: a quarter of the exponentials
+//   on the FMA pipe (B4 S2048 H32 causal, same run: POLY 0 0.1430 ms, one of eight 0.1405, one of four 0.1403, two of four
+//   0.1509; exponentials first 0.1542).
+// Timing-only ablations of this kernel before the masked loops were merged (B4 S2048 H32 causal, 0.163 ms on the box of
+//   that run): no P stores -6 %, no exponentials -7 %, QK^T or P V reduced to one instruction of eight -6 % / 0 %, no K / V
+//   loads -10 %, no output stage -3 %; all of them together still left 0.067 ms: the row threads' own instruction stream (two
+//   row warps per scheduler, several hundred instructions per row and key tile, issued in order) and the hand-offs between
+//   the roles bound the kernel, not one of the units. Also measured and not kept: on the diagonal tile, skipping the keys
+//   that no row of a warp may see (half of that tile's exponentials on average): 2-3 % slower.
 constexpr int NUM_THREADS2 = 320;
 constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
 
@@ -780,7 +771,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(S_FREE + t));   // S_t is in registers: the next Q K^T of this tile may run
-                const float mx = diag ? row_max128<true>(v, kmax) : row_max128<false>(v, kmax);
+                if (diag) {   // Keys after the query row score -inf: they lose every maximum and exponentiate to exactly 0, so ONE copy of
+                              // the maximum / exponential code serves masked and unmasked tiles. (A masked variant of both loops --
+                              // a select per score inside them, the maximum as one chain of 128 dependent selects -- cost 12 % of
+                              // the kernel on B4 S2048: the chain sits on every item's critical path, and the second copy of the
+                              // unrolled loops on the instruction cache.)
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i > kmax) v[i] = 0xff800000u;
+                }
+                const float mx = row_max128(v);
                 const float m_new = mx * p.scale_log2e;        // finite: the first key of a sequence is never masked
                 // lazy rescale: raise the offset only when the row maximum outgrew it by more than 2^8
                 float alpha = 1.f;
@@ -815,8 +815,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     l_run *= alpha;
                 }
                 uint32_t pk[64];
-                l_run += diag ? row_exp_pack128<true, POLY>(v, kmax, p.scale_log2e, m_used, pk)
-                              : row_exp_pack128<false, POLY>(v, kmax, p.scale_log2e, m_used, pk);
+                l_run += row_exp_pack128<POLY>(v, p.scale_log2e, m_used, pk);
                 if (!(WAIT_FIRST || rescale)) {
                     if (!wait_p_tile()) { ok = false; break; }
                 }
@@ -838,8 +837,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const int64_t cell = (int64_t)seq_row(p.q, p.S, it.b, qrow, it.h) * p.q.hblk + it.h % p.q.hblk;
                 p.lse_base[cell] = (m_used + log2f(l_run)) * 0.6931471805599453f;   // l is relative to the offset m_used
             }
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll 1
+            for (int cc = 0; cc < 4; ++cc) {   // not unrolled: the output stage runs once per item, and code size costs instruction fetches
                 uint32_t o[32];
                 tmem_ld32(tO + cc * 32, o);
                 tmem_ld_wait();
@@ -939,6 +938,7 @@ ja_status_t launch_two_tiles(int variant, dim3 grid, cudaStream_t st, const CUte
     switch (variant) {
         JA_ATTN_LAUNCH(0)
         JA_ATTN_LAUNCH(1)
+        JA_ATTN_LAUNCH(3)
         JA_ATTN_LAUNCH(4)
         default: return ja_fail(JA_ERR_INVALID_ARG, "unknown attention variant %d", variant);
     }
@@ -1020,7 +1020,7 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
             for (int i = 1; i < a.n_ends; ++i) longest = std::max(longest, a.ends[i] - a.ends[i - 1]);
         }
         const bool persist = cfg.attn_persistent >= 0 ? cfg.attn_persistent == 1 : longest <= 4096;
-        const int variant = cfg.attn_variant >= 0 ? cfg.attn_variant : 0;
+        const int variant = cfg.attn_variant >= 0 ? cfg.attn_variant : 1;
         ja_status_t s;
         if (persist) {
             int32_t* queues = nullptr;

@@ -25,7 +25,7 @@ def force_attention_form(form):
     ja.ja_debug_set("attn_mma_sync", 1 if form == "mma_sync" else 0)
     ja.ja_debug_set("attn_one_tile", 1 if form == "tcgen05_one_tile" else 0)
     ja.ja_debug_set("attn_persistent", 0 if form == "tcgen05_two_tiles" else 1)
-    ja.ja_debug_set("attn_variant", 1 if form.endswith("poly_exp") else 4 if form.endswith("exp_first") else 0)
+    ja.ja_debug_set("attn_variant", 3 if form.endswith("poly_exp") else 4 if form.endswith("exp_first") else 0 if form == "tcgen05_two_tiles" else -1)
 
 
 def _matmul_case(M, J, N, si_, sj, sk, dtype, cfg=1, std_b=1.0):
