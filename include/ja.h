@@ -148,8 +148,10 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  * (a cudaStream_t passed as void*; NULL = the legacy default stream), asynchronously.
  * inputs[k] must be tiled exactly as in_k(J), outputs[0] as out(J) (else JA_ERR_PARTITION_MISMATCH).
  * Supported forms (letters are free; shapes of the signature matter):
- *   "ij,jk->ik"            MUL / SUM        bf16 or f32 operands, f32 accumulate (tensor cores for bf16 on
- *                                            uniform 16-byte-aligned blocks, plain ALUs otherwise)
+ *   "ij,jk->ik"            MUL / SUM        bf16 or f32 operands, f32 accumulate. bf16: tensor cores under every tiling
+ *                                            (operands fetched by TMA on uniform blocks with 16-byte rows, by plain
+ *                                            asynchronous loads otherwise; plain ALUs only where blocks are smaller than
+ *                                            64 cells a side); f32: plain ALUs
  *   "ij,jk,ik->ik"         MATMUL_ADD / SUM   } fused chains: the accumulator of the contraction goes through the
  *   "ij,jk->ik"            MATMUL_ROPE / SUM  } next join-agg before its single rounding and store; bf16 relations
  *   "ij,jk,jk->ik"         SWIGLU_UP / SUM    } on uniform blocks only (JA_ERR_UNSUPPORTED otherwise: run the chain)

@@ -920,13 +920,18 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         const ja_relation *A = inputs[0], *B = inputs[1];
         if (A->dtype != B->dtype || A->dtype != out->dtype) return ja_fail(JA_ERR_DTYPE, "matmul operands must share one dtype");
         if (A->dtype == JA_BF16) {
+            const int loader = ja_config().gemm_loader;
             if (!plan->gemm_checked) {
                 bool ok = false;
                 if ((st = ja_gemm_tc_plan(A, B, out, nullptr, &plan->gemm, &ok)) != JA_OK) return st;
                 if (!ok) plan->gemm.reset();
                 plan->gemm_checked = true;
             }
-            if (plan->gemm) return ja_launch_gemm_tc(*plan->gemm, stream);
+            if (plan->gemm && loader != 1) return ja_launch_gemm_tc(*plan->gemm, stream);
+            if (loader != 0) {   // tilings TMA cannot address: the tensor cores fed by plain loads
+                bool launched = false;
+                if ((st = ja_launch_gemm_ld(A, B, out, stream, &launched)) != JA_OK || launched) return st;
+            }
         }
         return ja_launch_matmul_simt(A, B, out, stream);
     }

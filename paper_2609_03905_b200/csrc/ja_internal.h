@@ -94,7 +94,7 @@ struct JaConfig {
     int gemm_group_m = -1;      // JA_GEMM_GROUP_M      n: row tiles per rasterisation band
     int gemm_heavy_first = -1;  // JA_GEMM_HEAVY_FIRST  0: plain tile order
     int gemm_split = -1;        // JA_GEMM_SPLIT        0: the last partial wave is not split along the contracted index
-    int gemm_loader = -1;       // JA_GEMM_LOADER       1: operands staged by plain loads even where TMA could take them
+    int gemm_loader = -1;       // JA_GEMM_LOADER       1: operands staged by plain loads even where TMA could take them; 0: never
     int row_tma = -1;           // JA_ROW_TMA           0: row join-aggs without the TMA-staged kernel
     int row_team = -1;          // JA_ROW_TEAM          n: threads per row of the plain row kernel
     int64_t wait_cap_us = 2000000;   // JA_WAIT_CAP (nanoseconds in the environment): limit of every device-side wait
@@ -112,6 +112,10 @@ JaConfig& ja_config();
 // three relations must be on the device (ja_relation_to_device).
 ja_status_t ja_launch_matmul_simt(const ja_relation* A, const ja_relation* B, const ja_relation* C, cudaStream_t st,
                                   bool partials = false);
+
+// tcgen05 matmul join-agg for bf16 relations under any tiling, operands staged by plain loads (k_gemm_ld.cu); *launched
+// stays false when the blocks are too small for its tiles. Key tables must be on the device.
+ja_status_t ja_launch_gemm_ld(const ja_relation* A, const ja_relation* B, const ja_relation* C, cudaStream_t st, bool* launched);
 
 // Memory-bound join-aggs: flat key-aligned maps and row-structured maps / reductions.
 enum RowOp {

@@ -110,6 +110,30 @@ def test_matmul_tensor_core(M, J, N, gi, gj, gk, cta_group):
     assert np.abs(got - ref).max() <= 2.0 ** -7 * np.abs(ref).max() + 1e-6
 
 
+# the same contraction with operands staged by plain loads: the tensor-core form for tilings TMA cannot address
+@pytest.mark.parametrize("M,J,N,si_,sj,sk", [
+    (256, 256, 512, ES(256, 2), ES(256, 2), ES(512, 2)),                   # TMA-friendly blocks, loader forced
+    (384, 704, 640, ES(384, 3), ES(704, 2), ES(640, 1)),                   # 352-deep blocks (5.5 stages), three column tiles
+    (512, 1376, 344, ES(512, 2), ES(1376, 8), ES(344, 2)),                 # 172-cell block rows: 8-byte aligned only
+    (300, 330, 270, [0, 100, 300], [0, 130, 330], [0, 135, 270]),          # odd widths: 2-byte aligned rows, ragged everything
+    (260, 200, 522, [0, 129, 260], [0, 67, 200], [0, 261, 522]),           # irregular blocks a cell past a tile / stage boundary
+    (1024, 96, 256, ES(1024, 1), ES(96, 1), ES(256, 1)),                   # one block, 96-deep: a stage and a half
+])
+def test_matmul_tensor_core_plain_load_form(M, J, N, si_, sj, sk):
+    ja.ja_debug_set("gemm_loader", 1)
+    before = ja.ja_launch_count()
+    got, ref = _matmul_case(M, J, N, si_, sj, sk, BF, cfg=2, std_b=0.05)
+    assert ja.ja_launch_count() == before + 1
+    assert relfro(got, ref) <= TOL[BF]
+    assert np.abs(got - ref).max() <= 2.0 ** -7 * np.abs(ref).max() + 1e-6
+    # the plain-ALU kernel on the same tiling gives the same result up to its different summation order
+    ja.ja_debug_set("gemm_loader", 0)
+    ja.ja_debug_set("gemm_cta_group", 1)
+    if any(len(set(np.diff(sp))) > 1 or np.diff(sp)[0] % 8 for sp in (sj, sk)) or len(set(np.diff(si_))) > 1:
+        alu, _ = _matmul_case(M, J, N, si_, sj, sk, BF, cfg=2, std_b=0.05)      # this tiling has no TMA form: plain ALUs
+        assert relfro(got, alu) <= 1e-2
+
+
 def test_matmul_tensor_core_identity_is_exact():
     M = 256
     A = si.normal((M, M), 0.0, 1.0, BF, 2, 3)
