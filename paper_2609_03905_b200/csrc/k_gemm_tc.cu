@@ -35,9 +35,8 @@ using namespace ja_ptx;
 
 constexpr int BM = 128, BN = 256;
 constexpr int NUM_THREADS = 192;
-// BK = contraction depth of one pipeline stage. TMA throughput grows with the box size (measured on this part:
-// 8 KiB boxes ~10 TB/s, 16 KiB ~12.7 TB/s aggregate), so the two-CTA form stages 128-deep chunks: every box it
-// issues (A: 128 rows x 64 k, B: 128 k x 64 columns) is 16 KiB.
+// BK = contraction depth of one pipeline stage. The two-CTA form stages 128-deep chunks so that every box it issues
+// (A: 128 rows x 64 k, B: 128 k x 64 columns) is 16 KiB: fewer, larger TMA copies per flop than 64-deep stages.
 template <int CG> struct Cfg {
     static constexpr int BK = CG == 1 ? 64 : 128;
     static constexpr int STAGES = CG == 1 ? 4 : 3;
