@@ -521,7 +521,9 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   loads -10 %, no output stage -3 %; all of them together still left 0.067 ms: the row threads' own instruction stream (two
 //   row warps per scheduler, several hundred instructions per row and key tile, issued in order) and the hand-offs between
 //   the roles bound the kernel, not one of the units. Also measured and not kept: on the diagonal tile, skipping the keys
-//   that no row of a warp may see (half of that tile's exponentials on average): 2-3 % slower.
+//   that no row of a warp may see (half of that tile's exponentials on average): 2-3 % slower; TMA prefetches into L2
+//   (the next item's Q and first K / V tiles, claimed one item early, and the tiles two key steps ahead): 20 % slower --
+//   the prefetches queue in front of the loads the products wait for; claiming one item early alone: 2 % slower.
 constexpr int NUM_THREADS2 = 320;
 constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
 
