@@ -523,7 +523,9 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   the roles bound the kernel, not one of the units. Also measured and not kept: on the diagonal tile, skipping the keys
 //   that no row of a warp may see (half of that tile's exponentials on average): 2-3 % slower; TMA prefetches into L2
 //   (the next item's Q and first K / V tiles, claimed one item early, and the tiles two key steps ahead): 20 % slower --
-//   the prefetches queue in front of the loads the products wait for; claiming one item early alone: 2 % slower.
+//   the prefetches queue in front of the loads the products wait for; claiming one item early alone: 2 % slower; issuing
+//   the tensor-memory loads of the next key step's scores before handing P over (when they are already complete): 20 %
+//   slower.
 constexpr int NUM_THREADS2 = 320;
 constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
 
