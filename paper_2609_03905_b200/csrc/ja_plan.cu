@@ -112,10 +112,16 @@ void enum_specs(const Op& op, int32_t p, size_t l, Counts* cur, std::vector<Coun
     }
 }
 
-struct Choice {
-    Counts spec;
-    std::vector<Counts> in_tilings;   // chosen T_k per operand produced inside the tree (empty otherwise)
+// What a node can deliver, and at what price: one entry per distinct output tiling the node's specs can produce, holding the
+// cheapest total (the node's own Cost plus everything upstream of it inside the tree) of delivering the output in that tiling,
+// the spec that achieves it, and -- per operand produced inside the tree -- which entry of the producer's own table it uses.
+struct Delivery {
+    Counts tiling;                 // of the node's output
+    int64_t total;                 // cheapest summed Cost of the subtree that ends in this node, output tiled like this
+    Counts spec;                   // the node's spec in that cheapest solution
+    std::vector<int> supplier;     // per operand: entry of the producer's table (-1: operand not produced inside the tree)
 };
+typedef std::vector<Delivery> DeliveryTable;
 
 // allow_sharing = false: every node but the last must be consumed exactly once (a tree, Section 4.2)
 ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, bool allow_sharing, std::vector<Op>* ops, std::vector<int>* consumers) {
@@ -144,67 +150,67 @@ ja_status_t parse_all(const ja_plan_node_t* nodes, int32_t n_nodes, bool allow_s
     return JA_OK;
 }
 
-// Algorithm 1 on the tree `members` (ascending = topological) rooted at `root`. An operand produced outside the tree by a
-// node that already has a spec enters with that node's output tiling fixed (Cost charges the repartition on a mismatch);
-// any other outside operand enters like an input of the computation. If `charge_consumers`, the root's tiling is chosen
-// with the repartition charges of its already-planned consumers added. Fills plan[] for the members.
+// The dynamic program of Section 4.2 (Algorithm 1) on the tree `members` (ascending = topological) rooted at `root`, stated
+// on delivery tables: nodes are visited producers first; for every spec of a node each operand independently picks the
+// cheapest entry of its producer's table (entry total + the repartition charge if the entry's tiling is not the one the
+// spec reads -- Cost is a sum over operands, so the minimum over all combinations of producer tilings separates), and the
+// spec competes for the entry of its own output tiling. The plan is read back from the root's cheapest entry through the
+// recorded suppliers.
+// Operands from outside the tree: one produced by a node that already has a spec enters with that node's output tiling
+// fixed (a mismatch is charged); any other enters like an input of the computation. If `charge_consumers`, the root's entry
+// is chosen with the repartition charges of its already-planned consumers added. Fills plan[] for the members.
 ja_status_t optimize_tree(const std::vector<Op>& ops, const std::vector<int32_t>& members, int32_t root, int32_t p,
                           bool charge_consumers, std::vector<Counts>* plan, int64_t* tree_cost) {
     std::vector<char> inside(ops.size(), 0);
     for (int32_t i : members) inside[i] = 1;
-    std::map<int32_t, std::vector<Counts>> cand;
-    std::map<int32_t, std::map<Counts, int64_t>> opt;
-    std::map<int32_t, std::map<Counts, Choice>> choice;
+    std::map<int32_t, DeliveryTable> table;
     for (int32_t i : members) {
         const Op& op = ops[i];
         std::vector<Counts> specs;
-        Counts cur;
-        enum_specs(op, p, 0, &cur, &specs);
+        Counts scratch;
+        enum_specs(op, p, 0, &scratch, &specs);
         if (specs.empty()) return ja_fail(JA_ERR_TILING, "node %d has no decomposition into %d function specs", i, p);
         const size_t n = op.ins.size();
-        std::vector<Counts> fixed(n);               // tiling of an operand whose producer is planned outside the tree
-        std::vector<int> kind(n, 0);                // 0 free, 1 produced inside the tree, 2 fixed
+        enum Source { FREE, IN_TREE, PLANNED_OUTSIDE };
+        std::vector<Source> source(n, FREE);
+        std::vector<Counts> outside_tiling(n);
         for (size_t k = 0; k < n; ++k) {
             const int32_t q = op.producers[k];
             if (q < 0) continue;
-            if (inside[q]) kind[k] = 1;
-            else if (!(*plan)[q].empty()) { kind[k] = 2; fixed[k] = tiling(ops[q], (*plan)[q], ops[q].out); }
+            if (inside[q]) source[k] = IN_TREE;
+            else if (!(*plan)[q].empty()) { source[k] = PLANNED_OUTSIDE; outside_tiling[k] = tiling(ops[q], (*plan)[q], ops[q].out); }
         }
-        for (const Counts& J : specs) {
-            // B(J). Cost is a sum over operands (join and repartition terms) plus the aggregation term, so the minimum over
-            // the producers' candidate tilings separates: each operand picks its own cheapest (Opt + repartition charge).
-            std::vector<const Counts*> none(n, nullptr);
-            int64_t best = cost(op, J, none);
-            std::vector<size_t> best_idx(n, 0);
+        DeliveryTable& mine = table[i];
+        for (const Counts& spec : specs) {
+            const std::vector<const Counts*> no_producers(n, nullptr);
+            Delivery d;
+            d.tiling = tiling(op, spec, op.out);
+            d.spec = spec;
+            d.supplier.assign(n, -1);
+            d.total = cost(op, spec, no_producers);          // join + aggregation terms of this node
             for (size_t k = 0; k < n; ++k) {
-                const Counts need = tiling(op, J, op.ins[k]);
-                if (kind[k] == 2) {
-                    if (fixed[k] != need) best += card(op, op.ins[k]);
-                } else if (kind[k] == 1) {
-                    const std::vector<Counts>& cs = cand[op.producers[k]];
-                    int64_t bk = -1;
-                    for (size_t c = 0; c < cs.size(); ++c) {
-                        const int64_t v = opt[op.producers[k]][cs[c]] + (cs[c] != need ? card(op, op.ins[k]) : 0);
-                        if (bk < 0 || v < bk) { bk = v; best_idx[k] = c; }
+                const Counts reads = tiling(op, spec, op.ins[k]);
+                const int64_t relayout = card(op, op.ins[k]);  // what a mismatch on this operand is charged
+                if (source[k] == PLANNED_OUTSIDE) {
+                    if (outside_tiling[k] != reads) d.total += relayout;
+                } else if (source[k] == IN_TREE) {
+                    const DeliveryTable& theirs = table[op.producers[k]];
+                    int64_t cheapest = -1;
+                    for (size_t e = 0; e < theirs.size(); ++e) {
+                        const int64_t v = theirs[e].total + (theirs[e].tiling != reads ? relayout : 0);
+                        if (cheapest < 0 || v < cheapest) { cheapest = v; d.supplier[k] = (int)e; }
                     }
-                    best += bk;
+                    d.total += cheapest;
                 }
             }
-            const Counts T = tiling(op, J, op.out);
-            auto it = opt[i].find(T);
-            if (it == opt[i].end() || best < it->second) {
-                if (it == opt[i].end()) cand[i].push_back(T);
-                opt[i][T] = best;
-                Choice c;
-                c.spec = J;
-                c.in_tilings.resize(n);
-                for (size_t k = 0; k < n; ++k)
-                    if (kind[k] == 1) c.in_tilings[k] = cand[op.producers[k]][best_idx[k]];
-                choice[i][T] = c;
-            }
+            size_t slot = 0;
+            while (slot < mine.size() && mine[slot].tiling != d.tiling) ++slot;
+            if (slot == mine.size()) mine.push_back(d);
+            else if (d.total < mine[slot].total) mine[slot] = d;
         }
     }
-    auto consumer_charge = [&](const Counts& T) {
+    // the root's entry: cheapest once the relayouts its already-planned consumers would need are counted in
+    auto consumers_pay = [&](const Counts& T) {
         int64_t c = 0;
         if (!charge_consumers) return c;
         for (size_t j = 0; j < ops.size(); ++j) {
@@ -214,23 +220,23 @@ ja_status_t optimize_tree(const std::vector<Op>& ops, const std::vector<int32_t>
         }
         return c;
     };
-    const Counts* T_star = nullptr;
-    int64_t best_total = -1;
-    for (const Counts& T : cand[root]) {
-        const int64_t v = opt[root][T] + consumer_charge(T);
-        if (!T_star || v < best_total) { T_star = &T; best_total = v; }
+    const DeliveryTable& top = table[root];
+    int chosen = -1;
+    int64_t chosen_total = 0;
+    for (size_t e = 0; e < top.size(); ++e) {
+        const int64_t v = top[e].total + consumers_pay(top[e].tiling);
+        if (chosen < 0 || v < chosen_total) { chosen = (int)e; chosen_total = v; }
     }
-    if (tree_cost) *tree_cost = opt[root][*T_star];
-    std::vector<std::pair<int32_t, Counts>> stack;
-    stack.push_back({root, *T_star});
-    while (!stack.empty()) {
-        const int32_t i = stack.back().first;
-        const Counts T = stack.back().second;
-        stack.pop_back();
-        const Choice& c = choice[i][T];
-        (*plan)[i] = c.spec;
+    if (tree_cost) *tree_cost = top[chosen].total;
+    // read the plan back: (node, entry) pairs, following the suppliers
+    std::vector<std::pair<int32_t, int>> todo(1, std::make_pair(root, chosen));
+    while (!todo.empty()) {
+        const int32_t i = todo.back().first;
+        const Delivery& d = table[i][todo.back().second];
+        todo.pop_back();
+        (*plan)[i] = d.spec;
         for (size_t k = 0; k < ops[i].ins.size(); ++k)
-            if (ops[i].producers[k] >= 0 && inside[ops[i].producers[k]]) stack.push_back({ops[i].producers[k], c.in_tilings[k]});
+            if (d.supplier[k] >= 0) todo.push_back(std::make_pair(ops[i].producers[k], d.supplier[k]));
     }
     return JA_OK;
 }
