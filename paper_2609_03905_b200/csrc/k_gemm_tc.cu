@@ -37,6 +37,12 @@ constexpr int BM = 128, BN = 256;
 constexpr int NUM_THREADS = 192;
 // BK = contraction depth of one pipeline stage. The two-CTA form stages 128-deep chunks so that every box it issues
 // (A: 128 rows x 64 k, B: 128 k x 64 columns) is 16 KiB: fewer, larger TMA copies per flop than 64-deep stages.
+// What bounds this kernel is operand delivery, not the tensor pipe: timing-only ablations on [16384, 4096] x [4096, 4096]
+// with half of the B boxes not loaded ran at 1617 TFLOP/s against 1391, with half of A as well at 1821. A form that cuts
+// the bytes per flop by a quarter -- tiles of 256 x 512 on both accumulators, A fetched once per 512 columns -- was built,
+// passed the parity tests and measured SLOWER, because the shared memory left holds either four 64-deep stages of 8 KiB
+// B boxes (1196 TFLOP/s on the same product) or two 128-deep stages (1339; 1205 against 1330-1418 on the up-projections):
+// more, smaller copies or too shallow a pipeline cost more than the saved bytes bring.
 template <int CG> struct Cfg {
     static constexpr int BK = CG == 1 ? 64 : 128;
     static constexpr int STAGES = CG == 1 ? 4 : 3;
