@@ -525,7 +525,14 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   (the next item's Q and first K / V tiles, claimed one item early, and the tiles two key steps ahead): 20 % slower --
 //   the prefetches queue in front of the loads the products wait for; claiming one item early alone: 2 % slower; issuing
 //   the tensor-memory loads of the next key step's scores before handing P over (when they are already complete): 20 %
-//   slower.
+//   slower; a fourth group of four warps that takes O~ / l and the stores off the row warps (register allotments moved
+//   between the groups with setmaxnreg, output written straight from registers): 6 % slower -- the output stage is not
+//   what an item waits for. Not possible: P in f16 from ex2.approx.f16x2 (two exponentials per instruction) against bf16
+//   V -- tcgen05.mma kind::f16 with different formats for A and B is an illegal instruction.
+//   Counters of the steady state: per 128 x 128 x 128 product pair the two smem x smem products read 128 KiB of shared
+//   memory (1024 cycles of its 128 B/clk port, as long as the products themselves take), the P stores and the K / V fills
+//   add half as much again: the shared-memory port, not a pipe, bounds long sequences (tensor-core reads 53 % + stores
+//   19 % of its cycles over a whole launch of B4 S2048).
 constexpr int NUM_THREADS2 = 320;
 constexpr int SMEM_BYTES2 = 7 * TILE_BYTES + 1024 + 256;
 
