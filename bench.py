@@ -221,12 +221,12 @@ def run_gpu(args, shape):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     sampler = ClockSampler(local) if rank == 0 else None   # started during set-up so that it is polling long before the timed region
-    bf = torch.bfloat16
+    bf = torch.float16 if args.dtype == "f16" else torch.bfloat16     # cell type of every relation of the block
     Bt, S, hidden, heads, ffn = shape["batch"], shape["seq"], shape["hidden"], shape["heads"], shape["ffn"]
     T = Bt * S
     kvh = shape.get("kv_heads") or heads
-    weights = si.llama_weights(hidden, ffn, kv_hidden=hidden // heads * kvh)
-    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan, fused=not args.unfused, n_kv_heads=kvh)
+    weights = si.llama_weights(hidden, ffn, dtype=bf, kv_hidden=hidden // heads * kvh)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, weights, plan=args.plan, fused=not args.unfused, n_kv_heads=kvh, dtype=bf)
     x_host = si.normal((T, hidden), 0.0, 1.0, bf, 5, 0).pin_memory()
     out_host = torch.empty((T, hidden), dtype=bf).pin_memory()
     x_dev = torch.empty((T, hidden), dtype=bf, device="cuda")
@@ -428,7 +428,7 @@ def run_gpu(args, shape):
                          f"token rows ({cfl / 1e9:.1f} GFLOP)"}
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": args.dtype,
         "data": "synthetic",
         "config": {"workload": f"LLaMA-{args.shape} block forward as chained join-aggs, plan '{args.plan}' "
                                f"({blk.n_relayouts} ja_repartition relayouts per step; fused chains: {'on' if not args.unfused else 'off'})", **shape,
@@ -825,6 +825,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the kernels of configurations 1-4 after the headline region")
     ap.add_argument("--config-reps", type=int, default=20, help="timed launches per kernel of configurations 1-4")
+    ap.add_argument("--dtype", choices=["bf16", "f16"], default="bf16",
+                    help="cell type of the block's relations (--case block): bf16 as the benchmark configurations state, or f16, the paper's precision")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
     ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "

@@ -53,7 +53,10 @@ typedef enum {
     JA_ERR_TIMEOUT = 11            /* a bounded device-side wait ran out (reported through ja_stream_status) */
 } ja_status_t;
 
-typedef enum { JA_F32 = 0, JA_BF16 = 1 } ja_dtype_t;
+/* cell type of a relation. The two 16-bit types run through the same kernels (tensor cores for the contractions, f32
+ * accumulation and f32 row arithmetic, one rounding to nearest even at each store); JA_F16 is the precision of the
+ * paper's experiments (Section 6), JA_BF16 the one the benchmark configurations of this library are stated in. */
+typedef enum { JA_F32 = 0, JA_BF16 = 1, JA_F16 = 2 } ja_dtype_t;
 
 /* aggregation operator (+) of Definition 3.7 */
 typedef enum {
@@ -148,12 +151,13 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  * (a cudaStream_t passed as void*; NULL = the legacy default stream), asynchronously.
  * inputs[k] must be tiled exactly as in_k(J), outputs[0] as out(J) (else JA_ERR_PARTITION_MISMATCH).
  * Supported forms (letters are free; shapes of the signature matter):
- *   "ij,jk->ik"            MUL / SUM        bf16 or f32 operands, f32 accumulate. bf16: tensor cores under every tiling
+ *   "ij,jk->ik"            MUL / SUM        bf16, f16 or f32 operands (one dtype for all three relations), f32 accumulate.
+ *                                            bf16 / f16: tensor cores under every tiling
  *                                            (operands fetched by TMA on uniform blocks with 16-byte rows, by plain
  *                                            asynchronous loads otherwise; plain ALUs only where blocks are smaller than
  *                                            64 cells a side); f32: plain ALUs
  *   "ij,jk,ik->ik"         MATMUL_ADD / SUM   } fused chains: the accumulator of the contraction goes through the
- *   "ij,jk->ik"            MATMUL_ROPE / SUM  } next join-agg before its single rounding and store; bf16 relations
+ *   "ij,jk->ik"            MATMUL_ROPE / SUM  } next join-agg before its single rounding and store; bf16 or f16 relations
  *   "ij,jk,jk->ik"         SWIGLU_UP / SUM    } on uniform blocks only (JA_ERR_UNSUPPORTED otherwise: run the chain)
  *   "X,X->X", X any rank   ADD | SILU_MUL / NONE          key-aligned join
  *   "Rj->R"                SQUARE/SUM, IDENT/MAX          R = leading letters; f32 statistics output
@@ -163,7 +167,9 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  *   "Rj,j->Rj"             RMSNORM / NONE   (fused)       "Rj->Rj"  SOFTMAX / NONE (fused)
  *   "bshd->bshd"           ROPE / NONE
  *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128; q / k split points and sequence
- *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends multiples of 64 rows (tensor memory kernels: 128)
+ *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends multiples of 64 rows (tensor memory kernels: 128);
+ *                                                          Q, K, V, O of one 16-bit dtype (bf16 or f16; the probabilities
+ *                                                          enter the second product rounded to that dtype)
  * n_outputs is 1, except for ATTENTION where it may be 2: outputs[1] then receives lse[b, q, h] = log of the softmax
  * denominator of every query row (f32, tiled like the first three indices of outputs[0]) -- with it two results over
  * disjoint key ranges combine by the online-softmax aggregation: O = w1 O1 + w2 O2, w_i = exp(lse_i - lse).
@@ -188,14 +194,15 @@ ja_status_t ja_overlay_atoms(const ja_relation_t* src, const ja_relation_t* dst,
  * rank(out)+1 whose leading index is the copy index c, extent m = the number of function specs per output type
  * (it must be the same for all of them), cut into its m unit intervals; the other indices are those of the output,
  * tiled as out(J). Block (c, key) holds the output of the c-th function spec (ascending F) with output type `key`.
- * Supported: "ij,jk->ik" MUL/SUM -- copy c is A[:, block c] B[block c, :]. bf16 operands on uniform blocks: tensor
- * cores, partial relation bf16 (one rounding per copy) or f32 (the accumulator as it is); otherwise plain ALUs and a
+ * Supported: "ij,jk->ik" MUL/SUM -- copy c is A[:, block c] B[block c, :]. bf16 / f16 operands on uniform blocks: tensor
+ * cores, partial relation of the operands' dtype (one rounding per copy) or f32 (the accumulator as it is); otherwise plain ALUs and a
  * partial relation of the operands' dtype. Errors as ja_execute; JA_ERR_UNSUPPORTED for other forms.
  *
  * ja_repartition_agg is the one-processor image of an exchange program: every atom of the overlay of the partial
  * relation's tiling (copy index dropped) and dst's tiling has m copies; they are (+)-combined in ascending copy
  * order in f32 (agg = JA_AGG_SUM or JA_AGG_MAX; JA_AGG_NONE only when m == 1, a plain relayout) and stored once,
- * rounded once, in dst's block. partials may be f32 or bf16, dst f32 or bf16, independently. partials is borrowed and
+ * rounded once, in dst's block. partials and dst may each be f32 or a 16-bit type (the same one when both are 16-bit:
+ * JA_ERR_DTYPE otherwise). partials is borrowed and
  * unchanged. Asynchronous on `cuda_stream`; the first call per (partials, dst) pair builds and caches the copy plan
  * (one synchronous cudaMalloc + cudaMemcpy). Errors: JA_ERR_SHAPE, JA_ERR_TILING (copy index not cut into unit
  * intervals), JA_ERR_INVALID_ARG (aggregation missing; dst aliases partials). */

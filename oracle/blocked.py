@@ -288,7 +288,7 @@ def join_partials(einsum: str, parts: dict, inputs, fn="mul", agg="sum", params=
         lo, hi = spec.bounds(okey, -1)
         out[(c,) + tuple(slice(l, h) for l, h in zip(lo, hi))] = part
     assert not np.isnan(out).any()
-    return core.round_to(out, dtype) if dtype in ("f32", "bf16") else out
+    return core.round_to(out, dtype) if dtype in ("f32", "bf16", "f16") else out
 
 
 def partial_splits(m: int, splits):
@@ -319,4 +319,4 @@ def aggregate_repartition(partials: np.ndarray, src_splits, dst_splits, agg="sum
                 raise ValueError("an atom has several copies but there is no aggregation")
         out[sl] = acc
     assert not np.isnan(out).any()
-    return core.round_to(out, dtype) if dtype in ("f32", "bf16") else out
+    return core.round_to(out, dtype) if dtype in ("f32", "bf16", "f16") else out

@@ -61,9 +61,9 @@ def _ptr(a: np.ndarray):
 
 
 def round_to(a, dtype: str) -> np.ndarray:
-    """Round fp64 values to the nearest value of `dtype` ('f32' | 'bf16'), ties to even; result stays fp64."""
+    """Round fp64 values to the nearest value of `dtype` ('f32' | 'bf16' | 'f16'), ties to even; result stays fp64."""
     out = _f64(a).copy()
-    lib().orc_round_array(_ptr(out), ctypes.c_int64(out.size), ctypes.c_int({"f32": 0, "bf16": 1}[dtype]))
+    lib().orc_round_array(_ptr(out), ctypes.c_int64(out.size), ctypes.c_int({"f32": 0, "bf16": 1, "f16": 2}[dtype]))
     return out
 
 

@@ -78,9 +78,23 @@ double orc_round_bf16(double x) {
 
 double orc_round_f32(double x) { return (double)(float)x; }
 
-void orc_round_array(double* a, int64_t n, int dtype /* 0 = f32, 1 = bf16 */) {
+/* IEEE binary16 (the precision of the paper's experiments, Section 6): 10 explicit mantissa bits, lowest binade 2^-14,
+ * largest finite value 65504; one rounding from fp64, ties to even. */
+double orc_round_f16(double x) {
+    if (isnan(x) || isinf(x) || x == 0.0) return x;
+    int e;
+    (void)frexp(x, &e);
+    int lead = e - 1;
+    if (lead < -14) lead = -14;    /* subnormals share the quantum of the lowest binade */
+    int qexp = lead - 10;
+    double r = ldexp(nearbyint(ldexp(x, -qexp)), qexp);
+    if (fabs(r) >= ldexp(1.0, 16)) return x > 0 ? INFINITY : -INFINITY;
+    return r;
+}
+
+void orc_round_array(double* a, int64_t n, int dtype /* 0 = f32, 1 = bf16, 2 = f16 */) {
 #pragma omp parallel for schedule(static)
-    for (int64_t i = 0; i < n; ++i) a[i] = dtype ? orc_round_bf16(a[i]) : orc_round_f32(a[i]);
+    for (int64_t i = 0; i < n; ++i) a[i] = dtype == 2 ? orc_round_f16(a[i]) : dtype ? orc_round_bf16(a[i]) : orc_round_f32(a[i]);
 }
 
 static double apply_g(int fn, const double* v, int n, const double* p) {

@@ -19,7 +19,7 @@ from . import core
 
 
 def rnd(a, dtype):
-    return core.round_to(a, dtype) if dtype in ("f32", "bf16") else np.asarray(a, dtype=np.float64)
+    return core.round_to(a, dtype) if dtype in ("f32", "bf16", "f16") else np.asarray(a, dtype=np.float64)
 
 
 # ---- matmul -------------------------------------------------------------------------------------

@@ -18,7 +18,7 @@ JA_OK = 0
 STATUS = {0: "JA_OK", 1: "JA_ERR_INVALID_ARG", 2: "JA_ERR_PARSE", 3: "JA_ERR_SHAPE", 4: "JA_ERR_TILING",
           5: "JA_ERR_PARTITION_MISMATCH", 6: "JA_ERR_DTYPE", 7: "JA_ERR_UNSUPPORTED", 8: "JA_ERR_ALIGNMENT",
           9: "JA_ERR_OOM", 10: "JA_ERR_CUDA", 11: "JA_ERR_TIMEOUT"}
-JA_F32, JA_BF16 = 0, 1
+JA_F32, JA_BF16, JA_F16 = 0, 1, 2
 AGG = {"none": 0, "sum": 1, "max": 2, "online_softmax": 3}
 FN = {"mul": 0, "ident": 1, "square": 2, "add": 3, "silu_mul": 4, "rms_scale": 5, "exp_sub": 6, "exp_sub_div": 7,
       "rope": 8, "attention": 9, "rmsnorm": 10, "softmax": 11, "matmul_add": 12, "matmul_rope": 13, "swiglu_up": 14}

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -37,9 +38,30 @@ __device__ __forceinline__ int64_t ja_elem_off(const RelView& v, const int64_t* 
 
 __device__ __forceinline__ float ja_to_float(float x) { return x; }
 __device__ __forceinline__ float ja_to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float ja_to_float(__half x) { return __half2float(x); }
 template <typename T> __device__ __forceinline__ T ja_from_float(float x);
 template <> __device__ __forceinline__ float ja_from_float<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 ja_from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+template <> __device__ __forceinline__ __half ja_from_float<__half>(float x) { return __float2half_rn(x); }
+
+// cell type <-> ja_dtype_t, and the packed pair of a 16-bit type
+template <typename T> struct JaDtypeOf;
+template <> struct JaDtypeOf<float> { static constexpr ja_dtype_t value = JA_F32; };
+template <> struct JaDtypeOf<__nv_bfloat16> { static constexpr ja_dtype_t value = JA_BF16; };
+template <> struct JaDtypeOf<__half> { static constexpr ja_dtype_t value = JA_F16; };
+// two f32 -> one packed pair of 16-bit cells (round to nearest even), and back; F16: false = bf16, true = f16
+template <bool F16> __device__ __forceinline__ uint32_t ja_pack16(float lo, float hi) {
+    if (F16) {
+        const __half2 t = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&t);
+    }
+    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&t);
+}
+template <bool F16> __device__ __forceinline__ float2 ja_unpack16(uint32_t w) {
+    if (F16) return __half22float2(*reinterpret_cast<const __half2*>(&w));
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w));
+}
 
 // Launch order of the attention CTAs (CTAs are handed to SMs in order of blockIdx.x). One CTA = one query tile (or pair
 // of tiles) of one (batch, head). (batch, head) pairs are taken in sections of `sect` consecutive pairs and inside a

@@ -183,7 +183,7 @@ static ja_status_t fill_relation(ja_relation* r, int32_t rank, const int64_t* ex
                                  const int64_t* const* splits, ja_dtype_t dtype) {
     if (rank < 1 || rank > JA_MAX_RANK || !extents || !nparts || !splits)
         return ja_fail(JA_ERR_INVALID_ARG, "rank must be 1..%d and extents/nparts/splits non-NULL", JA_MAX_RANK);
-    if (dtype != JA_F32 && dtype != JA_BF16) return ja_fail(JA_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    if (dtype != JA_F32 && dtype != JA_BF16 && dtype != JA_F16) return ja_fail(JA_ERR_DTYPE, "unknown dtype %d", (int)dtype);
     r->rank = rank;
     r->dtype = dtype;
     r->esize = esize_of(dtype);
@@ -919,7 +919,7 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         in[0][1] == in[1][0] && o[0] == in[0][0] && o[1] == in[1][1] && in[0][0] != in[1][1]) {
         const ja_relation *A = inputs[0], *B = inputs[1];
         if (A->dtype != B->dtype || A->dtype != out->dtype) return ja_fail(JA_ERR_DTYPE, "matmul operands must share one dtype");
-        if (A->dtype == JA_BF16) {
+        if (A->dtype != JA_F32) {   // bf16 or f16: tensor cores
             const int loader = ja_config().gemm_loader;
             if (!plan->gemm_checked) {
                 bool ok = false;
@@ -942,8 +942,8 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         in[0][0] != in[1][1]) {
         const ja_relation *A = inputs[0], *B = inputs[1];
         for (int k = 0; k < n_in; ++k)
-            if (inputs[k]->dtype != JA_BF16) return ja_fail(JA_ERR_UNSUPPORTED, "fused matmul chains need bf16 relations");
-        if (out->dtype != JA_BF16) return ja_fail(JA_ERR_UNSUPPORTED, "fused matmul chains need bf16 relations");
+            if (inputs[k]->dtype == JA_F32 || inputs[k]->dtype != out->dtype)
+                return ja_fail(JA_ERR_UNSUPPORTED, "fused matmul chains need relations of one 16-bit dtype");
         GemmEpilogue ep;
         memset(&ep, 0, sizeof ep);
         if (fn == JA_FN_MATMUL_ADD) {
@@ -1084,14 +1084,15 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         in[1] == in[2] && o == x && in[1][0] == x[0] && in[1][3] == x[3] && in[1][1] != x[1] && in[1][2] != x[1] &&
         in[1][2] != x[0] && in[1][2] != x[3]) {
         const ja_relation *Q = inputs[0], *K = inputs[1], *V = inputs[2];
-        if (Q->dtype != JA_BF16 || K->dtype != JA_BF16 || V->dtype != JA_BF16 || out->dtype != JA_BF16)
-            return ja_fail(JA_ERR_DTYPE, "attention relations must be bf16");
+        if (Q->dtype == JA_F32 || K->dtype != Q->dtype || V->dtype != Q->dtype || out->dtype != Q->dtype)
+            return ja_fail(JA_ERR_DTYPE, "attention relations must share one 16-bit dtype");
         if (Q->extent[3] != 128 || Q->nblk[3] != 1) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs an unsplit last index of extent 128");
         if (Q->extent[1] != K->extent[1]) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs equal query and key extents");
         AttnArgs aa;
         memset(&aa, 0, sizeof aa);
         aa.cache = &plan->attn;
         aa.q = ja_view(Q); aa.k = ja_view(K); aa.v = ja_view(V); aa.o = ja_view(out);
+        aa.f16 = Q->dtype == JA_F16;
         if (n_outputs == 2) {   // second output: lse[b, q, h], f32, tiled like the (b, q, h) indices of the output
             ja_relation* L = outputs[1];
             if (!L || L->rank != 3 || L->dtype != JA_F32) return ja_fail(JA_ERR_DTYPE, "the second attention output is an f32 relation over (b, q, h)");
@@ -1185,7 +1186,7 @@ extern "C" ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_
         std::lock_guard<std::mutex> plans_lock(spec->plans_mu);
         std::shared_ptr<ExecPlan> plan = spec->plans[key];
         if (!plan) spec->plans[key] = plan = std::make_shared<ExecPlan>();
-        if (A->dtype == JA_BF16) {
+        if (A->dtype != JA_F32) {
             if (!plan->gemm_checked) {
                 bool ok = false;
                 GemmEpilogue ep;

@@ -194,6 +194,7 @@ struct AttnArgs {
     const int32_t* q_split;
     const int32_t* k_split;
     bool rows_layout;
+    bool f16;              // cell type of Q, K, V, O: false = bf16, true = f16
 };
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);
 // tcgen05 / TMEM form; *launched stays false when the tiling does not fit it

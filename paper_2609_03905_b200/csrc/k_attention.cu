@@ -40,15 +40,19 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+// F16: operands are f16 instead of bf16 (same fragments, f32 accumulate)
+template <bool F16>
+__device__ __forceinline__ void mma_16bit(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    if (F16)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // byte address inside a [rows][128] bf16 tile whose 16-byte chunks are XOR-swizzled by the row
@@ -64,7 +68,7 @@ __device__ __forceinline__ const char* row_ptr(const RelView& v, int b, int s, i
     return v.base + v.blk_off[flat] + ((((int64_t)(b - blo) * sw + (s - slo)) * hw + (h - hlo)) * D) * 2;
 }
 
-template <int QT>
+template <int QT, bool F16>
 __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     constexpr int NW = QT / 16;        // warps; each owns 16 query rows
     constexpr int NT = NW * 32;
@@ -156,8 +160,8 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
                 const int chunk = ks * 2 + (mi % 2);
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4(kbase + swz(krow, chunk), b0, b1, b2, b3);
-                mma_bf16(s[2 * np], qf[ks], b0, b1);
-                mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
+                mma_16bit<F16>(s[2 * np], qf[ks], b0, b1);
+                mma_16bit<F16>(s[2 * np + 1], qf[ks], b2, b3);
             }
         }
         // ---- scale, causal band inside the diagonal block, row max ---------------------------------------------
@@ -197,8 +201,8 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
             float p2 = exp2f(s[n][2] - m_use[1]), p3 = exp2f(s[n][3] - m_use[1]);
             ls[0] += p0 + p1;
             ls[1] += p2 + p3;
-            pf[n / 2][(n % 2) * 2 + 0] = pack_bf16(p0, p1);
-            pf[n / 2][(n % 2) * 2 + 1] = pack_bf16(p2, p3);
+            pf[n / 2][(n % 2) * 2 + 0] = ja_pack16<F16>(p0, p1);
+            pf[n / 2][(n % 2) * 2 + 1] = ja_pack16<F16>(p2, p3);
         }
 #pragma unroll
         for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * alpha[r] + ls[r];
@@ -217,8 +221,8 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
                 const int chunk = np * 2 + (mi / 2);
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(vbase + swz(vrow, chunk), b0, b1, b2, b3);
-                mma_bf16(o[2 * np], pf[ks], b0, b1);
-                mma_bf16(o[2 * np + 1], pf[ks], b2, b3);
+                mma_16bit<F16>(o[2 * np], pf[ks], b0, b1);
+                mma_16bit<F16>(o[2 * np + 1], pf[ks], b2, b3);
             }
         }
         __syncthreads();  // everyone is done with this buffer before it is refilled
@@ -243,8 +247,8 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
 #pragma unroll
         for (int n = 0; n < 16; ++n) {
             // columns n*8 + 2*t4, +1  -> chunk n, byte (2*t4)*2 inside it
-            *reinterpret_cast<uint32_t*>(sQ + swz(r_lo, n) + t4 * 4) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
-            *reinterpret_cast<uint32_t*>(sQ + swz(r_hi, n) + t4 * 4) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
+            *reinterpret_cast<uint32_t*>(sQ + swz(r_lo, n) + t4 * 4) = ja_pack16<F16>(o[n][0] * inv0, o[n][1] * inv0);
+            *reinterpret_cast<uint32_t*>(sQ + swz(r_hi, n) + t4 * 4) = ja_pack16<F16>(o[n][2] * inv1, o[n][3] * inv1);
         }
     }
     __syncthreads();
@@ -271,13 +275,19 @@ ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
     a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (ja_sm_count() + a.S / QT - 1) / (a.S / QT)));
     dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
+#define JA_ATTN_SYNC(Q, F)                                                                                          \
+    do {                                                                                                           \
+        JA_CUDA(cudaFuncSetAttribute(attention_kernel<Q, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); \
+        attention_kernel<Q, F><<<grid, 2 * Q, smem, st>>>(a2);                                                    \
+    } while (0)
     if (QT == 128) {
-        JA_CUDA(cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attention_kernel<128><<<grid, 256, smem, st>>>(a2);
+        if (a.f16) JA_ATTN_SYNC(128, true);
+        else JA_ATTN_SYNC(128, false);
     } else {
-        JA_CUDA(cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attention_kernel<64><<<grid, 128, smem, st>>>(a2);
+        if (a.f16) JA_ATTN_SYNC(64, true);
+        else JA_ATTN_SYNC(64, false);
     }
+#undef JA_ATTN_SYNC
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
     return JA_OK;

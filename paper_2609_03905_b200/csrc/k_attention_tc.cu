@@ -167,6 +167,7 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+template <bool F16>   // cell type of Q, K, V, O and of P: bf16 or f16
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnTcParams p) {
@@ -241,7 +242,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         {
             const uint32_t leader = elect_one();
             // S = Q K^T: M=128, N=128, A and B K-major.  O' = P V: A from TMEM, B MN-major.
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+            constexpr uint32_t FMT = F16 ? 0u : 1u;   // operand format of the instruction descriptor: f16 = 0, bf16 = 1
+            const uint32_t idesc_qk = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
             auto issue_qk = [&](int j) {
                 const int st = j & 1;
@@ -342,8 +344,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (diag && c * 32 + i > kmax) p0 = 0.f;
                     if (diag && c * 32 + i + 1 > kmax) p1 = 0.f;
                     sum += p0 + p1;
-                    __nv_bfloat162 t = __floats2bfloat162_rn(p0, p1);
-                    pk[i / 2] = *reinterpret_cast<uint32_t*>(&t);
+                    pk[i / 2] = ja_pack16<F16>(p0, p1);
                 }
                 tmem_st16(tS[st] + lane_addr + c * 16, pk);   // columns [16c, 16c+16): S columns already consumed
             }
@@ -378,9 +379,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
                 for (int g = 0; g < 16; ++g) {
                     uint4 ov;
-                    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
+                    uint32_t* po = reinterpret_cast<uint32_t*>(&ov);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
+                    for (int e = 0; e < 4; ++e) po[e] = ja_pack16<F16>(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
                     *reinterpret_cast<uint4*>(dst + g * 16) = ov;
                 }
             }
@@ -457,11 +458,11 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
     p1 = __int_as_float(__float_as_int(r1) + (__float_as_int(t1) << 23));
 }
 
-// One row of P = 2^(S * scale - m) for 128 keys as 64 packed bf16 pairs in registers; returns the row sum (f32, of the
+// One row of P = 2^(S * scale - m) for 128 keys as 64 packed bf16 (or f16) pairs in registers; returns the row sum (f32, of the
 // unrounded values); a score of -inf (a masked key) gives exactly 0. POLY: which pairs of every group of eight keys take the
 // FMA-pipe exponential instead of ex2 -- 0 none, 1 one of four, 2 two of four, 3 one of eight -- interleaved so that both
 // pipes stay busy.
-template <int POLY>
+template <int POLY, bool F16>
 __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float scale, float m_used, uint32_t (&pk)[64]) {
     const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_used, -m_used);
     uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
@@ -482,8 +483,7 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
             }
             if (i & 2) sum_a = add2(sum_a, pack2(p0, p1));
             else sum_b = add2(sum_b, pack2(p0, p1));
-            __nv_bfloat162 tt = __floats2bfloat162_rn(p0, p1);
-            pk[col / 2] = *reinterpret_cast<uint32_t*>(&tt);
+            pk[col / 2] = ja_pack16<F16>(p0, p1);
         }
     }
     float a0, a1, b0, b1;
@@ -564,7 +564,7 @@ __device__ __forceinline__ bool attn_item(const AttnTcParams& p, int rank, AttnI
     return true;
 }
 
-template <bool PERSIST, int VAR>
+template <bool PERSIST, int VAR, bool F16>
 __global__ void __launch_bounds__(NUM_THREADS2, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -675,7 +675,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     } else if (warp == 1) {
         // ================= MMA issuer: the whole warp runs the loop, one elected lane issues =================
         const uint32_t leader = elect_one();
-        const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+        constexpr uint32_t FMT = F16 ? 0u : 1u;   // operand format of the instruction descriptor: f16 = 0, bf16 = 1
+        const uint32_t idesc_qk = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
         const uint32_t idesc_pv = idesc_qk | (1u << 16);
         auto issue_qk = [&](int t, int sl) {          // S_t = Q_t K^T, K in slot sl
             const uint32_t kaddr = sKV + sl * TILE_BYTES, qaddr = sQ + t * TILE_BYTES;
@@ -826,7 +827,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     l_run *= alpha;
                 }
                 uint32_t pk[64];
-                l_run += row_exp_pack128<POLY>(v, p.scale_log2e, m_used, pk);
+                l_run += row_exp_pack128<POLY, F16>(v, p.scale_log2e, m_used, pk);
                 if (!(WAIT_FIRST || rescale)) {
                     if (!wait_p_tile()) { ok = false; break; }
                 }
@@ -856,10 +857,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     uint4 ov;
-                    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov);
+                    uint32_t* po = reinterpret_cast<uint32_t*>(&ov);
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        po[e] = __floats2bfloat162_rn(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
+                        po[e] = ja_pack16<F16>(__uint_as_float(o[g * 8 + 2 * e]) * inv, __uint_as_float(o[g * 8 + 2 * e + 1]) * inv);
                     const int ch = cc * 4 + g;                      // 16-byte chunk 0..15 of the row
                     *reinterpret_cast<uint4*>(prow + (ch >> 3) * HALF_BYTES + (((ch & 7) ^ sw) << 4)) = ov;
                 }
@@ -895,7 +896,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 }
 
 // "bshd" relation with uniform blocks along b and h as a rank-3 tensor (d, head in block, row of hblk x 128 cells)
-ja_status_t encode_rows(const RelView& v, CUtensorMap* tm) {
+ja_status_t encode_rows(const RelView& v, bool f16, CUtensorMap* tm) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     const int64_t hb = v.bs[2];
@@ -904,7 +905,7 @@ ja_status_t encode_rows(const RelView& v, CUtensorMap* tm) {
     cuuint64_t strides[2] = {(cuuint64_t)(D * 2), (cuuint64_t)(hb * D * 2)};
     cuuint32_t box[3] = {64, 1, 128};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    CUresult res = enc(tm, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (bshd rows) failed with code %d", (int)res);
     return JA_OK;
@@ -938,12 +939,17 @@ void ja_attention_reset_queues() {
 namespace {
 
 template <bool PERSIST>
-ja_status_t launch_two_tiles(int variant, dim3 grid, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                             const CUtensorMap& to, const AttnTcParams& p) {
+ja_status_t launch_two_tiles(int variant, bool f16, dim3 grid, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk,
+                             const CUtensorMap& tv, const CUtensorMap& to, const AttnTcParams& p) {
+    if (f16) {   // f16 cells: the default row-thread variant only
+        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel<PERSIST, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2));
+        attention_tc2_kernel<PERSIST, 1, true><<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);
+        return JA_OK;
+    }
 #define JA_ATTN_LAUNCH(V)                                                                                                          \
     case V: {                                                                                                                      \
-        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel<PERSIST, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2)); \
-        attention_tc2_kernel<PERSIST, V><<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);                             \
+        JA_CUDA(cudaFuncSetAttribute(attention_tc2_kernel<PERSIST, V, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES2)); \
+        attention_tc2_kernel<PERSIST, V, false><<<grid, NUM_THREADS2, SMEM_BYTES2, st>>>(tq, tk, tv, to, p);                      \
         return JA_OK;                                                                                                              \
     }
     switch (variant) {
@@ -974,10 +980,10 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
     CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(cache->maps);
     if (!cache->valid) {
         ja_status_t s;
-        if ((s = encode_rows(a.q, &maps[0])) != JA_OK) return s;
-        if ((s = encode_rows(a.k, &maps[1])) != JA_OK) return s;
-        if ((s = encode_rows(a.v, &maps[2])) != JA_OK) return s;
-        if ((s = encode_rows(a.o, &maps[3])) != JA_OK) return s;
+        if ((s = encode_rows(a.q, a.f16, &maps[0])) != JA_OK) return s;
+        if ((s = encode_rows(a.k, a.f16, &maps[1])) != JA_OK) return s;
+        if ((s = encode_rows(a.v, a.f16, &maps[2])) != JA_OK) return s;
+        if ((s = encode_rows(a.o, a.f16, &maps[3])) != JA_OK) return s;
         cache->valid = true;
     }
     const CUtensorMap &tq = maps[0], &tk = maps[1], &tv = maps[2], &to = maps[3];
@@ -1045,15 +1051,20 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
             const unsigned half = ATTN_QUEUES / 2;
             const unsigned slot = cap == cudaStreamCaptureStatusActive ? half + next_captured.fetch_add(1) % half : next_queue.fetch_add(1) % half;
             p.queue = queues + 2 * slot;
-            s = launch_two_tiles<true>(variant, dim3((unsigned)std::min<int64_t>(items, sms), 1, 1), st, tq, tk, tv, to, p);
+            s = launch_two_tiles<true>(variant, a.f16, dim3((unsigned)std::min<int64_t>(items, sms), 1, 1), st, tq, tk, tv, to, p);
         } else {
-            s = launch_two_tiles<false>(variant, dim3((unsigned)items, 1, 1), st, tq, tk, tv, to, p);
+            s = launch_two_tiles<false>(variant, a.f16, dim3((unsigned)items, 1, 1), st, tq, tk, tv, to, p);
         }
         if (s != JA_OK) return s;
     } else {
-        JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
-        attention_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+        if (a.f16) {
+            JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+            attention_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+        } else {
+            JA_CUDA(cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+            attention_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tq, tk, tv, p);
+        }
     }
     ja_count_launch();
     JA_CUDA(cudaGetLastError());

@@ -40,6 +40,7 @@ struct LdParams {
     uint32_t wait_cap_us;
     int32_t tiles_i, tiles_k;   // tiles per output block along i and k (of the LARGEST block)
     int32_t total_tiles;        // nblk_i * tiles_i * nblk_k * tiles_k
+    int32_t f16;                // cell type of all three relations: 0 = bf16, 1 = f16
 };
 
 __device__ __forceinline__ int64_t interval_width(const RelView& v, int d, int idx) {
@@ -137,7 +138,7 @@ __device__ __forceinline__ Tile tile_of(const LdParams& p, int t) {
 }
 
 // ASYNC: every block row of A and B starts on a 4-byte boundary
-template <bool ASYNC>
+template <bool ASYNC, bool F16>   // F16: cells are f16 instead of bf16
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_ld_kernel(const LdParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -254,7 +255,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_ld_kernel(const LdParams 
     } else if (warp == 8) {
         // ================= MMA issuer =================
         const uint32_t leader = elect_one();
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        constexpr uint32_t fmt = F16 ? 0u : 1u;   // A and B: bf16 (format 1) or f16 (format 0); D f32; B MN-major
+        const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         int stage = 0, it = 0;
         uint32_t phase = 0, acc_phase[2] = {0, 0};
         bool ok = true;
@@ -314,8 +316,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_ld_kernel(const LdParams 
                         uint32_t w[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[g * 8 + 2 * e]), __uint_as_float(v[g * 8 + 2 * e + 1]));
-                            w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+                            const float lo = __uint_as_float(v[g * 8 + 2 * e]), hi = __uint_as_float(v[g * 8 + 2 * e + 1]);
+                            w[e] = ja_pack16<F16>(lo, hi);
                         }
                         store8(c_row + (ch * 32 + g * 8) * 2, w, (int)min((int64_t)8, cols - ch * 32 - g * 8));
                     }
@@ -339,7 +341,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_ld_kernel(const LdParams 
 // *launched stays false when the relations are too small for 128 x 256 tiles to pay (the plain-ALU kernel takes them)
 ja_status_t ja_launch_gemm_ld(const ja_relation* Ar, const ja_relation* Br, const ja_relation* Cr, cudaStream_t st, bool* launched) {
     *launched = false;
-    if (Ar->dtype != JA_BF16 || Br->dtype != JA_BF16 || Cr->dtype != JA_BF16) return JA_OK;
+    if (Ar->dtype == JA_F32 || Br->dtype != Ar->dtype || Cr->dtype != Ar->dtype) return JA_OK;
     int64_t max_bm = 0, max_bn = 0;
     for (int i = 0; i < Ar->nblk[0]; ++i) max_bm = std::max(max_bm, Ar->splits[0][i + 1] - Ar->splits[0][i]);
     for (int i = 0; i < Br->nblk[1]; ++i) max_bn = std::max(max_bn, Br->splits[1][i + 1] - Br->splits[1][i]);
@@ -348,6 +350,7 @@ ja_status_t ja_launch_gemm_ld(const ja_relation* Ar, const ja_relation* Br, cons
     p.A = ja_view(Ar);
     p.B = ja_view(Br);
     p.C = ja_view(Cr);
+    p.f16 = Ar->dtype == JA_F16;
     p.status = ja_device_status_word(st);
     if (!p.status) return ja_fail(JA_ERR_CUDA, "cannot resolve the device status word");
     p.wait_cap_us = (uint32_t)ja_config().wait_cap_us;
@@ -363,13 +366,20 @@ ja_status_t ja_launch_gemm_ld(const ja_relation* Ar, const ja_relation* Br, cons
     int dev = 0;
     cudaGetDevice(&dev);
     if (!configured[dev & 63]) {
-        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        JA_CUDA(cudaFuncSetAttribute(gemm_ld_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         configured[dev & 63] = true;
     }
     const int grid = (int)std::min<int64_t>(total, ja_sm_count());
-    if (even) gemm_ld_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
-    else gemm_ld_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    if (p.f16) {
+        if (even) gemm_ld_kernel<true, true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
+        else gemm_ld_kernel<false, true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    } else {
+        if (even) gemm_ld_kernel<true, false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
+        else gemm_ld_kernel<false, false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    }
     JA_CUDA(cudaGetLastError());
     ja_count_launch();
     *launched = true;

@@ -72,7 +72,8 @@ struct GemmParams {
     int32_t bn_tile;           // output columns per tile: 256, or 128 for EPI_SWIGLU (two 128-column products per tile)
     int32_t n_copies;          // 1: SUM over all contracted blocks (aggregated output). nbk: join only -- tile (c, ., .) covers the
                                // single contracted block c and is stored to copy c of a partial relation [c, i, k]
-    int32_t c_esize;           // bytes per output cell: 2 (bf16) or 4 (f32, partial relations only)
+    int32_t c_esize;           // bytes per output cell: 2 (bf16 / f16) or 4 (f32, partial relations only)
+    int32_t f16;               // cell type of the operands (and of a 2-byte output): 0 = bf16, 1 = f16
     const char* r_base;        // EPI_ADD: payload of the relation added to the product (tiled exactly like the output)
     const float2* rope_table;  // EPI_ROPE: (cos, sin)[position][pair]
     int32_t rope_S, rope_D;    // EPI_ROPE: positions per sequence (row % rope_S), rotated extent (column % rope_D)
@@ -152,7 +153,9 @@ __device__ __forceinline__ int tile_of_iter(const GemmParams& p, int i, int firs
     return t < total ? t : -1;
 }
 
-template <int CG>
+// F16: cell type of the operands and of a 2-byte output -- bf16 or f16 (a compile-time choice: a select between the two
+// conversions in the epilogue cost the plain contraction a tenth of its rate)
+template <int CG, bool F16>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
@@ -279,7 +282,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const TileCoord tc = tile_coord<CG>(p, t, 0);
                 const int acc = it & 1;
                 const uint32_t n_mma = p.epi == EPI_SWIGLU ? (uint32_t)(2 * tc.width) : (uint32_t)((tc.width + 15) / 16 * 16);
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((n_mma >> 3) << 17) |
+                // D f32; A and B both bf16 (format 1) or both f16 (format 0); B MN-major
+                constexpr uint32_t fmt = F16 ? 0u : 1u;
+                const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((n_mma >> 3) << 17) |
                                        ((uint32_t)((BM * CG) >> 4) << 24);
                 if (!mbar_wait(tempty_bar(acc), acc_phase[acc] ^ 1, abort_flag, p.status)) { ok = false; break; }
                 acc_phase[acc] ^= 1;
@@ -385,18 +390,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[g * 8 + e]);
                             if (p.epi == EPI_ADD) {   // key-aligned join with the addend relation: same block, same cell
                                 const uint4 rv = *reinterpret_cast<const uint4*>(p.r_base + off + g * 16);
-                                const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&rv);
+                                const uint32_t* pr = reinterpret_cast<const uint32_t*>(&rv);
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    const float2 rf = __bfloat1622float2(pr[e]);
+                                    const float2 rf = ja_unpack16<F16>(pr[e]);
                                     f[2 * e] += rf.x;
                                     f[2 * e + 1] += rf.y;
                                 }
                             }
                             uint4 o;
-                            __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+                            uint32_t* po = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+                            for (int e = 0; e < 4; ++e) po[e] = ja_pack16<F16>(f[2 * e], f[2 * e + 1]);
                             *reinterpret_cast<uint4*>(dst + g * 16) = o;
                         }
                     }
@@ -433,7 +438,8 @@ ja_status_t encode_blocked_2d(const ja_relation* r, int box_inner, int box_rows,
     cuuint64_t strides[3] = {(cuuint64_t)(bc * 2), (cuuint64_t)blk_stride, (cuuint64_t)(blk_stride * r->nblk[1])};
     cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult res = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, r->base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const CUtensorMapDataType cell = r->dtype == JA_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUresult res = enc(tm, cell, 4, r->base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)res);
     return JA_OK;
@@ -452,6 +458,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
                             std::shared_ptr<GemmTcPlan>* out, bool* eligible) {
     *eligible = false;
     if (!A->equal_blocks || !B->equal_blocks || !C->equal_blocks) return JA_OK;
+    if (A->dtype == JA_F32 || B->dtype != A->dtype || (C->esize == 2 && C->dtype != A->dtype)) return JA_OK;
     const int epi = ep ? ep->epi : 0;
     const int bn_tile = epi == EPI_SWIGLU ? 128 : BN;
     if (epi == EPI_SWIGLU && (B->bs[1] % 128 != 0 || !ep->B2 || !ep->B2->equal_blocks)) return JA_OK;
@@ -474,6 +481,7 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     p.bn_tile = bn_tile;
     p.n_copies = (ep && ep->partials) ? p.nbk : 1;
     p.c_esize = C->esize;
+    p.f16 = A->dtype == JA_F16;
     if (p.c_esize == 4 && !(ep && ep->partials)) return JA_OK;
     p.r_base = (epi == EPI_ADD) ? (const char*)ep->addend->base : nullptr;
     p.rope_table = (epi == EPI_ROPE) ? ep->rope_table : nullptr;
@@ -501,8 +509,13 @@ ja_status_t ja_gemm_tc_plan(const ja_relation* A, const ja_relation* B, const ja
     const int sms = ja_sm_count();
     const int tiles = p.m_tiles * p.n_tiles * p.n_copies;
     plan->grid = two ? 2 * std::min(sms / 2, tiles) : std::min(sms, tiles);
-    cudaError_t e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
-                        : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES);
+    cudaError_t e;
+    if (p.f16)
+        e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
+                : cudaFuncSetAttribute(gemm_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES);
+    else
+        e = two ? cudaFuncSetAttribute(gemm_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES)
+                : cudaFuncSetAttribute(gemm_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES);
     if (e != cudaSuccess) return ja_cuda_fail(e, "cudaFuncSetAttribute(gemm_tc_kernel)");
     *out = plan;
     *eligible = true;
@@ -528,9 +541,11 @@ ja_status_t ja_launch_gemm_tc(const GemmTcPlan& plan, cudaStream_t st) {
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, plan.tmA, plan.tmB, plan.tmB2, p));
+        if (p.f16) JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, true>, plan.tmA, plan.tmB, plan.tmB2, p));
+        else JA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false>, plan.tmA, plan.tmB, plan.tmB2, p));
     } else {
-        gemm_tc_kernel<1><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, p);
+        if (p.f16) gemm_tc_kernel<1, true><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, p);
+        else gemm_tc_kernel<1, false><<<plan.grid, NUM_THREADS, Cfg<1>::SMEM_BYTES, st>>>(plan.tmA, plan.tmB, plan.tmB2, p);
         JA_CUDA(cudaGetLastError());
     }
     ja_count_launch();

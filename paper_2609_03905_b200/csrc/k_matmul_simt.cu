@@ -41,18 +41,21 @@ __device__ __forceinline__ int64_t block_offset(const RelView& v, int64_t flat) 
 template <typename T> struct VecOf;
 template <> struct VecOf<float> { typedef float4 type; static constexpr int W = 4; };
 template <> struct VecOf<__nv_bfloat16> { typedef uint4 type; static constexpr int W = 8; };
+template <> struct VecOf<__half> { typedef uint4 type; static constexpr int W = 8; };
 
 template <typename T, int W> __device__ __forceinline__ void unpack_vec(const typename VecOf<T>::type& v, float (&f)[W]);
 template <> __device__ __forceinline__ void unpack_vec<float, 4>(const float4& v, float (&f)[4]) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
-template <> __device__ __forceinline__ void unpack_vec<__nv_bfloat16, 8>(const uint4& v, float (&f)[8]) {
-    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+template <bool F16> __device__ __forceinline__ void unpack_16bit(const uint4& v, float (&f)[8]) {
+    const uint32_t* p = reinterpret_cast<const uint32_t*>(&v);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const float2 t = __bfloat1622float2(p[e]);
+        const float2 t = ja_unpack16<F16>(p[e]);
         f[2 * e] = t.x;
         f[2 * e + 1] = t.y;
     }
 }
+template <> __device__ __forceinline__ void unpack_vec<__nv_bfloat16, 8>(const uint4& v, float (&f)[8]) { unpack_16bit<false>(v, f); }
+template <> __device__ __forceinline__ void unpack_vec<__half, 8>(const uint4& v, float (&f)[8]) { unpack_16bit<true>(v, f); }
 
 // TM x TN output tile, 256 threads, (TM/16) x (TN/16) outputs per thread. VECTOR: 16-byte operand loads.
 // TK: contracted cells per chunk (64 with the small tiles: a small problem is bound by the latency of its chunk loads)
@@ -208,8 +211,8 @@ __global__ void __launch_bounds__(NT) matmul_simt_kernel(const SimtParams p) {
             if (sizeof(T) == 4) {
                 *reinterpret_cast<float4*>(dst) = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
             } else {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(acc[u][0], acc[u][1]), hi = __floats2bfloat162_rn(acc[u][2], acc[u][3]);
-                *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                constexpr bool F16 = JaDtypeOf<T>::value == JA_F16;
+                *reinterpret_cast<uint2*>(dst) = make_uint2(ja_pack16<F16>(acc[u][0], acc[u][1]), ja_pack16<F16>(acc[u][2], acc[u][3]));
             }
         } else {
 #pragma unroll
@@ -255,6 +258,9 @@ ja_status_t ja_launch_matmul_simt(const ja_relation* Ar, const ja_relation* Br, 
     if (dt == JA_F32) {
         if (small) launch<float, 32, 32>(p, grid, vec, st);
         else launch<float, 64, 64>(p, grid, vec, st);
+    } else if (dt == JA_F16) {
+        if (small) launch<__half, 32, 32>(p, grid, vec, st);
+        else launch<__half, 64, 64>(p, grid, vec, st);
     } else {
         if (small) launch<__nv_bfloat16, 32, 32>(p, grid, vec, st);
         else launch<__nv_bfloat16, 64, 64>(p, grid, vec, st);

@@ -3,6 +3,7 @@
 #include "k_membound_impl.cuh"
 
 ja_status_t ja_launch_row_f32(RowOp op, const RowArgs& a, cudaStream_t st);
+ja_status_t ja_launch_row_f16(RowOp op, const RowArgs& a, cudaStream_t st);
 
 ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,
                            cudaStream_t st) {
@@ -11,8 +12,11 @@ ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, 
     int64_t want = (n_vec + 255) / 256;
     unsigned grid = (unsigned)(want < (int64_t)148 * 32 ? (want > 0 ? want : 1) : (int64_t)148 * 32);
     if (dt == JA_BF16) {
-        if (fn == JA_FN_ADD) flat_bf16_kernel<JA_FN_ADD><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
-        else flat_bf16_kernel<JA_FN_SILU_MUL><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
+        if (fn == JA_FN_ADD) flat_16bit_kernel<JA_FN_ADD, false><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
+        else flat_16bit_kernel<JA_FN_SILU_MUL, false><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
+    } else if (dt == JA_F16) {
+        if (fn == JA_FN_ADD) flat_16bit_kernel<JA_FN_ADD, true><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
+        else flat_16bit_kernel<JA_FN_SILU_MUL, true><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, (uint4*)out, n_vec);
     } else {
         if (fn == JA_FN_ADD) flat_f32_kernel<JA_FN_ADD><<<grid, 256, 0, st>>>((const float4*)a, (const float4*)b, (float4*)out, n_vec);
         else flat_f32_kernel<JA_FN_SILU_MUL><<<grid, 256, 0, st>>>((const float4*)a, (const float4*)b, (float4*)out, n_vec);
@@ -27,5 +31,7 @@ ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_
     bool launched = false;
     ja_status_t s = ja_launch_row_tma(op, a, dt, st, &launched);
     if (s != JA_OK || launched) return s;
-    return dt == JA_F32 ? ja_launch_row_f32(op, a, st) : launch_row_typed<__nv_bfloat16>(op, a, st);
+    if (dt == JA_F32) return ja_launch_row_f32(op, a, st);
+    if (dt == JA_F16) return ja_launch_row_f16(op, a, st);
+    return launch_row_typed<__nv_bfloat16>(op, a, st);
 }

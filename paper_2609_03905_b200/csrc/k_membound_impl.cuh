@@ -27,18 +27,19 @@ __device__ __forceinline__ float flat_fn(float a, float b) {
     return FN == JA_FN_ADD ? a + b : silu_mul_f(a, b);
 }
 
-template <int FN>
-__global__ void __launch_bounds__(256) flat_bf16_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b,
-                                                        uint4* __restrict__ out, int64_t n_vec) {
+// eight 16-bit cells per 16-byte vector; F16: false = bf16, true = f16
+template <int FN, bool F16>
+__global__ void __launch_bounds__(256) flat_16bit_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b,
+                                                         uint4* __restrict__ out, int64_t n_vec) {
     for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * 256) {
         uint4 va = a[i], vb = b[i], vo;
-        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va);
-        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&vb);
-        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&vo);
+        const uint32_t* pa = reinterpret_cast<const uint32_t*>(&va);
+        const uint32_t* pb = reinterpret_cast<const uint32_t*>(&vb);
+        uint32_t* po = reinterpret_cast<uint32_t*>(&vo);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            float2 fa = __bfloat1622float2(pa[k]), fb = __bfloat1622float2(pb[k]);
-            po[k] = __floats2bfloat162_rn(flat_fn<FN>(fa.x, fb.x), flat_fn<FN>(fa.y, fb.y));
+            const float2 fa = ja_unpack16<F16>(pa[k]), fb = ja_unpack16<F16>(pb[k]);
+            po[k] = ja_pack16<F16>(flat_fn<FN>(fa.x, fb.x), flat_fn<FN>(fa.y, fb.y));
         }
         out[i] = vo;
     }
@@ -551,7 +552,7 @@ ja_status_t launch_row_op(RowOp op, const RowArgs& a, int vec, int64_t n_rows, i
 
 template <typename T>
 ja_status_t launch_row_typed(RowOp op, const RowArgs& a, cudaStream_t st) {
-    const ja_dtype_t dt = sizeof(T) == 4 ? JA_F32 : JA_BF16;
+    const ja_dtype_t dt = JaDtypeOf<T>::value;
     const int last = a.x.rank - 1;
     const int64_t n = a.x.extent[last];
     int64_t n_rows = 1;

@@ -11,6 +11,9 @@ namespace {
 template <typename T> struct VecOf;
 template <> struct VecOf<float> { static constexpr int N = 4; };            // 16 bytes
 template <> struct VecOf<__nv_bfloat16> { static constexpr int N = 8; };    // 16 bytes
+template <> struct VecOf<__half> { static constexpr int N = 8; };
+template <typename T> struct IsF16 { static constexpr bool value = false; };
+template <> struct IsF16<__half> { static constexpr bool value = true; };
 
 template <typename TS, int VEC> __device__ __forceinline__ void load_cells(const char* p, float* f) {
     if (VEC == 1) {
@@ -20,10 +23,10 @@ template <typename TS, int VEC> __device__ __forceinline__ void load_cells(const
         if (sizeof(TS) == 4) {
             f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
         } else {
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+            const uint32_t* h = reinterpret_cast<const uint32_t*>(&v);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float2 t = __bfloat1622float2(h[e]);
+                const float2 t = ja_unpack16<IsF16<TS>::value>(h[e]);
                 f[2 * e] = t.x;
                 f[2 * e + 1] = t.y;
             }
@@ -39,15 +42,14 @@ template <typename TD, int VEC> __device__ __forceinline__ void store_cells(char
         for (int e = 0; e < VEC; e += 4) *reinterpret_cast<float4*>(p + e * 4) = make_float4(f[e], f[e + 1], f[e + 2], f[e + 3]);
     } else if (VEC == 8) {
         uint4 o;
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+        uint32_t* h = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+        for (int e = 0; e < 4; ++e) h[e] = ja_pack16<IsF16<TD>::value>(f[2 * e], f[2 * e + 1]);
         *reinterpret_cast<uint4*>(p) = o;
-    } else {   // 4 bf16 cells
+    } else {   // 4 cells of 16 bits
         uint2 o;
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
-        h[0] = __floats2bfloat162_rn(f[0], f[1]);
-        h[1] = __floats2bfloat162_rn(f[2], f[3]);
+        o.x = ja_pack16<IsF16<TD>::value>(f[0], f[1]);
+        o.y = ja_pack16<IsF16<TD>::value>(f[2], f[3]);
         *reinterpret_cast<uint2*>(p) = o;
     }
 }
@@ -110,10 +112,19 @@ ja_status_t ja_launch_repartition_agg(const char* src, char* dst, const CopySlab
     if (n_slabs == 0) return JA_OK;
     const unsigned grid = (unsigned)(n_slabs < (int64_t)148 * 64 ? n_slabs : (int64_t)148 * 64);
     const bool is_max = agg == JA_AGG_MAX, v = vec > 1;
-    if (src_dt == JA_F32 && dst_dt == JA_F32) launch<float, float>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
-    else if (src_dt == JA_F32) launch<float, __nv_bfloat16>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
-    else if (dst_dt == JA_F32) launch<__nv_bfloat16, float>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
-    else launch<__nv_bfloat16, __nv_bfloat16>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st);
+    // partial and destination relations: f32 or one 16-bit type (never bf16 on one side and f16 on the other)
+    if (src_dt != JA_F32 && dst_dt != JA_F32 && src_dt != dst_dt)
+        return ja_fail(JA_ERR_DTYPE, "aggregating relayout: partials and destination of different 16-bit types");
+    const bool f16 = src_dt == JA_F16 || dst_dt == JA_F16;
+#define JA_AGG_LAUNCH(TS, TD) launch<TS, TD>(src, dst, d_slabs, n_slabs, n_copies, copy_stride, is_max, v, grid, st)
+    if (src_dt == JA_F32 && dst_dt == JA_F32) JA_AGG_LAUNCH(float, float);
+    else if (src_dt == JA_F32 && f16) JA_AGG_LAUNCH(float, __half);
+    else if (src_dt == JA_F32) JA_AGG_LAUNCH(float, __nv_bfloat16);
+    else if (dst_dt == JA_F32 && f16) JA_AGG_LAUNCH(__half, float);
+    else if (dst_dt == JA_F32) JA_AGG_LAUNCH(__nv_bfloat16, float);
+    else if (f16) JA_AGG_LAUNCH(__half, __half);
+    else JA_AGG_LAUNCH(__nv_bfloat16, __nv_bfloat16);
+#undef JA_AGG_LAUNCH
     ja_count_launch();
     JA_CUDA(cudaGetLastError());
     return JA_OK;

@@ -92,7 +92,7 @@ extern "C" ja_status_t ja_repartition_noalloc(int32_t rank, const int64_t* exten
                                               void* dst_device, void* cuda_stream) {
     if (rank < 1 || rank > JA_MAX_RANK || !extents || !src_nparts || !src_splits || !dst_nparts || !dst_splits)
         return ja_fail(JA_ERR_INVALID_ARG, "rank must be 1..%d and every array non-NULL", JA_MAX_RANK);
-    if (dtype != JA_F32 && dtype != JA_BF16) return ja_fail(JA_ERR_DTYPE, "unknown dtype %d", (int)dtype);
+    if (dtype != JA_F32 && dtype != JA_BF16 && dtype != JA_F16) return ja_fail(JA_ERR_DTYPE, "unknown dtype %d", (int)dtype);
     if (!src_device || !dst_device || src_device == dst_device) return ja_fail(JA_ERR_INVALID_ARG, "payload pointers must be distinct and non-NULL");
     if (((uintptr_t)src_device | (uintptr_t)dst_device) % JA_ALIGN) return ja_fail(JA_ERR_ALIGNMENT, "payloads must be %d-byte aligned", JA_ALIGN);
     const int es = dtype == JA_F32 ? 4 : 2;

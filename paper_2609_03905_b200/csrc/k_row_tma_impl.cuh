@@ -23,6 +23,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "ja_device.cuh"
 #include "ja_ptx.cuh"
@@ -513,7 +514,7 @@ __global__ void __launch_bounds__(NUM_THREADS, (ctas_per_sm<T, OP, VPL>())) row_
                 if (r >= rows || !team.ok) break;
                 uint8_t* rowp = stage + (size_t)r * row_seg_bytes;
                 const int64_t stat_off = lb * g.stat_blk_bytes + (int64_t)(r0 + r) * 4;
-                if constexpr (sizeof(T) == 2) {
+                if constexpr (std::is_same<T, __nv_bfloat16>::value) {
                     if (full_rows) row_bf16<OP, VPL, true>(a, g, rowp, off, g_s, stat_off, cur0[q], cur1[q], lane, team);
                     else row_bf16<OP, VPL, false>(a, g, rowp, off, g_s, stat_off, cur0[q], cur1[q], lane, team);
                 }
@@ -588,7 +589,10 @@ ja_status_t encode_rows4(const RelView& v, const RowTmaGeom& g, int64_t n_lead, 
     cuuint64_t strides[3] = {(cuuint64_t)g.bsc * es, (cuuint64_t)g.blk_bytes, (cuuint64_t)g.blk_bytes * g.nbc};
     cuuint32_t box[4] = {(cuuint32_t)g.bw, (cuuint32_t)g.R, (cuuint32_t)g.nbc, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult res = enc(tm, dt == JA_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, v.base, dims, strides, box,
+    const CUtensorMapDataType cell = dt == JA_F32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                     : dt == JA_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                    : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUresult res = enc(tm, cell, 4, v.base, dims, strides, box,
                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (res != CUDA_SUCCESS) return ja_fail(JA_ERR_CUDA, "cuTensorMapEncodeTiled (row strips) failed with code %d", (int)res);
@@ -600,7 +604,7 @@ ja_status_t encode_rows4(const RelView& v, const RowTmaGeom& g, int64_t n_lead, 
 // more than 256 column blocks, RoPE (its rotation needs the row's coordinates).
 template <typename T>
 ja_status_t row_tma_launch(RowOp op, const RowArgs& a, cudaStream_t st, bool* launched) {
-    const ja_dtype_t dt = sizeof(T) == 4 ? JA_F32 : JA_BF16;
+    const ja_dtype_t dt = JaDtypeOf<T>::value;
     *launched = false;
     if (op == ROW_ROPE) return JA_OK;
     if (ja_config().row_tma == 0) return JA_OK;

@@ -31,7 +31,8 @@ from .relations import Relation, Spec, equal_splits as ES, from_dense, repartiti
 class LlamaBlock:
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, plan: str = "seq",
                  theta: float = 1e4, eps: float = 1e-5, token_block: int = 128, col_blocks: int = 8,
-                 ffn_blocks: int | None = None, fused: bool = True, n_kv_heads: int | None = None):
+                 ffn_blocks: int | None = None, fused: bool = True, n_kv_heads: int | None = None,
+                 dtype: torch.dtype = torch.bfloat16):
         assert plan in ("seq", "head", "mixed")
         self.fused = fused
         assert hidden % n_heads == 0 and hidden // n_heads == 128, "attention kernel needs head dimension 128"
@@ -43,7 +44,8 @@ class LlamaBlock:
         kv_hidden = self.kv_hidden
         T = batch * seq
         self.T = T
-        bf = torch.bfloat16
+        assert dtype in (torch.bfloat16, torch.float16), "the block's relations are bf16 (the benchmark configurations) or f16 (the paper's precision)"
+        bf = self.dtype = dtype                          # cell type of every relation of the block
         D = hidden // n_heads
         t_sp = ES(T, T // token_block)
         io_c = ES(hidden, col_blocks)                    # column tiling of the block's input / output

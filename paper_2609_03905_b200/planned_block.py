@@ -82,7 +82,7 @@ class PlannedBlock:
     """counts: one {letter: intervals} dict per operator of block_graph(), e.g. the plan of ja_plan_optimize_graph."""
 
     def __init__(self, batch: int, seq: int, hidden: int, n_heads: int, ffn: int, weights: dict, counts, theta: float = 1e4,
-                 eps: float = 1e-5, fused: bool = True, share_relayouts: bool = False):
+                 eps: float = 1e-5, fused: bool = True, share_relayouts: bool = False, dtype: torch.dtype = torch.bfloat16):
         assert hidden // n_heads == 128, "the attention kernels need head dimension 128"
         self.B, self.S, self.hidden, self.H, self.ffn = batch, seq, hidden, n_heads, ffn
         self.T = batch * seq
@@ -92,7 +92,8 @@ class PlannedBlock:
         assert len(self.counts) == len(self.ops)
         for op, c in zip(self.ops, self.counts):
             assert c.get("d", 1) == 1, "the head dimension is not shardable"
-        bf = torch.bfloat16
+        assert dtype in (torch.bfloat16, torch.float16)
+        bf = self.dtype = dtype    # cell type of every relation of the block
         w = {n: weights[n].to("cuda", bf) for n in weights}
         ops, cn = self.ops, self.counts
         self.steps = []            # (name, callable) in execution order
@@ -101,7 +102,7 @@ class PlannedBlock:
 
         def out_tensor(i):
             _, out = _terms(ops[i]["einsum"])
-            return _Tensor(out, ops[i]["extents"], cn[i])
+            return self._tensor(out, ops[i]["extents"], cn[i])
         self.out_t = [out_tensor(i) for i in range(len(ops))]
 
         def operand(i, k, dense=None, name=""):
@@ -111,14 +112,14 @@ class PlannedBlock:
             term = ins[k]
             prod = ops[i]["inputs"][k]
             if prod is None:
-                return _Tensor(term, ops[i]["extents"], cn[i], dense=dense)
+                return self._tensor(term, ops[i]["extents"], cn[i], dense=dense)
             src = self.out_t[prod]
             want = tuple(cn[i][c] for c in term)
             if want == src.counts:
                 return src
             key = (prod, want) if share_relayouts else (prod, want, i, k)   # the plan's Cost charges every consuming operand
             if key not in self._relaid:
-                dst = _Tensor(term, ops[i]["extents"], cn[i])
+                dst = self._tensor(term, ops[i]["extents"], cn[i])
                 self._relaid[key] = dst
                 self.steps.append((f"repartition_{name or prod}_for_{i}", lambda s=src, d=dst: repartition(s.rel, d.rel)))
                 self.n_relayouts += 1
@@ -141,7 +142,7 @@ class PlannedBlock:
                 self.steps.append((name, run(Spec("ij,jk->ik", parts), [A2, W2], C2)))
 
         # ---- 0: n1 = RMSNorm(x, g1) -------------------------------------------------------------------------------
-        self.x = _Tensor("bse", ops[0]["extents"], cn[0])                   # block input, in the tiling operator 0 reads it in
+        self.x = self._tensor("bse", ops[0]["extents"], cn[0])                   # block input, in the tiling operator 0 reads it in
         g1 = operand(0, 1, w["g1"])
         x2, n1 = self.x.rows_view(2), self.out_t[0]
         self.steps.append(("rmsnorm_1", run(Spec("ij,j->ij", {"i": x2.splits[0], "j": x2.splits[1]}, "rmsnorm", (eps,), "none"),
@@ -157,7 +158,7 @@ class PlannedBlock:
             # rows of a two-index view follow the token order only when a row block never mixes sequences with a cut sequence
             natural = cn[i]["s"] == 1 or cn[i]["b"] == batch
             parts = {"i": A2.splits[0], "j": A2.splits[1], "k": W2.splits[1]}
-            pre = _Tensor(out.letters, ops[i]["extents"], cn[i])               # before the rotation (unfused chain)
+            pre = self._tensor(out.letters, ops[i]["extents"], cn[i])               # before the rotation (unfused chain)
             s_rope = Spec("bshd->bshd", dict(zip("bshd", pre.splits)), "rope", (theta,), "none")
 
             def unfused(parts=parts, A2=A2, W2=W2, pre=pre, out=out, s_rope=s_rope):
@@ -223,7 +224,7 @@ class PlannedBlock:
         want = tuple(counts[c] for c in letters)
         if want == x.counts:
             return x
-        dst = _Tensor(letters, extents, counts)
+        dst = self._tensor(letters, extents, counts)
         self.steps.append(("repartition_x", lambda: repartition(x.rel, dst.rel)))
         self.n_input_relayouts += 1
         return dst
@@ -252,6 +253,9 @@ class PlannedBlock:
                     state["chain"] = make_chain()
             state["chain"]()
         return call
+
+    def _tensor(self, letters, extents, counts, dense=None):
+        return _Tensor(letters, extents, counts, self.dtype, dense)
 
     def load_input(self, x_dense: torch.Tensor):
         """Pack a dense [batch * seq, hidden] CUDA tensor into the block's input relation (a relayout from one block)."""

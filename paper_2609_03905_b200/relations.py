@@ -8,7 +8,7 @@ import torch
 
 from . import binding as B
 
-_DT = {torch.float32: B.JA_F32, torch.bfloat16: B.JA_BF16}
+_DT = {torch.float32: B.JA_F32, torch.bfloat16: B.JA_BF16, torch.float16: B.JA_F16}
 
 
 def equal_splits(extent: int, n: int):

@@ -38,6 +38,31 @@ def test_round_bf16_matches_torch_and_ties_to_even():
     assert np.array_equal(core.round_to(x, "f32"), x.astype(np.float32).astype(np.float64))
 
 
+def test_round_f16_matches_numpy_and_torch_ties_range_and_subnormals():
+    """IEEE binary16, the storage type of the paper's experiments (Section 6): one rounding from fp64, ties to even,
+    overflow to infinity from 65520 on, subnormals in steps of 2^-24. numpy converts fp64 to float16 with one correct
+    rounding; torch is fed fp32-representable values (it rounds from fp32)."""
+    x = np.concatenate([RNG.standard_normal(20000) * 10.0 ** RNG.integers(-9, 5, 20000),
+                        [0.0, 1.0, 65504.0, 65519.9, 65520.0, -65520.0, 70000.0, 2.0 ** -14, 2.0 ** -24, 2.0 ** -25,
+                         1.5 * 2.0 ** -24, 2.5 * 2.0 ** -24, 2.0 ** -25 * (1 + 2.0 ** -30), 1e-9]])
+    with np.errstate(over="ignore"):
+        assert np.array_equal(core.round_to(x, "f16"), x.astype(np.float16).astype(np.float64))
+    x32 = x.astype(np.float32).astype(np.float64)
+    want = torch.from_numpy(x32.astype(np.float32)).to(torch.float16).to(torch.float64).numpy()
+    assert np.array_equal(core.round_to(x32, "f16"), want)
+    # exact ties: 1 + 2^-11 lies midway between 1 and 1 + 2^-10 -> 1.0 (even); 1 + 3 * 2^-11 -> 1 + 2^-9
+    assert core.round_to([1.0 + 2.0 ** -11], "f16")[0] == 1.0
+    assert core.round_to([1.0 + 3 * 2.0 ** -11], "f16")[0] == 1.0 + 2.0 ** -9
+    # one rounding from fp64, not two: just above the tie rounds up (fp64 -> fp32 -> f16 would land on the tie and round down)
+    assert core.round_to([1.0 + 2.0 ** -11 + 2.0 ** -40], "f16")[0] == 1.0 + 2.0 ** -10
+    # range and subnormals
+    r = core.round_to([65519.9, 65520.0, 2.0 ** -25, 1.5 * 2.0 ** -24, 2.5 * 2.0 ** -24], "f16")
+    assert r[0] == 65504.0 and np.isinf(r[1]) and r[2] == 0.0 and r[3] == 2.0 ** -23 and r[4] == 2.0 ** -23
+    # f16 keeps three more bits than bf16 on the same values
+    v = RNG.standard_normal(4096)
+    assert np.abs(core.round_to(v, "f16") - v).max() < np.abs(core.round_to(v, "bf16") - v).max() / 4
+
+
 # ---------------------------------------------------------------------------------------------
 # the three engines against brute force (tiny inputs, every extent <= 6)
 # ---------------------------------------------------------------------------------------------
