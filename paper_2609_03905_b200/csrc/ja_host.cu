@@ -62,6 +62,7 @@ JaConfig& ja_config() {
         cfg.gemm_loader = env_int("JA_GEMM_LOADER", -1);
         cfg.row_tma = env_int("JA_ROW_TMA", -1);
         cfg.row_team = env_int("JA_ROW_TEAM", -1);
+        cfg.row_reduce = env_int("JA_ROW_REDUCE", -1);
         if (const char* v = getenv("JA_WAIT_CAP")) {
             const long long ns = atoll(v);
             if (ns >= 1000 && ns <= 4000000000000ll) cfg.wait_cap_us = ns / 1000;
@@ -78,7 +79,8 @@ extern "C" ja_status_t ja_debug_set(const char* name, int64_t value) {
         {"attn_mma_sync", &c.attn_mma_sync}, {"attn_one_tile", &c.attn_one_tile}, {"attn_persistent", &c.attn_persistent},
         {"attn_section", &c.attn_section}, {"attn_variant", &c.attn_variant}, {"gemm_cta_group", &c.gemm_cta_group},
         {"gemm_group_m", &c.gemm_group_m}, {"gemm_heavy_first", &c.gemm_heavy_first}, {"gemm_split", &c.gemm_split},
-        {"gemm_loader", &c.gemm_loader}, {"row_tma", &c.row_tma}, {"row_team", &c.row_team}};
+        {"gemm_loader", &c.gemm_loader}, {"row_tma", &c.row_tma}, {"row_team", &c.row_team},
+        {"row_reduce", &c.row_reduce}};
     for (auto& e : ints)
         if (n == e.key) {
             *e.field = (int)value;

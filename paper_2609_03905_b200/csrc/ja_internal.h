@@ -97,6 +97,7 @@ struct JaConfig {
     int gemm_loader = -1;       // JA_GEMM_LOADER       1: operands staged by plain loads even where TMA could take them; 0: never
     int row_tma = -1;           // JA_ROW_TMA           0: row join-aggs without the TMA-staged kernel
     int row_team = -1;          // JA_ROW_TEAM          n: threads per row of the plain row kernel
+    int row_reduce = -1;        // JA_ROW_REDUCE        0: statistics-only row forms never take the plain read-stream kernel, 1: whenever the tiling fits
     int64_t wait_cap_us = 2000000;   // JA_WAIT_CAP (nanoseconds in the environment): limit of every device-side wait
 };
 JaConfig& ja_config();
@@ -135,6 +136,8 @@ struct RowArgs {
 ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st);
 // bulk-copy pipelined form for uniform tilings; *launched stays false when the shape does not fit it
 ja_status_t ja_launch_row_tma(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched);
+// statistics-only forms (sum of squares, row maximum, sum of exponentials) as a plain read stream; *launched as above
+ja_status_t ja_launch_row_reduce(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st, bool* launched);
 ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, int64_t n_elems, ja_dtype_t dt,
                            cudaStream_t st);
 

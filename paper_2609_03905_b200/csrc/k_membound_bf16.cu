@@ -27,9 +27,12 @@ ja_status_t ja_launch_flat(ja_fn_t fn, const void* a, const void* b, void* out, 
 }
 
 ja_status_t ja_launch_row(RowOp op, const RowArgs& a, ja_dtype_t dt, cudaStream_t st) {
-    // uniform tilings: bulk-copy pipeline through shared memory
     bool launched = false;
-    ja_status_t s = ja_launch_row_tma(op, a, dt, st, &launched);
+    // statistics-only forms on uniform tilings: a plain read stream
+    ja_status_t s = ja_launch_row_reduce(op, a, dt, st, &launched);
+    if (s != JA_OK || launched) return s;
+    // uniform tilings: bulk-copy pipeline through shared memory
+    s = ja_launch_row_tma(op, a, dt, st, &launched);
     if (s != JA_OK || launched) return s;
     if (dt == JA_F32) return ja_launch_row_f32(op, a, st);
     if (dt == JA_F16) return ja_launch_row_f16(op, a, st);

@@ -18,7 +18,7 @@ def golden_dir():
 
 
 SWITCHES = ("attn_mma_sync", "attn_one_tile", "attn_persistent", "attn_section", "attn_variant", "gemm_cta_group", "gemm_group_m",
-            "gemm_heavy_first", "gemm_split", "gemm_loader", "row_tma", "row_team")
+            "gemm_heavy_first", "gemm_split", "gemm_loader", "row_tma", "row_team", "row_reduce")
 
 
 @pytest.fixture(autouse=True)

@@ -243,6 +243,35 @@ def test_softmax_join_aggs(shape, sh, si_, sj, dtype):
 
 
 @pytest.mark.parametrize("dtype", [BF, F32, F16])
+@pytest.mark.parametrize("form", [1, 0])     # the plain read-stream kernel for all three statistics / never
+def test_row_statistics_both_forms(dtype, form):
+    """Sum of squares, row maximum and sum of exponentials as statistics-only join-aggs through both kernels that take
+    them on uniform tilings (by default the choice depends on the form and the size), incl. rows that are not a whole
+    number of 32-vector steps, three leading indices and more rows than resident warps."""
+    ja.ja_debug_set("row_reduce", form)
+    for shape, splits in (((6000, 1024), [ES(6000, 3), ES(1024, 8)]),
+                          ((3, 40, 2000), [ES(3, 3), ES(40, 2), ES(2000, 5)]),
+                          ((2, 3, 16, 264), [ES(2, 1), ES(3, 3), ES(16, 4), ES(264, 1)])):
+        X = si.normal(shape, 0.0, 2.0, dtype, 3, 7)
+        x64 = si.to_f64(X).reshape(-1, shape[-1])
+        rX = upload(X, splits)
+        letters = "abcd"[: len(shape) - 1]
+        parts = dict(zip(letters + "j", splits))
+        stat = lambda: empty_like_tiling(list(shape[:-1]), splits[:-1], F32, fill=float("nan"))
+        rSS, rM, rL = stat(), stat(), stat()
+        before = ja.ja_launch_count()
+        ja.Spec(f"{letters}j->{letters}", parts, "square", (), "sum").execute([rX], rSS)
+        ja.Spec(f"{letters}j->{letters}", parts, "ident", (), "max").execute([rX], rM)
+        ja.Spec(f"{letters}j,{letters}->{letters}", parts, "exp_sub", (), "sum").execute([rX, rM], rL)
+        assert ja.ja_launch_count() == before + 3
+        m = x64.max(axis=1)
+        assert relfro(download(rSS).reshape(-1), (x64 * x64).sum(axis=1)) <= 1e-5
+        assert np.array_equal(download(rM).reshape(-1), m)
+        assert relfro(download(rL).reshape(-1), np.exp(x64 - m[:, None]).sum(axis=1)) <= 1e-5
+    check_status()
+
+
+@pytest.mark.parametrize("dtype", [BF, F32, F16])
 def test_key_aligned_maps(dtype):
     for shape, sp in (((256, 1376), [ES(256, 2), ES(1376, 1)]), ((50, 70), [[0, 13, 50], [0, 33, 70]])):
         a = si.normal(shape, 0.0, 1.5, dtype, 2, 4)
