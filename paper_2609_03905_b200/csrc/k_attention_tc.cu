@@ -529,6 +529,12 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   between the groups with setmaxnreg, output written straight from registers): 6 % slower -- the output stage is not
 //   what an item waits for. Not possible: P in f16 from ex2.approx.f16x2 (two exponentials per instruction) against bf16
 //   V -- tcgen05.mma kind::f16 with different formats for A and B is an illegal instruction.
+//   Built, verified against the oracle and dropped for the same reason as the shared-memory analysis below suggested it:
+//   FOUR tiles on a pair of CTAs, both products as tcgen05.mma.cta_group::2 with M = 256 and the K / V tile split between
+//   the two SMs (each SM then reads and is filled with half of every K / V tile: a quarter less traffic on the
+//   shared-memory port per product). B4 S2048 causal 0.230 ms against 0.140, one sequence of 16384 rows 2.79 against
+//   1.80 ms: every key step then has two hand-offs that cross the cluster (the peer's P ready -> the leader's MMA warp;
+//   the products' commit -> the peer's row warps), and their latency sits on the chain that already bounds the kernel.
 //   Counters of the steady state: per 128 x 128 x 128 product pair the two smem x smem products read 128 KiB of shared
 //   memory (1024 cycles of its 128 B/clk port, as long as the products themselves take), the P stores and the K / V fills
 //   add half as much again: the shared-memory port, not a pipe, bounds long sequences (tensor-core reads 53 % + stores
