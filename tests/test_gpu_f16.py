@@ -198,3 +198,21 @@ def test_llama_block_f16(plan):
     got = download(blk.forward())
     check_status()
     assert relfro(got.reshape(Bt * S, hidden), ref) <= TOL[F16]
+
+
+def test_optimizer_plan_on_small_block_f16():
+    """The logical optimizer's p = 8 plan executed with every relation in f16: relayouts wherever the plan charges one."""
+    from paper_2609_03905_b200.planned_block import PlannedBlock, block_graph, plan_repartition_charges
+    Bt, S, hidden, heads, ffn = 2, 512, 512, 4, 1408
+    ops = block_graph(Bt, S, hidden, heads, ffn)
+    _, plan = ja.ja_plan_optimize_graph(ops, 8)
+    w = si.llama_weights(hidden, ffn, config=5, dtype=F16, first_ordinal=21)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, F16, 5, 20)
+    blk = PlannedBlock(Bt, S, hidden, heads, ffn, w, plan, dtype=F16)
+    assert blk.n_relayouts == plan_repartition_charges(ops, plan)[0] > 0
+    blk.load_input(x.cuda())
+    got = download(blk.forward()).reshape(Bt * S, hidden)
+    check_status()
+    w64 = {k: si.to_f64(v) for k, v in w.items()}
+    ref = np.concatenate([operators.llama_block(si.to_f64(x[b * S:(b + 1) * S]), w64, heads, dtype="f16")["out"] for b in range(Bt)])
+    assert relfro(got, ref) <= TOL[F16]
