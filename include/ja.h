@@ -166,8 +166,9 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  *   "Rj,R,R->Rj"           EXP_SUB_DIV / NONE
  *   "Rj,j->Rj"             RMSNORM / NONE   (fused)       "Rj->Rj"  SOFTMAX / NONE (fused)
  *   "bshd->bshd"           ROPE / NONE
- *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128; q / k split points and sequence
- *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends multiples of 64 rows (tensor memory kernels: 128);
+ *   "bqhd,bkhd,bkhd->bqhd" ATTENTION / ONLINE_SOFTMAX     d unsplit, extent 128; any length, split points and sequence
+ *   "bqhd,bkgd,bkgd->bqhd"   (grouped-query form)         ends (tensor-memory kernels where all are multiples of 128 rows,
+ *                                                          mma.sync tiles for multiples of 64, a per-row form otherwise);
  *                                                          Q, K, V, O of one 16-bit dtype (bf16 or f16; the probabilities
  *                                                          enter the second product rounded to that dtype)
  * n_outputs is 1, except for ATTENTION where it may be 2: outputs[1] then receives lse[b, q, h] = log of the softmax

@@ -1126,7 +1126,6 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
             g = std::__gcd(g, (int64_t)aa.ends[i]);
         }
         aa.align = (int32_t)g;
-        if (aa.align % 64) return ja_fail(JA_ERR_UNSUPPORTED, "attention needs q/k split points and sequence ends that are multiples of 64 rows");
         aa.scale = spec->params.size() >= 1 ? (float)spec->params[0] : 0.08838834764831845f;
         aa.causal = spec->params.size() >= 2 ? (spec->params[1] != 0.0) : 1;
         std::vector<int32_t> qs(Q->splits[1].begin(), Q->splits[1].end()), ks(K->splits[1].begin(), K->splits[1].end());

@@ -14,6 +14,10 @@
 // This file holds the mma.sync form (m16n8k16, bf16 in, fp32 accumulate; operands staged in shared memory with
 // cp.async under an XOR swizzle and read with ldmatrix). It serves tilings the tensor-memory kernel cannot
 // take (64-row blocks); everything else is dispatched to the tcgen05 kernel.
+// RAGGED form of the same kernel: ANY split points of the sequence index, any sequence length and any sequence ends. Output
+// key tiles are then 64 consecutive positions wherever they fall: a tile may straddle blocks and packed sequences and run
+// past the end of the index, so every row is located on its own (block lookup per row), rows past the end are zero, and
+// the selection predicate of the spec -- same sequence, and not after the query when causal -- is applied per score.
 #include <stdlib.h>
 
 #include <algorithm>
@@ -68,7 +72,17 @@ __device__ __forceinline__ const char* row_ptr(const RelView& v, int b, int s, i
     return v.base + v.blk_off[flat] + ((((int64_t)(b - blo) * sw + (s - slo)) * hw + (h - hlo)) * D) * 2;
 }
 
-template <int QT, bool F16>
+// the packed sequence [s0, s1) that holds position pos (the whole index when sequences are not packed)
+__device__ __forceinline__ void seq_bounds(const AttnArgs& a, int pos, int& s0, int& s1) {
+    s0 = 0;
+    s1 = a.S;
+    for (int i = 0; i < a.n_ends; ++i) {
+        if (a.ends[i] <= pos) s0 = a.ends[i];
+        else { s1 = a.ends[i]; break; }
+    }
+}
+
+template <int QT, bool F16, bool RAGGED>
 __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     constexpr int NW = QT / 16;        // warps; each owns 16 query rows
     constexpr int NT = NW * 32;
@@ -79,43 +93,56 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int g = lane / 4, t4 = lane % 4;
 
-    const int n_qt = a.S / QT;
+    const int n_qt = (a.S + QT - 1) / QT;
     int slot, bh;
     ja_attn_decode_cta((int)blockIdx.x, n_qt, a.H * a.B, a.sect, &slot, &bh);
     const int qt = n_qt - 1 - slot;              // heaviest output keys (most surviving tuples) first
     const int h = bh % a.H, b = bh / a.H;
     const int q0 = qt * QT;
     const int hk = h / a.group;                  // key/value head joined with this query head
-    int s0 = 0, s1 = a.S;                        // the packed sequence this tile lies in (no tile straddles an end)
-    for (int i = 0; i < a.n_ends; ++i) {
-        if (a.ends[i] <= q0) s0 = a.ends[i];
-        else { s1 = a.ends[i]; break; }
+    int s0, s1;                                  // the packed sequence the tile's first row lies in (RAGGED: later rows may lie in later ones)
+    seq_bounds(a, q0, s0, s1);
+    const int q_last = min(q0 + QT, a.S) - 1;    // last position of the tile that exists
+    if (RAGGED) {
+        int unused;
+        seq_bounds(a, q_last, unused, s1);       // the key walk ends where the last row's sequence ends
     }
 
     // ---- stage Q, read its A fragments ---------------------------------------------------------------------
     {
         int64_t pitch;
-        const char* qp = row_ptr(a.q, b, q0, h, &pitch);  // a q tile never leaves its block (QT divides qblk)
+        const char* qp = RAGGED ? nullptr : row_ptr(a.q, b, q0, h, &pitch);  // a q tile never leaves its block (QT divides qblk)
         for (int i = tid; i < QT * 16; i += NT) {
             int r = i / 16, c = i % 16;
-            cp_async16(smem_u32(sQ) + swz(r, c), qp + (int64_t)r * pitch + c * 16);
+            if (!RAGGED) cp_async16(smem_u32(sQ) + swz(r, c), qp + (int64_t)r * pitch + c * 16);
+            else if (q0 + r < a.S) cp_async16(smem_u32(sQ) + swz(r, c), row_ptr(a.q, b, q0 + r, h, &pitch) + c * 16);
+            else *reinterpret_cast<uint4*>(sQ + swz(r, c)) = make_uint4(0u, 0u, 0u, 0u);
         }
         cp_async_commit();
     }
     // number of 64-row key steps this output key joins with: keys [s0, q0 + QT) when causal, else [s0, s1)
-    const int k_end = a.causal ? min(s1, q0 + QT) : s1;
+    const int k_end = a.causal ? min(s1, (RAGGED ? q_last + 1 : q0 + QT)) : s1;
     const int n_steps = (k_end - s0 + KT - 1) / KT;
 
     auto load_kv = [&](int step, int buf) {
         const int k0 = s0 + step * KT;  // a 64-row step never straddles a key block (64 divides every split point)
-        int64_t pk, pv;
-        const char* kp = row_ptr(a.k, b, k0, hk, &pk);
-        const char* vp = row_ptr(a.v, b, k0, hk, &pv);
+        int64_t pk = 0, pv = 0;
+        const char* kp = RAGGED ? nullptr : row_ptr(a.k, b, k0, hk, &pk);
+        const char* vp = RAGGED ? nullptr : row_ptr(a.v, b, k0, hk, &pv);
         const uint32_t dk = smem_u32(sK) + buf * KT * ROW_BYTES, dv = smem_u32(sV) + buf * KT * ROW_BYTES;
         for (int i = tid; i < KT * 16; i += NT) {
             int r = i / 16, c = i % 16;
-            cp_async16(dk + swz(r, c), kp + (int64_t)r * pk + c * 16);
-            cp_async16(dv + swz(r, c), vp + (int64_t)r * pv + c * 16);
+            if (!RAGGED) {
+                cp_async16(dk + swz(r, c), kp + (int64_t)r * pk + c * 16);
+                cp_async16(dv + swz(r, c), vp + (int64_t)r * pv + c * 16);
+            } else if (k0 + r < a.S) {   // every row on its own: a step may straddle key blocks
+                cp_async16(dk + swz(r, c), row_ptr(a.k, b, k0 + r, hk, &pk) + c * 16);
+                cp_async16(dv + swz(r, c), row_ptr(a.v, b, k0 + r, hk, &pv) + c * 16);
+            } else {                     // past the end of the index: zeros (their scores are masked, 0 * V must not be NaN)
+                const uint32_t off = swz(r, c);
+                *reinterpret_cast<uint4*>(sK + buf * KT * ROW_BYTES + off) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(sV + buf * KT * ROW_BYTES + off) = make_uint4(0u, 0u, 0u, 0u);
+            }
         }
         cp_async_commit();
     };
@@ -139,6 +166,12 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
     const float sl2 = a.scale * 1.4426950408889634f;  // scores are kept in the base-2 exponent domain
     const int row0 = q0 + warp * 16 + g;              // sequence position of this thread's first row (second: +8)
+    int rs0[2] = {0, 0}, rs1[2] = {0, 0};             // RAGGED: keys [rs0, rs1) are the sequence of each of the two rows; empty past the end
+    if (RAGGED) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+            if (row0 + 8 * r < a.S) seq_bounds(a, row0 + 8 * r, rs0[r], rs1[r]);
+    }
 
     for (int step = 0; step < n_steps; ++step) {
         const int buf = step & 1;
@@ -173,7 +206,11 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float v = s[n][e] * sl2;
-                if (diag) {
+                if (RAGGED) {
+                    const int key = k0 + n * 8 + 2 * t4 + (e & 1);
+                    const int row = row0 + 8 * (e >> 1);
+                    if (key < rs0[e >> 1] || key >= rs1[e >> 1] || (a.causal && key > row)) v = -INFINITY;
+                } else if (diag) {
                     const int key = k0 + n * 8 + 2 * t4 + (e & 1);
                     const int row = row0 + 8 * (e >> 1);
                     if (key > row) v = -INFINITY;
@@ -238,6 +275,7 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     if (a.lse.base && t4 == 0) {   // second output: log of the softmax denominator (scores were kept in base 2)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
+            if (RAGGED && row0 + 8 * r >= a.S) continue;
             const int64_t x[3] = {b, row0 + 8 * r, h};
             *reinterpret_cast<float*>(a.lse.base + ja_elem_off(a.lse, x)) = (m_run[r] + log2f(l_run[r])) * 0.6931471805599453f;
         }
@@ -254,9 +292,13 @@ __global__ void __launch_bounds__(QT * 2, 1) attention_kernel(AttnArgs a) {
     __syncthreads();
     {
         int64_t pitch;
-        char* op = const_cast<char*>(row_ptr(a.o, b, q0, h, &pitch));
+        char* op = RAGGED ? nullptr : const_cast<char*>(row_ptr(a.o, b, q0, h, &pitch));
         for (int i = tid; i < QT * 16; i += NT) {
             int r = i / 16, c = i % 16;
+            if (RAGGED) {
+                if (q0 + r >= a.S) continue;
+                op = const_cast<char*>(row_ptr(a.o, b, q0 + r, h, &pitch)) - (int64_t)r * pitch;
+            }
             *reinterpret_cast<uint4*>(op + (int64_t)r * pitch + c * 16) = *reinterpret_cast<const uint4*>(sQ + swz(r, c));
         }
     }
@@ -270,22 +312,27 @@ ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st) {
         ja_status_t s = ja_launch_attention_tc(a, st, &launched);
         if (s != JA_OK || launched) return s;
     }
+    const bool ragged = a.align % 64 != 0;       // some split point, sequence end or the length itself is not a multiple of 64 rows
     const int QT = (a.align % 128 == 0) ? 128 : 64;
+    const int n_qt = (a.S + QT - 1) / QT;
     AttnArgs a2 = a;
-    a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (ja_sm_count() + a.S / QT - 1) / (a.S / QT)));
-    dim3 grid((unsigned)((int64_t)a.H * a.B * (a.S / QT)), 1, 1);
+    a2.sect = (a.causal || a.n_ends > 1) ? a.H * a.B : std::min<int>(a.H * a.B, std::max(1, (ja_sm_count() + n_qt - 1) / n_qt));
+    dim3 grid((unsigned)((int64_t)a.H * a.B * n_qt), 1, 1);
     const int smem = QT * ROW_BYTES + 4 * KT * ROW_BYTES;
-#define JA_ATTN_SYNC(Q, F)                                                                                          \
-    do {                                                                                                           \
-        JA_CUDA(cudaFuncSetAttribute(attention_kernel<Q, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); \
-        attention_kernel<Q, F><<<grid, 2 * Q, smem, st>>>(a2);                                                    \
+#define JA_ATTN_SYNC(Q, F, R)                                                                                          \
+    do {                                                                                                              \
+        JA_CUDA(cudaFuncSetAttribute(attention_kernel<Q, F, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); \
+        attention_kernel<Q, F, R><<<grid, 2 * Q, smem, st>>>(a2);                                                    \
     } while (0)
-    if (QT == 128) {
-        if (a.f16) JA_ATTN_SYNC(128, true);
-        else JA_ATTN_SYNC(128, false);
+    if (ragged) {
+        if (a.f16) JA_ATTN_SYNC(64, true, true);
+        else JA_ATTN_SYNC(64, false, true);
+    } else if (QT == 128) {
+        if (a.f16) JA_ATTN_SYNC(128, true, false);
+        else JA_ATTN_SYNC(128, false, false);
     } else {
-        if (a.f16) JA_ATTN_SYNC(64, true);
-        else JA_ATTN_SYNC(64, false);
+        if (a.f16) JA_ATTN_SYNC(64, true, false);
+        else JA_ATTN_SYNC(64, false, false);
     }
 #undef JA_ATTN_SYNC
     ja_count_launch();

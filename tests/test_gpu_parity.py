@@ -423,6 +423,45 @@ def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut
             assert np.array_equal(got[:, s0], np.repeat(si.to_f64(V)[:, s0], grp, axis=1))
 
 
+# Ragged attention: lengths, split points and sequence ends that are NOT multiples of 64 rows. Output key tiles then
+# straddle blocks and packed sequences and run past the end of the index; the same-sequence / causal selection is applied
+# per score and every row is located on its own.
+@pytest.mark.parametrize("dtype", [BF, F16])
+@pytest.mark.parametrize("B,S,Hq,Hkv,s_split,ends,causal", [
+    (2, 100, 2, 2, [0, 100], [], True),                         # one short sequence in one block: a tile of 64 rows and one of 36
+    (1, 200, 2, 2, [0, 37, 101, 200], [], False),               # odd split points, not causal
+    (1, 333, 4, 2, [0, 50, 64, 131, 200, 333], [50, 131, 333], True),   # packed sequences that end inside tiles (every end is a split point, as the spec requires), grouped heads
+    (2, 77, 2, 1, list(range(0, 77, 11)) + [77], [77], True),   # 11-row blocks
+    (1, 64, 1, 1, [0, 1, 64], [1, 64], True),                   # a sequence of one row
+])
+def test_attention_ragged(B, S, Hq, Hkv, s_split, ends, causal, dtype):
+    D, grp = 128, Hq // Hkv
+    Q = si.normal((B, S, Hq, D), 0.0, 1.0, dtype, 4, 41)
+    K, V = (si.normal((B, S, Hkv, D), 0.0, 1.0, dtype, 4, o) for o in (42, 43))
+    g_split, h_split = ES(Hkv, Hkv), [grp * x for x in ES(Hkv, Hkv)]
+    q_sp, k_sp = [ES(B, B), s_split, h_split, [0, D]], [ES(B, B), s_split, g_split, [0, D]]
+    rQ, rK, rV = upload(Q, q_sp), upload(K, k_sp), upload(V, k_sp)
+    rO = empty_like_tiling([B, S, Hq, D], q_sp, dtype, fill=float("nan"))
+    rL = empty_like_tiling([B, S, Hq], q_sp[:3], F32, fill=float("nan"))
+    parts = {"b": q_sp[0], "q": s_split, "h": h_split, "d": [0, D], "k": s_split, "g": g_split}
+    prm = (1.0 / np.sqrt(D), 1.0 if causal else 0.0) + tuple(float(e) for e in ends)
+    spec = ja.Spec("bqhd,bkgd,bkgd->bqhd" if grp > 1 else "bqhd,bkhd,bkhd->bqhd",
+                   parts if grp > 1 else {k: v for k, v in parts.items() if k != "g"}, "attention", prm, "online_softmax")
+    before = ja.ja_launch_count()
+    spec.execute([rQ, rK, rV], [rO, rL])
+    assert ja.ja_launch_count() == before + 1
+    got, lse = download(rO), download(rL)          # download() checks the guard zones around both payloads
+    check_status()
+    ref = operators.attention_gqa_packed(si.to_f64(Q), si.to_f64(K), si.to_f64(V), grp, ends or None, causal, ORC_DT[dtype])
+    assert relfro(got, ref) <= TOL[dtype]
+    assert np.isfinite(lse).all()
+    if causal:   # the first row of every sequence joins with its own key only: O = V exactly, lse = its one score
+        for s0 in [0] + list(ends[:-1]):
+            assert np.array_equal(got[:, s0], np.repeat(si.to_f64(V)[:, s0], grp, axis=1))
+            q64, k64 = si.to_f64(Q)[:, s0], np.repeat(si.to_f64(K)[:, s0], grp, axis=1)
+            assert np.abs(lse[:, s0] - (q64 * k64).sum(-1) / np.sqrt(D)).max() <= 2e-3
+
+
 # ---------------------------------------------------------------------------------------------------
 # fused chains on the tensor-core matmul: the accumulator goes through the next join-agg before its one store
 # ---------------------------------------------------------------------------------------------------
