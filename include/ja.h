@@ -171,6 +171,9 @@ ja_status_t ja_relation_get_keys(const ja_relation_t* rel, int32_t* coords, int6
  *                                                          mma.sync tiles for multiples of 64, a per-row form otherwise);
  *                                                          Q, K, V, O of one 16-bit dtype (bf16 or f16; the probabilities
  *                                                          enter the second product rounded to that dtype)
+ *   any other einsum       MUL | ADD | IDENT | SQUARE | SILU_MUL | EXP_SUB with SUM | MAX | NONE: up to four operands
+ *                          and four summed indices, any tilings and dtypes -- Definition 3.7 executed cell by cell (one
+ *                          thread per output cell walks its joined tuples in ascending order): complete, not fast
  * n_outputs is 1, except for ATTENTION where it may be 2: outputs[1] then receives lse[b, q, h] = log of the softmax
  * denominator of every query row (f32, tiled like the first three indices of outputs[0]) -- with it two results over
  * disjoint key ranges combine by the online-softmax aggregation: O = w1 O1 + w2 O2, w_i = exp(lse_i - lse).

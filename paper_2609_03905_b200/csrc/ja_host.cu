@@ -1137,6 +1137,11 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
         return ja_launch_attention(aa, stream);
     }
 
+    // ---- anything else whose operator is a scalar function of the joined cells: the definition, cell by cell --------
+    if (n_outputs == 1) {
+        bool launched = false;
+        if ((st = ja_launch_generic(spec, inputs, out, stream, &launched)) != JA_OK || launched) return st;
+    }
     return ja_fail(JA_ERR_UNSUPPORTED, "no kernel for einsum '%s' with fn %d / agg %d", spec->einsum.c_str(), (int)fn,
                    (int)agg);
 }

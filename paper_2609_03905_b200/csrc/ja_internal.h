@@ -111,6 +111,9 @@ JaConfig& ja_config();
 // ---- kernel launchers (one per .cu file) ------------------------------------------------------------
 // Plain-ALU tiled matmul join-agg over arbitrary tilings (f32 or bf16 operands, f32 accumulate). The key tables of the
 // three relations must be on the device (ja_relation_to_device).
+// the definition in its relational form, one thread per output cell: any spec whose operator is a scalar function of the
+// joined cells (*launched stays false otherwise)
+ja_status_t ja_launch_generic(const ja_spec* spec, const ja_relation* const* inputs, const ja_relation* out, cudaStream_t st, bool* launched);
 ja_status_t ja_launch_matmul_simt(const ja_relation* A, const ja_relation* B, const ja_relation* C, cudaStream_t st,
                                   bool partials = false);
 

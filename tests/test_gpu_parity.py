@@ -423,6 +423,39 @@ def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut
             assert np.array_equal(got[:, s0], np.repeat(si.to_f64(V)[:, s0], grp, axis=1))
 
 
+# ---------------------------------------------------------------------------------------------------
+# any other einsum: the definition executed cell by cell (no specialised kernel matches these signatures)
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("einsum,shapes,splits,fn,agg,dtype", [
+    ("bij,bjk->bik", [(3, 20, 17), (3, 17, 12)], {"b": [0, 1, 3], "i": [0, 7, 20], "j": [0, 5, 17], "k": [0, 12]}, "mul", "sum", F32),   # batched matmul
+    ("bij,bjk->bik", [(2, 16, 24), (2, 24, 8)], {"b": [0, 2], "i": ES(16, 2), "j": ES(24, 3), "k": ES(8, 1)}, "mul", "sum", BF),
+    ("ij,kj->ik", [(18, 30), (11, 30)], {"i": [0, 4, 18], "j": [0, 9, 30], "k": [0, 11]}, "mul", "sum", F16),                          # second operand transposed
+    ("ij,j->i", [(25, 40), (40,)], {"i": [0, 10, 25], "j": ES(40, 4)}, "mul", "sum", F32),                                             # matrix x vector
+    ("i,j->ij", [(9,), (14,)], {"i": [0, 2, 9], "j": [0, 14]}, "mul", "none", F32),                                                    # outer product: nothing aggregated
+    ("ij,jk,kl->il", [(6, 7), (7, 5), (5, 8)], {"i": [0, 6], "j": [0, 3, 7], "k": [0, 5], "l": [0, 1, 8]}, "mul", "sum", F32),         # three operands, two summed indices
+    ("ijk->ik", [(5, 33, 6)], {"i": [0, 5], "j": [0, 20, 33], "k": ES(6, 2)}, "ident", "max", BF),                                     # MAX over a middle index
+    ("ijk->i", [(7, 9, 10)], {"i": [0, 3, 7], "j": ES(9, 3), "k": [0, 10]}, "square", "sum", F32),                                     # two summed indices, one operand
+    ("ij,ji->ij", [(12, 15), (15, 12)], {"i": ES(12, 3), "j": [0, 4, 15]}, "add", "none", F32),                                        # x + y^T: a join that is not key-aligned in storage
+])
+def test_general_einsum_runs_as_the_definition(einsum, shapes, splits, fn, agg, dtype):
+    ins, out_letters = einsum.split("->")
+    terms = ins.split(",")
+    xs = [si.normal(sh, 0.0, 1.0, dtype, 1, 50 + k) for k, sh in enumerate(shapes)]
+    rels = [upload(x, [splits[c] for c in t]) for x, t in zip(xs, terms)]
+    ext = {c: splits[c][-1] for c in splits}
+    rO = empty_like_tiling([ext[c] for c in out_letters], [splits[c] for c in out_letters], dtype, fill=float("nan"))
+    before = ja.ja_launch_count()
+    ja.Spec(einsum, splits, fn, (), agg).execute(rels, rO)
+    assert ja.ja_launch_count() == before + 1
+    got = download(rO)
+    check_status()
+    ref = core.join_agg(einsum, [si.to_f64(x) for x in xs], fn, agg)        # the scalar-keyed join + aggregation of the oracle
+    if agg == "max":
+        assert np.array_equal(got, ref)                                     # no arithmetic: exact in any dtype
+    else:
+        assert relfro(got, core.round_to(ref, ORC_DT[dtype])) <= TOL[dtype]
+
+
 # Ragged attention: lengths, split points and sequence ends that are NOT multiples of 64 rows. Output key tiles then
 # straddle blocks and packed sequences and run past the end of the index; the same-sequence / causal selection is applied
 # per score and every row is located on its own.
