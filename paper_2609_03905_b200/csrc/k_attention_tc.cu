@@ -531,6 +531,9 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   V -- tcgen05.mma kind::f16 with different formats for A and B is an illegal instruction.
 //   The output written from the row threads' registers straight to global memory (no staging in the P tile, no wait for
 //   its TMA stores at the next item's first key step): 0.1495 ms against 0.1399.
+//   With f16 relations, exponentials in half precision (ex2.approx.f16x2: two per instruction, the result already the
+//   packed operand, the row sum from f16 partial sums): 0.1558 ms against 0.1405 -- half the special-function work
+//   buys nothing, the conversions and the sum cost more.
 //   Built, verified against the oracle and dropped for the same reason as the shared-memory analysis below suggested it:
 //   FOUR tiles on a pair of CTAs, both products as tcgen05.mma.cta_group::2 with M = 256 and the K / V tile split between
 //   the two SMs (each SM then reads and is filled with half of every K / V tile: a quarter less traffic on the
