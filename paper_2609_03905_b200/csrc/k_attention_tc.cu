@@ -534,6 +534,12 @@ __device__ __forceinline__ float row_exp_pack128(const uint32_t (&v)[128], float
 //   With f16 relations, exponentials in half precision (ex2.approx.f16x2: two per instruction, the result already the
 //   packed operand, the row sum from f16 partial sums): 0.1558 ms against 0.1405 -- half the special-function work
 //   buys nothing, the conversions and the sum cost more.
+//   TWO threads per query row (sixteen row warps, 64 keys each, the halves of a row agreeing on its maximum through shared
+//   memory at every key step; registers moved to the row warps with setmaxnreg): 0.1618 ms against 0.1399, 2.12 against
+//   1.79 ms on one sequence of 16384 rows. Halving the row threads' instruction chains does not shorten a key step:
+//   what a step waits for are the hand-offs themselves (commit -> barrier -> wake, the tensor-memory loads, P ready ->
+//   issue), and with S and O~ of two tiles the 512 columns of tensor memory are full -- a third tile to overlap them
+//   with does not fit at d = 128.
 //   Built, verified against the oracle and dropped for the same reason as the shared-memory analysis below suggested it:
 //   FOUR tiles on a pair of CTAs, both products as tcgen05.mma.cta_group::2 with M = 256 and the K / V tile split between
 //   the two SMs (each SM then reads and is filled with half of every K / V tile: a quarter less traffic on the
