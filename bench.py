@@ -768,6 +768,52 @@ def case_results(case, reps):
                                          "optimizer_host_ms": opt_ms, "launches": len(blk.steps), "plan": plan}
             del blk
             torch.cuda.empty_cache()
+        # the two other selectors of the paper's plan-selection experiment (Section 6, Experiment 3) at p = 8: greedy (the
+        # same program without the repartition sub-cost) and twenty uniform draws among the valid specs of every operator
+        cost, plan = ja.ja_plan_select_greedy(ops, 8)
+        blk = PlannedBlock(Bt, S, hidden, heads, ffn, weights, plan)
+        t = timeit(lambda r: blk.forward(), reps, True)
+        res["greedy_p8"] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "proxy_cost_cells": cost,
+                            "repartition_charges": plan_repartition_charges(ops, plan)[0], "relayouts_executed": blk.n_relayouts,
+                            "launches": len(blk.steps), "plan": plan}
+        del blk
+        torch.cuda.empty_cache()
+        import random
+
+        def valid_specs(op, p_):   # specs(Op): interval counts with product p over the shardable letters
+            letters = []
+            for term in op["einsum"].replace("->", ",").split(","):
+                letters += [c for c in term if c not in letters]
+            out = []
+
+            def rec(i, rest, acc):
+                if i == len(letters):
+                    if rest == 1:
+                        out.append(dict(zip(letters, acc)))
+                    return
+                if letters[i] in op.get("fixed", ()):
+                    rec(i + 1, rest, acc + [1])
+                    return
+                for c_ in range(1, rest + 1):
+                    if rest % c_ == 0 and c_ <= op["extents"][letters[i]]:
+                        rec(i + 1, rest // c_, acc + [c_])
+            rec(0, p_, [])
+            return out
+
+        rng = random.Random(3905)
+        cand = [valid_specs(op, 8) for op in ops]
+        draws = []
+        for _ in range(20):
+            plan = [rng.choice(c_) for c_ in cand]
+            blk = PlannedBlock(Bt, S, hidden, heads, ffn, weights, plan)
+            t = timeit(lambda r: blk.forward(), max(3, reps // 4), True)
+            draws.append({"ms_mean": t["ms_mean"], "proxy_cost_cells": ja.ja_plan_cost(ops, plan), "relayouts_executed": blk.n_relayouts})
+            del blk
+            torch.cuda.empty_cache()
+        ms = sorted(d["ms_mean"] for d in draws)
+        res["random_p8_20_draws"] = {"ms_mean": sum(ms) / len(ms), "ms_best": ms[0], "ms_median": (ms[9] + ms[10]) / 2, "ms_worst": ms[-1],
+                                     "proxy_cost_cells_median": sorted(d["proxy_cost_cells"] for d in draws)[10],
+                                     "relayouts_executed_median": sorted(d["relayouts_executed"] for d in draws)[10]}
     elif args.case == "chains":
         # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
         # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)

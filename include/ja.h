@@ -247,6 +247,11 @@ ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int
  * the repartition charges of its already-planned consumers added. total_cost is the summed Cost of the assembled plan
  * (what ja_plan_cost returns for it). On a tree the result equals ja_plan_optimize. */
 ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
+/* The greedy selector the paper compares its optimizer with (Section 6, Experiment 3): the same program without the
+ * repartition sub-cost, so every operator independently takes the spec of least join + aggregation cost (the first one in
+ * the enumeration order of its specs). Trees and graphs alike. *total_cost is the full Cost of the plan it returns,
+ * repartition charges included: never below what ja_plan_optimize finds on a tree. */
+ja_status_t ja_plan_select_greedy(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost);
 
 /* ---- relayout without allocation -------------------------------------------------------------------
  * (The paper has no counterpart to this call: it exists for callers of THIS library that cannot allocate.)

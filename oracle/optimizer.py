@@ -115,6 +115,17 @@ def optimize_tree(ops, p: int):
     return opt[(root, T_star)], chosen
 
 
+def greedy(ops, p: int):
+    """The greedy selector of Section 6, Experiment 3: the dynamic program with the repartition sub-cost removed.  Nothing
+    then couples an operator to its producers, so each takes the spec of least join + aggregation cost on its own (the
+    first such spec in the order of `specs`).  Returns (full cost of that plan, repartition charges included, plan)."""
+    plan = []
+    for op in ops:
+        free = [None] * len(op["inputs"])
+        plan.append(min(specs(op, p), key=lambda J: cost(op, J, free)))      # min() keeps the first of equal keys
+    return plan_cost(ops, plan), plan
+
+
 def plan_cost(ops, plan) -> int:
     """Cost of a complete assignment: every operator pays Cost with its producers' output tilings."""
     total = 0

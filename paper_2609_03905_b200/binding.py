@@ -42,9 +42,10 @@ class ja_index_part_t(ctypes.Structure):
 
 
 def _load() -> ctypes.CDLL:
-    if not os.path.exists(_LIB_PATH):
-        from .build import build
-        build()
+    # make-like: compiles what is missing or older than its sources, nothing when libja.so is up to date (a library left over
+    # from older sources would otherwise be loaded and lack the newer entry points)
+    from .build import build
+    build()
     lib = ctypes.CDLL(_LIB_PATH)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     P = ctypes.POINTER
@@ -67,6 +68,7 @@ def _load() -> ctypes.CDLL:
         "ja_plan_optimize": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_plan_cost": [P(ja_plan_node_t), i32, P(i32), P(i64)],
         "ja_plan_optimize_graph": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
+        "ja_plan_select_greedy": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_repartition_agg": [vp, ctypes.c_int, vp, vp],
         "ja_overlay_atoms": [vp, vp, P(i64), vp, vp, vp, vp],
         "ja_stream_status": [vp, P(ctypes.c_int)],
@@ -258,6 +260,16 @@ def ja_plan_optimize_graph(ops, p: int):
     counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
     total = ctypes.c_int64()
     _check(LIB.ja_plan_optimize_graph(arr, len(ops), p, counts, ctypes.byref(total)))
+    plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
+    return total.value, plan
+
+
+def ja_plan_select_greedy(ops, p: int):
+    """Experiment 3's greedy selector: every operator takes its cheapest spec with the repartition sub-cost ignored."""
+    arr, keep = _plan_nodes(ops)
+    counts = (ctypes.c_int32 * (len(ops) * JA_PLAN_MAX_LETTERS))()
+    total = ctypes.c_int64()
+    _check(LIB.ja_plan_select_greedy(arr, len(ops), p, counts, ctypes.byref(total)))
     plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
     return total.value, plan
 

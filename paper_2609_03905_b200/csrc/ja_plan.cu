@@ -310,6 +310,34 @@ extern "C" ja_status_t ja_plan_optimize_graph(const ja_plan_node_t* nodes, int32
     return JA_OK;
 }
 
+// The greedy selector of the paper's plan-selection experiment (Section 6, Experiment 3): the same program with the
+// repartition sub-cost removed. That sub-cost is the only one that depends on the producers' tilings, so the recurrence falls
+// apart and every operator takes, on its own, the spec with the least join + aggregation cost (the first such spec in the
+// enumeration order of specs(Op)). The cost reported is the plan's full Cost, repartition charges included.
+extern "C" ja_status_t ja_plan_select_greedy(const ja_plan_node_t* nodes, int32_t n_nodes, int32_t p, int32_t* counts, int64_t* total_cost) {
+    if (p < 1 || !counts) return ja_fail(JA_ERR_INVALID_ARG, "p must be positive and counts non-NULL");
+    std::vector<Op> ops;
+    std::vector<int> consumers;
+    ja_status_t st = parse_all(nodes, n_nodes, true, &ops, &consumers);
+    if (st != JA_OK) return st;
+    std::vector<Counts> plan(n_nodes);
+    for (int32_t i = 0; i < n_nodes; ++i) {
+        std::vector<Counts> cand;
+        Counts cur;
+        enum_specs(ops[i], p, 0, &cur, &cand);
+        if (cand.empty()) return ja_fail(JA_ERR_TILING, "node %d has no spec with %d function specs", i, p);
+        const std::vector<const Counts*> no_producers(ops[i].ins.size(), nullptr);
+        int64_t best = -1;
+        for (const Counts& J : cand) {
+            const int64_t c = cost(ops[i], J, no_producers);
+            if (best < 0 || c < best) { best = c; plan[i] = J; }
+        }
+    }
+    write_counts(plan, counts);
+    if (total_cost) *total_cost = assembled_cost(ops, plan);
+    return JA_OK;
+}
+
 extern "C" ja_status_t ja_plan_cost(const ja_plan_node_t* nodes, int32_t n_nodes, const int32_t* counts, int64_t* total_cost) {
     if (!counts || !total_cost) return ja_fail(JA_ERR_INVALID_ARG, "counts / total_cost is NULL");
     std::vector<Op> ops;

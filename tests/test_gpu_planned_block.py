@@ -96,3 +96,21 @@ def test_optimizer_plan_on_the_7b_block_sampled_rows(p):
     hand = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan="seq")
     ja.repartition(ja.from_dense(x.cuda(), [hand.t_sp, hand.io_c]), hand.x)
     assert relfro(out, download(hand.forward())) <= TOL[BF]
+
+
+def test_greedy_plan_on_small_block():
+    """The greedy selector's plan (Section 6, Experiment 3: no repartition sub-cost in the selection) executes like any
+    other: one relayout per repartition charge, every intermediate against the oracle; its cost is not below the optimizer's."""
+    Bt, S, hidden, heads, ffn = 2, 512, 512, 4, 1408
+    ops = block_graph(Bt, S, hidden, heads, ffn)
+    cost, plan = ja.ja_plan_select_greedy(ops, 8)
+    assert cost == optimizer.plan_cost(ops, plan) and plan == optimizer.greedy(ops, 8)[1]
+    assert cost >= ja.ja_plan_optimize_graph(ops, 8)[0]
+    w = si.llama_weights(hidden, ffn, config=5, first_ordinal=21)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 20)
+    blk = PlannedBlock(Bt, S, hidden, heads, ffn, w, plan)
+    assert blk.n_relayouts == plan_repartition_charges(ops, plan)[0]
+    blk.load_input(x.cuda())
+    blk.forward()
+    check_status()
+    _check_all(blk, _oracle_block(x, w, Bt, S, heads), Bt, S, hidden, heads)

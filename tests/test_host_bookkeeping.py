@@ -298,3 +298,31 @@ def test_logical_optimizer_on_graphs_with_shared_tensors():
         assert got == want == optimizer.plan_cost(ops, plan) == ja.ja_plan_cost(ops, plan)
     tree = _mlp_tree(100, 36, 50)
     assert ja.ja_plan_optimize_graph(tree, 12)[0] == ja.ja_plan_optimize(tree, 12)[0]
+
+
+def test_greedy_selector_against_the_oracle_and_the_optimizer():
+    """The greedy selector of the plan-selection experiment (Section 6, Experiment 3): per operator the spec of least join +
+    aggregation cost, the repartition sub-cost ignored. The library's choice equals the oracle's, its cost is the full
+    cost of that plan, and on trees it is never below the optimizer's (equal where no relayout can be saved)."""
+    from oracle import optimizer
+    from test_oracle_pins import _block_graph
+    worse = 0
+    for tree, p in ((_mlp_tree(64, 32, 48), 4), (_mlp_tree(100, 36, 50), 12), (_mlp_tree(16, 16, 16), 8)):
+        want_cost, want_plan = optimizer.greedy(tree, p)
+        got_cost, got_plan = ja.ja_plan_select_greedy(tree, p)
+        assert got_plan == want_plan and got_cost == want_cost == optimizer.plan_cost(tree, got_plan) == ja.ja_plan_cost(tree, got_plan)
+        best = ja.ja_plan_optimize(tree, p)[0]
+        assert got_cost >= best
+        worse += got_cost > best
+    assert worse > 0       # the cases are not all degenerate: somewhere ignoring the relayouts costs something
+    for dims, p in (((16, 8, 12), 4), ((64, 32, 48), 8)):       # graphs with multiply consumed tensors
+        ops = _block_graph(*dims)
+        want_cost, want_plan = optimizer.greedy(ops, p)
+        got_cost, got_plan = ja.ja_plan_select_greedy(ops, p)
+        assert got_plan == want_plan and got_cost == want_cost == ja.ja_plan_cost(ops, got_plan)
+    # every operator's choice really is its own minimum: brute force over its specs with no producer tilings
+    ops = _block_graph(16, 8, 12)
+    _, plan = ja.ja_plan_select_greedy(ops, 4)
+    for op, J in zip(ops, plan):
+        free = [None] * len(op["inputs"])
+        assert optimizer.cost(op, J, free) == min(optimizer.cost(op, K, free) for K in optimizer.specs(op, 4))
