@@ -235,13 +235,14 @@ def test_small_grouped_query_block_every_intermediate():
         assert relfro(out, cat("out")) <= TOL[BF], (plan, fused)
 
 
-def test_paper_block_shape_grouped_query_sampled():
+@pytest.mark.parametrize("dtype", [BF, torch.float16])      # bf16 as the benchmark configurations state; f16 is the paper's precision
+def test_paper_block_shape_grouped_query_sampled(dtype):
     """Hidden 4096, 32 query heads on 8 key/value heads of 128, FFN 14336 (Section 6), eight sequences of 1K tokens;
     sampled token rows of one sequence against the oracle."""
     Bt, S, hidden, heads, kvh, ffn = 8, 1024, 4096, 32, 8, 14336
-    w = si.llama_weights(hidden, ffn, config=5, first_ordinal=61, kv_hidden=kvh * 128)
-    x = si.normal((Bt * S, hidden), 0.0, 1.0, BF, 5, 60)
-    blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan="seq", n_kv_heads=kvh)
+    w = si.llama_weights(hidden, ffn, config=5, dtype=dtype, first_ordinal=61, kv_hidden=kvh * 128)
+    x = si.normal((Bt * S, hidden), 0.0, 1.0, dtype, 5, 60)
+    blk = LlamaBlock(Bt, S, hidden, heads, ffn, w, plan="seq", n_kv_heads=kvh, dtype=dtype)
     ja.repartition(ja.from_dense(x.cuda(), [blk.t_sp, blk.io_c]), blk.x)
     out = download(blk.forward())
     check_status()
@@ -249,8 +250,9 @@ def test_paper_block_shape_grouped_query_sampled():
     seq_id, prefix = 5, 512
     rows = np.unique(np.concatenate([[0, 1, 127, 128, prefix - 1], np.linspace(0, prefix - 1, 6).astype(int)]))
     xs = si.to_f64(x[seq_id * S: seq_id * S + prefix])
-    ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows, n_kv_heads=kvh)["out"]
-    assert relfro(out[seq_id * S + rows], ref) <= TOL[BF]
+    ref = operators.llama_block(xs, {k: si.to_f64(v) for k, v in w.items()}, heads, 1e4, 1e-5, rows=rows, n_kv_heads=kvh,
+                                dtype="bf16" if dtype == BF else "f16")["out"]
+    assert relfro(out[seq_id * S + rows], ref) <= TOL[dtype]
 
 
 def test_join_only_and_aggregating_relayout_full_size():
