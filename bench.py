@@ -495,6 +495,17 @@ def case_results(case, reps):
         ts.sort()
         return {"ms_mean": sum(ts) / len(ts), "ms_min": ts[0], "ms_median": ts[len(ts) // 2]}
 
+    def timeit_graph(fn, reps, flush_l2):
+        """As timeit, for launches shorter than the host's own marshalling of the call (~15 us per relation through
+        Python): the call is recorded into a CUDA graph once and each timed region is one replay."""
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn(0)
+        return timeit(lambda r: g.replay(), reps, flush_l2)
+
     def rel(shape, splits, dtype=bf, std=1.0):
         r = ja.Relation(list(shape), splits, dtype)
         r.payload.normal_(0.0, std)
@@ -647,6 +658,28 @@ def case_results(case, reps):
             es = 4 if pdt == f32 else 2
             res["aggregating_relayout_" + tag] = hb((m * es + 2.0) * T * d, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
             del h, W2, P, y, spec
+        # the same for attention: the key index of B4 x 8192 keys cut into m ranges of 2048, one ja_execute (O_c, lse_c) per
+        # range against the 2048 queries, then the online-softmax aggregation as its own step (ja_attention_combine)
+        Bn, S, H, D = 4, 2048, 32, 128
+        sp = [ES(Bn, Bn), ES(S, S // 128), ES(H, H), [0, D]]
+        parts = {"b": sp[0], "q": sp[1], "h": sp[2], "d": sp[3], "k": sp[1]}
+        aspec = ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / D ** 0.5, 0.0), "online_softmax")
+        Q = rel((Bn, S, H, D), sp)
+        for m in (2, 4):
+            KV = [(rel((Bn, S, H, D), sp), rel((Bn, S, H, D), sp)) for _ in range(m)]
+            Oc = [ja.Relation([Bn, S, H, D], sp, bf) for _ in range(m)]
+            Lc = [ja.Relation([Bn, S, H], sp[:3], f32) for _ in range(m)]
+            O, L = ja.Relation([Bn, S, H, D], sp, bf), ja.Relation([Bn, S, H], sp[:3], f32)
+
+            def partials(r):
+                for c in range(m):
+                    aspec.execute([Q, KV[c][0], KV[c][1]], [Oc[c], Lc[c]])
+            t = timeit(partials, reps, True)
+            fl = 4.0 * Bn * H * S * (m * S) * D
+            res["attention_partials_m%d" % m] = {**t, "TFLOPs": fl / (t["ms_mean"] * 1e-3) / 1e12, "frac_of_burst_bf16_peak": fl / (t["ms_mean"] * 1e-3) / 1e12 / peaks["bf16"]}
+            nbytes = (m + 1.0) * Bn * S * H * (D * 2 + 4)
+            res["attention_combine_m%d" % m] = hb(nbytes, timeit_graph(lambda r: ja.attention_combine(Oc, Lc, O, L), reps, True))
+            del KV, Oc, Lc, O, L
     elif args.case == "opt":
         # logical optimization (Algorithm 1) of the SwiGLU MLP tree of config 2, then the chosen plan and three hand
         # plans executed as join-aggs (a relayout wherever a producer's tiling differs from what its consumer's spec needs)

@@ -214,6 +214,21 @@ ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_t* const* i
                             ja_relation_t* partials, void* cuda_stream);
 ja_status_t ja_repartition_agg(const ja_relation_t* partials, ja_agg_t agg, ja_relation_t* dst, void* cuda_stream);
 
+/* ---- the online-softmax aggregation as a step of its own (Definition 3.7 step 2 for ATTENTION; Section 5.1) ------
+ * When the function specs of an attention output key are executed apart -- m calls of ja_execute with n_outputs = 2,
+ * each over its own range of the key index -- every call leaves a partial result O_c (already divided by its own
+ * denominator) and lse_c. Their (+)-combination is  lse = log sum_c exp(lse_c),  O = sum_c exp(lse_c - lse) O_c,
+ * the (O~, m, l) aggregation of JA_AGG_ONLINE_SOFTMAX written for normalised partials; copies are combined in
+ * ascending order in f32 and O is rounded once. A partial whose lse is -inf for a row (no key of its range joined with
+ * it) contributes nothing to that row; a row with no key at all gets O = 0 and lse = -inf.
+ *   o_parts, lse_parts  host arrays of m (1..8) relations: O_c [b, s, h, 128] and lse_c [b, s, h] (f32); borrowed, unchanged
+ *   o, lse              outputs: o of the dtype of the partials; lse f32 or NULL. Every relation may have its own tiling
+ *                       (the last index unsplit).
+ * Asynchronous on `cuda_stream`. Errors: JA_ERR_INVALID_ARG (NULL, aliasing), JA_ERR_SHAPE, JA_ERR_DTYPE,
+ * JA_ERR_UNSUPPORTED (m outside 1..8). */
+ja_status_t ja_attention_combine(const ja_relation_t* const* o_parts, const ja_relation_t* const* lse_parts, int32_t m,
+                                 ja_relation_t* o, ja_relation_t* lse, void* cuda_stream);
+
 /* ---- logical optimization (Section 4.2, Algorithm 1; cost proxy of Section 4.3) -------------------------------
  * Chooses one join-agg spec per abstract operator of a computation TREE (every node but the last is consumed by
  * exactly one later node; the last node produces the result) for p processors = p function specs per operator.

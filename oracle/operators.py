@@ -88,7 +88,10 @@ def attention_lse(Q, K, causal=True, scale=None, qpos=None):
         pos = np.arange(Q.shape[1]) if qpos is None else np.asarray(qpos)
         s = np.where(np.arange(K.shape[1])[None, None, None, :] <= pos[None, :, None, None], s, -np.inf)
     m = s.max(axis=-1)
-    return rnd(m + np.log(np.exp(s - m[..., None]).sum(axis=-1)), "f32")
+    some = np.isfinite(m)                         # a row that joins with no key: the sum is empty, its log is -inf
+    ms = np.where(some, m, 0.0)
+    with np.errstate(divide="ignore"):
+        return rnd(np.where(some, ms + np.log(np.exp(s - ms[..., None]).sum(axis=-1)), -np.inf), "f32")
 
 
 def attention_gqa_packed(Q, K, V, group=1, ends=None, causal=True, out_dtype="bf16", scale=None):
@@ -127,6 +130,22 @@ def attention_as_join_aggs(Q, K, V, causal=True, scale=None):
         q_i, k_i = np.arange(S.shape[2])[:, None], np.arange(S.shape[3])[None, :]
         P = np.where(k_i <= q_i, P, 0.0)  # tuples removed by the selection contribute nothing to the SUM
     return core.join_agg("bhqk,bkhd->bqhd", [P, V], fn="mul", agg="sum")
+
+
+def attention_combine(o_parts, lse_parts, out_dtype="bf16"):
+    """The online-softmax aggregation of normalised partial attention results (O_c, lse_c) over disjoint key ranges:
+    lse = log sum_c exp(lse_c), O = sum_c exp(lse_c - lse) O_c -- the (O~, m, l) combine of softmax_triple_combine with
+    O_c = O~_c / l_c and lse_c = m_c + log l_c.  A partial with lse = -inf contributes nothing; a row without any key
+    gets O = 0, lse = -inf.  Returns (O rounded once to out_dtype, lse rounded to f32), fp64 inside."""
+    ls = np.stack([np.asarray(l, dtype=np.float64) for l in lse_parts])
+    os_ = np.stack([np.asarray(o, dtype=np.float64) for o in o_parts])
+    with np.errstate(divide="ignore", invalid="ignore"):
+        mx = ls.max(axis=0)
+        safe = np.where(np.isfinite(mx), mx, 0.0)
+        tot = np.where(np.isfinite(mx), safe + np.log(np.exp(ls - safe).sum(axis=0)), -np.inf)
+        w = np.where(np.isfinite(tot), np.exp(ls - np.where(np.isfinite(tot), tot, 0.0)), 0.0)
+    O = np.where(w[..., None] > 0, w[..., None] * np.nan_to_num(os_), 0.0).sum(axis=0)   # an empty partial's O is never looked at
+    return rnd(O, out_dtype), tot.astype(np.float32).astype(np.float64)
 
 
 def softmax_triple_combine(a, b):

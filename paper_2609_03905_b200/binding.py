@@ -67,6 +67,7 @@ def _load() -> ctypes.CDLL:
         "ja_execute_join": [vp, P(vp), i32, vp, vp],
         "ja_plan_optimize": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_plan_cost": [P(ja_plan_node_t), i32, P(i32), P(i64)],
+        "ja_attention_combine": [P(vp), P(vp), i32, vp, vp, vp],
         "ja_plan_optimize_graph": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_plan_select_greedy": [P(ja_plan_node_t), i32, i32, P(i32), P(i64)],
         "ja_repartition_agg": [vp, ctypes.c_int, vp, vp],
@@ -262,6 +263,15 @@ def ja_plan_optimize_graph(ops, p: int):
     _check(LIB.ja_plan_optimize_graph(arr, len(ops), p, counts, ctypes.byref(total)))
     plan = [{c: counts[i * JA_PLAN_MAX_LETTERS + l] for l, c in enumerate(op["_letters"])} for i, op in enumerate(ops)]
     return total.value, plan
+
+
+def ja_attention_combine(o_parts, lse_parts, o: int, lse: int | None = None, stream: int = 0):
+    """Handles of m partial attention results (O_c, lse_c) -> their online-softmax combination in `o` (and `lse`)."""
+    m = len(o_parts)
+    assert len(lse_parts) == m
+    oa = (ctypes.c_void_p * m)(*o_parts)
+    la = (ctypes.c_void_p * m)(*lse_parts)
+    _check(LIB.ja_attention_combine(oa, la, m, ctypes.c_void_p(o), ctypes.c_void_p(lse) if lse else None, ctypes.c_void_p(stream)))
 
 
 def ja_plan_select_greedy(ops, p: int):

@@ -1147,6 +1147,37 @@ extern "C" ja_status_t ja_execute(const ja_spec_t* spec, const ja_relation_t* co
 }
 
 // ---------------------------------------------------------------------------------------------------
+// ja_attention_combine: the online-softmax aggregation of partial attention results as a step of its own
+// ---------------------------------------------------------------------------------------------------
+extern "C" ja_status_t ja_attention_combine(const ja_relation_t* const* o_parts, const ja_relation_t* const* lse_parts, int32_t m,
+                                            ja_relation_t* o, ja_relation_t* lse, void* cuda_stream) {
+    if (!o_parts || !lse_parts || !o) return ja_fail(JA_ERR_INVALID_ARG, "o_parts / lse_parts / o is NULL");
+    if (m < 1 || m > 8) return ja_fail(JA_ERR_UNSUPPORTED, "between 1 and 8 partial results, %d given", m);
+    if (o->rank != 4 || o->extent[3] != 128 || o->nblk[3] != 1) return ja_fail(JA_ERR_SHAPE, "o is a [b, s, h, 128] relation with an unsplit last index");
+    if (o->dtype != JA_F32 && o->dtype != JA_BF16 && o->dtype != JA_F16) return ja_fail(JA_ERR_DTYPE, "unknown dtype");
+    auto stat_like = [&](const ja_relation* r) {
+        if (!r || r->rank != 3 || r->dtype != JA_F32) return false;
+        for (int d = 0; d < 3; ++d)
+            if (r->extent[d] != o->extent[d]) return false;
+        return true;
+    };
+    if (lse && !stat_like(lse)) return ja_fail(JA_ERR_SHAPE, "lse is an f32 relation over (b, s, h)");
+    ja_status_t st;
+    for (int c = 0; c < m; ++c) {
+        const ja_relation* p = o_parts[c];
+        if (!p || p->rank != 4 || p->dtype != o->dtype || p->nblk[3] != 1) return ja_fail(JA_ERR_SHAPE, "partial result %d: a relation like o (same dtype, unsplit last index)", c);
+        for (int d = 0; d < 4; ++d)
+            if (p->extent[d] != o->extent[d]) return ja_fail(JA_ERR_SHAPE, "partial result %d: extents differ from o", c);
+        if (!stat_like(lse_parts[c])) return ja_fail(JA_ERR_SHAPE, "lse of partial result %d: an f32 relation over (b, s, h)", c);
+        if (p->base == o->base || (lse && lse_parts[c]->base == lse->base)) return ja_fail(JA_ERR_INVALID_ARG, "an output aliases partial result %d", c);
+        if ((st = ja_relation_to_device(p)) != JA_OK || (st = ja_relation_to_device(lse_parts[c])) != JA_OK) return st;
+    }
+    if ((st = ja_relation_to_device(o)) != JA_OK) return st;
+    if (lse && (st = ja_relation_to_device(lse)) != JA_OK) return st;
+    return ja_launch_attention_combine(o_parts, lse_parts, m, o, lse, (cudaStream_t)cuda_stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // ja_execute_join: step (1) of Definition 3.7 alone (Section 5.1: a producer compiled through its join)
 // ---------------------------------------------------------------------------------------------------
 extern "C" ja_status_t ja_execute_join(const ja_spec_t* spec, const ja_relation_t* const* inputs, int32_t n_inputs,

@@ -205,4 +205,7 @@ struct AttnArgs {
 ja_status_t ja_launch_attention(const AttnArgs& a, cudaStream_t st);
 // tcgen05 / TMEM form; *launched stays false when the tiling does not fit it
 ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* launched);
+// the online-softmax aggregation of m partial attention results (O_c, lse_c) into (O, lse); l may be nullptr
+ja_status_t ja_launch_attention_combine(const ja_relation* const* op, const ja_relation* const* lp, int m, const ja_relation* o,
+                                        const ja_relation* l, cudaStream_t st);
 void ja_attention_reset_queues();   // zeroes the work counters of the persistent attention kernel (after a device-side failure)

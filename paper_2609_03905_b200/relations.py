@@ -87,6 +87,12 @@ def repartition_agg(partials: Relation, agg: str, dst: Relation, stream: int | N
     B.ja_repartition_agg(partials.handle, agg, dst.handle, current_stream() if stream is None else stream)
 
 
+def attention_combine(o_parts, lse_parts, o: Relation, lse: Relation | None = None, stream: int | None = None):
+    """Partial attention results over disjoint key ranges -> one result (the online-softmax aggregation as its own step)."""
+    B.ja_attention_combine([r.handle for r in o_parts], [r.handle for r in lse_parts], o.handle, lse.handle if lse is not None else None,
+                           current_stream() if stream is None else stream)
+
+
 def partial_relation(copies: int, extents, splits, dtype) -> Relation:
     """Empty partial relation [c, x...]: the copy index in front, cut into its unit intervals."""
     return Relation([copies] + list(extents), [list(range(copies + 1))] + [list(s) for s in splits], dtype)

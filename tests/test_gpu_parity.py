@@ -424,6 +424,67 @@ def test_attention_grouped_heads_packed_sequences(B, S, Hq, Hkv, gblk, ends, cut
 
 
 # ---------------------------------------------------------------------------------------------------
+# the online-softmax aggregation as a step of its own: partial attention results over disjoint key ranges, combined
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", [BF, F16, F32])
+@pytest.mark.parametrize("m,same_tiling", [(1, False), (3, False), (3, True)])
+def test_attention_combine_of_partial_results(m, same_tiling, dtype):
+    """Function specs of one output key executed apart: m attention calls (n_outputs = 2), each over its own 256 keys, then
+    ja_attention_combine -- against attention over all m * 256 keys at once (oracle), with the partial and the output
+    relations each in a tiling of its own. f32 partials come from the oracle (attention itself takes 16-bit relations)."""
+    B, S, H, D = 2, 256, 4, 128
+    adt = BF if dtype == F32 else dtype
+    Q = si.normal((B, S, H, D), 0.0, 1.0, adt, 4, 61)
+    K, V = (si.normal((B, m * S, H, D), 0.0, 1.0, adt, 4, o) for o in (62, 63))
+    tilings = [[ES(B, B), ES(S, 2), ES(H, H), [0, D]], [ES(B, 1), ES(S, 4), ES(H, 2), [0, D]], [ES(B, B), [0, 100, 256], [0, 1, 4], [0, D]]]
+    if same_tiling:      # one tiling for every relation: rows addressed by arithmetic instead of through the key tables
+        tilings = [tilings[0]] * 3
+    o_parts, l_parts, ref_o, ref_l = [], [], [], []
+    for c in range(m):
+        sp = tilings[c % 3]
+        Kc, Vc = K[:, c * S:(c + 1) * S].contiguous(), V[:, c * S:(c + 1) * S].contiguous()
+        ref_o.append(operators.attention(si.to_f64(Q), si.to_f64(Kc), si.to_f64(Vc), False, ORC_DT[dtype]))
+        ref_l.append(operators.attention_lse(si.to_f64(Q), si.to_f64(Kc), False))
+        if dtype == F32 or (c % 3 == 2 and not same_tiling):      # oracle partials (f32, or the irregular tiling attention is not run on here)
+            o_parts.append(upload(torch.from_numpy(ref_o[-1]).to(dtype), sp))
+            l_parts.append(upload(torch.from_numpy(ref_l[-1]).to(F32), sp[:3]))
+            continue
+        rQ, rK, rV = upload(Q, sp), upload(Kc, sp), upload(Vc, sp)
+        rO = empty_like_tiling([B, S, H, D], sp, dtype, fill=float("nan"))
+        rL = empty_like_tiling([B, S, H], sp[:3], F32, fill=float("nan"))
+        parts = {"b": sp[0], "q": sp[1], "h": sp[2], "d": sp[3], "k": sp[1]}
+        ja.Spec("bqhd,bkhd,bkhd->bqhd", parts, "attention", (1.0 / np.sqrt(D), 0.0), "online_softmax").execute([rQ, rK, rV], [rO, rL])
+        o_parts.append(rO)
+        l_parts.append(rL)
+    out_sp = tilings[0] if same_tiling else [ES(B, B), ES(S, 1), ES(H, 4), [0, D]]
+    rO = empty_like_tiling([B, S, H, D], out_sp, dtype, fill=float("nan"))
+    rL = empty_like_tiling([B, S, H], out_sp[:3], F32, fill=float("nan"))
+    before = ja.ja_launch_count()
+    ja.attention_combine(o_parts, l_parts, rO, rL)
+    assert ja.ja_launch_count() == before + 1
+    got, got_l = download(rO), download(rL)
+    check_status()
+    want = operators.attention(si.to_f64(Q), si.to_f64(K), si.to_f64(V), False, ORC_DT[dtype])           # all keys at once
+    want_l = operators.attention_lse(si.to_f64(Q), si.to_f64(K), False)
+    assert relfro(got, want) <= (2e-3 if dtype == F32 else TOL[dtype])        # f32: the partials were rounded to f32, the exponentials are fast ones
+    assert np.abs(got_l - want_l).max() <= 2e-3
+    # the combine itself, on exactly the partials the GPU saw, is the oracle's combine up to rounding
+    exact_o, exact_l = operators.attention_combine([download(r) for r in o_parts], [download(r) for r in l_parts], ORC_DT[dtype])
+    assert relfro(got, exact_o) <= (1e-5 if dtype == F32 else 3e-3 if dtype == BF else 4e-4)
+    assert np.abs(got_l - exact_l).max() <= 1e-5
+    # a partial that holds nothing for some rows (lse = -inf, O unspecified -- here NaN) drops out of those rows
+    if m == 3:
+        l_parts[1].payload.fill_(float("-inf"))
+        o_parts[1].payload.fill_(float("nan"))
+        ja.attention_combine(o_parts, l_parts, rO, None)
+        exact2, _ = operators.attention_combine([download(o_parts[0]), download(o_parts[2])], [download(l_parts[0]), download(l_parts[2])], ORC_DT[dtype])
+        assert relfro(download(rO), exact2) <= (1e-5 if dtype == F32 else 3e-3 if dtype == BF else 4e-4)
+        check_status()
+    with pytest.raises(ja.JaError):      # an output may not alias a partial
+        ja.attention_combine(o_parts, l_parts, o_parts[0], None)
+
+
+# ---------------------------------------------------------------------------------------------------
 # any other einsum: the definition executed cell by cell (no specialised kernel matches these signatures)
 # ---------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("einsum,shapes,splits,fn,agg,dtype", [

@@ -585,6 +585,41 @@ def test_attention_lse_combines_partial_results():
     np.testing.assert_allclose(operators.attention_lse(Q, K1, causal=False), np.einsum("bqhd,bhd->bqh", Q, K[:, 0]) / np.sqrt(D) + np.log(S), rtol=1e-6, atol=1e-6)
 
 
+def test_attention_combine_equals_attention_over_all_keys():
+    """operators.attention_combine against the plain definition: attention over three disjoint key ranges, combined,
+    equals attention over all keys -- also causal, where a whole key range lies after some query rows (their partial is
+    empty: lse = -inf, and must drop out), and the order of the partials does not matter."""
+    B, S, H, D = 2, 24, 3, 8
+    Q, K, V = (RNG.standard_normal((B, S, H, D)) for _ in range(3))
+    ranges = ((0, 7), (7, 16), (16, 24))
+    for causal in (False, True):
+        want = operators.attention(Q, K, V, causal=causal, out_dtype=None)
+        want_l = operators.attention_lse(Q, K, causal=causal)
+        o_parts, l_parts = [], []
+        for k0, k1 in ranges:
+            if causal:   # key i of the range sits at position k0 + i: query q sees it iff i <= q - k0; rows before k0 see none of it
+                o = np.zeros_like(Q)                             # what an empty partial holds is never looked at
+                o[:, k0:] = operators.attention(Q[:, k0:], K[:, k0:k1], V[:, k0:k1], causal=True, out_dtype=None,
+                                                qpos=np.minimum(np.arange(k0, S) - k0, k1 - k0 - 1))
+                o_parts.append(o)
+                l_parts.append(operators.attention_lse(Q, K[:, k0:k1], causal=True, qpos=np.arange(S) - k0))
+            else:
+                o_parts.append(operators.attention(Q, K[:, k0:k1], V[:, k0:k1], causal=False, out_dtype=None))
+                l_parts.append(operators.attention_lse(Q, K[:, k0:k1], causal=False))
+        if causal:
+            assert np.isneginf(l_parts[2][:, :16]).all() and np.isfinite(l_parts[2][:, 16:]).all()     # the case does hold empty partials
+        got, got_l = operators.attention_combine(o_parts, l_parts, out_dtype=None)
+        np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-6)
+        np.testing.assert_allclose(got_l, want_l, rtol=1e-6, atol=1e-6)
+        rev, rev_l = operators.attention_combine(o_parts[::-1], l_parts[::-1], out_dtype=None)
+        np.testing.assert_allclose(rev, got, rtol=1e-12, atol=1e-12)
+        # one partial alone is returned as it is; a row without any key gives O = 0 and lse = -inf
+        one, one_l = operators.attention_combine(o_parts[:1], l_parts[:1], out_dtype=None)
+        np.testing.assert_allclose(one, o_parts[0], rtol=1e-12, atol=0)
+    z, zl = operators.attention_combine([np.ones((1, 2, 1, 4))], [np.full((1, 2, 1), -np.inf)], out_dtype=None)
+    assert np.array_equal(z, np.zeros((1, 2, 1, 4))) and np.isneginf(zl).all()
+
+
 def _block_graph(T=16, d=8, f=12, S=4):
     """The operators of a transformer block as a DAG with multiply consumed tensors (x, n1, h): small extents."""
     E = lambda **k: k
