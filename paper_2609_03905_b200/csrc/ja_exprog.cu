@@ -1,0 +1,1376 @@
+// Exchange programs (Section 5): the ExProg language of Section 5.2, Definition "Closure; validity" and the rewriting
+// rules of Section 5.4, the cost model of the hardware simulator, preamble generation of Section 5.3. Host code only.
+//
+// An aggregate is a 64-bit mask over the atoms in declaration order, a state a set of (mask, site) pairs. A program is a
+// SET of actions; wherever an order is needed it is the order of the text.
+#include <ctype.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <charconv>
+#include <map>
+#include <set>
+#include <string>
+#include <tuple>
+#include <utility>
+#include <vector>
+
+#include "ja_exprog.h"
+#include "ja_internal.h"
+
+struct ExTarget {
+    int part = -1;                 // >= 0: a partition, else the list of sites
+    std::vector<int> sites;
+    bool operator==(const ExTarget& o) const { return part == o.part && sites == o.sites; }
+};
+struct ExAction {
+    uint64_t agg = 0;
+    ExTarget src;
+    std::vector<int> dests;
+    bool operator==(const ExAction& o) const { return agg == o.agg && src == o.src && dests == o.dests; }
+};
+struct ExPartition {
+    std::string name;
+    int size = 0;
+    bool bound = false;
+    std::vector<int> members;
+};
+struct ExAtom {
+    std::string name;
+    int site = 0;
+    double gb = 1.0;
+};
+struct ja_exprog {
+    std::vector<int> gpus;
+    std::vector<ExPartition> parts;
+    std::vector<ExAtom> atoms;
+    std::vector<std::pair<uint64_t, ExTarget>> out;
+    std::vector<ExAction> actions;
+};
+
+namespace {
+
+typedef ja_exprog Prog;
+struct Flat {              // an expanded action
+    uint64_t agg;
+    int site;
+    std::vector<int> dests;
+    bool operator==(const Flat& o) const { return agg == o.agg && site == o.site && dests == o.dests; }
+};
+typedef std::set<std::pair<int, uint64_t>> State;    // (site, aggregate)
+
+// ------------------------------------------------------------------------------------------------------ text
+std::string trim(const std::string& s) {
+    size_t a = s.find_first_not_of(" \t\r\n"), b = s.find_last_not_of(" \t\r\n");
+    return a == std::string::npos ? std::string() : s.substr(a, b - a + 1);
+}
+std::vector<std::string> split(const std::string& s, const char* seps) {
+    std::vector<std::string> res;
+    std::string cur;
+    for (char c : s) {
+        if (strchr(seps, c)) {
+            res.push_back(cur);
+            cur.clear();
+        } else {
+            cur.push_back(c);
+        }
+    }
+    res.push_back(cur);
+    return res;
+}
+bool is_word(const std::string& s) {
+    if (s.empty()) return false;
+    for (char c : s)
+        if (!(isalnum((unsigned char)c) || c == '_')) return false;
+    return true;
+}
+bool parse_int(const std::string& t, int* v) {
+    std::string s = trim(t);
+    if (s.empty() || s.size() > 9) return false;
+    for (char c : s)
+        if (!isdigit((unsigned char)c)) return false;
+    *v = atoi(s.c_str());
+    return true;
+}
+bool parse_sites(const std::string& text, std::vector<int>* sites) {
+    sites->clear();
+    for (const std::string& t : split(text, ",")) {
+        if (trim(t).empty()) continue;
+        int v;
+        if (!parse_int(t, &v)) return false;
+        sites->push_back(v);
+    }
+    return true;
+}
+std::vector<std::string> items(const std::string& text) {
+    std::vector<std::string> res;
+    for (const std::string& t : split(text, ";\n"))
+        if (!trim(t).empty()) res.push_back(trim(t));
+    return res;
+}
+int find_part(const Prog& p, const std::string& name) {
+    for (size_t i = 0; i < p.parts.size(); ++i)
+        if (p.parts[i].name == name) return (int)i;
+    return -1;
+}
+int find_atom(const Prog& p, const std::string& name) {
+    for (size_t i = 0; i < p.atoms.size(); ++i)
+        if (p.atoms[i].name == name) return (int)i;
+    return -1;
+}
+bool parse_target(const Prog& p, const std::string& text, ExTarget* t) {
+    std::string s = trim(text);
+    t->part = find_part(p, s);
+    t->sites.clear();
+    if (t->part >= 0) return true;
+    return parse_sites(s, &t->sites) && !t->sites.empty();
+}
+bool parse_aggregate(const Prog& p, const std::string& text, uint64_t* mask) {
+    *mask = 0;
+    for (const std::string& t : split(text, "+")) {
+        int a = find_atom(p, trim(t));
+        if (a < 0 || (*mask >> a) & 1) return false;
+        *mask |= 1ull << a;
+    }
+    return *mask != 0;
+}
+// position of keyword "KW:" (KW preceded by a non-word character, optional blanks before the colon); npos if absent
+size_t find_keyword(const std::string& s, const char* kw, size_t from, size_t* after) {
+    size_t n = strlen(kw);
+    for (size_t i = s.find(kw, from); i != std::string::npos; i = s.find(kw, i + 1)) {
+        if (i > 0 && (isalnum((unsigned char)s[i - 1]) || s[i - 1] == '_')) continue;
+        size_t j = i + n;
+        while (j < s.size() && (s[j] == ' ' || s[j] == '\t')) ++j;
+        if (j < s.size() && s[j] == ':') {
+            *after = j + 1;
+            return i;
+        }
+    }
+    return std::string::npos;
+}
+
+ja_status_t check_static(const Prog& p) {
+    std::set<int> g(p.gpus.begin(), p.gpus.end());
+    if (g.size() != p.gpus.size()) return ja_fail(JA_ERR_INVALID_ARG, "a site is listed twice in GPUS");
+    for (int s : p.gpus)
+        if (s < 0 || s > 63) return ja_fail(JA_ERR_INVALID_ARG, "site %d: sites are 0..63", s);
+    std::set<int> fixed;
+    int total = 0;
+    for (const ExPartition& q : p.parts) {
+        total += q.size;
+        if (!q.bound) continue;
+        for (int s : q.members) {
+            if (!g.count(s) || !fixed.insert(s).second)
+                return ja_fail(JA_ERR_INVALID_ARG, "partitions overlap or name an undeclared site (%s)", q.name.c_str());
+        }
+    }
+    if (!p.parts.empty() && total != (int)p.gpus.size())
+        return ja_fail(JA_ERR_INVALID_ARG, "the partitions must cover the declared GPUs");
+    for (const ExAtom& a : p.atoms)
+        if (!g.count(a.site)) return ja_fail(JA_ERR_INVALID_ARG, "atom %s at an undeclared site", a.name.c_str());
+    auto sized = [&](uint64_t m) {
+        double gb = -1.0;
+        for (size_t i = 0; i < p.atoms.size(); ++i)
+            if ((m >> i) & 1) {
+                if (gb >= 0 && p.atoms[i].gb != gb) return false;
+                gb = p.atoms[i].gb;
+            }
+        return true;
+    };
+    for (const auto& o : p.out)
+        if (!sized(o.first)) return ja_fail(JA_ERR_INVALID_ARG, "the atoms of one aggregate differ in size");
+    for (const ExAction& a : p.actions)
+        if (!sized(a.agg)) return ja_fail(JA_ERR_INVALID_ARG, "the atoms of one aggregate differ in size");
+    return JA_OK;
+}
+
+ja_status_t parse_program(const std::string& text, Prog* p) {
+    size_t out_after = 0, out_at = find_keyword(text, "OUT", 0, &out_after);
+    if (out_at == std::string::npos) return ja_fail(JA_ERR_PARSE, "no OUT declaration");
+    // the body starts after the first blank line that follows OUT
+    size_t pre_end = text.size(), body_at = text.size();
+    for (size_t i = text.find('\n', out_after); i != std::string::npos; i = text.find('\n', i + 1)) {
+        size_t j = i + 1;
+        while (j < text.size() && (text[j] == ' ' || text[j] == '\t')) ++j;
+        if (j < text.size() && text[j] == '\n') {
+            pre_end = i;
+            body_at = j + 1;
+            break;
+        }
+    }
+    const std::string pre = text.substr(0, pre_end), body = text.substr(body_at);
+    struct Mark {
+        size_t at, after;
+        int kw;
+    };
+    static const char* const KW[4] = {"GPUS", "PARTITIONS", "IN", "OUT"};
+    std::vector<Mark> marks;
+    for (int k = 0; k < 4; ++k) {
+        size_t after = 0, from = 0, at;
+        while ((at = find_keyword(pre, KW[k], from, &after)) != std::string::npos) {
+            marks.push_back({at, after, k});
+            from = at + 1;
+        }
+    }
+    std::sort(marks.begin(), marks.end(), [](const Mark& a, const Mark& b) { return a.at < b.at; });
+    std::string sect[4];
+    bool has[4] = {false, false, false, false};
+    for (size_t i = 0; i < marks.size(); ++i) {
+        size_t end = i + 1 < marks.size() ? marks[i + 1].at : pre.size();
+        sect[marks[i].kw] = pre.substr(marks[i].after, end - marks[i].after);
+        has[marks[i].kw] = true;
+    }
+    if (!has[2]) return ja_fail(JA_ERR_PARSE, "no IN declaration");
+    // PARTITIONS: name { size n } | name { s, s, .. }
+    {
+        const std::string& s = sect[1];
+        size_t i = 0;
+        while ((i = s.find('{', i)) != std::string::npos) {
+            size_t close = s.find('}', i);
+            if (close == std::string::npos) return ja_fail(JA_ERR_PARSE, "PARTITIONS: missing '}'");
+            size_t b = i;
+            while (b > 0 && (s[b - 1] == ' ' || s[b - 1] == '\t')) --b;
+            size_t a = b;
+            while (a > 0 && (isalnum((unsigned char)s[a - 1]) || s[a - 1] == '_')) --a;
+            ExPartition q;
+            q.name = s.substr(a, b - a);
+            if (!is_word(q.name)) return ja_fail(JA_ERR_PARSE, "PARTITIONS: a partition needs a name");
+            std::string inner = trim(s.substr(i + 1, close - i - 1));
+            if (inner.compare(0, 4, "size") == 0 && inner.size() > 4 && (inner[4] == ' ' || inner[4] == '\t')) {
+                if (!parse_int(inner.substr(4), &q.size)) return ja_fail(JA_ERR_PARSE, "PARTITIONS: bad size of %s", q.name.c_str());
+            } else {
+                if (!parse_sites(inner, &q.members)) return ja_fail(JA_ERR_PARSE, "PARTITIONS: bad members of %s", q.name.c_str());
+                q.size = (int)q.members.size();
+                q.bound = true;
+            }
+            p->parts.push_back(q);
+            i = close + 1;
+        }
+    }
+    for (const std::string& it : items(sect[2])) {          // IN: name @ site [(size: x GB)]
+        size_t at = it.find('@');
+        if (at == std::string::npos) return ja_fail(JA_ERR_PARSE, "bad IN item: %s", it.c_str());
+        ExAtom a;
+        a.name = trim(it.substr(0, at));
+        std::string rest = trim(it.substr(at + 1));
+        size_t par = rest.find('(');
+        std::string site = trim(par == std::string::npos ? rest : rest.substr(0, par));
+        if (!is_word(a.name) || !parse_int(site, &a.site)) return ja_fail(JA_ERR_PARSE, "bad IN item: %s", it.c_str());
+        if (par != std::string::npos) {
+            std::string in = trim(rest.substr(par + 1));
+            if (in.empty() || in.back() != ')') return ja_fail(JA_ERR_PARSE, "bad IN item: %s", it.c_str());
+            in = trim(in.substr(0, in.size() - 1));
+            size_t colon = in.find(':');
+            if (trim(in.substr(0, colon == std::string::npos ? 0 : colon)) != "size" || in.size() < 2 ||
+                in.compare(in.size() - 2, 2, "GB") != 0)
+                return ja_fail(JA_ERR_PARSE, "bad IN item: %s", it.c_str());
+            std::string num = trim(in.substr(colon + 1, in.size() - 2 - colon - 1));
+            char* end = nullptr;
+            a.gb = strtod(num.c_str(), &end);
+            if (num.empty() || *end) return ja_fail(JA_ERR_PARSE, "bad size in IN item: %s", it.c_str());
+        }
+        if (find_atom(*p, a.name) >= 0) return ja_fail(JA_ERR_PARSE, "atom %s declared twice", a.name.c_str());
+        if (p->atoms.size() == 64) return ja_fail(JA_ERR_INVALID_ARG, "more than 64 atoms");
+        p->atoms.push_back(a);
+    }
+    for (const std::string& it : items(sect[3])) {          // OUT: aggregate @ sites | partition
+        size_t at = it.find('@');
+        std::pair<uint64_t, ExTarget> o;
+        if (at == std::string::npos || !parse_aggregate(*p, it.substr(0, at), &o.first) || !parse_target(*p, it.substr(at + 1), &o.second))
+            return ja_fail(JA_ERR_PARSE, "bad OUT item: %s", it.c_str());
+        p->out.push_back(o);
+    }
+    for (const std::string& it : items(body)) {             // aggregate @ source(s) [-> destinations]
+        size_t arrow = it.find("->"), at = it.find('@');
+        ExAction a;
+        std::string left = arrow == std::string::npos ? it : it.substr(0, arrow);
+        if (at == std::string::npos || at > left.size() || !parse_aggregate(*p, left.substr(0, at), &a.agg) ||
+            !parse_target(*p, left.substr(at + 1), &a.src))
+            return ja_fail(JA_ERR_PARSE, "bad action: %s", it.c_str());
+        if (arrow != std::string::npos && !trim(it.substr(arrow + 2)).empty()) {
+            if (!parse_sites(it.substr(arrow + 2), &a.dests)) return ja_fail(JA_ERR_PARSE, "bad action: %s", it.c_str());
+            if (a.src.part >= 0 || a.src.sites.size() != 1)
+                return ja_fail(JA_ERR_PARSE, "an action with an arrow has one source site: %s", it.c_str());
+        }
+        if (std::find(p->actions.begin(), p->actions.end(), a) == p->actions.end()) p->actions.push_back(a);   // a set
+    }
+    if (has[0]) {
+        if (!parse_sites(sect[0], &p->gpus)) return ja_fail(JA_ERR_PARSE, "bad GPUS list");
+    } else {
+        std::set<int> seen;
+        for (const ExAtom& a : p->atoms) seen.insert(a.site);
+        for (const auto& o : p->out) seen.insert(o.second.sites.begin(), o.second.sites.end());
+        for (const ExAction& a : p->actions) {
+            seen.insert(a.dests.begin(), a.dests.end());
+            seen.insert(a.src.sites.begin(), a.src.sites.end());
+        }
+        for (const ExPartition& q : p->parts) seen.insert(q.members.begin(), q.members.end());
+        p->gpus.assign(seen.begin(), seen.end());
+    }
+    return check_static(*p);
+}
+
+std::string number(double v) {           // the shortest text that reads back to v, always with a '.' or an exponent
+    char buf[64];
+    auto r = std::to_chars(buf, buf + sizeof buf, v);
+    std::string s(buf, r.ptr);
+    if (s.find_first_of(".einf") == std::string::npos) s += ".0";
+    return s;
+}
+std::string agg_text(const Prog& p, uint64_t m) {
+    std::string s;
+    for (size_t i = 0; i < p.atoms.size(); ++i)
+        if ((m >> i) & 1) s += (s.empty() ? "" : "+") + p.atoms[i].name;
+    return s;
+}
+std::string sites_text(const std::vector<int>& v) {
+    std::string s;
+    for (size_t i = 0; i < v.size(); ++i) s += (i ? ", " : "") + std::to_string(v[i]);
+    return s;
+}
+std::string target_text(const Prog& p, const ExTarget& t) { return t.part >= 0 ? p.parts[t.part].name : sites_text(t.sites); }
+std::string format_program(const Prog& p) {
+    std::string s = "GPUS: " + sites_text(p.gpus) + "\n";
+    if (!p.parts.empty()) {
+        s += "PARTITIONS:";
+        for (const ExPartition& q : p.parts)
+            s += " " + q.name + " {" + (q.bound ? sites_text(q.members) : "size " + std::to_string(q.size)) + "}";
+        s += "\n";
+    }
+    s += "IN: ";
+    for (size_t i = 0; i < p.atoms.size(); ++i) {
+        const ExAtom& a = p.atoms[i];
+        s += (i ? "; " : "") + a.name + " @ " + std::to_string(a.site);
+        if (a.gb != 1.0) s += " (size: " + number(a.gb) + " GB)";
+    }
+    s += "\nOUT: ";
+    for (size_t i = 0; i < p.out.size(); ++i) s += (i ? "; " : "") + agg_text(p, p.out[i].first) + " @ " + target_text(p, p.out[i].second);
+    s += "\n\n";
+    for (const ExAction& a : p.actions) {
+        s += agg_text(p, a.agg) + " @ " + target_text(p, a.src);
+        if (!a.dests.empty()) s += " -> " + sites_text(a.dests);
+        s += "\n";
+    }
+    return s;
+}
+
+// ------------------------------------------------------------------------------------------ memberships, expansion
+bool all_bound(const Prog& p) {
+    for (const ExPartition& q : p.parts)
+        if (!q.bound) return false;
+    return true;
+}
+bool resolve(const Prog& p, const ExTarget& t, std::vector<int>* sites) {
+    if (t.part < 0) {
+        *sites = t.sites;
+        return true;
+    }
+    if (!p.parts[t.part].bound) return false;
+    *sites = p.parts[t.part].members;
+    return true;
+}
+bool expand(const Prog& p, std::vector<Flat>* res) {
+    res->clear();
+    std::vector<int> sites;
+    for (const ExAction& a : p.actions) {
+        if (!resolve(p, a.src, &sites)) return false;
+        for (int s : sites) {
+            Flat f{a.agg, s, a.dests};
+            if (std::find(res->begin(), res->end(), f) == res->end()) res->push_back(f);
+        }
+    }
+    return true;
+}
+bool requirements(const Prog& p, std::vector<std::pair<uint64_t, int>>* res) {
+    res->clear();
+    std::vector<int> sites;
+    for (const auto& o : p.out) {
+        if (!resolve(p, o.second, &sites)) return false;
+        for (int s : sites) res->push_back({o.first, s});
+    }
+    return true;
+}
+// all memberships in enumeration order: per unbound partition (declaration order) a combination of what is left
+void enumerate_memberships(const Prog& p, std::vector<std::vector<std::vector<int>>>* all) {
+    std::vector<int> unbound;
+    std::set<int> taken;
+    for (size_t i = 0; i < p.parts.size(); ++i) {
+        if (p.parts[i].bound) taken.insert(p.parts[i].members.begin(), p.parts[i].members.end());
+        else unbound.push_back((int)i);
+    }
+    std::vector<int> free_sites;
+    for (int s : p.gpus)
+        if (!taken.count(s)) free_sites.push_back(s);
+    std::vector<std::vector<int>> cur;
+    struct Rec {
+        const Prog& p;
+        const std::vector<int>& unbound;
+        std::vector<std::vector<std::vector<int>>>* all;
+        std::vector<std::vector<int>>& cur;
+        void go(size_t i, const std::vector<int>& rest) {
+            if (i == unbound.size()) {
+                all->push_back(cur);
+                return;
+            }
+            const int k = p.parts[unbound[i]].size, n = (int)rest.size();
+            if (k > n) return;
+            std::vector<int> idx(k);
+            for (int t = 0; t < k; ++t) idx[t] = t;
+            while (true) {
+                std::vector<int> mem, left;
+                size_t q = 0;
+                for (int t = 0; t < n; ++t) {
+                    if (q < idx.size() && idx[q] == t) {
+                        mem.push_back(rest[t]);
+                        ++q;
+                    } else {
+                        left.push_back(rest[t]);
+                    }
+                }
+                cur.push_back(mem);
+                go(i + 1, left);
+                cur.pop_back();
+                int t = k - 1;
+                while (t >= 0 && idx[t] == n - k + t) --t;
+                if (t < 0) break;
+                ++idx[t];
+                for (int u = t + 1; u < k; ++u) idx[u] = idx[u - 1] + 1;
+            }
+        }
+    } rec{p, unbound, all, cur};
+    rec.go(0, free_sites);
+}
+void bind_membership(Prog* p, const std::vector<std::vector<int>>& mem) {
+    size_t k = 0;
+    for (ExPartition& q : p->parts)
+        if (!q.bound) {
+            q.members = mem[k++];
+            std::sort(q.members.begin(), q.members.end());
+            q.bound = true;
+        }
+}
+
+// ---------------------------------------------------------------------------- Definition "Closure; validity"
+// a partition of x into members of `avail` with the fewest parts; returns the number of parts, 0 if there is none
+struct Cover {
+    std::vector<uint64_t> cands;
+    int best = 0;
+    void rec(uint64_t rest, int parts) {
+        if (best && parts >= best) return;
+        if (!rest) {
+            best = parts;
+            return;
+        }
+        const uint64_t pivot = rest & (~rest + 1);
+        for (uint64_t y : cands)
+            if ((y & pivot) && (y & ~rest) == 0) rec(rest & ~y, parts + 1);
+    }
+};
+int exact_cover(uint64_t x, const std::vector<uint64_t>& avail) {
+    Cover c;
+    for (uint64_t y : avail)
+        if (y && (y & ~x) == 0) c.cands.push_back(y);
+    c.rec(x, 0);
+    return c.best;
+}
+std::vector<uint64_t> at_site(const State& st, int site) {
+    std::vector<uint64_t> res;
+    for (auto it = st.lower_bound({site, 0}); it != st.end() && it->first == site; ++it) res.push_back(it->second);
+    return res;
+}
+State closure_of(const Prog& p, const std::vector<Flat>& acts) {
+    State st;
+    for (size_t i = 0; i < p.atoms.size(); ++i) st.insert({p.atoms[i].site, 1ull << i});
+    bool changed = true;
+    while (changed) {
+        changed = false;
+        for (const Flat& a : acts) {
+            if (!exact_cover(a.agg, at_site(st, a.site))) continue;
+            if (st.insert({a.site, a.agg}).second) changed = true;
+            for (int d : a.dests)
+                if (st.insert({d, a.agg}).second) changed = true;
+        }
+    }
+    return st;
+}
+void check_bound(const Prog& p, bool* wf, bool* valid) {
+    std::vector<Flat> acts;
+    expand(p, &acts);
+    const State st = closure_of(p, acts);
+    *wf = true;
+    for (const Flat& a : acts)
+        if (!exact_cover(a.agg, at_site(st, a.site))) *wf = false;
+    *valid = *wf;
+    std::vector<std::pair<uint64_t, int>> req;
+    requirements(p, &req);
+    for (const auto& r : req)
+        if (!st.count({r.second, r.first})) *valid = false;
+}
+bool valid_bound(const Prog& p) {
+    bool wf, v;
+    check_bound(p, &wf, &v);
+    return v;
+}
+
+// --------------------------------------------------------------------------------------------------- simulator
+double atom_gb(const Prog& p, uint64_t agg) {
+    for (size_t i = 0; i < p.atoms.size(); ++i)
+        if ((agg >> i) & 1) return p.atoms[i].gb;
+    return 0.0;
+}
+// kind 0: a direct link of the given capacity, 1: the bridge
+void mesh_link(const ja_machine_t& m, int a, int b, int* kind, double* cap) {
+    if (abs(a - b) == 4) {
+        *kind = 0;
+        *cap = m.double_gbs;
+    } else if (a / 4 == b / 4) {
+        *kind = 0;
+        *cap = m.link_gbs;
+    } else {
+        *kind = 1;
+        *cap = m.pcie_gbs;
+    }
+}
+struct FlowRec {
+    int act, dst;
+    double rem;
+};
+bool simulate(const Prog& p, const ja_machine_t& m, double* completion_ms, double* t_start, double* t_agg, double* t_fin) {
+    std::vector<Flat> acts;
+    expand(p, &acts);
+    const int n = (int)acts.size();
+    std::map<int, std::map<uint64_t, double>> have;
+    for (size_t i = 0; i < p.atoms.size(); ++i) have[p.atoms[i].site][1ull << i] = 0.0;
+    enum { WAIT, AGG, XFER, DONE };
+    std::vector<int> st(n, WAIT);
+    std::vector<double> rem_agg(n, 0.0), ts(n, -1.0), ta(n, -1.0), tf(n, -1.0);
+    std::vector<FlowRec> flows;
+    double now = 0.0;
+    auto begin_transfer = [&](int i) {
+        if (!acts[i].dests.empty()) {
+            st[i] = XFER;
+            for (int d : acts[i].dests) flows.push_back({i, d, atom_gb(p, acts[i].agg)});
+        } else {
+            st[i] = DONE;
+            tf[i] = now;
+        }
+    };
+    while (true) {
+        bool progress = true;
+        while (progress) {              // start whatever is enabled now; steps of no cost may enable more
+            progress = false;
+            for (int i = 0; i < n; ++i) {
+                if (st[i] != WAIT) continue;
+                std::vector<uint64_t> avail;
+                for (const auto& kv : have[acts[i].site]) avail.push_back(kv.first);
+                const int parts = exact_cover(acts[i].agg, avail);
+                if (!parts) continue;
+                ts[i] = now;
+                progress = true;
+                if (parts >= 2) {
+                    st[i] = AGG;
+                    rem_agg[i] = (parts + 1) * atom_gb(p, acts[i].agg);
+                } else {
+                    ta[i] = now;
+                    begin_transfer(i);
+                }
+            }
+        }
+        std::vector<int> active;
+        for (int i = 0; i < n; ++i)
+            if (st[i] == AGG) active.push_back(i);
+        if (active.empty() && flows.empty()) break;
+        std::map<int, int> per_site;
+        for (int i : active) ++per_site[acts[i].site];
+        std::vector<double> rate_agg(active.size()), rate_flow(flows.size());
+        for (size_t k = 0; k < active.size(); ++k) rate_agg[k] = m.hbm_gbs / per_site[acts[active[k]].site];
+        if (m.fabric == JA_FABRIC_NVSWITCH) {
+            std::map<int, int> out_n, in_n;
+            for (const FlowRec& f : flows) {
+                ++out_n[acts[f.act].site];
+                ++in_n[f.dst];
+            }
+            for (size_t k = 0; k < flows.size(); ++k)
+                rate_flow[k] = std::min(m.link_gbs / out_n[acts[flows[k].act].site], m.link_gbs / in_n[flows[k].dst]);
+        } else {
+            std::map<std::pair<int, int>, int> on;      // (-1, -1) = the bridge
+            for (const FlowRec& f : flows) {
+                int kind;
+                double cap;
+                mesh_link(m, acts[f.act].site, f.dst, &kind, &cap);
+                ++on[kind ? std::make_pair(-1, -1) : std::make_pair(acts[f.act].site, f.dst)];
+            }
+            for (size_t k = 0; k < flows.size(); ++k) {
+                int kind;
+                double cap;
+                mesh_link(m, acts[flows[k].act].site, flows[k].dst, &kind, &cap);
+                rate_flow[k] = cap / on[kind ? std::make_pair(-1, -1) : std::make_pair(acts[flows[k].act].site, flows[k].dst)];
+            }
+        }
+        double dt = INFINITY;
+        for (size_t k = 0; k < active.size(); ++k) dt = std::min(dt, rem_agg[active[k]] / rate_agg[k]);
+        for (size_t k = 0; k < flows.size(); ++k) dt = std::min(dt, flows[k].rem / rate_flow[k]);
+        now += dt;
+        for (size_t k = 0; k < active.size(); ++k) rem_agg[active[k]] -= rate_agg[k] * dt;
+        for (size_t k = 0; k < flows.size(); ++k) flows[k].rem -= rate_flow[k] * dt;
+        const double eps = 1e-12;
+        std::vector<FlowRec> keep;
+        for (size_t k = 0; k < flows.size(); ++k) {
+            if (flows[k].rem <= eps * (1.0 + rate_flow[k] * dt)) {
+                have[flows[k].dst].insert({acts[flows[k].act].agg, now});
+            } else {
+                keep.push_back(flows[k]);
+            }
+        }
+        flows.swap(keep);
+        for (size_t k = 0; k < active.size(); ++k) {
+            const int i = active[k];
+            if (rem_agg[i] <= eps * (1.0 + rate_agg[k] * dt)) {
+                have[acts[i].site].insert({acts[i].agg, now});
+                ta[i] = now;
+                begin_transfer(i);
+            }
+        }
+        for (int i = 0; i < n; ++i) {
+            if (st[i] != XFER) continue;
+            bool any = false;
+            for (const FlowRec& f : flows) any |= f.act == i;
+            if (!any) {
+                st[i] = DONE;
+                tf[i] = now;
+            }
+        }
+    }
+    for (int i = 0; i < n; ++i)
+        if (st[i] != DONE) return false;
+    *completion_ms = now * 1e3;
+    for (int i = 0; i < n; ++i) {
+        if (t_start) t_start[i] = ts[i] * 1e3;
+        if (t_agg) t_agg[i] = ta[i] * 1e3;
+        if (t_fin) t_fin[i] = tf[i] * 1e3;
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------------------ bodies
+ExTarget one_site(int s) {
+    ExTarget t;
+    t.sites.push_back(s);
+    return t;
+}
+void add_action(Prog* p, const ExAction& a) {
+    if (std::find(p->actions.begin(), p->actions.end(), a) == p->actions.end()) p->actions.push_back(a);
+}
+void naive_body(Prog* p) {
+    p->actions.clear();
+    std::vector<std::pair<uint64_t, int>> req;
+    requirements(*p, &req);
+    std::vector<std::set<int>> need(p->atoms.size());
+    for (const auto& r : req)
+        for (size_t a = 0; a < p->atoms.size(); ++a)
+            if (((r.first >> a) & 1) && p->atoms[a].site != r.second) need[a].insert(r.second);
+    for (size_t a = 0; a < p->atoms.size(); ++a) {
+        if (need[a].empty()) continue;
+        ExAction act;
+        act.agg = 1ull << a;
+        act.src = one_site(p->atoms[a].site);
+        act.dests.assign(need[a].begin(), need[a].end());
+        p->actions.push_back(act);
+    }
+    for (const auto& o : p->out) {
+        if (!(o.first & (o.first - 1))) continue;      // a single atom needs no aggregation
+        ExAction act;
+        act.agg = o.first;
+        act.src = o.second;
+        add_action(p, act);
+    }
+}
+void butterfly_body(Prog* p) {
+    p->actions.clear();
+    std::vector<std::pair<uint64_t, int>> req;
+    requirements(*p, &req);
+    std::vector<uint64_t> order;                       // aggregates in order of first appearance
+    std::map<uint64_t, std::set<int>> groups;
+    for (const auto& r : req) {
+        if (!groups.count(r.first)) order.push_back(r.first);
+        groups[r.first].insert(r.second);
+    }
+    std::vector<std::set<int>> need(p->atoms.size());
+    std::vector<std::pair<uint64_t, std::vector<int>>> local;
+    for (uint64_t x : order) {
+        std::vector<int> t(groups[x].begin(), groups[x].end());
+        std::vector<uint64_t> held(t.size(), 0);
+        std::set<int> atom_sites;
+        for (size_t a = 0; a < p->atoms.size(); ++a) {
+            if (!((x >> a) & 1)) continue;
+            atom_sites.insert(p->atoms[a].site);
+            for (size_t i = 0; i < t.size(); ++i)
+                if (t[i] == p->atoms[a].site) held[i] |= 1ull << a;
+        }
+        int k = 0;
+        while ((2u << k) <= t.size()) ++k;
+        bool ok = t.size() >= 2 && (1u << k) == t.size() && atom_sites == groups[x];
+        for (size_t i = 1; ok && i < t.size(); ++i) ok = __builtin_popcountll(held[i]) == __builtin_popcountll(held[0]);
+        if (!ok) {
+            for (int s : t)
+                for (size_t a = 0; a < p->atoms.size(); ++a)
+                    if (((x >> a) & 1) && p->atoms[a].site != s) need[a].insert(s);
+            if (x & (x - 1)) local.push_back({x, t});
+            continue;
+        }
+        std::vector<uint64_t> cur = held;
+        for (int b = 0; b < k; ++b) {
+            for (size_t i = 0; i < t.size(); ++i) {
+                ExAction act;
+                act.agg = cur[i];
+                act.src = one_site(t[i]);
+                act.dests.push_back(t[i ^ (1u << b)]);
+                add_action(p, act);
+            }
+            std::vector<uint64_t> nxt(t.size());
+            for (size_t i = 0; i < t.size(); ++i) nxt[i] = cur[i] | cur[i ^ (1u << b)];
+            cur.swap(nxt);
+        }
+        local.push_back({x, t});
+    }
+    for (size_t a = 0; a < p->atoms.size(); ++a) {
+        if (need[a].empty()) continue;
+        ExAction act;
+        act.agg = 1ull << a;
+        act.src = one_site(p->atoms[a].site);
+        act.dests.assign(need[a].begin(), need[a].end());
+        add_action(p, act);
+    }
+    for (const auto& l : local) {
+        ExAction act;
+        act.agg = l.first;
+        act.src.sites = l.second;
+        add_action(p, act);
+    }
+}
+void normalise(Prog* p) {
+    std::vector<Flat> acts;
+    expand(*p, &acts);
+    p->actions.clear();
+    for (const Flat& f : acts) {
+        ExAction a;
+        a.agg = f.agg;
+        a.src = one_site(f.site);
+        a.dests = f.dests;
+        p->actions.push_back(a);
+    }
+}
+bool is_normal(const Prog& p) {
+    for (const ExAction& a : p.actions)
+        if (a.src.part >= 0 || a.src.sites.size() != 1) return false;
+    return true;
+}
+bool same_size(const Prog& p, uint64_t m) {
+    double gb = -1;
+    for (size_t i = 0; i < p.atoms.size(); ++i)
+        if ((m >> i) & 1) {
+            if (gb >= 0 && p.atoms[i].gb != gb) return false;
+            gb = p.atoms[i].gb;
+        }
+    return true;
+}
+std::vector<int> mask_sites(uint64_t m) {
+    std::vector<int> v;
+    for (int s = 0; s < 64; ++s)
+        if ((m >> s) & 1) v.push_back(s);
+    return v;
+}
+bool contains(const std::vector<int>& v, int s) { return std::find(v.begin(), v.end(), s) != v.end(); }
+
+// one rule application on a normalised, bound program; q receives the rewritten program; false if the rule does not
+// match or its guard fails
+bool rewrite(const Prog& p, int rule, int i, int j, uint64_t a, uint64_t b, Prog* q) {
+    const int n = (int)p.actions.size();
+    *q = p;
+    auto idx = [&](int k) { return k >= 0 && k < n; };
+    switch (rule) {
+    case JA_RULE_INSERT: {
+        if (!a || (p.atoms.size() < 64 && (a >> p.atoms.size())) || !same_size(p, a) || !contains(p.gpus, i)) return false;
+        ExAction act;
+        act.agg = a;
+        act.src = one_site(i);
+        act.dests = mask_sites(b);
+        for (int d : act.dests)
+            if (!contains(p.gpus, d)) return false;
+        add_action(q, act);
+        bool wf, v;
+        check_bound(*q, &wf, &v);
+        return wf;
+    }
+    case JA_RULE_DELETE:
+        if (!idx(i)) return false;
+        q->actions.erase(q->actions.begin() + i);
+        return valid_bound(*q);
+    case JA_RULE_FISSION: {
+        if (!idx(i)) return false;
+        std::vector<int> d1, d2;
+        for (int t : p.actions[i].dests) ((a >> t) & 1 ? d1 : d2).push_back(t);
+        if (d1.empty() || d2.empty()) return false;
+        q->actions[i].dests = d1;
+        ExAction act = p.actions[i];
+        act.dests = d2;
+        q->actions.push_back(act);
+        return valid_bound(*q);
+    }
+    case JA_RULE_FUSION: {
+        if (!idx(i) || !idx(j) || i == j) return false;
+        const ExAction &x = p.actions[i], &y = p.actions[j];
+        if (x.agg != y.agg || !(x.src == y.src) || x.dests.empty() || y.dests.empty()) return false;
+        std::set<int> u(x.dests.begin(), x.dests.end());
+        u.insert(y.dests.begin(), y.dests.end());
+        q->actions[i].dests.assign(u.begin(), u.end());
+        q->actions.erase(q->actions.begin() + j);
+        return valid_bound(*q);
+    }
+    case JA_RULE_RELAY_IN: {
+        if (!idx(i)) return false;
+        const ExAction& x = p.actions[i];
+        const int dest = j, relay = (int)a;
+        if (!contains(x.dests, dest) || relay == x.src.sites[0] || contains(x.dests, relay) || !contains(p.gpus, relay)) return false;
+        std::vector<int> rest;
+        for (int t : x.dests)
+            if (t != dest) rest.push_back(t);
+        rest.push_back(relay);
+        std::sort(rest.begin(), rest.end());
+        q->actions[i].dests = rest;
+        ExAction hop;
+        hop.agg = x.agg;
+        hop.src = one_site(relay);
+        hop.dests.push_back(dest);
+        add_action(q, hop);
+        return valid_bound(*q);
+    }
+    case JA_RULE_RELAY_OUT: {
+        if (!idx(i) || !idx(j) || i == j) return false;
+        const ExAction &x = p.actions[i], &y = p.actions[j];
+        const int r = y.src.sites[0];
+        if (x.agg != y.agg || x.dests.size() != 1 || x.dests[0] != r || y.dests.size() != 1) return false;
+        q->actions[i].dests = y.dests;
+        q->actions.erase(q->actions.begin() + j);
+        return valid_bound(*q);
+    }
+    case JA_RULE_PUSHDOWN: {
+        if (!idx(i) || !idx(j) || i == j) return false;
+        const ExAction &x = p.actions[i], &y = p.actions[j];
+        if (!(x.src == y.src) || x.dests != y.dests || x.dests.empty() || (x.agg & y.agg) || !same_size(p, x.agg | y.agg)) return false;
+        q->actions[i].agg = x.agg | y.agg;
+        q->actions.erase(q->actions.begin() + j);
+        return valid_bound(*q);
+    }
+    case JA_RULE_PULLUP: {
+        if (!idx(i)) return false;
+        const ExAction& xy = p.actions[i];
+        const uint64_t x = a, y = xy.agg & ~a;
+        if (xy.dests.empty() || !x || !y || (x & ~xy.agg)) return false;
+        q->actions[i].agg = x;
+        ExAction other = xy;
+        other.agg = y;
+        q->actions.push_back(other);
+        if (b)
+            for (int t : xy.dests) {
+                ExAction loc;
+                loc.agg = xy.agg;
+                loc.src = one_site(t);
+                add_action(q, loc);
+            }
+        return valid_bound(*q);
+    }
+    case JA_RULE_SOURCE: {
+        if (!idx(i)) return false;
+        const ExAction& x = p.actions[i];
+        if (x.dests.empty() || j == x.src.sites[0] || contains(x.dests, j)) return false;
+        std::vector<Flat> acts;
+        expand(p, &acts);
+        if (!closure_of(p, acts).count({j, x.agg})) return false;
+        q->actions[i].src = one_site(j);
+        return valid_bound(*q);
+    }
+    }
+    return false;
+}
+
+// every program one rule application away, in a fixed order (per action: delete, fissions, substitutions, relays,
+// pullups; then per pair: relay elimination, fusion, pushdown)
+void neighbours(const Prog& p, std::vector<Prog>* res) {
+    res->clear();
+    const int n = (int)p.actions.size();
+    std::vector<Flat> acts;
+    expand(p, &acts);
+    const State st = closure_of(p, acts);
+    Prog q;
+    auto tryr = [&](int rule, int i, int j, uint64_t a, uint64_t b) {
+        if (rewrite(p, rule, i, j, a, b, &q)) res->push_back(q);
+    };
+    for (int i = 0; i < n; ++i) {
+        const ExAction& x = p.actions[i];
+        tryr(JA_RULE_DELETE, i, 0, 0, 0);
+        if (x.dests.size() > 1)
+            for (int t : x.dests) tryr(JA_RULE_FISSION, i, 0, 1ull << t, 0);
+        if (!x.dests.empty()) {
+            for (int s : p.gpus)
+                if (st.count({s, x.agg})) tryr(JA_RULE_SOURCE, i, s, 0, 0);
+            for (int t : x.dests)
+                for (int r : p.gpus) tryr(JA_RULE_RELAY_IN, i, t, (uint64_t)r, 0);
+            if (x.agg & (x.agg - 1))
+                for (size_t a = 0; a < p.atoms.size(); ++a)
+                    if ((x.agg >> a) & 1) tryr(JA_RULE_PULLUP, i, 0, 1ull << a, 1);
+        }
+        for (int j = 0; j < n; ++j) {
+            if (j != i) tryr(JA_RULE_RELAY_OUT, i, j, 0, 0);
+            if (j > i) {
+                tryr(JA_RULE_FUSION, i, j, 0, 0);
+                tryr(JA_RULE_PUSHDOWN, i, j, 0, 0);
+            }
+        }
+    }
+}
+typedef std::vector<std::tuple<uint64_t, int, std::vector<int>>> Key;
+Key key_of(const Prog& p) {
+    std::vector<Flat> acts;
+    expand(p, &acts);
+    Key k;
+    for (const Flat& f : acts) {
+        std::vector<int> d = f.dests;
+        std::sort(d.begin(), d.end());
+        k.push_back(std::make_tuple(f.agg, f.site, d));
+    }
+    std::sort(k.begin(), k.end());
+    return k;
+}
+bool best_constructed(const Prog& bound, const ja_machine_t& m, int body, Prog* best, double* ms) {
+    std::vector<Prog> cands;
+    if (body == JA_BODY_OWN) {
+        cands.push_back(bound);
+    } else {
+        if (body == JA_BODY_NAIVE || body == JA_BODY_BEST) {
+            cands.push_back(bound);
+            naive_body(&cands.back());
+        }
+        if (body == JA_BODY_BUTTERFLY || body == JA_BODY_BEST) {
+            cands.push_back(bound);
+            butterfly_body(&cands.back());
+        }
+    }
+    bool found = false;
+    for (Prog& c : cands) {
+        double t;
+        if (!valid_bound(c) || !simulate(c, m, &t, nullptr, nullptr, nullptr)) continue;
+        if (!found || t < *ms) {
+            *best = c;
+            *ms = t;
+            found = true;
+        }
+    }
+    return found;
+}
+
+ja_status_t need_bound(const Prog* p) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    if (!all_bound(*p)) return ja_fail(JA_ERR_INVALID_ARG, "a partition declared by size has no members yet: bind or place the program first");
+    return JA_OK;
+}
+ja_status_t check_machine(const ja_machine_t* m, const Prog& p) {
+    if (!m) return ja_fail(JA_ERR_INVALID_ARG, "null machine");
+    if (!(m->hbm_gbs > 0) || !(m->link_gbs > 0)) return ja_fail(JA_ERR_INVALID_ARG, "machine: bandwidths must be positive");
+    if (m->fabric == JA_FABRIC_CUBE_MESH) {
+        if (!(m->double_gbs > 0) || !(m->pcie_gbs > 0)) return ja_fail(JA_ERR_INVALID_ARG, "machine: bandwidths must be positive");
+        for (int s : p.gpus)
+            if (s > 7) return ja_fail(JA_ERR_INVALID_ARG, "the cube mesh has sites 0..7");
+    } else if (m->fabric != JA_FABRIC_NVSWITCH) {
+        return ja_fail(JA_ERR_INVALID_ARG, "machine: unknown fabric");
+    }
+    return JA_OK;
+}
+
+}  // namespace
+
+// ============================================================================================================ C ABI
+extern "C" ja_status_t ja_machine_preset(const char* name, ja_machine_t* out) {
+    if (!name || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    ja_machine_t m = {JA_FABRIC_NVSWITCH, 8, 0, 0, 0, 0};
+    if (!strcmp(name, "dgx_h100")) {
+        m.link_gbs = 450.0;
+        m.hbm_gbs = 3350.0;
+    } else if (!strcmp(name, "dgx_a100")) {
+        m.link_gbs = 300.0;
+        m.hbm_gbs = 2039.0;
+    } else if (!strcmp(name, "hgx_b200")) {
+        m.link_gbs = 900.0;
+        m.hbm_gbs = 7700.0;
+    } else if (!strcmp(name, "dgx_v100")) {
+        m.fabric = JA_FABRIC_CUBE_MESH;
+        m.link_gbs = 25.0;
+        m.double_gbs = 50.0;
+        m.pcie_gbs = 15.75;
+        m.hbm_gbs = 900.0;
+    } else {
+        return ja_fail(JA_ERR_INVALID_ARG, "unknown machine '%s'", name);
+    }
+    *out = m;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_parse(const char* text, ja_exprog_t** out) {
+    if (!text || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    Prog* p = new Prog();
+    ja_status_t st = parse_program(text, p);
+    if (st != JA_OK) {
+        delete p;
+        return st;
+    }
+    *out = p;
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_clone(const ja_exprog_t* p, ja_exprog_t** out) {
+    if (!p || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    *out = new Prog(*p);
+    return JA_OK;
+}
+extern "C" void ja_exprog_destroy(ja_exprog_t* p) { delete p; }
+
+extern "C" ja_status_t ja_exprog_format(const ja_exprog_t* p, char* buf, int64_t cap, int64_t* needed) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    const std::string s = format_program(*p);
+    if (needed) *needed = (int64_t)s.size() + 1;
+    if (!buf) return JA_OK;
+    if (cap < (int64_t)s.size() + 1) return ja_fail(JA_ERR_INVALID_ARG, "buffer too small: %lld bytes needed", (long long)s.size() + 1);
+    memcpy(buf, s.c_str(), s.size() + 1);
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_counts(const ja_exprog_t* p, int32_t* n_gpus, int32_t* n_partitions, int32_t* n_atoms,
+                                        int32_t* n_out, int32_t* n_actions, int32_t* n_expanded) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    if (n_gpus) *n_gpus = (int32_t)p->gpus.size();
+    if (n_partitions) *n_partitions = (int32_t)p->parts.size();
+    if (n_atoms) *n_atoms = (int32_t)p->atoms.size();
+    if (n_out) *n_out = (int32_t)p->out.size();
+    if (n_actions) *n_actions = (int32_t)p->actions.size();
+    if (n_expanded) {
+        std::vector<Flat> acts;
+        *n_expanded = expand(*p, &acts) ? (int32_t)acts.size() : -1;
+    }
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_get_actions(const ja_exprog_t* p, uint64_t* aggregate, int32_t* source, uint64_t* dests) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    std::vector<Flat> acts;
+    if (!expand(*p, &acts)) return ja_fail(JA_ERR_INVALID_ARG, "a partition used by the body has no members yet");
+    for (size_t i = 0; i < acts.size(); ++i) {
+        if (aggregate) aggregate[i] = acts[i].agg;
+        if (source) source[i] = acts[i].site;
+        if (dests) {
+            dests[i] = 0;
+            for (int d : acts[i].dests) dests[i] |= 1ull << d;
+        }
+    }
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_get_requirements(const ja_exprog_t* p, int32_t* n, uint64_t* aggregate, int32_t* site) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    std::vector<std::pair<uint64_t, int>> req;
+    if (!requirements(*p, &req)) return ja_fail(JA_ERR_INVALID_ARG, "a partition named in OUT has no members yet");
+    if (n) *n = (int32_t)req.size();
+    for (size_t i = 0; i < req.size(); ++i) {
+        if (aggregate) aggregate[i] = req[i].first;
+        if (site) site[i] = req[i].second;
+    }
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_get_atoms(const ja_exprog_t* p, int32_t* site, double* size_gb) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    for (size_t i = 0; i < p->atoms.size(); ++i) {
+        if (site) site[i] = p->atoms[i].site;
+        if (size_gb) size_gb[i] = p->atoms[i].gb;
+    }
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_num_memberships(const ja_exprog_t* p, int64_t* n) {
+    if (!p || !n) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    std::vector<std::vector<std::vector<int>>> all;
+    enumerate_memberships(*p, &all);
+    *n = (int64_t)all.size();
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_bind(ja_exprog_t* p, int64_t index) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    std::vector<std::vector<std::vector<int>>> all;
+    enumerate_memberships(*p, &all);
+    if (index < 0 || index >= (int64_t)all.size()) return ja_fail(JA_ERR_INVALID_ARG, "membership %lld of %lld", (long long)index, (long long)all.size());
+    bind_membership(p, all[index]);
+    return check_static(*p);
+}
+extern "C" ja_status_t ja_exprog_membership(const ja_exprog_t* p, const char* partition, uint64_t* members) {
+    if (!p || !partition || !members) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    const int k = find_part(*p, partition);
+    if (k < 0) return ja_fail(JA_ERR_INVALID_ARG, "no partition '%s'", partition);
+    if (!p->parts[k].bound) return ja_fail(JA_ERR_INVALID_ARG, "partition '%s' has no members yet", partition);
+    *members = 0;
+    for (int s : p->parts[k].members) *members |= 1ull << s;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_closure(const ja_exprog_t* p, int64_t* n, uint64_t* aggregate, int32_t* site) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    std::vector<Flat> acts;
+    expand(*p, &acts);
+    const State st = closure_of(*p, acts);
+    if (n) *n = (int64_t)st.size();
+    int64_t i = 0;
+    for (const auto& e : st) {
+        if (aggregate) aggregate[i] = e.second;
+        if (site) site[i] = e.first;
+        ++i;
+    }
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_check(const ja_exprog_t* p, int32_t* well_formed, int32_t* valid) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    bool wf, v;
+    check_bound(*p, &wf, &v);
+    if (well_formed) *well_formed = wf;
+    if (valid) *valid = v;
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_valid_any(const ja_exprog_t* p, int32_t* valid) {
+    if (!p || !valid) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    std::vector<std::vector<std::vector<int>>> all;
+    enumerate_memberships(*p, &all);
+    *valid = 0;
+    for (const auto& mem : all) {
+        Prog q = *p;
+        bind_membership(&q, mem);
+        if (valid_bound(q)) {
+            *valid = 1;
+            break;
+        }
+    }
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_simulate(const ja_exprog_t* p, const ja_machine_t* machine, double* completion_ms,
+                                          double* start_ms, double* aggregated_ms, double* finish_ms) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    if ((s = check_machine(machine, *p)) != JA_OK) return s;
+    double ms = 0;
+    if (!simulate(*p, *machine, &ms, start_ms, aggregated_ms, finish_ms))
+        return ja_fail(JA_ERR_INVALID_ARG, "the program is not well-formed: an action never becomes enabled");
+    if (completion_ms) *completion_ms = ms;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_body(ja_exprog_t* p, int32_t body) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    if (body == JA_BODY_NAIVE) naive_body(p);
+    else if (body == JA_BODY_BUTTERFLY) butterfly_body(p);
+    else if (body != JA_BODY_OWN) return ja_fail(JA_ERR_INVALID_ARG, "body %d", body);
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_normalise(ja_exprog_t* p) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    normalise(p);
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_rewrite(ja_exprog_t* p, int32_t rule, int32_t i, int32_t j, uint64_t a, uint64_t b, int32_t* applied) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    if (!applied) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    if (!is_normal(*p)) return ja_fail(JA_ERR_INVALID_ARG, "the rules work on a normalised program (ja_exprog_normalise)");
+    if (rule < JA_RULE_INSERT || rule > JA_RULE_SOURCE) return ja_fail(JA_ERR_INVALID_ARG, "rule %d", rule);
+    Prog q;
+    *applied = rewrite(*p, rule, i, j, a, b, &q) ? 1 : 0;
+    if (*applied) *p = q;
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_synthesize(ja_exprog_t* p, const ja_machine_t* machine, int32_t depth, int32_t beam, double* ms) {
+    ja_status_t s = need_bound(p);
+    if (s != JA_OK) return s;
+    if ((s = check_machine(machine, *p)) != JA_OK) return s;
+    if (depth < 0 || beam < 1) return ja_fail(JA_ERR_INVALID_ARG, "depth >= 0 and beam >= 1");
+    Prog start;
+    double t0 = 0;
+    if (!p->actions.empty()) {
+        start = *p;
+        normalise(&start);
+        if (!valid_bound(start) || !simulate(start, *machine, &t0, nullptr, nullptr, nullptr))
+            return ja_fail(JA_ERR_INVALID_ARG, "the program's own body is not valid");
+    } else {
+        if (!best_constructed(*p, *machine, JA_BODY_BEST, &start, &t0)) return ja_fail(JA_ERR_INVALID_ARG, "OUT cannot be satisfied");
+        normalise(&start);
+    }
+    std::pair<double, Prog> best(t0, start);
+    std::vector<std::pair<double, Prog>> level(1, best);
+    std::set<Key> seen;
+    seen.insert(key_of(start));
+    std::vector<Prog> nb;
+    for (int d = 0; d < depth; ++d) {
+        std::vector<std::pair<double, Prog>> nxt;
+        for (const auto& cur : level) {
+            neighbours(cur.second, &nb);
+            for (const Prog& r : nb) {
+                if (!seen.insert(key_of(r)).second) continue;
+                double t;
+                if (!simulate(r, *machine, &t, nullptr, nullptr, nullptr)) continue;
+                nxt.push_back({t, r});
+            }
+        }
+        if (nxt.empty()) break;
+        std::stable_sort(nxt.begin(), nxt.end(), [](const std::pair<double, Prog>& x, const std::pair<double, Prog>& y) {
+            return x.first != y.first ? x.first < y.first : x.second.actions.size() < y.second.actions.size();
+        });
+        if ((int)nxt.size() > beam) nxt.resize(beam);
+        level.swap(nxt);
+        if (level[0].first < best.first * (1.0 - 1e-12)) best = level[0];
+    }
+    *p = best.second;
+    if (ms) *ms = best.first;
+    return JA_OK;
+}
+extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machine, int32_t body, double* ms) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    ja_status_t s = check_machine(machine, *p);
+    if (s != JA_OK) return s;
+    if (body < JA_BODY_OWN || body > JA_BODY_BEST) return ja_fail(JA_ERR_INVALID_ARG, "body %d", body);
+    std::vector<std::vector<std::vector<int>>> all;
+    enumerate_memberships(*p, &all);
+    bool found = false;
+    Prog best;
+    double best_ms = 0;
+    for (const auto& mem : all) {
+        Prog q = *p;
+        bind_membership(&q, mem);
+        Prog c;
+        double t;
+        if (!best_constructed(q, *machine, body, &c, &t)) continue;
+        if (!found || t < best_ms * (1.0 - 1e-12)) {
+            best = c;
+            best_ms = t;
+            found = true;
+        }
+    }
+    if (!found) return ja_fail(JA_ERR_INVALID_ARG, "no membership makes the program valid");
+    *p = best;
+    if (ms) *ms = best_ms;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, const int32_t* n_producer_splits,
+                                          const int64_t* consumer_splits, const int32_t* n_consumer_splits, int32_t m,
+                                          const int32_t* copy_site, const int32_t* consumer_specs, int32_t n_specs,
+                                          int32_t width_bytes, ja_exprog_t** out) {
+    if (rank < 1 || rank > 8 || !producer_splits || !n_producer_splits || !consumer_splits || !n_consumer_splits || m < 1 ||
+        !copy_site || !consumer_specs || n_specs < 1 || width_bytes < 1 || !out)
+        return ja_fail(JA_ERR_INVALID_ARG, "bad argument");
+    std::vector<std::vector<int64_t>> ps(rank), cs(rank), ov(rank);
+    const int64_t *pp = producer_splits, *cp = consumer_splits;
+    int64_t n_pblocks = 1, n_cblocks = 1, n_cells = 1;
+    for (int d = 0; d < rank; ++d) {
+        if (n_producer_splits[d] < 2 || n_consumer_splits[d] < 2) return ja_fail(JA_ERR_TILING, "index %d: at least two split points", d);
+        ps[d].assign(pp, pp + n_producer_splits[d]);
+        cs[d].assign(cp, cp + n_consumer_splits[d]);
+        pp += n_producer_splits[d];
+        cp += n_consumer_splits[d];
+        for (const auto* v : {&ps[d], &cs[d]}) {
+            if ((*v)[0] != 0) return ja_fail(JA_ERR_TILING, "index %d: split points start at 0", d);
+            for (size_t i = 1; i < v->size(); ++i)
+                if ((*v)[i] <= (*v)[i - 1]) return ja_fail(JA_ERR_TILING, "index %d: split points must increase", d);
+        }
+        if (ps[d].back() != cs[d].back()) return ja_fail(JA_ERR_SHAPE, "index %d: the two tilings differ in extent", d);
+        std::set<int64_t> u(ps[d].begin(), ps[d].end());
+        u.insert(cs[d].begin(), cs[d].end());
+        ov[d].assign(u.begin(), u.end());
+        n_pblocks *= (int64_t)ps[d].size() - 1;
+        n_cblocks *= (int64_t)cs[d].size() - 1;
+        n_cells *= (int64_t)ov[d].size() - 1;
+    }
+    if (n_cells * m > 64) return ja_fail(JA_ERR_INVALID_ARG, "%lld atoms x %d copies: at most 64 ExProg atoms", (long long)n_cells, m);
+    Prog* p = new Prog();
+    std::set<int> g;
+    for (int64_t i = 0; i < n_pblocks * m; ++i) g.insert(copy_site[i]);
+    for (int i = 0; i < n_specs; ++i) g.insert(i);
+    p->gpus.assign(g.begin(), g.end());
+    for (int i = 0; i < n_specs; ++i) {
+        ExPartition q;
+        q.name = "S" + std::to_string(i + 1);
+        q.size = 1;
+        p->parts.push_back(q);
+    }
+    auto owner = [](const std::vector<int64_t>& s, int64_t lo) {
+        int i = 0;
+        while (!(s[i] <= lo && lo < s[i + 1])) ++i;
+        return i;
+    };
+    struct Cell {
+        int64_t j, pb, cb;
+        double gb;
+    };
+    std::vector<Cell> cells;
+    std::vector<int> c(rank, 0);
+    for (int64_t j = 0; j < n_cells; ++j) {
+        int64_t card = 1, pb = 0, cb = 0;
+        for (int d = 0; d < rank; ++d) {
+            const int64_t lo = ov[d][c[d]];
+            card *= ov[d][c[d] + 1] - lo;
+            pb = pb * ((int64_t)ps[d].size() - 1) + owner(ps[d], lo);
+            cb = cb * ((int64_t)cs[d].size() - 1) + owner(cs[d], lo);
+        }
+        cells.push_back({j, pb, cb, (double)(card * width_bytes) / 1e9});
+        for (int d = rank - 1; d >= 0; --d) {
+            if (++c[d] < (int)ov[d].size() - 1) break;
+            c[d] = 0;
+        }
+    }
+    // IN: by site, then atom, then copy
+    std::vector<std::tuple<int, int64_t, int, double>> entries;
+    for (const Cell& ce : cells)
+        for (int k = 0; k < m; ++k) entries.push_back(std::make_tuple(copy_site[ce.pb * m + k], ce.j, k, ce.gb));
+    std::sort(entries.begin(), entries.end());
+    std::map<std::pair<int64_t, int>, int> index;
+    for (const auto& e : entries) {
+        ExAtom a;
+        a.name = "a" + std::to_string(std::get<1>(e)) + "_" + std::to_string(std::get<2>(e));
+        a.site = std::get<0>(e);
+        a.gb = std::get<3>(e);
+        index[{std::get<1>(e), std::get<2>(e)}] = (int)p->atoms.size();
+        p->atoms.push_back(a);
+    }
+    for (const Cell& ce : cells) {
+        uint64_t x = 0;
+        for (int k = 0; k < m; ++k) x |= 1ull << index[{ce.j, k}];
+        for (int i = 0; i < n_specs; ++i) {
+            if (consumer_specs[i] < 0 || consumer_specs[i] >= n_cblocks) {
+                delete p;
+                return ja_fail(JA_ERR_INVALID_ARG, "function spec %d names block %d of %lld", i, consumer_specs[i], (long long)n_cblocks);
+            }
+            if (consumer_specs[i] == ce.cb) {
+                ExTarget t;
+                t.part = i;
+                p->out.push_back({x, t});
+            }
+        }
+    }
+    if ((int)p->gpus.size() != n_specs) {
+        delete p;
+        return ja_fail(JA_ERR_INVALID_ARG, "one function spec of op per GPU: the partitions of size one must cover the GPUs");
+    }
+    ja_status_t st = check_static(*p);
+    if (st != JA_OK) {
+        delete p;
+        return st;
+    }
+    *out = p;
+    return JA_OK;
+}

@@ -1,0 +1,219 @@
+"""ctypes binding of the exchange-program part of libja's C ABI (include/ja_exprog.h): the same names, argument
+marshalling only.  `ExchangeProgram` owns a handle.  Aggregates are masks over the atoms in declaration order, sets of
+sites masks over site numbers, as in the header."""
+from __future__ import annotations
+
+import ctypes
+
+from .binding import LIB, _check
+
+JA_FABRIC_NVSWITCH, JA_FABRIC_CUBE_MESH = 0, 1
+BODY = {"own": 0, "naive": 1, "butterfly": 2, "best": 3}
+RULE = {"insert": 0, "delete": 1, "fission": 2, "fusion": 3, "relay_in": 4, "relay_out": 5, "pushdown": 6, "pullup": 7,
+        "source": 8}
+
+
+class ja_machine_t(ctypes.Structure):
+    _fields_ = [("fabric", ctypes.c_int32), ("n_sites", ctypes.c_int32), ("hbm_gbs", ctypes.c_double),
+                ("link_gbs", ctypes.c_double), ("double_gbs", ctypes.c_double), ("pcie_gbs", ctypes.c_double)]
+
+
+def _declare():
+    vp, i32, i64, u64, dbl = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64, ctypes.c_double
+    P = ctypes.POINTER
+    sigs = {
+        "ja_machine_preset": [ctypes.c_char_p, P(ja_machine_t)],
+        "ja_exprog_parse": [ctypes.c_char_p, P(vp)],
+        "ja_exprog_clone": [vp, P(vp)],
+        "ja_exprog_format": [vp, ctypes.c_char_p, i64, P(i64)],
+        "ja_exprog_counts": [vp, P(i32), P(i32), P(i32), P(i32), P(i32), P(i32)],
+        "ja_exprog_get_actions": [vp, P(u64), P(i32), P(u64)],
+        "ja_exprog_get_requirements": [vp, P(i32), P(u64), P(i32)],
+        "ja_exprog_get_atoms": [vp, P(i32), P(dbl)],
+        "ja_exprog_num_memberships": [vp, P(i64)],
+        "ja_exprog_bind": [vp, i64],
+        "ja_exprog_membership": [vp, ctypes.c_char_p, P(u64)],
+        "ja_exprog_closure": [vp, P(i64), P(u64), P(i32)],
+        "ja_exprog_check": [vp, P(i32), P(i32)],
+        "ja_exprog_valid_any": [vp, P(i32)],
+        "ja_exprog_simulate": [vp, P(ja_machine_t), P(dbl), P(dbl), P(dbl), P(dbl)],
+        "ja_exprog_body": [vp, i32],
+        "ja_exprog_normalise": [vp],
+        "ja_exprog_rewrite": [vp, i32, i32, i32, u64, u64, P(i32)],
+        "ja_exprog_synthesize": [vp, P(ja_machine_t), i32, i32, P(dbl)],
+        "ja_exprog_place": [vp, P(ja_machine_t), i32, P(dbl)],
+        "ja_exprog_preamble": [i32, P(i64), P(i32), P(i64), P(i32), i32, P(i32), P(i32), i32, i32, P(vp)],
+    }
+    for name, argtypes in sigs.items():
+        fn = getattr(LIB, name)
+        fn.argtypes = argtypes
+        fn.restype = ctypes.c_int
+    LIB.ja_exprog_destroy.argtypes = [vp]
+    LIB.ja_exprog_destroy.restype = None
+
+
+_declare()
+
+
+def ja_machine_preset(name: str) -> ja_machine_t:
+    m = ja_machine_t()
+    _check(LIB.ja_machine_preset(name.encode(), ctypes.byref(m)))
+    return m
+
+
+def ja_exprog_parse(text: str) -> int:
+    h = ctypes.c_void_p()
+    _check(LIB.ja_exprog_parse(text.encode(), ctypes.byref(h)))
+    return h.value
+
+
+def ja_exprog_clone(prog: int) -> int:
+    h = ctypes.c_void_p()
+    _check(LIB.ja_exprog_clone(prog, ctypes.byref(h)))
+    return h.value
+
+
+def ja_exprog_destroy(prog: int):
+    LIB.ja_exprog_destroy(prog)
+
+
+def ja_exprog_format(prog: int) -> str:
+    need = ctypes.c_int64()
+    _check(LIB.ja_exprog_format(prog, None, 0, ctypes.byref(need)))
+    buf = ctypes.create_string_buffer(need.value)
+    _check(LIB.ja_exprog_format(prog, buf, need.value, ctypes.byref(need)))
+    return buf.value.decode()
+
+
+def ja_exprog_counts(prog: int) -> dict:
+    v = [ctypes.c_int32() for _ in range(6)]
+    _check(LIB.ja_exprog_counts(prog, *[ctypes.byref(x) for x in v]))
+    return dict(zip(("gpus", "partitions", "atoms", "out", "actions", "expanded"), (x.value for x in v)))
+
+
+def ja_exprog_get_actions(prog: int):
+    """[(aggregate mask, source site, destination mask)] of the expanded actions."""
+    n = ja_exprog_counts(prog)["expanded"]
+    agg, src, dst = (ctypes.c_uint64 * max(n, 1))(), (ctypes.c_int32 * max(n, 1))(), (ctypes.c_uint64 * max(n, 1))()
+    _check(LIB.ja_exprog_get_actions(prog, agg, src, dst))
+    return [(agg[i], src[i], dst[i]) for i in range(max(n, 0))]
+
+
+def ja_exprog_get_requirements(prog: int):
+    n = ctypes.c_int32()
+    _check(LIB.ja_exprog_get_requirements(prog, ctypes.byref(n), None, None))
+    agg, site = (ctypes.c_uint64 * max(n.value, 1))(), (ctypes.c_int32 * max(n.value, 1))()
+    _check(LIB.ja_exprog_get_requirements(prog, ctypes.byref(n), agg, site))
+    return [(agg[i], site[i]) for i in range(n.value)]
+
+
+def ja_exprog_get_atoms(prog: int):
+    n = ja_exprog_counts(prog)["atoms"]
+    site, gb = (ctypes.c_int32 * max(n, 1))(), (ctypes.c_double * max(n, 1))()
+    _check(LIB.ja_exprog_get_atoms(prog, site, gb))
+    return [(site[i], gb[i]) for i in range(n)]
+
+
+def ja_exprog_num_memberships(prog: int) -> int:
+    n = ctypes.c_int64()
+    _check(LIB.ja_exprog_num_memberships(prog, ctypes.byref(n)))
+    return n.value
+
+
+def ja_exprog_bind(prog: int, index: int):
+    _check(LIB.ja_exprog_bind(prog, index))
+
+
+def ja_exprog_membership(prog: int, partition: str) -> int:
+    m = ctypes.c_uint64()
+    _check(LIB.ja_exprog_membership(prog, partition.encode(), ctypes.byref(m)))
+    return m.value
+
+
+def ja_exprog_closure(prog: int):
+    n = ctypes.c_int64()
+    _check(LIB.ja_exprog_closure(prog, ctypes.byref(n), None, None))
+    agg, site = (ctypes.c_uint64 * max(n.value, 1))(), (ctypes.c_int32 * max(n.value, 1))()
+    _check(LIB.ja_exprog_closure(prog, ctypes.byref(n), agg, site))
+    return [(agg[i], site[i]) for i in range(n.value)]
+
+
+def ja_exprog_check(prog: int):
+    wf, v = ctypes.c_int32(), ctypes.c_int32()
+    _check(LIB.ja_exprog_check(prog, ctypes.byref(wf), ctypes.byref(v)))
+    return bool(wf.value), bool(v.value)
+
+
+def ja_exprog_valid_any(prog: int) -> bool:
+    v = ctypes.c_int32()
+    _check(LIB.ja_exprog_valid_any(prog, ctypes.byref(v)))
+    return bool(v.value)
+
+
+def ja_exprog_simulate(prog: int, machine: ja_machine_t, trace: bool = False):
+    ms = ctypes.c_double()
+    if not trace:
+        _check(LIB.ja_exprog_simulate(prog, ctypes.byref(machine), ctypes.byref(ms), None, None, None))
+        return ms.value
+    n = max(ja_exprog_counts(prog)["expanded"], 1)
+    a, b, c = (ctypes.c_double * n)(), (ctypes.c_double * n)(), (ctypes.c_double * n)()
+    _check(LIB.ja_exprog_simulate(prog, ctypes.byref(machine), ctypes.byref(ms), a, b, c))
+    return ms.value, [(a[i], b[i], c[i]) for i in range(n)]
+
+
+def ja_exprog_body(prog: int, body: str):
+    _check(LIB.ja_exprog_body(prog, BODY[body]))
+
+
+def ja_exprog_normalise(prog: int):
+    _check(LIB.ja_exprog_normalise(prog))
+
+
+def ja_exprog_rewrite(prog: int, rule: str, i: int = 0, j: int = 0, a: int = 0, b: int = 0) -> bool:
+    applied = ctypes.c_int32()
+    _check(LIB.ja_exprog_rewrite(prog, RULE[rule], i, j, a, b, ctypes.byref(applied)))
+    return bool(applied.value)
+
+
+def ja_exprog_synthesize(prog: int, machine: ja_machine_t, depth: int = 4, beam: int = 16) -> float:
+    ms = ctypes.c_double()
+    _check(LIB.ja_exprog_synthesize(prog, ctypes.byref(machine), depth, beam, ctypes.byref(ms)))
+    return ms.value
+
+
+def ja_exprog_place(prog: int, machine: ja_machine_t, body: str = "best") -> float:
+    ms = ctypes.c_double()
+    _check(LIB.ja_exprog_place(prog, ctypes.byref(machine), BODY[body], ctypes.byref(ms)))
+    return ms.value
+
+
+def ja_exprog_preamble(producer_splits, consumer_splits, m: int, copy_site, consumer_specs, width_bytes: int) -> int:
+    rank = len(producer_splits)
+    flat_p = [int(x) for s in producer_splits for x in s]
+    flat_c = [int(x) for s in consumer_splits for x in s]
+    h = ctypes.c_void_p()
+    _check(LIB.ja_exprog_preamble(
+        rank, (ctypes.c_int64 * len(flat_p))(*flat_p), (ctypes.c_int32 * rank)(*[len(s) for s in producer_splits]),
+        (ctypes.c_int64 * len(flat_c))(*flat_c), (ctypes.c_int32 * rank)(*[len(s) for s in consumer_splits]), m,
+        (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
+        (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs), width_bytes,
+        ctypes.byref(h)))
+    return h.value
+
+
+class ExchangeProgram:
+    """A handle with its lifetime; methods are the calls above."""
+
+    def __init__(self, text: str | None = None, handle: int | None = None):
+        self.handle = ja_exprog_parse(text) if handle is None else handle
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            ja_exprog_destroy(self.handle)
+            self.handle = None
+
+    def clone(self):
+        return ExchangeProgram(handle=ja_exprog_clone(self.handle))
+
+    def __str__(self):
+        return ja_exprog_format(self.handle)
