@@ -145,6 +145,24 @@ ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, con
                                const int32_t* copy_site, const int32_t* consumer_specs, int32_t n_specs,
                                int32_t width_bytes, ja_exprog_t** out);
 
+/* ---- an exchange program executed on ONE GPU (Sections 5.2 - 5.3) ----------------------------------------------------
+ * The sites of the program are regions of this GPU's memory.  `partials` is a partial relation (ja.h: rank(dst) + 1, the
+ * copy index in front, cut into its m unit intervals, the other indices tiled as the producer's out(J_k)); `dst` is tiled
+ * as in_k(J), same cell type; copy_site and consumer_specs are those given to ja_exprog_preamble, and `prog` must be a
+ * bound, valid program over exactly the preamble they generate (JA_ERR_INVALID_ARG otherwise).  Steps, all enqueued on
+ * `cuda_stream`: decompose (every resident copy of a producer block is sliced into its atoms, one batched launch), the
+ * actions in a firing order of the program (repeated passes over the expanded actions in body order; an action fires the
+ * first time aggregates at its source partition its aggregate) -- a local aggregation of m >= 2 parts is one launch that
+ * combines them in ascending order of their first atoms in f32 (SUM or MAX) and rounds once to the cell type, a transfer
+ * one device-to-device copy -- and recompose (the aggregated atoms at the site of function spec i are concatenated into
+ * the block it consumes; a block consumed by several specs is written from the lowest one).  At most 16 parts per
+ * aggregation, tensors of rank <= 3.  Scratch memory for the atom buffers comes from the stream-ordered allocator and is
+ * returned to it at the end of the call.  stats (optional, HOST, 4 values): local aggregations launched, transfers,
+ * bytes transferred, scratch bytes. */
+ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                int64_t* stats, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -228,8 +228,9 @@ def requirements(prog: Program):
 
 
 # ------------------------------------------------------------------------- Definition "Closure; validity" (Section 5.4)
-def exact_cover(x: frozenset, available):
-    """A partition of x into members of `available` with the fewest parts (None if there is none)."""
+def exact_cover(x: frozenset, available, order=None):
+    """A partition of x into members of `available` with the fewest parts (None if there is none).  With `order` (atom ->
+    position) the search branches on the first uncovered atom in that order, so the parts come out by their first atoms."""
     cands = [y for y in available if y and y <= x]
     best = [None]
 
@@ -239,7 +240,7 @@ def exact_cover(x: frozenset, available):
         if not rest:
             best[0] = list(parts)
             return
-        pivot = min(rest)
+        pivot = min(rest) if order is None else min(rest, key=order.get)
         for y in cands:
             if pivot in y and y <= rest:
                 parts.append(y)
@@ -737,3 +738,108 @@ def synthesize(prog: Program, mach: dict, depth: int = 6, beam: int = 24):
         if level[0][0] < best[0] * (1.0 - 1e-12):
             best = level[0]
     return best[1], best[0]
+
+
+# ------------------------------------------------------------------ executing a program over tensors (Sections 5.1 - 5.3)
+def schedule(prog: Program):
+    """A firing order of a valid bound program and, per fired action, the parts it aggregates: repeated passes over the
+    expanded actions in body order, an action fires the first time aggregates at its source partition its aggregate
+    (the partition with the fewest parts; candidates tried in ascending order of their atom masks, so the parts come out
+    in ascending order of their first atoms).  Returns [(aggregate, site, destinations, [parts])]."""
+    order = _name_order(prog)
+
+    def mask(y):
+        return sum(1 << order[a] for a in y)
+
+    have = {}
+    for a, (s, _) in prog.atoms.items():
+        have.setdefault(s, set()).add(frozenset([a]))
+    acts = expanded(prog)
+    fired = [False] * len(acts)
+    res = []
+    progress = True
+    while progress:
+        progress = False
+        for i, (x, s, d) in enumerate(acts):
+            if fired[i]:
+                continue
+            cover = exact_cover(x, sorted(have.get(s, ()), key=mask), order)
+            if cover is None:
+                continue
+            fired[i] = True
+            progress = True
+            res.append((x, s, d, cover))
+            have.setdefault(s, set()).add(x)
+            for t in d:
+                have.setdefault(t, set()).add(x)
+    if not all(fired):
+        raise ValueError("the program is not well-formed")
+    return res
+
+
+def execute(prog: Program, values: dict, agg: str = "sum", dtype=None, combine=None):
+    """Runs a valid bound program on tensors: values[atom name] = array.  Every fired action materialises its aggregate at
+    its source -- the (+)-combination of its parts in the order `schedule` gives, in fp64, rounded once to `dtype` -- and
+    copies it to its destinations.  Returns {(aggregate, site): array}.  `combine(parts) -> array` replaces the fp64
+    combination (a test restates the same order in another precision with it)."""
+    import numpy as np
+
+    from . import core
+
+    def default(parts):
+        acc = np.asarray(parts[0], dtype=np.float64).copy()
+        for p in parts[1:]:
+            acc = acc + p if agg == "sum" else np.maximum(acc, p)
+        return core.round_to(acc, dtype) if dtype in ("f32", "bf16", "f16") else acc
+
+    if agg not in ("sum", "max"):
+        raise ValueError(agg)
+    combine = combine or default
+    store = {(frozenset([a]), s): values[a] for a, (s, _) in prog.atoms.items()}
+    for x, s, d, cover in schedule(prog):
+        if len(cover) >= 2:
+            store[(x, s)] = combine([store[(y, s)] for y in cover])
+        for t in d:
+            store.setdefault((x, t), store[(x, s)])
+    return store
+
+
+def exchange(prog: Program, partials, producer_splits, consumer_splits, consumer_specs, agg="sum", dtype=None,
+             combine=None, name=None):
+    """Section 5.3 end to end for one input of op: decompose (every resident copy of a producer block is sliced into its
+    atoms), the exchange program, recompose (the aggregated atoms delivered to the GPU of function spec i are concatenated
+    into the block it consumes).  `partials` is the dense tensor P[c, x...] whose copy c of producer block b is the slice
+    of P[c] over that block; `prog` a valid bound program over the preamble `preamble(...)` generates for these tilings.
+    Returns the dense tensor assembled from the blocks of all function specs (for a block consumed by several specs, the
+    lowest one's) -- NaN where no spec consumes."""
+    import numpy as np
+
+    name = name or (lambda j, c: "a%d_%d" % (j, c))
+    P = np.asarray(partials)
+    m = P.shape[0]
+    rank = P.ndim - 1
+    over = [sorted(set(producer_splits[d]) | set(consumer_splits[d])) for d in range(rank)]
+    cells = list(itertools.product(*[range(len(o) - 1) for o in over]))
+    boxes = [tuple(slice(over[d][cell[d]], over[d][cell[d] + 1]) for d in range(rank)) for cell in cells]
+    values = {name(j, c): P[(c,) + boxes[j]] for j in range(len(cells)) for c in range(m) if name(j, c) in prog.atoms}
+    store = execute(prog, values, agg, dtype, combine)
+    out = np.full(P.shape[1:], np.nan)
+    done = set()
+
+    def cblock(j):
+        k = 0
+        for d in range(rank):
+            lo = over[d][cells[j][d]]
+            idx = max(i for i in range(len(consumer_splits[d]) - 1) if consumer_splits[d][i] <= lo)
+            k = k * (len(consumer_splits[d]) - 1) + idx
+        return k
+
+    for i, blk in enumerate(consumer_specs):
+        site = prog.partitions["S%d" % (i + 1)]["members"][0]
+        for j in range(len(cells)):
+            if cblock(j) != blk or j in done:
+                continue
+            x = frozenset(name(j, c) for c in range(m))
+            out[boxes[j]] = store[(x, site)]
+            done.add(j)
+    return out

@@ -469,6 +469,25 @@ struct Cover {
             if ((y & pivot) && (y & ~rest) == 0) rec(rest & ~y, parts + 1);
     }
 };
+// the same search, keeping the parts: candidates in the order given (callers pass them ascending), so the parts come out in
+// ascending order of their first atoms and the first minimal partition found wins
+struct CoverParts {
+    std::vector<uint64_t> cands, cur, best;
+    void rec(uint64_t rest) {
+        if (!best.empty() && cur.size() >= best.size()) return;
+        if (!rest) {
+            best = cur;
+            return;
+        }
+        const uint64_t pivot = rest & (~rest + 1);
+        for (uint64_t y : cands)
+            if ((y & pivot) && (y & ~rest) == 0) {
+                cur.push_back(y);
+                rec(rest & ~y);
+                cur.pop_back();
+            }
+    }
+};
 int exact_cover(uint64_t x, const std::vector<uint64_t>& avail) {
     Cover c;
     for (uint64_t y : avail)
@@ -1267,22 +1286,31 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
     return JA_OK;
 }
 
-extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, const int32_t* n_producer_splits,
-                                          const int64_t* consumer_splits, const int32_t* n_consumer_splits, int32_t m,
-                                          const int32_t* copy_site, const int32_t* consumer_specs, int32_t n_specs,
-                                          int32_t width_bytes, ja_exprog_t** out) {
-    if (rank < 1 || rank > 8 || !producer_splits || !n_producer_splits || !consumer_splits || !n_consumer_splits || m < 1 ||
-        !copy_site || !consumer_specs || n_specs < 1 || width_bytes < 1 || !out)
-        return ja_fail(JA_ERR_INVALID_ARG, "bad argument");
-    std::vector<std::vector<int64_t>> ps(rank), cs(rank), ov(rank);
-    const int64_t *pp = producer_splits, *cp = consumer_splits;
+namespace {
+
+// the overlay of a producer's and a consumer's tiling of one tensor and the preamble built on it (Section 5.3)
+struct OverlayCell {
+    int64_t j, pb, cb;                 // atom number (row-major over the overlay), flat producer block, flat consumer block
+    int64_t lo[8], hi[8];              // its box
+    double gb;
+};
+struct Overlay {
+    int rank = 0;
+    std::vector<std::vector<int64_t>> ps, cs, ov;
+    std::vector<OverlayCell> cells;
+    std::vector<std::pair<int64_t, int>> atom_jc;   // per ExProg atom (declaration order): (atom number, copy)
+};
+
+ja_status_t make_preamble(int rank, const std::vector<std::vector<int64_t>>& ps, const std::vector<std::vector<int64_t>>& cs,
+                          int m, const int32_t* copy_site, const int32_t* consumer_specs, int n_specs, int width_bytes,
+                          Prog* p, Overlay* o) {
+    o->rank = rank;
+    o->ps = ps;
+    o->cs = cs;
+    o->ov.assign(rank, {});
     int64_t n_pblocks = 1, n_cblocks = 1, n_cells = 1;
     for (int d = 0; d < rank; ++d) {
-        if (n_producer_splits[d] < 2 || n_consumer_splits[d] < 2) return ja_fail(JA_ERR_TILING, "index %d: at least two split points", d);
-        ps[d].assign(pp, pp + n_producer_splits[d]);
-        cs[d].assign(cp, cp + n_consumer_splits[d]);
-        pp += n_producer_splits[d];
-        cp += n_consumer_splits[d];
+        if (ps[d].size() < 2 || cs[d].size() < 2) return ja_fail(JA_ERR_TILING, "index %d: at least two split points", d);
         for (const auto* v : {&ps[d], &cs[d]}) {
             if ((*v)[0] != 0) return ja_fail(JA_ERR_TILING, "index %d: split points start at 0", d);
             for (size_t i = 1; i < v->size(); ++i)
@@ -1291,18 +1319,19 @@ extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_
         if (ps[d].back() != cs[d].back()) return ja_fail(JA_ERR_SHAPE, "index %d: the two tilings differ in extent", d);
         std::set<int64_t> u(ps[d].begin(), ps[d].end());
         u.insert(cs[d].begin(), cs[d].end());
-        ov[d].assign(u.begin(), u.end());
+        o->ov[d].assign(u.begin(), u.end());
         n_pblocks *= (int64_t)ps[d].size() - 1;
         n_cblocks *= (int64_t)cs[d].size() - 1;
-        n_cells *= (int64_t)ov[d].size() - 1;
+        n_cells *= (int64_t)o->ov[d].size() - 1;
     }
     if (n_cells * m > 64) return ja_fail(JA_ERR_INVALID_ARG, "%lld atoms x %d copies: at most 64 ExProg atoms", (long long)n_cells, m);
-    Prog* p = new Prog();
     std::set<int> g;
     for (int64_t i = 0; i < n_pblocks * m; ++i) g.insert(copy_site[i]);
     for (int i = 0; i < n_specs; ++i) g.insert(i);
     p->gpus.assign(g.begin(), g.end());
     for (int i = 0; i < n_specs; ++i) {
+        if (consumer_specs[i] < 0 || consumer_specs[i] >= n_cblocks)
+            return ja_fail(JA_ERR_INVALID_ARG, "function spec %d names block %d of %lld", i, consumer_specs[i], (long long)n_cblocks);
         ExPartition q;
         q.name = "S" + std::to_string(i + 1);
         q.size = 1;
@@ -1313,29 +1342,29 @@ extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_
         while (!(s[i] <= lo && lo < s[i + 1])) ++i;
         return i;
     };
-    struct Cell {
-        int64_t j, pb, cb;
-        double gb;
-    };
-    std::vector<Cell> cells;
     std::vector<int> c(rank, 0);
     for (int64_t j = 0; j < n_cells; ++j) {
-        int64_t card = 1, pb = 0, cb = 0;
+        OverlayCell ce;
+        ce.j = j;
+        ce.pb = ce.cb = 0;
+        int64_t card = 1;
         for (int d = 0; d < rank; ++d) {
-            const int64_t lo = ov[d][c[d]];
-            card *= ov[d][c[d] + 1] - lo;
-            pb = pb * ((int64_t)ps[d].size() - 1) + owner(ps[d], lo);
-            cb = cb * ((int64_t)cs[d].size() - 1) + owner(cs[d], lo);
+            ce.lo[d] = o->ov[d][c[d]];
+            ce.hi[d] = o->ov[d][c[d] + 1];
+            card *= ce.hi[d] - ce.lo[d];
+            ce.pb = ce.pb * ((int64_t)ps[d].size() - 1) + owner(ps[d], ce.lo[d]);
+            ce.cb = ce.cb * ((int64_t)cs[d].size() - 1) + owner(cs[d], ce.lo[d]);
         }
-        cells.push_back({j, pb, cb, (double)(card * width_bytes) / 1e9});
+        ce.gb = (double)(card * width_bytes) / 1e9;
+        o->cells.push_back(ce);
         for (int d = rank - 1; d >= 0; --d) {
-            if (++c[d] < (int)ov[d].size() - 1) break;
+            if (++c[d] < (int)o->ov[d].size() - 1) break;
             c[d] = 0;
         }
     }
     // IN: by site, then atom, then copy
     std::vector<std::tuple<int, int64_t, int, double>> entries;
-    for (const Cell& ce : cells)
+    for (const OverlayCell& ce : o->cells)
         for (int k = 0; k < m; ++k) entries.push_back(std::make_tuple(copy_site[ce.pb * m + k], ce.j, k, ce.gb));
     std::sort(entries.begin(), entries.end());
     std::map<std::pair<int64_t, int>, int> index;
@@ -1345,32 +1374,256 @@ extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_
         a.site = std::get<0>(e);
         a.gb = std::get<3>(e);
         index[{std::get<1>(e), std::get<2>(e)}] = (int)p->atoms.size();
+        o->atom_jc.push_back({std::get<1>(e), std::get<2>(e)});
         p->atoms.push_back(a);
     }
-    for (const Cell& ce : cells) {
+    for (const OverlayCell& ce : o->cells) {
         uint64_t x = 0;
         for (int k = 0; k < m; ++k) x |= 1ull << index[{ce.j, k}];
-        for (int i = 0; i < n_specs; ++i) {
-            if (consumer_specs[i] < 0 || consumer_specs[i] >= n_cblocks) {
-                delete p;
-                return ja_fail(JA_ERR_INVALID_ARG, "function spec %d names block %d of %lld", i, consumer_specs[i], (long long)n_cblocks);
-            }
+        for (int i = 0; i < n_specs; ++i)
             if (consumer_specs[i] == ce.cb) {
                 ExTarget t;
                 t.part = i;
                 p->out.push_back({x, t});
             }
-        }
     }
-    if ((int)p->gpus.size() != n_specs) {
-        delete p;
+    if ((int)p->gpus.size() != n_specs)
         return ja_fail(JA_ERR_INVALID_ARG, "one function spec of op per GPU: the partitions of size one must cover the GPUs");
+    return check_static(*p);
+}
+
+}  // namespace
+
+extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, const int32_t* n_producer_splits,
+                                          const int64_t* consumer_splits, const int32_t* n_consumer_splits, int32_t m,
+                                          const int32_t* copy_site, const int32_t* consumer_specs, int32_t n_specs,
+                                          int32_t width_bytes, ja_exprog_t** out) {
+    if (rank < 1 || rank > 8 || !producer_splits || !n_producer_splits || !consumer_splits || !n_consumer_splits || m < 1 ||
+        !copy_site || !consumer_specs || n_specs < 1 || width_bytes < 1 || !out)
+        return ja_fail(JA_ERR_INVALID_ARG, "bad argument");
+    std::vector<std::vector<int64_t>> ps(rank), cs(rank);
+    const int64_t *pp = producer_splits, *cp = consumer_splits;
+    for (int d = 0; d < rank; ++d) {
+        if (n_producer_splits[d] < 2 || n_consumer_splits[d] < 2) return ja_fail(JA_ERR_TILING, "index %d: at least two split points", d);
+        ps[d].assign(pp, pp + n_producer_splits[d]);
+        cs[d].assign(cp, cp + n_consumer_splits[d]);
+        pp += n_producer_splits[d];
+        cp += n_consumer_splits[d];
     }
-    ja_status_t st = check_static(*p);
+    Prog* p = new Prog();
+    Overlay o;
+    ja_status_t st = make_preamble(rank, ps, cs, m, copy_site, consumer_specs, n_specs, width_bytes, p, &o);
     if (st != JA_OK) {
         delete p;
         return st;
     }
     *out = p;
+    return JA_OK;
+}
+
+// ---------------------------------------------------------------------------------- execution on one GPU (Section 5.3)
+// The sites of the program are regions of this GPU's memory; a transfer is a device-to-device copy (on a machine with
+// several GPUs it would be a peer copy), a local aggregation one launch of the combine kernel, decompose and recompose
+// one batched box-copy launch each. Actions are issued on one stream in a firing order of the program.
+extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                           const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                           int64_t* stats, void* cuda_stream) {
+    ja_status_t st = need_bound(prog);
+    if (st != JA_OK) return st;
+    if (!partials || !dst || !copy_site || !consumer_specs || n_specs < 1) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    const int rank = dst->rank;
+    if (partials->rank != rank + 1) return ja_fail(JA_ERR_SHAPE, "a partial relation has the copy index in front: rank %d expected, got %d", rank + 1, partials->rank);
+    if (partials->nblk[0] != partials->extent[0]) return ja_fail(JA_ERR_TILING, "the copy index of a partial relation must be cut into unit intervals");
+    for (int d = 0; d < rank; ++d)
+        if (partials->extent[d + 1] != dst->extent[d]) return ja_fail(JA_ERR_SHAPE, "extent of dimension %d differs", d);
+    if (partials->dtype != dst->dtype) return ja_fail(JA_ERR_DTYPE, "the exchange moves and aggregates atoms in the partial relation's cell type: the consumer relation must have it too");
+    if (partials->base == dst->base) return ja_fail(JA_ERR_INVALID_ARG, "the consumer relation aliases the partial relation");
+    const int m = (int)partials->extent[0];
+    if (agg != JA_AGG_SUM && agg != JA_AGG_MAX && !(agg == JA_AGG_NONE && m == 1))
+        return ja_fail(JA_ERR_INVALID_ARG, "%d copies of every atom need SUM or MAX aggregation", m);
+    // the preamble these relations generate must be the program's
+    std::vector<std::vector<int64_t>> ps(rank), cs(rank);
+    for (int d = 0; d < rank; ++d) {
+        ps[d] = partials->splits[d + 1];
+        cs[d] = dst->splits[d];
+    }
+    Prog pre;
+    Overlay ov;
+    if ((st = make_preamble(rank, ps, cs, m, copy_site, consumer_specs, n_specs, partials->esize, &pre, &ov)) != JA_OK) return st;
+    bool same = pre.gpus == prog->gpus && pre.atoms.size() == prog->atoms.size() && pre.out.size() == prog->out.size() &&
+                pre.parts.size() == prog->parts.size();
+    for (size_t i = 0; same && i < pre.atoms.size(); ++i)
+        same = pre.atoms[i].name == prog->atoms[i].name && pre.atoms[i].site == prog->atoms[i].site && pre.atoms[i].gb == prog->atoms[i].gb;
+    for (size_t i = 0; same && i < pre.out.size(); ++i) same = pre.out[i].first == prog->out[i].first && pre.out[i].second == prog->out[i].second;
+    for (size_t i = 0; same && i < pre.parts.size(); ++i) same = pre.parts[i].name == prog->parts[i].name && prog->parts[i].members.size() == 1;
+    if (!same) return ja_fail(JA_ERR_INVALID_ARG, "the program's preamble is not the one these relations, copy sites and function specs generate");
+    if (!valid_bound(*prog)) return ja_fail(JA_ERR_INVALID_ARG, "the program is not valid (Definition \"Closure; validity\")");
+
+    // firing order and the parts of every aggregation: repeated passes over the expanded actions in body order
+    std::vector<Flat> acts;
+    expand(*prog, &acts);
+    struct Fired {
+        int act;
+        std::vector<uint64_t> parts;
+    };
+    std::vector<Fired> order;
+    {
+        std::map<int, std::set<uint64_t>> have;
+        for (size_t i = 0; i < prog->atoms.size(); ++i) have[prog->atoms[i].site].insert(1ull << i);
+        std::vector<bool> fired(acts.size(), false);
+        bool progress = true;
+        while (progress) {
+            progress = false;
+            for (size_t i = 0; i < acts.size(); ++i) {
+                if (fired[i]) continue;
+                CoverParts cp;
+                for (uint64_t y : have[acts[i].site])
+                    if ((y & ~acts[i].agg) == 0) cp.cands.push_back(y);
+                cp.rec(acts[i].agg);
+                if (cp.best.empty()) continue;
+                fired[i] = true;
+                progress = true;
+                order.push_back({(int)i, cp.best});
+                have[acts[i].site].insert(acts[i].agg);
+                for (int d : acts[i].dests) have[d].insert(acts[i].agg);
+            }
+        }
+    }
+    // buffers: one per (aggregate, site) materialisation
+    auto atom_bytes = [&](uint64_t agg_mask) {
+        const int a = __builtin_ctzll(agg_mask);
+        const OverlayCell& ce = ov.cells[ov.atom_jc[a].first];
+        int64_t cells = 1;
+        for (int d = 0; d < rank; ++d) cells *= ce.hi[d] - ce.lo[d];
+        return cells * partials->esize;
+    };
+    std::map<std::pair<int, uint64_t>, int64_t> buf;     // (site, aggregate) -> offset in the scratch allocation
+    int64_t scratch = 0;
+    auto alloc = [&](int site, uint64_t x) {
+        auto key = std::make_pair(site, x);
+        if (buf.count(key)) return;
+        buf[key] = scratch;
+        scratch += (atom_bytes(x) + 255) / 256 * 256;
+    };
+    for (size_t a = 0; a < prog->atoms.size(); ++a) alloc(prog->atoms[a].site, 1ull << a);
+    int64_t n_aggregations = 0, n_transfers = 0, transfer_bytes = 0;
+    for (const Fired& f : order) {
+        const Flat& a = acts[f.act];
+        if (f.parts.size() > JA_EXCHANGE_MAX_PARTS)
+            return ja_fail(JA_ERR_UNSUPPORTED, "an aggregation of %d parts (at most %d)", (int)f.parts.size(), JA_EXCHANGE_MAX_PARTS);
+        alloc(a.site, a.agg);
+        for (int d : a.dests) alloc(d, a.agg);
+    }
+    // decompose and recompose tables
+    const int64_t ntrail = partials->nblocks / m;
+    std::vector<JaBoxCopy> boxes;
+    bool vec_in = true, vec_out = true;
+    int64_t max_in = 0, max_out = 0;
+    auto box_of = [&](const OverlayCell& ce, const std::vector<std::vector<int64_t>>& tiling, int64_t blk, int64_t blk_off, bool from_block, int64_t buf_off) {
+        // the block's extents and the box's offset inside it, padded to three dimensions in front
+        int64_t bext[3] = {1, 1, 1}, off[3] = {0, 0, 0}, n[3] = {1, 1, 1};
+        int64_t rem = blk;
+        for (int d = rank - 1; d >= 0; --d) {
+            const int64_t nb = (int64_t)tiling[d].size() - 1, k = rem % nb;
+            rem /= nb;
+            bext[3 - rank + d] = tiling[d][k + 1] - tiling[d][k];
+            off[3 - rank + d] = ce.lo[d] - tiling[d][k];
+            n[3 - rank + d] = ce.hi[d] - ce.lo[d];
+        }
+        const int64_t es = partials->esize;
+        JaBoxCopy b;
+        b.n0 = n[0];
+        b.n1 = n[1];
+        b.run_bytes = n[2] * es;
+        const int64_t blk_pitch1 = bext[2] * es, blk_pitch0 = bext[1] * blk_pitch1;
+        const int64_t in_blk = blk_off + off[0] * blk_pitch0 + off[1] * blk_pitch1 + off[2] * es;
+        const int64_t dense1 = n[2] * es, dense0 = n[1] * dense1;
+        if (from_block) {
+            b.src_off = in_blk; b.src_pitch0 = blk_pitch0; b.src_pitch1 = blk_pitch1;
+            b.dst_off = buf_off; b.dst_pitch0 = dense0; b.dst_pitch1 = dense1;
+        } else {
+            b.dst_off = in_blk; b.dst_pitch0 = blk_pitch0; b.dst_pitch1 = blk_pitch1;
+            b.src_off = buf_off; b.src_pitch0 = dense0; b.src_pitch1 = dense1;
+        }
+        return b;
+    };
+    auto aligned16 = [](const JaBoxCopy& b) {
+        return ((b.src_off | b.dst_off | b.src_pitch0 | b.src_pitch1 | b.dst_pitch0 | b.dst_pitch1 | b.run_bytes) & 15) == 0;
+    };
+    if (rank > 3) return ja_fail(JA_ERR_UNSUPPORTED, "tensors of rank above 3");
+    for (size_t a = 0; a < prog->atoms.size(); ++a) {
+        const OverlayCell& ce = ov.cells[ov.atom_jc[a].first];
+        const int c = ov.atom_jc[a].second;
+        const JaBoxCopy b = box_of(ce, ps, ce.pb, partials->blk_off[c * ntrail + ce.pb], true, buf[{prog->atoms[a].site, 1ull << a}]);
+        vec_in = vec_in && aligned16(b);
+        max_in = std::max(max_in, b.n0 * b.n1 * b.run_bytes);
+        boxes.push_back(b);
+    }
+    const int n_in = (int)boxes.size();
+    std::set<int64_t> done;
+    for (int i = 0; i < n_specs; ++i) {
+        const int site = prog->parts[i].members[0];
+        for (const OverlayCell& ce : ov.cells) {
+            if (ce.cb != consumer_specs[i] || done.count(ce.j)) continue;
+            done.insert(ce.j);
+            uint64_t x = 0;
+            for (size_t a = 0; a < prog->atoms.size(); ++a)
+                if (ov.atom_jc[a].first == ce.j) x |= 1ull << a;
+            auto it = buf.find({site, x});
+            if (it == buf.end()) return ja_fail(JA_ERR_INVALID_ARG, "internal: a required aggregate was never materialised");
+            const JaBoxCopy b = box_of(ce, cs, ce.cb, dst->blk_off[ce.cb], false, it->second);
+            vec_out = vec_out && aligned16(b);
+            max_out = std::max(max_out, b.n0 * b.n1 * b.run_bytes);
+            boxes.push_back(b);
+        }
+    }
+    const int n_out = (int)boxes.size() - n_in;
+    const int64_t table_bytes = (int64_t)boxes.size() * (int64_t)sizeof(JaBoxCopy);
+    const int64_t table_off = scratch;
+    scratch += (table_bytes + 255) / 256 * 256;
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* pool = nullptr;
+    JA_CUDA(cudaMallocAsync((void**)&pool, (size_t)scratch, stream));
+    ja_status_t rc = JA_OK;
+    do {
+        if (cudaMemcpyAsync(pool + table_off, boxes.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+            rc = ja_fail(JA_ERR_CUDA, "copying the box tables failed");
+            break;
+        }
+        const JaBoxCopy* d_boxes = (const JaBoxCopy*)(pool + table_off);
+        if ((rc = ja_launch_box_copies((const char*)partials->base, pool, d_boxes, n_in, max_in, vec_in, partials->esize, stream)) != JA_OK) break;
+        for (const Fired& f : order) {
+            const Flat& a = acts[f.act];
+            char* here = pool + buf[{a.site, a.agg}];
+            if (f.parts.size() >= 2) {
+                const void* parts[JA_EXCHANGE_MAX_PARTS];
+                for (size_t k = 0; k < f.parts.size(); ++k) parts[k] = pool + buf[{a.site, f.parts[k]}];
+                if ((rc = ja_launch_exchange_combine(parts, (int)f.parts.size(), here, atom_bytes(a.agg), partials->dtype, agg, stream)) != JA_OK) break;
+                ++n_aggregations;
+            }
+            for (int d : a.dests) {
+                char* there = pool + buf[{d, a.agg}];
+                if (there == here) continue;
+                if (cudaMemcpyAsync(there, here, (size_t)atom_bytes(a.agg), cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+                    rc = ja_fail(JA_ERR_CUDA, "a transfer failed");
+                    break;
+                }
+                ++n_transfers;
+                transfer_bytes += atom_bytes(a.agg);
+            }
+            if (rc != JA_OK) break;
+        }
+        if (rc != JA_OK) break;
+        rc = ja_launch_box_copies(pool, (char*)dst->base, d_boxes + n_in, n_out, max_out, vec_out, partials->esize, stream);
+    } while (false);
+    cudaFreeAsync(pool, stream);
+    if (rc != JA_OK) return rc;
+    if (stats) {
+        stats[0] = n_aggregations;
+        stats[1] = n_transfers;
+        stats[2] = transfer_bytes;
+        stats[3] = scratch;
+    }
     return JA_OK;
 }

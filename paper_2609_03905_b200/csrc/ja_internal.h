@@ -208,4 +208,16 @@ ja_status_t ja_launch_attention_tc(const AttnArgs& a, cudaStream_t st, bool* lau
 // the online-softmax aggregation of m partial attention results (O_c, lse_c) into (O, lse); l may be nullptr
 ja_status_t ja_launch_attention_combine(const ja_relation* const* op, const ja_relation* const* lp, int m, const ja_relation* o,
                                         const ja_relation* l, cudaStream_t st);
+// an exchange program on one GPU: batched copies of boxes between relation blocks and dense atom buffers (decompose / recompose),
+// and the local aggregation of an action -- out = parts[0] (+) parts[1] (+) ... in that order, f32, one rounding
+struct JaBoxCopy {
+    int64_t src_off, dst_off;                // bytes from the two base pointers
+    int64_t n0, n1, run_bytes;               // n0 x n1 runs of run_bytes contiguous bytes
+    int64_t src_pitch0, src_pitch1, dst_pitch0, dst_pitch1;   // bytes between consecutive indices of the two outer dimensions
+};
+#define JA_EXCHANGE_MAX_PARTS 16
+ja_status_t ja_launch_box_copies(const char* src, char* dst, const JaBoxCopy* d_boxes, int n_boxes, int64_t max_box_bytes,
+                                 bool vec16, int esize, cudaStream_t st);
+ja_status_t ja_launch_exchange_combine(const void* const* parts, int n_parts, void* out, int64_t bytes, ja_dtype_t dt,
+                                       ja_agg_t agg, cudaStream_t st);
 void ja_attention_reset_queues();   // zeroes the work counters of the persistent attention kernel (after a device-side failure)

@@ -43,6 +43,7 @@ def _declare():
         "ja_exprog_synthesize": [vp, P(ja_machine_t), i32, i32, P(dbl)],
         "ja_exprog_place": [vp, P(ja_machine_t), i32, P(dbl)],
         "ja_exprog_preamble": [i32, P(i64), P(i32), P(i64), P(i32), i32, P(i32), P(i32), i32, i32, P(vp)],
+        "ja_exchange_execute": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i64), vp],
     }
     for name, argtypes in sigs.items():
         fn = getattr(LIB, name)
@@ -201,6 +202,16 @@ def ja_exprog_preamble(producer_splits, consumer_splits, m: int, copy_site, cons
     return h.value
 
 
+def ja_exchange_execute(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int, stream: int = 0) -> dict:
+    """Relation handles as in binding.ja_repartition_agg; returns the call's statistics."""
+    from .binding import AGG
+    stats = (ctypes.c_int64 * 4)()
+    _check(LIB.ja_exchange_execute(prog, partials, (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
+                                   (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs),
+                                   AGG[agg] if isinstance(agg, str) else int(agg), dst, stats, stream))
+    return {"aggregations": stats[0], "transfers": stats[1], "transfer_bytes": stats[2], "scratch_bytes": stats[3]}
+
+
 class ExchangeProgram:
     """A handle with its lifetime; methods are the calls above."""
 
@@ -217,3 +228,9 @@ class ExchangeProgram:
 
     def __str__(self):
         return ja_exprog_format(self.handle)
+
+    def execute(self, partials, copy_site, consumer_specs, agg, dst, stream=None):
+        """partials, dst: relations.Relation objects (payloads on the GPU); enqueues on torch's current stream by default."""
+        import torch
+        st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        return ja_exchange_execute(self.handle, partials.handle, copy_site, consumer_specs, agg, dst.handle, st)

@@ -1,0 +1,139 @@
+"""An exchange program executed on one GPU (ja_exchange_execute) against the oracle's executor (oracle/exprog.py) on the
+same seeded partial relations: decompose, the program's aggregations and transfers, recompose.  MAX and programs whose
+aggregations have two parts of f32 cells are bit-exact; sums are compared with the same firing order restated in f32
+(bit-exact) and with the oracle (tolerance)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import blocked, core
+from oracle import exprog as E
+from paper_2609_03905_b200 import exprog as X
+from paper_2609_03905_b200.binding import JaError
+import synth_inputs as si
+from gpu_util import TOL, check_status, download, download_bits, empty_like_tiling, relfro, upload
+
+pytestmark = pytest.mark.gpu
+BF, F16, F32 = torch.bfloat16, torch.float16, torch.float32
+ORC_DT = {BF: "bf16", F16: "f16", F32: "f32"}
+ES = blocked.equal_splits
+G = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "exprog_examples.json")))
+
+CASES = {
+    # the preamble example of Section 5.3: 2 copies, four GPUs
+    "preamble": dict(ext=[256, 256], ps=[[0, 128, 256], [0, 256]], cs=[[0, 64, 128, 192, 256], [0, 256]], m=2,
+                     copy_site=[0, 1, 2, 3], specs=[0, 1, 2, 3]),
+    # an all-to-all: every GPU holds a copy of every producer block's share, consumer cut the other way
+    "crossed": dict(ext=[192, 160], ps=[ES(192, 2), ES(160, 1)], cs=[ES(192, 1), ES(160, 4)], m=4,
+                    copy_site=[0, 1, 2, 3, 3, 2, 1, 0], specs=[0, 1, 2, 3]),
+    # replication: two function specs consume the same block; odd sizes (scalar accesses); rank 3
+    "replicated": dict(ext=[6, 33, 10], ps=[ES(6, 2), [0, 10, 33], [0, 10]], cs=[ES(6, 1), [0, 33], [0, 3, 10]], m=3,
+                       copy_site=[0, 1, 2, 2, 0, 1, 1, 2, 0, 0, 2, 1], specs=[0, 1, 1]),
+    # an all-reduce shape: every GPU holds one copy of the one block and every GPU consumes it
+    "allreduce": dict(ext=[128, 64], ps=[[0, 128], [0, 64]], cs=[[0, 128], [0, 64]], m=4, copy_site=[0, 1, 2, 3],
+                      specs=[0, 0, 0, 0]),
+}
+
+
+def build(case, body, machine="hgx_b200"):
+    c = CASES[case]
+    pre_o = E.preamble(c["ext"], c["ps"], {(b, k): c["copy_site"][b * c["m"] + k] for b in range(len(c["copy_site"]) // c["m"]) for k in range(c["m"])},
+                       c["cs"], c["specs"], 2)
+    h = X.ExchangeProgram(handle=X.ja_exprog_preamble(c["ps"], c["cs"], c["m"], c["copy_site"], c["specs"], 2))
+    m = X.ja_machine_preset(machine)
+    if body == "synth":
+        X.ja_exprog_place(h.handle, m, "best")
+        X.ja_exprog_synthesize(h.handle, m, 2, 6)
+    else:
+        X.ja_exprog_place(h.handle, m, body)
+    return h, E.parse(str(h))        # the oracle executes the library's program, read from its text
+
+
+@pytest.mark.parametrize("dtype", [BF, F16, F32])
+@pytest.mark.parametrize("agg", ["sum", "max"])
+@pytest.mark.parametrize("body", ["naive", "butterfly", "synth"])
+@pytest.mark.parametrize("case", list(CASES))
+def test_exchange_program_on_one_gpu(case, body, agg, dtype):
+    c = CASES[case]
+    m = c["m"]
+    es = 4 if dtype == F32 else 2
+    # the preamble's sizes depend on the cell width: rebuild for this dtype
+    h = X.ExchangeProgram(handle=X.ja_exprog_preamble(c["ps"], c["cs"], m, c["copy_site"], c["specs"], es))
+    mach = X.ja_machine_preset("hgx_b200")
+    X.ja_exprog_place(h.handle, mach, "best" if body == "synth" else body)
+    if body == "synth":
+        X.ja_exprog_synthesize(h.handle, mach, 2, 6)
+    assert X.ja_exprog_check(h.handle) == (True, True)
+    q = E.parse(str(h))
+    assert E.valid_bound(q)
+    P = si.normal([m] + c["ext"], 0.0, 1.0, dtype, 5, 17)
+    rP = upload(P, blocked.partial_splits(m, c["ps"]))
+    rD = empty_like_tiling(c["ext"], c["cs"], dtype, fill=float("nan"))
+    before = download_bits(rP).copy()
+    stats = h.execute(rP, c["copy_site"], c["specs"], agg, rD)
+    got = download(rD)
+    check_status()
+    assert np.array_equal(download_bits(rP), before)                      # partials are borrowed, unchanged
+    P64 = si.to_f64(P)
+    sched = E.schedule(q)
+    assert stats["aggregations"] == sum(len(cover) >= 2 for _, _, _, cover in sched)
+    assert stats["transfers"] == sum(len(d) for _, _, d, _ in sched)
+    want = E.exchange(q, P64, c["ps"], c["cs"], c["specs"], agg, ORC_DT[dtype])
+    consumed = ~np.isnan(want)
+    assert consumed.all()                                                  # every block of these cases is consumed
+    if agg == "max":
+        assert np.array_equal(got, want)                                   # bit-exact
+        assert np.array_equal(got, blocked.aggregate_repartition(P64, c["ps"], c["cs"], "max", ORC_DT[dtype]))
+        return
+
+    def f32_sum(parts):                                                    # the kernel's arithmetic: f32, the order given, one rounding
+        acc = np.asarray(parts[0], dtype=np.float64).astype(np.float32)
+        for p in parts[1:]:
+            acc = acc + np.asarray(p, dtype=np.float64).astype(np.float32)
+        return core.round_to(acc.astype(np.float64), ORC_DT[dtype])
+
+    same_order = E.exchange(q, P64, c["ps"], c["cs"], c["specs"], "sum", ORC_DT[dtype], combine=f32_sum)
+    assert np.array_equal(got, same_order)
+    assert relfro(got, want) <= (1e-6 if dtype == F32 else 1e-3)
+    # whatever the program, the result is the aggregate of all m copies (intermediate aggregates are rounded to the cell type)
+    assert relfro(got, blocked.aggregate_repartition(P64, c["ps"], c["cs"], "sum", ORC_DT[dtype])) <= TOL[dtype]
+
+
+def test_the_doubling_body_is_what_runs_for_the_allreduce_shape():
+    h, q = build("allreduce", "best", "dgx_h100")
+    acts = X.ja_exprog_get_actions(h.handle)
+    assert sum(1 for a, s, d in acts if d) == 8 and max(bin(a).count("1") for a, s, d in acts if d) == 2   # two rounds of four sends
+    hn, _ = build("allreduce", "naive", "dgx_h100")
+    assert X.ja_exprog_simulate(h.handle, X.ja_machine_preset("dgx_h100")) < X.ja_exprog_simulate(hn.handle, X.ja_machine_preset("dgx_h100"))
+
+
+def test_exchange_refusals():
+    c = CASES["preamble"]
+    h, q = build("preamble", "naive")
+    P = si.normal([2] + c["ext"], 0.0, 1.0, BF, 1, 2)
+    rP = upload(P, blocked.partial_splits(2, c["ps"]))
+    rD = empty_like_tiling(c["ext"], c["cs"], BF)
+    with pytest.raises(JaError) as e:                      # other copy sites than the program's preamble
+        h.execute(rP, [1, 0, 2, 3], c["specs"], "sum", rD)
+    assert e.value.status_name == "JA_ERR_INVALID_ARG"
+    with pytest.raises(JaError) as e:                      # another consumer tiling
+        h.execute(rP, c["copy_site"], c["specs"], "sum", empty_like_tiling(c["ext"], [ES(256, 2), [0, 256]], BF))
+    assert e.value.status_name == "JA_ERR_INVALID_ARG"
+    with pytest.raises(JaError) as e:
+        h.execute(rP, c["copy_site"], c["specs"], "sum", empty_like_tiling(c["ext"], c["cs"], F32))
+    assert e.value.status_name == "JA_ERR_DTYPE"
+    with pytest.raises(JaError) as e:                      # two copies need an aggregation
+        h.execute(rP, c["copy_site"], c["specs"], "none", rD)
+    assert e.value.status_name == "JA_ERR_INVALID_ARG"
+    # a body that does not satisfy OUT
+    bad = X.ExchangeProgram(str(h).split("\n\n")[0] + "\n\n")
+    with pytest.raises(JaError) as e:
+        bad.execute(rP, c["copy_site"], c["specs"], "sum", rD)
+    assert e.value.status_name == "JA_ERR_INVALID_ARG"
+    unbound = X.ExchangeProgram(handle=X.ja_exprog_preamble(c["ps"], c["cs"], 2, c["copy_site"], c["specs"], 2))
+    with pytest.raises(JaError):
+        unbound.execute(rP, c["copy_site"], c["specs"], "sum", rD)
+    check_status()

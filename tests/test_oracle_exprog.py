@@ -249,3 +249,40 @@ def test_rule_families_keep_validity_and_their_closures():
         cur = rng.choice(nb)
     q, ms = E.synthesize(cur, H100, depth=2, beam=6)
     assert E.valid_bound(q) and ms <= E.simulate(cur, H100) * (1 + 1e-12)
+
+
+def test_executing_any_valid_program_gives_the_aggregate_of_all_copies():
+    """The oracle's executor (decompose, fire the actions, recompose) against the plain definition it must reach: the
+    consumer's tensor is the (+)-aggregate of the m copies, whatever the program's route (oracle/blocked.py
+    aggregate_repartition, itself pinned to the preamble example and to brute force)."""
+    import numpy as np
+
+    from oracle import blocked
+    rng = np.random.default_rng(4)
+    mo = E.machine("dgx_h100")
+    cases = [
+        ([256, 256], [[0, 128, 256], [0, 256]], [[0, 64, 128, 192, 256], [0, 256]], 2, [0, 1, 2, 3], [0, 1, 2, 3]),
+        ([6, 33, 10], [[0, 3, 6], [0, 10, 33], [0, 10]], [[0, 6], [0, 33], [0, 3, 10]], 3, [0, 1, 2, 2, 0, 1, 1, 2, 0, 0, 2, 1], [0, 1, 1]),
+        ([128, 64], [[0, 128], [0, 64]], [[0, 128], [0, 64]], 4, [0, 1, 2, 3], [0, 0, 0, 0]),
+    ]
+    for ext, ps, cs, m, sites, specs in cases:
+        pre = E.preamble(ext, ps, {(b, c): sites[b * m + c] for b in range(len(sites) // m) for c in range(m)}, cs, specs, 4)
+        P = rng.standard_normal([m] + ext)
+        for body in (E.naive_body, E.butterfly_body, lambda b: E.synthesize(b, mo, depth=2, beam=5)[0]):
+            _, q, _ = E.place(pre, mo, body=body)
+            for agg in ("sum", "max"):
+                out = E.exchange(q, P, ps, cs, specs, agg)
+                ref = blocked.aggregate_repartition(P, ps, cs, agg)
+                assert np.abs(out - ref).max() <= (1e-12 if agg == "sum" else 0.0)
+        # a rewritten program: the walk changes the aggregation trees, not the result
+        rnd = random.Random(7)
+        _, cur, _ = E.place(pre, mo, body=E.naive_body)
+        cur = E.normalised(cur)
+        for _ in range(6):
+            cur = rnd.choice(E.neighbours(cur))
+        assert np.abs(E.exchange(cur, P, ps, cs, specs, "sum") - blocked.aggregate_repartition(P, ps, cs, "sum")).max() <= 1e-12
+    # the schedule fires every action once, in an order in which each is enabled
+    q = E.parse(G["doubling"]["program"])
+    sched = E.schedule(q)
+    assert len(sched) == len(E.expanded(q))
+    assert [len(c) for x, s, d, c in sched if len(x) == 4] == [2, 2, 2, 2]          # A+B and C+D, not four atoms
