@@ -847,6 +847,40 @@ def case_results(case, reps):
         res["random_p8_20_draws"] = {"ms_mean": sum(ms) / len(ms), "ms_best": ms[0], "ms_median": (ms[9] + ms[10]) / 2, "ms_worst": ms[-1],
                                      "proxy_cost_cells_median": sorted(d["proxy_cost_cells"] for d in draws)[10],
                                      "relayouts_executed_median": sorted(d["relayouts_executed"] for d in draws)[10]}
+    elif args.case == "exchange":
+        # Section 5: the exchange that links the down projection of the 7B block, compiled through its join with the contracted
+        # index cut four ways (copy c of the one output block on GPU c), to a consumer cut into four row intervals (one function
+        # spec per GPU: a reduce-scatter) or to four function specs that all consume the whole tensor (an all-reduce, rows cut
+        # into four atoms by giving the producer four row blocks). Per case: the simulator's completion time of the naive and
+        # of the synthesised program on the nominal NVSwitch model of this part, and the SAME program executed on this one GPU
+        # (sites = regions of its memory) beside the fused aggregating relayout.
+        from paper_2609_03905_b200 import exprog as X
+        hb = lambda nbytes, t: {**t, "GBps": nbytes / (t["ms_mean"] * 1e-3) / 1e9, "frac_of_measured_hbm": nbytes / (t["ms_mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        T, d, m = 16384, 4096, 4
+        mach = X.ja_machine_preset("hgx_b200")
+        for tag, ps, cs, specs in (("reduce_scatter", [[0, T], [0, d]], [ES(T, 4), [0, d]], [0, 1, 2, 3]),
+                                   ("all_reduce", [ES(T, 4), [0, d]], [[0, T], [0, d]], [0, 0, 0, 0])):
+            npb = (len(ps[0]) - 1) * (len(ps[1]) - 1)
+            copy_site = [c for _ in range(npb) for c in range(m)]
+            P = ja.partial_relation(m, [T, d], ps, bf)
+            P.payload.normal_(0.0, 1.0)
+            y = ja.Relation([T, d], cs, bf)
+            for body in ("naive", "best"):
+                h = X.ExchangeProgram(handle=X.ja_exprog_preamble(ps, cs, m, copy_site, specs, 2))
+                sim = X.ja_exprog_place(h.handle, mach, body)
+                if body == "best":
+                    sim = X.ja_exprog_synthesize(h.handle, mach, 2, 8)
+                stats = h.execute(P, copy_site, specs, "sum", y)
+                t = timeit(lambda r: h.execute(P, copy_site, specs, "sum", y), reps, True)
+                acts = X.ja_exprog_get_actions(h.handle)
+                # HBM traffic on this GPU: decompose reads and writes every copy once, recompose the tensor once, a transfer reads
+                # and writes its atom, an aggregation reads its parts and writes one atom
+                nbytes = 2.0 * m * T * d * 2 + 2.0 * T * d * 2 + 2.0 * stats["transfer_bytes"] + stats["aggregation_bytes"]
+                res["%s_%s" % (tag, "synthesised" if body == "best" else body)] = {
+                    **hb(nbytes, t), "simulated_ms_hgx_b200_nominal": sim, "actions": len(acts), "aggregations": stats["aggregations"],
+                    "transfers": stats["transfers"], "transfer_MB": stats["transfer_bytes"] / 1e6, "scratch_MB": stats["scratch_bytes"] / 1e6}
+            res["%s_fused_aggregating_relayout" % tag] = hb((m + 1.0) * T * d * 2, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
+            del P, y
     elif args.case == "chains":
         # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
         # join-aggs (every intermediate stored once, in bf16); operands N(0, 1/rows) so that magnitudes stay O(1)
@@ -907,11 +941,12 @@ def main():
     ap.add_argument("--dtype", choices=["bf16", "f16"], default="bf16",
                     help="cell type of the block's relations (--case block): bf16 as the benchmark configurations state, or f16, the paper's precision")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains"], default="block",
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains", "exchange"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "
                          "gqa = grouped-query attention over packed sequences; agg = join-only matmul + aggregating relayout; "
                          "opt = logical optimizer's plan for the MLP tree against hand plans; optblock = the optimizer's plans for the whole "
-                         "7B block against the hand decompositions; chains = the five matrix chains")
+                         "7B block against the hand decompositions; chains = the five matrix chains; exchange = exchange programs for a "
+                         "reduce-scatter and an all-reduce of the down projection's partial copies, simulated and executed on this GPU")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
     if args.case != "block":

@@ -156,12 +156,14 @@ ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, con
  * combines them in ascending order of their first atoms in f32 (SUM or MAX) and rounds once to the cell type, a transfer
  * one device-to-device copy -- and recompose (the aggregated atoms at the site of function spec i are concatenated into
  * the block it consumes; a block consumed by several specs is written from the lowest one).  At most 16 parts per
- * aggregation, tensors of rank <= 3.  Scratch memory for the atom buffers comes from the stream-ordered allocator and is
- * returned to it at the end of the call.  stats (optional, HOST, 4 values): local aggregations launched, transfers,
- * bytes transferred, scratch bytes. */
+ * aggregation, tensors of rank <= 3.  Scratch memory for the atom buffers comes from a stream-ordered memory pool of the
+ * library's own and goes back to it, in stream order, at the end of the call; the pool keeps it for the next call until
+ * ja_exchange_trim (which the caller synchronises before) hands it back to the driver.  stats (optional, HOST, 5 values):
+ * local aggregations launched, transfers, bytes transferred, scratch bytes, bytes read and written by the aggregations. */
 ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
                                 const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
                                 int64_t* stats, void* cuda_stream);
+ja_status_t ja_exchange_trim(void);
 
 #ifdef __cplusplus
 }

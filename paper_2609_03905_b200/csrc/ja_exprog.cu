@@ -12,6 +12,7 @@
 #include <algorithm>
 #include <charconv>
 #include <map>
+#include <mutex>
 #include <set>
 #include <string>
 #include <tuple>
@@ -1421,6 +1422,41 @@ extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_
     return JA_OK;
 }
 
+// Scratch of ja_exchange_execute: a stream-ordered pool of the library's own per device that keeps what it has been given
+// (the default pool hands memory back to the driver at every synchronisation, and getting a gigabyte again costs milliseconds);
+// ja_exchange_trim returns it.
+namespace {
+std::mutex g_pool_mu;
+std::map<int, cudaMemPool_t> g_pools;
+ja_status_t exchange_pool(cudaMemPool_t* out) {
+    int dev = 0;
+    JA_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(g_pool_mu);
+    auto it = g_pools.find(dev);
+    if (it == g_pools.end()) {
+        cudaMemPoolProps props;
+        memset(&props, 0, sizeof props);
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t mp = nullptr;
+        JA_CUDA(cudaMemPoolCreate(&mp, &props));
+        uint64_t keep = UINT64_MAX;
+        JA_CUDA(cudaMemPoolSetAttribute(mp, cudaMemPoolAttrReleaseThreshold, &keep));
+        it = g_pools.insert({dev, mp}).first;
+    }
+    *out = it->second;
+    return JA_OK;
+}
+}  // namespace
+
+extern "C" ja_status_t ja_exchange_trim(void) {
+    std::lock_guard<std::mutex> lk(g_pool_mu);
+    for (auto& kv : g_pools) JA_CUDA(cudaMemPoolTrimTo(kv.second, 0));
+    return JA_OK;
+}
+
 // ---------------------------------------------------------------------------------- execution on one GPU (Section 5.3)
 // The sites of the program are regions of this GPU's memory; a transfer is a device-to-device copy (on a machine with
 // several GPUs it would be a peer copy), a local aggregation one launch of the combine kernel, decompose and recompose
@@ -1506,7 +1542,7 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
         scratch += (atom_bytes(x) + 255) / 256 * 256;
     };
     for (size_t a = 0; a < prog->atoms.size(); ++a) alloc(prog->atoms[a].site, 1ull << a);
-    int64_t n_aggregations = 0, n_transfers = 0, transfer_bytes = 0;
+    int64_t n_aggregations = 0, n_transfers = 0, transfer_bytes = 0, aggregation_bytes = 0;
     for (const Fired& f : order) {
         const Flat& a = acts[f.act];
         if (f.parts.size() > JA_EXCHANGE_MAX_PARTS)
@@ -1584,7 +1620,9 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* pool = nullptr;
-    JA_CUDA(cudaMallocAsync((void**)&pool, (size_t)scratch, stream));
+    cudaMemPool_t mp = nullptr;
+    if ((st = exchange_pool(&mp)) != JA_OK) return st;
+    JA_CUDA(cudaMallocFromPoolAsync((void**)&pool, (size_t)scratch, mp, stream));
     ja_status_t rc = JA_OK;
     do {
         if (cudaMemcpyAsync(pool + table_off, boxes.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
@@ -1601,6 +1639,7 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
                 for (size_t k = 0; k < f.parts.size(); ++k) parts[k] = pool + buf[{a.site, f.parts[k]}];
                 if ((rc = ja_launch_exchange_combine(parts, (int)f.parts.size(), here, atom_bytes(a.agg), partials->dtype, agg, stream)) != JA_OK) break;
                 ++n_aggregations;
+                aggregation_bytes += ((int64_t)f.parts.size() + 1) * atom_bytes(a.agg);
             }
             for (int d : a.dests) {
                 char* there = pool + buf[{d, a.agg}];
@@ -1624,6 +1663,7 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
         stats[1] = n_transfers;
         stats[2] = transfer_bytes;
         stats[3] = scratch;
+        stats[4] = aggregation_bytes;
     }
     return JA_OK;
 }

@@ -49,6 +49,8 @@ def _declare():
         fn = getattr(LIB, name)
         fn.argtypes = argtypes
         fn.restype = ctypes.c_int
+    LIB.ja_exchange_trim.argtypes = []
+    LIB.ja_exchange_trim.restype = ctypes.c_int
     LIB.ja_exprog_destroy.argtypes = [vp]
     LIB.ja_exprog_destroy.restype = None
 
@@ -205,11 +207,16 @@ def ja_exprog_preamble(producer_splits, consumer_splits, m: int, copy_site, cons
 def ja_exchange_execute(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int, stream: int = 0) -> dict:
     """Relation handles as in binding.ja_repartition_agg; returns the call's statistics."""
     from .binding import AGG
-    stats = (ctypes.c_int64 * 4)()
+    stats = (ctypes.c_int64 * 5)()
     _check(LIB.ja_exchange_execute(prog, partials, (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
                                    (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs),
                                    AGG[agg] if isinstance(agg, str) else int(agg), dst, stats, stream))
-    return {"aggregations": stats[0], "transfers": stats[1], "transfer_bytes": stats[2], "scratch_bytes": stats[3]}
+    return {"aggregations": stats[0], "transfers": stats[1], "transfer_bytes": stats[2], "scratch_bytes": stats[3],
+            "aggregation_bytes": stats[4]}
+
+
+def ja_exchange_trim():
+    _check(LIB.ja_exchange_trim())
 
 
 class ExchangeProgram:
