@@ -165,6 +165,20 @@ ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* pa
                                 int64_t* stats, void* cuda_stream);
 ja_status_t ja_exchange_trim(void);
 
+/* ---- the pieces a program needs when its sites are different processes (one per GPU) ------------------------------------
+ * ja_exprog_schedule: the firing order ja_exchange_execute uses, for a driver that issues the actions itself: fired action
+ * k is expanded action action[k] and aggregates parts[part_begin[k] .. part_begin[k + 1]) (masks, in combination order;
+ * one part = the aggregate is already materialised, nothing to compute).  Every process derives the same order from the
+ * same program.  NULL arrays to get the two counts; part_begin has n_fired + 1 entries.  JA_ERR_INVALID_ARG if the
+ * program is not well-formed.  Host only.
+ * ja_exchange_combine: the local aggregation stage of one action on DEVICE buffers: out = parts[0] (+) parts[1] (+) ... in
+ * that order (2..16 parts; SUM or MAX in f32, one rounding to `dtype`).  All buffers hold `bytes` bytes, a multiple of 16,
+ * and are 16-byte aligned (JA_ERR_ALIGNMENT otherwise); out may not alias a part.  Asynchronous on cuda_stream. */
+ja_status_t ja_exprog_schedule(const ja_exprog_t* p, int32_t* n_fired, int32_t* n_parts_total, int32_t* action,
+                               int32_t* part_begin, uint64_t* parts);
+ja_status_t ja_exchange_combine(const void* const* parts, int32_t n_parts, void* out, int64_t bytes, ja_dtype_t dtype,
+                                ja_agg_t agg, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

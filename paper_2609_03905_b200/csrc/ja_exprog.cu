@@ -1422,6 +1422,76 @@ extern "C" ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_
     return JA_OK;
 }
 
+namespace {
+// A firing order of a bound program and the parts of every aggregation: repeated passes over the expanded actions in body
+// order; an action fires the first time aggregates at its source partition its aggregate (the partition with the fewest parts,
+// candidates in ascending order of their masks, so the parts come out in ascending order of their first atoms). Actions that
+// never become enabled are left out (the program is then not well-formed).
+struct Fired {
+    int act;
+    std::vector<uint64_t> parts;
+};
+void firing_order(const Prog& p, const std::vector<Flat>& acts, std::vector<Fired>* order) {
+    order->clear();
+    std::map<int, std::set<uint64_t>> have;
+    for (size_t i = 0; i < p.atoms.size(); ++i) have[p.atoms[i].site].insert(1ull << i);
+    std::vector<bool> fired(acts.size(), false);
+    bool progress = true;
+    while (progress) {
+        progress = false;
+        for (size_t i = 0; i < acts.size(); ++i) {
+            if (fired[i]) continue;
+            CoverParts cp;
+            for (uint64_t y : have[acts[i].site])
+                if ((y & ~acts[i].agg) == 0) cp.cands.push_back(y);
+            cp.rec(acts[i].agg);
+            if (cp.best.empty()) continue;
+            fired[i] = true;
+            progress = true;
+            order->push_back({(int)i, cp.best});
+            have[acts[i].site].insert(acts[i].agg);
+            for (int d : acts[i].dests) have[d].insert(acts[i].agg);
+        }
+    }
+}
+}  // namespace
+
+extern "C" ja_status_t ja_exprog_schedule(const ja_exprog_t* p, int32_t* n_fired, int32_t* n_parts_total, int32_t* action,
+                                          int32_t* part_begin, uint64_t* parts) {
+    ja_status_t st = need_bound(p);
+    if (st != JA_OK) return st;
+    std::vector<Flat> acts;
+    expand(*p, &acts);
+    std::vector<Fired> order;
+    firing_order(*p, acts, &order);
+    if (order.size() != acts.size()) return ja_fail(JA_ERR_INVALID_ARG, "the program is not well-formed: an action never becomes enabled");
+    int32_t total = 0;
+    for (size_t i = 0; i < order.size(); ++i) {
+        if (action) action[i] = order[i].act;
+        if (part_begin) part_begin[i] = total;
+        for (uint64_t y : order[i].parts) {
+            if (parts) parts[total] = y;
+            ++total;
+        }
+    }
+    if (part_begin) part_begin[order.size()] = total;
+    if (n_fired) *n_fired = (int32_t)order.size();
+    if (n_parts_total) *n_parts_total = total;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exchange_combine(const void* const* parts, int32_t n_parts, void* out, int64_t bytes, ja_dtype_t dtype,
+                                           ja_agg_t agg, void* cuda_stream) {
+    if (!parts || !out || bytes < 1) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    if (agg != JA_AGG_SUM && agg != JA_AGG_MAX) return ja_fail(JA_ERR_INVALID_ARG, "SUM or MAX");
+    if (dtype != JA_F32 && dtype != JA_BF16 && dtype != JA_F16) return ja_fail(JA_ERR_DTYPE, "unknown cell type");
+    if (bytes % 16) return ja_fail(JA_ERR_ALIGNMENT, "the buffers are read and written in 16-byte accesses: %lld bytes is not a whole number of them", (long long)bytes);
+    if ((uintptr_t)out % 16) return ja_fail(JA_ERR_ALIGNMENT, "out must be 16-byte aligned");
+    for (int i = 0; i < n_parts; ++i)
+        if (!parts[i] || (uintptr_t)parts[i] % 16) return ja_fail(JA_ERR_ALIGNMENT, "part %d must be a 16-byte aligned device pointer", i);
+    return ja_launch_exchange_combine(parts, n_parts, out, bytes, dtype, agg, (cudaStream_t)cuda_stream);
+}
+
 // Scratch of ja_exchange_execute: a stream-ordered pool of the library's own per device that keeps what it has been given
 // (the default pool hands memory back to the driver at every synchronisation, and getting a gigabyte again costs milliseconds);
 // ja_exchange_trim returns it.
@@ -1495,36 +1565,11 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
     if (!same) return ja_fail(JA_ERR_INVALID_ARG, "the program's preamble is not the one these relations, copy sites and function specs generate");
     if (!valid_bound(*prog)) return ja_fail(JA_ERR_INVALID_ARG, "the program is not valid (Definition \"Closure; validity\")");
 
-    // firing order and the parts of every aggregation: repeated passes over the expanded actions in body order
+    // firing order and the parts of every aggregation
     std::vector<Flat> acts;
     expand(*prog, &acts);
-    struct Fired {
-        int act;
-        std::vector<uint64_t> parts;
-    };
     std::vector<Fired> order;
-    {
-        std::map<int, std::set<uint64_t>> have;
-        for (size_t i = 0; i < prog->atoms.size(); ++i) have[prog->atoms[i].site].insert(1ull << i);
-        std::vector<bool> fired(acts.size(), false);
-        bool progress = true;
-        while (progress) {
-            progress = false;
-            for (size_t i = 0; i < acts.size(); ++i) {
-                if (fired[i]) continue;
-                CoverParts cp;
-                for (uint64_t y : have[acts[i].site])
-                    if ((y & ~acts[i].agg) == 0) cp.cands.push_back(y);
-                cp.rec(acts[i].agg);
-                if (cp.best.empty()) continue;
-                fired[i] = true;
-                progress = true;
-                order.push_back({(int)i, cp.best});
-                have[acts[i].site].insert(acts[i].agg);
-                for (int d : acts[i].dests) have[d].insert(acts[i].agg);
-            }
-        }
-    }
+    firing_order(*prog, acts, &order);
     // buffers: one per (aggregate, site) materialisation
     auto atom_bytes = [&](uint64_t agg_mask) {
         const int a = __builtin_ctzll(agg_mask);

@@ -44,6 +44,8 @@ def _declare():
         "ja_exprog_place": [vp, P(ja_machine_t), i32, P(dbl)],
         "ja_exprog_preamble": [i32, P(i64), P(i32), P(i64), P(i32), i32, P(i32), P(i32), i32, i32, P(vp)],
         "ja_exchange_execute": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i64), vp],
+        "ja_exprog_schedule": [vp, P(i32), P(i32), P(i32), P(i32), P(u64)],
+        "ja_exchange_combine": [P(vp), i32, vp, i64, ctypes.c_int, ctypes.c_int, vp],
     }
     for name, argtypes in sigs.items():
         fn = getattr(LIB, name)
@@ -213,6 +215,21 @@ def ja_exchange_execute(prog: int, partials: int, copy_site, consumer_specs, agg
                                    AGG[agg] if isinstance(agg, str) else int(agg), dst, stats, stream))
     return {"aggregations": stats[0], "transfers": stats[1], "transfer_bytes": stats[2], "scratch_bytes": stats[3],
             "aggregation_bytes": stats[4]}
+
+
+def ja_exprog_schedule(prog: int):
+    """[(expanded action index, [part masks in combination order])] in firing order."""
+    n, total = ctypes.c_int32(), ctypes.c_int32()
+    _check(LIB.ja_exprog_schedule(prog, ctypes.byref(n), ctypes.byref(total), None, None, None))
+    act, begin, parts = (ctypes.c_int32 * max(n.value, 1))(), (ctypes.c_int32 * (n.value + 1))(), (ctypes.c_uint64 * max(total.value, 1))()
+    _check(LIB.ja_exprog_schedule(prog, ctypes.byref(n), ctypes.byref(total), act, begin, parts))
+    return [(act[k], [parts[i] for i in range(begin[k], begin[k + 1])]) for k in range(n.value)]
+
+
+def ja_exchange_combine(part_ptrs, out_ptr: int, nbytes: int, dtype: int, agg, stream: int = 0):
+    from .binding import AGG
+    arr = (ctypes.c_void_p * len(part_ptrs))(*[int(p) for p in part_ptrs])
+    _check(LIB.ja_exchange_combine(arr, len(part_ptrs), out_ptr, nbytes, dtype, AGG[agg] if isinstance(agg, str) else int(agg), stream))
 
 
 def ja_exchange_trim():

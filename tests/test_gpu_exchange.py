@@ -137,3 +137,30 @@ def test_exchange_refusals():
     with pytest.raises(JaError):
         unbound.execute(rP, c["copy_site"], c["specs"], "sum", rD)
     check_status()
+
+
+@pytest.mark.parametrize("dtype", [BF, F16, F32])
+@pytest.mark.parametrize("agg", ["sum", "max"])
+@pytest.mark.parametrize("n_parts", [2, 5, 16])
+def test_the_local_aggregation_primitive(n_parts, agg, dtype):
+    from paper_2609_03905_b200 import exchange_dist
+    n = 4096 + 8 * 37                                                   # whole 16-byte accesses, several blocks and a ragged last one
+    parts = [si.normal([n], 0.0, 1.0, dtype, 9, k).cuda() for k in range(n_parts)]
+    out = exchange_dist.library_combine(parts, agg)
+    torch.cuda.synchronize()
+    check_status()
+    P64 = [si.to_f64(p.cpu()) for p in parts]
+    if agg == "max":
+        assert np.array_equal(si.to_f64(out.cpu()), np.max(np.stack(P64), axis=0))
+    else:
+        acc = P64[0].astype(np.float32)
+        for p in P64[1:]:
+            acc = acc + p.astype(np.float32)
+        assert np.array_equal(si.to_f64(out.cpu()), core.round_to(acc.astype(np.float64), ORC_DT[dtype]))
+        assert relfro(si.to_f64(out.cpu()), core.round_to(np.sum(np.stack(P64), axis=0), ORC_DT[dtype])) <= (1e-6 if dtype == F32 else 1e-3)
+    with pytest.raises(JaError) as e:
+        X.ja_exchange_combine([parts[0].data_ptr(), parts[1].data_ptr() + 2], out.data_ptr(), 64, 1, "sum")
+    assert e.value.status_name == "JA_ERR_ALIGNMENT"
+    with pytest.raises(JaError) as e:
+        X.ja_exchange_combine([parts[0].data_ptr(), parts[1].data_ptr()], out.data_ptr(), 40, 1, "sum")
+    assert e.value.status_name == "JA_ERR_ALIGNMENT"

@@ -305,3 +305,34 @@ def test_generated_preamble_against_the_oracle_and_the_paper():
     mo = E.machine("hgx_b200")
     _, _, ms_o = E.place(want2, mo, body=lambda b: E.synthesize(b, mo, depth=0)[0])
     assert close(ms, ms_o)
+
+
+def test_firing_order_against_the_oracle():
+    rng = random.Random(23)
+    texts = [G[n]["program"] for n in ("swap", "doubling")]
+    for _ in range(25):
+        n_sites = rng.randint(2, 4)
+        atoms = list("ABCDE")[:rng.randint(2, 5)]
+        t = "GPUS: " + ", ".join(str(s) for s in range(n_sites)) + "\nIN: " + "; ".join("%s @ %d" % (a, rng.randrange(n_sites)) for a in atoms)
+        t += "\nOUT: " + "+".join(atoms) + " @ " + ", ".join(str(s) for s in range(n_sites)) + "\n"
+        texts.append(t)
+    for t in texts:
+        h = X.ExchangeProgram(t)
+        p = E.parse(t)
+        if not p.actions:
+            X.ja_exprog_body(h.handle, "naive")
+            X.ja_exprog_normalise(h.handle)
+            p = E.normalised(E.naive_body(p))
+            for _ in range(4):                                   # a few rewrites so that aggregation trees differ
+                nb = E.neighbours(p)
+                if nb:
+                    p = rng.choice(nb)
+            h = X.ExchangeProgram(E.format_program(p))
+        mk = masks(p)
+        acts = E.expanded(p)
+        want = [(acts.index((x, s, d)), [mk(y) for y in cover]) for x, s, d, cover in E.schedule(p)]
+        assert X.ja_exprog_schedule(h.handle) == want
+    from paper_2609_03905_b200.binding import JaError
+    never = X.ExchangeProgram("IN: A @ 0; B @ 1\nOUT: A+B @ 0\n\nA+B @ 0\n")       # kept alive: the handle dies with the object
+    with pytest.raises(JaError):
+        X.ja_exprog_schedule(never.handle)
