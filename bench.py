@@ -847,6 +847,20 @@ def case_results(case, reps):
         res["random_p8_20_draws"] = {"ms_mean": sum(ms) / len(ms), "ms_best": ms[0], "ms_median": (ms[9] + ms[10]) / 2, "ms_worst": ms[-1],
                                      "proxy_cost_cells_median": sorted(d["proxy_cost_cells"] for d in draws)[10],
                                      "relayouts_executed_median": sorted(d["relayouts_executed"] for d in draws)[10]}
+        # Section 6, Experiment 5 in miniature: Pearson correlation between the proxy cost of a plan and its measured time, over
+        # the twenty draws and over all p = 8 plans timed here (draws, greedy, optimizer, hand plans)
+
+        def pearson(xs, ys):
+            n = len(xs)
+            mx, my = sum(xs) / n, sum(ys) / n
+            sxy = sum((x - mx) * (y - my) for x, y in zip(xs, ys))
+            sxx, syy = sum((x - mx) ** 2 for x in xs), sum((y - my) ** 2 for y in ys)
+            return sxy / (sxx * syy) ** 0.5 if sxx > 0 and syy > 0 else float("nan")
+
+        pts = [(d["proxy_cost_cells"], d["ms_mean"]) for d in draws]
+        more = [(v["proxy_cost_cells"], v["ms_mean"]) for k, v in res.items() if k.endswith("p8") and "proxy_cost_cells" in v]
+        res["proxy_cost_against_time_p8"] = {"pearson_r_random_draws": pearson(*zip(*pts)), "n_random_draws": len(pts),
+                                             "pearson_r_all_p8_plans": pearson(*zip(*(pts + more))), "n_all": len(pts) + len(more)}
     elif args.case == "exchange":
         # Section 5: the exchange that links the down projection of the 7B block, compiled through its join with the contracted
         # index cut four ways (copy c of the one output block on GPU c), to a consumer cut into four row intervals (one function
