@@ -448,8 +448,47 @@ def run_gpu(args, shape):
 L2_NOTE = "512 MiB flush buffer written, then a 256 MiB buffer read (clean lines), before every timed launch"
 
 
+def physical_results():
+    """Section 6, Experiment 4 in miniature, on the library's simulator (host only, no GPU): the exchange programs that link the
+    operators of a plan the logical optimizer chose for eight GPUs -- the 7B block and matrix chains A and B -- compiled
+    naively (function spec i on GPU i, every aggregated block gathered and aggregated where it is consumed) and with
+    placement and synthesis, on the NVSwitch model of the DGX-A100 and on the cube mesh of the DGX-V100."""
+    import paper_2609_03905_b200 as ja
+    from paper_2609_03905_b200 import exprog as X, physical
+    from paper_2609_03905_b200.planned_block import block_graph
+    workloads = {}
+    ops = block_graph(8, 2048, 4096, 32, 11008)
+    workloads["llama7b_block"] = (ops, ja.ja_plan_optimize_graph(ops, 8)[1])
+    chains = {"chain_A": ([10240] + [16384, 6144] * 4 + [10240], ((0, 1), (((2, 3), ((4, 5), (6, 7))), 8))),
+              "chain_B": ([9216, 20480, 5120, 20480, 5120, 9216], ((0, 1), ((2, 3), 4)))}
+    for name, (dims, tree) in chains.items():
+        ops = []
+
+        def build(t):   # returns (producer index or None, rows, cols)
+            if isinstance(t, int):
+                return None, dims[t], dims[t + 1]
+            (a, m, j), (b, _, n) = build(t[0]), build(t[1])
+            ops.append({"einsum": "ij,jk->ik", "extents": {"i": m, "j": j, "k": n}, "inputs": [a, b]})
+            return len(ops) - 1, m, n
+        build(tree)
+        workloads[name] = (ops, ja.ja_plan_optimize(ops, 8)[1])
+    res = {}
+    for name, (ops, plan) in workloads.items():
+        for mname in ("dgx_a100", "dgx_v100"):
+            mach = X.ja_machine_preset(mname)
+            naive, en = physical.compile_exchanges(ops, plan, mach, False)
+            opt, eo = physical.compile_exchanges(ops, plan, mach, True, depth=2, beam=6)
+            res["%s_%s" % (name, mname)] = {"naive_ms": naive, "optimised_ms": opt, "naive_over_optimised": naive / opt if opt > 0 else 1.0,
+                                            "edges": len(en), "edges_with_traffic": sum(1 for e in en if e["ms"] > 0),
+                                            "proxy_cost_cells": ja.ja_plan_cost(ops, plan)}
+    return res
+
+
 def run_case(args):
     """Times the kernels of one benchmark configuration in isolation and prints one JSON line."""
+    if args.case == "physical":
+        print(json.dumps({"case": "physical", "simulated": True, "results": physical_results()}))
+        return
     import torch
     torch.cuda.set_device(0)
     res = case_results(args.case, args.steps)
@@ -955,12 +994,13 @@ def main():
     ap.add_argument("--dtype", choices=["bf16", "f16"], default="bf16",
                     help="cell type of the block's relations (--case block): bf16 as the benchmark configurations state, or f16, the paper's precision")
     ap.add_argument("--unfused", action="store_true", help="run every join-agg of the block as its own launch (no fused chains)")
-    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains", "exchange"], default="block",
+    ap.add_argument("--case", choices=["block", "cfg1", "cfg2", "cfg3", "cfg4", "gqa", "agg", "opt", "optblock", "chains", "exchange", "physical"], default="block",
                     help="block = the headline step; cfgN = the kernels of benchmark configuration N in isolation; "
                          "gqa = grouped-query attention over packed sequences; agg = join-only matmul + aggregating relayout; "
                          "opt = logical optimizer's plan for the MLP tree against hand plans; optblock = the optimizer's plans for the whole "
                          "7B block against the hand decompositions; chains = the five matrix chains; exchange = exchange programs for a "
-                         "reduce-scatter and an all-reduce of the down projection's partial copies, simulated and executed on this GPU")
+                         "reduce-scatter and an all-reduce of the down projection's partial copies, simulated and executed on this GPU; "
+                         "physical = naive against optimised exchange programs for the block and chains A, B on the simulator (host only)")
     args = ap.parse_args()
     shape = SHAPES[args.shape]
     if args.case != "block":

@@ -76,6 +76,9 @@ ja_status_t ja_exprog_get_atoms(const ja_exprog_t* p, int32_t* site, double* siz
 ja_status_t ja_exprog_num_memberships(const ja_exprog_t* p, int64_t* n);
 ja_status_t ja_exprog_bind(ja_exprog_t* p, int64_t index);
 ja_status_t ja_exprog_membership(const ja_exprog_t* p, const char* partition, uint64_t* members);
+/* Gives one size-declared partition explicit members (n = its size; JA_ERR_INVALID_ARG if they overlap another
+ * partition's, are not declared GPUs, or the partition already has members). */
+ja_status_t ja_exprog_bind_members(ja_exprog_t* p, const char* partition, const int32_t* sites, int32_t n);
 
 /* ---- Definition "Closure; validity" (Section 5.4) -------------------------------------------------------------------
  * ja_exprog_closure: S*(P) as (aggregate, site) pairs sorted by site, then by mask; NULL arrays to get the count.
@@ -119,6 +122,9 @@ ja_status_t ja_exprog_simulate(const ja_exprog_t* p, const ja_machine_t* machine
  * ja_exprog_place: chooses the members of the size-declared partitions -- among the memberships under which the program
  * is valid the one with the least simulated time (the first of equals), with body = JA_BODY_OWN (the program's body as it
  * is), JA_BODY_NAIVE, JA_BODY_BUTTERFLY or JA_BODY_BEST (the better of the two constructed ones) rebuilt per membership.
+ * Above 5000 memberships they are not enumerated: the search starts from the first one (the free sites dealt to the
+ * partitions in ascending order) and repeatedly takes the exchange of two sites between two partitions that lowers the
+ * simulated time most (the first of equals, pairs in ascending order), until none does.
  * The program is left bound to the chosen membership with the chosen body.  JA_ERR_INVALID_ARG if none is valid. */
 typedef enum { JA_BODY_OWN = 0, JA_BODY_NAIVE = 1, JA_BODY_BUTTERFLY = 2, JA_BODY_BEST = 3 } ja_body_t;
 typedef enum {
@@ -158,7 +164,9 @@ ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, con
  * the block it consumes; a block consumed by several specs is written from the lowest one).  At most 16 parts per
  * aggregation, tensors of rank <= 3.  Scratch memory for the atom buffers comes from a stream-ordered memory pool of the
  * library's own and goes back to it, in stream order, at the end of the call; the pool keeps it for the next call until
- * ja_exchange_trim (which the caller synchronises before) hands it back to the driver.  stats (optional, HOST, 5 values):
+ * ja_exchange_trim (which the caller synchronises before) hands it back to the driver.  Not capturable: a call on a stream
+ * that is being captured is refused (JA_ERR_UNSUPPORTED, nothing enqueued); the call may block the host briefly while its
+ * tables are staged.  stats (optional, HOST, 5 values):
  * local aggregations launched, transfers, bytes transferred, scratch bytes, bytes read and written by the aggregations. */
 ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
                                 const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,

@@ -32,6 +32,7 @@ Readings where the paper is silent (each also listed in the design notes of the 
 from __future__ import annotations
 
 import itertools
+import math
 import re
 from dataclasses import dataclass, field
 
@@ -473,20 +474,63 @@ def butterfly_body(prog: Program) -> Program:
     return q
 
 
-def place(prog: Program, mach: dict, body=None):
+def place(prog: Program, mach: dict, body=None, enumeration_limit: int = 5000):
     """Choose the members of the size-declared partitions: among the memberships under which the program (its own body,
     or body(bound preamble) if a synthesiser is given) is valid, the one with the least simulated completion time; ties go to
-    the first in enumeration order.  Returns (membership, bound program, milliseconds)."""
-    best = None
-    for m in memberships(prog):
+    the first in enumeration order.  Above `enumeration_limit` memberships: steepest descent over exchanges of two sites
+    between two partitions instead.  Returns (membership, bound program, milliseconds)."""
+    def cost(m):
         q = bind(prog, m)
         if body is not None:
             q = body(q)
         if not valid_bound(q):
-            continue
-        ms = simulate(q, mach)
-        if best is None or ms < best[2] * (1.0 - 1e-12):
-            best = (m, q, ms)
+            return None
+        return (m, q, simulate(q, mach))
+
+    names = [n for n, p in prog.partitions.items() if p["members"] is None]
+    taken = {s for p in prog.partitions.values() if p["members"] is not None for s in p["members"]}
+    n_free = len([s for s in prog.gpus if s not in taken])
+    total = 1
+    for n in names:
+        k = prog.partitions[n]["size"]
+        total *= math.comb(n_free, k)
+        n_free -= k
+    best = None
+    if total <= enumeration_limit:
+        for m in memberships(prog):
+            c = cost(m)
+            if c is not None and (best is None or c[2] < best[2] * (1.0 - 1e-12)):
+                best = c
+    else:
+        # steepest descent over exchanges of two sites between partitions, from the first membership in enumeration order
+        free = [s for s in prog.gpus if s not in taken]
+        cur, at = {}, 0
+        for n in names:
+            cur[n] = tuple(free[at: at + prog.partitions[n]["size"]])
+            at += prog.partitions[n]["size"]
+        best = cost(cur)
+        improved = True
+        while improved:
+            improved = False
+            pick = None
+            for ia, a in enumerate(names):
+                for b in names[ia + 1:]:
+                    for i in range(len(cur[a])):
+                        for j in range(len(cur[b])):
+                            nxt = dict(cur)
+                            la, lb = list(cur[a]), list(cur[b])
+                            la[i], lb[j] = lb[j], la[i]
+                            nxt[a], nxt[b] = tuple(la), tuple(lb)
+                            c = cost(nxt)
+                            if c is None:
+                                continue
+                            bar = pick[2] if pick is not None else (best[2] if best is not None else math.inf)
+                            if c[2] < bar * (1.0 - 1e-12):
+                                pick = (nxt, c[1], c[2])
+            if pick is not None:
+                cur = pick[0]
+                best = ({n: tuple(sorted(v)) for n, v in pick[0].items()}, pick[1], pick[2])
+                improved = True
     if best is None:
         raise ValueError("no membership makes the program valid")
     return best

@@ -1259,31 +1259,129 @@ extern "C" ja_status_t ja_exprog_synthesize(ja_exprog_t* p, const ja_machine_t* 
     if (ms) *ms = best.first;
     return JA_OK;
 }
+// memberships above this count are searched by pairwise swaps instead of being enumerated
+constexpr int64_t PLACE_ENUMERATION_LIMIT = 5000;
+namespace {
+int64_t count_memberships(const Prog& p) {      // the multinomial, capped well above the limit
+    std::set<int> taken;
+    int64_t n_free = 0;
+    for (const ExPartition& q : p.parts)
+        if (q.bound) taken.insert(q.members.begin(), q.members.end());
+    for (int s : p.gpus) n_free += !taken.count(s);
+    double total = 1.0;
+    for (const ExPartition& q : p.parts) {
+        if (q.bound) continue;
+        double c = 1.0;
+        for (int i = 0; i < q.size; ++i) c = c * (double)(n_free - i) / (double)(i + 1);
+        total *= c;
+        n_free -= q.size;
+        if (total > 1e15) return (int64_t)1e15;
+    }
+    return (int64_t)(total + 0.5);
+}
+}  // namespace
+
 extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machine, int32_t body, double* ms) {
     if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
     ja_status_t s = check_machine(machine, *p);
     if (s != JA_OK) return s;
     if (body < JA_BODY_OWN || body > JA_BODY_BEST) return ja_fail(JA_ERR_INVALID_ARG, "body %d", body);
-    std::vector<std::vector<std::vector<int>>> all;
-    enumerate_memberships(*p, &all);
     bool found = false;
     Prog best;
     double best_ms = 0;
-    for (const auto& mem : all) {
-        Prog q = *p;
-        bind_membership(&q, mem);
-        Prog c;
-        double t;
-        if (!best_constructed(q, *machine, body, &c, &t)) continue;
-        if (!found || t < best_ms * (1.0 - 1e-12)) {
-            best = c;
-            best_ms = t;
-            found = true;
+    if (count_memberships(*p) <= PLACE_ENUMERATION_LIMIT) {
+        std::vector<std::vector<std::vector<int>>> all;
+        enumerate_memberships(*p, &all);
+        for (const auto& mem : all) {
+            Prog q = *p;
+            bind_membership(&q, mem);
+            Prog c;
+            double t;
+            if (!best_constructed(q, *machine, body, &c, &t)) continue;
+            if (!found || t < best_ms * (1.0 - 1e-12)) {
+                best = c;
+                best_ms = t;
+                found = true;
+            }
+        }
+    } else {
+        // steepest descent over exchanges of two sites between partitions, from the first membership in enumeration order
+        // (the free sites dealt to the size-declared partitions in ascending order)
+        std::vector<int> unbound;
+        std::set<int> taken;
+        for (size_t i = 0; i < p->parts.size(); ++i) {
+            if (p->parts[i].bound) taken.insert(p->parts[i].members.begin(), p->parts[i].members.end());
+            else unbound.push_back((int)i);
+        }
+        std::vector<std::vector<int>> cur;
+        {
+            std::vector<int> free_sites;
+            for (int g : p->gpus)
+                if (!taken.count(g)) free_sites.push_back(g);
+            size_t at = 0;
+            for (int k : unbound) {
+                cur.push_back(std::vector<int>(free_sites.begin() + at, free_sites.begin() + at + p->parts[k].size));
+                at += p->parts[k].size;
+            }
+        }
+        auto cost_of = [&](const std::vector<std::vector<int>>& mem, Prog* c, double* t) {
+            Prog q = *p;
+            bind_membership(&q, mem);
+            return best_constructed(q, *machine, body, c, t);
+        };
+        found = cost_of(cur, &best, &best_ms);
+        bool improved = true;
+        while (improved) {
+            improved = false;
+            std::vector<std::vector<int>> pick;
+            Prog pick_prog;
+            double pick_ms = 0;
+            bool any = false;
+            for (size_t a = 0; a < cur.size(); ++a)
+                for (size_t b = a + 1; b < cur.size(); ++b)
+                    for (size_t i = 0; i < cur[a].size(); ++i)
+                        for (size_t j = 0; j < cur[b].size(); ++j) {
+                            std::vector<std::vector<int>> nxt = cur;
+                            std::swap(nxt[a][i], nxt[b][j]);
+                            Prog c;
+                            double t;
+                            if (!cost_of(nxt, &c, &t)) continue;
+                            const double bar = any ? pick_ms : (found ? best_ms : INFINITY);
+                            if (t < bar * (1.0 - 1e-12)) {
+                                pick = nxt;
+                                pick_prog = c;
+                                pick_ms = t;
+                                any = true;
+                            }
+                        }
+            if (any) {
+                cur = pick;
+                best = pick_prog;
+                best_ms = pick_ms;
+                found = true;
+                improved = true;
+            }
         }
     }
     if (!found) return ja_fail(JA_ERR_INVALID_ARG, "no membership makes the program valid");
     *p = best;
     if (ms) *ms = best_ms;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exprog_bind_members(ja_exprog_t* p, const char* partition, const int32_t* sites, int32_t n) {
+    if (!p || !partition || !sites) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    const int k = find_part(*p, partition);
+    if (k < 0) return ja_fail(JA_ERR_INVALID_ARG, "no partition '%s'", partition);
+    if (p->parts[k].bound) return ja_fail(JA_ERR_INVALID_ARG, "partition '%s' already has members", partition);
+    if (n != p->parts[k].size) return ja_fail(JA_ERR_INVALID_ARG, "partition '%s' has size %d", partition, p->parts[k].size);
+    Prog q = *p;
+    q.parts[k].members.assign(sites, sites + n);
+    std::sort(q.parts[k].members.begin(), q.parts[k].members.end());
+    q.parts[k].bound = true;
+    ja_status_t st = check_static(q);
+    if (st != JA_OK) return st;
+    *p = q;
     return JA_OK;
 }
 
@@ -1664,6 +1762,13 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
     scratch += (table_bytes + 255) / 256 * 256;
 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        JA_CUDA(cudaStreamIsCapturing(stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone)
+            return ja_fail(JA_ERR_UNSUPPORTED, "ja_exchange_execute was called on a stream that is being captured: its box tables are staged from "
+                                               "host memory of this call, which a replay would read too late");
+    }
     char* pool = nullptr;
     cudaMemPool_t mp = nullptr;
     if ((st = exchange_pool(&mp)) != JA_OK) return st;

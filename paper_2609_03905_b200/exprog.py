@@ -33,6 +33,7 @@ def _declare():
         "ja_exprog_num_memberships": [vp, P(i64)],
         "ja_exprog_bind": [vp, i64],
         "ja_exprog_membership": [vp, ctypes.c_char_p, P(u64)],
+        "ja_exprog_bind_members": [vp, ctypes.c_char_p, P(i32), i32],
         "ja_exprog_closure": [vp, P(i64), P(u64), P(i32)],
         "ja_exprog_check": [vp, P(i32), P(i32)],
         "ja_exprog_valid_any": [vp, P(i32)],
@@ -133,6 +134,10 @@ def ja_exprog_membership(prog: int, partition: str) -> int:
     m = ctypes.c_uint64()
     _check(LIB.ja_exprog_membership(prog, partition.encode(), ctypes.byref(m)))
     return m.value
+
+
+def ja_exprog_bind_members(prog: int, partition: str, sites):
+    _check(LIB.ja_exprog_bind_members(prog, partition.encode(), (ctypes.c_int32 * len(sites))(*[int(x) for x in sites]), len(sites)))
 
 
 def ja_exprog_closure(prog: int):

@@ -164,3 +164,25 @@ def test_the_local_aggregation_primitive(n_parts, agg, dtype):
     with pytest.raises(JaError) as e:
         X.ja_exchange_combine([parts[0].data_ptr(), parts[1].data_ptr()], out.data_ptr(), 40, 1, "sum")
     assert e.value.status_name == "JA_ERR_ALIGNMENT"
+
+
+def test_exchange_refuses_a_stream_that_is_being_captured():
+    c = CASES["preamble"]
+    h, q = build("preamble", "naive")
+    rP = upload(si.normal([2] + c["ext"], 0.0, 1.0, BF, 1, 3), blocked.partial_splits(2, c["ps"]))
+    rD = empty_like_tiling(c["ext"], c["cs"], BF)
+    h.execute(rP, c["copy_site"], c["specs"], "sum", rD)                      # outside any capture: fine
+    torch.cuda.synchronize()
+    want = download_bits(rD).copy()
+    g = torch.cuda.CUDAGraph()
+    marker = torch.zeros(1, device="cuda")
+    with torch.cuda.graph(g):
+        marker.add_(1.0)                                                        # so that the capture is not empty
+        with pytest.raises(JaError, match="captured") as e:
+            h.execute(rP, c["copy_site"], c["specs"], "sum", rD)
+        assert e.value.status_name == "JA_ERR_UNSUPPORTED"
+    g.replay()
+    torch.cuda.synchronize()
+    assert marker.item() == 1.0 and np.array_equal(download_bits(rD), want)    # the refused call recorded nothing
+    X.ja_exchange_trim()
+    check_status()
