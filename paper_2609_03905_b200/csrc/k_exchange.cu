@@ -5,12 +5,28 @@
 
 namespace {
 
-// 16-byte accesses when every offset, pitch and run of the launch allows, else one cell per access
+// 16-byte accesses when every offset, pitch and run of the launch allows, else one cell per access. Long runs: a CTA takes whole
+// runs (the run's two offsets are computed once, the threads stride along it); short runs: the box is walked as one flat range.
 template <typename V>
 __global__ void __launch_bounds__(256) box_copy_kernel(const char* __restrict__ src, char* __restrict__ dst,
                                                         const JaBoxCopy* __restrict__ boxes) {
     const JaBoxCopy b = boxes[blockIdx.y];
-    const int64_t per_row = b.run_bytes / (int64_t)sizeof(V), rows = b.n0 * b.n1, total = rows * per_row;
+    const int64_t per_row = b.run_bytes / (int64_t)sizeof(V), rows = b.n0 * b.n1;
+    if (per_row >= 256) {
+        for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+            const int64_t r0 = row / b.n1, r1 = row - r0 * b.n1;
+            const V* s = reinterpret_cast<const V*>(src + b.src_off + r0 * b.src_pitch0 + r1 * b.src_pitch1);
+            V* d = reinterpret_cast<V*>(dst + b.dst_off + r0 * b.dst_pitch0 + r1 * b.dst_pitch1);
+            int64_t x = threadIdx.x;
+            for (; x + 768 < per_row; x += 1024) {          // four independent accesses in flight per thread
+                const V v0 = s[x], v1 = s[x + 256], v2 = s[x + 512], v3 = s[x + 768];
+                d[x] = v0; d[x + 256] = v1; d[x + 512] = v2; d[x + 768] = v3;
+            }
+            for (; x < per_row; x += 256) d[x] = s[x];
+        }
+        return;
+    }
+    const int64_t total = rows * per_row;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t row = i / per_row, x = i - row * per_row, r0 = row / b.n1, r1 = row - r0 * b.n1;
         const V v = *reinterpret_cast<const V*>(src + b.src_off + r0 * b.src_pitch0 + r1 * b.src_pitch1 + x * (int64_t)sizeof(V));
