@@ -15,7 +15,7 @@ Text form accepted (a reading of the printed examples):
 An action with an arrow has one source site; without an arrow the source may be a list of sites or a partition name
 (one local aggregation per site).
 
-Readings where the paper is silent (each also listed in the design notes of the repository):
+Readings where the paper is silent:
   * all atoms of one aggregate are copies of one tensor block, so an aggregate has the size of any of its atoms;
   * a local aggregation of m >= 2 materialised parts reads m and writes 1 block of that size at the site's HBM bandwidth;
     an aggregate that is already materialised at the source costs nothing (m = 1);
