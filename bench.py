@@ -929,8 +929,16 @@ def case_results(case, reps):
                 # HBM traffic on this GPU: decompose reads and writes every copy once, recompose the tensor once, a transfer reads
                 # and writes its atom, an aggregation reads its parts and writes one atom
                 nbytes = 2.0 * m * T * d * 2 + 2.0 * T * d * 2 + 2.0 * stats["transfer_bytes"] + stats["aggregation_bytes"]
+                # the same program as an exchange plan: buffers and tables resident, one stream per site (dataflow), and the
+                # plan's run captured into a CUDA graph and replayed
+                plan = X.ExchangePlan(h, P, copy_site, specs, "sum", y)
+                tp = timeit(lambda r: plan.run(), reps, True)
+                tg = timeit_graph(lambda r: plan.run(), reps, True)
+                plan.close()
                 res["%s_%s" % (tag, "synthesised" if body == "best" else body)] = {
-                    **hb(nbytes, t), "simulated_ms_hgx_b200_nominal": sim, "actions": len(acts), "aggregations": stats["aggregations"],
+                    **hb(nbytes, t), "plan_dataflow_ms": tp["ms_mean"], "plan_graph_replay_ms": tg["ms_mean"],
+                    "plan_graph_replay_frac_of_measured_hbm": nbytes / (tg["ms_mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "simulated_ms_hgx_b200_nominal": sim, "actions": len(acts), "aggregations": stats["aggregations"],
                     "transfers": stats["transfers"], "transfer_MB": stats["transfer_bytes"] / 1e6, "scratch_MB": stats["scratch_bytes"] / 1e6}
             res["%s_fused_aggregating_relayout" % tag] = hb((m + 1.0) * T * d * 2, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
             del P, y

@@ -162,7 +162,7 @@ ja_status_t ja_exprog_preamble(int32_t rank, const int64_t* producer_splits, con
  * combines them in ascending order of their first atoms in f32 (SUM or MAX) and rounds once to the cell type, a transfer
  * one device-to-device copy -- and recompose (the aggregated atoms at the site of function spec i are concatenated into
  * the block it consumes; a block consumed by several specs is written from the lowest one).  At most 16 parts per
- * aggregation, tensors of rank <= 3.  Scratch memory for the atom buffers comes from a stream-ordered memory pool of the
+ * aggregation, tensors of rank <= 3; a second delivery of an aggregate to a site that already holds it moves nothing.  Scratch memory for the atom buffers comes from a stream-ordered memory pool of the
  * library's own and goes back to it, in stream order, at the end of the call; the pool keeps it for the next call until
  * ja_exchange_trim (which the caller synchronises before) hands it back to the driver.  Not capturable: a call on a stream
  * that is being captured is refused (JA_ERR_UNSUPPORTED, nothing enqueued); the call may block the host briefly while its
@@ -172,6 +172,25 @@ ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* pa
                                 const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
                                 int64_t* stats, void* cuda_stream);
 ja_status_t ja_exchange_trim(void);
+
+/* ---- an exchange plan: the executable artifact (Section 5.1: "a CUDA graph in which each vertex is a GPU kernel or a
+ * network operation") ---------------------------------------------------------------------------------------------------
+ * ja_exchange_plan_create does once what ja_exchange_execute does per call -- checks, firing order, buffers, tables --
+ * and keeps the atom buffers and tables in device memory of its own (synchronous cudaMalloc / cudaMemcpy; JA_ERR_OOM if
+ * the buffers do not fit).  The relations' payload addresses are bound into the plan: both relations must outlive it
+ * and keep their payloads in place; what the payloads hold may change between runs.
+ * ja_exchange_plan_run only enqueues: decompose on `cuda_stream`; then every step on the stream of its SITE (the plan
+ * owns one stream per site that acts), after the events of the buffers that other sites' streams write -- so actions
+ * proceed as dataflow allows, as Section 5.2 says a program does, and transfers (copy engines) overlap aggregations --
+ * then recompose on `cuda_stream` once every site's stream has been joined.  It may be called while `cuda_stream` is
+ * being captured: the capture then holds the program's dependency graph, and replaying it needs no host work.  Runs of
+ * one plan must not overlap (they share the buffers); the results are those of ja_exchange_execute, bit for bit. */
+typedef struct ja_exchange_plan ja_exchange_plan_t;
+ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                    const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                    int64_t* stats, ja_exchange_plan_t** out);
+ja_status_t ja_exchange_plan_run(ja_exchange_plan_t* plan, void* cuda_stream);
+void ja_exchange_plan_destroy(ja_exchange_plan_t* plan);
 
 /* ---- the pieces a program needs when its sites are different processes (one per GPU) ------------------------------------
  * ja_exprog_schedule: the firing order ja_exchange_execute uses, for a driver that issues the actions itself: fired action

@@ -1629,9 +1629,39 @@ extern "C" ja_status_t ja_exchange_trim(void) {
 // The sites of the program are regions of this GPU's memory; a transfer is a device-to-device copy (on a machine with
 // several GPUs it would be a peer copy), a local aggregation one launch of the combine kernel, decompose and recompose
 // one batched box-copy launch each. Actions are issued on one stream in a firing order of the program.
-extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
-                                           const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
-                                           int64_t* stats, void* cuda_stream) {
+namespace {
+
+// Everything ja_exchange_execute and an exchange plan need beyond the relations' payloads, worked out on the host.
+struct ExBuffer {
+    int site;
+    uint64_t agg;
+    int64_t off, bytes;
+    int producer_site;      // whose stream writes it: -1 = decompose (before the sites' streams fork)
+};
+struct ExStep {
+    int site;
+    int out;                        // buffer of the aggregate at the source
+    std::vector<int> parts;         // >= 2: a local aggregation into `out`; 1: `out` is already materialised
+    std::vector<int> dests;         // buffers the aggregate is transferred to
+};
+struct ExBuild {
+    std::vector<ExBuffer> bufs;
+    std::vector<ExStep> steps;
+    std::vector<JaBoxCopy> boxes;   // n_in decompose boxes, then n_out recompose boxes
+    int n_in = 0, n_out = 0;
+    bool vec_in = true, vec_out = true;
+    int64_t max_in = 0, max_out = 0, scratch = 0, table_off = 0, table_bytes = 0;
+    int64_t n_aggregations = 0, n_transfers = 0, transfer_bytes = 0, aggregation_bytes = 0;
+    std::vector<int> sites;         // the sites that run a step
+    ja_dtype_t dtype = JA_BF16;
+    int esize = 2;
+    ja_agg_t agg = JA_AGG_SUM;
+    const char* src_base = nullptr;
+    char* dst_base = nullptr;
+};
+
+ja_status_t build_exchange(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site, const int32_t* consumer_specs,
+                           int32_t n_specs, ja_agg_t agg, ja_relation_t* dst, ExBuild* B) {
     ja_status_t st = need_bound(prog);
     if (st != JA_OK) return st;
     if (!partials || !dst || !copy_site || !consumer_specs || n_specs < 1) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
@@ -1642,6 +1672,7 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
         if (partials->extent[d + 1] != dst->extent[d]) return ja_fail(JA_ERR_SHAPE, "extent of dimension %d differs", d);
     if (partials->dtype != dst->dtype) return ja_fail(JA_ERR_DTYPE, "the exchange moves and aggregates atoms in the partial relation's cell type: the consumer relation must have it too");
     if (partials->base == dst->base) return ja_fail(JA_ERR_INVALID_ARG, "the consumer relation aliases the partial relation");
+    if (rank > 3) return ja_fail(JA_ERR_UNSUPPORTED, "tensors of rank above 3");
     const int m = (int)partials->extent[0];
     if (agg != JA_AGG_SUM && agg != JA_AGG_MAX && !(agg == JA_AGG_NONE && m == 1))
         return ja_fail(JA_ERR_INVALID_ARG, "%d copies of every atom need SUM or MAX aggregation", m);
@@ -1663,6 +1694,11 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
     if (!same) return ja_fail(JA_ERR_INVALID_ARG, "the program's preamble is not the one these relations, copy sites and function specs generate");
     if (!valid_bound(*prog)) return ja_fail(JA_ERR_INVALID_ARG, "the program is not valid (Definition \"Closure; validity\")");
 
+    B->dtype = partials->dtype;
+    B->esize = partials->esize;
+    B->agg = agg;
+    B->src_base = (const char*)partials->base;
+    B->dst_base = (char*)dst->base;
     // firing order and the parts of every aggregation
     std::vector<Flat> acts;
     expand(*prog, &acts);
@@ -1674,30 +1710,49 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
         const OverlayCell& ce = ov.cells[ov.atom_jc[a].first];
         int64_t cells = 1;
         for (int d = 0; d < rank; ++d) cells *= ce.hi[d] - ce.lo[d];
-        return cells * partials->esize;
+        return cells * (int64_t)partials->esize;
     };
-    std::map<std::pair<int, uint64_t>, int64_t> buf;     // (site, aggregate) -> offset in the scratch allocation
-    int64_t scratch = 0;
-    auto alloc = [&](int site, uint64_t x) {
+    std::map<std::pair<int, uint64_t>, int> index;
+    auto buffer = [&](int site, uint64_t x, int producer_site) {
         auto key = std::make_pair(site, x);
-        if (buf.count(key)) return;
-        buf[key] = scratch;
-        scratch += (atom_bytes(x) + 255) / 256 * 256;
+        auto it = index.find(key);
+        if (it != index.end()) return it->second;
+        B->bufs.push_back({site, x, B->scratch, atom_bytes(x), producer_site});
+        B->scratch += (atom_bytes(x) + 255) / 256 * 256;
+        index[key] = (int)B->bufs.size() - 1;
+        return (int)B->bufs.size() - 1;
     };
-    for (size_t a = 0; a < prog->atoms.size(); ++a) alloc(prog->atoms[a].site, 1ull << a);
-    int64_t n_aggregations = 0, n_transfers = 0, transfer_bytes = 0, aggregation_bytes = 0;
+    for (size_t a = 0; a < prog->atoms.size(); ++a) buffer(prog->atoms[a].site, 1ull << a, -1);
+    std::set<int> step_sites;
     for (const Fired& f : order) {
         const Flat& a = acts[f.act];
         if (f.parts.size() > JA_EXCHANGE_MAX_PARTS)
             return ja_fail(JA_ERR_UNSUPPORTED, "an aggregation of %d parts (at most %d)", (int)f.parts.size(), JA_EXCHANGE_MAX_PARTS);
-        alloc(a.site, a.agg);
-        for (int d : a.dests) alloc(d, a.agg);
+        ExStep stp;
+        stp.site = a.site;
+        for (uint64_t y : f.parts) stp.parts.push_back(index.at({a.site, y}));
+        stp.out = buffer(a.site, a.agg, a.site);
+        if (f.parts.size() >= 2) {
+            ++B->n_aggregations;
+            B->aggregation_bytes += ((int64_t)f.parts.size() + 1) * atom_bytes(a.agg);
+        }
+        for (int d : a.dests) {
+            const bool fresh = !index.count({d, a.agg});
+            const int b = buffer(d, a.agg, a.site);
+            if (fresh && b != stp.out) {               // a second delivery of an aggregate that is already there moves nothing
+                stp.dests.push_back(b);
+                ++B->n_transfers;
+                B->transfer_bytes += atom_bytes(a.agg);
+            }
+        }
+        if (f.parts.size() >= 2 || !stp.dests.empty()) {
+            step_sites.insert(a.site);
+            B->steps.push_back(stp);
+        }
     }
+    B->sites.assign(step_sites.begin(), step_sites.end());
     // decompose and recompose tables
     const int64_t ntrail = partials->nblocks / m;
-    std::vector<JaBoxCopy> boxes;
-    bool vec_in = true, vec_out = true;
-    int64_t max_in = 0, max_out = 0;
     auto box_of = [&](const OverlayCell& ce, const std::vector<std::vector<int64_t>>& tiling, int64_t blk, int64_t blk_off, bool from_block, int64_t buf_off) {
         // the block's extents and the box's offset inside it, padded to three dimensions in front
         int64_t bext[3] = {1, 1, 1}, off[3] = {0, 0, 0}, n[3] = {1, 1, 1};
@@ -1729,16 +1784,15 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
     auto aligned16 = [](const JaBoxCopy& b) {
         return ((b.src_off | b.dst_off | b.src_pitch0 | b.src_pitch1 | b.dst_pitch0 | b.dst_pitch1 | b.run_bytes) & 15) == 0;
     };
-    if (rank > 3) return ja_fail(JA_ERR_UNSUPPORTED, "tensors of rank above 3");
     for (size_t a = 0; a < prog->atoms.size(); ++a) {
         const OverlayCell& ce = ov.cells[ov.atom_jc[a].first];
         const int c = ov.atom_jc[a].second;
-        const JaBoxCopy b = box_of(ce, ps, ce.pb, partials->blk_off[c * ntrail + ce.pb], true, buf[{prog->atoms[a].site, 1ull << a}]);
-        vec_in = vec_in && aligned16(b);
-        max_in = std::max(max_in, b.n0 * b.n1 * b.run_bytes);
-        boxes.push_back(b);
+        const JaBoxCopy b = box_of(ce, ps, ce.pb, partials->blk_off[c * ntrail + ce.pb], true, B->bufs[index.at({prog->atoms[a].site, 1ull << a})].off);
+        B->vec_in = B->vec_in && aligned16(b);
+        B->max_in = std::max(B->max_in, b.n0 * b.n1 * b.run_bytes);
+        B->boxes.push_back(b);
     }
-    const int n_in = (int)boxes.size();
+    B->n_in = (int)B->boxes.size();
     std::set<int64_t> done;
     for (int i = 0; i < n_specs; ++i) {
         const int site = prog->parts[i].members[0];
@@ -1748,72 +1802,171 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
             uint64_t x = 0;
             for (size_t a = 0; a < prog->atoms.size(); ++a)
                 if (ov.atom_jc[a].first == ce.j) x |= 1ull << a;
-            auto it = buf.find({site, x});
-            if (it == buf.end()) return ja_fail(JA_ERR_INVALID_ARG, "internal: a required aggregate was never materialised");
-            const JaBoxCopy b = box_of(ce, cs, ce.cb, dst->blk_off[ce.cb], false, it->second);
-            vec_out = vec_out && aligned16(b);
-            max_out = std::max(max_out, b.n0 * b.n1 * b.run_bytes);
-            boxes.push_back(b);
+            auto it = index.find({site, x});
+            if (it == index.end()) return ja_fail(JA_ERR_INVALID_ARG, "internal: a required aggregate was never materialised");
+            const JaBoxCopy b = box_of(ce, cs, ce.cb, dst->blk_off[ce.cb], false, B->bufs[it->second].off);
+            B->vec_out = B->vec_out && aligned16(b);
+            B->max_out = std::max(B->max_out, b.n0 * b.n1 * b.run_bytes);
+            B->boxes.push_back(b);
         }
     }
-    const int n_out = (int)boxes.size() - n_in;
-    const int64_t table_bytes = (int64_t)boxes.size() * (int64_t)sizeof(JaBoxCopy);
-    const int64_t table_off = scratch;
-    scratch += (table_bytes + 255) / 256 * 256;
+    B->n_out = (int)B->boxes.size() - B->n_in;
+    B->table_bytes = (int64_t)B->boxes.size() * (int64_t)sizeof(JaBoxCopy);
+    B->table_off = B->scratch;
+    B->scratch += (B->table_bytes + 255) / 256 * 256;
+    return JA_OK;
+}
 
+void fill_stats(const ExBuild& B, int64_t* stats) {
+    if (!stats) return;
+    stats[0] = B.n_aggregations;
+    stats[1] = B.n_transfers;
+    stats[2] = B.transfer_bytes;
+    stats[3] = B.scratch;
+    stats[4] = B.aggregation_bytes;
+}
+
+// one step on `stream`: the local aggregation, then the transfers
+ja_status_t issue_step(const ExBuild& B, const ExStep& s, char* pool, cudaStream_t stream) {
+    char* here = pool + B.bufs[s.out].off;
+    if (s.parts.size() >= 2) {
+        const void* parts[JA_EXCHANGE_MAX_PARTS];
+        for (size_t k = 0; k < s.parts.size(); ++k) parts[k] = pool + B.bufs[s.parts[k]].off;
+        ja_status_t rc = ja_launch_exchange_combine(parts, (int)s.parts.size(), here, B.bufs[s.out].bytes, B.dtype, B.agg, stream);
+        if (rc != JA_OK) return rc;
+    }
+    for (int d : s.dests)
+        if (cudaMemcpyAsync(pool + B.bufs[d].off, here, (size_t)B.bufs[s.out].bytes, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+            return ja_fail(JA_ERR_CUDA, "a transfer failed");
+    return JA_OK;
+}
+
+}  // namespace
+
+extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                           const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                           int64_t* stats, void* cuda_stream) {
+    ExBuild B;
+    ja_status_t st = build_exchange(prog, partials, copy_site, consumer_specs, n_specs, agg, dst, &B);
+    if (st != JA_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     {
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         JA_CUDA(cudaStreamIsCapturing(stream, &cap));
         if (cap != cudaStreamCaptureStatusNone)
             return ja_fail(JA_ERR_UNSUPPORTED, "ja_exchange_execute was called on a stream that is being captured: its box tables are staged from "
-                                               "host memory of this call, which a replay would read too late");
+                                               "host memory of this call, which a replay would read too late (an exchange plan can be captured)");
     }
     char* pool = nullptr;
     cudaMemPool_t mp = nullptr;
     if ((st = exchange_pool(&mp)) != JA_OK) return st;
-    JA_CUDA(cudaMallocFromPoolAsync((void**)&pool, (size_t)scratch, mp, stream));
+    JA_CUDA(cudaMallocFromPoolAsync((void**)&pool, (size_t)B.scratch, mp, stream));
     ja_status_t rc = JA_OK;
     do {
-        if (cudaMemcpyAsync(pool + table_off, boxes.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        if (cudaMemcpyAsync(pool + B.table_off, B.boxes.data(), (size_t)B.table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
             rc = ja_fail(JA_ERR_CUDA, "copying the box tables failed");
             break;
         }
-        const JaBoxCopy* d_boxes = (const JaBoxCopy*)(pool + table_off);
-        if ((rc = ja_launch_box_copies((const char*)partials->base, pool, d_boxes, n_in, max_in, vec_in, partials->esize, stream)) != JA_OK) break;
-        for (const Fired& f : order) {
-            const Flat& a = acts[f.act];
-            char* here = pool + buf[{a.site, a.agg}];
-            if (f.parts.size() >= 2) {
-                const void* parts[JA_EXCHANGE_MAX_PARTS];
-                for (size_t k = 0; k < f.parts.size(); ++k) parts[k] = pool + buf[{a.site, f.parts[k]}];
-                if ((rc = ja_launch_exchange_combine(parts, (int)f.parts.size(), here, atom_bytes(a.agg), partials->dtype, agg, stream)) != JA_OK) break;
-                ++n_aggregations;
-                aggregation_bytes += ((int64_t)f.parts.size() + 1) * atom_bytes(a.agg);
-            }
-            for (int d : a.dests) {
-                char* there = pool + buf[{d, a.agg}];
-                if (there == here) continue;
-                if (cudaMemcpyAsync(there, here, (size_t)atom_bytes(a.agg), cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
-                    rc = ja_fail(JA_ERR_CUDA, "a transfer failed");
-                    break;
-                }
-                ++n_transfers;
-                transfer_bytes += atom_bytes(a.agg);
-            }
-            if (rc != JA_OK) break;
-        }
+        const JaBoxCopy* d_boxes = (const JaBoxCopy*)(pool + B.table_off);
+        if ((rc = ja_launch_box_copies(B.src_base, pool, d_boxes, B.n_in, B.max_in, B.vec_in, B.esize, stream)) != JA_OK) break;
+        for (const ExStep& s : B.steps)
+            if ((rc = issue_step(B, s, pool, stream)) != JA_OK) break;
         if (rc != JA_OK) break;
-        rc = ja_launch_box_copies(pool, (char*)dst->base, d_boxes + n_in, n_out, max_out, vec_out, partials->esize, stream);
+        rc = ja_launch_box_copies(pool, B.dst_base, d_boxes + B.n_in, B.n_out, B.max_out, B.vec_out, B.esize, stream);
     } while (false);
     cudaFreeAsync(pool, stream);
     if (rc != JA_OK) return rc;
-    if (stats) {
-        stats[0] = n_aggregations;
-        stats[1] = n_transfers;
-        stats[2] = transfer_bytes;
-        stats[3] = scratch;
-        stats[4] = aggregation_bytes;
-    }
+    fill_stats(B, stats);
     return JA_OK;
+}
+
+// ---- an exchange plan: the same program with its buffers and tables kept on the device, issued as dataflow ------------------
+// Every site that runs a step has a stream of its own; a step waits for the buffers other sites' streams write (events), so what
+// a capture of ja_exchange_plan_run records is the program's dependency graph -- kernels and copies as vertices -- and actions of
+// different sites may run at the same time, copies on the copy engines beside the aggregation kernels.
+struct ja_exchange_plan {
+    ExBuild B;
+    char* pool = nullptr;
+    int device = 0;
+    std::map<int, cudaStream_t> stream;       // per site
+    std::vector<cudaEvent_t> ready;           // per buffer: written
+    std::map<int, cudaEvent_t> done;          // per site: its last step issued
+    cudaEvent_t start = nullptr;
+};
+
+extern "C" void ja_exchange_plan_destroy(ja_exchange_plan_t* p) {
+    if (!p) return;
+    for (auto& kv : p->stream) cudaStreamDestroy(kv.second);
+    for (cudaEvent_t e : p->ready)
+        if (e) cudaEventDestroy(e);
+    for (auto& kv : p->done) cudaEventDestroy(kv.second);
+    if (p->start) cudaEventDestroy(p->start);
+    if (p->pool) cudaFree(p->pool);
+    delete p;
+}
+
+extern "C" ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                               const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                               int64_t* stats, ja_exchange_plan_t** out) {
+    if (!out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    ja_exchange_plan* p = new ja_exchange_plan();
+    ja_status_t st = build_exchange(prog, partials, copy_site, consumer_specs, n_specs, agg, dst, &p->B);
+    if (st != JA_OK) {
+        delete p;
+        return st;
+    }
+    const ExBuild& B = p->B;
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->pool, (size_t)B.scratch);
+    if (e == cudaSuccess) e = cudaMemcpy(p->pool + B.table_off, B.boxes.data(), (size_t)B.table_bytes, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->start, cudaEventDisableTiming);
+    p->ready.assign(B.bufs.size(), nullptr);
+    for (size_t i = 0; e == cudaSuccess && i < B.bufs.size(); ++i)
+        if (B.bufs[i].producer_site >= 0) e = cudaEventCreateWithFlags(&p->ready[i], cudaEventDisableTiming);
+    for (size_t i = 0; e == cudaSuccess && i < B.sites.size(); ++i) {
+        cudaStream_t s = nullptr;
+        e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+        if (e == cudaSuccess) p->stream[B.sites[i]] = s;
+        cudaEvent_t ev = nullptr;
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e == cudaSuccess) p->done[B.sites[i]] = ev;
+    }
+    if (e != cudaSuccess) {
+        ja_exchange_plan_destroy(p);
+        return ja_fail(e == cudaErrorMemoryAllocation ? JA_ERR_OOM : JA_ERR_CUDA, "exchange plan: %s", cudaGetErrorString(e));
+    }
+    fill_stats(B, stats);
+    *out = p;
+    return JA_OK;
+}
+
+extern "C" ja_status_t ja_exchange_plan_run(ja_exchange_plan_t* p, void* cuda_stream) {
+    if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null plan");
+    const ExBuild& B = p->B;
+    cudaStream_t user = (cudaStream_t)cuda_stream;
+    const JaBoxCopy* d_boxes = (const JaBoxCopy*)(p->pool + B.table_off);
+    ja_status_t rc = ja_launch_box_copies(B.src_base, p->pool, d_boxes, B.n_in, B.max_in, B.vec_in, B.esize, user);
+    if (rc != JA_OK) return rc;
+    if (!B.steps.empty()) {
+        // fork: every site's stream starts after decompose
+        JA_CUDA(cudaEventRecord(p->start, user));
+        for (auto& kv : p->stream) JA_CUDA(cudaStreamWaitEvent(kv.second, p->start, 0));
+        for (const ExStep& s : B.steps) {
+            cudaStream_t st = p->stream.at(s.site);
+            for (int b : s.parts)
+                if (B.bufs[b].producer_site >= 0 && B.bufs[b].producer_site != s.site) JA_CUDA(cudaStreamWaitEvent(st, p->ready[b], 0));
+            if (s.parts.size() == 1 && B.bufs[s.out].producer_site >= 0 && B.bufs[s.out].producer_site != s.site)
+                JA_CUDA(cudaStreamWaitEvent(st, p->ready[s.out], 0));
+            if ((rc = issue_step(B, s, p->pool, st)) != JA_OK) return rc;
+            // what this step wrote: its aggregate (if it computed one) and the copies at the destinations
+            if (s.parts.size() >= 2) JA_CUDA(cudaEventRecord(p->ready[s.out], st));
+            for (int d : s.dests) JA_CUDA(cudaEventRecord(p->ready[d], st));
+        }
+        // join
+        for (auto& kv : p->stream) {
+            JA_CUDA(cudaEventRecord(p->done.at(kv.first), kv.second));
+            JA_CUDA(cudaStreamWaitEvent(user, p->done.at(kv.first), 0));
+        }
+    }
+    return ja_launch_box_copies(p->pool, B.dst_base, d_boxes + B.n_in, B.n_out, B.max_out, B.vec_out, B.esize, user);
 }

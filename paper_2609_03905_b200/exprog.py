@@ -46,12 +46,16 @@ def _declare():
         "ja_exprog_preamble": [i32, P(i64), P(i32), P(i64), P(i32), i32, P(i32), P(i32), i32, i32, P(vp)],
         "ja_exchange_execute": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i64), vp],
         "ja_exprog_schedule": [vp, P(i32), P(i32), P(i32), P(i32), P(u64)],
+        "ja_exchange_plan_create": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i64), P(vp)],
+        "ja_exchange_plan_run": [vp, vp],
         "ja_exchange_combine": [P(vp), i32, vp, i64, ctypes.c_int, ctypes.c_int, vp],
     }
     for name, argtypes in sigs.items():
         fn = getattr(LIB, name)
         fn.argtypes = argtypes
         fn.restype = ctypes.c_int
+    LIB.ja_exchange_plan_destroy.argtypes = [vp]
+    LIB.ja_exchange_plan_destroy.restype = None
     LIB.ja_exchange_trim.argtypes = []
     LIB.ja_exchange_trim.restype = ctypes.c_int
     LIB.ja_exprog_destroy.argtypes = [vp]
@@ -237,8 +241,52 @@ def ja_exchange_combine(part_ptrs, out_ptr: int, nbytes: int, dtype: int, agg, s
     _check(LIB.ja_exchange_combine(arr, len(part_ptrs), out_ptr, nbytes, dtype, AGG[agg] if isinstance(agg, str) else int(agg), stream))
 
 
+def _stats(stats):
+    return {"aggregations": stats[0], "transfers": stats[1], "transfer_bytes": stats[2], "scratch_bytes": stats[3],
+            "aggregation_bytes": stats[4]}
+
+
+def ja_exchange_plan_create(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int):
+    """Returns (plan handle, statistics)."""
+    from .binding import AGG
+    stats = (ctypes.c_int64 * 5)()
+    h = ctypes.c_void_p()
+    _check(LIB.ja_exchange_plan_create(prog, partials, (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
+                                       (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs),
+                                       AGG[agg] if isinstance(agg, str) else int(agg), dst, stats, ctypes.byref(h)))
+    return h.value, _stats(stats)
+
+
+def ja_exchange_plan_run(plan: int, stream: int = 0):
+    _check(LIB.ja_exchange_plan_run(plan, stream))
+
+
+def ja_exchange_plan_destroy(plan: int):
+    LIB.ja_exchange_plan_destroy(plan)
+
+
 def ja_exchange_trim():
     _check(LIB.ja_exchange_trim())
+
+
+class ExchangePlan:
+    """An exchange plan with its lifetime; keeps the two relations alive, as the plan holds their payload addresses."""
+
+    def __init__(self, prog: "ExchangeProgram", partials, copy_site, consumer_specs, agg, dst):
+        self.partials, self.dst = partials, dst
+        self.handle, self.stats = ja_exchange_plan_create(prog.handle, partials.handle, copy_site, consumer_specs, agg, dst.handle)
+
+    def run(self, stream=None):
+        import torch
+        ja_exchange_plan_run(self.handle, torch.cuda.current_stream().cuda_stream if stream is None else stream)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            ja_exchange_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
 
 
 class ExchangeProgram:
