@@ -142,9 +142,16 @@ def _check_static(prog: Program):
     for s, _ in prog.atoms.values():
         if s not in g:
             raise ValueError("atom at an undeclared site")
-    for agg, _ in prog.out:
+    for agg, tg in prog.out:
         if len({prog.atoms[a][1] for a in agg}) != 1:
             raise ValueError("atoms of one aggregate differ in size")
+        if tg[0] == "sites" and not set(tg[1]) <= g:
+            raise ValueError("OUT names an undeclared site")
+    for agg, src, d in prog.actions:
+        if len({prog.atoms[a][1] for a in agg}) != 1:
+            raise ValueError("atoms of one aggregate differ in size")
+        if not set(d) <= g or (src[0] == "sites" and not set(src[1]) <= g):
+            raise ValueError("an action names an undeclared site")
 
 
 def _name_order(prog):

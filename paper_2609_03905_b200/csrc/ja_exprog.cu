@@ -181,10 +181,18 @@ ja_status_t check_static(const Prog& p) {
             }
         return true;
     };
-    for (const auto& o : p.out)
+    for (const auto& o : p.out) {
         if (!sized(o.first)) return ja_fail(JA_ERR_INVALID_ARG, "the atoms of one aggregate differ in size");
-    for (const ExAction& a : p.actions)
+        for (int t : o.second.sites)
+            if (!g.count(t)) return ja_fail(JA_ERR_INVALID_ARG, "OUT names the undeclared site %d", t);
+    }
+    for (const ExAction& a : p.actions) {
         if (!sized(a.agg)) return ja_fail(JA_ERR_INVALID_ARG, "the atoms of one aggregate differ in size");
+        for (int t : a.src.sites)
+            if (!g.count(t)) return ja_fail(JA_ERR_INVALID_ARG, "an action names the undeclared site %d", t);
+        for (int t : a.dests)
+            if (!g.count(t)) return ja_fail(JA_ERR_INVALID_ARG, "an action names the undeclared site %d", t);
+    }
     return JA_OK;
 }
 

@@ -62,6 +62,9 @@ def test_sizes_round_trip_through_text():
     ("GPUS: 0, 1\nPARTITIONS: P {0, 1} Q {1}\nIN: A @ 0\nOUT: A @ P\n", "JA_ERR_INVALID_ARG"),
     ("GPUS: 0, 1\nIN: A @ 2\nOUT: A @ 0\n", "JA_ERR_INVALID_ARG"),
     ("IN: A @ 0; B @ 0 (size: 2 GB)\nOUT: A+B @ 0\n", "JA_ERR_INVALID_ARG"),
+    ("GPUS: 0, 1\nIN: A @ 0\nOUT: A @ 1\n\nA @ 0 -> 1, 70\n", "JA_ERR_INVALID_ARG"),
+    ("GPUS: 0, 1\nIN: A @ 0\nOUT: A @ 2\n", "JA_ERR_INVALID_ARG"),
+    ("GPUS: 0, 1\nIN: A @ 0; B @ 0 (size: 3 GB)\nOUT: A @ 1\n\nA+B @ 0 -> 1\n", "JA_ERR_INVALID_ARG"),
 ])
 def test_malformed_programs_are_refused(bad, status):
     from paper_2609_03905_b200.binding import JaError
