@@ -473,6 +473,54 @@ def physical_results():
         build(tree)
         workloads[name] = (ops, ja.ja_plan_optimize(ops, 8)[1])
     res = {}
+    # Experiments 3 and 5 in miniature on the simulator: the three plan selectors for the block at p = 8 -- the dynamic program,
+    # greedy (no repartition sub-cost), twenty uniform draws -- by the simulated time of their optimised exchange programs, and
+    # the Pearson correlation between a plan's proxy cost and that time over all 22 plans
+    import random
+    ops = workloads["llama7b_block"][0]
+
+    def valid_specs(op, p_):
+        letters = []
+        for term in op["einsum"].replace("->", ",").split(","):
+            letters += [c for c in term if c not in letters]
+        out = []
+
+        def rec(i, rest, acc):
+            if i == len(letters):
+                if rest == 1:
+                    out.append(dict(zip(letters, acc)))
+                return
+            if letters[i] in op.get("fixed", ()):
+                rec(i + 1, rest, acc + [1])
+                return
+            for c_ in range(1, rest + 1):
+                if rest % c_ == 0 and c_ <= op["extents"][letters[i]]:
+                    rec(i + 1, rest // c_, acc + [c_])
+        rec(0, p_, [])
+        return out
+
+    def pearson(xs, ys):
+        n = len(xs)
+        mx, my = sum(xs) / n, sum(ys) / n
+        sxy = sum((x - mx) * (y - my) for x, y in zip(xs, ys))
+        sxx, syy = sum((x - mx) ** 2 for x in xs), sum((y - my) ** 2 for y in ys)
+        return sxy / (sxx * syy) ** 0.5 if sxx > 0 and syy > 0 else float("nan")
+
+    rng = random.Random(3905)
+    cand = [valid_specs(op, 8) for op in ops]
+    plans = {"optimizer": workloads["llama7b_block"][1], "greedy": ja.ja_plan_select_greedy(ops, 8)[1]}
+    for i in range(20):
+        plans["random_%02d" % i] = [rng.choice(c_) for c_ in cand]
+    for mname in ("dgx_a100", "dgx_v100"):
+        mach = X.ja_machine_preset(mname)
+        ms = {k: physical.compile_exchanges(ops, pl, mach, True, depth=1, beam=4)[0] for k, pl in plans.items()}
+        cost = {k: ja.ja_plan_cost(ops, pl) for k, pl in plans.items()}
+        draws = sorted(v for k, v in ms.items() if k.startswith("random"))
+        res["plan_selection_p8_%s" % mname] = {
+            "optimizer_exchange_ms": ms["optimizer"], "greedy_exchange_ms": ms["greedy"], "random_best_ms": draws[0],
+            "random_median_ms": (draws[9] + draws[10]) / 2, "random_worst_ms": draws[-1],
+            "plans_beating_the_optimizer": sum(1 for k, v in ms.items() if v < ms["optimizer"] * (1 - 1e-9)),
+            "pearson_r_proxy_cost_vs_exchange_ms": pearson([cost[k] for k in plans], [ms[k] for k in plans]), "n_plans": len(plans)}
     for name, (ops, plan) in workloads.items():
         for mname in ("dgx_a100", "dgx_v100"):
             mach = X.ja_machine_preset(mname)
