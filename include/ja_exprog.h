@@ -72,7 +72,8 @@ ja_status_t ja_exprog_get_atoms(const ja_exprog_t* p, int32_t* site, double* siz
  * The memberships are enumerated partition by partition in declaration order, each taking a combination (in
  * lexicographic order) of the sites that the explicit partitions and the earlier ones left.  ja_exprog_bind writes the
  * index-th membership into the program (partitions then have explicit members); ja_exprog_membership reports the
- * members of one partition as a site mask. */
+ * members of one partition as a site mask.  ja_exprog_num_memberships is the closed-form count; ja_exprog_bind by index
+ * and ja_exprog_valid_any list the memberships and refuse (JA_ERR_UNSUPPORTED) more than a million of them. */
 ja_status_t ja_exprog_num_memberships(const ja_exprog_t* p, int64_t* n);
 ja_status_t ja_exprog_bind(ja_exprog_t* p, int64_t index);
 ja_status_t ja_exprog_membership(const ja_exprog_t* p, const char* partition, uint64_t* members);
@@ -120,11 +121,12 @@ ja_status_t ja_exprog_simulate(const ja_exprog_t* p, const ja_machine_t* machine
  * simulator) from the program's own body, or, if it is empty, from the better of the naive and the butterfly body; keeps
  * the best program seen and reports its time.  The paper leaves the search procedure open.
  * ja_exprog_place: chooses the members of the size-declared partitions -- among the memberships under which the program
- * is valid the one with the least simulated time (the first of equals), with body = JA_BODY_OWN (the program's body as it
- * is), JA_BODY_NAIVE, JA_BODY_BUTTERFLY or JA_BODY_BEST (the better of the two constructed ones) rebuilt per membership.
- * Above 5000 memberships they are not enumerated: the search starts from the first one (the free sites dealt to the
- * partitions in ascending order) and repeatedly takes the exchange of two sites between two partitions that lowers the
- * simulated time most (the first of equals, pairs in ascending order), until none does.
+ * is valid the one with the least simulated time (among equal times the one that sends the fewest bytes, then the
+ * first), with body = JA_BODY_OWN (the program's body as it is), JA_BODY_NAIVE, JA_BODY_BUTTERFLY or JA_BODY_BEST (the
+ * better of the two constructed ones) rebuilt per membership.  Above 5000 memberships they are not enumerated: the
+ * search starts from the first one (the free sites dealt to the partitions in ascending order) and repeatedly takes the
+ * exchange of two sites between two partitions that lowers the simulated time most -- or, at equal time, the bytes
+ * sent -- (the first of equals, pairs in ascending order), until none does.
  * The program is left bound to the chosen membership with the chosen body.  JA_ERR_INVALID_ARG if none is valid. */
 typedef enum { JA_BODY_OWN = 0, JA_BODY_NAIVE = 1, JA_BODY_BUTTERFLY = 2, JA_BODY_BEST = 3 } ja_body_t;
 typedef enum {

@@ -483,8 +483,8 @@ def butterfly_body(prog: Program) -> Program:
 
 def place(prog: Program, mach: dict, body=None, enumeration_limit: int = 5000):
     """Choose the members of the size-declared partitions: among the memberships under which the program (its own body,
-    or body(bound preamble) if a synthesiser is given) is valid, the one with the least simulated completion time; ties go to
-    the first in enumeration order.  Above `enumeration_limit` memberships: steepest descent over exchanges of two sites
+    or body(bound preamble) if a synthesiser is given) is valid, the one with the least simulated completion time, among
+    equal times the one that sends the fewest bytes, then the first in enumeration order.  Above `enumeration_limit` memberships: steepest descent over exchanges of two sites
     between two partitions instead.  Returns (membership, bound program, milliseconds)."""
     def cost(m):
         q = bind(prog, m)
@@ -492,7 +492,15 @@ def place(prog: Program, mach: dict, body=None, enumeration_limit: int = 5000):
             q = body(q)
         if not valid_bound(q):
             return None
-        return (m, q, simulate(q, mach))
+        moved = sum(q.atoms[next(iter(x))][1] * len(d) for x, _, d in expanded(q))
+        return (m, q, simulate(q, mach), moved)
+
+    def better(c, ref):      # less simulated time; among equal times, fewer bytes sent
+        if ref is None:
+            return True
+        if c[2] < ref[2] * (1.0 - 1e-12):
+            return True
+        return c[2] <= ref[2] * (1.0 + 1e-12) and c[3] < ref[3] * (1.0 - 1e-12)
 
     names = [n for n, p in prog.partitions.items() if p["members"] is None]
     taken = {s for p in prog.partitions.values() if p["members"] is not None for s in p["members"]}
@@ -506,7 +514,7 @@ def place(prog: Program, mach: dict, body=None, enumeration_limit: int = 5000):
     if total <= enumeration_limit:
         for m in memberships(prog):
             c = cost(m)
-            if c is not None and (best is None or c[2] < best[2] * (1.0 - 1e-12)):
+            if c is not None and better(c, best):
                 best = c
     else:
         # steepest descent over exchanges of two sites between partitions, from the first membership in enumeration order
@@ -531,16 +539,15 @@ def place(prog: Program, mach: dict, body=None, enumeration_limit: int = 5000):
                             c = cost(nxt)
                             if c is None:
                                 continue
-                            bar = pick[2] if pick is not None else (best[2] if best is not None else math.inf)
-                            if c[2] < bar * (1.0 - 1e-12):
-                                pick = (nxt, c[1], c[2])
+                            if better(c, pick if pick is not None else best):
+                                pick = (nxt, c[1], c[2], c[3])
             if pick is not None:
                 cur = pick[0]
-                best = ({n: tuple(sorted(v)) for n, v in pick[0].items()}, pick[1], pick[2])
+                best = ({n: tuple(sorted(v)) for n, v in pick[0].items()}, pick[1], pick[2], pick[3])
                 improved = True
     if best is None:
         raise ValueError("no membership makes the program valid")
-    return best
+    return best[:3]
 
 
 # ----------------------------------------------------------------------------------- preamble generation (Section 5.3)

@@ -973,6 +973,19 @@ Key key_of(const Prog& p) {
     std::sort(k.begin(), k.end());
     return k;
 }
+double bytes_sent(const Prog& p) {      // GB put on links: every transfer of every action
+    std::vector<Flat> acts;
+    expand(p, &acts);
+    double gb = 0.0;
+    for (const Flat& a : acts) gb += atom_gb(p, a.agg) * (double)a.dests.size();
+    return gb;
+}
+// less simulated time; among equal times, fewer bytes sent
+bool better_placement(double t, double gb, bool have_ref, double ref_t, double ref_gb) {
+    if (!have_ref) return true;
+    if (t < ref_t * (1.0 - 1e-12)) return true;
+    return t <= ref_t * (1.0 + 1e-12) && gb < ref_gb * (1.0 - 1e-12);
+}
 bool best_constructed(const Prog& bound, const ja_machine_t& m, int body, Prog* best, double* ms) {
     std::vector<Prog> cands;
     if (body == JA_BODY_OWN) {
@@ -1018,6 +1031,30 @@ ja_status_t check_machine(const ja_machine_t* m, const Prog& p) {
     return JA_OK;
 }
 
+}  // namespace
+
+// memberships above this count are searched by pairwise swaps instead of being enumerated
+constexpr int64_t PLACE_ENUMERATION_LIMIT = 5000;
+// and above this one they are not listed at all (ja_exprog_bind by index, ja_exprog_valid_any)
+constexpr int64_t MEMBERSHIP_LIST_LIMIT = 1000000;
+namespace {
+int64_t count_memberships(const Prog& p) {      // the multinomial, capped well above the limit
+    std::set<int> taken;
+    int64_t n_free = 0;
+    for (const ExPartition& q : p.parts)
+        if (q.bound) taken.insert(q.members.begin(), q.members.end());
+    for (int s : p.gpus) n_free += !taken.count(s);
+    double total = 1.0;
+    for (const ExPartition& q : p.parts) {
+        if (q.bound) continue;
+        double c = 1.0;
+        for (int i = 0; i < q.size; ++i) c = c * (double)(n_free - i) / (double)(i + 1);
+        total *= c;
+        n_free -= q.size;
+        if (total > 1e15) return (int64_t)1e15;
+    }
+    return (int64_t)(total + 0.5);
+}
 }  // namespace
 
 // ============================================================================================================ C ABI
@@ -1123,13 +1160,14 @@ extern "C" ja_status_t ja_exprog_get_atoms(const ja_exprog_t* p, int32_t* site, 
 
 extern "C" ja_status_t ja_exprog_num_memberships(const ja_exprog_t* p, int64_t* n) {
     if (!p || !n) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
-    std::vector<std::vector<std::vector<int>>> all;
-    enumerate_memberships(*p, &all);
-    *n = (int64_t)all.size();
+    *n = count_memberships(*p);
     return JA_OK;
 }
 extern "C" ja_status_t ja_exprog_bind(ja_exprog_t* p, int64_t index) {
     if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
+    if (count_memberships(*p) > MEMBERSHIP_LIST_LIMIT)
+        return ja_fail(JA_ERR_UNSUPPORTED, "more than %lld memberships: bind the partitions with ja_exprog_bind_members or let ja_exprog_place choose",
+                       (long long)MEMBERSHIP_LIST_LIMIT);
     std::vector<std::vector<std::vector<int>>> all;
     enumerate_memberships(*p, &all);
     if (index < 0 || index >= (int64_t)all.size()) return ja_fail(JA_ERR_INVALID_ARG, "membership %lld of %lld", (long long)index, (long long)all.size());
@@ -1172,6 +1210,8 @@ extern "C" ja_status_t ja_exprog_check(const ja_exprog_t* p, int32_t* well_forme
 }
 extern "C" ja_status_t ja_exprog_valid_any(const ja_exprog_t* p, int32_t* valid) {
     if (!p || !valid) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    if (count_memberships(*p) > MEMBERSHIP_LIST_LIMIT)
+        return ja_fail(JA_ERR_UNSUPPORTED, "more than %lld memberships to try", (long long)MEMBERSHIP_LIST_LIMIT);
     std::vector<std::vector<std::vector<int>>> all;
     enumerate_memberships(*p, &all);
     *valid = 0;
@@ -1267,28 +1307,6 @@ extern "C" ja_status_t ja_exprog_synthesize(ja_exprog_t* p, const ja_machine_t* 
     if (ms) *ms = best.first;
     return JA_OK;
 }
-// memberships above this count are searched by pairwise swaps instead of being enumerated
-constexpr int64_t PLACE_ENUMERATION_LIMIT = 5000;
-namespace {
-int64_t count_memberships(const Prog& p) {      // the multinomial, capped well above the limit
-    std::set<int> taken;
-    int64_t n_free = 0;
-    for (const ExPartition& q : p.parts)
-        if (q.bound) taken.insert(q.members.begin(), q.members.end());
-    for (int s : p.gpus) n_free += !taken.count(s);
-    double total = 1.0;
-    for (const ExPartition& q : p.parts) {
-        if (q.bound) continue;
-        double c = 1.0;
-        for (int i = 0; i < q.size; ++i) c = c * (double)(n_free - i) / (double)(i + 1);
-        total *= c;
-        n_free -= q.size;
-        if (total > 1e15) return (int64_t)1e15;
-    }
-    return (int64_t)(total + 0.5);
-}
-}  // namespace
-
 extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machine, int32_t body, double* ms) {
     if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null program");
     ja_status_t s = check_machine(machine, *p);
@@ -1296,7 +1314,7 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
     if (body < JA_BODY_OWN || body > JA_BODY_BEST) return ja_fail(JA_ERR_INVALID_ARG, "body %d", body);
     bool found = false;
     Prog best;
-    double best_ms = 0;
+    double best_ms = 0, best_gb = 0;
     if (count_memberships(*p) <= PLACE_ENUMERATION_LIMIT) {
         std::vector<std::vector<std::vector<int>>> all;
         enumerate_memberships(*p, &all);
@@ -1306,9 +1324,11 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
             Prog c;
             double t;
             if (!best_constructed(q, *machine, body, &c, &t)) continue;
-            if (!found || t < best_ms * (1.0 - 1e-12)) {
+            const double gb = bytes_sent(c);
+            if (better_placement(t, gb, found, best_ms, best_gb)) {
                 best = c;
                 best_ms = t;
+                best_gb = gb;
                 found = true;
             }
         }
@@ -1338,12 +1358,13 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
             return best_constructed(q, *machine, body, c, t);
         };
         found = cost_of(cur, &best, &best_ms);
+        if (found) best_gb = bytes_sent(best);
         bool improved = true;
         while (improved) {
             improved = false;
             std::vector<std::vector<int>> pick;
             Prog pick_prog;
-            double pick_ms = 0;
+            double pick_ms = 0, pick_gb = 0;
             bool any = false;
             for (size_t a = 0; a < cur.size(); ++a)
                 for (size_t b = a + 1; b < cur.size(); ++b)
@@ -1354,11 +1375,12 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
                             Prog c;
                             double t;
                             if (!cost_of(nxt, &c, &t)) continue;
-                            const double bar = any ? pick_ms : (found ? best_ms : INFINITY);
-                            if (t < bar * (1.0 - 1e-12)) {
+                            const double gb = bytes_sent(c);
+                            if (any ? better_placement(t, gb, true, pick_ms, pick_gb) : better_placement(t, gb, found, best_ms, best_gb)) {
                                 pick = nxt;
                                 pick_prog = c;
                                 pick_ms = t;
+                                pick_gb = gb;
                                 any = true;
                             }
                         }
@@ -1366,6 +1388,7 @@ extern "C" ja_status_t ja_exprog_place(ja_exprog_t* p, const ja_machine_t* machi
                 cur = pick;
                 best = pick_prog;
                 best_ms = pick_ms;
+                best_gb = pick_gb;
                 found = true;
                 improved = true;
             }

@@ -90,6 +90,22 @@ def test_the_interface_limits_of_the_library():
     assert abs(X.ja_exprog_simulate(ok.handle, X.ja_machine_preset("dgx_h100")) - (63 / 450 + 65 / 3350) * 1e3) < 1e-6
 
 
+def test_membership_spaces_too_large_to_list():
+    from paper_2609_03905_b200.binding import JaError
+    n = 12
+    text = ("GPUS: " + ", ".join(str(i) for i in range(n)) + "\nPARTITIONS: " + " ".join("S%d {size 1}" % i for i in range(n)) +
+            "\nIN: " + "; ".join("a%d @ %d" % (i, i) for i in range(n)) + "\nOUT: " + "; ".join("a%d @ S%d" % (i, (i + 1) % n) for i in range(n)) + "\n")
+    h = X.ExchangeProgram(text)
+    import math
+    assert X.ja_exprog_num_memberships(h.handle) == math.factorial(n)         # counted, not listed
+    for call in (lambda: X.ja_exprog_bind(h.handle, 5), lambda: X.ja_exprog_valid_any(h.handle)):
+        with pytest.raises(JaError) as e:
+            call()
+        assert e.value.status_name == "JA_ERR_UNSUPPORTED"
+    ms = X.ja_exprog_place(h.handle, X.ja_machine_preset("dgx_h100"), "naive")   # the swap descent still places it
+    assert X.ja_exprog_check(h.handle) == (True, True) and ms == 0.0             # every atom's requirement put where the atom is
+
+
 def library_state(handle):
     return set(X.ja_exprog_closure(handle))
 
