@@ -235,3 +235,70 @@ def download_packed(dense, splits):
     from gpu_util import from_bits, np_bits
     packed = blocked.pack(np_bits(dense), splits)
     return from_bits(packed, dense.dtype).cuda()
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_randomly_rewritten_programs_on_random_preambles(seed):
+    """Random tilings, copy sites and function specs; the body is the trivial program after a random walk through the
+    rewriting rules (relays, fissions, eager and lazy aggregation, redirected sources), so the aggregation trees, the
+    duplicates and the order of arrival differ from anything a constructor emits."""
+    import random
+    rng = random.Random(100 + seed)
+    rank = rng.choice([1, 2, 2, 3])
+    ext = [rng.choice([24, 40, 64, 96]) for _ in range(rank)]
+
+    def cut(e, n):
+        pts = sorted(rng.sample(range(1, e), n - 1)) if n > 1 else []
+        return [0] + pts + [e]
+
+    n_sites = rng.choice([2, 3, 4])
+    while True:
+        ps = [cut(e, rng.choice([1, 2])) for e in ext]
+        cs = [cut(e, rng.choice([1, 2, 3])) for e in ext]
+        n_pb = int(np.prod([len(s) - 1 for s in ps]))
+        n_cb = int(np.prod([len(s) - 1 for s in cs]))
+        m = rng.choice([1, 2, 3])
+        cells = int(np.prod([len(set(a) | set(b)) - 1 for a, b in zip(ps, cs)]))
+        if cells * m <= 24:
+            break
+    copy_site = [rng.randrange(n_sites) for _ in range(n_pb * m)]
+    specs = [rng.randrange(n_cb) for _ in range(n_sites)]
+    dtype = rng.choice([BF, F16, F32])
+    agg = rng.choice(["sum", "max"]) if m > 1 else "none"
+    es = 4 if dtype == F32 else 2
+    h0 = X.ExchangeProgram(handle=X.ja_exprog_preamble(ps, cs, m, copy_site, specs, es))
+    X.ja_exprog_bind(h0.handle, rng.randrange(X.ja_exprog_num_memberships(h0.handle)))
+    X.ja_exprog_body(h0.handle, "naive")
+    q = E.normalised(E.parse(str(h0)))
+    for _ in range(rng.randint(0, 8)):
+        nb = E.neighbours(q)
+        if nb:
+            q = rng.choice(nb)
+    assert E.valid_bound(q)
+    h = X.ExchangeProgram(E.format_program(q))
+    assert X.ja_exprog_check(h.handle) == (True, True)
+    P = si.normal([m] + ext, 0.0, 1.0, dtype, 7, seed)
+    rP = upload(P, blocked.partial_splits(m, ps))
+    rD = empty_like_tiling(ext, cs, dtype, fill=float("nan"))
+    h.execute(rP, copy_site, specs, agg, rD)
+    plan = X.ExchangePlan(h, rP, copy_site, specs, agg, empty_like_tiling(ext, cs, dtype, fill=float("nan")))
+    plan.run()
+    got, got_plan = download(rD), download(plan.dst)
+    check_status()
+    P64 = si.to_f64(P)
+    want = E.exchange(q, P64, ps, cs, specs, "sum" if agg == "none" else agg, ORC_DT[dtype])
+    consumed = ~np.isnan(want)                                              # blocks no function spec consumes stay untouched
+    assert consumed.any() and np.isnan(got[~consumed]).all()
+    assert np.array_equal(got_plan[consumed], got[consumed]) and np.isnan(got_plan[~consumed]).all()
+    if agg != "sum":
+        assert np.array_equal(got[consumed], want[consumed])
+    else:
+        def f32_sum(parts):
+            acc = np.asarray(parts[0], dtype=np.float64).astype(np.float32)
+            for p in parts[1:]:
+                acc = acc + np.asarray(p, dtype=np.float64).astype(np.float32)
+            return core.round_to(acc.astype(np.float64), ORC_DT[dtype])
+        same = E.exchange(q, P64, ps, cs, specs, "sum", ORC_DT[dtype], combine=f32_sum)
+        assert np.array_equal(got[consumed], same[consumed])
+        assert relfro(got[consumed], want[consumed]) <= (1e-6 if dtype == F32 else 2e-3)
+    plan.close()
