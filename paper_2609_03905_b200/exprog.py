@@ -280,9 +280,9 @@ class ExchangePlan:
         import torch
         ja_exchange_plan_run(self.handle, torch.cuda.current_stream().cuda_stream if stream is None else stream)
 
-    def close(self):
+    def close(self, _destroy=LIB.ja_exchange_plan_destroy):   # bound at definition: module globals may be gone at interpreter exit
         if getattr(self, "handle", None):
-            ja_exchange_plan_destroy(self.handle)
+            _destroy(self.handle)
             self.handle = None
 
     def __del__(self):
@@ -295,9 +295,9 @@ class ExchangeProgram:
     def __init__(self, text: str | None = None, handle: int | None = None):
         self.handle = ja_exprog_parse(text) if handle is None else handle
 
-    def __del__(self):
+    def __del__(self, _destroy=LIB.ja_exprog_destroy):       # bound at definition: module globals may be gone at interpreter exit
         if getattr(self, "handle", None):
-            ja_exprog_destroy(self.handle)
+            _destroy(self.handle)
             self.handle = None
 
     def clone(self):
