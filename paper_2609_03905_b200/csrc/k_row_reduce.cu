@@ -13,7 +13,9 @@
 // and the sum of exponentials pays about half of its special-function time on top in either form. Measured and not kept:
 // issuing the loads of the next chunk before reducing this one (two buffers in registers halve what is in flight: 17.4 /
 // 51.4 / 71.9 us), sixteen vectors per lane (occupancy halves: 20.5 / 72.9 / 92.7), and asking for the warp's next row
-// with one bulk L2 prefetch per column block (21.3 / 69.7 / 88.2: the prefetches queue in front of the loads).
+// with one bulk L2 prefetch per column block (21.3 / 69.7 / 88.2: the prefetches queue in front of the loads); a quarter or
+// half of the exponentials as a degree-5 polynomial on the FMA pipe instead of ex2.approx (73.8 / 83.5 us against 66.2: what
+// the sum of exponentials pays on top of the row maximum is instruction issue, not the special-function unit).
 #include <stdlib.h>
 #include <string.h>
 
