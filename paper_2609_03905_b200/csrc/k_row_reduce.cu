@@ -15,7 +15,9 @@
 // 51.4 / 71.9 us), sixteen vectors per lane (occupancy halves: 20.5 / 72.9 / 92.7), and asking for the warp's next row
 // with one bulk L2 prefetch per column block (21.3 / 69.7 / 88.2: the prefetches queue in front of the loads); a quarter or
 // half of the exponentials as a degree-5 polynomial on the FMA pipe instead of ex2.approx (73.8 / 83.5 us against 66.2: what
-// the sum of exponentials pays on top of the row maximum is instruction issue, not the special-function unit).
+// the sum of exponentials pays on top of the row maximum is instruction issue, not the special-function unit); the scale,
+// the subtraction and the two running sums as packed f32x2 instructions (64.4 us against 66.2, sum of squares unchanged: not
+// worth a second code path).
 #include <stdlib.h>
 #include <string.h>
 
