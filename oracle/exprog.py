@@ -59,7 +59,7 @@ def _items(text):
 
 
 def _sites(text):
-    return tuple(int(t) for t in text.replace(" ", "").split(",") if t != "")
+    return tuple(int(t) for t in (u.strip() for u in text.split(",")) if t != "")
 
 
 def _target(text, partitions):
@@ -97,6 +97,8 @@ def parse(text: str) -> Program:
         if mi.group(1) in prog.atoms:
             raise ValueError("atom declared twice: " + mi.group(1))
         prog.atoms[mi.group(1)] = (int(mi.group(2)), float(mi.group(3)) if mi.group(3) else 1.0)
+    if not prog.atoms:
+        raise ValueError("IN declares no atom")
 
     def aggregate(t):
         names = [n.strip() for n in t.split("+")]

@@ -285,6 +285,7 @@ ja_status_t parse_program(const std::string& text, Prog* p) {
         if (p->atoms.size() == 64) return ja_fail(JA_ERR_INVALID_ARG, "more than 64 atoms");
         p->atoms.push_back(a);
     }
+    if (p->atoms.empty()) return ja_fail(JA_ERR_PARSE, "IN declares no atom");
     for (const std::string& it : items(sect[3])) {          // OUT: aggregate @ sites | partition
         size_t at = it.find('@');
         std::pair<uint64_t, ExTarget> o;

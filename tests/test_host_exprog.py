@@ -355,3 +355,58 @@ def test_firing_order_against_the_oracle():
     never = X.ExchangeProgram("IN: A @ 0; B @ 1\nOUT: A+B @ 0\n\nA+B @ 0\n")       # kept alive: the handle dies with the object
     with pytest.raises(JaError):
         X.ja_exprog_schedule(never.handle)
+
+
+def test_parser_fuzz_agrees_with_the_oracle_and_never_crashes():
+    from paper_2609_03905_b200.binding import JaError
+    rng = random.Random(77)
+    tokens = ["IN:", "OUT:", "GPUS:", "PARTITIONS:", "A", "B", "C", "G1", "G2", "@", "->", "+", ";", ",", "\n", "\n\n", " ", "0", "1", "2", "3",
+              "{", "}", "size", "(size:", "GB)", "1.5", "(", ")", ":", "x9", "70", "-1", "A+B", "A @ 0", "B @ 1", "OUT: A+B @ 0, 1", "IN: A @ 0; B @ 1"]
+    accepted = 0
+    for _ in range(1500):
+        text = "".join(rng.choice(tokens) + rng.choice(["", " ", " "]) for _ in range(rng.randint(1, 25)))
+        try:
+            p = E.parse(text)
+            ok_o = True
+        except Exception:
+            ok_o = False
+        try:
+            h = X.ExchangeProgram(text)
+            ok_l = True
+        except JaError:
+            ok_l = False
+        if ok_o and ok_l:
+            accepted += 1
+            same_program(h.handle, p)
+        # the two parsers may differ on malformed text only in WHICH of them is stricter; neither may accept what the other
+        # reads as a different program, which same_program above checks whenever both accept
+    assert accepted > 5
+    # mutations of the paper's printed programs: a token dropped, doubled or replaced
+    both = 0
+    for _ in range(1500):
+        base = G[rng.choice(["swap", "doubling", "v100", "preamble"])]["program"]
+        parts = base.replace("\n", " \n ").split(" ")
+        for _ in range(rng.randint(1, 3)):
+            i = rng.randrange(len(parts))
+            k = rng.random()
+            if k < 0.4:
+                del parts[i]
+            elif k < 0.7:
+                parts.insert(i, parts[i])
+            else:
+                parts[i] = rng.choice(tokens)
+        text = " ".join(parts).replace(" \n ", "\n")
+        try:
+            p = E.parse(text)
+        except Exception:
+            p = None
+        try:
+            h = X.ExchangeProgram(text)
+        except JaError:
+            h = None
+        if p is not None and h is not None:
+            both += 1
+            same_program(h.handle, p)
+            if not p.partitions or all(q["members"] is not None for q in p.partitions.values()):
+                assert X.ja_exprog_check(h.handle) == (E.well_formed(p), E.valid_bound(p))
+    assert both > 100
