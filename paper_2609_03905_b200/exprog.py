@@ -311,3 +311,24 @@ class ExchangeProgram:
         import torch
         st = torch.cuda.current_stream().cuda_stream if stream is None else stream
         return ja_exchange_execute(self.handle, partials.handle, copy_site, consumer_specs, agg, dst.handle, st)
+
+
+def best_valid_body(preamble: str, bodies, machine: ja_machine_t):
+    """Candidate bodies for one (bound) preamble from any source -- the paper has a language model propose them -- filtered by
+    Definition "Closure; validity" and ranked by the simulator.  Returns (index of the winner, its milliseconds, verdicts) where
+    verdicts[i] is None for a candidate that does not parse, is not valid, or is not for this preamble's sites, else its time;
+    (None, None, verdicts) if no candidate is valid."""
+    from .binding import JaError
+    verdicts, best = [], None
+    head = preamble.strip("\n").split("\n\n")[0]
+    for i, body in enumerate(bodies):
+        try:
+            h = ExchangeProgram(head + "\n\n" + body.strip("\n") + "\n")
+            ok = ja_exprog_check(h.handle)[1]
+            ms = ja_exprog_simulate(h.handle, machine) if ok else None
+        except JaError:
+            ms = None
+        verdicts.append(ms)
+        if ms is not None and (best is None or ms < verdicts[best]):
+            best = i
+    return best, (verdicts[best] if best is not None else None), verdicts

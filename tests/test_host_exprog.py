@@ -410,3 +410,19 @@ def test_parser_fuzz_agrees_with_the_oracle_and_never_crashes():
             if not p.partitions or all(q["members"] is not None for q in p.partitions.values()):
                 assert X.ja_exprog_check(h.handle) == (E.well_formed(p), E.valid_bound(p))
     assert both > 100
+
+
+def test_candidate_bodies_are_filtered_by_validity_and_ranked_by_the_simulator():
+    pre, printed_body = G["doubling"]["program"].split("\n\n", 1)
+    gather = "A @ 0 -> 1, 2, 3; B @ 1 -> 0, 2, 3; C @ 2 -> 0, 1, 3; D @ 3 -> 0, 1, 2; A+B+C+D @ 0, 1, 2, 3"
+    bodies = ["A+B @ 0 -> 1",                                  # not enabled: B never reaches site 0
+              gather,
+              "A @ 0 -> 1; B @ 1 -> 0; A+B+C+D @ 0",            # not well-formed either
+              printed_body,
+              "A @ 0 -> 9",                                     # names an undeclared site
+              gather.replace("A+B+C+D @ 0, 1, 2, 3", "A+B+C+D @ 0, 1, 2")]   # well-formed, a requirement unmet
+    best, ms, verdicts = X.best_valid_body(pre, bodies, X.ja_machine_preset("dgx_h100"))
+    assert best == 3 and round(ms, 1) == G["doubling"]["completion_ms"]
+    assert [v is not None for v in verdicts] == [False, True, False, True, False, False]
+    assert verdicts[1] > verdicts[3]
+    assert X.best_valid_body(pre, bodies[:1], X.ja_machine_preset("dgx_h100"))[0] is None
