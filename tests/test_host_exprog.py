@@ -426,3 +426,27 @@ def test_candidate_bodies_are_filtered_by_validity_and_ranked_by_the_simulator()
     assert [v is not None for v in verdicts] == [False, True, False, True, False, False]
     assert verdicts[1] > verdicts[3]
     assert X.best_valid_body(pre, bodies[:1], X.ja_machine_preset("dgx_h100"))[0] is None
+
+
+def test_beam_search_against_the_oracle_on_random_preambles():
+    rng = random.Random(5)
+    for trial in range(12):
+        n_sites = rng.choice([3, 4])
+        atoms = list("ABCDEF")[:rng.randint(2, 5)]
+        text = "GPUS: " + ", ".join(map(str, range(n_sites))) + "\nIN: " + "; ".join("%s @ %d" % (a, rng.randrange(n_sites)) for a in atoms)
+        outs = []
+        for _ in range(rng.randint(1, 2)):
+            x = rng.sample(atoms, rng.randint(1, len(atoms)))
+            outs.append("+".join(sorted(x)) + " @ " + ", ".join(map(str, sorted(rng.sample(range(n_sites), rng.randint(1, n_sites))))))
+        text += "\nOUT: " + "; ".join(outs) + "\n"
+        for mname in ("dgx_h100", "dgx_v100"):
+            h = X.ExchangeProgram(text)
+            ms = X.ja_exprog_synthesize(h.handle, X.ja_machine_preset(mname), 2, 5)
+            q, ms_o = E.synthesize(E.parse(text), E.machine(mname), depth=2, beam=5)
+            assert close(ms, ms_o)
+            mk = masks(q)
+            assert set(X.ja_exprog_get_actions(h.handle)) == {(mk(x), s, sites_mask(d)) for x, s, d in E.expanded(q)}
+            assert X.ja_exprog_check(h.handle) == (True, True)
+            start = X.ExchangeProgram(text)
+            X.ja_exprog_body(start.handle, "naive")
+            assert ms <= X.ja_exprog_simulate(start.handle, X.ja_machine_preset(mname)) * (1 + 1e-12)
