@@ -227,6 +227,15 @@ def test_exchange_plan_runs_as_dataflow_and_inside_a_graph(case, body):
     assert np.array_equal(download(rB), download(rA))                      # cell for cell (the payloads' padding was cleared in one only)
     want = E.exchange(q, si.to_f64(P2), c["ps"], c["cs"], c["specs"], "sum", "bf16")
     assert relfro(download(rB), want) <= 1e-3
+    # and eagerly again after the capture, on another stream
+    rB.payload.zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        plan.run()
+    side.synchronize()
+    check_status()
+    assert np.array_equal(download(rB), download(rA))
     plan.close()
 
 
