@@ -32,15 +32,19 @@ typedef struct ja_exprog ja_exprog_t;
  * endpoints: every site sends at most link_gbs and receives at most link_gbs; a multicast to k sites is k flows.
  * CUBE_MESH: eight sites; i <-> i + 4 are double links (double_gbs per direction), pairs inside {0..3} and inside {4..7}
  * single links (link_gbs), every other pair shares one bridge of pcie_gbs in total (the paper names the four double
- * links and "single links inside a socket"; the rest of the table is this library's reading). */
-typedef enum { JA_FABRIC_NVSWITCH = 0, JA_FABRIC_CUBE_MESH = 1 } ja_fabric_t;
+ * links and "single links inside a socket"; the rest of the table is this library's reading).
+ * LINKS: any point-to-point topology given as a table of directed link capacities; flows on one directed link share it,
+ * flows between unlinked pairs share the bridge -- the cube mesh is the special case ja_machine_preset("dgx_v100") fills in. */
+typedef enum { JA_FABRIC_NVSWITCH = 0, JA_FABRIC_CUBE_MESH = 1, JA_FABRIC_LINKS = 2 } ja_fabric_t;
 typedef struct {
     int32_t fabric;    /* ja_fabric_t */
     int32_t n_sites;
     double hbm_gbs;    /* local aggregation: an aggregate of m >= 2 parts reads m and writes 1 block at this rate */
     double link_gbs;
     double double_gbs; /* CUBE_MESH only */
-    double pcie_gbs;   /* CUBE_MESH only */
+    double pcie_gbs;   /* CUBE_MESH and LINKS: the bridge that every transfer between unlinked pairs shares */
+    const double* links; /* LINKS only: n_sites x n_sites, links[a * n_sites + b] = GB/s of the direct link a -> b, 0 = none
+                            (the transfer goes over the bridge); HOST memory that outlives the calls given this machine */
 } ja_machine_t;
 /* "dgx_h100" (450 / 3350), "dgx_a100" (300 / 2039), "hgx_b200" (900 / 7700), "dgx_v100" (25, 50, 15.75 / 900).  The H100
  * and V100 figures reproduce the completion times of the paper's three examples. JA_ERR_INVALID_ARG for another name. */

@@ -313,7 +313,11 @@ def machine(name: str) -> dict:
 
 
 def _link(mach, a, b):
-    """("link", capacity) of the direct link a -> b of the cube mesh, or ("pcie", capacity)."""
+    """("link", capacity) of the direct link a -> b of the cube mesh (or of a machine given as a table of directed links,
+    {"kind": "links", "links": [[GB/s]], "pcie": bridge, "hbm": ...}), or ("pcie", capacity)."""
+    if mach["kind"] == "links":
+        c = mach["links"][a][b]
+        return ("link", c) if c > 0 else ("pcie", mach["pcie"])
     if abs(a - b) == 4:
         return ("link", mach["double"])
     if a // 4 == b // 4:

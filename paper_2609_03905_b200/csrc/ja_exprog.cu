@@ -552,6 +552,12 @@ double atom_gb(const Prog& p, uint64_t agg) {
 }
 // kind 0: a direct link of the given capacity, 1: the bridge
 void mesh_link(const ja_machine_t& m, int a, int b, int* kind, double* cap) {
+    if (m.fabric == JA_FABRIC_LINKS) {
+        const double c = m.links[a * m.n_sites + b];
+        *kind = c > 0 ? 0 : 1;
+        *cap = c > 0 ? c : m.pcie_gbs;
+        return;
+    }
     if (abs(a - b) == 4) {
         *kind = 0;
         *cap = m.double_gbs;
@@ -1026,6 +1032,17 @@ ja_status_t check_machine(const ja_machine_t* m, const Prog& p) {
         if (!(m->double_gbs > 0) || !(m->pcie_gbs > 0)) return ja_fail(JA_ERR_INVALID_ARG, "machine: bandwidths must be positive");
         for (int s : p.gpus)
             if (s > 7) return ja_fail(JA_ERR_INVALID_ARG, "the cube mesh has sites 0..7");
+    } else if (m->fabric == JA_FABRIC_LINKS) {
+        if (!m->links || m->n_sites < 1 || m->n_sites > 64) return ja_fail(JA_ERR_INVALID_ARG, "machine: a link table of n_sites x n_sites entries is needed");
+        bool bridge_needed = false;
+        for (int a = 0; a < m->n_sites; ++a)
+            for (int b = 0; b < m->n_sites; ++b) {
+                if (m->links[a * m->n_sites + b] < 0) return ja_fail(JA_ERR_INVALID_ARG, "machine: negative link capacity");
+                if (a != b && m->links[a * m->n_sites + b] == 0) bridge_needed = true;
+            }
+        if (bridge_needed && !(m->pcie_gbs > 0)) return ja_fail(JA_ERR_INVALID_ARG, "machine: unlinked pairs need a bridge capacity");
+        for (int s : p.gpus)
+            if (s >= m->n_sites) return ja_fail(JA_ERR_INVALID_ARG, "site %d is not in the machine's link table", s);
     } else if (m->fabric != JA_FABRIC_NVSWITCH) {
         return ja_fail(JA_ERR_INVALID_ARG, "machine: unknown fabric");
     }
@@ -1061,7 +1078,7 @@ int64_t count_memberships(const Prog& p) {      // the multinomial, capped well 
 // ============================================================================================================ C ABI
 extern "C" ja_status_t ja_machine_preset(const char* name, ja_machine_t* out) {
     if (!name || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
-    ja_machine_t m = {JA_FABRIC_NVSWITCH, 8, 0, 0, 0, 0};
+    ja_machine_t m = {JA_FABRIC_NVSWITCH, 8, 0, 0, 0, 0, nullptr};
     if (!strcmp(name, "dgx_h100")) {
         m.link_gbs = 450.0;
         m.hbm_gbs = 3350.0;

@@ -7,7 +7,7 @@ import ctypes
 
 from .binding import LIB, _check
 
-JA_FABRIC_NVSWITCH, JA_FABRIC_CUBE_MESH = 0, 1
+JA_FABRIC_NVSWITCH, JA_FABRIC_CUBE_MESH, JA_FABRIC_LINKS = 0, 1, 2
 BODY = {"own": 0, "naive": 1, "butterfly": 2, "best": 3}
 RULE = {"insert": 0, "delete": 1, "fission": 2, "fusion": 3, "relay_in": 4, "relay_out": 5, "pushdown": 6, "pullup": 7,
         "source": 8}
@@ -15,7 +15,17 @@ RULE = {"insert": 0, "delete": 1, "fission": 2, "fusion": 3, "relay_in": 4, "rel
 
 class ja_machine_t(ctypes.Structure):
     _fields_ = [("fabric", ctypes.c_int32), ("n_sites", ctypes.c_int32), ("hbm_gbs", ctypes.c_double),
-                ("link_gbs", ctypes.c_double), ("double_gbs", ctypes.c_double), ("pcie_gbs", ctypes.c_double)]
+                ("link_gbs", ctypes.c_double), ("double_gbs", ctypes.c_double), ("pcie_gbs", ctypes.c_double),
+                ("links", ctypes.POINTER(ctypes.c_double))]
+
+
+def machine_from_links(links, hbm_gbs: float, bridge_gbs: float = 0.0) -> ja_machine_t:
+    """A point-to-point topology from a square table links[a][b] = GB/s of the direct link a -> b (0 = none: over the bridge)."""
+    n = len(links)
+    flat = (ctypes.c_double * (n * n))(*[float(links[a][b]) for a in range(n) for b in range(n)])
+    m = ja_machine_t(JA_FABRIC_LINKS, n, hbm_gbs, 1.0, 0.0, bridge_gbs, ctypes.cast(flat, ctypes.POINTER(ctypes.c_double)))
+    m._keep = flat           # the table must outlive the machine
+    return m
 
 
 def _declare():

@@ -450,3 +450,51 @@ def test_beam_search_against_the_oracle_on_random_preambles():
             start = X.ExchangeProgram(text)
             X.ja_exprog_body(start.handle, "naive")
             assert ms <= X.ja_exprog_simulate(start.handle, X.ja_machine_preset(mname)) * (1 + 1e-12)
+
+
+def test_a_machine_given_as_a_table_of_links():
+    from paper_2609_03905_b200.binding import JaError
+    # the cube mesh written out as a table is the preset
+    table = [[0.0] * 8 for _ in range(8)]
+    for a in range(8):
+        for b in range(8):
+            if a != b:
+                table[a][b] = 50.0 if abs(a - b) == 4 else (25.0 if a // 4 == b // 4 else 0.0)
+    m = X.machine_from_links(table, 900.0, 15.75)
+    mo = {"kind": "links", "links": table, "pcie": 15.75, "hbm": 900.0}
+    h = X.ExchangeProgram(G["v100"]["program"])
+    ms = X.ja_exprog_place(h.handle, m, "own")
+    assert round(ms) == G["v100"]["completion_ms"]
+    g = X.ExchangeProgram(G["v100"]["program"])
+    assert close(X.ja_exprog_place(g.handle, X.ja_machine_preset("dgx_v100"), "own"), ms)
+    assert close(E.place(E.parse(G["v100"]["program"]), mo)[2], ms)
+    # a directed ring of four sites: 0 -> 1 -> 2 -> 3 -> 0 at 10 GB/s, nothing else, no bridge needed by this program
+    ring = [[0.0] * 4 for _ in range(4)]
+    for a in range(4):
+        ring[a][(a + 1) % 4] = 10.0
+    text = "IN: A @ 0 (size: 2 GB)\nOUT: A @ 3\n\nA @ 0 -> 1; A @ 1 -> 2; A @ 2 -> 3\n"
+    mr = X.machine_from_links(ring, 1000.0, 5.0)
+    assert close(X.ja_exprog_simulate(X.ExchangeProgram(text).handle, mr), 3 * 2 / 10 * 1e3)          # three hops, one after the other
+    direct = "IN: A @ 0 (size: 2 GB)\nOUT: A @ 3\n\nA @ 0 -> 3\n"
+    assert close(X.ja_exprog_simulate(X.ExchangeProgram(direct).handle, mr), 2 / 5 * 1e3)            # unlinked: over the bridge
+    with pytest.raises(JaError):                                                                       # unlinked pairs but no bridge
+        X.ja_exprog_simulate(X.ExchangeProgram(direct).handle, X.machine_from_links(ring, 1000.0, 0.0))
+    with pytest.raises(JaError):                                                                       # a site outside the table
+        X.ja_exprog_simulate(X.ExchangeProgram("IN: A @ 5\nOUT: A @ 5\n").handle, mr)
+    # random tables and random programs against the oracle
+    rng = random.Random(41)
+    for _ in range(25):
+        n = rng.randint(2, 5)
+        links = [[0.0 if a == b or rng.random() < 0.3 else rng.choice([5.0, 12.5, 40.0]) for b in range(n)] for a in range(n)]
+        ml, mlo = X.machine_from_links(links, 800.0, 3.0), {"kind": "links", "links": links, "pcie": 3.0, "hbm": 800.0}
+        atoms = list("ABCD")[:rng.randint(2, 4)]
+        t = "GPUS: " + ", ".join(map(str, range(n))) + "\nIN: " + "; ".join("%s @ %d" % (a, rng.randrange(n)) for a in atoms)
+        t += "\nOUT: " + "+".join(atoms) + " @ " + ", ".join(map(str, sorted(rng.sample(range(n), rng.randint(1, n))))) + "\n"
+        for body in ("naive", "butterfly"):
+            hh = X.ExchangeProgram(t)
+            X.ja_exprog_body(hh.handle, body)
+            q = (E.naive_body if body == "naive" else E.butterfly_body)(E.parse(t))
+            assert close(X.ja_exprog_simulate(hh.handle, ml), E.simulate(q, mlo))
+        hs = X.ExchangeProgram(t)
+        ms_s = X.ja_exprog_synthesize(hs.handle, ml, 1, 4)
+        assert close(ms_s, E.synthesize(E.parse(t), mlo, depth=1, beam=4)[1])
