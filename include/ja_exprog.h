@@ -57,6 +57,12 @@ ja_status_t ja_machine_preset(const char* name, ja_machine_t* out);
  * than 64 atoms or a site above 63.  The handle is owned by the caller (ja_exprog_destroy). */
 ja_status_t ja_exprog_parse(const char* text, ja_exprog_t** out);
 ja_status_t ja_exprog_clone(const ja_exprog_t* p, ja_exprog_t** out);
+/* One program out of two over the same GPUS and PARTITIONS (names, sizes and members must agree) -- the exchanges of two
+ * operands of one operator, which share the placement of its function specs and run at the same time: a's atoms, renamed
+ * prefix_a + name, then b's, renamed prefix_b + name; OUT and the bodies likewise, a's first.  JA_ERR_INVALID_ARG if the
+ * preambles disagree, names clash, or there are more than 64 atoms. */
+ja_status_t ja_exprog_merge(const ja_exprog_t* a, const ja_exprog_t* b, const char* prefix_a, const char* prefix_b,
+                            ja_exprog_t** out);
 void ja_exprog_destroy(ja_exprog_t* p);
 /* The program as text that ja_exprog_parse reads back to the same program.  Writes at most cap bytes including the
  * terminating zero; *needed receives the size of the whole text with its zero (JA_ERR_INVALID_ARG if cap is smaller). */

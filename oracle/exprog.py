@@ -156,6 +156,26 @@ def _check_static(prog: Program):
             raise ValueError("an action names an undeclared site")
 
 
+def merge(a: Program, b: Program, prefix_a: str, prefix_b: str) -> Program:
+    """One program out of two over the same GPUS and PARTITIONS: the exchanges of two operands of one operator, which share
+    the placement of its function specs and run at the same time (Section 5.1 compiles one program per operator)."""
+    if a.gpus != b.gpus or a.partitions != b.partitions:
+        raise ValueError("the two preambles disagree")
+    q = Program(list(a.gpus), {k: dict(v) for k, v in a.partitions.items()})
+    for prog, pre in ((a, prefix_a), (b, prefix_b)):
+        for n, v in prog.atoms.items():
+            if pre + n in q.atoms:
+                raise ValueError("atom names clash")
+            q.atoms[pre + n] = v
+        q.out += [(frozenset(pre + n for n in x), t) for x, t in prog.out]
+        for x, src, d in prog.actions:
+            act = (frozenset(pre + n for n in x), src, d)
+            if act not in q.actions:
+                q.actions.append(act)
+    _check_static(q)
+    return q
+
+
 def _name_order(prog):
     return {a: i for i, a in enumerate(prog.atoms)}
 

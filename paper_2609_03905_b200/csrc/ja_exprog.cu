@@ -1112,6 +1112,48 @@ extern "C" ja_status_t ja_exprog_parse(const char* text, ja_exprog_t** out) {
     *out = p;
     return JA_OK;
 }
+extern "C" ja_status_t ja_exprog_merge(const ja_exprog_t* a, const ja_exprog_t* b, const char* prefix_a, const char* prefix_b,
+                                       ja_exprog_t** out) {
+    if (!a || !b || !prefix_a || !prefix_b || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
+    if (a->gpus != b->gpus) return ja_fail(JA_ERR_INVALID_ARG, "the two programs declare different GPUS");
+    if (a->parts.size() != b->parts.size()) return ja_fail(JA_ERR_INVALID_ARG, "the two programs declare different PARTITIONS");
+    for (size_t i = 0; i < a->parts.size(); ++i)
+        if (a->parts[i].name != b->parts[i].name || a->parts[i].size != b->parts[i].size || a->parts[i].bound != b->parts[i].bound ||
+            a->parts[i].members != b->parts[i].members)
+            return ja_fail(JA_ERR_INVALID_ARG, "partition %s differs between the two programs", a->parts[i].name.c_str());
+    if (a->atoms.size() + b->atoms.size() > 64) return ja_fail(JA_ERR_INVALID_ARG, "%d atoms: at most 64", (int)(a->atoms.size() + b->atoms.size()));
+    Prog* p = new Prog(*a);
+    const int shift = (int)a->atoms.size();
+    for (ExAtom& at : p->atoms) at.name = std::string(prefix_a) + at.name;
+    for (ExAtom at : b->atoms) {
+        at.name = std::string(prefix_b) + at.name;
+        if (!is_word(at.name) || find_atom(*p, at.name) >= 0) {
+            delete p;
+            return ja_fail(JA_ERR_INVALID_ARG, "atom name %s clashes or is not a word", at.name.c_str());
+        }
+        p->atoms.push_back(at);
+    }
+    for (const ExAtom& at : p->atoms)
+        if (!is_word(at.name)) {
+            delete p;
+            return ja_fail(JA_ERR_INVALID_ARG, "atom name %s is not a word", at.name.c_str());
+        }
+    for (auto o : b->out) {
+        o.first <<= shift;
+        p->out.push_back(o);
+    }
+    for (ExAction act : b->actions) {
+        act.agg <<= shift;
+        add_action(p, act);
+    }
+    ja_status_t st = check_static(*p);
+    if (st != JA_OK) {
+        delete p;
+        return st;
+    }
+    *out = p;
+    return JA_OK;
+}
 extern "C" ja_status_t ja_exprog_clone(const ja_exprog_t* p, ja_exprog_t** out) {
     if (!p || !out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
     *out = new Prog(*p);

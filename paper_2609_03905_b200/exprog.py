@@ -35,6 +35,7 @@ def _declare():
         "ja_machine_preset": [ctypes.c_char_p, P(ja_machine_t)],
         "ja_exprog_parse": [ctypes.c_char_p, P(vp)],
         "ja_exprog_clone": [vp, P(vp)],
+        "ja_exprog_merge": [vp, vp, ctypes.c_char_p, ctypes.c_char_p, P(vp)],
         "ja_exprog_format": [vp, ctypes.c_char_p, i64, P(i64)],
         "ja_exprog_counts": [vp, P(i32), P(i32), P(i32), P(i32), P(i32), P(i32)],
         "ja_exprog_get_actions": [vp, P(u64), P(i32), P(u64)],
@@ -75,6 +76,17 @@ def _declare():
 _declare()
 
 
+def _program_arg(fn):
+    """Lets a call take an ExchangeProgram object where it takes a handle; the object stays referenced for the call's duration
+    (a handle taken from a temporary object would die before the call runs)."""
+    import functools
+
+    @functools.wraps(fn)
+    def inner(prog, *args, **kw):
+        return fn(getattr(prog, "handle", prog), *args, **kw)
+    return inner
+
+
 def ja_machine_preset(name: str) -> ja_machine_t:
     m = ja_machine_t()
     _check(LIB.ja_machine_preset(name.encode(), ctypes.byref(m)))
@@ -87,9 +99,16 @@ def ja_exprog_parse(text: str) -> int:
     return h.value
 
 
+@_program_arg
 def ja_exprog_clone(prog: int) -> int:
     h = ctypes.c_void_p()
     _check(LIB.ja_exprog_clone(prog, ctypes.byref(h)))
+    return h.value
+
+
+def ja_exprog_merge(a, b, prefix_a: str, prefix_b: str) -> int:
+    h = ctypes.c_void_p()
+    _check(LIB.ja_exprog_merge(getattr(a, "handle", a), getattr(b, "handle", b), prefix_a.encode(), prefix_b.encode(), ctypes.byref(h)))
     return h.value
 
 
@@ -97,6 +116,7 @@ def ja_exprog_destroy(prog: int):
     LIB.ja_exprog_destroy(prog)
 
 
+@_program_arg
 def ja_exprog_format(prog: int) -> str:
     need = ctypes.c_int64()
     _check(LIB.ja_exprog_format(prog, None, 0, ctypes.byref(need)))
@@ -105,12 +125,14 @@ def ja_exprog_format(prog: int) -> str:
     return buf.value.decode()
 
 
+@_program_arg
 def ja_exprog_counts(prog: int) -> dict:
     v = [ctypes.c_int32() for _ in range(6)]
     _check(LIB.ja_exprog_counts(prog, *[ctypes.byref(x) for x in v]))
     return dict(zip(("gpus", "partitions", "atoms", "out", "actions", "expanded"), (x.value for x in v)))
 
 
+@_program_arg
 def ja_exprog_get_actions(prog: int):
     """[(aggregate mask, source site, destination mask)] of the expanded actions."""
     n = ja_exprog_counts(prog)["expanded"]
@@ -119,6 +141,7 @@ def ja_exprog_get_actions(prog: int):
     return [(agg[i], src[i], dst[i]) for i in range(max(n, 0))]
 
 
+@_program_arg
 def ja_exprog_get_requirements(prog: int):
     n = ctypes.c_int32()
     _check(LIB.ja_exprog_get_requirements(prog, ctypes.byref(n), None, None))
@@ -127,6 +150,7 @@ def ja_exprog_get_requirements(prog: int):
     return [(agg[i], site[i]) for i in range(n.value)]
 
 
+@_program_arg
 def ja_exprog_get_atoms(prog: int):
     n = ja_exprog_counts(prog)["atoms"]
     site, gb = (ctypes.c_int32 * max(n, 1))(), (ctypes.c_double * max(n, 1))()
@@ -134,26 +158,31 @@ def ja_exprog_get_atoms(prog: int):
     return [(site[i], gb[i]) for i in range(n)]
 
 
+@_program_arg
 def ja_exprog_num_memberships(prog: int) -> int:
     n = ctypes.c_int64()
     _check(LIB.ja_exprog_num_memberships(prog, ctypes.byref(n)))
     return n.value
 
 
+@_program_arg
 def ja_exprog_bind(prog: int, index: int):
     _check(LIB.ja_exprog_bind(prog, index))
 
 
+@_program_arg
 def ja_exprog_membership(prog: int, partition: str) -> int:
     m = ctypes.c_uint64()
     _check(LIB.ja_exprog_membership(prog, partition.encode(), ctypes.byref(m)))
     return m.value
 
 
+@_program_arg
 def ja_exprog_bind_members(prog: int, partition: str, sites):
     _check(LIB.ja_exprog_bind_members(prog, partition.encode(), (ctypes.c_int32 * len(sites))(*[int(x) for x in sites]), len(sites)))
 
 
+@_program_arg
 def ja_exprog_closure(prog: int):
     n = ctypes.c_int64()
     _check(LIB.ja_exprog_closure(prog, ctypes.byref(n), None, None))
@@ -162,18 +191,21 @@ def ja_exprog_closure(prog: int):
     return [(agg[i], site[i]) for i in range(n.value)]
 
 
+@_program_arg
 def ja_exprog_check(prog: int):
     wf, v = ctypes.c_int32(), ctypes.c_int32()
     _check(LIB.ja_exprog_check(prog, ctypes.byref(wf), ctypes.byref(v)))
     return bool(wf.value), bool(v.value)
 
 
+@_program_arg
 def ja_exprog_valid_any(prog: int) -> bool:
     v = ctypes.c_int32()
     _check(LIB.ja_exprog_valid_any(prog, ctypes.byref(v)))
     return bool(v.value)
 
 
+@_program_arg
 def ja_exprog_simulate(prog: int, machine: ja_machine_t, trace: bool = False):
     ms = ctypes.c_double()
     if not trace:
@@ -185,26 +217,31 @@ def ja_exprog_simulate(prog: int, machine: ja_machine_t, trace: bool = False):
     return ms.value, [(a[i], b[i], c[i]) for i in range(n)]
 
 
+@_program_arg
 def ja_exprog_body(prog: int, body: str):
     _check(LIB.ja_exprog_body(prog, BODY[body]))
 
 
+@_program_arg
 def ja_exprog_normalise(prog: int):
     _check(LIB.ja_exprog_normalise(prog))
 
 
+@_program_arg
 def ja_exprog_rewrite(prog: int, rule: str, i: int = 0, j: int = 0, a: int = 0, b: int = 0) -> bool:
     applied = ctypes.c_int32()
     _check(LIB.ja_exprog_rewrite(prog, RULE[rule], i, j, a, b, ctypes.byref(applied)))
     return bool(applied.value)
 
 
+@_program_arg
 def ja_exprog_synthesize(prog: int, machine: ja_machine_t, depth: int = 4, beam: int = 16) -> float:
     ms = ctypes.c_double()
     _check(LIB.ja_exprog_synthesize(prog, ctypes.byref(machine), depth, beam, ctypes.byref(ms)))
     return ms.value
 
 
+@_program_arg
 def ja_exprog_place(prog: int, machine: ja_machine_t, body: str = "best") -> float:
     ms = ctypes.c_double()
     _check(LIB.ja_exprog_place(prog, ctypes.byref(machine), BODY[body], ctypes.byref(ms)))
@@ -225,6 +262,7 @@ def ja_exprog_preamble(producer_splits, consumer_splits, m: int, copy_site, cons
     return h.value
 
 
+@_program_arg
 def ja_exchange_execute(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int, stream: int = 0) -> dict:
     """Relation handles as in binding.ja_repartition_agg; returns the call's statistics."""
     from .binding import AGG
@@ -236,6 +274,7 @@ def ja_exchange_execute(prog: int, partials: int, copy_site, consumer_specs, agg
             "aggregation_bytes": stats[4]}
 
 
+@_program_arg
 def ja_exprog_schedule(prog: int):
     """[(expanded action index, [part masks in combination order])] in firing order."""
     n, total = ctypes.c_int32(), ctypes.c_int32()
@@ -256,6 +295,7 @@ def _stats(stats):
             "aggregation_bytes": stats[4]}
 
 
+@_program_arg
 def ja_exchange_plan_create(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int):
     """Returns (plan handle, statistics)."""
     from .binding import AGG
@@ -300,7 +340,8 @@ class ExchangePlan:
 
 
 class ExchangeProgram:
-    """A handle with its lifetime; methods are the calls above."""
+    """A handle with its lifetime; methods are the calls above.  The handle is destroyed with the object: keep the object
+    for as long as its `.handle` is in use (do not pass `ExchangeProgram(text).handle` of a temporary)."""
 
     def __init__(self, text: str | None = None, handle: int | None = None):
         self.handle = ja_exprog_parse(text) if handle is None else handle
@@ -312,6 +353,9 @@ class ExchangeProgram:
 
     def clone(self):
         return ExchangeProgram(handle=ja_exprog_clone(self.handle))
+
+    def merge(self, other: "ExchangeProgram", prefix_self: str, prefix_other: str):
+        return ExchangeProgram(handle=ja_exprog_merge(self.handle, other.handle, prefix_self, prefix_other))
 
     def __str__(self):
         return ja_exprog_format(self.handle)

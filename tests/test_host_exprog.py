@@ -474,13 +474,13 @@ def test_a_machine_given_as_a_table_of_links():
         ring[a][(a + 1) % 4] = 10.0
     text = "IN: A @ 0 (size: 2 GB)\nOUT: A @ 3\n\nA @ 0 -> 1; A @ 1 -> 2; A @ 2 -> 3\n"
     mr = X.machine_from_links(ring, 1000.0, 5.0)
-    assert close(X.ja_exprog_simulate(X.ExchangeProgram(text).handle, mr), 3 * 2 / 10 * 1e3)          # three hops, one after the other
+    assert close(X.ja_exprog_simulate(X.ExchangeProgram(text), mr), 3 * 2 / 10 * 1e3)          # three hops, one after the other
     direct = "IN: A @ 0 (size: 2 GB)\nOUT: A @ 3\n\nA @ 0 -> 3\n"
-    assert close(X.ja_exprog_simulate(X.ExchangeProgram(direct).handle, mr), 2 / 5 * 1e3)            # unlinked: over the bridge
+    assert close(X.ja_exprog_simulate(X.ExchangeProgram(direct), mr), 2 / 5 * 1e3)            # unlinked: over the bridge
     with pytest.raises(JaError):                                                                       # unlinked pairs but no bridge
-        X.ja_exprog_simulate(X.ExchangeProgram(direct).handle, X.machine_from_links(ring, 1000.0, 0.0))
+        X.ja_exprog_simulate(X.ExchangeProgram(direct), X.machine_from_links(ring, 1000.0, 0.0))
     with pytest.raises(JaError):                                                                       # a site outside the table
-        X.ja_exprog_simulate(X.ExchangeProgram("IN: A @ 5\nOUT: A @ 5\n").handle, mr)
+        X.ja_exprog_simulate(X.ExchangeProgram("IN: A @ 5\nOUT: A @ 5\n"), mr)
     # random tables and random programs against the oracle
     rng = random.Random(41)
     for _ in range(25):
@@ -498,3 +498,33 @@ def test_a_machine_given_as_a_table_of_links():
         hs = X.ExchangeProgram(t)
         ms_s = X.ja_exprog_synthesize(hs.handle, ml, 1, 4)
         assert close(ms_s, E.synthesize(E.parse(t), mlo, depth=1, beam=4)[1])
+
+
+def test_merged_programs_run_their_exchanges_at_the_same_time():
+    from paper_2609_03905_b200.binding import JaError
+    a_text = "GPUS: 0, 1, 2, 3\nIN: A @ 0; B @ 1\nOUT: A+B @ 2\n\nA @ 0 -> 2; B @ 1 -> 2; A+B @ 2\n"
+    b_text = "GPUS: 0, 1, 2, 3\nIN: A @ 3; B @ 2\nOUT: A+B @ 0, 1\n\nA @ 3 -> 0, 1; B @ 2 -> 0, 1; A+B @ 0, 1\n"
+    a, b = X.ExchangeProgram(a_text), X.ExchangeProgram(b_text)
+    m = X.ExchangeProgram(handle=X.ja_exprog_merge(a.handle, b.handle, "x_", "w_"))
+    mo = E.merge(E.parse(a_text), E.parse(b_text), "x_", "w_")
+    same_program(m.handle, mo)
+    assert X.ja_exprog_check(m.handle) == (True, True) and E.valid_bound(mo)
+    mk = masks(mo)
+    assert library_state(m.handle) == {(mk(x), s) for x, s in E.closure(mo)}
+    for name in ("dgx_h100", "dgx_v100"):
+        mach, macho = X.ja_machine_preset(name), E.machine(name)
+        ta, tb, tm = (X.ja_exprog_simulate(h.handle, mach) for h in (a, b, m))
+        assert close(tm, E.simulate(mo, macho))
+        assert max(ta, tb) * (1 - 1e-12) <= tm <= (ta + tb) * (1 + 1e-12)       # concurrent, sharing endpoints and memory
+    with pytest.raises(JaError):
+        X.ja_exprog_merge(a.handle, b.handle, "", "")                            # names clash
+    other = X.ExchangeProgram("GPUS: 0, 1\nIN: A @ 0\nOUT: A @ 1\n")          # objects are kept: a handle dies with its object
+    with pytest.raises(JaError):
+        X.ja_exprog_merge(a.handle, other.handle, "p", "q")
+    # the merged preamble of a partitioned pair places both operands with one membership
+    p1 = "GPUS: 0, 1\nPARTITIONS: S1 {size 1} S2 {size 1}\nIN: A @ 0; B @ 1\nOUT: A @ S1; B @ S2\n"
+    p2 = "GPUS: 0, 1\nPARTITIONS: S1 {size 1} S2 {size 1}\nIN: C @ 1 (size: 4 GB); D @ 0 (size: 4 GB)\nOUT: C @ S1; D @ S2\n"
+    h1, h2 = X.ExchangeProgram(p1), X.ExchangeProgram(p2)
+    j = h1.merge(h2, "a_", "b_")
+    ms = X.ja_exprog_place(j.handle, X.ja_machine_preset("dgx_h100"), "naive")
+    assert X.ja_exprog_membership(j.handle, "S1") == 1 << 1 and close(ms, 1 / 450 * 1e3)      # the 4 GB operand decides: S1 where C is
