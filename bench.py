@@ -527,7 +527,7 @@ def physical_results():
             naive, en = physical.compile_exchanges(ops, plan, mach, False)
             opt, eo = physical.compile_exchanges(ops, plan, mach, True, depth=2, beam=6)
             res["%s_%s" % (name, mname)] = {"naive_ms": naive, "optimised_ms": opt, "naive_over_optimised": naive / opt if opt > 0 else 1.0,
-                                            "edges": len(en), "edges_with_traffic": sum(1 for e in en if e["ms"] > 0),
+                                            "operators_with_produced_operands": len(en), "of_them_with_traffic": sum(1 for e in en if e["ms"] > 0),
                                             "proxy_cost_cells": ja.ja_plan_cost(ops, plan)}
     return res
 

@@ -69,25 +69,28 @@ def edge(ops, plan, consumer: int, operand: int, producer_sites, width_bytes: in
             "tensor_bytes": math.prod(ext) * width_bytes}
 
 
-def compile_exchanges(ops, plan, machine, optimise: bool, depth: int = 2, beam: int = 6, width_bytes: int = 2):
+def compile_exchanges(ops, plan, machine, optimise: bool, depth: int = 2, beam: int = 6, width_bytes: int = 2, joint: bool = True):
     """Every producer -> consumer edge of the planned graph as an exchange program, operators in topological order.
+    joint: the exchanges of all operands of one operator form ONE program (`ja_exprog_merge`), as Section 5.1 compiles one
+    program per operator -- they share the placement of its function specs and run at the same time; operators whose operands
+    together have more than 64 atoms, and joint = False, fall back to one program per operand, their times added.
     optimise = False: the naive programs of the paper's Experiment 4 -- function spec i on GPU i, every aggregated block
     gathered and aggregated where it is consumed.  optimise = True: every body goes through ja_exprog_synthesize, and the
-    placement of a consumer's function specs is the best, by the summed simulated time of its operands' exchanges, of
-    spec i on GPU i and of what ja_exprog_place chooses for each one of its operands; since a placement also moves the copies
-    the next operator starts from, the whole compilation is done a second time with every operator left at spec i on GPU i and
-    the faster of the two is returned.  Returns (total simulated ms, per-edge records)."""
+    placement of a consumer's function specs is the best, by simulated time, of spec i on GPU i and of what ja_exprog_place
+    chooses (for the joint program, or for each operand by itself); since a placement also moves the copies the next operator
+    starts from, the whole compilation is done a second time with every operator left at spec i on GPU i and the faster of the
+    two is returned.  Returns (total simulated ms, per-operator records)."""
     if not optimise:
-        return _compile(ops, plan, machine, "naive", depth, beam, width_bytes)
-    placed = _compile(ops, plan, machine, "placed", depth, beam, width_bytes)
-    fixed = _compile(ops, plan, machine, "fixed", depth, beam, width_bytes)
+        return _compile(ops, plan, machine, "naive", depth, beam, width_bytes, joint)
+    placed = _compile(ops, plan, machine, "placed", depth, beam, width_bytes, joint)
+    fixed = _compile(ops, plan, machine, "fixed", depth, beam, width_bytes, joint)
     return placed if placed[0] <= fixed[0] else fixed
 
 
-def _compile(ops, plan, machine, mode, depth, beam, width_bytes):
+def _compile(ops, plan, machine, mode, depth, beam, width_bytes, joint):
     p = None
     placement = {}
-    edges = []
+    records = []
     total = 0.0
     for j, op in enumerate(ops):
         _, _, letters = _terms(op["einsum"])
@@ -102,45 +105,52 @@ def _compile(ops, plan, machine, mode, depth, beam, width_bytes):
             continue
         args = {k: edge(ops, plan, j, k, placement[op["inputs"][k]], width_bytes) for k in operands}
 
-        def program(k, sites=None):
+        def operand_program(k, sites):
             a = args[k]
             h = X.ExchangeProgram(handle=X.ja_exprog_preamble(a["producer_splits"], a["consumer_splits"], a["m"], a["copy_site"],
                                                               a["consumer_specs"], a["width_bytes"]))
             if sites is not None:
                 for i, s in enumerate(sites):
-                    X.ja_exprog_bind_members(h.handle, "S%d" % (i + 1), [s])
+                    X.ja_exprog_bind_members(h, "S%d" % (i + 1), [s])
             return h
 
-        def record(k, ms, h):
-            return {"consumer": j, "operand": k, "ms": ms, "m": args[k]["m"], "tensor_MB": args[k]["tensor_bytes"] / 1e6,
-                    "actions": X.ja_exprog_counts(h.handle)["expanded"]}
+        def programs(sites):
+            """The operator's exchange as a list of programs: one (all operands merged) or one per operand."""
+            hs = [operand_program(k, sites) for k in operands]
+            if joint and len(hs) > 1 and sum(X.ja_exprog_counts(h)["atoms"] for h in hs) <= 64:
+                merged = hs[0]
+                for n, h in enumerate(hs[1:], 1):
+                    merged = merged.merge(h, "k0_" if n == 1 else "", "k%d_" % n)
+                return [merged]
+            return hs
 
-        if mode == "naive":
-            placement[j] = identity
-            for k in operands:
-                h = program(k, identity)
-                X.ja_exprog_body(h.handle, "naive")
-                edges.append(record(k, X.ja_exprog_simulate(h.handle, machine), h))
-                total += edges[-1]["ms"]
-            continue
+        def sites_of(h):
+            return [X.ja_exprog_membership(h, "S%d" % (i + 1)).bit_length() - 1 for i in range(p)]
+
+        def cost_with(sites):
+            hs = programs(sites)
+            if mode == "naive":
+                for h in hs:
+                    X.ja_exprog_body(h, "naive")
+                ms = [X.ja_exprog_simulate(h, machine) for h in hs]
+            else:
+                ms = [X.ja_exprog_synthesize(h, machine, depth, beam) for h in hs]
+            return sum(ms), sum(X.ja_exprog_counts(h)["expanded"] for h in hs), len(hs)
+
         candidates = [identity]
         if mode == "placed":
-            for k in operands:
-                h = program(k)
-                X.ja_exprog_place(h.handle, machine, "best")
-                sites = [X.ja_exprog_membership(h.handle, "S%d" % (i + 1)).bit_length() - 1 for i in range(p)]
+            for h in programs(None):
+                X.ja_exprog_place(h, machine, "best")
+                sites = sites_of(h)
                 if sites not in candidates:
                     candidates.append(sites)
         best = None
         for sites in candidates:
-            recs = []
-            for k in operands:
-                h = program(k, sites)
-                recs.append(record(k, X.ja_exprog_synthesize(h.handle, machine, depth, beam), h))
-            cost = sum(r["ms"] for r in recs)
-            if best is None or cost < best[0] * (1.0 - 1e-12):
-                best = (cost, sites, recs)
+            ms, n_actions, n_programs = cost_with(sites)
+            if best is None or ms < best[0] * (1.0 - 1e-12):
+                best = (ms, sites, n_actions, n_programs)
         placement[j] = best[1]
-        edges += best[2]
+        records.append({"consumer": j, "operands": operands, "ms": best[0], "actions": best[2], "programs": best[3],
+                        "m": [args[k]["m"] for k in operands], "tensor_MB": [args[k]["tensor_bytes"] / 1e6 for k in operands]})
         total += best[0]
-    return total, edges
+    return total, records

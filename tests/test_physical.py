@@ -41,16 +41,21 @@ def test_naive_against_optimised_exchanges_of_a_planned_block():
         mach = X.ja_machine_preset(name)
         naive, en = physical.compile_exchanges(ops, plan, mach, False)
         opt, eo = physical.compile_exchanges(ops, plan, mach, True, depth=1, beam=4)
-        assert len(en) == len(eo) == sum(1 for op in ops for i in op["inputs"] if i is not None)
+        assert len(en) == len(eo) == sum(1 for op in ops if any(i is not None for i in op["inputs"]))
         assert opt <= naive * (1 + 1e-12)                       # the naive program is in the search space
-        # edges whose producer and consumer agree on tiling and placement and have one copy move nothing
-        charged = {(j, k) for j, op in enumerate(ops) for k, i in enumerate(op["inputs"]) if i is not None and
-                   tuple(plan[i][c] for c in op_out(ops[i])) != tuple(plan[j][c] for c in op_in(op, k))}
-        for e in en:
-            if e["m"] == 1 and (e["consumer"], e["operand"]) not in charged:
-                replicated = any(c not in op_in(ops[e["consumer"]], e["operand"]) and plan[e["consumer"]][c] > 1
-                                 for c in letters(ops[e["consumer"]]))
-                assert replicated or e["ms"] == 0.0
+        # one program per operator runs its operands' exchanges at the same time: never slower than one after the other
+        naive_sep, en_sep = physical.compile_exchanges(ops, plan, mach, False, joint=False)
+        assert naive <= naive_sep * (1 + 1e-12)
+        assert all(e["programs"] == 1 for e in en) and any(e["programs"] > 1 for e in en_sep)
+        # operators whose producers and they agree on tiling and placement, with one copy and nothing replicated, move nothing
+        for e in en_sep:
+            j = e["consumer"]
+            quiet = all(m == 1 for m in e["m"])
+            for k in e["operands"]:
+                i = ops[j]["inputs"][k]
+                quiet = quiet and tuple(plan[i][c] for c in op_out(ops[i])) == tuple(plan[j][c] for c in op_in(ops[j], k))
+                quiet = quiet and not any(c not in op_in(ops[j], k) and plan[j][c] > 1 for c in letters(ops[j]))
+            assert not quiet or e["ms"] == 0.0
         out[name] = naive / opt if opt > 0 else 1.0
     assert out["dgx_a100"] < 1.02                               # nothing to exploit on a non-blocking fabric
     assert out["dgx_v100"] >= out["dgx_a100"] - 1e-12
