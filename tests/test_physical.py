@@ -103,3 +103,29 @@ def test_swap_descent_placement_matches_the_oracle_and_enumeration():
     desc = E.place(p, mo, body=E.naive_body, enumeration_limit=0)
     assert desc[2] >= full[2] * (1 - 1e-12)                      # enumeration is exact; descent may stop in a local minimum
     assert E.valid_bound(desc[1])
+
+
+def test_the_plan_for_one_long_sequence_is_the_one_the_paper_reports():
+    """Section 6, Experiment 1: for the 1 x 128K workload the optimizer "discovers" the DeepSpeed-Ulysses decomposition --
+    tokens sharded everywhere outside attention, heads sharded inside it, a repartition at the boundary.  With the sequence
+    index of attention not shardable inside one sequence (Example 3.10) the library's optimizer and the oracle's both return
+    exactly that for eight processors, and the four boundary exchanges are all-to-alls."""
+    from oracle import optimizer as O
+    from paper_2609_03905_b200.planned_block import plan_repartition_charges
+    ops = block_graph(1, 131072, 4096, 32, 14336)
+    ops[4] = dict(ops[4], fixed={"d", "q", "k"})
+    cost, plan = ja.ja_plan_optimize_graph(ops, 8)
+    for j, counts in enumerate(plan):
+        cut = {k: v for k, v in counts.items() if v > 1}
+        assert cut == ({"h": 8} if j == 4 else {"s": 8}), (j, cut)
+    assert plan_repartition_charges(ops, plan)[0] == 4                     # q, k, v into attention, its output back
+    cost_o, plan_o = O.optimize_graph(ops, 8)
+    assert cost_o == cost and [dict(p) for p in plan_o] == [dict(p) for p in plan]
+    mach = X.ja_machine_preset("dgx_a100")
+    total, recs = physical.compile_exchanges(ops, plan, mach, True, depth=0)
+    moving = [r for r in recs if r["ms"] > 0]
+    assert [r["consumer"] for r in moving] == [4, 5]                       # attention (q, k, v as one program) and the output projection
+    # an all-to-all: every GPU sends 7/8 of its eighth of each tensor, one eighth to each other GPU, at full egress
+    eighth_gb = 131072 * 4096 * 2 / 8 / 1e9
+    assert abs(moving[1]["ms"] - 7 / 8 * eighth_gb / 300 * 1e3) < 1e-6
+    assert abs(moving[0]["ms"] - 3 * 7 / 8 * eighth_gb / 300 * 1e3) < 1e-6  # q, k and v together share the endpoints
