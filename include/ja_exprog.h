@@ -201,6 +201,19 @@ typedef struct ja_exchange_plan ja_exchange_plan_t;
 ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
                                     const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
                                     int64_t* stats, ja_exchange_plan_t** out);
+/* The same with the sites spread over the devices of this process: site s lives on the device with label site_device[s]
+ * (s < n_site_device; other sites, and all of them when site_device is NULL, live on the HOME device, the one current at
+ * creation, whose label is its ordinal).  A site's buffers are allocated on its device, its aggregations launched there on
+ * its own stream, and a transfer is a copy between the two devices' buffers (cudaMemcpyAsync under unified addressing, which a
+ * stream capture can record) -- no kernel ever reads another device's memory.  Both relations live on the home device: atoms of sites elsewhere are sliced
+ * into a staging area at home and sent to their sites before the program starts, and the aggregates that function specs
+ * elsewhere end with are brought home before recompose (on a machine whose producers and consumers run on those devices
+ * these two hops are the operators' own outputs and inputs).  A label beyond the visible devices wraps around (label modulo
+ * the device count), so every path of a multi-device plan also runs on fewer GPUs, down to one.  ja_exchange_plan_run must
+ * be called with the home device current. */
+ja_status_t ja_exchange_plan_create_on(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                       const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                       const int32_t* site_device, int32_t n_site_device, int64_t* stats, ja_exchange_plan_t** out);
 ja_status_t ja_exchange_plan_run(ja_exchange_plan_t* plan, void* cuda_stream);
 void ja_exchange_plan_destroy(ja_exchange_plan_t* plan);
 

@@ -1738,7 +1738,8 @@ struct ExStep {
 struct ExBuild {
     std::vector<ExBuffer> bufs;
     std::vector<ExStep> steps;
-    std::vector<JaBoxCopy> boxes;   // n_in decompose boxes, then n_out recompose boxes
+    std::vector<JaBoxCopy> boxes;   // n_in decompose boxes (box a fills buffer a, the atoms come first), then n_out recompose boxes
+    std::vector<int> out_box_buf;   // the buffer every recompose box reads
     int n_in = 0, n_out = 0;
     bool vec_in = true, vec_out = true;
     int64_t max_in = 0, max_out = 0, scratch = 0, table_off = 0, table_bytes = 0;
@@ -1899,6 +1900,7 @@ ja_status_t build_exchange(const ja_exprog_t* prog, const ja_relation_t* partial
             B->vec_out = B->vec_out && aligned16(b);
             B->max_out = std::max(B->max_out, b.n0 * b.n1 * b.run_bytes);
             B->boxes.push_back(b);
+            B->out_box_buf.push_back(it->second);
         }
     }
     B->n_out = (int)B->boxes.size() - B->n_in;
@@ -1975,30 +1977,53 @@ extern "C" ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_rel
 // Every site that runs a step has a stream of its own; a step waits for the buffers other sites' streams write (events), so what
 // a capture of ja_exchange_plan_run records is the program's dependency graph -- kernels and copies as vertices -- and actions of
 // different sites may run at the same time, copies on the copy engines beside the aggregation kernels.
+// Sites may live on different devices of this process: every site has a device label, the buffers of a site are allocated on its
+// device, its aggregations launched there, and a transfer is a copy from the source's device to the destination's. The two
+// relations live on the HOME device (the one current at creation): atoms of sites elsewhere are sliced into a staging area at
+// home and sent to their sites before the program starts, and the aggregates a function spec elsewhere ends with are brought
+// home before recompose. Labels beyond the visible devices wrap around, which runs every one of these paths on fewer GPUs.
+struct ExPlace {
+    int label;            // device label of the buffer's site
+    int64_t off;          // offset in that label's pool
+    int64_t stage = -1;   // offset of its staging copy in the home pool (buffers that decompose fills or recompose reads, away from home)
+};
 struct ja_exchange_plan {
     ExBuild B;
-    char* pool = nullptr;
-    int device = 0;
+    std::vector<ExPlace> place;               // per buffer
+    std::map<int, char*> pool;                // per label
+    std::map<int, int> phys;                  // label -> device ordinal
+    std::map<int, int> site_label;
+    int home = 0;                             // label of the home device
+    int64_t table_off = 0;                    // box tables, in the home pool
     std::map<int, cudaStream_t> stream;       // per site
     std::vector<cudaEvent_t> ready;           // per buffer: written
     std::map<int, cudaEvent_t> done;          // per site: its last step issued
     cudaEvent_t start = nullptr;
+    char* at(int b) const { return pool.at(place[b].label) + place[b].off; }
 };
 
 extern "C" void ja_exchange_plan_destroy(ja_exchange_plan_t* p) {
     if (!p) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
     for (auto& kv : p->stream) cudaStreamDestroy(kv.second);
     for (cudaEvent_t e : p->ready)
         if (e) cudaEventDestroy(e);
     for (auto& kv : p->done) cudaEventDestroy(kv.second);
     if (p->start) cudaEventDestroy(p->start);
-    if (p->pool) cudaFree(p->pool);
+    for (auto& kv : p->pool)
+        if (kv.second) {
+            cudaSetDevice(p->phys[kv.first]);
+            cudaFree(kv.second);
+        }
+    cudaSetDevice(cur);
     delete p;
 }
 
-extern "C" ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
-                                               const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
-                                               int64_t* stats, ja_exchange_plan_t** out) {
+extern "C" ja_status_t ja_exchange_plan_create_on(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                                  const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                                  const int32_t* site_device, int32_t n_site_device, int64_t* stats,
+                                                  ja_exchange_plan_t** out) {
     if (!out) return ja_fail(JA_ERR_INVALID_ARG, "null argument");
     ja_exchange_plan* p = new ja_exchange_plan();
     ja_status_t st = build_exchange(prog, partials, copy_site, consumer_specs, n_specs, agg, dst, &p->B);
@@ -2006,22 +2031,80 @@ extern "C" ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja
         delete p;
         return st;
     }
-    const ExBuild& B = p->B;
-    cudaError_t e = cudaGetDevice(&p->device);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->pool, (size_t)B.scratch);
-    if (e == cudaSuccess) e = cudaMemcpy(p->pool + B.table_off, B.boxes.data(), (size_t)B.table_bytes, cudaMemcpyHostToDevice);
+    ExBuild& B = p->B;
+    int home_dev = 0, n_dev = 1;
+    cudaError_t e = cudaGetDevice(&home_dev);
+    if (e == cudaSuccess) e = cudaGetDeviceCount(&n_dev);
+    if (e != cudaSuccess || n_dev < 1) {
+        delete p;
+        return ja_fail(JA_ERR_CUDA, "exchange plan: no device");
+    }
+    // labels: the home device's own ordinal is its label; a site without an entry lives at home
+    p->home = home_dev;
+    p->phys[p->home] = home_dev;
+    for (int s : prog->gpus) {
+        int label = p->home;
+        if (site_device && s < n_site_device) {
+            if (site_device[s] < 0) {
+                delete p;
+                return ja_fail(JA_ERR_INVALID_ARG, "site %d: negative device label", s);
+            }
+            label = site_device[s];
+        }
+        p->site_label[s] = label;
+        p->phys[label] = label % n_dev;
+    }
+    // place every buffer in its site's pool; staging at home for what decompose fills or recompose reads away from home
+    std::map<int, int64_t> size;
+    auto take = [&](int label, int64_t bytes) {
+        const int64_t off = size[label];
+        size[label] += (bytes + 255) / 256 * 256;
+        return off;
+    };
+    p->place.resize(B.bufs.size());
+    for (size_t b = 0; b < B.bufs.size(); ++b) {
+        p->place[b].label = p->site_label.at(B.bufs[b].site);
+        p->place[b].off = take(p->place[b].label, B.bufs[b].bytes);
+    }
+    for (int a = 0; a < B.n_in; ++a)
+        if (p->place[a].label != p->home) p->place[a].stage = take(p->home, B.bufs[a].bytes);
+    for (int b : B.out_box_buf)
+        if (p->place[b].label != p->home && p->place[b].stage < 0) p->place[b].stage = take(p->home, B.bufs[b].bytes);
+    p->table_off = take(p->home, B.table_bytes);
+    // the boxes address the home pool: a buffer at home directly, one elsewhere through its staging copy
+    for (int i = 0; i < B.n_in; ++i) B.boxes[i].dst_off = p->place[i].stage >= 0 ? p->place[i].stage : p->place[i].off;
+    for (int i = 0; i < B.n_out; ++i) {
+        const ExPlace& pl = p->place[B.out_box_buf[i]];
+        B.boxes[B.n_in + i].src_off = pl.stage >= 0 ? pl.stage : pl.off;
+    }
+    B.scratch = 0;
+    for (auto& kv : size) B.scratch += kv.second;
+    for (auto& kv : size) {
+        if (e != cudaSuccess) break;
+        e = cudaSetDevice(p->phys[kv.first]);
+        char* mem = nullptr;
+        if (e == cudaSuccess) e = cudaMalloc((void**)&mem, (size_t)std::max<int64_t>(kv.second, 256));
+        if (e == cudaSuccess) p->pool[kv.first] = mem;
+    }
+    if (e == cudaSuccess) e = cudaSetDevice(home_dev);
+    if (e == cudaSuccess) e = cudaMemcpy(p->pool[p->home] + p->table_off, B.boxes.data(), (size_t)B.table_bytes, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->start, cudaEventDisableTiming);
     p->ready.assign(B.bufs.size(), nullptr);
     for (size_t i = 0; e == cudaSuccess && i < B.bufs.size(); ++i)
-        if (B.bufs[i].producer_site >= 0) e = cudaEventCreateWithFlags(&p->ready[i], cudaEventDisableTiming);
+        if (B.bufs[i].producer_site >= 0) {
+            e = cudaSetDevice(p->phys[p->site_label.at(B.bufs[i].producer_site)]);      // recorded on the producer's stream
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ready[i], cudaEventDisableTiming);
+        }
     for (size_t i = 0; e == cudaSuccess && i < B.sites.size(); ++i) {
+        e = cudaSetDevice(p->phys[p->site_label.at(B.sites[i])]);
         cudaStream_t s = nullptr;
-        e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
         if (e == cudaSuccess) p->stream[B.sites[i]] = s;
         cudaEvent_t ev = nullptr;
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
         if (e == cudaSuccess) p->done[B.sites[i]] = ev;
     }
+    cudaSetDevice(home_dev);
     if (e != cudaSuccess) {
         ja_exchange_plan_destroy(p);
         return ja_fail(e == cudaErrorMemoryAllocation ? JA_ERR_OOM : JA_ERR_CUDA, "exchange plan: %s", cudaGetErrorString(e));
@@ -2031,13 +2114,47 @@ extern "C" ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja
     return JA_OK;
 }
 
+extern "C" ja_status_t ja_exchange_plan_create(const ja_exprog_t* prog, const ja_relation_t* partials, const int32_t* copy_site,
+                                               const int32_t* consumer_specs, int32_t n_specs, ja_agg_t agg, ja_relation_t* dst,
+                                               int64_t* stats, ja_exchange_plan_t** out) {
+    return ja_exchange_plan_create_on(prog, partials, copy_site, consumer_specs, n_specs, agg, dst, nullptr, 0, stats, out);
+}
+
+namespace {
+// a device switch only when the device changes
+cudaError_t set_device_if(int dev) {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return e;
+    return cur == dev ? cudaSuccess : cudaSetDevice(dev);
+}
+// Between two buffers of this process, on one device or two: under unified addressing the runtime finds the devices from the
+// pointers, and the copy can be recorded by a stream capture (cudaMemcpyPeerAsync cannot: a capture that meets it is invalidated).
+cudaError_t copy_between(void* dst, const void* src, size_t bytes, cudaStream_t st) {
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, st);
+}
+}  // namespace
+
 extern "C" ja_status_t ja_exchange_plan_run(ja_exchange_plan_t* p, void* cuda_stream) {
     if (!p) return ja_fail(JA_ERR_INVALID_ARG, "null plan");
     const ExBuild& B = p->B;
     cudaStream_t user = (cudaStream_t)cuda_stream;
-    const JaBoxCopy* d_boxes = (const JaBoxCopy*)(p->pool + B.table_off);
-    ja_status_t rc = ja_launch_box_copies(B.src_base, p->pool, d_boxes, B.n_in, B.max_in, B.vec_in, B.esize, user);
+    const int home_dev = p->phys.at(p->home);
+    int cur = 0;
+    JA_CUDA(cudaGetDevice(&cur));
+    if (cur != home_dev) return ja_fail(JA_ERR_INVALID_ARG, "the plan was created with device %d current, now it is %d", home_dev, cur);
+    char* home = p->pool.at(p->home);
+    const JaBoxCopy* d_boxes = (const JaBoxCopy*)(home + p->table_off);
+    struct Restore {
+        int dev;
+        ~Restore() { set_device_if(dev); }
+    } restore{cur};
+    auto dev_of = [&](int b) { return p->phys.at(p->place[b].label); };
+    ja_status_t rc = ja_launch_box_copies(B.src_base, home, d_boxes, B.n_in, B.max_in, B.vec_in, B.esize, user);
     if (rc != JA_OK) return rc;
+    for (int a = 0; a < B.n_in; ++a)          // atoms of sites on other devices leave home
+        if (p->place[a].stage >= 0)
+            JA_CUDA(copy_between(p->at(a), home + p->place[a].stage, (size_t)B.bufs[a].bytes, user));
     if (!B.steps.empty()) {
         // fork: every site's stream starts after decompose
         JA_CUDA(cudaEventRecord(p->start, user));
@@ -2048,16 +2165,29 @@ extern "C" ja_status_t ja_exchange_plan_run(ja_exchange_plan_t* p, void* cuda_st
                 if (B.bufs[b].producer_site >= 0 && B.bufs[b].producer_site != s.site) JA_CUDA(cudaStreamWaitEvent(st, p->ready[b], 0));
             if (s.parts.size() == 1 && B.bufs[s.out].producer_site >= 0 && B.bufs[s.out].producer_site != s.site)
                 JA_CUDA(cudaStreamWaitEvent(st, p->ready[s.out], 0));
-            if ((rc = issue_step(B, s, p->pool, st)) != JA_OK) return rc;
-            // what this step wrote: its aggregate (if it computed one) and the copies at the destinations
-            if (s.parts.size() >= 2) JA_CUDA(cudaEventRecord(p->ready[s.out], st));
-            for (int d : s.dests) JA_CUDA(cudaEventRecord(p->ready[d], st));
+            JA_CUDA(set_device_if(dev_of(s.out)));
+            char* here = p->at(s.out);
+            if (s.parts.size() >= 2) {
+                const void* parts[JA_EXCHANGE_MAX_PARTS];
+                for (size_t k = 0; k < s.parts.size(); ++k) parts[k] = p->at(s.parts[k]);
+                if ((rc = ja_launch_exchange_combine(parts, (int)s.parts.size(), here, B.bufs[s.out].bytes, B.dtype, B.agg, st)) != JA_OK) return rc;
+                JA_CUDA(cudaEventRecord(p->ready[s.out], st));
+            }
+            for (int d : s.dests) {
+                JA_CUDA(copy_between(p->at(d), here, (size_t)B.bufs[s.out].bytes, st));
+                JA_CUDA(cudaEventRecord(p->ready[d], st));
+            }
         }
         // join
+        JA_CUDA(set_device_if(home_dev));
         for (auto& kv : p->stream) {
             JA_CUDA(cudaEventRecord(p->done.at(kv.first), kv.second));
             JA_CUDA(cudaStreamWaitEvent(user, p->done.at(kv.first), 0));
         }
     }
-    return ja_launch_box_copies(p->pool, B.dst_base, d_boxes + B.n_in, B.n_out, B.max_out, B.vec_out, B.esize, user);
+    std::set<int> brought;
+    for (int b : B.out_box_buf)              // what function specs on other devices ended with comes home
+        if (p->place[b].stage >= 0 && brought.insert(b).second)
+            JA_CUDA(copy_between(home + p->place[b].stage, p->at(b), (size_t)B.bufs[b].bytes, user));
+    return ja_launch_box_copies(home, B.dst_base, d_boxes + B.n_in, B.n_out, B.max_out, B.vec_out, B.esize, user);
 }

@@ -59,6 +59,7 @@ def _declare():
         "ja_exprog_schedule": [vp, P(i32), P(i32), P(i32), P(i32), P(u64)],
         "ja_exchange_plan_create": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i64), P(vp)],
         "ja_exchange_plan_run": [vp, vp],
+        "ja_exchange_plan_create_on": [vp, vp, P(i32), P(i32), i32, ctypes.c_int, vp, P(i32), i32, P(i64), P(vp)],
         "ja_exchange_combine": [P(vp), i32, vp, i64, ctypes.c_int, ctypes.c_int, vp],
     }
     for name, argtypes in sigs.items():
@@ -296,14 +297,16 @@ def _stats(stats):
 
 
 @_program_arg
-def ja_exchange_plan_create(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int):
-    """Returns (plan handle, statistics)."""
+def ja_exchange_plan_create(prog: int, partials: int, copy_site, consumer_specs, agg, dst: int, site_device=None):
+    """Returns (plan handle, statistics).  site_device[s] = device label of site s (None: every site on the current device)."""
     from .binding import AGG
     stats = (ctypes.c_int64 * 5)()
     h = ctypes.c_void_p()
-    _check(LIB.ja_exchange_plan_create(prog, partials, (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
-                                       (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs),
-                                       AGG[agg] if isinstance(agg, str) else int(agg), dst, stats, ctypes.byref(h)))
+    sd = None if site_device is None else (ctypes.c_int32 * len(site_device))(*[int(x) for x in site_device])
+    _check(LIB.ja_exchange_plan_create_on(prog, partials, (ctypes.c_int32 * len(copy_site))(*[int(x) for x in copy_site]),
+                                          (ctypes.c_int32 * len(consumer_specs))(*[int(x) for x in consumer_specs]), len(consumer_specs),
+                                          AGG[agg] if isinstance(agg, str) else int(agg), dst, sd,
+                                          0 if site_device is None else len(site_device), stats, ctypes.byref(h)))
     return h.value, _stats(stats)
 
 
@@ -322,9 +325,10 @@ def ja_exchange_trim():
 class ExchangePlan:
     """An exchange plan with its lifetime; keeps the two relations alive, as the plan holds their payload addresses."""
 
-    def __init__(self, prog: "ExchangeProgram", partials, copy_site, consumer_specs, agg, dst):
+    def __init__(self, prog: "ExchangeProgram", partials, copy_site, consumer_specs, agg, dst, site_device=None):
         self.partials, self.dst = partials, dst
-        self.handle, self.stats = ja_exchange_plan_create(prog.handle, partials.handle, copy_site, consumer_specs, agg, dst.handle)
+        self.handle, self.stats = ja_exchange_plan_create(prog.handle, partials.handle, copy_site, consumer_specs, agg, dst.handle,
+                                                          site_device)
 
     def run(self, stream=None):
         import torch

@@ -311,3 +311,39 @@ def test_randomly_rewritten_programs_on_random_preambles(seed):
         assert np.array_equal(got[consumed], same[consumed])
         assert relfro(got[consumed], want[consumed]) <= (1e-6 if dtype == F32 else 2e-3)
     plan.close()
+
+
+@pytest.mark.parametrize("case,body", [("preamble", "naive"), ("crossed", "synth"), ("replicated", "naive"), ("allreduce", "butterfly")])
+def test_exchange_plan_with_sites_on_device_labels(case, body):
+    """Every site on a device label of its own.  With fewer devices than labels the labels wrap around, so on one GPU this
+    runs every path a plan over several devices takes -- per-device pools, staging at home, copies for the atoms that leave
+    home, for every transfer and for the aggregates that come home -- and must give the one-stream execution's bits."""
+    c = CASES[case]
+    m = c["m"]
+    h, q = build(case, body)
+    P = si.normal([m] + c["ext"], 0.0, 1.0, BF, 6, 29)
+    rP = upload(P, blocked.partial_splits(m, c["ps"]))
+    rA = empty_like_tiling(c["ext"], c["cs"], BF, fill=float("nan"))
+    rB = empty_like_tiling(c["ext"], c["cs"], BF, fill=float("nan"))
+    stats = h.execute(rP, c["copy_site"], c["specs"], "sum", rA)
+    n_sites = X.ja_exprog_counts(h)["gpus"]
+    for labels in ([s + 1 for s in range(n_sites)],            # nobody at home: everything is staged
+                   [0] + [5] * (n_sites - 1),                  # site 0 at home, the others together elsewhere
+                   [torch.cuda.current_device()] * n_sites):   # everybody at home: the plan of the test above
+        plan = X.ExchangePlan(h, rP, c["copy_site"], c["specs"], "sum", rB, site_device=labels)
+        assert {k: v for k, v in plan.stats.items() if k != "scratch_bytes"} == {k: v for k, v in stats.items() if k != "scratch_bytes"}
+        rB.payload.zero_()
+        plan.run()
+        torch.cuda.synchronize()
+        check_status()
+        assert np.array_equal(download(rB), download(rA))
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            plan.run()
+        rB.payload.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(download(rB), download(rA))
+        plan.close()
+    with pytest.raises(JaError):
+        X.ExchangePlan(h, rP, c["copy_site"], c["specs"], "sum", rB, site_device=[-1] * n_sites)
