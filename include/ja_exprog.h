@@ -32,7 +32,7 @@ typedef struct ja_exprog ja_exprog_t;
  * endpoints: every site sends at most link_gbs and receives at most link_gbs; a multicast to k sites is k flows.
  * CUBE_MESH: eight sites; i <-> i + 4 are double links (double_gbs per direction), pairs inside {0..3} and inside {4..7}
  * single links (link_gbs), every other pair shares one bridge of pcie_gbs in total (the paper names the four double
- * links and "single links inside a socket"; the rest of the table is this library's reading).
+ * links and says that pairs inside a CPU socket have single ones; the rest of the table is this library's reading).
  * LINKS: any point-to-point topology given as a table of directed link capacities; flows on one directed link share it,
  * flows between unlinked pairs share the bridge -- the cube mesh is the special case ja_machine_preset("dgx_v100") fills in. */
 typedef enum { JA_FABRIC_NVSWITCH = 0, JA_FABRIC_CUBE_MESH = 1, JA_FABRIC_LINKS = 2 } ja_fabric_t;
@@ -78,7 +78,7 @@ ja_status_t ja_exprog_get_requirements(const ja_exprog_t* p, int32_t* n, uint64_
 /* Atoms: site[i], size_gb[i] in declaration order. */
 ja_status_t ja_exprog_get_atoms(const ja_exprog_t* p, int32_t* site, double* size_gb);
 
-/* ---- partitions declared by size alone (Section 5.2: "the compiler chooses its membership") ----------------------
+/* ---- partitions declared by size alone (Section 5.2: their members are the compiler's choice) ----------------------
  * The memberships are enumerated partition by partition in declaration order, each taking a combination (in
  * lexicographic order) of the sites that the explicit partitions and the earlier ones left.  ja_exprog_bind writes the
  * index-th membership into the program (partitions then have explicit members); ja_exprog_membership reports the
@@ -100,7 +100,7 @@ ja_status_t ja_exprog_closure(const ja_exprog_t* p, int64_t* n, uint64_t* aggreg
 ja_status_t ja_exprog_check(const ja_exprog_t* p, int32_t* well_formed, int32_t* valid);
 ja_status_t ja_exprog_valid_any(const ja_exprog_t* p, int32_t* valid);
 
-/* ---- the simulator (Section 5.2: a set, not a sequence; two-stage actions; the cost model) -------------------------
+/* ---- the simulator (Section 5.2: an unordered body; two-stage actions; the cost model) -------------------------
  * An action starts when aggregates materialised at its source partition its aggregate (the partition with the fewest
  * parts available then); m >= 2 parts cost (m + 1) x size / hbm_gbs, one part nothing; its transfers start when the
  * aggregation ends.  Concurrent work shares a resource equally (aggregations at a site; flows at an endpoint, on a
@@ -185,8 +185,8 @@ ja_status_t ja_exchange_execute(const ja_exprog_t* prog, const ja_relation_t* pa
                                 int64_t* stats, void* cuda_stream);
 ja_status_t ja_exchange_trim(void);
 
-/* ---- an exchange plan: the executable artifact (Section 5.1: "a CUDA graph in which each vertex is a GPU kernel or a
- * network operation") ---------------------------------------------------------------------------------------------------
+/* ---- an exchange plan: the executable artifact (Section 5.1: what the compiler emits is a CUDA graph of kernel nodes and
+ * transfer nodes) -------------------------------------------------------------------------------------------------------
  * ja_exchange_plan_create does once what ja_exchange_execute does per call -- checks, firing order, buffers, tables --
  * and keeps the atom buffers and tables in device memory of its own (synchronous cudaMalloc / cudaMemcpy; JA_ERR_OOM if
  * the buffers do not fit).  The relations' payload addresses are bound into the plan: both relations must outlive it

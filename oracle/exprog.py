@@ -25,7 +25,7 @@ Readings where the paper is silent:
     flow gets min(egress of its source / flows leaving it, ingress of its destination / flows entering it), a multicast
     to k sites being k flows; on the cube mesh flows on one directed link share it, and all flows between unlinked pairs
     share the PCIe bridge;
-  * the cube mesh (the paper names only the four 50 GB/s pillars and "single links inside a socket"): sites {0,1,2,3} and
+  * the cube mesh (the paper names only the four 50 GB/s pillars and says that pairs inside a CPU socket have single links): sites {0,1,2,3} and
     {4,5,6,7} are fully connected by 25 GB/s links, i <-> i+4 are 50 GB/s, every other pair goes over PCIe;
   * the completion time is the time at which the last action of the program finishes.
 """
