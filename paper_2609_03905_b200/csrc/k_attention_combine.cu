@@ -51,11 +51,13 @@ template <> __device__ __forceinline__ uint4 pack_vec<__half>(const float (&f)[8
 }
 
 // MC: capacity in copies (2, 4 or 8). A lane holds one 16-byte vector of a row, so a row of 128 cells takes 16 lanes (16-bit
-// cells) or 32 (f32) and a warp-wide load covers RPL = 2 or 1 rows; a warp takes 8 / MC such loads per copy and round --
-// 4 KiB of loads in flight per warp whatever m is, kept packed in registers until they are used.
+// cells) or 32 (f32) and a warp-wide load covers RPL = 2 or 1 rows; a warp takes R = 2 (MC = 2) or 1 such loads per copy and
+// round, kept packed in registers until they are used. More rows per round (R = 8 / MC: 4 KiB in flight per warp) cost more in
+// registers, and so in resident warps, than they brought: 45.9 / 75.0 us against 37.0 / 58.7 for m = 2 / 4 on
+// 4 x 2048 x 32 rows of bf16.
 template <typename T, bool FAST, int MC>
 __global__ void __launch_bounds__(256) attention_combine_kernel(const CombineParams p) {
-    constexpr int R = MAX_COPIES / MC, CELLS = Vec16<T>::CELLS, LPR = 128 / CELLS, RPL = 32 / LPR, ROWS = R * RPL;
+    constexpr int R = (MAX_COPIES / MC + 1) / 2, CELLS = Vec16<T>::CELLS, LPR = 128 / CELLS, RPL = 32 / LPR, ROWS = R * RPL;
     const int lane = threadIdx.x & 31, sub = lane / LPR, col = (lane % LPR) * 16;      // col: byte offset of the lane's vector in its row
     const uint32_t warps = gridDim.x * 8u, n_rows = (uint32_t)(p.B * p.S * p.H);   // the host keeps the row count below 2^31
     for (uint32_t row0 = (blockIdx.x * 8u + (threadIdx.x >> 5)) * ROWS; row0 < n_rows; row0 += warps * ROWS) {
@@ -163,7 +165,7 @@ ja_status_t ja_launch_attention_combine(const ja_relation* const* op, const ja_r
         p.o_blk_stride = o->nblocks > 1 ? o->blk_off[1] - o->blk_off[0] : 0;
         p.l_blk_stride = l_stride;
     }
-    const int rows_per_warp = (m <= 2 ? 4 : m <= 4 ? 2 : 1) * (o->dtype == JA_F32 ? 1 : 2);
+    const int rows_per_warp = (m <= 2 ? 2 : 1) * (o->dtype == JA_F32 ? 1 : 2);
     const int64_t n_rows = p.B * p.S * p.H, want = (n_rows + 8 * rows_per_warp - 1) / (8 * rows_per_warp), cap = (int64_t)ja_sm_count() * 16;
     if (n_rows >= (1ll << 31)) return ja_fail(JA_ERR_UNSUPPORTED, "more than 2^31 (batch, position, head) rows");
     const unsigned grid = (unsigned)(want < cap ? (want > 0 ? want : 1) : cap);
