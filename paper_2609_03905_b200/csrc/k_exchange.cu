@@ -68,7 +68,28 @@ template <> __device__ __forceinline__ uint4 pack16<__half>(const float (&f)[8])
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(const CombineParams p) {
     constexpr int N = Cells16<T>::N;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_vec; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p.n_parts == 2) {
+        // two parts: two vectors of a thread at a time, so that four loads are in flight per thread as with more parts
+        const uint4 *a = reinterpret_cast<const uint4*>(p.part[0]), *b = reinterpret_cast<const uint4*>(p.part[1]);
+        for (; i + stride < p.n_vec; i += 2 * stride) {
+            const uint4 a0 = a[i], a1 = a[i + stride], b0 = b[i], b1 = b[i + stride];
+            float x0[N], x1[N], y0[N], y1[N];
+            unpack16<T>(a0, x0);
+            unpack16<T>(b0, y0);
+            unpack16<T>(a1, x1);
+            unpack16<T>(b1, y1);
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                x0[e] = p.is_max ? fmaxf(x0[e], y0[e]) : x0[e] + y0[e];
+                x1[e] = p.is_max ? fmaxf(x1[e], y1[e]) : x1[e] + y1[e];
+            }
+            reinterpret_cast<uint4*>(p.out)[i] = pack16<T>(x0);
+            reinterpret_cast<uint4*>(p.out)[i + stride] = pack16<T>(x1);
+        }
+    }
+    for (; i < p.n_vec; i += stride) {
         float acc[N];
         unpack16<T>(reinterpret_cast<const uint4*>(p.part[0])[i], acc);
         for (int c0 = 1; c0 < p.n_parts; c0 += 4) {

@@ -64,7 +64,30 @@ __global__ void __launch_bounds__(256) repartition_agg_kernel(const char* __rest
         const CopySlab sl = slabs[s];
         const int vpr = sl.row_bytes / (int)(VEC * sizeof(TS));  // accesses per row
         const int total = vpr * sl.rows;
-        for (int i = threadIdx.x; i < total; i += 256) {
+        int i = threadIdx.x;
+        if (n_copies <= 2) {
+            // few copies: two accesses of a thread at a time, so that four loads are in flight per thread as with many copies
+            for (; i + 256 < total; i += 512) {
+                const int r0 = i / vpr, c0 = i - r0 * vpr, r1 = (i + 256) / vpr, c1 = i + 256 - r1 * vpr;
+                const char* sp0 = src + sl.src_off + (int64_t)r0 * sl.src_pitch + (int64_t)c0 * (VEC * sizeof(TS));
+                const char* sp1 = src + sl.src_off + (int64_t)r1 * sl.src_pitch + (int64_t)c1 * (VEC * sizeof(TS));
+                float a0[VEC], a1[VEC], b0[VEC], b1[VEC];
+                load_cells<TS, VEC>(sp0, a0);
+                load_cells<TS, VEC>(sp1, a1);
+                if (n_copies == 2) {
+                    load_cells<TS, VEC>(sp0 + copy_stride, b0);
+                    load_cells<TS, VEC>(sp1 + copy_stride, b1);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        a0[e] = combine<IS_MAX>(a0[e], b0[e]);
+                        a1[e] = combine<IS_MAX>(a1[e], b1[e]);
+                    }
+                }
+                store_cells<TD, VEC>(dst + sl.dst_off + (int64_t)r0 * sl.dst_pitch + (int64_t)c0 * (VEC * sizeof(TD)), a0);
+                store_cells<TD, VEC>(dst + sl.dst_off + (int64_t)r1 * sl.dst_pitch + (int64_t)c1 * (VEC * sizeof(TD)), a1);
+            }
+        }
+        for (; i < total; i += 256) {
             const int r = i / vpr, c = i - r * vpr;
             const char* sp = src + sl.src_off + (int64_t)r * sl.src_pitch + (int64_t)c * (VEC * sizeof(TS));
             float acc[VEC];
