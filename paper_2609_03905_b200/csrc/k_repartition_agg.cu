@@ -15,22 +15,26 @@ template <> struct VecOf<__half> { static constexpr int N = 8; };
 template <typename T> struct IsF16 { static constexpr bool value = false; };
 template <> struct IsF16<__half> { static constexpr bool value = true; };
 
+// the cells of one 16-byte access that is already in registers
+template <typename TS> __device__ __forceinline__ void unpack_cells(const uint4& v, float* f) {
+    if (sizeof(TS) == 4) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    } else {
+        const uint32_t h[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 t = ja_unpack16<IsF16<TS>::value>(h[e]);
+            f[2 * e] = t.x;
+            f[2 * e + 1] = t.y;
+        }
+    }
+}
+// p points into GLOBAL memory (the read-only path is used)
 template <typename TS, int VEC> __device__ __forceinline__ void load_cells(const char* p, float* f) {
     if (VEC == 1) {
         f[0] = ja_to_float(*reinterpret_cast<const TS*>(p));
     } else {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
-        if (sizeof(TS) == 4) {
-            f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
-        } else {
-            const uint32_t* h = reinterpret_cast<const uint32_t*>(&v);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 t = ja_unpack16<IsF16<TS>::value>(h[e]);
-                f[2 * e] = t.x;
-                f[2 * e + 1] = t.y;
-            }
-        }
+        unpack_cells<TS>(__ldg(reinterpret_cast<const uint4*>(p)), f);
     }
 }
 
@@ -56,7 +60,9 @@ template <typename TD, int VEC> __device__ __forceinline__ void store_cells(char
 
 template <bool IS_MAX> __device__ __forceinline__ float combine(float a, float b) { return IS_MAX ? fmaxf(a, b) : a + b; }
 
-template <typename TS, typename TD, int VEC, bool IS_MAX>
+// FEW: at most four copies (a form of its own: the two-at-a-time path costs registers that the many-copies loop pays for in
+// resident warps -- eight copies ran in 288 us instead of 200 with both in one kernel)
+template <typename TS, typename TD, int VEC, bool IS_MAX, bool FEW>
 __global__ void __launch_bounds__(256) repartition_agg_kernel(const char* __restrict__ src, char* __restrict__ dst,
                                                               const CopySlab* __restrict__ slabs, int64_t n_slabs, int n_copies,
                                                               int64_t copy_stride) {
@@ -65,24 +71,35 @@ __global__ void __launch_bounds__(256) repartition_agg_kernel(const char* __rest
         const int vpr = sl.row_bytes / (int)(VEC * sizeof(TS));  // accesses per row
         const int total = vpr * sl.rows;
         int i = threadIdx.x;
-        if (n_copies <= 2) {
-            // few copies: two accesses of a thread at a time, so that four loads are in flight per thread as with many copies
+        if (FEW && VEC > 1) {
+            // few copies: two accesses of a thread at a time, every load of both issued first and kept as it came (16 bytes
+            // each) until it is combined, so that a thread has as many loads in flight as with many copies
             for (; i + 256 < total; i += 512) {
                 const int r0 = i / vpr, c0 = i - r0 * vpr, r1 = (i + 256) / vpr, c1 = i + 256 - r1 * vpr;
                 const char* sp0 = src + sl.src_off + (int64_t)r0 * sl.src_pitch + (int64_t)c0 * (VEC * sizeof(TS));
                 const char* sp1 = src + sl.src_off + (int64_t)r1 * sl.src_pitch + (int64_t)c1 * (VEC * sizeof(TS));
-                float a0[VEC], a1[VEC], b0[VEC], b1[VEC];
-                load_cells<TS, VEC>(sp0, a0);
-                load_cells<TS, VEC>(sp1, a1);
-                if (n_copies == 2) {
-                    load_cells<TS, VEC>(sp0 + copy_stride, b0);
-                    load_cells<TS, VEC>(sp1 + copy_stride, b1);
+                uint4 raw0[4], raw1[4];
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) {
-                        a0[e] = combine<IS_MAX>(a0[e], b0[e]);
-                        a1[e] = combine<IS_MAX>(a1[e], b1[e]);
+                for (int c = 0; c < 4; ++c)
+                    if (c < n_copies) {
+                        raw0[c] = __ldg(reinterpret_cast<const uint4*>(sp0 + (int64_t)c * copy_stride));
+                        raw1[c] = __ldg(reinterpret_cast<const uint4*>(sp1 + (int64_t)c * copy_stride));
                     }
-                }
+                float a0[VEC], a1[VEC];
+                unpack_cells<TS>(raw0[0], a0);
+                unpack_cells<TS>(raw1[0], a1);
+#pragma unroll
+                for (int c = 1; c < 4; ++c)
+                    if (c < n_copies) {
+                        float b0[VEC], b1[VEC];
+                        unpack_cells<TS>(raw0[c], b0);
+                        unpack_cells<TS>(raw1[c], b1);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) {
+                            a0[e] = combine<IS_MAX>(a0[e], b0[e]);
+                            a1[e] = combine<IS_MAX>(a1[e], b1[e]);
+                        }
+                    }
                 store_cells<TD, VEC>(dst + sl.dst_off + (int64_t)r0 * sl.dst_pitch + (int64_t)c0 * (VEC * sizeof(TD)), a0);
                 store_cells<TD, VEC>(dst + sl.dst_off + (int64_t)r1 * sl.dst_pitch + (int64_t)c1 * (VEC * sizeof(TD)), a1);
             }
@@ -118,13 +135,21 @@ template <typename TS, typename TD>
 void launch(const char* src, char* dst, const CopySlab* d_slabs, int64_t n_slabs, int n_copies, int64_t copy_stride, bool is_max,
             bool vec, unsigned grid, cudaStream_t st) {
     constexpr int V = VecOf<TS>::N;
+#define JA_AGG_LAUNCH(VV, MAXF, FEWF) repartition_agg_kernel<TS, TD, VV, MAXF, FEWF><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride)
+    const bool few = vec && n_copies <= 4;
     if (vec) {
-        if (is_max) repartition_agg_kernel<TS, TD, V, true><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
-        else repartition_agg_kernel<TS, TD, V, false><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+        if (few) {
+            if (is_max) JA_AGG_LAUNCH(V, true, true);
+            else JA_AGG_LAUNCH(V, false, true);
+        } else {
+            if (is_max) JA_AGG_LAUNCH(V, true, false);
+            else JA_AGG_LAUNCH(V, false, false);
+        }
     } else {
-        if (is_max) repartition_agg_kernel<TS, TD, 1, true><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
-        else repartition_agg_kernel<TS, TD, 1, false><<<grid, 256, 0, st>>>(src, dst, d_slabs, n_slabs, n_copies, copy_stride);
+        if (is_max) JA_AGG_LAUNCH(1, true, false);
+        else JA_AGG_LAUNCH(1, false, false);
     }
+#undef JA_AGG_LAUNCH
 }
 
 }  // namespace
