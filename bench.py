@@ -983,9 +983,15 @@ def case_results(case, reps):
                 tp = timeit(lambda r: plan.run(), reps, True)
                 tg = timeit_graph(lambda r: plan.run(), reps, True)
                 plan.close()
+                # every site on a device label of its own (the labels wrap around on one GPU): the paths a plan over several devices
+                # takes -- atoms leave the relations' device through a staging area, aggregates come back before recompose
+                staged = X.ExchangePlan(h, P, copy_site, specs, "sum", y, site_device=[s + 1 for s in range(4)])
+                ts = timeit_graph(lambda r: staged.run(), reps, True)
+                staged.close()
                 res["%s_%s" % (tag, "synthesised" if body == "best" else body)] = {
                     **hb(nbytes, t), "plan_dataflow_ms": tp["ms_mean"], "plan_graph_replay_ms": tg["ms_mean"],
                     "plan_graph_replay_frac_of_measured_hbm": nbytes / (tg["ms_mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "plan_all_sites_staged_graph_replay_ms": ts["ms_mean"],
                     "simulated_ms_hgx_b200_nominal": sim, "actions": len(acts), "aggregations": stats["aggregations"],
                     "transfers": stats["transfers"], "transfer_MB": stats["transfer_bytes"] / 1e6, "scratch_MB": stats["scratch_bytes"] / 1e6}
             res["%s_fused_aggregating_relayout" % tag] = hb((m + 1.0) * T * d * 2, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
