@@ -996,7 +996,7 @@ def case_results(case, reps):
                     "transfers": stats["transfers"], "transfer_MB": stats["transfer_bytes"] / 1e6, "scratch_MB": stats["scratch_bytes"] / 1e6}
             res["%s_fused_aggregating_relayout" % tag] = hb((m + 1.0) * T * d * 2, timeit(lambda r: ja.repartition_agg(P, "sum", y), reps, True))
             del P, y
-        # the oracle's executor beside it, on the host cores, on one sixteenth of the rows (the programs and their traffic per
+        # cpu_baseline leg of this case: the oracle's executor beside it, on the host cores, on one sixteenth of the rows (the programs and their traffic per
         # byte of tensor are the same at that size): the naive reduce-scatter program, fp64 sums, one rounding to bf16 per aggregate
         import time
         import numpy as np
@@ -1009,7 +1009,7 @@ def case_results(case, reps):
         t0 = time.perf_counter()
         OE.exchange(q, Ph, ps, cs, specs, "sum", "bf16")
         dt = time.perf_counter() - t0
-        res["oracle_reduce_scatter_naive_on_host"] = {"seconds": dt, "rows": Ts, "GBps_of_bf16_tensor_traffic": (2.82e9 / 16) / dt / 1e9,
+        res["cpu_baseline_oracle_reduce_scatter_naive"] = {"kind": "oracle", "seconds": dt, "rows": Ts, "GBps_of_bf16_tensor_traffic": (2.82e9 / 16) / dt / 1e9,
                                                       "note": "oracle/exprog.py executor, numpy fp64, 1/16 of the rows"}
     elif args.case == "chains":
         # Section 6, second workload: five fixed matrix chains, each parenthesization executed as a sequence of matmul
