@@ -27,6 +27,9 @@
  *
  * Payload layout of a relation ("block-key layout"): blocks in row-major key order, each block a dense
  * row-major array of its own extents, blocks back to back, each starting on a 128-byte boundary.
+ *
+ * Exchange programs (Section 5: the ExProg language, validity, the simulator, synthesis, placement, preamble
+ * generation, and a program's execution on one GPU) are declared in ja_exprog.h, which includes this header.
  */
 #ifndef JA_H_
 #define JA_H_
