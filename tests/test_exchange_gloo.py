@@ -12,6 +12,7 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
+import paper_2609_03905_b200  # noqa: F401  (loads, and if need be builds, the library once here, before the ranks start)
 from oracle import exprog as E
 
 G = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "exprog_examples.json")))
